@@ -1,0 +1,312 @@
+/*
+ * H2O (Heavy-Hitter Oracle) eviction policy — plain fp64 CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, by-the-definition restatement
+ * of the method that the CUDA path is checked against.  It shares no code with
+ * the CUDA path and must never be called from it.  Only the tests, the smoke
+ * check and the benchmark's CPU-baseline leg may use it.
+ *
+ * What it follows (paper section / algorithm):
+ *   - Attention of token i over a kept set S: o_i = D_i^{-1} exp(Q_i K_S^T),
+ *     evicted tokens absent from numerator and normaliser (Definition 2.2, "generative
+ *     process with eviction policy"; Appendix D.5 "approximate version").
+ *   - With S = [i] this is ordinary causal attention (Definition 2.2, last bullet;
+ *     Appendix D "generative process with full knowledge").
+ *   - Accumulated score o~_i = o~_{i-1} + o_i and victim
+ *     u = argmax_v F_score(G_i \ {v}), F_score(T) = h(sum_{s in T} o~_s)
+ *     (Algorithm 2, formal version of Algorithm 1).  For increasing h the argmax is
+ *     the candidate with the smallest accumulated score; the tests brute-force the
+ *     literal argmax to pin that.
+ *   - Budget split into heavy hitters and the most recent tokens; prefill keeps
+ *     K heavy + K recent (all if the prompt is shorter); eviction is skipped
+ *     while the cache is not full (Appendix A, system details and pseudocode).
+ *
+ * Readings taken where the paper leaves a choice (each is listed in the design notes):
+ *   - token t attends to the kept set plus itself, then one entry is evicted;
+ *   - scores are accumulated at every step, also while the cache is filling, and
+ *     the prompt's column sums are carried into decoding;
+ *   - after step t the protected window is positions t-r+1..t, so eviction
+ *     candidates are the entries with pos <= t - r;
+ *   - total order for eviction: smaller accumulated score first, equal scores
+ *     broken by lower token position;
+ *   - logits are multiplied by an explicit softmax scale c.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms for uniform attention, brute force of the literal argmax, textbook
+ * causal / sliding-window attention as special cases, explicit column sums).
+ * The paper prints no worked numeric example, so no stored golden values exist.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* <a, b> over d elements, inputs widened to double, summed in index order. */
+static double dot_fd(const float* a, const float* b, long d) {
+  double s = 0.0;
+  for (long c = 0; c < d; ++c) s += (double)a[c] * (double)b[c];
+  return s;
+}
+
+int h2o_oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/*
+ * Causal softmax attention of one (sequence, head) and the column sums of its
+ * probability matrix.
+ *   Q, K, V : n rows of d floats, consecutive rows `stride` floats apart.
+ *   c       : softmax scale.
+ *   O       : [n][d]  O_i = sum_{j<=i} P[i][j] V_j
+ *   rowmax, rowsum : [n]  m_i = max_j s_ij,  l_i = sum_j exp(s_ij - m_i)
+ *   acc0    : [n]     acc0[j] = sum_{i>=j} P[i][j]   (summed for increasing i)
+ *   P_out   : optional [n][n] (NULL to skip), zero above the diagonal.
+ * P[i][j] = exp(s_ij - m_i) / l_i with s_ij = c <Q_i, K_j>, j <= i.
+ */
+int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const float* V, long n, long d, long stride,
+                                       double c, double* O, double* rowmax, double* rowsum, double* acc0,
+                                       double* P_out) {
+  if (n < 0 || d <= 0 || stride < d) return -1;
+  int failed = 0;
+#pragma omp parallel
+  {
+    double* e = (double*)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    if (!e) {
+#pragma omp atomic write
+      failed = 1;
+    }
+#pragma omp for schedule(dynamic, 4)
+    for (long i = 0; i < n; ++i) {
+      if (!e) continue;
+      const float* qi = Q + i * stride;
+      double m = -INFINITY;
+      for (long j = 0; j <= i; ++j) {
+        e[j] = c * dot_fd(qi, K + j * stride, d);
+        if (e[j] > m) m = e[j];
+      }
+      double l = 0.0;
+      for (long j = 0; j <= i; ++j) {
+        e[j] = exp(e[j] - m);
+        l += e[j];
+      }
+      rowmax[i] = m;
+      rowsum[i] = l;
+      double* oi = O + i * d;
+      for (long x = 0; x < d; ++x) oi[x] = 0.0;
+      for (long j = 0; j <= i; ++j) {
+        const double p = e[j] / l;
+        const float* vj = V + j * stride;
+        for (long x = 0; x < d; ++x) oi[x] += p * (double)vj[x];
+        if (P_out) P_out[i * n + j] = p;
+      }
+      if (P_out)
+        for (long j = i + 1; j < n; ++j) P_out[i * n + j] = 0.0;
+    }
+    free(e);
+    /* Column sums straight from the definition: the same s_ij, m_i and l_i again. */
+#pragma omp for schedule(dynamic, 4)
+    for (long j = 0; j < n; ++j) {
+      const float* kj = K + j * stride;
+      double a = 0.0;
+      for (long i = j; i < n; ++i) {
+        const double s = c * dot_fd(Q + i * stride, kj, d);
+        a += exp(s - rowmax[i]) / rowsum[i];
+      }
+      acc0[j] = a;
+    }
+  }
+  return failed ? -2 : 0;
+}
+
+/* Eviction order: x before y iff acc_x < acc_y, or equal and pos_x < pos_y. */
+static int precedes(double acc_x, long pos_x, double acc_y, long pos_y) {
+  if (acc_x < acc_y) return 1;
+  if (acc_x > acc_y) return 0;
+  return pos_x < pos_y;
+}
+
+static double rel_gap(double a, double b) {
+  const double m = fmax(fabs(a), fabs(b));
+  return m > 0.0 ? fabs(a - b) / m : 0.0;
+}
+
+typedef struct {
+  double acc;
+  long pos;
+} scored_t;
+
+static int scored_cmp(const void* a, const void* b) {
+  const scored_t* x = (const scored_t*)a;
+  const scored_t* y = (const scored_t*)b;
+  if (precedes(x->acc, x->pos, y->acc, y->pos)) return -1;
+  if (precedes(y->acc, y->pos, x->acc, x->pos)) return 1;
+  return 0;
+}
+
+/*
+ * One-shot selection after the prompt (Appendix A: "K heavy hitters and K recent
+ * tokens if the prompt has length >= 2K, otherwise all").
+ *   acc0 [n], heavy budget k, recent window r.
+ *   kept : out, ascending positions, min(n, k + r) of them; returns that count.
+ *   boundary : out [2] = accumulated score of the weakest kept heavy hitter and of
+ *              the strongest dropped candidate (NaN where there is none).
+ * Heavy hitters are the k largest of positions [0, n - r) under the eviction order.
+ */
+long h2o_oracle_select(const double* acc0, long n, long k, long r, int32_t* kept, double* boundary) {
+  boundary[0] = boundary[1] = NAN;
+  if (n <= k + r) {
+    for (long j = 0; j < n; ++j) kept[j] = (int32_t)j;
+    return n;
+  }
+  const long nc = n - r; /* candidates 0..nc-1, nc > k */
+  scored_t* c = (scored_t*)malloc(sizeof(scored_t) * (size_t)nc);
+  if (!c) return -1;
+  for (long j = 0; j < nc; ++j) {
+    c[j].acc = acc0[j];
+    c[j].pos = j;
+  }
+  qsort(c, (size_t)nc, sizeof(scored_t), scored_cmp); /* weakest first */
+  char* keep = (char*)calloc((size_t)n, 1);
+  if (!keep) {
+    free(c);
+    return -1;
+  }
+  for (long x = nc - k; x < nc; ++x) keep[c[x].pos] = 1;
+  for (long j = nc; j < n; ++j) keep[j] = 1;
+  if (k > 0) boundary[0] = c[nc - k].acc;
+  boundary[1] = c[nc - k - 1].acc;
+  long m = 0;
+  for (long j = 0; j < n; ++j)
+    if (keep[j]) kept[m++] = (int32_t)j;
+  free(keep);
+  free(c);
+  return m;
+}
+
+/*
+ * One decoding step for `units` independent (sequence, head) caches
+ * (Algorithm 2 body: scores over G = S u {t}, accumulate, evict one).
+ *
+ * State, per unit u, in rows of capacity `cap` (>= k+r+1) entries:
+ *   cnt[u], t[u], pos[u][cap], acc[u][cap], Kc[u][cap][d], Vc[u][cap][d]
+ * Entry order carries no meaning; only `pos` does.
+ * Inputs: q, knew, vnew [units][d]; kbud, rwin [units]; scale c.
+ * hint  : optional [units]; a decision made elsewhere for this step (-1 none,
+ *         >= 0 evicted position, -2 = no hint).  The oracle always computes its own
+ *         victim first.  If the hint names a different candidate whose accumulated
+ *         score is within `tie_rel` (relative) of the oracle's minimum, the hint is
+ *         applied instead so that later steps stay comparable, and status = 1.
+ *         Any other disagreement is status = 2 and the oracle's own choice is applied.
+ * Outputs: out [units][d]; evicted [units] = oracle's own decision (-1 none);
+ *          status [units]; gap [units] = relative gap between the two smallest
+ *          candidate scores (inf when fewer than two); p_out optional [units][cap]
+ *          = probabilities of the entries in state order, the new token last.
+ */
+int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, const int32_t* rwin, int32_t* t,
+                           int32_t* cnt, int32_t* pos, double* acc, double* Kc, double* Vc, const float* q,
+                           const float* knew, const float* vnew, double c, const int32_t* hint, double tie_rel,
+                           double* out, int32_t* evicted, int32_t* status, double* gap, double* p_out) {
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 8)
+  for (long u = 0; u < units; ++u) {
+    const long B = (long)kbud[u] + (long)rwin[u];
+    const long r = rwin[u];
+    long m = cnt[u];
+    int32_t* up = pos + u * cap;
+    double* ua = acc + u * cap;
+    double* uk = Kc + u * cap * d;
+    double* uv = Vc + u * cap * d;
+    if (m + 1 > cap || m > B) {
+#pragma omp atomic write
+      bad = 1;
+      continue;
+    }
+    const long tt = t[u];
+    /* G = S u {t}: append the new token with zero accumulated score. */
+    up[m] = (int32_t)tt;
+    ua[m] = 0.0;
+    for (long x = 0; x < d; ++x) {
+      uk[m * d + x] = (double)knew[u * d + x];
+      uv[m * d + x] = (double)vnew[u * d + x];
+    }
+    m += 1;
+    /* scores, softmax, output */
+    double* e = (double*)malloc(sizeof(double) * (size_t)m);
+    double mx = -INFINITY;
+    for (long j = 0; j < m; ++j) {
+      double s = 0.0;
+      for (long x = 0; x < d; ++x) s += (double)q[u * d + x] * uk[j * d + x];
+      e[j] = c * s;
+      if (e[j] > mx) mx = e[j];
+    }
+    double l = 0.0;
+    for (long j = 0; j < m; ++j) {
+      e[j] = exp(e[j] - mx);
+      l += e[j];
+    }
+    double* o = out + u * d;
+    for (long x = 0; x < d; ++x) o[x] = 0.0;
+    for (long j = 0; j < m; ++j) {
+      const double p = e[j] / l;
+      for (long x = 0; x < d; ++x) o[x] += p * uv[j * d + x];
+      ua[j] += p; /* accumulate */
+      if (p_out) p_out[u * cap + j] = p;
+    }
+    free(e);
+    /* eviction */
+    evicted[u] = -1;
+    status[u] = 0;
+    gap[u] = INFINITY;
+    long victim = -1;
+    if (m > B) {
+      long second = -1;
+      for (long j = 0; j < m; ++j) {
+        if ((long)up[j] > tt - r) continue; /* protected recent window */
+        if (victim < 0 || precedes(ua[j], up[j], ua[victim], up[victim])) {
+          second = victim;
+          victim = j;
+        } else if (second < 0 || precedes(ua[j], up[j], ua[second], up[second])) {
+          second = j;
+        }
+      }
+      if (victim < 0) { /* cannot happen with distinct positions < t; flagged, not hidden */
+#pragma omp atomic write
+        bad = 1;
+        continue;
+      }
+      if (second >= 0) gap[u] = rel_gap(ua[victim], ua[second]);
+      evicted[u] = up[victim];
+      if (hint && hint[u] != -2 && hint[u] != evicted[u]) {
+        long alt = -1;
+        for (long j = 0; j < m; ++j)
+          if (up[j] == hint[u] && (long)up[j] <= tt - r) alt = j;
+        if (alt >= 0 && rel_gap(ua[alt], ua[victim]) < tie_rel) {
+          status[u] = 1;
+          victim = alt;
+        } else {
+          status[u] = 2;
+        }
+      }
+      /* S = G \ {u}: close the gap, keeping the remaining order */
+      for (long j = victim; j + 1 < m; ++j) {
+        up[j] = up[j + 1];
+        ua[j] = ua[j + 1];
+        memcpy(uk + j * d, uk + (j + 1) * d, sizeof(double) * (size_t)d);
+        memcpy(uv + j * d, uv + (j + 1) * d, sizeof(double) * (size_t)d);
+      }
+      m -= 1;
+    } else if (hint && hint[u] != -2 && hint[u] != -1) {
+      status[u] = 2;
+    }
+    cnt[u] = (int32_t)m;
+    t[u] = (int32_t)(tt + 1);
+  }
+  return bad ? -1 : 0;
+}

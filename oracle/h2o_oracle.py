@@ -1,0 +1,222 @@
+"""ctypes front end of the fp64 CPU oracle (``h2o_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  The CUDA package never imports this module and
+this module never imports the CUDA package.
+
+The arithmetic lives in the C file; this wrapper only owns the per-unit state
+arrays, slices ragged inputs into units and gathers the rows the C selection
+named.  A *unit* is one (sequence, head); units never interact.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "h2o_oracle.c")
+_LIB = os.path.join(_HERE, "libh2o_oracle.so")
+_lib = None
+
+NO_HINT = -2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over independent rows/units)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c = ctypes
+        dp, fp, ip = c.POINTER(c.c_double), c.POINTER(c.c_float), c.POINTER(c.c_int32)
+        lib.h2o_oracle_num_threads.restype = c.c_int
+        lib.h2o_oracle_causal_attention_colsum.restype = c.c_int
+        lib.h2o_oracle_causal_attention_colsum.argtypes = [fp, fp, fp, c.c_long, c.c_long, c.c_long, c.c_double, dp, dp, dp, dp, dp]
+        lib.h2o_oracle_select.restype = c.c_long
+        lib.h2o_oracle_select.argtypes = [dp, c.c_long, c.c_long, c.c_long, ip, dp]
+        lib.h2o_oracle_decode_step.restype = c.c_int
+        lib.h2o_oracle_decode_step.argtypes = [c.c_long, c.c_long, c.c_long, ip, ip, ip, ip, ip, dp, dp, dp, fp, fp, fp,
+                                               c.c_double, ip, c.c_double, dp, ip, ip, dp, dp]
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().h2o_oracle_num_threads())
+
+
+def _p(a: Optional[np.ndarray], ty):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ty))
+
+
+def _f32(x) -> np.ndarray:
+    """Widen any input (numpy or torch CPU tensor, f32 or bf16) to contiguous float32, exactly."""
+    if hasattr(x, "detach"):
+        x = x.detach().to("cpu").float().numpy()
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False):
+    """One unit: q, k, v ``[n, d]`` views (row stride may exceed d).  Returns O, acc0, (P)."""
+    n, d = q.shape
+    assert q.dtype == np.float32 and k.dtype == np.float32 and v.dtype == np.float32
+    stride = q.strides[0] // 4
+    assert q.strides == k.strides == v.strides and q.strides[1] == 4
+    O = np.empty((n, d), dtype=np.float64)
+    rowmax = np.empty(n, dtype=np.float64)
+    rowsum = np.empty(n, dtype=np.float64)
+    acc0 = np.empty(n, dtype=np.float64)
+    P = np.empty((n, n), dtype=np.float64) if want_p else None
+    rc = _load().h2o_oracle_causal_attention_colsum(
+        _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), n, d, stride, float(scale),
+        _p(O, ctypes.c_double), _p(rowmax, ctypes.c_double), _p(rowsum, ctypes.c_double), _p(acc0, ctypes.c_double),
+        _p(P, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError("oracle attention failed: %d" % rc)
+    return (O, acc0, P) if want_p else (O, acc0)
+
+
+def select(acc0: np.ndarray, k: int, r: int):
+    """Kept positions (ascending) and the two boundary scores (weakest kept heavy, strongest dropped)."""
+    n = acc0.shape[0]
+    acc0 = np.ascontiguousarray(acc0, dtype=np.float64)
+    kept = np.empty(max(1, min(n, k + r)), dtype=np.int32)
+    boundary = np.empty(2, dtype=np.float64)
+    m = _load().h2o_oracle_select(_p(acc0, ctypes.c_double), n, k, r, _p(kept, ctypes.c_int32), _p(boundary, ctypes.c_double))
+    if m < 0:
+        raise RuntimeError("oracle select failed")
+    return kept[:m].copy(), boundary
+
+
+class OracleCache:
+    """State of ``batch * n_heads`` independent units; unit index = sequence * n_heads + head."""
+
+    def __init__(self, batch: int, n_heads: int, head_dim: int, heavy: Sequence[int], recent: Sequence[int], scale: Optional[float] = None):
+        assert len(heavy) == batch and len(recent) == batch
+        self.batch, self.n_heads, self.d = batch, n_heads, head_dim
+        self.units = batch * n_heads
+        self.scale = float(scale) if scale and scale > 0 else 1.0 / float(np.sqrt(head_dim))
+        self.kbud = np.repeat(np.asarray(heavy, dtype=np.int32), n_heads)
+        self.rwin = np.repeat(np.asarray(recent, dtype=np.int32), n_heads)
+        self.cap = int((self.kbud + self.rwin).max()) + 1
+        self.t = np.zeros(self.units, dtype=np.int32)
+        self.cnt = np.zeros(self.units, dtype=np.int32)
+        self.pos = np.full((self.units, self.cap), -1, dtype=np.int32)
+        self.acc = np.zeros((self.units, self.cap), dtype=np.float64)
+        self.K = np.zeros((self.units, self.cap, head_dim), dtype=np.float64)
+        self.V = np.zeros((self.units, self.cap, head_dim), dtype=np.float64)
+        self.last_acc0: List[np.ndarray] = []
+        self.last_boundary: List[np.ndarray] = []
+
+    # -- prefill ---------------------------------------------------------
+    def prefill(self, q, k, v, cu_seqlens, units: Optional[Sequence[int]] = None, forced_kept=None):
+        """Causal attention, column sums and one-shot selection for every unit (or only ``units``).
+
+        q, k, v: ``[total_tokens, n_heads, d]``.  Returns (out ``[total_tokens, n_heads, d]`` float64 with
+        untouched units left NaN, kept: dict unit -> ascending positions).  ``forced_kept`` maps a unit to
+        a kept set chosen elsewhere (used to re-synchronise after an excused near-tie).
+        """
+        q, k, v = _f32(q), _f32(k), _f32(v)
+        cu = np.asarray(cu_seqlens, dtype=np.int64)
+        out = np.full(q.shape, np.nan, dtype=np.float64)
+        todo = range(self.units) if units is None else units
+        kept_all = {}
+        self.last_acc0 = [None] * self.units
+        self.last_boundary = [None] * self.units
+        for u in todo:
+            s, h = divmod(u, self.n_heads)
+            lo, hi = int(cu[s]), int(cu[s + 1])
+            O, acc0 = causal_attention_colsum(q[lo:hi, h], k[lo:hi, h], v[lo:hi, h], self.scale)
+            out[lo:hi, h] = O
+            kept, boundary = select(acc0, int(self.kbud[u]), int(self.rwin[u]))
+            self.last_acc0[u], self.last_boundary[u] = acc0, boundary
+            kept_all[u] = kept
+            use = kept if forced_kept is None or u not in forced_kept else np.asarray(forced_kept[u], dtype=np.int32)
+            self.load_unit(u, use, acc0[use], k[lo:hi, h][use], v[lo:hi, h][use], hi - lo)
+        return out, kept_all
+
+    def load_unit(self, u: int, positions, acc, k_rows, v_rows, t: int):
+        m = len(positions)
+        assert m <= self.cap - 1
+        self.cnt[u] = m
+        self.t[u] = t
+        self.pos[u, :m] = positions
+        self.acc[u, :m] = acc
+        self.K[u, :m] = k_rows
+        self.V[u, :m] = v_rows
+
+    # -- decode ----------------------------------------------------------
+    def decode_step(self, q, k_new, v_new, hint: Optional[np.ndarray] = None, tie_rel: float = 1e-6, want_p: bool = False,
+                    units: Optional[Sequence[int]] = None):
+        """One step for all units (or the listed ones).  q, k_new, v_new: ``[batch, n_heads, d]``.
+
+        Returns dict(out [units, d], evicted [units], status [units], gap [units], p [units, cap] or None).
+        """
+        qf = _f32(q).reshape(self.units, self.d)
+        kf = _f32(k_new).reshape(self.units, self.d)
+        vf = _f32(v_new).reshape(self.units, self.d)
+        if units is not None:
+            return self._decode_subset(qf, kf, vf, hint, tie_rel, want_p, list(units))
+        return self._decode(self, qf, kf, vf, hint, tie_rel, want_p)
+
+    @staticmethod
+    def _decode(st, qf, kf, vf, hint, tie_rel, want_p):
+        n = st.cnt.shape[0]
+        out = np.empty((n, st.d), dtype=np.float64)
+        evicted = np.empty(n, dtype=np.int32)
+        status = np.empty(n, dtype=np.int32)
+        gap = np.empty(n, dtype=np.float64)
+        p = np.zeros((n, st.cap), dtype=np.float64) if want_p else None
+        h = None if hint is None else np.ascontiguousarray(hint, dtype=np.int32)
+        rc = _load().h2o_oracle_decode_step(
+            n, st.d, st.cap, _p(st.kbud, ctypes.c_int32), _p(st.rwin, ctypes.c_int32), _p(st.t, ctypes.c_int32),
+            _p(st.cnt, ctypes.c_int32), _p(st.pos, ctypes.c_int32), _p(st.acc, ctypes.c_double), _p(st.K, ctypes.c_double),
+            _p(st.V, ctypes.c_double), _p(qf, ctypes.c_float), _p(kf, ctypes.c_float), _p(vf, ctypes.c_float), st.scale,
+            _p(h, ctypes.c_int32), float(tie_rel), _p(out, ctypes.c_double), _p(evicted, ctypes.c_int32),
+            _p(status, ctypes.c_int32), _p(gap, ctypes.c_double), _p(p, ctypes.c_double))
+        if rc != 0:
+            raise RuntimeError("oracle decode step failed: inconsistent state (%d)" % rc)
+        return dict(out=out, evicted=evicted, status=status, gap=gap, p=p)
+
+    def _decode_subset(self, qf, kf, vf, hint, tie_rel, want_p, units):
+        """Step only some units: copy their state out, step, copy back (units are independent)."""
+        idx = np.asarray(units, dtype=np.int64)
+
+        class _S:
+            pass
+
+        st = _S()
+        st.d, st.cap, st.scale = self.d, self.cap, self.scale
+        for name in ("kbud", "rwin", "t", "cnt", "pos", "acc", "K", "V"):
+            setattr(st, name, np.ascontiguousarray(getattr(self, name)[idx]))
+        res = self._decode(st, np.ascontiguousarray(qf[idx]), np.ascontiguousarray(kf[idx]), np.ascontiguousarray(vf[idx]),
+                           None if hint is None else np.asarray(hint)[idx], tie_rel, want_p)
+        for name in ("t", "cnt", "pos", "acc", "K", "V"):
+            getattr(self, name)[idx] = getattr(st, name)
+        return res
+
+    # -- inspection ------------------------------------------------------
+    def export(self, u: int):
+        """Positions (ascending) and their accumulated scores for unit ``u``."""
+        m = int(self.cnt[u])
+        order = np.argsort(self.pos[u, :m], kind="stable")
+        return self.pos[u, :m][order].copy(), self.acc[u, :m][order].copy()
+
+    def permute_entries(self, rng: np.random.Generator):
+        """Shuffle the storage order of every unit's entries (semantics must not change)."""
+        for u in range(self.units):
+            m = int(self.cnt[u])
+            perm = rng.permutation(m)
+            for a in (self.pos, self.acc, self.K, self.V):
+                a[u, :m] = a[u, :m][perm]

@@ -1,0 +1,406 @@
+"""Pins for the fp64 CPU oracle: closed forms, brute force and textbook special cases.
+
+None of these tests re-types the oracle's own loops.  Each compares it with
+something fixed by the paper or by mathematics:
+
+* uniform attention (q = 0) has a closed form in harmonic numbers, evaluated
+  here in exact rational arithmetic;
+* a pure-Python simulator materialises the whole (masked) probability matrix,
+  takes accumulated scores as explicit column sums and picks the victim by the
+  literal ``argmax_v F_score(G \\ {v})`` of the policy's definition, for three
+  choices of ``h``;
+* a budget at least as large as the sequence reduces to ordinary causal softmax
+  attention, a zero heavy budget to sliding-window attention (library softmax);
+* structural invariants of the eviction policy (budget, one eviction per step,
+  no resurrection, recent window always present).
+"""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+from scipy.special import softmax as scipy_softmax
+
+
+def _rand_qkv(rng, n, d, heavy_tail=True):
+    q = rng.standard_normal((n, d)).astype(np.float32)
+    k = rng.standard_normal((n, d)).astype(np.float32)
+    v = rng.standard_normal((n, d)).astype(np.float32)
+    if heavy_tail:
+        u = rng.standard_normal(d)
+        u /= np.linalg.norm(u)
+        q += (1.5 * u).astype(np.float32)
+        hot = rng.random(n) < 0.1
+        k[hot] += (4.0 * u).astype(np.float32)
+    return q, k, v
+
+
+def _as_thd(x):  # [n, d] -> [n, 1, d]
+    return np.ascontiguousarray(x[:, None, :])
+
+
+def _harmonic(m):
+    return sum(Fraction(1, x) for x in range(1, m + 1))
+
+
+# --------------------------------------------------------------------------
+# closed form: uniform attention
+# --------------------------------------------------------------------------
+def test_uniform_attention_closed_form(oracle):
+    n, d, k, r, steps = 23, 3, 4, 5, 9
+    rng = np.random.default_rng(0)
+    q = np.zeros((n + steps, d), dtype=np.float32)
+    kk = rng.standard_normal((n + steps, d)).astype(np.float32)
+    v = rng.standard_normal((n + steps, d)).astype(np.float32)
+
+    O, acc0, P = oracle.causal_attention_colsum(q[:n], kk[:n], v[:n], 0.37, want_p=True)
+    Hn = _harmonic(n)
+    for j in range(n):
+        assert acc0[j] == pytest.approx(float(Hn - _harmonic(j)), rel=1e-14)
+    for i in range(n):
+        np.testing.assert_allclose(P[i, : i + 1], 1.0 / (i + 1), rtol=1e-15)
+        assert np.all(P[i, i + 1:] == 0.0)
+        np.testing.assert_allclose(O[i], v[: i + 1].astype(np.float64).mean(axis=0), rtol=1e-13, atol=1e-15)
+
+    # harmonic tails decrease with position, so the heavy hitters are the first k tokens
+    kept, boundary = oracle.select(acc0, k, r)
+    assert kept.tolist() == list(range(k)) + list(range(n - r, n))
+    assert boundary[0] == pytest.approx(float(Hn - _harmonic(k - 1)), rel=1e-14)
+    assert boundary[1] == pytest.approx(float(Hn - _harmonic(k)), rel=1e-14)
+
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=0.37)
+    cache.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    B = k + r
+    expect = {j: Hn - _harmonic(j) for j in kept.tolist()}
+    for s in range(steps):
+        t = n + s
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        # B cached entries plus the new token share the probability mass equally
+        np.testing.assert_allclose(res["p"][0, : B + 1], 1.0 / (B + 1), rtol=1e-15)
+        members = sorted(expect) + [t]
+        np.testing.assert_allclose(res["out"][0], v[members].astype(np.float64).mean(axis=0), rtol=1e-12, atol=1e-14)
+        expect[t] = Fraction(0)
+        for j in expect:
+            expect[j] += Fraction(1, B + 1)
+        # the token that just left the recent window has the smallest accumulated score
+        assert res["evicted"][0] == t - r
+        del expect[t - r]
+        pos, acc = cache.export(0)
+        assert pos.tolist() == sorted(expect)
+        np.testing.assert_allclose(acc, [float(expect[j]) for j in sorted(expect)], rtol=1e-13)
+
+
+# --------------------------------------------------------------------------
+# brute force of the literal definition
+# --------------------------------------------------------------------------
+class LiteralH2O:
+    """Token-by-token policy, written for clarity only (pure Python, O(T^3)).
+
+    Keeps the full T x T matrix of attention probabilities (zero where a token was
+    not attended), so accumulated scores are explicit column sums, and evaluates
+    F_score(G \\ {v}) = h(sum of accumulated scores of G without v) for every
+    candidate v, taking the argmax.
+    """
+
+    def __init__(self, k, r, scale, h):
+        self.k, self.r, self.c, self.h = k, r, scale, h
+        self.S = []  # kept positions
+        self.rows = []  # rows[i][j] = probability token i gave token j
+        self.K, self.V = {}, {}
+        self.t = 0
+
+    def preload_rows(self, rows):
+        self.rows = [dict(r_) for r_ in rows]
+
+    def column_sum(self, j):
+        return math.fsum(row.get(j, 0.0) for row in self.rows)
+
+    def step(self, q, k_new, v_new):
+        t = self.t
+        self.K[t], self.V[t] = k_new, v_new
+        G = self.S + [t]
+        logits = [self.c * math.fsum(float(a) * float(b) for a, b in zip(q, self.K[j])) for j in G]
+        mx = max(logits)
+        w = [math.exp(x - mx) for x in logits]
+        tot = math.fsum(w)
+        probs = [x / tot for x in w]
+        self.rows.append({j: p for j, p in zip(G, probs)})
+        out = [math.fsum(p * float(self.V[j][x]) for j, p in zip(G, probs)) for x in range(len(q))]
+        evicted = -1
+        min_gap = math.inf
+        if len(G) > self.k + self.r:
+            cand = [j for j in G if j <= t - self.r]
+            colsum = {j: self.column_sum(j) for j in G}
+            best, best_val = None, None
+            for v_ in sorted(cand):  # ascending position: first maximum wins = lowest position
+                val = self.h(math.fsum(colsum[s] for s in G if s != v_))
+                if best is None or val > best_val:
+                    best, best_val = v_, val
+            evicted = best
+            cs = sorted(colsum[j] for j in cand)
+            if len(cs) > 1:
+                min_gap = (cs[1] - cs[0]) / max(abs(cs[1]), 1e-300)
+            G.remove(evicted)
+        self.S = G
+        self.t += 1
+        return out, evicted, probs, min_gap
+
+
+@pytest.mark.parametrize("hname", ["identity", "sqrt", "log"])
+@pytest.mark.parametrize("k,r", [(3, 0), (2, 2), (0, 3), (4, 1), (1, 4)])
+def test_sequential_policy_matches_literal_argmax(oracle, hname, k, r):
+    h = {"identity": lambda z: z, "sqrt": lambda z: math.sqrt(z + 1.0), "log": lambda z: math.log(z + 1.0)}[hname]
+    T, d, scale = 16, 4, 0.6
+    rng = np.random.default_rng(100 + 10 * k + r)
+    q, kk, v = _rand_qkv(rng, T, d)
+    lit = LiteralH2O(k, r, scale, h)
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    ever_evicted = set()
+    prev = set()
+    checked = 0
+    for t in range(T):
+        out_l, ev_l, probs, gap = lit.step(q[t], kk[t], v[t])
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        m = len(probs)
+        # every softmax row sums to one; same probabilities as the literal simulation
+        assert math.fsum(res["p"][0, :m]) == pytest.approx(1.0, abs=1e-14)
+        np.testing.assert_allclose(np.sort(res["p"][0, :m]), np.sort(probs), rtol=1e-12)
+        np.testing.assert_allclose(res["out"][0], out_l, rtol=1e-11, atol=1e-13)
+        if gap > 1e-9:  # the sum-minus-one form loses a few ulps; skip decisions it cannot resolve
+            assert res["evicted"][0] == ev_l
+            checked += 1
+        else:
+            pytest.skip("tiny accidental near-tie in random data")
+        pos, acc = cache.export(0)
+        # accumulated scores are explicit column sums of everything attended so far
+        np.testing.assert_allclose(acc, [lit.column_sum(j) for j in pos], rtol=1e-12)
+        now = set(pos.tolist())
+        assert now == set(lit.S)
+        assert len(now) <= k + r  # budget
+        assert len(now - prev) <= 1  # at most one new entry per step
+        if ev_l >= 0:
+            ever_evicted.add(ev_l)
+        assert not (now & ever_evicted)  # evicted entries never come back
+        assert set(range(max(0, t - r + 1), t + 1)) <= now  # recent window always present
+        prev = now
+    assert checked >= T - (k + r)
+
+
+def test_budget_three_example_structure(oracle):
+    """Budget 3: the fourth step still sees four tokens, then drops one for good (Figure 2's story)."""
+    rng = np.random.default_rng(5)
+    q, kk, v = _rand_qkv(rng, 8, 4)
+    cache = oracle.OracleCache(1, 1, 4, [3], [0], scale=0.5)
+    gone = None
+    for t in range(8):
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        if t < 3:
+            assert res["evicted"][0] == -1 and cache.cnt[0] == t + 1
+        if t == 3:
+            assert np.count_nonzero(res["p"][0]) == 4
+            gone = int(res["evicted"][0])
+            assert 0 <= gone <= 3
+        if t >= 3:
+            assert cache.cnt[0] == 3
+            assert gone not in cache.export(0)[0].tolist()
+
+
+# --------------------------------------------------------------------------
+# special cases that reduce to textbook attention
+# --------------------------------------------------------------------------
+def _textbook_causal(q, k, v, scale, window=None):
+    n = q.shape[0]
+    s = scale * (q.astype(np.float64) @ k.astype(np.float64).T)
+    i, j = np.indices((n, n))
+    mask = j <= i
+    if window is not None:
+        mask &= j >= i - window
+    s = np.where(mask, s, -np.inf)
+    p = scipy_softmax(s, axis=1)
+    return p @ v.astype(np.float64), p
+
+
+def test_budget_at_least_length_is_full_causal_attention(oracle):
+    n, steps, d, scale = 40, 12, 8, 0.3
+    rng = np.random.default_rng(7)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+    ref_out, ref_p = _textbook_causal(q, kk, v, scale)
+    cache = oracle.OracleCache(1, 1, d, [30], [n + steps - 30], scale=scale)
+    out, kept = cache.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    np.testing.assert_allclose(out[:, 0], ref_out[:n], rtol=1e-11, atol=1e-13)
+    assert kept[0].tolist() == list(range(n))
+    np.testing.assert_allclose(cache.export(0)[1], ref_p[:n].sum(axis=0)[:n], rtol=1e-12)
+    for s in range(steps):
+        t = n + s
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        assert res["evicted"][0] == -1
+        np.testing.assert_allclose(res["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+    pos, acc = cache.export(0)
+    assert pos.tolist() == list(range(n + steps))
+    np.testing.assert_allclose(acc, ref_p.sum(axis=0), rtol=1e-12)
+
+
+def test_prefill_outputs_are_full_causal_whatever_the_budget(oracle):
+    n, d, scale = 64, 8, 0.4
+    rng = np.random.default_rng(8)
+    q, kk, v = _rand_qkv(rng, n, d)
+    ref_out, ref_p = _textbook_causal(q, kk, v, scale)
+    O, acc0, P = oracle.causal_attention_colsum(q, kk, v, scale, want_p=True)
+    np.testing.assert_allclose(O, ref_out, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(P, ref_p, rtol=1e-11, atol=1e-300)
+    np.testing.assert_allclose(acc0, ref_p.sum(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(P.sum(axis=1), 1.0, rtol=1e-14)
+
+
+def test_zero_heavy_budget_is_sliding_window(oracle):
+    T, d, r, scale = 48, 8, 6, 0.5
+    rng = np.random.default_rng(9)
+    q, kk, v = _rand_qkv(rng, T, d)
+    ref_out, _ = _textbook_causal(q, kk, v, scale, window=r)
+    # token by token from an empty cache: every output is windowed attention
+    cache = oracle.OracleCache(1, 1, d, [0], [r], scale=scale)
+    for t in range(T):
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        np.testing.assert_allclose(res["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+        assert res["evicted"][0] == (t - r if t >= r else -1)
+    # after a one-shot prefill the decode steps are windowed as well
+    n = 30
+    cache = oracle.OracleCache(1, 1, d, [0], [r], scale=scale)
+    out, kept = cache.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    assert kept[0].tolist() == list(range(n - r, n))
+    np.testing.assert_allclose(out[:, 0], _textbook_causal(q[:n], kk[:n], v[:n], scale)[0], rtol=1e-11, atol=1e-13)
+    for t in range(n, T):
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        np.testing.assert_allclose(res["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+
+
+def test_sequential_fill_equals_prefill_when_nothing_is_evicted(oracle):
+    n, steps, d, scale = 20, 6, 4, 0.7
+    rng = np.random.default_rng(10)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+    a = oracle.OracleCache(1, 1, d, [n], [steps], scale=scale)
+    b = oracle.OracleCache(1, 1, d, [n], [steps], scale=scale)
+    out_a, _ = a.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    for t in range(n + steps):
+        rb = b.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        if t < n:
+            np.testing.assert_allclose(rb["out"][0], out_a[t, 0], rtol=1e-12, atol=1e-14)
+        else:
+            ra = a.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+            np.testing.assert_allclose(rb["out"][0], ra["out"][0], rtol=1e-12, atol=1e-14)
+    np.testing.assert_array_equal(a.export(0)[0], b.export(0)[0])
+    np.testing.assert_allclose(a.export(0)[1], b.export(0)[1], rtol=1e-12)
+
+
+# --------------------------------------------------------------------------
+# selection and tie-breaking
+# --------------------------------------------------------------------------
+def _select_by_repeated_eviction(acc0, k, r):
+    n = len(acc0)
+    if n <= k + r:
+        return list(range(n))
+    cand = list(range(n - r))
+    while len(cand) > k:
+        worst = min(cand, key=lambda j: (acc0[j], j))
+        cand.remove(worst)
+    return sorted(cand) + list(range(n - r, n))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_equals_repeated_min_eviction(oracle, seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(5, 60))
+    k = int(rng.integers(0, 12))
+    r = int(rng.integers(0, 12))
+    acc0 = rng.random(n)
+    acc0[rng.integers(0, n, size=n // 2)] = 0.5  # plenty of exact ties
+    kept, _ = oracle.select(acc0, k, r)
+    assert kept.tolist() == _select_by_repeated_eviction(acc0.tolist(), k, r)
+
+
+def test_select_ties_drop_lowest_position_first(oracle):
+    acc0 = np.array([1.0, 1.0, 1.0, 1.0, 9.0, 0.1, 0.2], dtype=np.float64)
+    kept, boundary = oracle.select(acc0, 2, 2)
+    assert kept.tolist() == [3, 4, 5, 6]
+    assert boundary.tolist() == [1.0, 1.0]
+    kept, _ = oracle.select(acc0, 0, 3)
+    assert kept.tolist() == [4, 5, 6]
+    kept, _ = oracle.select(acc0, 3, 0)
+    assert kept.tolist() == [2, 3, 4]
+
+
+def test_decode_tie_evicts_lowest_position_and_hint_protocol(oracle):
+    d = 2
+    cache = oracle.OracleCache(1, 1, d, [2], [1], scale=1.0)
+    kv = np.ones((3, d))
+    # stored out of position order on purpose; positions 7 and 4 tie
+    cache.load_unit(0, [7, 4, 9], [1.25, 1.25, 3.0], kv, kv, t=10)
+    snap = {n_: getattr(cache, n_).copy() for n_ in ("t", "cnt", "pos", "acc", "K", "V")}
+    z = np.zeros((1, 1, d), dtype=np.float32)
+    res = cache.decode_step(z, z + 1, z + 1)
+    assert res["evicted"][0] == 4 and res["status"][0] == 0 and res["gap"][0] == 0.0
+    assert cache.export(0)[0].tolist() == [7, 9, 10]
+
+    def restore():
+        for n_, a in snap.items():
+            getattr(cache, n_)[...] = a
+
+    restore()
+    res = cache.decode_step(z, z + 1, z + 1, hint=np.array([7], dtype=np.int32))
+    assert res["evicted"][0] == 4 and res["status"][0] == 1  # excused, and the hint is applied
+    assert cache.export(0)[0].tolist() == [4, 9, 10]
+    restore()
+    res = cache.decode_step(z, z + 1, z + 1, hint=np.array([9], dtype=np.int32))
+    assert res["status"][0] == 2  # a real disagreement; oracle's own choice stands
+    assert cache.export(0)[0].tolist() == [7, 9, 10]
+    restore()
+    res = cache.decode_step(z, z + 1, z + 1, hint=np.array([10], dtype=np.int32))
+    assert res["status"][0] == 2  # the new token is inside the recent window, not a candidate
+
+
+def test_entry_order_is_irrelevant(oracle):
+    n, steps, d, scale = 50, 20, 8, 0.35
+    rng = np.random.default_rng(11)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+    a = oracle.OracleCache(1, 1, d, [5], [4], scale=scale)
+    b = oracle.OracleCache(1, 1, d, [5], [4], scale=scale)
+    a.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    b.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    shuffler = np.random.default_rng(12)
+    for t in range(n, n + steps):
+        b.permute_entries(shuffler)
+        ra = a.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        rb = b.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        assert ra["evicted"][0] == rb["evicted"][0]
+        np.testing.assert_allclose(ra["out"], rb["out"], rtol=1e-12, atol=1e-14)
+    np.testing.assert_array_equal(a.export(0)[0], b.export(0)[0])
+    np.testing.assert_allclose(a.export(0)[1], b.export(0)[1], rtol=1e-12)
+
+
+def test_heads_and_sequences_are_independent(oracle):
+    """Batched, ragged call equals per-unit calls (different kept sets per head)."""
+    rng = np.random.default_rng(13)
+    lens, H, d = [9, 17, 5], 2, 4
+    heavy, recent = [2, 3, 4], [2, 3, 4]
+    tot = sum(lens)
+    q = rng.standard_normal((tot, H, d)).astype(np.float32)
+    k = rng.standard_normal((tot, H, d)).astype(np.float32)
+    v = rng.standard_normal((tot, H, d)).astype(np.float32)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    cache = oracle.OracleCache(len(lens), H, d, heavy, recent)
+    out, kept = cache.prefill(q, k, v, cu)
+    for s, n in enumerate(lens):
+        for h in range(H):
+            sl = slice(cu[s], cu[s + 1])
+            O, acc0 = oracle.causal_attention_colsum(q[sl, h], k[sl, h], v[sl, h], cache.scale)
+            np.testing.assert_array_equal(out[sl, h], O)
+            ks, _ = oracle.select(acc0, heavy[s], recent[s])
+            np.testing.assert_array_equal(kept[s * H + h], ks)
+    dq = rng.standard_normal((len(lens), H, d)).astype(np.float32)
+    full = oracle.OracleCache(len(lens), H, d, heavy, recent)
+    full.prefill(q, k, v, cu)
+    r_all = cache.decode_step(dq, dq * 0.5, dq * 2)
+    r_sub = full.decode_step(dq, dq * 0.5, dq * 2, units=[1, 4])
+    np.testing.assert_array_equal(r_sub["out"], r_all["out"][[1, 4]])
+    np.testing.assert_array_equal(r_sub["evicted"], r_all["evicted"][[1, 4]])
+    assert full.t[1] == lens[0] + 1 and full.t[0] == lens[0]
