@@ -78,26 +78,6 @@ def ragged_prompt_lengths(batch: int, lo: int, hi: int, seed: int) -> Tuple[int,
     return tuple(int(x) for x in torch.randint(lo, hi + 1, (batch,), generator=g))
 
 
-def _uniform(name, batch, heads, d, dtype, n, steps, k, r, layers=1, seed=20230614) -> Workload:
-    return Workload(name, batch, heads, d, dtype, (n,) * batch, steps, (k,) * batch, (r,) * batch, layers, seed)
-
-
-def _config5() -> Workload:
-    seed = 20230614 + 4
-    lens = ragged_prompt_lengths(128, 128, 4096, seed)
-    k, r = budgets_for(lens, 0.2)
-    return Workload("c5_ragged_32layer", 128, 32, 128, "bf16", lens, 128, k, r, 32, seed)
-
-
-CONFIGS = {
-    "c1_tiny": _uniform("c1_tiny", 1, 4, 64, "f32", 256, 64, 32, 32, seed=20230614 + 0),
-    "c2_opt6p7b": _uniform("c2_opt6p7b", 8, 32, 128, "bf16", 2048, 256, 205, 205, seed=20230614 + 1),
-    "c3_opt30b": _uniform("c3_opt30b", 64, 56, 128, "bf16", 512, 32, 52, 52, seed=20230614 + 2),
-    "c4_longctx": _uniform("c4_longctx", 1, 32, 128, "bf16", 32768, 512, 1024, 1024, seed=20230614 + 3),
-    "c5_ragged_32layer": _config5(),
-}
-
-
 def _mix(seed: int, layer: int, kind: int, step: int) -> int:
     """Derive an independent 63-bit stream seed from the four counters."""
     x = (seed * 0x9E3779B97F4A7C15 + layer * 0xBF58476D1CE4E5B9 + kind * 0x94D049BB133111EB + step * 0xD6E8FEB86659FD93) & (
@@ -152,3 +132,23 @@ def make_prompt_inputs(wl: Workload, layer: int = 0, device="cpu"):
 def make_decode_inputs(wl: Workload, step: int, layer: int = 0, device="cpu"):
     """q, k_new, v_new of shape ``[batch, n_heads, head_dim]`` for decode step ``step`` (0-based)."""
     return _make(wl, layer, 1 + step, wl.batch, device)
+
+
+def _uniform(name, batch, heads, d, dtype, n, steps, k, r, layers=1, seed=20230614) -> Workload:
+    return Workload(name, batch, heads, d, dtype, (n,) * batch, steps, (k,) * batch, (r,) * batch, layers, seed)
+
+
+def _config5() -> Workload:
+    seed = 20230614 + 4
+    lens = ragged_prompt_lengths(128, 128, 4096, seed)
+    k, r = budgets_for(lens, 0.2)
+    return Workload("c5_ragged_32layer", 128, 32, 128, "bf16", lens, 128, k, r, 32, seed)
+
+
+CONFIGS = {
+    "c1_tiny": _uniform("c1_tiny", 1, 4, 64, "f32", 256, 64, 32, 32, seed=20230614 + 0),
+    "c2_opt6p7b": _uniform("c2_opt6p7b", 8, 32, 128, "bf16", 2048, 256, 205, 205, seed=20230614 + 1),
+    "c3_opt30b": _uniform("c3_opt30b", 64, 56, 128, "bf16", 512, 32, 52, 52, seed=20230614 + 2),
+    "c4_longctx": _uniform("c4_longctx", 1, 32, 128, "bf16", 32768, 512, 1024, 1024, seed=20230614 + 3),
+    "c5_ragged_32layer": _config5(),
+}
