@@ -1,0 +1,174 @@
+/*
+ * h2o.h — C ABI of the B200 (sm_100a) implementation of the H2O KV-cache
+ * eviction hot path: attention over a budget-limited KV cache whose slots are
+ * kept or evicted by accumulated attention score.
+ *
+ * Vocabulary.  A *unit* is one (sequence, head); units never interact (the
+ * paper evicts "for each head", Appendix A).  Per sequence s the cache holds
+ * B_s = k_s + r_s *slots* per head: k_s heavy hitters and the r_s most recent
+ * tokens (Section 5 "evenly assigns the caching budget", Appendix A "first K
+ * entries heavy hitters, last K entries most recent").  Slot order carries no
+ * meaning; each slot records the token position it holds.
+ *
+ * Conventions common to every call
+ *   - Returns 0 (H2O_OK) or a negative H2O_ERR_* code; nothing is printed, thrown
+ *     or aborted.  On error no kernel has been launched by that call.
+ *   - "dev" pointers are CUDA device pointers on the cache's device, "host"
+ *     pointers are ordinary host memory.  The library never allocates or frees
+ *     device memory and keeps no caller pointer after a call returns, except the
+ *     workspace given to h2o_cache_create, which the caller must keep alive and
+ *     untouched until h2o_cache_destroy.
+ *   - Calls taking a stream are asynchronous on that stream (a cudaStream_t
+ *     passed as void*; NULL is the legacy default stream).  A cache must be
+ *     driven from one stream at a time.
+ *   - Tensors are dense, row-major, 16-byte aligned, of the cache's dtype.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x
+ *     h2o_cache_create fails with H2O_ERR_CUDA / H2O_ERR_UNSUPPORTED.
+ */
+#ifndef H2O_B200_H_
+#define H2O_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define H2O_OK 0
+#define H2O_ERR_INVALID_ARG (-1) /* NULL pointer, non-positive size, negative budget, ...      */
+#define H2O_ERR_UNSUPPORTED (-2) /* dtype / head_dim / device the kernels are not written for   */
+#define H2O_ERR_WORKSPACE (-3)   /* workspace or scratch too small or misaligned                */
+#define H2O_ERR_STATE (-4)       /* call order violated (e.g. second prefill on one cache)      */
+#define H2O_ERR_CUDA (-5)        /* a CUDA runtime call or kernel launch failed                 */
+#define H2O_ERR_TIMEOUT (-6)     /* a bounded device-side wait gave up (seen by h2o_cache_status) */
+
+typedef enum { H2O_F32 = 0, H2O_BF16 = 1 } h2o_dtype_t;
+
+typedef struct h2o_cache h2o_cache_t; /* opaque, host-side */
+
+/*
+ * Problem statement (Section 2.1: Q, K in R^{n x d} and a space budget;
+ * Appendix A: parameter K heavy + K recent, chosen per sequence here).
+ */
+typedef struct {
+  int32_t batch;                /* number of sequences, >= 1                                   */
+  int32_t n_heads;              /* heads per sequence, >= 1                                    */
+  int32_t head_dim;             /* d: 64 or 128                                                */
+  int32_t dtype;                /* h2o_dtype_t of q/k/v/out and of the stored K/V slots        */
+  const int32_t* heavy_budget;  /* host [batch]: k_s >= 0                                      */
+  const int32_t* recent_window; /* host [batch]: r_s >= 0, k_s + r_s >= 1                      */
+  float softmax_scale;          /* c in exp(c q.k); <= 0 selects 1/sqrt(head_dim)              */
+  int32_t device;               /* CUDA device ordinal                                         */
+} h2o_config_t;
+
+/* Bytes of device workspace h2o_cache_create needs for this configuration
+ * (K/V slots, accumulated scores, positions, counters).  Pure host arithmetic.
+ * Returns 0 for an invalid or unsupported configuration. */
+size_t h2o_cache_workspace_bytes(const h2o_config_t* cfg);
+
+/* Bytes of device scratch one h2o_prefill_select call needs for prompts of
+ * `total_tokens` tokens in all (row statistics and column sums, per head).
+ * Pure host arithmetic; 0 for invalid arguments. */
+size_t h2o_prefill_scratch_bytes(const h2o_config_t* cfg, int64_t total_tokens);
+
+/*
+ * Create an empty cache (every unit holds 0 tokens, next position t = 0) inside
+ * the caller's device workspace (256-byte aligned, at least
+ * h2o_cache_workspace_bytes(cfg) bytes).  The budget arrays are copied.  Small
+ * tables are copied to the device synchronously; no kernel state survives a
+ * failed create.  *out is set only on success.
+ * Pre-allocated storage that is overwritten in place follows Section 4.2
+ * ("do not swap memory ... directly fill with newly-added KV") and Appendix A.
+ */
+int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes);
+
+/*
+ * Prefill selection (Appendix A pseudocode, prefill branch: attention over the
+ * whole prompt, then "select K heavy hitters and K recent tokens", all tokens
+ * if the prompt is not longer than the budget).  For every unit:
+ *   P[i][j] = softmax_j(c q_i.k_j), j <= i          causal attention, n_s rows
+ *   out_i   = sum_j P[i][j] v_j
+ *   acc0[j] = sum_{i >= j} P[i][j]                   accumulated score (Algorithm 2, accumulation line)
+ *   keep the last r_s positions and the k_s positions of [0, n_s - r_s) with the
+ *   largest acc0 (equal scores: the higher position is kept), copy their K/V rows,
+ *   acc0 and position into the unit's slots; t = n_s.
+ * q, k, v, out : dev [total_tokens, n_heads, head_dim], sequences concatenated
+ *                token-major; out may not alias the inputs.
+ * cu_seqlens   : host [batch + 1], cu[0] = 0, non-decreasing; n_s = cu[s+1]-cu[s] >= 1.
+ * scratch      : dev, 256-byte aligned, >= h2o_prefill_scratch_bytes(cfg, cu[batch]);
+ *                used only by the work this call enqueues.
+ * Allowed once per cache and only before any decode step (H2O_ERR_STATE otherwise).
+ */
+int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const void* v,
+                       const int32_t* cu_seqlens, void* out, void* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * One decoding step for every unit, fused in one kernel (Algorithm 2 loop body
+ * with the cache layout of Appendix A).  With S the unit's kept set and t its
+ * next position:
+ *   p      = softmax over S u {t} of c q.k_x           (the new token attends to itself)
+ *   out    = sum_x p_x v_x
+ *   acc_x += p_x for x in S;  acc_t = p_t
+ *   if the unit already holds B_s tokens: evict the candidate (pos <= t - r_s) with
+ *   the smallest acc (equal: lowest position) and store the new token in its slot;
+ *   otherwise append.  With r_s = 0 the new token itself is a candidate and may be
+ *   the one dropped.  t += 1.
+ * q, k_new, v_new, out : dev [batch, n_heads, head_dim].
+ * evicted_pos          : dev [batch, n_heads] int32 or NULL; position evicted by this
+ *                        step, -1 if none.
+ * May be called on a cache that was never prefilled (token-by-token mode, the
+ * fill phase of Algorithm 2).
+ */
+int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const void* v_new, void* out,
+                    int32_t* evicted_pos, void* stream);
+
+/*
+ * The same two calls for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous).  Inputs are copied to `staging` (dev, 256-byte
+ * aligned) on the stream, the device call above runs on the staged copies, and the
+ * results are copied back to the host buffers on the same stream; the host buffers
+ * must stay valid until the stream has finished this work.
+ *   h2o_prefill_select_host: staging >= 4 tensors of [total_tokens, n_heads, head_dim]
+ *                            (each rounded up to 256 bytes); scratch as above.
+ *   h2o_decode_step_host   : staging >= 4 tensors of [batch, n_heads, head_dim] plus
+ *                            [batch, n_heads] int32 (each rounded up to 256 bytes).
+ * h2o_host_staging_bytes(cfg, tokens) gives the size for `tokens` rows per tensor
+ * (tokens = total_tokens for prefill, batch for decode); 0 for invalid arguments.
+ * No counterpart in the paper; the semantics are those of the device calls.
+ */
+size_t h2o_host_staging_bytes(const h2o_config_t* cfg, int64_t tokens);
+int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* k_host, const void* v_host,
+                            const int32_t* cu_seqlens, void* out_host, void* staging, size_t staging_bytes,
+                            void* scratch, size_t scratch_bytes, void* stream);
+int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_new_host, const void* v_new_host,
+                         void* out_host, int32_t* evicted_pos_host, void* staging, size_t staging_bytes, void* stream);
+
+/*
+ * Return the cache to the empty state of h2o_cache_create (every unit holds 0
+ * tokens, t = 0, status cleared) with work enqueued on the stream, so that a
+ * workspace can serve a new batch of prompts without a new handle.
+ */
+int h2o_cache_reset(h2o_cache_t* cache, void* stream);
+
+/* Free the host-side handle.  NULL is accepted.  The workspace stays the caller's. */
+int h2o_cache_destroy(h2o_cache_t* cache);
+
+/*
+ * Diagnostics (no counterpart in the paper).
+ * h2o_cache_export copies, for every unit u = s * n_heads + h, its slot table into
+ * host arrays with a fixed row pitch: pos [units][pitch] (unused entries -1),
+ * acc [units][pitch], count [units], t [units]; pitch >= max_s B_s.  Synchronises
+ * the stream.  Any output pointer may be NULL.
+ * h2o_cache_status synchronises the stream and returns the device status word
+ * (H2O_OK, or the first H2O_ERR_* a kernel recorded).
+ */
+int h2o_cache_export(h2o_cache_t* cache, int32_t* pos, double* acc, int32_t* count, int32_t* t, int32_t pitch,
+                     void* stream);
+int h2o_cache_status(h2o_cache_t* cache, void* stream);
+const char* h2o_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* H2O_B200_H_ */

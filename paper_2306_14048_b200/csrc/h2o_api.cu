@@ -1,0 +1,440 @@
+// Host side of the C ABI declared in include/h2o.h: argument checks, workspace
+// carving, call-order state machine and kernel launches.  No device memory is
+// allocated here; everything lives in the caller's workspace / scratch.
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <numeric>
+#include <vector>
+
+#include "h2o_internal.cuh"
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMaxSlotsPerUnit = 49152;  // scores of one unit must fit in shared memory
+constexpr int kMaxUnits = 65535;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+size_t elem_size(int dtype) { return dtype == H2O_F32 ? 4 : 2; }
+
+struct Layout {
+  size_t K, V, acc, pos, count, tpos, status, slot_off, kbud, rwin, order, total;
+  int64_t total_slots;
+  int max_B;
+};
+
+// 0 = fine, otherwise an H2O_ERR_* code.
+int check_config(const h2o_config_t* cfg) {
+  if (!cfg || !cfg->heavy_budget || !cfg->recent_window) return H2O_ERR_INVALID_ARG;
+  if (cfg->batch < 1 || cfg->n_heads < 1 || cfg->device < 0) return H2O_ERR_INVALID_ARG;
+  if (cfg->dtype != H2O_F32 && cfg->dtype != H2O_BF16) return H2O_ERR_UNSUPPORTED;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return H2O_ERR_UNSUPPORTED;
+  if ((int64_t)cfg->batch * cfg->n_heads > kMaxUnits) return H2O_ERR_UNSUPPORTED;
+  for (int s = 0; s < cfg->batch; ++s) {
+    const int64_t k = cfg->heavy_budget[s], r = cfg->recent_window[s];
+    if (k < 0 || r < 0 || k + r < 1) return H2O_ERR_INVALID_ARG;
+    if (k + r > kMaxSlotsPerUnit) return H2O_ERR_UNSUPPORTED;
+  }
+  if (std::isnan(cfg->softmax_scale) || std::isinf(cfg->softmax_scale)) return H2O_ERR_INVALID_ARG;
+  return H2O_OK;
+}
+
+Layout make_layout(const h2o_config_t* cfg) {
+  Layout L{};
+  int64_t slots = 0;
+  int max_B = 0;
+  for (int s = 0; s < cfg->batch; ++s) {
+    const int B = cfg->heavy_budget[s] + cfg->recent_window[s];
+    slots += (int64_t)B * cfg->n_heads;
+    max_B = std::max(max_B, B);
+  }
+  const size_t units = (size_t)cfg->batch * cfg->n_heads;
+  const size_t row = (size_t)cfg->head_dim * elem_size(cfg->dtype);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes);
+    return at;
+  };
+  L.K = take((size_t)slots * row);
+  L.V = take((size_t)slots * row);
+  L.acc = take((size_t)slots * sizeof(double));
+  L.pos = take((size_t)slots * sizeof(int32_t));
+  L.count = take(units * sizeof(int32_t));
+  L.tpos = take(units * sizeof(int32_t));
+  L.status = take(sizeof(int32_t));
+  L.slot_off = take(units * sizeof(int64_t));
+  L.kbud = take(units * sizeof(int32_t));
+  L.rwin = take(units * sizeof(int32_t));
+  L.order = take(units * sizeof(int32_t));
+  L.total = off;
+  L.total_slots = slots;
+  L.max_B = max_B;
+  return L;
+}
+
+struct ScratchLayout {
+  size_t rowmax, rowsum, acc0, cu, total;
+};
+
+ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens) {
+  ScratchLayout S{};
+  const size_t cells = (size_t)total_tokens * cfg->n_heads;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes);
+    return at;
+  };
+  S.rowmax = take(cells * sizeof(float));
+  S.rowsum = take(cells * sizeof(float));
+  S.acc0 = take(cells * sizeof(double));
+  S.cu = take(((size_t)cfg->batch + 1) * sizeof(int32_t));
+  S.total = off;
+  return S;
+}
+
+enum class Phase { Empty, Prefilled, Decoding };
+
+}  // namespace
+
+struct h2o_cache {
+  h2o_config_t cfg;
+  std::vector<int32_t> heavy, recent, cu;
+  Layout layout;
+  h2o::CacheView view;
+  Phase phase;
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = prev == dev || cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (ok && prev >= 0) {
+      int cur = -1;
+      if (cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+  }
+};
+
+}  // namespace
+
+extern "C" {
+
+size_t h2o_cache_workspace_bytes(const h2o_config_t* cfg) {
+  if (check_config(cfg) != H2O_OK) return 0;
+  return make_layout(cfg).total;
+}
+
+size_t h2o_prefill_scratch_bytes(const h2o_config_t* cfg, int64_t total_tokens) {
+  if (check_config(cfg) != H2O_OK || total_tokens < 1 || total_tokens > INT32_MAX) return 0;
+  return make_scratch_layout(cfg, total_tokens).total;
+}
+
+int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes) {
+  if (!out) return H2O_ERR_INVALID_ARG;
+  const int rc = check_config(cfg);
+  if (rc != H2O_OK) return rc;
+  if (!dev_workspace) return H2O_ERR_INVALID_ARG;
+  const Layout L = make_layout(cfg);
+  if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(dev_workspace) % kAlign) != 0) return H2O_ERR_WORKSPACE;
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  if (cfg->device >= ndev) return H2O_ERR_INVALID_ARG;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, cfg->device) != cudaSuccess) return H2O_ERR_CUDA;
+  if (major != 10) return H2O_ERR_UNSUPPORTED;  // the kernels are built for sm_100a only
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+
+  h2o_cache* c = new (std::nothrow) h2o_cache();
+  if (!c) return H2O_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->heavy.assign(cfg->heavy_budget, cfg->heavy_budget + cfg->batch);
+  c->recent.assign(cfg->recent_window, cfg->recent_window + cfg->batch);
+  c->cfg.heavy_budget = c->heavy.data();
+  c->cfg.recent_window = c->recent.data();
+  c->layout = L;
+  c->phase = Phase::Empty;
+
+  const int units = cfg->batch * cfg->n_heads;
+  std::vector<int64_t> slot_off(units);
+  std::vector<int32_t> kbud(units), rwin(units), order(units);
+  int64_t at = 0;
+  for (int u = 0; u < units; ++u) {
+    const int s = u / cfg->n_heads;
+    slot_off[u] = at;
+    kbud[u] = c->heavy[s];
+    rwin[u] = c->recent[s];
+    at += c->heavy[s] + c->recent[s];
+  }
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(),
+                   [&](int a, int b) { return kbud[a] + rwin[a] > kbud[b] + rwin[b]; });  // longest first
+
+  char* ws = static_cast<char*>(dev_workspace);
+  h2o::CacheView& v = c->view;
+  v.K = ws + L.K;
+  v.V = ws + L.V;
+  v.acc = reinterpret_cast<double*>(ws + L.acc);
+  v.pos = reinterpret_cast<int32_t*>(ws + L.pos);
+  v.count = reinterpret_cast<int32_t*>(ws + L.count);
+  v.tpos = reinterpret_cast<int32_t*>(ws + L.tpos);
+  v.status = reinterpret_cast<int32_t*>(ws + L.status);
+  v.slot_off = reinterpret_cast<const int64_t*>(ws + L.slot_off);
+  v.kbud = reinterpret_cast<const int32_t*>(ws + L.kbud);
+  v.rwin = reinterpret_cast<const int32_t*>(ws + L.rwin);
+  v.order = reinterpret_cast<const int32_t*>(ws + L.order);
+  v.units = units;
+  v.n_heads = cfg->n_heads;
+  v.head_dim = cfg->head_dim;
+  v.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+
+  bool ok = true;
+  ok = ok && cudaMemset(ws + L.acc, 0, L.slot_off - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
+  ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
+  ok = ok && cudaMemcpy(ws + L.slot_off, slot_off.data(), units * sizeof(int64_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(ws + L.kbud, kbud.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(ws + L.rwin, rwin.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(ws + L.order, order.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    delete c;
+    return H2O_ERR_CUDA;
+  }
+  *out = c;
+  return H2O_OK;
+}
+
+int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                       void* out, void* scratch, size_t scratch_bytes, void* stream) {
+  if (!cache || !q || !k || !v || !cu_seqlens || !out || !scratch) return H2O_ERR_INVALID_ARG;
+  if (cache->phase != Phase::Empty) return H2O_ERR_STATE;
+  const h2o_config_t& cfg = cache->cfg;
+  if (cu_seqlens[0] != 0) return H2O_ERR_INVALID_ARG;
+  int max_seqlen = 0;
+  for (int s = 0; s < cfg.batch; ++s) {
+    const int64_t n = (int64_t)cu_seqlens[s + 1] - cu_seqlens[s];
+    if (n < 1) return H2O_ERR_INVALID_ARG;
+    max_seqlen = std::max<int64_t>(max_seqlen, n);
+  }
+  const int64_t total = cu_seqlens[cfg.batch];
+  if (max_seqlen > kMaxSlotsPerUnit - 1) return H2O_ERR_UNSUPPORTED;  // limit of the shared-memory score row
+  const ScratchLayout S = make_scratch_layout(&cfg, total);
+  if (scratch_bytes < S.total || (reinterpret_cast<uintptr_t>(scratch) % kAlign) != 0) return H2O_ERR_WORKSPACE;
+  for (const void* p : {q, k, v, (const void*)out})
+    if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
+  if (out == q || out == k || out == v) return H2O_ERR_INVALID_ARG;
+
+  DeviceGuard guard(cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* sc = static_cast<char*>(scratch);
+  h2o::PrefillScratch ps;
+  ps.rowmax = reinterpret_cast<float*>(sc + S.rowmax);
+  ps.rowsum = reinterpret_cast<float*>(sc + S.rowsum);
+  ps.acc0 = reinterpret_cast<double*>(sc + S.acc0);
+  ps.cu = reinterpret_cast<int32_t*>(sc + S.cu);
+  ps.total_tokens = total;
+  cache->cu.assign(cu_seqlens, cu_seqlens + cfg.batch + 1);  // pageable source: staged before the call returns
+  if (cudaMemcpyAsync(ps.cu, cache->cu.data(), cache->cu.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  cudaError_t e = h2o::launch_prefill_naive(cache->view, ps, cfg.dtype, cfg.batch, max_seqlen, q, k, v, out, st);
+  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, cfg.dtype, cache->layout.max_B, k, v, st);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  cache->phase = Phase::Prefilled;
+  return H2O_OK;
+}
+
+int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const void* v_new, void* out,
+                    int32_t* evicted_pos, void* stream) {
+  if (!cache || !q || !k_new || !v_new || !out) return H2O_ERR_INVALID_ARG;
+  for (const void* p : {q, k_new, v_new, (const void*)out})
+    if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->layout.max_B, q, k_new, v_new, out,
+                                           evicted_pos, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  cache->phase = Phase::Decoding;
+  return H2O_OK;
+}
+
+size_t h2o_host_staging_bytes(const h2o_config_t* cfg, int64_t tokens) {
+  if (check_config(cfg) != H2O_OK || tokens < 1 || tokens > INT32_MAX) return 0;
+  const size_t tensor = align_up((size_t)tokens * cfg->n_heads * cfg->head_dim * elem_size(cfg->dtype));
+  return 4 * tensor + align_up((size_t)tokens * cfg->n_heads * sizeof(int32_t));
+}
+
+int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* k_host, const void* v_host,
+                            const int32_t* cu_seqlens, void* out_host, void* staging, size_t staging_bytes,
+                            void* scratch, size_t scratch_bytes, void* stream) {
+  if (!cache || !q_host || !k_host || !v_host || !cu_seqlens || !out_host || !staging) return H2O_ERR_INVALID_ARG;
+  if (cache->phase != Phase::Empty) return H2O_ERR_STATE;
+  const h2o_config_t& cfg = cache->cfg;
+  const int64_t total = cu_seqlens[cfg.batch];
+  if (total < 1) return H2O_ERR_INVALID_ARG;
+  if (staging_bytes < h2o_host_staging_bytes(&cfg, total) || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0)
+    return H2O_ERR_WORKSPACE;
+  DeviceGuard guard(cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)total * cfg.n_heads * cfg.head_dim * elem_size(cfg.dtype);
+  const size_t pitch = align_up(bytes);
+  char* sg = static_cast<char*>(staging);
+  bool ok = cudaMemcpyAsync(sg, q_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sg + pitch, k_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sg + 2 * pitch, v_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  const int rc = h2o_prefill_select(cache, sg, sg + pitch, sg + 2 * pitch, cu_seqlens, sg + 3 * pitch, scratch,
+                                    scratch_bytes, stream);
+  if (rc != H2O_OK) return rc;
+  if (cudaMemcpyAsync(out_host, sg + 3 * pitch, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  return H2O_OK;
+}
+
+int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_new_host, const void* v_new_host,
+                         void* out_host, int32_t* evicted_pos_host, void* staging, size_t staging_bytes, void* stream) {
+  if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !staging) return H2O_ERR_INVALID_ARG;
+  const h2o_config_t& cfg = cache->cfg;
+  if (staging_bytes < h2o_host_staging_bytes(&cfg, cfg.batch) || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0)
+    return H2O_ERR_WORKSPACE;
+  DeviceGuard guard(cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)cfg.batch * cfg.n_heads * cfg.head_dim * elem_size(cfg.dtype);
+  const size_t pitch = align_up(bytes);
+  char* sg = static_cast<char*>(staging);
+  int32_t* ev_dev = reinterpret_cast<int32_t*>(sg + 4 * pitch);
+  bool ok = cudaMemcpyAsync(sg, q_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sg + pitch, k_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sg + 2 * pitch, v_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  const int rc = h2o_decode_step(cache, sg, sg + pitch, sg + 2 * pitch, sg + 3 * pitch,
+                                 evicted_pos_host ? ev_dev : nullptr, stream);
+  if (rc != H2O_OK) return rc;
+  ok = cudaMemcpyAsync(out_host, sg + 3 * pitch, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (evicted_pos_host)
+    ok = ok && cudaMemcpyAsync(evicted_pos_host, ev_dev, (size_t)cfg.batch * cfg.n_heads * sizeof(int32_t),
+                               cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  return H2O_OK;
+}
+
+int h2o_cache_reset(h2o_cache_t* cache, void* stream) {
+  if (!cache) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Layout& L = cache->layout;
+  char* ws = static_cast<char*>(cache->view.K) - L.K;
+  bool ok = cudaMemsetAsync(ws + L.acc, 0, L.slot_off - L.acc, st) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t), st) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  cache->phase = Phase::Empty;
+  return H2O_OK;
+}
+
+int h2o_cache_destroy(h2o_cache_t* cache) {
+  delete cache;
+  return H2O_OK;
+}
+
+int h2o_cache_export(h2o_cache_t* cache, int32_t* pos, double* acc, int32_t* count, int32_t* t, int32_t pitch,
+                     void* stream) {
+  if (!cache) return H2O_ERR_INVALID_ARG;
+  if ((pos || acc) && pitch < cache->layout.max_B) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const h2o::CacheView& v = cache->view;
+  const size_t slots = (size_t)cache->layout.total_slots;
+  std::vector<int32_t> hpos(pos ? slots : 0);
+  std::vector<double> hacc(acc ? slots : 0);
+  bool ok = cudaStreamSynchronize(st) == cudaSuccess;
+  if (pos) ok = ok && cudaMemcpy(hpos.data(), v.pos, slots * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (acc) ok = ok && cudaMemcpy(hacc.data(), v.acc, slots * sizeof(double), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (count) ok = ok && cudaMemcpy(count, v.count, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (t) ok = ok && cudaMemcpy(t, v.tpos, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  size_t at = 0;
+  for (int u = 0; u < v.units; ++u) {
+    const int s = u / v.n_heads;
+    const int B = cache->heavy[s] + cache->recent[s];
+    for (int x = 0; x < pitch; ++x) {
+      if (pos) pos[(size_t)u * pitch + x] = x < B ? hpos[at + x] : -1;
+      if (acc) acc[(size_t)u * pitch + x] = x < B ? hacc[at + x] : 0.0;
+    }
+    at += B;
+  }
+  return H2O_OK;
+}
+
+int h2o_cache_status(h2o_cache_t* cache, void* stream) {
+  if (!cache) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  int32_t word = 0;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess ||
+      cudaMemcpy(&word, cache->view.status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  return word;
+}
+
+const char* h2o_strerror(int code) {
+  switch (code) {
+    case H2O_OK: return "ok";
+    case H2O_ERR_INVALID_ARG: return "invalid argument";
+    case H2O_ERR_UNSUPPORTED: return "unsupported dtype, head_dim, size or device";
+    case H2O_ERR_WORKSPACE: return "workspace or scratch too small or misaligned";
+    case H2O_ERR_STATE: return "call order violated or inconsistent cache state";
+    case H2O_ERR_CUDA: return "CUDA runtime error";
+    case H2O_ERR_TIMEOUT: return "bounded device-side wait timed out";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Internal declarations shared by the translation units of libh2o_b200.so.
+// Nothing here is part of the public ABI (see include/h2o.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "h2o.h"
+
+namespace h2o {
+
+// Device-side view of a cache.  All pointers live inside the caller's workspace.
+struct CacheView {
+  void* K;                  // [total_slots][d] storage dtype
+  void* V;                  // [total_slots][d]
+  double* acc;              // [total_slots] accumulated attention score
+  int32_t* pos;             // [total_slots] token position held by the slot
+  int32_t* count;           // [units] occupied slots
+  int32_t* tpos;            // [units] position of the next token
+  int32_t* status;          // [1] first error recorded by a kernel
+  const int64_t* slot_off;  // [units] first slot of the unit
+  const int32_t* kbud;      // [units] heavy budget k
+  const int32_t* rwin;      // [units] recent window r
+  const int32_t* order;     // [units] launch order (largest budget first)
+  int32_t units, n_heads, head_dim;
+  float scale;              // softmax scale c
+};
+
+// Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
+// index = h * total_tokens + token.
+struct PrefillScratch {
+  float* rowmax;   // m_i
+  float* rowsum;   // l_i
+  double* acc0;    // column sums
+  int32_t* cu;     // [batch + 1] device copy of cu_seqlens
+  int64_t total_tokens;
+};
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_decode(const CacheView& c, int dtype, int max_B, const void* q, const void* k_new, const void* v_new,
+                          void* out, int32_t* evicted_pos, cudaStream_t stream);
+cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int batch, int max_seqlen,
+                                 const void* q, const void* k, const void* v, void* out, cudaStream_t stream);
+cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
+                                 const void* v, cudaStream_t stream);
+
+// ---------------------------------------------------------------------------
+// Small device helpers
+// ---------------------------------------------------------------------------
+template <typename T>
+struct Vec16;  // 16-byte vector of T, widened to float on load
+
+template <>
+struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ __forceinline__ static void load(const float* p, float (&f)[4]) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+  }
+  __device__ __forceinline__ static void store(float* p, const float (&f)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+  }
+};
+
+template <>
+struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ __forceinline__ static void unpack(const uint4& v, float (&f)[8]) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+  __device__ __forceinline__ static void load(const __nv_bfloat16* p, float (&f)[8]) {
+    unpack(*reinterpret_cast<const uint4*>(p), f);
+  }
+  __device__ __forceinline__ static uint32_t pack2(float lo, float hi) {
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&b);
+  }
+  __device__ __forceinline__ static void store(__nv_bfloat16* p, const float (&f)[8]) {
+    uint4 v;
+    v.x = pack2(f[0], f[1]); v.y = pack2(f[2], f[3]); v.z = pack2(f[4], f[5]); v.w = pack2(f[6], f[7]);
+    *reinterpret_cast<uint4*>(p) = v;
+  }
+};
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+}  // namespace h2o

@@ -1,0 +1,119 @@
+// Prompt attention and column sums on the fp32 FMA pipe, for every dtype and head_dim.
+// This is the path of fp32 inputs (tensor cores would round them to TF32, which the
+// exact-decision requirement cannot afford) and of head_dim 64.
+//
+//   rows kernel   : one thread block per (unit, query row i): P[i][0..i], out_i, m_i, l_i
+//   colsum kernel : one thread per key column j: acc0[j] = sum_{i >= j} exp(c q_i.k_j - m_i) / l_i
+//
+// Paper: causal attention of the prompt (Appendix A pseudocode, prefill branch) and the
+// accumulated score of Algorithm 2 evaluated for all prompt rows at once.
+#include "attend.cuh"
+
+namespace h2o {
+
+namespace {
+
+constexpr int kRowThreads = 128;
+constexpr int kColThreads = 128;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kRowThreads)
+prefill_rows_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, const T* __restrict__ k,
+                    const T* __restrict__ v, T* __restrict__ out) {
+  using A = Attend<T, D, kRowThreads>;
+  constexpr int VEC = A::VEC, LPR = A::LPR;
+  extern __shared__ float p[];
+  __shared__ typename A::Smem sm;
+  const int u = blockIdx.y;
+  const int seq = u / c.n_heads, h = u % c.n_heads;
+  const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
+  const int i = blockIdx.x;
+  if (i >= n) return;
+  const int64_t stride = (int64_t)c.n_heads * D;
+  const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
+  float o[VEC], m, l;
+  A::run(q + base + i * stride, k + base, v + base, stride, i + 1, nullptr, nullptr, c.scale, p, sm, o, m, l);
+  if (threadIdx.x < LPR) Vec16<T>::store(out + base + i * stride + threadIdx.x * VEC, o);
+  if (threadIdx.x == 0) {
+    s.rowmax[(int64_t)h * s.total_tokens + lo + i] = m;
+    s.rowsum[(int64_t)h * s.total_tokens + lo + i] = l;
+  }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kColThreads)
+prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, const T* __restrict__ k) {
+  constexpr int VEC = Vec16<T>::N;
+  const int u = blockIdx.y;
+  const int seq = u / c.n_heads, h = u % c.n_heads;
+  const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
+  const int j0 = blockIdx.x * kColThreads;
+  if (j0 >= n) return;
+  const int j = j0 + threadIdx.x;
+  const int64_t stride = (int64_t)c.n_heads * D;
+  const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
+  const float* rowmax = s.rowmax + (int64_t)h * s.total_tokens + lo;
+  const float* rowsum = s.rowsum + (int64_t)h * s.total_tokens + lo;
+
+  float kf[D];
+  if (j < n) {
+#pragma unroll
+    for (int x = 0; x < D; x += VEC) {
+      float t[VEC];
+      Vec16<T>::load(k + base + j * stride + x, t);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) kf[x + e] = t[e];
+    }
+  } else {
+#pragma unroll
+    for (int x = 0; x < D; ++x) kf[x] = 0.f;
+  }
+  double a = 0.0;
+  for (int i = j0; i < n; ++i) {  // every thread of the block reads the same query row (broadcast)
+    const T* qi = q + base + i * stride;
+    float dot = 0.f;
+#pragma unroll
+    for (int x = 0; x < D; x += VEC) {
+      float t[VEC];
+      Vec16<T>::load(qi + x, t);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) dot = fmaf(t[e], kf[x + e], dot);
+    }
+    if (i >= j) a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
+  }
+  if (j < n) s.acc0[(int64_t)h * s.total_tokens + lo + j] = a;
+}
+
+template <typename T, int D>
+cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
+                   const void* v, void* out, cudaStream_t stream) {
+  const size_t smem = sizeof(float) * (size_t)(max_seqlen + 1);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(prefill_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  dim3 grid_rows((unsigned)max_seqlen, (unsigned)c.units);
+  prefill_rows_kernel<T, D><<<grid_rows, kRowThreads, smem, stream>>>(
+      c, s, static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(out));
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  dim3 grid_cols((unsigned)((max_seqlen + kColThreads - 1) / kColThreads), (unsigned)c.units);
+  prefill_colsum_kernel<T, D><<<grid_cols, kColThreads, 0, stream>>>(c, s, static_cast<const T*>(q),
+                                                                    static_cast<const T*>(k));
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int batch, int max_seqlen,
+                                 const void* q, const void* k, const void* v, void* out, cudaStream_t stream) {
+  (void)batch;
+  if (dtype == H2O_F32) {
+    if (c.head_dim == 64) return launch<float, 64>(c, s, max_seqlen, q, k, v, out, stream);
+    return launch<float, 128>(c, s, max_seqlen, q, k, v, out, stream);
+  }
+  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, s, max_seqlen, q, k, v, out, stream);
+  return launch<__nv_bfloat16, 128>(c, s, max_seqlen, q, k, v, out, stream);
+}
+
+}  // namespace h2o

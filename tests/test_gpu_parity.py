@@ -1,0 +1,74 @@
+"""CUDA path vs oracle, element by element, through the C ABI (needs a B200)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from workloads import CONFIGS, Workload
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H2OCache():
+    import paper_2306_14048_b200 as pkg
+
+    assert torch.cuda.is_available(), "these tests need a CUDA device; there is no CPU fallback"
+    return pkg.H2OCache
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _oracle_built(oracle):
+    return oracle
+
+
+def _wl(name, batch, heads, d, dtype, lens, steps, heavy, recent, seed=1234):
+    return Workload(name, batch, heads, d, dtype, tuple(lens), steps, tuple(heavy), tuple(recent), 1, seed)
+
+
+def test_config1_tiny_fp32_full(H2OCache):
+    from parity_harness import run_parity
+
+    st = run_parity(CONFIGS["c1_tiny"], H2OCache, export_every=8)
+    assert st.decisions == 4 + 4 * 64
+    print(st)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
+def test_small_ragged_all_dtypes(H2OCache, dtype, d):
+    """Ragged batch spanning several tiles and ragged tails; one prompt shorter than its budget."""
+    from parity_harness import run_parity
+
+    wl = _wl("small", 4, 3, d, dtype, [300, 77, 513, 40], 48, [20, 9, 33, 30], [24, 5, 31, 30], seed=77 + d)
+    st = run_parity(wl, H2OCache, export_every=8)
+    print(st)
+
+
+@pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([1, 0], [0, 1]), ([3, 2], [1, 2])])
+def test_edge_budgets(H2OCache, heavy, recent):
+    """k = 0 (sliding window), r = 0 (the new token may be the one dropped), single-slot caches."""
+    from parity_harness import run_parity
+
+    wl = _wl("edge", 2, 2, 64, "f32", [37, 21], 40, heavy, recent, seed=5)
+    st = run_parity(wl, H2OCache, export_every=4)
+    print(st)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_token_by_token_from_empty_cache(H2OCache, dtype, d):
+    """No prefill: the fill phase of Algorithm 2, then steady-state eviction."""
+    from parity_harness import run_parity
+
+    wl = _wl("seq", 2, 2, d, dtype, [1, 1], 90, [10, 4], [6, 20], seed=9)
+    st = run_parity(wl, H2OCache, prefill=False, export_every=5)
+    print(st)
+
+
+def test_peaky_softmax_stress(H2OCache):
+    """Four times the default scale: many tiny probabilities, more near-equal scores."""
+    from parity_harness import run_parity
+
+    wl = _wl("peaky", 2, 4, 128, "bf16", [700, 450], 64, [40, 30], [40, 30], seed=21)
+    st = run_parity(wl, H2OCache, scale=4.0 / np.sqrt(128.0), export_every=16)
+    print(st)
