@@ -191,6 +191,10 @@ def main():
     ap.add_argument("--layers", type=int, default=8, help="independent layer caches rotated per decode step")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the config's decode step count")
     ap.add_argument("--ref-units", type=int, default=4)
+    ap.add_argument("--split", type=int, default=0, help="decode thread blocks per unit (0 = library default)")
+    ap.add_argument("--stages", type=int, default=0, help="decode ring depth (0 = library default)")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="launch every decode step from the host instead of replaying a CUDA graph of the decode loop")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -227,6 +231,8 @@ def main():
     esize = 4 if wl.dtype == "f32" else 2
     stream = torch.cuda.Stream(device=dev)
     caches = [pkg.H2OCache(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, device=local) for _ in range(L)]
+    for cch in caches:
+        cch.set_decode_shape(args.split, args.stages)
     cu = wl.cu_seqlens()
     prompts, dec = [], []
     for l in range(L):  # each rank draws its own data: the units are independent, nothing is exchanged
@@ -238,6 +244,33 @@ def main():
                     torch.empty(S, wl.batch, H, dtype=torch.int32, device=dev)))
     torch.cuda.synchronize()
 
+    # raw pointers once, so that the host loop is a bare C call per launch
+    sp = int(stream.cuda_stream)
+    dec_args = [[(caches[l]._h, dec[l][0][s].data_ptr(), dec[l][1][s].data_ptr(), dec[l][2][s].data_ptr(),
+                  dec[l][3][s].data_ptr(), dec[l][4][s].data_ptr(), sp) for l in range(L)] for s in range(S)]
+    c_decode = pkg.lib.h2o_decode_step
+
+    def decode_loop():
+        for s in range(S):
+            for a in dec_args[s]:
+                rc = c_decode(*a)
+                if rc != 0:
+                    raise pkg.H2OError(rc, "h2o_decode_step")
+
+    graph = None
+    if args.graph:
+        # the decode loop of one step (S x L launches of h2o_decode_step) as one CUDA graph
+        for l in range(L):
+            q, k, v, o = prompts[l]
+            caches[l].reset(stream)
+            caches[l].prefill_select(q, k, v, cu, o, stream)
+        decode_loop()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            decode_loop()
+        torch.cuda.synchronize()
+
     def one_step(ev=None):
         if ev:
             ev[0].record(stream)
@@ -247,10 +280,11 @@ def main():
             caches[l].prefill_select(q, k, v, cu, o, stream)
         if ev:
             ev[1].record(stream)
-        for s in range(S):
-            for l in range(L):
-                dq, dk, dv, do, de = dec[l]
-                caches[l].decode_step(dq[s], dk[s], dv[s], do[s], de[s], stream)
+        if graph is not None:
+            with torch.cuda.stream(stream):
+                graph.replay()
+        else:
+            decode_loop()
         if ev:
             ev[2].record(stream)
 
@@ -333,6 +367,7 @@ def main():
                 "workload": "%s x %d layer caches" % (wl.name, L), "batch": wl.batch, "n_heads": H, "head_dim": d,
                 "prompt_len": int(np.mean(wl.prompt_lens)), "decode_steps": S, "heavy": int(np.mean(wl.heavy)),
                 "recent": int(np.mean(wl.recent)), "layers": L,
+                "decode_launch": "cuda graph of the decode loop" if graph is not None else "one host call per launch",
                 "l2": "inputs larger than L2: %d layer caches of %.0f MB rotated every decode launch" % (
                     L, bytes_launch / 1e6),
             },

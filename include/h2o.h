@@ -166,6 +166,14 @@ int h2o_cache_destroy(h2o_cache_t* cache);
 int h2o_cache_export(h2o_cache_t* cache, int32_t* pos, double* acc, int32_t* count, int32_t* t, int32_t pitch,
                      void* stream);
 int h2o_cache_status(h2o_cache_t* cache, void* stream);
+/*
+ * Tuning knob (no counterpart in the paper): how the decode kernel is laid out.
+ * split  = thread blocks (one cluster) sharing a unit: 1, 2, 4 or 8; 0 keeps the
+ *          value chosen at create time from the number of units and the budgets.
+ * stages = depth of the shared-memory ring of 16 KB (K tile + V tile) stages, 1..8;
+ *          0 = default.  Results do not depend on either value beyond summation order.
+ */
+int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages);
 const char* h2o_strerror(int code);
 
 #ifdef __cplusplus

@@ -39,6 +39,7 @@ EXPORTED = (
     "h2o_decode_step_host",
     "h2o_cache_export",
     "h2o_cache_status",
+    "h2o_cache_set_decode_shape",
     "h2o_strerror",
 )
 
@@ -88,6 +89,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_export.argtypes = [vp, i32p, c.POINTER(c.c_double), i32p, i32p, c.c_int32, vp]
     lib.h2o_cache_status.restype = c.c_int
     lib.h2o_cache_status.argtypes = [vp, vp]
+    lib.h2o_cache_set_decode_shape.restype = c.c_int
+    lib.h2o_cache_set_decode_shape.argtypes = [vp, c.c_int32, c.c_int32]
     lib.h2o_strerror.restype = c.c_char_p
     lib.h2o_strerror.argtypes = [c.c_int]
     return lib
@@ -214,6 +217,9 @@ class H2OCache:
                                     count.ctypes.data_as(i32p), t.ctypes.data_as(i32p), pitch, _stream_ptr(stream)),
                "h2o_cache_export")
         return pos, acc, count, t
+
+    def set_decode_shape(self, split: int = 0, stages: int = 0):
+        _check(lib.h2o_cache_set_decode_shape(self._h, int(split), int(stages)), "h2o_cache_set_decode_shape")
 
     def status(self, stream=None) -> int:
         return int(lib.h2o_cache_status(self._h, _stream_ptr(stream)))

@@ -1,152 +1,517 @@
 // Fused decode step: scores over the occupied slots, softmax, weighted values,
-// score accumulation, victim search and in-place replacement — one kernel, one
-// thread block per (sequence, head), the cache read exactly once.
+// score accumulation, victim search and in-place replacement — one kernel launch,
+// the cache read exactly once.
 //
-// Paper: Algorithm 2 loop body (scores, accumulate, argmax of F_score(G \ {v}) which
+// Paper: Algorithm 2 loop body (scores, accumulate, argmax of F_score(G \ {v}), which
 // for the summation score is the candidate with the smallest accumulated score) on
 // the pre-allocated, overwritten-in-place cache of Section 4.2 / Appendix A.
-#include <cfloat>
+//
+// Shape of the kernel (the step is bound by HBM traffic, about one flop per byte):
+//   - A unit's slots are split over `split` thread blocks that form one cluster; each
+//     block owns `chunk` consecutive slots.  split = 1 for many small units, up to 8
+//     for few long ones, so that every SM has several blocks resident.
+//   - K tiles, then V tiles, of 8 KB each are streamed into a shared-memory ring with
+//     cp.async.bulk (the TMA engine, one elected thread issues, completion counted on
+//     an mbarrier).  The first STAGES tiles are issued before anything else happens, so
+//     V tiles are already in flight while the softmax of the K pass is computed.
+//   - Raw scores stay in shared memory; the softmax is exact (two passes over on-chip
+//     scores, no online rescaling).  Blocks of a cluster exchange (max, sum), partial
+//     outputs and victim candidates through distributed shared memory.
+//   - Accumulated scores are fp64 in memory: eviction decisions compare sums of
+//     hundreds of probabilities and must not depend on fp32 rounding of the sum.
+// Every wait on an mbarrier is bounded; a wait that gives up records H2O_ERR_TIMEOUT in
+// the status word and the block carries on (results of that step are then invalid).
+#include <climits>
+#include <cooperative_groups.h>
 
-#include "attend.cuh"
+#include "h2o_internal.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace h2o {
 
 namespace {
 
-constexpr int kDecodeThreads = 256;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kTileBytes = 8192;
+constexpr int kMaxStages = 8;
+constexpr int kDefaultStages = 4;
+constexpr int kMaxSplit = 8;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kMaxDynSmem = 200 * 1024;  // plus ~9 KB static shared memory stays below the 227 KB limit
 
+// Eviction candidate.  Accumulated scores are sums of probabilities (>= 0), so the bit
+// pattern of the double orders like its value; comparing the integer key keeps the
+// (slow) fp64 pipe out of the search.
 struct Cand {
-  double acc;
+  unsigned long long key;  // bit pattern of the accumulated score
   int pos;
-  int slot;  // -1: none, -2: the new token itself
+  int slot;  // slot index inside the unit; -1: none, -2: the new token itself
 };
-
+__device__ __forceinline__ Cand cand_none() { return Cand{~0ull, INT_MAX, -1}; }
+__device__ __forceinline__ Cand cand_make(double acc, int pos, int slot) {
+  return Cand{(unsigned long long)__double_as_longlong(acc), pos, slot};
+}
 __device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {
   if (a.slot == -1) return false;
   if (b.slot == -1) return true;
-  return a.acc < b.acc || (a.acc == b.acc && a.pos < b.pos);
+  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
 }
 
-__device__ __forceinline__ Cand cand_shfl_xor(const Cand& a, int off) {
+// Warp-wide minimum under the eviction order; every lane gets the winner.  Accumulated
+// scores are >= 0, so their bit patterns order like the values and three 32-bit
+// hardware reductions (high word, low word, position) find the winner.
+__device__ __forceinline__ Cand warp_argmin(const Cand& a) {
+  const bool valid = a.slot != -1;
+  const unsigned long long bits = valid ? a.key : ~0ull;
+  const unsigned hi = (unsigned)(bits >> 32), lo = (unsigned)bits;
+  const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
+  const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+  const bool tie = valid && hi == mh && lo == ml;
+  const unsigned mp = __reduce_min_sync(0xffffffffu, tie ? (unsigned)a.pos : 0xffffffffu);
+  const unsigned who = __ballot_sync(0xffffffffu, tie && (unsigned)a.pos == mp);
+  if (who == 0) return cand_none();
+  const int src = __ffs(who) - 1;
   Cand b;
-  b.acc = __shfl_xor_sync(0xffffffffu, a.acc, off);
-  b.pos = __shfl_xor_sync(0xffffffffu, a.pos, off);
-  b.slot = __shfl_xor_sync(0xffffffffu, a.slot, off);
+  b.key = ((unsigned long long)mh << 32) | ml;
+  b.pos = (int)mp;
+  b.slot = __shfl_sync(0xffffffffu, a.slot, src);
   return b;
 }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kDecodeThreads)
-decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
-              T* __restrict__ out, int32_t* __restrict__ evicted_pos) {
-  using A = Attend<T, D, kDecodeThreads>;
-  constexpr int VEC = A::VEC, LPR = A::LPR, WARPS = A::WARPS;
-  extern __shared__ float p[];  // [cnt + 1] scores, then probabilities
-  __shared__ typename A::Smem sm;
-  __shared__ Cand wbest[WARPS];
-  __shared__ int victim_sh;
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false after kSpinLimit unsuccessful polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// global -> shared bulk copy (16-byte aligned addresses, size a multiple of 16)
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// Optional phase timers (compile with -DH2O_PHASE_TIMERS): thread 0 of every block records
+// %globaltimer at a few points; h2o_debug_phase_timers copies them out.  Off in normal builds.
+#ifdef H2O_PHASE_TIMERS
+__device__ unsigned long long g_phase[8192 * 16];
+#define H2O_STAMP(i)                                                                   \
+  do {                                                                                 \
+    if (threadIdx.x == 0 && blockIdx.x < 8192) {                                       \
+      unsigned long long ts_;                                                          \
+      asm volatile("mov.u64 %0, %%clock64;" : "=l"(ts_));                             \
+      g_phase[blockIdx.x * 16 + (i)] = ts_;                                             \
+    }                                                                                  \
+  } while (0)
+#else
+#define H2O_STAMP(i) do { } while (0)
+#endif
+
+template <typename T, int D>
+struct Cfg {
+  static constexpr int VEC = Vec16<T>::N;
+  static constexpr int LPR = D / VEC;                  // lanes per row
+  static constexpr int RPW = 32 / LPR;                 // rows per warp pass (= row groups per warp)
+  static constexpr int RPC = kWarps * RPW;             // rows per block pass
+  static constexpr int GROUPS = kWarps * RPW;          // independent online-softmax streams per block
+  static constexpr int ROW_BYTES = D * (int)sizeof(T);
+  static constexpr int TILE_ROWS = kTileBytes / ROW_BYTES;
+  static constexpr int PASSES = TILE_ROWS / RPC;
+  static_assert(TILE_ROWS % RPC == 0 && PASSES >= 1, "tile must be a whole number of block passes");
+  static_assert(GROUPS <= 32, "group statistics are combined by one warp");
+};
+
+template <int GROUPS, int D>
+struct Shared {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t aux;
+  float red[GROUPS][D];  // per-group partial outputs (unnormalised, relative to the group's maximum)
+  float gm[GROUPS], gl[GROUPS];
+  Cand wbest[kWarps];
+  float m_c, l_c;      // block statistics, also read by the other blocks of the cluster
+  float x_out[D];      // block partial output relative to m_c (read by rank 0)
+  Cand x_cand;
+};
+
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads + 32)
+decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
+              T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages) {
+  using C = Cfg<T, D>;
+  constexpr int VEC = C::VEC, LPR = C::LPR, RPW = C::RPW, RPC = C::RPC, TILE_ROWS = C::TILE_ROWS, GROUPS = C::GROUPS;
+  extern __shared__ __align__(128) unsigned char dyn[];
+  __shared__ Shared<GROUPS, D> sh;
+  // dynamic layout: ring[stages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk + 1] f32
+  unsigned char* ring = dyn;
+  double* acc_s = reinterpret_cast<double*>(dyn + (size_t)stages * 2 * kTileBytes);
+  int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
+  float* p = reinterpret_cast<float*>(pos_s + chunk);
+
+  H2O_STAMP(1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int u = c.order[blockIdx.x];
-  const int cnt = c.count[u];
-  const int t = c.tpos[u];
-  const int r = c.rwin[u];
-  const int B = c.kbud[u] + r;
-  const int64_t s0 = c.slot_off[u];
-  T* Kb = reinterpret_cast<T*>(c.K) + s0 * D;
-  T* Vb = reinterpret_cast<T*>(c.V) + s0 * D;
-  double* acc = c.acc + s0;
-  int32_t* pos = c.pos + s0;
+  const int sub = lane / LPR, ch = lane % LPR;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = split > 1 ? (int)cluster.block_rank() : 0;
+  const int su = blockIdx.x / split;  // launch position of the unit
+  const UnitMeta mt = c.meta[su];     // static table, written once at create time
+  // Programmatic dependent launch: this grid may have been started while the previous kernel of
+  // the stream was still draining.  Let the next one start as early as it can, and wait for the
+  // previous one to finish (and flush) before reading anything it may have written.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int cnt = c.count[su];
+  const int t = c.tpos[su];
+  const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
+  const int lo = rank * chunk;                            // first slot of this block
+  const int nloc = max(0, min(cnt - lo, chunk));          // occupied slots of this block
+  const int ntile = (nloc + TILE_ROWS - 1) / TILE_ROWS;   // stages to stream (one K tile + one V tile each)
+  T* Kb = reinterpret_cast<T*>(c.K) + (mt.slot_off + lo) * D;
+  T* Vb = reinterpret_cast<T*>(c.V) + (mt.slot_off + lo) * D;
+  double* acc_g = c.acc + mt.slot_off + lo;
+  int32_t* pos_g = c.pos + mt.slot_off + lo;
   const T* qu = q + (int64_t)u * D;
   const T* ku = k_new + (int64_t)u * D;
   const T* vu = v_new + (int64_t)u * D;
+  bool timed_out = false;
 
-  float o[VEC], m, l;
-  A::run(qu, Kb, Vb, D, cnt, ku, vu, c.scale, p, sm, o, m, l);
-  if (tid < LPR) Vec16<T>::store(out + (int64_t)u * D + tid * VEC, o);
+  auto issue_stage = [&](int j) {  // producer lane only
+    const int s = j % stages;
+    const int rows = min(TILE_ROWS, nloc - j * TILE_ROWS);
+    const uint32_t bytes = (uint32_t)rows * C::ROW_BYTES;
+    unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
+    mbar_expect_tx(&sh.full[s], 2 * bytes);
+    bulk_g2s(dst, Kb + (int64_t)j * TILE_ROWS * D, bytes, &sh.full[s]);
+    bulk_g2s(dst + kTileBytes, Vb + (int64_t)j * TILE_ROWS * D, bytes, &sh.full[s]);
+  };
+  if (tid == kThreads) {  // producer lane: set up the barriers and get the first tiles moving at once
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], kWarps);
+    }
+    mbar_init(&sh.aux, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int j = 0; j < min(stages, ntile); ++j) issue_stage(j);
+    if (nloc > 0) {
+      const int npad = (nloc + 3) & ~3;  // stays inside the unit's padded slot range
+      mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
+      bulk_g2s(acc_s, acc_g, (uint32_t)npad * 8u, &sh.aux);
+      bulk_g2s(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
+    }
+  }
+  __syncthreads();  // barriers are initialised before any consumer polls them
 
-  // accumulate (Algorithm 2: o~_i = o~_{i-1} + o_i) and search the victim among the
-  // entries outside the recent window
-  const bool full = cnt >= B;
-  Cand best{DBL_MAX, INT_MAX, -1};
-  for (int x = tid; x < cnt; x += kDecodeThreads) {
-    const double a = acc[x] + (double)p[x];
-    acc[x] = a;
-    const int px = pos[x];
-    if (full && px <= t - r) {
-      const Cand cx{a, px, x};
-      if (cand_before(cx, best)) best = cx;
+  // the new token's own key/value: loaded now, used after the stream
+  float qf[VEC], ksf[VEC], vself = 0.f;
+  Vec16<T>::load(qu + ch * VEC, qf);
+  Vec16<T>::load(ku + ch * VEC, ksf);
+  if (tid < D) {
+    if constexpr (sizeof(T) == 4) vself = *reinterpret_cast<const float*>(vu + tid);
+    else vself = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(vu + tid));
+  }
+  float m = 0.f, l = 1.f, s_self = -INFINITY;
+
+  if (warp == kWarps) {
+    // ---- producer warp: one lane streams the tiles through the ring ------------------
+    if (lane == 0) {
+      for (int j = stages; j < ntile; ++j) {
+        if (!mbar_wait(&sh.empty[j % stages], (uint32_t)(j / stages - 1) & 1u)) timed_out = true;
+        issue_stage(j);
+      }
     }
-  }
-  if (full && r == 0 && tid == 0) {  // without a recent window the new token competes too
-    const Cand cs{(double)p[cnt], t, -2};
-    if (cand_before(cs, best)) best = cs;
-  }
+    if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    __syncwarp();
+    if (split > 1) {  // the producer warp only keeps the cluster barriers balanced
+      cluster.sync();
+      cluster.sync();
+    }
+  } else {
+    // ---- consumer warps: every row group keeps its own online softmax ------------------
+    float o[VEC];
 #pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const Cand other = cand_shfl_xor(best, off);
-    if (cand_before(other, best)) best = other;
-  }
-  if (lane == 0) wbest[warp] = best;
-  __syncthreads();
-  if (tid == 0) {
-    Cand b = wbest[0];
+    for (int v = 0; v < VEC; ++v) o[v] = 0.f;
+    float mg = -INFINITY, lg = 0.f;
+    {  // score of the new token against itself (every warp computes the same value)
+      float part = 0.f;
 #pragma unroll
-    for (int w = 1; w < WARPS; ++w)
-      if (cand_before(wbest[w], b)) b = wbest[w];
-    int slot, ev;
-    if (!full) {
-      slot = cnt;
-      ev = -1;
-      c.count[u] = cnt + 1;
-    } else if (b.slot == -2) {
-      slot = -1;
-      ev = t;
-    } else if (b.slot >= 0) {
-      slot = b.slot;
-      ev = b.pos;
-    } else {  // a full cache always has a candidate; record instead of corrupting
-      slot = -1;
-      ev = -1;
-      atomicCAS(c.status, 0, H2O_ERR_STATE);
+      for (int v = 0; v < VEC; ++v) part = fmaf(qf[v], ksf[v], part);
+#pragma unroll
+      for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+      s_self = c.scale * __shfl_sync(0xffffffffu, part, 0);
     }
-    if (slot >= 0) {
-      acc[slot] = (double)p[cnt];
-      pos[slot] = t;
+    for (int j = 0; j < ntile; ++j) {
+      const int s = j % stages;
+      if (!mbar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
+      if (j == 0) H2O_STAMP(2);
+      const T* kt = reinterpret_cast<const T*>(ring + (size_t)s * 2 * kTileBytes);
+      const T* vt = reinterpret_cast<const T*>(ring + (size_t)s * 2 * kTileBytes + kTileBytes);
+      const int rows = min(TILE_ROWS, nloc - j * TILE_ROWS);
+      float sc[C::PASSES], vf[C::PASSES][VEC];
+#pragma unroll
+      for (int ps = 0; ps < C::PASSES; ++ps) {  // independent dot products first
+        const int row = ps * RPC + warp * RPW + sub;
+        float part = 0.f;
+        if (row < rows) {
+          float kf[VEC];
+          Vec16<T>::load(kt + row * D + ch * VEC, kf);
+          Vec16<T>::load(vt + row * D + ch * VEC, vf[ps]);
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) part = fmaf(qf[v], kf[v], part);
+        } else {
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) vf[ps][v] = 0.f;
+        }
+#pragma unroll
+        for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+        sc[ps] = row < rows ? c.scale * part : -INFINITY;
+        if (ch == 0 && row < rows) p[j * TILE_ROWS + row] = sc[ps];  // raw score, finalised after the stream
+      }
+      float mnew = mg;
+#pragma unroll
+      for (int ps = 0; ps < C::PASSES; ++ps) mnew = fmaxf(mnew, sc[ps]);
+      if (mnew > -INFINITY) {  // at least one real row so far in this group
+        const float f = expf(mg - mnew);  // expf(-inf) = 0 for the group's first rows
+        lg *= f;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) o[v] *= f;
+#pragma unroll
+        for (int ps = 0; ps < C::PASSES; ++ps) {
+          const float e = expf(sc[ps] - mnew);  // 0 for rows past the end
+          lg += e;
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) o[v] = fmaf(e, vf[ps][v], o[v]);
+        }
+        mg = mnew;
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.empty[s])) : "memory");
     }
-    if (evicted_pos) evicted_pos[u] = ev;
-    c.tpos[u] = t + 1;
-    victim_sh = slot;
+    H2O_STAMP(3);
+    const int g = warp * RPW + sub;
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) sh.red[g][ch * VEC + v] = o[v];
+    if (ch == 0) {
+      sh.gm[g] = mg;
+      sh.gl[g] = lg;
+    }
+    consumer_sync();
+#ifdef H2O_EPI_REPS
+    for (int rep_ = 0; rep_ < H2O_EPI_REPS; ++rep_) {  // debug: run the epilogue again to time a warm pass
+    const bool last_rep_ = rep_ == H2O_EPI_REPS - 1;
+    if (!last_rep_) consumer_sync();
+#else
+    {
+    const bool last_rep_ = true;
+#endif
+    H2O_STAMP(8);
+
+    // ---- block statistics, computed by every warp alike (fixed order, same result) -------
+    const float m_i = lane < GROUPS ? sh.gm[lane] : -INFINITY;
+    float mc = warp_max(m_i);
+    if (rank == 0) mc = fmaxf(mc, s_self);
+    // weight of group `lane` relative to the block maximum (0 for empty groups and for an empty block)
+    const float w_i = (lane < GROUPS && m_i > -INFINITY) ? expf(m_i - mc) : 0.f;
+    float lc = warp_sum(lane < GROUPS ? sh.gl[lane] * w_i : 0.f);
+    const float w_self = rank == 0 ? expf(s_self - mc) : 0.f;
+    lc += w_self;
+    H2O_STAMP(9);
+    float part_o = 0.f;  // block partial output relative to mc
+#pragma unroll
+    for (int g2 = 0; g2 < GROUPS; ++g2) {
+      const float w = __shfl_sync(0xffffffffu, w_i, g2);
+      if (tid < D) part_o = fmaf(sh.red[g2][tid], w, part_o);
+    }
+    part_o = fmaf(w_self, vself, part_o);
+    if (split > 1) {
+      if (tid == 0) {
+        sh.m_c = mc;
+        sh.l_c = lc;
+      }
+      if (tid < D) sh.x_out[tid] = part_o;
+      cluster.sync();
+      const float mr = lane < split ? *cluster.map_shared_rank(&sh.m_c, lane) : -INFINITY;
+      const float lr = lane < split ? *cluster.map_shared_rank(&sh.l_c, lane) : 0.f;
+      m = warp_max(mr);
+      l = warp_sum(mr > -INFINITY ? lr * expf(mr - m) : 0.f);
+      if (rank == 0 && tid < D) {
+        part_o *= expf(mc - m);
+        for (int rk = 1; rk < split; ++rk) {
+          const float mrk = *cluster.map_shared_rank(&sh.m_c, rk);
+          if (mrk > -INFINITY) part_o = fmaf(cluster.map_shared_rank(sh.x_out, rk)[tid], expf(mrk - m), part_o);
+        }
+      }
+    } else {
+      m = mc;
+      l = lc;
+    }
+    H2O_STAMP(4);
+    if (rank == 0 && tid < D) {
+      const float res = part_o / l;  // (kept as a division: one per output element)
+      if constexpr (sizeof(T) == 4) reinterpret_cast<float*>(out)[(int64_t)u * D + tid] = res;
+      else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)u * D + tid] = __float2bfloat16_rn(res);
+    }
+
+    // ---- final probabilities, accumulation (Algorithm 2: o~_i = o~_{i-1} + o_i), victim search ----
+    if (nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
+    const bool full = cnt >= B;
+    const float inv_l = 1.0f / l;
+    const float p_self = expf(s_self - m) * inv_l;
+    Cand best = cand_none();
+#pragma unroll 2
+    for (int x = tid; x < nloc; x += kThreads) {
+      const float px = expf(p[x] - m) * inv_l;
+      const double a = acc_s[x] + (double)px;
+      acc_g[x] = a;
+      const int ps = pos_s[x];
+      if (full && ps <= t - r) {
+        const Cand cx = cand_make(a, ps, lo + x);
+        if (cand_before(cx, best)) best = cx;
+      }
+    }
+    if (rank == 0 && tid == 0 && full && r == 0) {  // without a recent window the new token competes too
+      const Cand cs = cand_make((double)p_self, t, -2);
+      if (cand_before(cs, best)) best = cs;
+    }
+    H2O_STAMP(10);
+    best = warp_argmin(best);
+    H2O_STAMP(11);
+    if (lane == 0) sh.wbest[warp] = best;
+    if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    consumer_sync();
+    H2O_STAMP(5);
+    if (warp == 0) {
+      Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+      H2O_STAMP(7);
+      if (split > 1) {
+        if (lane == 0) sh.x_cand = b;
+      }
+      if (split > 1) {
+        cluster.sync();
+        if (rank == 0) {
+          Cand o2 = lane < split ? *cluster.map_shared_rank(&sh.x_cand, lane) : cand_none();
+          b = warp_argmin(o2);
+        }
+      }
+      if (rank == 0 && last_rep_) {  // replace the victim in place (or append while the cache is filling)
+        int slot, ev;
+        if (!full) {
+          slot = cnt;
+          ev = -1;
+        } else if (b.slot == -2) {
+          slot = -1;
+          ev = t;
+        } else if (b.slot >= 0) {
+          slot = b.slot;
+          ev = b.pos;
+        } else {  // a full cache always has a candidate; record instead of corrupting
+          slot = -1;
+          ev = -1;
+          if (lane == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
+        }
+        if (lane == 0) {
+          if (!full) c.count[su] = cnt + 1;
+          if (slot >= 0) {
+            c.acc[mt.slot_off + slot] = (double)p_self;
+            c.pos[mt.slot_off + slot] = t;
+          }
+          if (evicted_pos) evicted_pos[u] = ev;
+          c.tpos[su] = t + 1;
+        }
+        if (slot >= 0) {
+          for (int i = lane; i < 2 * LPR; i += 32) {  // the new K/V row goes straight into the freed slot
+            const int c16 = i % LPR;
+            const uint4 val = *reinterpret_cast<const uint4*>((i < LPR ? ku : vu) + c16 * VEC);
+            T* base = reinterpret_cast<T*>(i < LPR ? c.K : c.V) + (mt.slot_off + slot) * D;
+            *reinterpret_cast<uint4*>(base + c16 * VEC) = val;
+          }
+        }
+      }
+    } else if (split > 1) {
+      cluster.sync();
+    }
+    }  // epilogue scope
   }
-  __syncthreads();
-  const int slot = victim_sh;
-  if (slot >= 0 && tid < 2 * LPR) {  // in-place replacement: the new K/V row goes into the freed slot
-    const int ch = tid % LPR;
-    const uint4 val = *reinterpret_cast<const uint4*>((tid < LPR ? ku : vu) + ch * VEC);
-    *reinterpret_cast<uint4*>((tid < LPR ? Kb : Vb) + (int64_t)slot * D + ch * VEC) = val;
-  }
+  if (split > 1) cluster.sync();  // nobody leaves while rank 0 still reads its peers' shared memory
+  H2O_STAMP(6);
 }
 
 template <typename T, int D>
-cudaError_t launch(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
-                   int32_t* evicted_pos, cudaStream_t stream) {
-  const size_t smem = sizeof(float) * (size_t)(max_B + 1);
-  decode_kernel<T, D><<<c.units, kDecodeThreads, smem, stream>>>(
-      c, static_cast<const T*>(q), static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
-      evicted_pos);
-  return cudaGetLastError();
+cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, const void* q, const void* k_new,
+                   const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  using C = Cfg<T, D>;
+  // ring depth: the whole chunk if it is short, otherwise enough to keep ~64 KB in flight per block
+  const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : kDefaultStages;
+  int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
+  stages = stages < 1 ? 1 : (stages > want ? want : stages);
+  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
+  static bool attr_done = false;  // one flag per template instance; setting it twice is harmless
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(c.units * split));
+  cfg.blockDim = dim3(kThreads + 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)split;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D>, c, static_cast<const T*>(q), static_cast<const T*>(k_new),
+                            static_cast<const T*>(v_new), static_cast<T*>(out), evicted_pos, split, chunk, stages);
 }
 
 }  // namespace
 
-cudaError_t launch_decode(const CacheView& c, int dtype, int max_B, const void* q, const void* k_new, const void* v_new,
-                          void* out, int32_t* evicted_pos, cudaStream_t stream) {
+#ifdef H2O_PHASE_TIMERS
+extern "C" int h2o_debug_phase_timers(unsigned long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_phase, sizeof(unsigned long long) * (size_t)n);
+}
+#endif
+
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, const void* q,
+                          const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  if (split < 1 || split > kMaxSplit) return cudaErrorInvalidValue;
   if (dtype == H2O_F32) {
-    if (c.head_dim == 64) return launch<float, 64>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
-    return launch<float, 128>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
+    if (c.head_dim == 64) return launch<float, 64>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
+    return launch<float, 128>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
   }
-  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
-  return launch<__nv_bfloat16, 128>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
+  if (c.head_dim == 64)
+    return launch<__nv_bfloat16, 64>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
+  return launch<__nv_bfloat16, 128>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace h2o

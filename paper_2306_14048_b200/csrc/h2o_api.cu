@@ -14,7 +14,9 @@
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kMaxSlotsPerUnit = 49152;  // scores of one unit must fit in shared memory
+constexpr int kMaxSlotsPerUnit = 65536;  // bounded by the decode kernel's shared-memory score rows
+constexpr int kMaxPromptLen = 49151;     // the ALU prefill keeps one score row in shared memory
+constexpr int kMaxChunk = 8192;          // slots per decode thread block
 constexpr int kMaxUnits = 65535;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -22,7 +24,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 size_t elem_size(int dtype) { return dtype == H2O_F32 ? 4 : 2; }
 
 struct Layout {
-  size_t K, V, acc, pos, count, tpos, status, slot_off, kbud, rwin, order, total;
+  size_t K, V, acc, pos, count, tpos, status, meta, total;
   int64_t total_slots;
   int max_B;
 };
@@ -49,7 +51,7 @@ Layout make_layout(const h2o_config_t* cfg) {
   int max_B = 0;
   for (int s = 0; s < cfg->batch; ++s) {
     const int B = cfg->heavy_budget[s] + cfg->recent_window[s];
-    slots += (int64_t)B * cfg->n_heads;
+    slots += (int64_t)((B + 3) & ~3) * cfg->n_heads;  // units start on a multiple of 4 slots (16-byte bulk copies)
     max_B = std::max(max_B, B);
   }
   const size_t units = (size_t)cfg->batch * cfg->n_heads;
@@ -67,10 +69,7 @@ Layout make_layout(const h2o_config_t* cfg) {
   L.count = take(units * sizeof(int32_t));
   L.tpos = take(units * sizeof(int32_t));
   L.status = take(sizeof(int32_t));
-  L.slot_off = take(units * sizeof(int64_t));
-  L.kbud = take(units * sizeof(int32_t));
-  L.rwin = take(units * sizeof(int32_t));
-  L.order = take(units * sizeof(int32_t));
+  L.meta = take(units * sizeof(h2o::UnitMeta));
   L.total = off;
   L.total_slots = slots;
   L.max_B = max_B;
@@ -105,6 +104,8 @@ enum class Phase { Empty, Prefilled, Decoding };
 struct h2o_cache {
   h2o_config_t cfg;
   std::vector<int32_t> heavy, recent, cu;
+  std::vector<h2o::UnitMeta> meta;  // launch order
+  int split, chunk, stages;
   Layout layout;
   h2o::CacheView view;
   Phase phase;
@@ -172,19 +173,26 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
   c->phase = Phase::Empty;
 
   const int units = cfg->batch * cfg->n_heads;
-  std::vector<int64_t> slot_off(units);
-  std::vector<int32_t> kbud(units), rwin(units), order(units);
+  std::vector<h2o::UnitMeta> meta(units);
   int64_t at = 0;
   for (int u = 0; u < units; ++u) {
     const int s = u / cfg->n_heads;
-    slot_off[u] = at;
-    kbud[u] = c->heavy[s];
-    rwin[u] = c->recent[s];
-    at += c->heavy[s] + c->recent[s];
+    meta[u] = h2o::UnitMeta{at, u, c->heavy[s], c->recent[s], 0};
+    at += (c->heavy[s] + c->recent[s] + 3) & ~3;
   }
-  std::iota(order.begin(), order.end(), 0);
-  std::stable_sort(order.begin(), order.end(),
-                   [&](int a, int b) { return kbud[a] + rwin[a] > kbud[b] + rwin[b]; });  // longest first
+  std::stable_sort(meta.begin(), meta.end(), [](const h2o::UnitMeta& a, const h2o::UnitMeta& b) {
+    return a.kbud + a.rwin > b.kbud + b.rwin;  // longest first
+  });
+  c->meta = meta;
+  // Thread blocks per unit.  One block per unit unless there are fewer units than SMs: sharing a
+  // unit costs three cluster barriers per step, which only pays when SMs would otherwise idle.
+  int split = 1;
+  while (split < 8 && (((int64_t)units * split < 148 && L.max_B / (2 * split) >= 64) ||
+                       (L.max_B + split - 1) / split > kMaxChunk))
+    split *= 2;
+  c->split = split;
+  c->stages = 0;
+  c->chunk = (((L.max_B + split - 1) / split) + 3) & ~3;
 
   char* ws = static_cast<char*>(dev_workspace);
   h2o::CacheView& v = c->view;
@@ -195,22 +203,16 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
   v.count = reinterpret_cast<int32_t*>(ws + L.count);
   v.tpos = reinterpret_cast<int32_t*>(ws + L.tpos);
   v.status = reinterpret_cast<int32_t*>(ws + L.status);
-  v.slot_off = reinterpret_cast<const int64_t*>(ws + L.slot_off);
-  v.kbud = reinterpret_cast<const int32_t*>(ws + L.kbud);
-  v.rwin = reinterpret_cast<const int32_t*>(ws + L.rwin);
-  v.order = reinterpret_cast<const int32_t*>(ws + L.order);
+  v.meta = reinterpret_cast<const h2o::UnitMeta*>(ws + L.meta);
   v.units = units;
   v.n_heads = cfg->n_heads;
   v.head_dim = cfg->head_dim;
   v.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
 
   bool ok = true;
-  ok = ok && cudaMemset(ws + L.acc, 0, L.slot_off - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
+  ok = ok && cudaMemset(ws + L.acc, 0, L.meta - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
   ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
-  ok = ok && cudaMemcpy(ws + L.slot_off, slot_off.data(), units * sizeof(int64_t), cudaMemcpyHostToDevice) == cudaSuccess;
-  ok = ok && cudaMemcpy(ws + L.kbud, kbud.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
-  ok = ok && cudaMemcpy(ws + L.rwin, rwin.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
-  ok = ok && cudaMemcpy(ws + L.order, order.data(), units * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(ws + L.meta, meta.data(), units * sizeof(h2o::UnitMeta), cudaMemcpyHostToDevice) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     delete c;
@@ -233,7 +235,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
     max_seqlen = std::max<int64_t>(max_seqlen, n);
   }
   const int64_t total = cu_seqlens[cfg.batch];
-  if (max_seqlen > kMaxSlotsPerUnit - 1) return H2O_ERR_UNSUPPORTED;  // limit of the shared-memory score row
+  if (max_seqlen > kMaxPromptLen) return H2O_ERR_UNSUPPORTED;  // limit of the shared-memory score row
   const ScratchLayout S = make_scratch_layout(&cfg, total);
   if (scratch_bytes < S.total || (reinterpret_cast<uintptr_t>(scratch) % kAlign) != 0) return H2O_ERR_WORKSPACE;
   for (const void* p : {q, k, v, (const void*)out})
@@ -273,8 +275,8 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
     if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
   DeviceGuard guard(cache->cfg.device);
   if (!guard.ok) return H2O_ERR_CUDA;
-  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->layout.max_B, q, k_new, v_new, out,
-                                           evicted_pos, static_cast<cudaStream_t>(stream));
+  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, q,
+                                           k_new, v_new, out, evicted_pos, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
@@ -363,13 +365,26 @@ int h2o_cache_reset(h2o_cache_t* cache, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Layout& L = cache->layout;
   char* ws = static_cast<char*>(cache->view.K) - L.K;
-  bool ok = cudaMemsetAsync(ws + L.acc, 0, L.slot_off - L.acc, st) == cudaSuccess;
+  bool ok = cudaMemsetAsync(ws + L.acc, 0, L.meta - L.acc, st) == cudaSuccess;
   ok = ok && cudaMemsetAsync(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t), st) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
   cache->phase = Phase::Empty;
+  return H2O_OK;
+}
+
+int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages) {
+  if (!cache || stages < 0 || stages > 8) return H2O_ERR_INVALID_ARG;
+  if (split != 0 && split != 1 && split != 2 && split != 4 && split != 8) return H2O_ERR_INVALID_ARG;
+  if (split != 0) {
+    const int chunk = (((cache->layout.max_B + split - 1) / split) + 3) & ~3;
+    if (chunk > kMaxChunk) return H2O_ERR_UNSUPPORTED;
+    cache->split = split;
+    cache->chunk = chunk;
+  }
+  cache->stages = stages;
   return H2O_OK;
 }
 
@@ -392,21 +407,22 @@ int h2o_cache_export(h2o_cache_t* cache, int32_t* pos, double* acc, int32_t* cou
   bool ok = cudaStreamSynchronize(st) == cudaSuccess;
   if (pos) ok = ok && cudaMemcpy(hpos.data(), v.pos, slots * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
   if (acc) ok = ok && cudaMemcpy(hacc.data(), v.acc, slots * sizeof(double), cudaMemcpyDeviceToHost) == cudaSuccess;
-  if (count) ok = ok && cudaMemcpy(count, v.count, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
-  if (t) ok = ok && cudaMemcpy(t, v.tpos, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+  std::vector<int32_t> hcount(count ? v.units : 0), ht(t ? v.units : 0);
+  if (count) ok = ok && cudaMemcpy(hcount.data(), v.count, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
+  if (t) ok = ok && cudaMemcpy(ht.data(), v.tpos, v.units * sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
-  size_t at = 0;
-  for (int u = 0; u < v.units; ++u) {
-    const int s = u / v.n_heads;
-    const int B = cache->heavy[s] + cache->recent[s];
+  for (int su = 0; su < v.units; ++su) {  // device tables are in launch order
+    const h2o::UnitMeta& mt = cache->meta[su];
+    const int u = mt.unit, B = mt.kbud + mt.rwin;
     for (int x = 0; x < pitch; ++x) {
-      if (pos) pos[(size_t)u * pitch + x] = x < B ? hpos[at + x] : -1;
-      if (acc) acc[(size_t)u * pitch + x] = x < B ? hacc[at + x] : 0.0;
+      if (pos) pos[(size_t)u * pitch + x] = x < B ? hpos[mt.slot_off + x] : -1;
+      if (acc) acc[(size_t)u * pitch + x] = x < B ? hacc[mt.slot_off + x] : 0.0;
     }
-    at += B;
+    if (count) count[u] = hcount[su];
+    if (t) t[u] = ht[su];
   }
   return H2O_OK;
 }

@@ -10,21 +10,28 @@
 
 namespace h2o {
 
+// Static description of one unit, stored in launch order (largest budget first).
+struct UnitMeta {
+  int64_t slot_off;  // first slot of the unit (a multiple of 4)
+  int32_t unit;      // sequence * n_heads + head
+  int32_t kbud;      // heavy budget k
+  int32_t rwin;      // recent window r
+  int32_t pad_;
+};
+
 // Device-side view of a cache.  All pointers live inside the caller's workspace.
+// `meta`, `count` and `tpos` are indexed by launch position, not by unit.
 struct CacheView {
-  void* K;                  // [total_slots][d] storage dtype
-  void* V;                  // [total_slots][d]
-  double* acc;              // [total_slots] accumulated attention score
-  int32_t* pos;             // [total_slots] token position held by the slot
-  int32_t* count;           // [units] occupied slots
-  int32_t* tpos;            // [units] position of the next token
-  int32_t* status;          // [1] first error recorded by a kernel
-  const int64_t* slot_off;  // [units] first slot of the unit
-  const int32_t* kbud;      // [units] heavy budget k
-  const int32_t* rwin;      // [units] recent window r
-  const int32_t* order;     // [units] launch order (largest budget first)
+  void* K;               // [total_slots][d] storage dtype
+  void* V;               // [total_slots][d]
+  double* acc;           // [total_slots] accumulated attention score
+  int32_t* pos;          // [total_slots] token position held by the slot
+  int32_t* count;        // [units] occupied slots
+  int32_t* tpos;         // [units] position of the next token
+  int32_t* status;       // [1] first error recorded by a kernel
+  const UnitMeta* meta;  // [units]
   int32_t units, n_heads, head_dim;
-  float scale;              // softmax scale c
+  float scale;           // softmax scale c
 };
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
@@ -38,8 +45,10 @@ struct PrefillScratch {
 };
 
 // Launchers (each returns the cudaError_t of its launch).
-cudaError_t launch_decode(const CacheView& c, int dtype, int max_B, const void* q, const void* k_new, const void* v_new,
-                          void* out, int32_t* evicted_pos, cudaStream_t stream);
+// `split` thread blocks (one cluster) share a unit, each owning `chunk` consecutive slots.
+// `stages` is the depth of the shared-memory ring (0 = default).
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, const void* q,
+                          const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream);
 cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int batch, int max_seqlen,
                                  const void* q, const void* k, const void* v, void* out, cudaStream_t stream);
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,

@@ -60,10 +60,12 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
   __shared__ int remaining_sh;
 
   const int tid = threadIdx.x;
-  const int u = c.order[blockIdx.x];
+  const int su = blockIdx.x;  // launch position
+  const UnitMeta mt = c.meta[su];
+  const int u = mt.unit;
   const int seq = u / c.n_heads, h = u % c.n_heads;
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
-  const int kb = c.kbud[u], r = c.rwin[u], B = kb + r;
+  const int kb = mt.kbud, r = mt.rwin, B = kb + r;
   const double* acc0 = s.acc0 + (int64_t)h * s.total_tokens + lo;
   const int m = n <= B ? n : B;  // entries kept
 
@@ -137,7 +139,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
   __syncthreads();
 
   // gather into the unit's slots
-  const int64_t s0 = c.slot_off[u];
+  const int64_t s0 = mt.slot_off;
   const int64_t stride = (int64_t)c.n_heads * D;
   const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
   T* Kb = reinterpret_cast<T*>(c.K) + s0 * D;
@@ -154,8 +156,8 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
     *reinterpret_cast<uint4*>(Vb + (int64_t)slot * D + ch * VEC) = *reinterpret_cast<const uint4*>(v + src);
   }
   if (tid == 0) {
-    c.count[u] = m;
-    c.tpos[u] = n;
+    c.count[su] = m;
+    c.tpos[su] = n;
   }
 }
 

@@ -74,6 +74,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     units = list(range(wl.units)) if units is None else sorted(set(int(u) for u in units))
     stats.units_checked = len(units)
     steps = wl.decode_steps if steps is None else steps
+    # the C ABI takes the softmax scale as a float: both sides get that same fp32 value
+    scale = float(np.float32(scale if scale > 0 else 1.0 / np.sqrt(float(d))))
     gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
     ora = h2o_oracle.OracleCache(wl.batch, H, d, wl.heavy, wl.recent, scale=scale)
     if prefill:

@@ -72,3 +72,26 @@ def test_peaky_softmax_stress(H2OCache):
     wl = _wl("peaky", 2, 4, 128, "bf16", [700, 450], 64, [40, 30], [40, 30], seed=21)
     st = run_parity(wl, H2OCache, scale=4.0 / np.sqrt(128.0), export_every=16)
     print(st)
+
+
+@pytest.mark.parametrize("dtype,d,heavy,recent", [
+    ("bf16", 128, [150, 30], [150, 40]),      # split over 4 thread blocks; the short sequence leaves blocks empty
+    ("bf16", 128, [600, 500], [500, 600]),    # split over 8
+    ("f32", 64, [100, 64], [100, 64]),
+])
+def test_units_split_over_a_cluster(H2OCache, dtype, d, heavy, recent):
+    """Few units with long budgets: one unit is shared by several thread blocks of a cluster."""
+    from parity_harness import run_parity
+
+    wl = _wl("cluster", 2, 2, d, dtype, [1500, 1300], 40, heavy, recent, seed=31)
+    st = run_parity(wl, H2OCache, export_every=8)
+    print(st)
+
+
+def test_cluster_split_fill_phase_from_empty(H2OCache):
+    """Token-by-token fill of a cache that is split over a cluster: most blocks start empty."""
+    from parity_harness import run_parity
+
+    wl = _wl("clusterfill", 1, 2, 128, "bf16", [1], 330, [150], [150], seed=32)
+    st = run_parity(wl, H2OCache, prefill=False, export_every=30)
+    print(st)
