@@ -174,6 +174,16 @@ int h2o_cache_status(h2o_cache_t* cache, void* stream);
  *          0 = default.  Results do not depend on either value beyond summation order.
  */
 int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages);
+/*
+ * Diagnostics for the prefill (no counterpart in the paper).
+ * h2o_cache_set_prefill_path: 0 = automatic (tensor-core kernels for bf16 with head_dim
+ *   128, fp32-FMA kernels otherwise), 1 = always the fp32-FMA kernels.
+ * h2o_prefill_scratch_layout: byte offset, inside the scratch buffer of
+ *   h2o_prefill_select, of the column sums acc0 (double, [n_heads][total_tokens]); valid
+ *   once the stream has finished the call.
+ */
+int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
+int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, size_t* acc0_offset);
 const char* h2o_strerror(int code);
 
 #ifdef __cplusplus

@@ -40,6 +40,8 @@ EXPORTED = (
     "h2o_cache_export",
     "h2o_cache_status",
     "h2o_cache_set_decode_shape",
+    "h2o_cache_set_prefill_path",
+    "h2o_prefill_scratch_layout",
     "h2o_strerror",
 )
 
@@ -91,6 +93,10 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_status.argtypes = [vp, vp]
     lib.h2o_cache_set_decode_shape.restype = c.c_int
     lib.h2o_cache_set_decode_shape.argtypes = [vp, c.c_int32, c.c_int32]
+    lib.h2o_cache_set_prefill_path.restype = c.c_int
+    lib.h2o_cache_set_prefill_path.argtypes = [vp, c.c_int32]
+    lib.h2o_prefill_scratch_layout.restype = c.c_int
+    lib.h2o_prefill_scratch_layout.argtypes = [cfgp, c.c_int64, c.POINTER(c.c_size_t)]
     lib.h2o_strerror.restype = c.c_char_p
     lib.h2o_strerror.argtypes = [c.c_int]
     return lib
@@ -220,6 +226,19 @@ class H2OCache:
 
     def set_decode_shape(self, split: int = 0, stages: int = 0):
         _check(lib.h2o_cache_set_decode_shape(self._h, int(split), int(stages)), "h2o_cache_set_decode_shape")
+
+    def set_prefill_path(self, path: int):
+        _check(lib.h2o_cache_set_prefill_path(self._h, int(path)), "h2o_cache_set_prefill_path")
+
+    def prefill_column_sums(self, total_tokens: int):
+        """acc0 of the last prefill_select as a [n_heads, total_tokens] float64 tensor (a view of the scratch)."""
+        acc_off = ctypes.c_size_t()
+        _check(lib.h2o_prefill_scratch_layout(ctypes.byref(self.cfg), int(total_tokens), ctypes.byref(acc_off)),
+               "h2o_prefill_scratch_layout")
+        base = (self._scratch.data_ptr() + 255) // 256 * 256 - self._scratch.data_ptr()
+        n = self.n_heads * int(total_tokens)
+        raw = self._scratch[base + acc_off.value: base + acc_off.value + 8 * n]
+        return raw.view(torch.float64).view(self.n_heads, int(total_tokens))
 
     def status(self, stream=None) -> int:
         return int(lib.h2o_cache_status(self._h, _stream_ptr(stream)))

@@ -77,7 +77,7 @@ Layout make_layout(const h2o_config_t* cfg) {
 }
 
 struct ScratchLayout {
-  size_t rowmax, rowsum, acc0, cu, total;
+  size_t rowstat, acc0, cu, total;
 };
 
 ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens) {
@@ -89,8 +89,7 @@ ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens)
     off = align_up(off + bytes);
     return at;
   };
-  S.rowmax = take(cells * sizeof(float));
-  S.rowsum = take(cells * sizeof(float));
+  S.rowstat = take(cells * 2 * sizeof(float));  // row maximum and row sum (planar or interleaved)
   S.acc0 = take(cells * sizeof(double));
   S.cu = take(((size_t)cfg->batch + 1) * sizeof(int32_t));
   S.total = off;
@@ -106,6 +105,7 @@ struct h2o_cache {
   std::vector<int32_t> heavy, recent, cu;
   std::vector<h2o::UnitMeta> meta;  // launch order
   int split, chunk, stages;
+  int prefill_path;  // 0 = automatic, 1 = force the ALU kernels
   Layout layout;
   h2o::CacheView view;
   Phase phase;
@@ -192,6 +192,7 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
     split *= 2;
   c->split = split;
   c->stages = 0;
+  c->prefill_path = 0;
   c->chunk = (((L.max_B + split - 1) / split) + 3) & ~3;
 
   char* ws = static_cast<char*>(dev_workspace);
@@ -247,8 +248,9 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* sc = static_cast<char*>(scratch);
   h2o::PrefillScratch ps;
-  ps.rowmax = reinterpret_cast<float*>(sc + S.rowmax);
-  ps.rowsum = reinterpret_cast<float*>(sc + S.rowsum);
+  ps.rowmax = reinterpret_cast<float*>(sc + S.rowstat);
+  ps.rowsum = ps.rowmax + (size_t)total * cfg.n_heads;
+  ps.rowstat = reinterpret_cast<float2*>(sc + S.rowstat);
   ps.acc0 = reinterpret_cast<double*>(sc + S.acc0);
   ps.cu = reinterpret_cast<int32_t*>(sc + S.cu);
   ps.total_tokens = total;
@@ -258,7 +260,15 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
-  cudaError_t e = h2o::launch_prefill_naive(cache->view, ps, cfg.dtype, cfg.batch, max_seqlen, q, k, v, out, st);
+  // bf16 / head_dim 128 runs on the tensor cores; every other combination on the fp32 FMA pipe
+  const bool tc = cache->prefill_path != 1 && h2o::prefill_tc_supported(cfg.dtype, cfg.head_dim);
+  cudaError_t e = cudaSuccess;
+  if (tc) {
+    e = h2o::launch_fwd_tc(cache->view, ps, max_seqlen, q, k, v, out, st);
+    if (e == cudaSuccess) e = h2o::launch_colsum_tc(cache->view, ps, max_seqlen, q, k, st);
+  } else {
+    e = h2o::launch_prefill_naive(cache->view, ps, cfg.dtype, max_seqlen, q, k, v, out, true, true, st);
+  }
   if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, cfg.dtype, cache->layout.max_B, k, v, st);
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -385,6 +395,19 @@ int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages
     cache->chunk = chunk;
   }
   cache->stages = stages;
+  return H2O_OK;
+}
+
+int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path) {
+  if (!cache || (path != 0 && path != 1)) return H2O_ERR_INVALID_ARG;
+  cache->prefill_path = path;
+  return H2O_OK;
+}
+
+int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, size_t* acc0_offset) {
+  if (check_config(cfg) != H2O_OK || total_tokens < 1 || total_tokens > INT32_MAX) return H2O_ERR_INVALID_ARG;
+  const ScratchLayout S = make_scratch_layout(cfg, total_tokens);
+  if (acc0_offset) *acc0_offset = S.acc0;
   return H2O_OK;
 }
 

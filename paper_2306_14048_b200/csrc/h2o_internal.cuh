@@ -39,6 +39,7 @@ struct CacheView {
 struct PrefillScratch {
   float* rowmax;   // m_i
   float* rowsum;   // l_i
+  float2* rowstat; // tensor-core path: {reference maximum (log2 domain), 1 / row sum}; aliases rowmax/rowsum
   double* acc0;    // column sums
   int32_t* cu;     // [batch + 1] device copy of cu_seqlens
   int64_t total_tokens;
@@ -49,8 +50,15 @@ struct PrefillScratch {
 // `stages` is the depth of the shared-memory ring (0 = default).
 cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, const void* q,
                           const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream);
-cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int batch, int max_seqlen,
-                                 const void* q, const void* k, const void* v, void* out, cudaStream_t stream);
+// ALU path; `rows` = attention rows + row statistics, `colsum` = column sums.
+cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int max_seqlen, const void* q,
+                                 const void* k, const void* v, void* out, bool rows, bool colsum, cudaStream_t stream);
+// Tensor-core path (bf16, head_dim 128 only).
+bool prefill_tc_supported(int dtype, int head_dim);
+cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
+                          const void* v, void* out, cudaStream_t stream);
+cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
+                             cudaStream_t stream);
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
                                  const void* v, cudaStream_t stream);
 

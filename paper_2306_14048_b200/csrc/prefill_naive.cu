@@ -86,34 +86,39 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
 
 template <typename T, int D>
 cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
-                   const void* v, void* out, cudaStream_t stream) {
-  const size_t smem = sizeof(float) * (size_t)(max_seqlen + 1);
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                   const void* v, void* out, bool rows, bool colsum, cudaStream_t stream) {
+  if (rows) {
+    const size_t smem = sizeof(float) * (size_t)(max_seqlen + 1);
+    if (smem > 48 * 1024) {
+      cudaError_t e =
+          cudaFuncSetAttribute(prefill_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    dim3 grid_rows((unsigned)max_seqlen, (unsigned)c.units);
+    prefill_rows_kernel<T, D><<<grid_rows, kRowThreads, smem, stream>>>(
+        c, s, static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(out));
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  dim3 grid_rows((unsigned)max_seqlen, (unsigned)c.units);
-  prefill_rows_kernel<T, D><<<grid_rows, kRowThreads, smem, stream>>>(
-      c, s, static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(out));
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  dim3 grid_cols((unsigned)((max_seqlen + kColThreads - 1) / kColThreads), (unsigned)c.units);
-  prefill_colsum_kernel<T, D><<<grid_cols, kColThreads, 0, stream>>>(c, s, static_cast<const T*>(q),
-                                                                    static_cast<const T*>(k));
-  return cudaGetLastError();
+  if (colsum) {
+    dim3 grid_cols((unsigned)((max_seqlen + kColThreads - 1) / kColThreads), (unsigned)c.units);
+    prefill_colsum_kernel<T, D><<<grid_cols, kColThreads, 0, stream>>>(c, s, static_cast<const T*>(q),
+                                                                      static_cast<const T*>(k));
+    return cudaGetLastError();
+  }
+  return cudaSuccess;
 }
 
 }  // namespace
 
-cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int batch, int max_seqlen,
-                                 const void* q, const void* k, const void* v, void* out, cudaStream_t stream) {
-  (void)batch;
+cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int max_seqlen, const void* q,
+                                 const void* k, const void* v, void* out, bool rows, bool colsum, cudaStream_t stream) {
   if (dtype == H2O_F32) {
-    if (c.head_dim == 64) return launch<float, 64>(c, s, max_seqlen, q, k, v, out, stream);
-    return launch<float, 128>(c, s, max_seqlen, q, k, v, out, stream);
+    if (c.head_dim == 64) return launch<float, 64>(c, s, max_seqlen, q, k, v, out, rows, colsum, stream);
+    return launch<float, 128>(c, s, max_seqlen, q, k, v, out, rows, colsum, stream);
   }
-  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, s, max_seqlen, q, k, v, out, stream);
-  return launch<__nv_bfloat16, 128>(c, s, max_seqlen, q, k, v, out, stream);
+  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, s, max_seqlen, q, k, v, out, rows, colsum, stream);
+  return launch<__nv_bfloat16, 128>(c, s, max_seqlen, q, k, v, out, rows, colsum, stream);
 }
 
 }  // namespace h2o

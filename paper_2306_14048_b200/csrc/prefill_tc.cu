@@ -1,0 +1,545 @@
+// Prompt attention on the tensor cores (bf16, head_dim 128): tcgen05.mma with TMEM
+// accumulators, operands staged in shared memory by TMA, warp-specialised roles.
+//
+// Column sums (this file, first kernel).  acc0[j] = sum_{i >= j} exp(c q_i.k_j - lse_i) needs the
+// final row normalisers, so scores are recomputed after the forward pass.  The kernel is
+// K-stationary and computes the TRANSPOSED tile S^T = K_j Q_i^T: a TMEM lane (= one thread of the
+// epilogue) then owns one key column j and sums over queries in registers — no atomics, fixed
+// order, reproducible.  A thread block takes key block j and its mirror nb-1-j, so every block
+// does the same number of tiles of the causal triangle.
+//
+// Paper: accumulated attention score of Algorithm 2 evaluated over all prompt rows (the prefill
+// branch of the Appendix A pseudocode).
+#include <cstring>
+
+#include "h2o_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace h2o {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kD = 128;           // head_dim handled here
+constexpr int kTile = 128;        // rows of a Q / K tile
+constexpr int kBoxBytes = kTile * 128;   // one TMA box: 128 rows x 64 bf16
+constexpr int kTileBytes = 2 * kBoxBytes;  // two boxes cover head_dim 128
+constexpr double kLog2eD = 1.4426950408889634074;
+
+// softmax scale times log2(e) as an unevaluated sum hi + lo of two floats, so that the product
+// with a raw score carries no rounding error of the constant
+struct Scale2 {
+  float hi, lo;
+};
+
+// ---- abortable waits: the first role that times out raises a flag every other wait observes ----
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 1023u) == 1023u && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Column sums
+// ---------------------------------------------------------------------------------------------
+constexpr int kCsThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kCsQStages = 2;
+constexpr int kCsTmemCols = 256;  // two accumulator buffers of 128 columns
+
+struct CsShared {
+  uint64_t k_full, k_empty;
+  uint64_t q_full[kCsQStages], q_empty[kCsQStages];
+  uint64_t acc_full[2], acc_empty[2];
+  uint64_t nl_full[2];  // the 128 epilogue threads have staged the tile's row statistics
+  uint32_t tmem_base;
+  int abort_flag;
+  float2 rstat[2][kTile];  // per query of the tile: {minus reference maximum (log2 domain), 1 / row sum}
+};
+
+__global__ void __launch_bounds__(kCsThreads)
+colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 PrefillScratch s, int n_heads, Scale2 scale2, int32_t* status) {
+  extern __shared__ unsigned char dyn_raw[];
+  __shared__ CsShared sh;
+  unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
+  unsigned char* k_tile = dyn;                       // [2 boxes][128 rows][128 B]
+  unsigned char* q_ring = dyn + kTileBytes;          // [stages][2 boxes][128 rows][128 B]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u = blockIdx.y;
+  const int seq = u / n_heads, h = u % n_heads;
+  const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
+  const int nb = (n + kTile - 1) / kTile;
+  const int pi = blockIdx.x;
+  if (pi >= (nb + 1) / 2) return;  // whole block leaves before any barrier or TMEM exists
+  const int jb0 = pi, jb1 = nb - 1 - pi;
+  const int ncb = jb1 > jb0 ? 2 : 1;
+  // tiles of column block jb: row blocks jb .. nb-1
+  const int t0 = nb - jb0;                        // tiles of the first column block
+  const int total = t0 + (ncb == 2 ? nb - jb1 : 0);
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.k_full, 1);
+    mbar_init(&sh.k_empty, 1);
+    for (int i = 0; i < kCsQStages; ++i) {
+      mbar_init(&sh.q_full[i], 1);
+      mbar_init(&sh.q_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh.acc_full[i], 1);
+      mbar_init(&sh.acc_empty[i], 4);  // one arrival per epilogue warp
+      mbar_init(&sh.nl_full[i], 128);
+    }
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, kCsTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      for (int t = 0; t < total; ++t) {
+        const int cb = t < t0 ? 0 : 1;
+        const int jb = cb == 0 ? jb0 : jb1;
+        const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
+        if (t == 0 || t == t0) {
+          if (cb == 1 && !wait_or_abort(&sh.k_empty, 0, abort_flag)) break;
+          mbar_expect_tx(&sh.k_full, kTileBytes);
+          tma_load_3d(k_tile, &map_k, 0, h, lo + jb * kTile, &sh.k_full);
+          tma_load_3d(k_tile + kBoxBytes, &map_k, 64, h, lo + jb * kTile, &sh.k_full);
+        }
+        const int st = t % kCsQStages;
+        if (!wait_or_abort(&sh.q_empty[st], ((t / kCsQStages) & 1) ^ 1, abort_flag)) break;
+        unsigned char* dst = q_ring + st * kTileBytes;
+        mbar_expect_tx(&sh.q_full[st], kTileBytes);
+        tma_load_3d(dst, &map_q, 0, h, lo + ib * kTile, &sh.q_full[st]);
+        tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + ib * kTile, &sh.q_full[st]);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_f16(kTile, kTile, kFmtBF16, kFmtBF16, false, false);
+      for (int t = 0; t < total; ++t) {
+        const int cb = t < t0 ? 0 : 1;
+        if (t == 0 || t == t0) {
+          if (!wait_or_abort(&sh.k_full, cb, abort_flag)) break;
+        }
+        const int st = t % kCsQStages, b = t & 1;
+        if (!wait_or_abort(&sh.q_full[st], (t / kCsQStages) & 1, abort_flag)) break;
+        if (!wait_or_abort(&sh.acc_empty[b], ((t >> 1) & 1) ^ 1, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t a0 = smem_u32(k_tile), b0 = smem_u32(q_ring + st * kTileBytes);
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t off = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+          mma_ss(tmem + (uint32_t)b * kTile, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
+                 idesc, ks > 0);
+        }
+        mma_commit(&sh.q_empty[st]);   // the Q stage may be refilled once these MMAs have read it
+        mma_commit(&sh.acc_full[b]);   // and the accumulator is ready for the epilogue
+        if (t == t0 - 1 && ncb == 2) mma_commit(&sh.k_empty);
+      }
+    }
+  } else {
+    // ---------------- epilogue: exp and in-thread column sums ----------------
+    const int e = threadIdx.x - 64;          // 0..127
+    const int quarter = warp & 3;            // TMEM lane quarter this warp may access
+    const int row = quarter * 32 + lane;     // key row inside the tile = TMEM lane
+    const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
+    double total_sum = 0.0;
+    auto fetch_nlse = [&](int t) -> float2 {
+      const int ib = t < t0 ? jb0 + t : jb1 + (t - t0);
+      const int qi = ib * kTile + e;
+      if (qi >= n) return make_float2(-INFINITY, 0.f);  // rows past the end: exp2(-inf) * 0 = 0
+      const float2 v2 = rowstat[qi];
+      return make_float2(-v2.x, v2.y);
+    };
+    float2 nl_next = fetch_nlse(0);
+    bool ok = true;
+    for (int t = 0; t < total && ok; ++t) {
+      const int cb = t < t0 ? 0 : 1;
+      const int jb = cb == 0 ? jb0 : jb1;
+      const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
+      const int b = t & 1;
+      sh.rstat[b][e] = nl_next;
+      if (t + 1 < total) nl_next = fetch_nlse(t + 1);
+      mbar_arrive(&sh.nl_full[b]);
+      ok = wait_or_abort(&sh.nl_full[b], (t >> 1) & 1, abort_flag) && wait_or_abort(&sh.acc_full[b], (t >> 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
+      if (!ok) break;
+      tc_fence_after();
+      const bool diag = ib == jb;
+      float tile_sum = 0.f;
+#pragma unroll
+      for (int cc = 0; cc < kTile / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(tmem + (uint32_t)b * kTile + (uint32_t)cc * 32u + ((uint32_t)(quarter * 32) << 16), r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c2 = 0; c2 < 32; ++c2) {
+          const int ql = cc * 32 + c2;  // query inside the tile
+          const float2 st2 = sh.rstat[b][ql];
+          const float sv = __uint_as_float(r[c2]);
+          const float pval = ex2(fmaf(sv, scale2.hi, fmaf(sv, scale2.lo, st2.x))) * st2.y;
+          tile_sum += (diag && ql < row) ? 0.f : pval;  // causal: query >= key
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
+      total_sum += (double)tile_sum;
+      if (t == t0 - 1 || t == total - 1) {  // last tile of this key block
+        const int key = jb * kTile + row;
+        if (key < n) s.acc0[(int64_t)h * s.total_tokens + lo + key] = total_sum;
+        total_sum = 0.0;
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(status, 0, H2O_ERR_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kCsTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward: out = softmax(c Q K^T) V over the causal triangle, plus the row log-sum-exp
+// ---------------------------------------------------------------------------------------------
+// One thread block per (unit, block of 128 queries); key tiles of 64.  Per key tile:
+//   MMA warp     : S = Q K_j^T            (M 128, N 64, K 128; accumulator in TMEM)
+//   softmax warps: one thread per query row reads its S row from TMEM, updates the running
+//                  maximum lazily (the reference maximum only moves when it would grow by more
+//                  than 8 in the log2 domain, so the O rows in TMEM are rescaled rarely),
+//                  writes P = exp2(S - m) as bf16 into a 128B-swizzled shared-memory tile
+//   MMA warp     : O += P V_j             (M 128, N 128, K 64; V is the MN-major operand)
+//                  (P is split into a bf16 hi and a bf16 lo part, multiplied one after the other,
+//                  so that the output does not carry the 2^-9 rounding of a single bf16 P)
+// Two blocks fit on an SM (96 KB of shared memory, 256 TMEM columns each); one block's softmax
+// overlaps the other's matrix instructions.
+constexpr int kFwThreads = 192;
+constexpr int kFwKeys = 64;                       // keys per tile
+constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
+constexpr int kFwKvSlots = 2;                     // slot 0 holds K tiles, slot 1 holds V tiles
+constexpr int kFwTmemCols = 256;                  // O: columns 0..127, S: columns 128..191
+constexpr float kRescaleThreshold = 8.0f;
+
+struct FwShared {
+  uint64_t q_full;
+  uint64_t kv_full[kFwKvSlots], kv_empty[kFwKvSlots];
+  uint64_t s_full, p_full, o_done;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <typename OutT>
+__global__ void __launch_bounds__(kFwThreads)
+fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+              const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, Scale2 scale2,
+              OutT* __restrict__ out, int32_t* status) {
+  extern __shared__ unsigned char dyn_raw[];
+  __shared__ FwShared sh;
+  unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
+  unsigned char* q_tile = dyn;                                   // 32 KB
+  unsigned char* kv_ring = dyn + kTileBytes;                     // 3 x 16 KB
+  unsigned char* p_tile = kv_ring + kFwKvSlots * kFwKvSlotBytes;  // 2 x 16 KB: hi and lo parts, [128 rows][64 bf16], swizzled
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u = blockIdx.y;
+  const int seq = u / n_heads, h = u % n_heads;
+  const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
+  const int nb = (n + kTile - 1) / kTile;
+  if ((int)blockIdx.x >= nb) return;
+  const int ib = nb - 1 - (int)blockIdx.x;  // long row blocks first
+  const int kmax = min(n, (ib + 1) * kTile);               // keys 0 .. kmax-1 are visible to this block
+  const int nt = (kmax + kFwKeys - 1) / kFwKeys;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.q_full, 1);
+    for (int i = 0; i < kFwKvSlots; ++i) {
+      mbar_init(&sh.kv_full[i], 1);
+      mbar_init(&sh.kv_empty[i], 1);
+    }
+    mbar_init(&sh.s_full, 1);
+    mbar_init(&sh.p_full, 4);
+    mbar_init(&sh.o_done, 1);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, kFwTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  const uint32_t tmem_o = tmem, tmem_s = tmem + 128u;
+  volatile int* abort_flag = &sh.abort_flag;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: Q once, then K_0, V_0, K_1, V_1, ... through three slots ----
+    if (lane == 0) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      prefetch_tensormap(&map_v);
+      mbar_expect_tx(&sh.q_full, kTileBytes);
+      tma_load_3d(q_tile, &map_q, 0, h, lo + ib * kTile, &sh.q_full);
+      tma_load_3d(q_tile + kBoxBytes, &map_q, 64, h, lo + ib * kTile, &sh.q_full);
+      for (int r = 0; r < 2 * nt; ++r) {
+        const int slot = r % kFwKvSlots;
+        if (!wait_or_abort(&sh.kv_empty[slot], ((r / kFwKvSlots) & 1) ^ 1, abort_flag)) break;
+        const CUtensorMap* map = (r & 1) ? &map_v : &map_k;
+        unsigned char* dst = kv_ring + slot * kFwKvSlotBytes;
+        const int row0 = lo + (r >> 1) * kFwKeys;
+        mbar_expect_tx(&sh.kv_full[slot], kFwKvSlotBytes);
+        tma_load_3d(dst, map, 0, h, row0, &sh.kv_full[slot]);
+        tma_load_3d(dst + kFwKvSlotBytes / 2, map, 64, h, row0, &sh.kv_full[slot]);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
+      // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
+      // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
+      constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
+      bool ok = wait_or_abort(&sh.q_full, 0, abort_flag);
+      const uint32_t q0 = smem_u32(q_tile), p0 = smem_u32(p_tile);
+      for (int j = 0; j < nt && ok; ++j) {
+        const int rk = 2 * j, rv = 2 * j + 1;
+        const int sk = rk % kFwKvSlots, sv = rv % kFwKvSlots;
+        ok = wait_or_abort(&sh.kv_full[sk], (rk / kFwKvSlots) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t k0 = smem_u32(kv_ring + sk * kFwKvSlotBytes);
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+          const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
+          mma_ss(tmem_s, smem_desc_sw128(q0 + qoff, 16, 1024), smem_desc_sw128(k0 + koff, 16, 1024), idesc_s, ks > 0);
+        }
+        mma_commit(&sh.kv_empty[sk]);
+        mma_commit(&sh.s_full);
+        ok = wait_or_abort(&sh.p_full, j & 1, abort_flag) && wait_or_abort(&sh.kv_full[sv], (rv / kFwKvSlots) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t v0 = smem_u32(kv_ring + sv * kFwKvSlotBytes);
+#pragma unroll
+        for (int ks = 0; ks < 2 * (kFwKeys / 16); ++ks) {  // hi part, then lo part, against the same V tile
+          const uint32_t part = (uint32_t)(ks >> 2), kk = (uint32_t)(ks & 3);
+          mma_ss(tmem_o, smem_desc_sw128(p0 + part * (kTile * 128) + kk * 32u, 16, 1024),
+                 smem_desc_sw128(v0 + kk * 2048u, kFwKvSlotBytes / 2, 1024), idesc_o, j > 0 || ks > 0);
+        }
+        mma_commit(&sh.kv_empty[sv]);
+      }
+      mma_commit(&sh.o_done);
+    }
+  } else {
+    // ---------------- softmax: one thread per query row ----------------
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int qi = ib * kTile + row;  // query position inside the sequence
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nt && ok; ++j) {
+      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full, j & 1, abort_flag));  // collectives below
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t r0[32], r1[32];
+      tmem_ld32(tmem_s + lane_addr, r0);
+      tmem_ld32(tmem_s + lane_addr + 32u, r1);
+      tmem_wait_ld();
+      const int key0 = j * kFwKeys;
+      const bool masked_tile = key0 + kFwKeys - 1 > ib * kTile;  // tile reaches past this block's first query
+      float sc[kFwKeys];
+      float m_tile = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < kFwKeys; ++c2) {
+        const float sv = __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]);
+        float x = fmaf(sv, scale2.hi, sv * scale2.lo);
+        if (masked_tile && key0 + c2 > qi) x = -INFINITY;  // causal: key <= query
+        sc[c2] = x;
+        m_tile = fmaxf(m_tile, x);
+      }
+      const bool need = m_tile > m_used + kRescaleThreshold;
+      if (j == 0) {
+        m_used = m_tile;  // key 0 is visible to every row, so this is finite
+      } else if (__any_sync(0xffffffffu, need)) {
+        // rescale this warp's O rows (the previous P V product has completed: s_full follows it)
+        const float m_new = need ? m_tile : m_used;
+        const float alpha = ex2(m_used - m_new);
+        l *= alpha;
+        m_used = m_new;
+#pragma unroll
+        for (int cc = 0; cc < kD / 32; ++cc) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c2 = 0; c2 < 32; ++c2) o[c2] = __float_as_uint(__uint_as_float(o[c2]) * alpha);
+          tmem_st32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
+        }
+        tmem_wait_st();
+      }
+      // probabilities relative to the reference maximum; bf16 copy for the P V product
+      unsigned char* prow = p_tile + row * 128;
+#pragma unroll
+      for (int c16 = 0; c16 < 8; ++c16) {
+        float pv[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          pv[e] = ex2(sc[c16 * 8 + e] - m_used);
+          l += pv[e];
+        }
+        // P = hi + lo with both parts bf16: the product with V then carries ~16 significant bits
+        uint4 w, wl;
+        uint32_t* wp = &w.x;
+        uint32_t* wlp = &wl.x;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pv[2 * e], pv[2 * e + 1]);
+          const float2 hf = __bfloat1622float2(hi2);
+          wp[e] = *reinterpret_cast<const uint32_t*>(&hi2);
+          wlp[e] = Vec16<__nv_bfloat16>::pack2(pv[2 * e] - hf.x, pv[2 * e + 1] - hf.y);
+        }
+        *reinterpret_cast<uint4*>(prow + ((c16 ^ (row & 7)) << 4)) = w;
+        *reinterpret_cast<uint4*>(prow + kTile * 128 + ((c16 ^ (row & 7)) << 4)) = wl;
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.p_full);
+    }
+    if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.o_done, 0, abort_flag));
+    if (ok) {
+      tc_fence_after();
+      const float inv_l = 1.0f / l;
+      OutT* orow = out + ((int64_t)(lo + qi) * n_heads + h) * kD;
+#pragma unroll
+      for (int cc = 0; cc < kD / 32; ++cc) {
+        uint32_t o[32];
+        tmem_ld32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
+        tmem_wait_ld();
+        if (qi < n) {
+#pragma unroll
+          for (int c8 = 0; c8 < 4; ++c8) {
+            float f[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[c8 * 8 + e]) * inv_l;
+            Vec16<__nv_bfloat16>::store(orow + cc * 32 + c8 * 8, f);
+          }
+        }
+      }
+      if (qi < n) s.rowstat[(int64_t)h * s.total_tokens + lo + qi] = make_float2(m_used, inv_l);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(status, 0, H2O_ERR_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kFwTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor maps
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [total_tokens, n_heads, 128] bf16, box = rows x 1 head x 64 elements (128 bytes), 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_heads, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)n_heads, (cuuint64_t)total_tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)n_heads * kD * 2};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+Scale2 make_scale2(float c) {
+  const double x = (double)c * kLog2eD;
+  Scale2 r;
+  r.hi = (float)x;
+  r.lo = (float)(x - (double)r.hi);
+  return r;
+}
+
+}  // namespace
+
+cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
+                          const void* v, void* out, cudaStream_t stream) {
+  CUtensorMap map_q, map_k, map_v;
+  if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
+      !make_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
+    return cudaErrorInvalidValue;
+  const int smem = kTileBytes + kFwKvSlots * kFwKvSlotBytes + 2 * kTile * 128 + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int nb = (max_seqlen + kTile - 1) / kTile;
+  dim3 grid((unsigned)nb, (unsigned)c.units);
+  fwd_tc_kernel<__nv_bfloat16><<<grid, kFwThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
+                                                                  static_cast<__nv_bfloat16*>(out), c.status);
+  return cudaGetLastError();
+}
+
+bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 && head_dim == kD && encode_fn() != nullptr; }
+
+cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
+                             cudaStream_t stream) {
+  CUtensorMap map_q, map_k;
+  if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
+    return cudaErrorInvalidValue;
+  const int smem = kTileBytes * (1 + kCsQStages) + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int nb = (max_seqlen + kTile - 1) / kTile;
+  dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
+  colsum_tc_kernel<<<grid, kCsThreads, smem, stream>>>(map_q, map_k, s, c.n_heads, make_scale2(c.scale), c.status);
+  return cudaGetLastError();
+}
+
+}  // namespace h2o

@@ -53,22 +53,37 @@ def _rel(a, b):
 
 def compare_state(gpu_cache, ora, units, dtype, stats: ParityStats, where: str):
     pos, acc, count, t = gpu_cache.export()
-    for u in units:
-        opos, oacc = ora.export(u)
+    for x, u in enumerate(units):  # oracle unit x mirrors GPU unit u
+        opos, oacc = ora.export(x)
         m = int(count[u])
         assert m == len(opos), "%s unit %d: count %d vs oracle %d" % (where, u, m, len(opos))
-        assert int(t[u]) == int(ora.t[u]), "%s unit %d: t" % (where, u)
+        assert int(t[u]) == int(ora.t[x]), "%s unit %d: t" % (where, u)
         order = np.argsort(pos[u, :m], kind="stable")
         gpos = pos[u, :m][order]
         assert np.array_equal(gpos, opos), "%s unit %d: kept positions differ" % (where, u)
-        assert np.all(pos[u, m:] == -1) or True
         stats.max_acc_err = max(stats.max_acc_err, assert_close(acc[u, :m][order], oacc, dtype, "%s unit %d acc" % (where, u)))
+
+
+def _gather_units(x, cu, units, H):
+    """Rows of the sampled units, packed as [sum n_u, 1, d] float32 on the host, plus their cu_seqlens."""
+    parts, lens = [], []
+    for u in units:
+        s, h = divmod(u, H)
+        parts.append(x[int(cu[s]):int(cu[s + 1]), h])
+        lens.append(int(cu[s + 1] - cu[s]))
+    packed = torch.cat(parts, dim=0).float().cpu().numpy()[:, None, :]
+    return np.ascontiguousarray(packed), np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
 
 
 def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
-               device: str = "cuda") -> ParityStats:
-    """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes."""
+               device: str = "cuda", prefill_path: int = 0) -> ParityStats:
+    """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
+
+    The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
+    (all of them by default) as a batch of single-head sequences, which is exact because units never
+    interact.
+    """
     stats = ParityStats()
     H, d = wl.n_heads, wl.head_dim
     units = list(range(wl.units)) if units is None else sorted(set(int(u) for u in units))
@@ -77,54 +92,61 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     # the C ABI takes the softmax scale as a float: both sides get that same fp32 value
     scale = float(np.float32(scale if scale > 0 else 1.0 / np.sqrt(float(d))))
     gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
-    ora = h2o_oracle.OracleCache(wl.batch, H, d, wl.heavy, wl.recent, scale=scale)
+    gpu.set_prefill_path(prefill_path)
+    ora = h2o_oracle.OracleCache(len(units), 1, d, [wl.heavy[u // H] for u in units], [wl.recent[u // H] for u in units],
+                                 scale=scale)
+    uidx = torch.as_tensor(units, dtype=torch.long, device=device)
     if prefill:
         q, k, v, cu = make_prompt_inputs(wl, layer=layer, device=device)
         out = torch.empty_like(q)
         gpu.prefill_select(q, k, v, cu, out)
         assert gpu.status() == 0
-        qh, kh, vh = (x.float().cpu().numpy() for x in (q, k, v))
-        out_h = out.float().cpu().numpy()
-        o_out, o_kept = ora.prefill(qh, kh, vh, cu, units=units)
+        qh, ocu = _gather_units(q, cu, units, H)
+        kh, _ = _gather_units(k, cu, units, H)
+        vh, _ = _gather_units(v, cu, units, H)
+        out_h, _ = _gather_units(out, cu, units, H)
+        o_out, o_kept = ora.prefill(qh, kh, vh, ocu)
         pos, acc, count, t = gpu.export()
-        for u in units:
-            s, h = divmod(u, H)
-            lo, hi = int(cu[s]), int(cu[s + 1])
-            stats.max_out_err = max(stats.max_out_err, assert_close(out_h[lo:hi, h], o_out[lo:hi, h], wl.dtype,
+        for x, u in enumerate(units):
+            lo, hi = int(ocu[x]), int(ocu[x + 1])
+            stats.max_out_err = max(stats.max_out_err, assert_close(out_h[lo:hi, 0], o_out[lo:hi, 0], wl.dtype,
                                                                     "prefill out unit %d" % u))
             m = int(count[u])
             gkept = np.sort(pos[u, :m])
-            if not np.array_equal(gkept, o_kept[u]):
-                acc0, (b_keep, b_drop) = ora.last_acc0[u], ora.last_boundary[u]
-                diff = set(gkept.tolist()) ^ set(o_kept[u].tolist())
-                assert len(gkept) == len(o_kept[u]), "prefill unit %d: kept count" % u
+            if not np.array_equal(gkept, o_kept[x]):
+                acc0, (b_keep, b_drop) = ora.last_acc0[x], ora.last_boundary[x]
+                diff = set(gkept.tolist()) ^ set(o_kept[x].tolist())
+                assert len(gkept) == len(o_kept[x]), "prefill unit %d: kept count" % u
                 for j in diff:  # every disputed position must sit on the k-th / (k+1)-th boundary
                     assert _rel(acc0[j], b_keep) < TIE_REL and _rel(acc0[j], b_drop) < TIE_REL, (
                         "prefill unit %d: position %d (score %.17g) kept/dropped against the oracle "
                         "(boundary %.17g / %.17g)" % (u, j, acc0[j], b_keep, b_drop))
                 stats.near_ties_prefill += 1
-                ora.load_unit(u, gkept, acc0[gkept], kh[lo:hi, h][gkept], vh[lo:hi, h][gkept], hi - lo)
+                ora.load_unit(x, gkept, acc0[gkept], kh[lo:hi, 0][gkept], vh[lo:hi, 0][gkept], hi - lo)
             stats.decisions += 1
         compare_state(gpu, ora, units, wl.dtype, stats, "after prefill")
         del q, k, v, out, qh, kh, vh, out_h
     ev = torch.empty(wl.batch, H, dtype=torch.int32, device=device)
+
+    def pick(x):  # [batch, H, d] -> the sampled units as [len(units), 1, d] float32 on the host
+        return x.reshape(wl.units, d)[uidx].float().cpu().numpy()[:, None, :]
+
     for step in range(steps):
         q, k, v = make_decode_inputs(wl, step, layer=layer, device=device)
         out = torch.empty_like(q)
         ev.fill_(-7)
         gpu.decode_step(q, k, v, out, ev)
-        g_ev = ev.cpu().numpy().reshape(-1)
-        g_out = out.float().cpu().numpy().reshape(wl.units, d)
-        res = ora.decode_step(q.float().cpu().numpy(), k.float().cpu().numpy(), v.float().cpu().numpy(),
-                              hint=g_ev, tie_rel=TIE_REL, units=units)
+        g_ev = ev.reshape(-1)[uidx].cpu().numpy()
+        g_out = out.reshape(wl.units, d)[uidx].float().cpu().numpy()
+        res = ora.decode_step(pick(q), pick(k), pick(v), hint=g_ev, tie_rel=TIE_REL)
         for x, u in enumerate(units):
             st = int(res["status"][x])
             if st == 2:
                 raise AssertionError("step %d unit %d: evicted %d, oracle %d (gap %.3g)" % (
-                    step, u, g_ev[u], res["evicted"][x], res["gap"][x]))
+                    step, u, g_ev[x], res["evicted"][x], res["gap"][x]))
             stats.near_ties_decode += st == 1
         stats.decisions += len(units)
-        stats.max_out_err = max(stats.max_out_err, assert_close(g_out[units], res["out"], wl.dtype, "decode out step %d" % step))
+        stats.max_out_err = max(stats.max_out_err, assert_close(g_out, res["out"], wl.dtype, "decode out step %d" % step))
         if (step + 1) % export_every == 0 or step == steps - 1:
             compare_state(gpu, ora, units, wl.dtype, stats, "after step %d" % step)
     assert gpu.status() == 0

@@ -95,3 +95,22 @@ def test_cluster_split_fill_phase_from_empty(H2OCache):
     wl = _wl("clusterfill", 1, 2, 128, "bf16", [1], 330, [150], [150], seed=32)
     st = run_parity(wl, H2OCache, prefill=False, export_every=30)
     print(st)
+
+
+def test_bf16_alu_prefill_path(H2OCache):
+    """bf16 / head_dim 128 forced onto the fp32-FMA prefill kernels (the tensor-core path is the default)."""
+    from parity_harness import run_parity
+
+    wl = _wl("alu", 2, 2, 128, "bf16", [333, 129], 8, [20, 10], [20, 10], seed=41)
+    st = run_parity(wl, H2OCache, export_every=4, prefill_path=1)
+    print(st)
+
+
+def test_tensor_core_prefill_tile_edges(H2OCache):
+    """Prompt lengths around the 64/128 tile edges of the tensor-core kernels, ragged batch."""
+    from parity_harness import run_parity
+
+    lens = [1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 640]
+    wl = _wl("edges", len(lens), 2, 128, "bf16", lens, 6, [5] * len(lens), [4] * len(lens), seed=43)
+    st = run_parity(wl, H2OCache, export_every=3)
+    print(st)
