@@ -124,6 +124,33 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
                     int32_t* evicted_pos, void* stream);
 
 /*
+ * h2o_prefill_select for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment convenience).  Some hosts of this library may not call
+ * cudaMalloc at all: a plugin inside a serving process whose memory pool is owned by someone
+ * else, a real-time loop that must not touch the allocator's lock or trigger its implicit
+ * synchronisation, a runtime that hands out device memory only at start-up.  They can pass
+ * the inputs and outputs they already hold, but have no buffer to offer as scratch.  This entry
+ * point takes none: the scratch is a fixed array of h2o_prefill_static_scratch_bytes() bytes
+ * (16 MiB) that is part of the library image, so every GPU that loads the library holds that
+ * much memory until the process exits.
+ *   - Arguments and semantics are those of h2o_prefill_select, minus scratch / scratch_bytes.
+ *   - Limit: prompts whose scratch need, h2o_prefill_scratch_bytes(cfg, cu[batch]), exceeds the
+ *     array are refused with H2O_ERR_WORKSPACE and nothing is launched (16 MiB covers about one
+ *     million (token, head) pairs, e.g. 8 prompts of 2048 tokens with 32 heads).
+ *   - It performs no device allocation or free and calls no allocating library routine.
+ *   - The first call on a device looks up the array's device address (one runtime query, with
+ *     that device made current for the query); make that first call before starting any stream
+ *     capture on the device.
+ *   - All calls on a device share the one array, and the array keeps whatever the last call
+ *     left in it.  Nothing in it needs to start at zero, so no clearing is done; but two calls
+ *     whose work overlaps on the GPU (different streams, no ordering between them) race on it
+ *     and corrupt each other.  Order such calls, or use h2o_prefill_select with own buffers.
+ */
+size_t h2o_prefill_static_scratch_bytes(void);
+int h2o_prefill_select_static(h2o_cache_t* cache, const void* q, const void* k, const void* v,
+                              const int32_t* cu_seqlens, void* out, void* stream);
+
+/*
  * The same two calls for callers whose tensors live in HOST memory (pinned memory
  * makes the copies asynchronous).  Inputs are copied to `staging` (dev, 256-byte
  * aligned) on the stream, the device call above runs on the staged copies, and the

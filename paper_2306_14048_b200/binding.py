@@ -31,6 +31,8 @@ EXPORTED = (
     "h2o_prefill_scratch_bytes",
     "h2o_cache_create",
     "h2o_prefill_select",
+    "h2o_prefill_select_static",
+    "h2o_prefill_static_scratch_bytes",
     "h2o_decode_step",
     "h2o_cache_destroy",
     "h2o_cache_reset",
@@ -75,6 +77,10 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_create.argtypes = [c.POINTER(vp), cfgp, vp, c.c_size_t]
     lib.h2o_prefill_select.restype = c.c_int
     lib.h2o_prefill_select.argtypes = [vp, vp, vp, vp, i32p, vp, vp, c.c_size_t, vp]
+    lib.h2o_prefill_select_static.restype = c.c_int
+    lib.h2o_prefill_select_static.argtypes = [vp, vp, vp, vp, i32p, vp, vp]
+    lib.h2o_prefill_static_scratch_bytes.restype = c.c_size_t
+    lib.h2o_prefill_static_scratch_bytes.argtypes = []
     lib.h2o_decode_step.restype = c.c_int
     lib.h2o_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.h2o_cache_reset.restype = c.c_int
@@ -173,6 +179,13 @@ class H2OCache:
         _check(lib.h2o_prefill_select(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                       cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), out.data_ptr(), sp, need,
                                       _stream_ptr(stream)), "h2o_prefill_select")
+
+    def prefill_select_static(self, q, k, v, cu_seqlens, out, stream=None):
+        """h2o_prefill_select_static: the scratch is the library's built-in array, nothing is allocated here."""
+        cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+        _check(lib.h2o_prefill_select_static(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                             cu.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), out.data_ptr(),
+                                             _stream_ptr(stream)), "h2o_prefill_select_static")
 
     def decode_step(self, q, k_new, v_new, out, evicted_pos=None, stream=None):
         _check(lib.h2o_decode_step(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),

@@ -130,6 +130,10 @@ struct DeviceGuard {
 
 }  // namespace
 
+namespace h2o {
+const h2o_config_t* cache_config(const h2o_cache_t* cache) { return &cache->cfg; }
+}  // namespace h2o
+
 extern "C" {
 
 size_t h2o_cache_workspace_bytes(const h2o_config_t* cfg) {

@@ -45,6 +45,9 @@ struct PrefillScratch {
   int64_t total_tokens;
 };
 
+// Read-only view of a handle's configuration (budget arrays are the handle's own copies).
+const h2o_config_t* cache_config(const h2o_cache_t* cache);
+
 // Launchers (each returns the cudaError_t of its launch).
 // `split` thread blocks (one cluster) share a unit, each owning `chunk` consecutive slots.
 // `stages` is the depth of the shared-memory ring (0 = default).
