@@ -374,6 +374,8 @@ def main():
             "prefill_ms": prefill_ms, "decode_ms": decode_ms,
             "decode_only_seq_heads_per_s": wl.units * L * S / (decode_ms * 1e-3),
             "prefill_tflops_algorithmic": flops / (prefill_ms * 1e-3) / 1e12,
+            # tensor-core work actually issued: S, P_hi V, P_lo V and S^T (four triangle products for two)
+            "prefill_tflops_executed_mma": 2.0 * flops / (prefill_ms * 1e-3) / 1e12,
             "gpu_launches": args.steps * L * (3 + S),
             "clocks": clocks,
             "roofline": {
