@@ -210,6 +210,14 @@ int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages
  *   once the stream has finished the call.
  */
 int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
+/*
+ * Process-wide diagnostic switch (no counterpart in the paper).  A decode kernel launched right
+ * after a decode / prefill / reset of a DIFFERENT cache on the same stream starts copying its own
+ * cache tiles into shared memory before the preceding kernel has finished (inputs q/k/v are still
+ * read only afterwards).  0 turns that off, so that every launch waits first; results must be
+ * identical either way.  Returns the previous setting.
+ */
+int h2o_debug_set_early_prefetch(int32_t enabled);
 int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, size_t* acc0_offset);
 const char* h2o_strerror(int code);
 

@@ -43,6 +43,7 @@ EXPORTED = (
     "h2o_cache_status",
     "h2o_cache_set_decode_shape",
     "h2o_cache_set_prefill_path",
+    "h2o_debug_set_early_prefetch",
     "h2o_prefill_scratch_layout",
     "h2o_strerror",
 )
@@ -103,6 +104,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_set_prefill_path.argtypes = [vp, c.c_int32]
     lib.h2o_prefill_scratch_layout.restype = c.c_int
     lib.h2o_prefill_scratch_layout.argtypes = [cfgp, c.c_int64, c.POINTER(c.c_size_t)]
+    lib.h2o_debug_set_early_prefetch.restype = c.c_int
+    lib.h2o_debug_set_early_prefetch.argtypes = [c.c_int32]
     lib.h2o_strerror.restype = c.c_char_p
     lib.h2o_strerror.argtypes = [c.c_int]
     return lib

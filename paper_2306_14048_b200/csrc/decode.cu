@@ -161,7 +161,8 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads + 32)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
-              T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages) {
+              T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
+              int cache_is_quiescent) {
   using C = Cfg<T, D>;
   constexpr int VEC = C::VEC, LPR = C::LPR, RPW = C::RPW, RPC = C::RPC, TILE_ROWS = C::TILE_ROWS, GROUPS = C::GROUPS;
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -180,10 +181,18 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   const int su = blockIdx.x / split;  // launch position of the unit
   const UnitMeta mt = c.meta[su];     // static table, written once at create time
   // Programmatic dependent launch: this grid may have been started while the previous kernel of
-  // the stream was still draining.  Let the next one start as early as it can, and wait for the
-  // previous one to finish (and flush) before reading anything it may have written.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // the stream was still running.  What it may touch before that kernel has finished
+  // (griddepcontrol.wait) depends on who wrote what:
+  //   - q / k_new / v_new can come from any kernel, so they are read only after the wait;
+  //   - the cache itself is written by this library alone.  The host tells us whether its previous
+  //     launch on this stream could have written THIS cache; if not (`cache_is_quiescent`), the cache
+  //     tiles are prefetched into shared memory before the wait, which hides the start-up latency.
+  // The next grid is released (launch_dependents) only after this grid's own wait: when a grid
+  // starts, everything older than its immediate predecessor has therefore completed.
+  if (!cache_is_quiescent) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   const int cnt = c.count[su];
   const int t = c.tpos[su];
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
@@ -225,6 +234,10 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
   }
   __syncthreads();  // barriers are initialised before any consumer polls them
+  if (cache_is_quiescent) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
 
   // the new token's own key/value: loaded now, used after the stream
   float qf[VEC], ksf[VEC], vself = 0.f;
@@ -461,8 +474,8 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
 }
 
 template <typename T, int D>
-cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, const void* q, const void* k_new,
-                   const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
+                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   using C = Cfg<T, D>;
   // ring depth: the whole chunk if it is short, otherwise enough to keep ~64 KB in flight per block
   const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : kDefaultStages;
@@ -491,7 +504,8 @@ cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, con
   cfg.attrs = at;
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, decode_kernel<T, D>, c, static_cast<const T*>(q), static_cast<const T*>(k_new),
-                            static_cast<const T*>(v_new), static_cast<T*>(out), evicted_pos, split, chunk, stages);
+                            static_cast<const T*>(v_new), static_cast<T*>(out), evicted_pos, split, chunk, stages,
+                            quiescent ? 1 : 0);
 }
 
 }  // namespace
@@ -502,16 +516,18 @@ extern "C" int h2o_debug_phase_timers(unsigned long long* host, int n) {
 }
 #endif
 
-cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, const void* q,
-                          const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent,
+                          const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+                          cudaStream_t stream) {
   if (split < 1 || split > kMaxSplit) return cudaErrorInvalidValue;
   if (dtype == H2O_F32) {
-    if (c.head_dim == 64) return launch<float, 64>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
-    return launch<float, 128>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
+    if (c.head_dim == 64)
+      return launch<float, 64>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+    return launch<float, 128>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);
   }
   if (c.head_dim == 64)
-    return launch<__nv_bfloat16, 64>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
-  return launch<__nv_bfloat16, 128>(c, split, chunk, stages, q, k_new, v_new, out, evicted_pos, stream);
+    return launch<__nv_bfloat16, 64>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+  return launch<__nv_bfloat16, 128>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace h2o

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <numeric>
 #include <vector>
@@ -112,6 +113,43 @@ struct h2o_cache {
 };
 
 namespace {
+
+// Which cache did this library's most recent launch on a stream write?  Only this library writes a
+// cache workspace, so if the answer is "another cache" (or the stream has since run foreign work,
+// which completes our earlier kernel first), a decode kernel may read its cache before the preceding
+// kernel of the stream has finished.  Unknown streams are treated as "this cache" (no early reads).
+class LastWriter {
+ public:
+  // returns true if the last recorded writer on `stream` is a different cache; then records `cache`
+  bool note_and_check(cudaStream_t stream, const void* cache) {
+    std::lock_guard<std::mutex> lock(mu_);
+    for (auto& e : entries_) {
+      if (e.stream == stream) {
+        const bool other = e.cache != nullptr && e.cache != cache;
+        e.cache = cache;
+        return other;
+      }
+    }
+    if (entries_.size() >= 64) entries_.erase(entries_.begin());
+    entries_.push_back({stream, cache});
+    return false;
+  }
+  void forget(const void* cache) {
+    std::lock_guard<std::mutex> lock(mu_);
+    for (auto& e : entries_)
+      if (e.cache == cache) e.cache = nullptr;
+  }
+
+ private:
+  struct Entry {
+    cudaStream_t stream;
+    const void* cache;
+  };
+  std::mutex mu_;
+  std::vector<Entry> entries_;
+};
+LastWriter g_last_writer;
+bool g_early_prefetch = true;  // diagnostic switch, see h2o_debug_set_early_prefetch
 
 struct DeviceGuard {
   int prev = -1;
@@ -278,6 +316,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
+  g_last_writer.note_and_check(st, cache->view.K);  // select/gather wrote this cache
   cache->phase = Phase::Prefilled;
   return H2O_OK;
 }
@@ -289,8 +328,11 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
     if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
   DeviceGuard guard(cache->cfg.device);
   if (!guard.ok) return H2O_ERR_CUDA;
-  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, q,
-                                           k_new, v_new, out, evicted_pos, static_cast<cudaStream_t>(stream));
+  // the cache workspace is the identity: two handles on one workspace must count as the same cache
+  const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
+  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages,
+                                           quiescent, q, k_new, v_new, out, evicted_pos,
+                                           static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
@@ -385,6 +427,7 @@ int h2o_cache_reset(h2o_cache_t* cache, void* stream) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
+  g_last_writer.note_and_check(st, cache->view.K);  // the memsets wrote this cache
   cache->phase = Phase::Empty;
   return H2O_OK;
 }
@@ -415,7 +458,14 @@ int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, si
   return H2O_OK;
 }
 
+int h2o_debug_set_early_prefetch(int32_t enabled) {
+  const int prev = g_early_prefetch ? 1 : 0;
+  g_early_prefetch = enabled != 0;
+  return prev;
+}
+
 int h2o_cache_destroy(h2o_cache_t* cache) {
+  if (cache) g_last_writer.forget(cache->view.K);
   delete cache;
   return H2O_OK;
 }

@@ -50,9 +50,12 @@ const h2o_config_t* cache_config(const h2o_cache_t* cache);
 
 // Launchers (each returns the cudaError_t of its launch).
 // `split` thread blocks (one cluster) share a unit, each owning `chunk` consecutive slots.
-// `stages` is the depth of the shared-memory ring (0 = default).
-cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, const void* q,
-                          const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream);
+// `stages` is the depth of the shared-memory ring (0 = default).  `quiescent`: nothing this library
+// launched immediately before on the stream can have written this cache, so the kernel may read the
+// cache before the previous kernel of the stream has finished (it still waits before reading q/k/v).
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent,
+                          const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+                          cudaStream_t stream);
 // ALU path; `rows` = attention rows + row statistics, `colsum` = column sums.
 cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int max_seqlen, const void* q,
                                  const void* k, const void* v, void* out, bool rows, bool colsum, cudaStream_t stream);

@@ -27,12 +27,6 @@ constexpr int kBoxBytes = kTile * 128;   // one TMA box: 128 rows x 64 bf16
 constexpr int kTileBytes = 2 * kBoxBytes;  // two boxes cover head_dim 128
 constexpr double kLog2eD = 1.4426950408889634074;
 
-// softmax scale times log2(e) as an unevaluated sum hi + lo of two floats, so that the product
-// with a raw score carries no rounding error of the constant
-struct Scale2 {
-  float hi, lo;
-};
-
 // ---- abortable waits: the first role that times out raises a flag every other wait observes ----
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -52,7 +46,7 @@ __device__ __forceinline__ float ex2(float x) {
 // ---------------------------------------------------------------------------------------------
 // Column sums
 // ---------------------------------------------------------------------------------------------
-constexpr int kCsThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kCsThreads = 320;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kCsQStages = 2;
 constexpr int kCsTmemCols = 256;  // two accumulator buffers of 128 columns
 
@@ -60,15 +54,17 @@ struct CsShared {
   uint64_t k_full, k_empty;
   uint64_t q_full[kCsQStages], q_empty[kCsQStages];
   uint64_t acc_full[2], acc_empty[2];
-  uint64_t nl_full[2];  // the 128 epilogue threads have staged the tile's row statistics
+  uint64_t nl_full[2];  // 128 epilogue threads have staged the tile's row statistics
+  uint64_t ps_full, ps_empty;  // hand-over of the second query half's partial sums
   uint32_t tmem_base;
   int abort_flag;
-  float2 rstat[2][kTile];  // per query of the tile: {minus reference maximum (log2 domain), 1 / row sum}
+  __align__(16) float2 rstat[2][kTile];  // per query of the tile: {minus reference maximum (log2 domain), 1 / row sum}
+  double psum[kTile];
 };
 
 __global__ void __launch_bounds__(kCsThreads)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 PrefillScratch s, int n_heads, Scale2 scale2, int32_t* status) {
+                 PrefillScratch s, int n_heads, float scale2, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ CsShared sh;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
@@ -97,9 +93,11 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.acc_full[i], 1);
-      mbar_init(&sh.acc_empty[i], 4);  // one arrival per epilogue warp
+      mbar_init(&sh.acc_empty[i], 8);  // one arrival per epilogue warp
       mbar_init(&sh.nl_full[i], 128);
     }
+    mbar_init(&sh.ps_full, 128);
+    mbar_init(&sh.ps_empty, 128);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -160,15 +158,18 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     }
   } else {
     // ---------------- epilogue: exp and in-thread column sums ----------------
-    const int e = threadIdx.x - 64;          // 0..127
+    // Eight warps: warps w and w+4 share a TMEM lane quarter (the same 32 key rows); the first
+    // takes queries 0..63 of the tile, the second queries 64..127.
+    const int e = threadIdx.x - 64;          // 0..255
     const int quarter = warp & 3;            // TMEM lane quarter this warp may access
+    const int half = e >> 7;                 // which 64 queries of the tile
     const int row = quarter * 32 + lane;     // key row inside the tile = TMEM lane
     const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
     double total_sum = 0.0;
     auto fetch_nlse = [&](int t) -> float2 {
       const int ib = t < t0 ? jb0 + t : jb1 + (t - t0);
       const int qi = ib * kTile + e;
-      if (qi >= n) return make_float2(-INFINITY, 0.f);  // rows past the end: exp2(-inf) * 0 = 0
+      if (e >= kTile || qi >= n) return make_float2(-INFINITY, 0.f);  // rows past the end: exp2(-inf) * 0 = 0
       const float2 v2 = rowstat[qi];
       return make_float2(-v2.x, v2.y);
     };
@@ -179,36 +180,61 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int jb = cb == 0 ? jb0 : jb1;
       const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
       const int b = t & 1;
-      sh.rstat[b][e] = nl_next;
+      if (e < kTile) {
+        sh.rstat[b][e] = nl_next;
+        mbar_arrive(&sh.nl_full[b]);
+      }
       if (t + 1 < total) nl_next = fetch_nlse(t + 1);
-      mbar_arrive(&sh.nl_full[b]);
       ok = wait_or_abort(&sh.nl_full[b], (t >> 1) & 1, abort_flag) && wait_or_abort(&sh.acc_full[b], (t >> 1) & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
       if (!ok) break;
       tc_fence_after();
-      const bool diag = ib == jb;
-      float tile_sum = 0.f;
+      const uint32_t taddr = tmem + (uint32_t)b * kTile + (uint32_t)half * 64u + ((uint32_t)(quarter * 32) << 16);
+      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b][half * 64]);  // {-m, 1/l} of two queries
+      uint32_t r0[32], r1[32];
+      tmem_ld32(taddr, r0);
+      tmem_wait_ld();
+      tmem_ld32(taddr + 32u, r1);  // in flight while the first 32 columns are processed
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      auto chunk = [&](const uint32_t (&r)[32], int c0, bool masked) {
 #pragma unroll
-      for (int cc = 0; cc < kTile / 32; ++cc) {
-        uint32_t r[32];
-        tmem_ld32(tmem + (uint32_t)b * kTile + (uint32_t)cc * 32u + ((uint32_t)(quarter * 32) << 16), r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int c2 = 0; c2 < 32; ++c2) {
-          const int ql = cc * 32 + c2;  // query inside the tile
-          const float2 st2 = sh.rstat[b][ql];
-          const float sv = __uint_as_float(r[c2]);
-          const float pval = ex2(fmaf(sv, scale2.hi, fmaf(sv, scale2.lo, st2.x))) * st2.y;
-          tile_sum += (diag && ql < row) ? 0.f : pval;  // causal: query >= key
+        for (int c2 = 0; c2 < 32; c2 += 2) {
+          const float4 st = st4[(c0 + c2) >> 1];
+          float pa = ex2(fmaf(__uint_as_float(r[c2]), scale2, st.x)) * st.y;
+          float pb = ex2(fmaf(__uint_as_float(r[c2 + 1]), scale2, st.z)) * st.w;
+          if (masked) {  // causal: query >= key (diagonal tile only)
+            const int ql = half * 64 + c0 + c2;
+            if (ql < row) pa = 0.f;
+            if (ql + 1 < row) pb = 0.f;
+          }
+          sum4[(c2 >> 1) & 3] += pa + pb;
         }
+      };
+      if (ib == jb) {
+        chunk(r0, 0, true);
+        tmem_wait_ld();
+        chunk(r1, 32, true);
+      } else {
+        chunk(r0, 0, false);
+        tmem_wait_ld();
+        chunk(r1, 32, false);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
-      total_sum += (double)tile_sum;
-      if (t == t0 - 1 || t == total - 1) {  // last tile of this key block
-        const int key = jb * kTile + row;
-        if (key < n) s.acc0[(int64_t)h * s.total_tokens + lo + key] = total_sum;
+      total_sum += (double)((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      if (t == t0 - 1 || t == total - 1) {  // last tile of this key block: add the two query halves
+        if (half == 1) {
+          sh.psum[row] = total_sum;
+          mbar_arrive(&sh.ps_full);
+        } else {
+          ok = wait_or_abort(&sh.ps_full, cb, abort_flag);
+          const int key = jb * kTile + row;
+          if (ok && key < n) s.acc0[(int64_t)h * s.total_tokens + lo + key] = total_sum + sh.psum[row];
+          if (ok) mbar_arrive(&sh.ps_empty);
+        }
+        if (half == 1 && cb == 0 && ncb == 2) ok = wait_or_abort(&sh.ps_empty, 0, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);  // keep the warp together for the next tile's collectives
         total_sum = 0.0;
       }
     }
@@ -254,7 +280,7 @@ struct FwShared {
 template <typename OutT>
 __global__ void __launch_bounds__(kFwThreads)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, Scale2 scale2,
+              const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, float scale2,
               OutT* __restrict__ out, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FwShared sh;
@@ -373,8 +399,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       float m_tile = -INFINITY;
 #pragma unroll
       for (int c2 = 0; c2 < kFwKeys; ++c2) {
-        const float sv = __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]);
-        float x = fmaf(sv, scale2.hi, sv * scale2.lo);
+        float x = __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]) * scale2;
         if (masked_tile && key0 + c2 > qi) x = -INFINITY;  // causal: key <= query
         sc[c2] = x;
         m_tile = fmaxf(m_tile, x);
@@ -492,13 +517,9 @@ bool make_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_he
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-Scale2 make_scale2(float c) {
-  const double x = (double)c * kLog2eD;
-  Scale2 r;
-  r.hi = (float)x;
-  r.lo = (float)(x - (double)r.hi);
-  return r;
-}
+// Softmax scale times log2(e), rounded once.  The forward and the column-sum kernel use the same
+// value, so a row's probabilities sum to one exactly as the forward pass normalised them.
+float make_scale2(float c) { return (float)((double)c * kLog2eD); }
 
 }  // namespace
 

@@ -114,3 +114,50 @@ def test_tensor_core_prefill_tile_edges(H2OCache):
     wl = _wl("edges", len(lens), 2, 128, "bf16", lens, 6, [5] * len(lens), [4] * len(lens), seed=43)
     st = run_parity(wl, H2OCache, export_every=3)
     print(st)
+
+
+def test_rotating_caches_early_prefetch_equals_waiting_first(H2OCache):
+    """Several caches stepped in rotation on one stream (the benchmark's pattern).  The kernels then
+    prefetch their cache before the previous launch has finished; everything observable must be
+    bit-identical to the run in which every launch waits first."""
+    import paper_2306_14048_b200 as pkg
+    from workloads import make_decode_inputs, make_prompt_inputs
+
+    wl = _wl("rot", 6, 8, 128, "bf16", [700] * 6, 24, [60] * 6, [60] * 6, seed=51)
+    n_caches = 3
+
+    def run(early):
+        prev = pkg.lib.h2o_debug_set_early_prefetch(1 if early else 0)
+        try:
+            caches = [H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent) for _ in range(n_caches)]
+            for l, c in enumerate(caches):
+                q, k, v, cu = make_prompt_inputs(wl, layer=l, device="cuda")
+                c.prefill_select(q, k, v, cu, torch.empty_like(q))
+            outs, evs = [], []
+            ins = [[make_decode_inputs(wl, s, layer=l, device="cuda") for l in range(n_caches)] for s in range(wl.decode_steps)]
+            torch.cuda.synchronize()
+            for s in range(wl.decode_steps):
+                for l, c in enumerate(caches):
+                    q, k, v = ins[s][l]
+                    o = torch.empty_like(q)
+                    e = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32, device="cuda")
+                    c.decode_step(q, k, v, o, e)
+                    outs.append(o)
+                    evs.append(e)
+            torch.cuda.synchronize()
+            state = [c.export() for c in caches]
+            assert all(c.status() == 0 for c in caches)
+            for c in caches:
+                c.close()
+            return [o.float().cpu().numpy() for o in outs], [e.cpu().numpy() for e in evs], state
+        finally:
+            pkg.lib.h2o_debug_set_early_prefetch(prev)
+
+    a, b = run(True), run(False)
+    for x, y in zip(a[0], b[0]):
+        assert np.array_equal(x, y)
+    for x, y in zip(a[1], b[1]):
+        assert np.array_equal(x, y)
+    for sa, sb in zip(a[2], b[2]):
+        for x, y in zip(sa, sb):
+            assert np.array_equal(x, y)
