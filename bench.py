@@ -53,6 +53,24 @@ def decode_bytes_per_unit_step(cnt: int, d: int, esize: int) -> int:
     return 2 * cnt * d * esize + 16 * cnt + 4 * cnt + 6 * d * esize
 
 
+# DRAM bytes (read + write) of one decode launch, from the ncu capture summarised in
+# profiles/decode_kernel__c2_opt6p7b.md (55.26 MB read + 0.07 MB written for config 2).
+NCU_DECODE_TRAFFIC_PER_LAUNCH = {"c2_opt6p7b": 55.33e6}
+
+
+def aggregate_over_ranks(values, world: int, device, dist=None):
+    """Max over ranks of per-rank timings (the job is as slow as its slowest replica)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_value(units_per_rank: int, layers: int, decode_steps: int, bench_steps: int, world: int, total_ms: float):
+    """(sequence, head) decode steps per second over all replicas."""
+    return units_per_rank * layers * world * decode_steps * bench_steps / (total_ms * 1e-3)
+
+
 def prefill_flops(n: int, d: int) -> float:
     """Algorithmic flops of one unit's prompt attention: QK^T and PV over the causal triangle."""
     return 4.0 * d * n * (n + 1) / 2.0
@@ -344,15 +362,13 @@ def main():
         e2e = {"ms_per_step": e2e_ms, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
         del hp, hd
 
-    ms = torch.tensor([total_ms, prefill_ms, decode_ms, e2e["ms_per_step"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    total_ms, prefill_ms, decode_ms, e2e_ms = (float(x) for x in ms.cpu())
+    total_ms, prefill_ms, decode_ms, e2e_ms = aggregate_over_ranks(
+        [total_ms, prefill_ms, decode_ms, e2e["ms_per_step"] if e2e else 0.0], world, dev, dist if world > 1 else None)
 
     if rank == 0:
         units_all = wl.units * L * world
         unit_steps = units_all * S
-        value = unit_steps * args.steps / (total_ms * 1e-3)
+        value = whole_job_value(wl.units, L, S, args.steps, world, total_ms)
         hbm_peak, peak_kind = _peaks()
         cnt = [min(n, kk + rr) for n, kk, rr in zip(wl.prompt_lens, wl.heavy, wl.recent)]
         bytes_launch = sum(decode_bytes_per_unit_step(c, d, esize) for c in cnt) * H
@@ -380,7 +396,8 @@ def main():
             "clocks": clocks,
             "roofline": {
                 "kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "peak_source": peak_kind, "traffic": None,
+                "frac": achieved / hbm_peak, "peak_source": peak_kind,
+                "traffic": NCU_DECODE_TRAFFIC_PER_LAUNCH.get(wl.name),
                 "bytes_per_launch": bytes_launch, "avg_launch_us": launch_us,
                 "frac_of_nominal_8TBs": achieved / 8000.0,
             },
