@@ -27,6 +27,16 @@ constexpr int kBoxBytes = kTile * 128;   // one TMA box: 128 rows x 64 bf16
 constexpr int kTileBytes = 2 * kBoxBytes;  // two boxes cover head_dim 128
 constexpr double kLog2eD = 1.4426950408889634074;
 
+// Optional cycle accounting of the forward kernel's softmax loop (compile with -DH2O_PHASE_TIMERS).
+#ifdef H2O_PHASE_TIMERS
+__device__ unsigned long long g_fwd_prof[8];
+#define FWD_CLK(v) const long long v = clock64()
+#define FWD_ADD(i, a, b) prof_[i] += (b) - (a)
+#else
+#define FWD_CLK(v) do { } while (0)
+#define FWD_ADD(i, a, b) do { } while (0)
+#endif
+
 // ---- abortable waits: the first role that times out raises a flag every other wait observes ----
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -132,28 +142,31 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
+    {
       constexpr uint32_t idesc = instr_desc_f16(kTile, kTile, kFmtBF16, kFmtBF16, false, false);
       for (int t = 0; t < total; ++t) {
         const int cb = t < t0 ? 0 : 1;
-        if (t == 0 || t == t0) {
-          if (!wait_or_abort(&sh.k_full, cb, abort_flag)) break;
-        }
+        bool ok = true;
+        if (t == 0 || t == t0) ok = wait_or_abort(&sh.k_full, cb, abort_flag);
         const int st = t % kCsQStages, b = t & 1;
-        if (!wait_or_abort(&sh.q_full[st], (t / kCsQStages) & 1, abort_flag)) break;
-        if (!wait_or_abort(&sh.acc_empty[b], ((t >> 1) & 1) ^ 1, abort_flag)) break;
+        ok = ok && wait_or_abort(&sh.q_full[st], (t / kCsQStages) & 1, abort_flag);
+        ok = ok && wait_or_abort(&sh.acc_empty[b], ((t >> 1) & 1) ^ 1, abort_flag);
+        if (!__all_sync(0xffffffffu, ok)) break;
         tc_fence_after();
         const uint32_t a0 = smem_u32(k_tile), b0 = smem_u32(q_ring + st * kTileBytes);
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t off = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
-          mma_ss(tmem + (uint32_t)b * kTile, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
-                 idesc, ks > 0);
+          for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t off = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+            mma_ss(tmem + (uint32_t)b * kTile, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
+                   idesc, ks > 0);
+          }
+          mma_commit(&sh.q_empty[st]);   // the Q stage may be refilled once these MMAs have read it
+          mma_commit(&sh.acc_full[b]);   // and the accumulator is ready for the epilogue
+          if (t == t0 - 1 && ncb == 2) mma_commit(&sh.k_empty);
         }
-        mma_commit(&sh.q_empty[st]);   // the Q stage may be refilled once these MMAs have read it
-        mma_commit(&sh.acc_full[b]);   // and the accumulator is ready for the epilogue
-        if (t == t0 - 1 && ncb == 2) mma_commit(&sh.k_empty);
+        __syncwarp();
       }
     }
   } else {
@@ -249,65 +262,81 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------
-// Forward: out = softmax(c Q K^T) V over the causal triangle, plus the row log-sum-exp
+// Forward: out = softmax(c Q K^T) V over the causal triangle, plus per-row {max, 1/sum}
 // ---------------------------------------------------------------------------------------------
-// One thread block per (unit, block of 128 queries); key tiles of 64.  Per key tile:
-//   MMA warp     : S = Q K_j^T            (M 128, N 64, K 128; accumulator in TMEM)
-//   softmax warps: one thread per query row reads its S row from TMEM, updates the running
-//                  maximum lazily (the reference maximum only moves when it would grow by more
-//                  than 8 in the log2 domain, so the O rows in TMEM are rescaled rarely),
-//                  writes P = exp2(S - m) as bf16 into a 128B-swizzled shared-memory tile
-//   MMA warp     : O += P V_j             (M 128, N 128, K 64; V is the MN-major operand)
-//                  (P is split into a bf16 hi and a bf16 lo part, multiplied one after the other,
-//                  so that the output does not carry the 2^-9 rounding of a single bf16 P)
-// Two blocks fit on an SM (96 KB of shared memory, 256 TMEM columns each); one block's softmax
-// overlaps the other's matrix instructions.
-constexpr int kFwThreads = 192;
+// One thread block per (unit, PAIR of 128-query blocks); key tiles of 64, loaded once (TMA) for
+// both query blocks.  Two softmax warpgroups (A, B), one per query block, and one MMA-issuing warp
+// that runs a small event loop.  Per group g and key tile j:
+//   S_g(j) = Q_g K_j^T           M 128, N 64, K 128; Q and K from shared memory, fp32 accumulator
+//                                in TMEM.  Issued as soon as the softmax has READ S_g(j-1) into
+//                                registers, so it runs while that softmax is still computing.
+//   P_g(j) = exp2(c S_g(j) - m)  written by the softmax threads into TMEM as bf16 hi | bf16 lo
+//                                (a single bf16 P would put its 2^-9 rounding into the output)
+//   O_g   += P_hi V_j + P_lo V_j M 128, N 128, K 64 twice; P is the TMEM operand, V the MN-major
+//                                shared-memory operand (with P in shared memory as well the
+//                                instruction is bound by shared-memory bandwidth)
+// The softmax keeps one thread per query row (row max / sum need no shuffles) and updates the
+// reference maximum lazily: O rows in TMEM are rescaled only when the maximum grows by more than
+// 8 in the log2 domain.  One block per SM: all 512 TMEM columns, 161 KB of shared memory.
+constexpr int kFwThreads = 320;                   // warp 0: TMA, warp 1: MMA, warps 2..5: group A, 6..9: group B
 constexpr int kFwKeys = 64;                       // keys per tile
 constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
-constexpr int kFwKvSlots = 2;                     // slot 0 holds K tiles, slot 1 holds V tiles
-constexpr int kFwTmemCols = 256;                  // O: columns 0..127, S: columns 128..191
+constexpr int kFwKvSlots = 6;                     // K_j, V_j, K_j+1, V_j+1, K_j+2, V_j+2
+constexpr int kFwTmemCols = 512;
+constexpr uint32_t kFwColO = 0;                   // O_g : 128 columns each
+constexpr uint32_t kFwColS = 256;                 // S_g : 64 columns each
+constexpr uint32_t kFwColP = 384;                 // P_g : 64 columns each (hi 0..31, lo 32..63)
 constexpr float kRescaleThreshold = 8.0f;
+constexpr uint32_t kFwLoopLimit = 1u << 26;       // passes of the MMA event loop before it gives up
 
 struct FwShared {
-  uint64_t q_full;
+  uint64_t q_full[2];
   uint64_t kv_full[kFwKvSlots], kv_empty[kFwKvSlots];
-  uint64_t s_full, p_full, o_done;
+  uint64_t s_full[2];   // MMA -> softmax: S_g(j) complete
+  uint64_t s_free[2];   // softmax -> MMA: S_g(j) is in registers, the columns may be overwritten
+  uint64_t p_full[2];   // softmax -> MMA: P_g(j) is in tensor memory
+  uint64_t pv_done[2];  // MMA -> softmax: O_g includes tile j (P_g may be overwritten, O_g may be rescaled)
   uint32_t tmem_base;
   int abort_flag;
 };
 
-template <typename OutT>
 __global__ void __launch_bounds__(kFwThreads)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, float scale2,
-              OutT* __restrict__ out, int32_t* status) {
+              __nv_bfloat16* __restrict__ out, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FwShared sh;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
-  unsigned char* q_tile = dyn;                                   // 32 KB
-  unsigned char* kv_ring = dyn + kTileBytes;                     // 3 x 16 KB
-  unsigned char* p_tile = kv_ring + kFwKvSlots * kFwKvSlotBytes;  // 2 x 16 KB: hi and lo parts, [128 rows][64 bf16], swizzled
+  unsigned char* q_tiles = dyn;                       // 2 x 32 KB
+  unsigned char* kv_ring = dyn + 2 * kTileBytes;      // 6 x 16 KB
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u = blockIdx.y;
   const int seq = u / n_heads, h = u % n_heads;
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
   const int nb = (n + kTile - 1) / kTile;
-  if ((int)blockIdx.x >= nb) return;
-  const int ib = nb - 1 - (int)blockIdx.x;  // long row blocks first
-  const int kmax = min(n, (ib + 1) * kTile);               // keys 0 .. kmax-1 are visible to this block
-  const int nt = (kmax + kFwKeys - 1) / kFwKeys;
+  const int npair = (nb + 1) / 2;
+  if ((int)blockIdx.x >= npair) return;
+  const int pr = npair - 1 - (int)blockIdx.x;  // long pairs first
+  const int ibA = 2 * pr, ibB = 2 * pr + 1;
+  const bool hasB = ibB < nb;
+  // key tiles visible to each group (keys 0 .. min(n, (ib+1)*128) - 1)
+  const int ntA = (min(n, (ibA + 1) * kTile) + kFwKeys - 1) / kFwKeys;
+  const int ntB = hasB ? (min(n, (ibB + 1) * kTile) + kFwKeys - 1) / kFwKeys : 0;
+  const int nt = max(ntA, ntB);
 
   if (threadIdx.x == 0) {
-    mbar_init(&sh.q_full, 1);
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(&sh.q_full[g], 1);
+      mbar_init(&sh.s_full[g], 1);
+      mbar_init(&sh.s_free[g], 4);
+      mbar_init(&sh.p_full[g], 4);
+      mbar_init(&sh.pv_done[g], 1);
+    }
     for (int i = 0; i < kFwKvSlots; ++i) {
       mbar_init(&sh.kv_full[i], 1);
       mbar_init(&sh.kv_empty[i], 1);
     }
-    mbar_init(&sh.s_full, 1);
-    mbar_init(&sh.p_full, 4);
-    mbar_init(&sh.o_done, 1);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -316,18 +345,20 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
-  const uint32_t tmem_o = tmem, tmem_s = tmem + 128u;
   volatile int* abort_flag = &sh.abort_flag;
 
   if (warp == 0) {
-    // ---------------- TMA producer: Q once, then K_0, V_0, K_1, V_1, ... through three slots ----
+    // ---------------- TMA producer: Q tiles, then K_0, V_0, K_1, V_1, ... through the slot ring ----
     if (lane == 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      mbar_expect_tx(&sh.q_full, kTileBytes);
-      tma_load_3d(q_tile, &map_q, 0, h, lo + ib * kTile, &sh.q_full);
-      tma_load_3d(q_tile + kBoxBytes, &map_q, 64, h, lo + ib * kTile, &sh.q_full);
+      for (int g = 0; g < (hasB ? 2 : 1); ++g) {
+        unsigned char* dst = q_tiles + g * kTileBytes;
+        mbar_expect_tx(&sh.q_full[g], kTileBytes);
+        tma_load_3d(dst, &map_q, 0, h, lo + (ibA + g) * kTile, &sh.q_full[g]);
+        tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + (ibA + g) * kTile, &sh.q_full[g]);
+      }
       for (int r = 0; r < 2 * nt; ++r) {
         const int slot = r % kFwKvSlots;
         if (!wait_or_abort(&sh.kv_empty[slot], ((r / kFwKvSlots) & 1) ^ 1, abort_flag)) break;
@@ -340,140 +371,211 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
-      // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
-      // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
-      constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
-      bool ok = wait_or_abort(&sh.q_full, 0, abort_flag);
-      const uint32_t q0 = smem_u32(q_tile), p0 = smem_u32(p_tile);
-      for (int j = 0; j < nt && ok; ++j) {
-        const int rk = 2 * j, rv = 2 * j + 1;
-        const int sk = rk % kFwKvSlots, sv = rv % kFwKvSlots;
-        ok = wait_or_abort(&sh.kv_full[sk], (rk / kFwKvSlots) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t k0 = smem_u32(kv_ring + sk * kFwKvSlotBytes);
+    // ---------------- MMA issuer: the whole warp runs an event loop, one elected lane issues ----------
+    constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
+    // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
+    // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
+    constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
+    auto slot_of = [&](int r) { return r % kFwKvSlots; };
+    auto par_of = [&](int r) { return (uint32_t)(r / kFwKvSlots) & 1u; };
+    const int ntg[2] = {ntA, ntB};
+    int next_s[2] = {0, 0};    // next S tile to issue per group
+    int next_pv[2] = {0, 0};   // next P V tile to issue per group
+    bool ok = wait_or_abort(&sh.q_full[0], 0, abort_flag) && (!hasB || wait_or_abort(&sh.q_full[1], 0, abort_flag));
+    ok = __all_sync(0xffffffffu, ok) != 0;
+    if (ok) tc_fence_after();
+    uint32_t idle = 0;
+    while (ok && (next_pv[0] < ntg[0] || next_pv[1] < ntg[1])) {
+      bool progressed = false;
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
-          const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
-          mma_ss(tmem_s, smem_desc_sw128(q0 + qoff, 16, 1024), smem_desc_sw128(k0 + koff, 16, 1024), idesc_s, ks > 0);
+      for (int g = 0; g < 2; ++g) {
+        // ---- S_g(j): needs K_j in shared memory and the previous S_g read out by the softmax ----
+        int j = next_s[g];
+        if (j < ntg[g]) {
+          bool ready = mbar_test_wait(&sh.kv_full[slot_of(2 * j)], par_of(2 * j));
+          if (ready && j > 0) ready = mbar_test_wait(&sh.s_free[g], (uint32_t)(j - 1) & 1u);
+          if (__all_sync(0xffffffffu, ready)) {
+            tc_fence_after();
+            const uint32_t q0 = smem_u32(q_tiles + g * kTileBytes);
+            const uint32_t k0 = smem_u32(kv_ring + slot_of(2 * j) * kFwKvSlotBytes);
+            if (elect_one()) {
+#pragma unroll
+              for (int ks = 0; ks < kD / 16; ++ks) {
+                const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+                const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
+                mma_ss(tmem + kFwColS + (uint32_t)g * 64u, smem_desc_sw128(q0 + qoff, 16, 1024),
+                       smem_desc_sw128(k0 + koff, 16, 1024), idesc_s, ks > 0);
+              }
+              mma_commit(&sh.s_full[g]);
+              // K_j may be refilled once both groups' scores have read it
+              const int other = g ^ 1;
+              if (j >= ntg[other] || next_s[other] > j) mma_commit(&sh.kv_empty[slot_of(2 * j)]);
+            }
+            __syncwarp();
+            next_s[g] = j + 1;
+            progressed = true;
+          }
         }
-        mma_commit(&sh.kv_empty[sk]);
-        mma_commit(&sh.s_full);
-        ok = wait_or_abort(&sh.p_full, j & 1, abort_flag) && wait_or_abort(&sh.kv_full[sv], (rv / kFwKvSlots) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t v0 = smem_u32(kv_ring + sv * kFwKvSlotBytes);
+        // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
+        j = next_pv[g];
+        if (j < ntg[g]) {
+          bool ready = mbar_test_wait(&sh.p_full[g], (uint32_t)j & 1u);
+          if (ready) ready = mbar_test_wait(&sh.kv_full[slot_of(2 * j + 1)], par_of(2 * j + 1));
+          if (__all_sync(0xffffffffu, ready)) {
+            tc_fence_after();
+            const uint32_t v0 = smem_u32(kv_ring + slot_of(2 * j + 1) * kFwKvSlotBytes);
+            if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < 2 * (kFwKeys / 16); ++ks) {  // hi part, then lo part, against the same V tile
-          const uint32_t part = (uint32_t)(ks >> 2), kk = (uint32_t)(ks & 3);
-          mma_ss(tmem_o, smem_desc_sw128(p0 + part * (kTile * 128) + kk * 32u, 16, 1024),
-                 smem_desc_sw128(v0 + kk * 2048u, kFwKvSlotBytes / 2, 1024), idesc_o, j > 0 || ks > 0);
-        }
-        mma_commit(&sh.kv_empty[sv]);
-      }
-      mma_commit(&sh.o_done);
-    }
-  } else {
-    // ---------------- softmax: one thread per query row ----------------
-    const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;
-    const int qi = ib * kTile + row;  // query position inside the sequence
-    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    float m_used = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < nt && ok; ++j) {
-      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full, j & 1, abort_flag));  // collectives below
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t r0[32], r1[32];
-      tmem_ld32(tmem_s + lane_addr, r0);
-      tmem_ld32(tmem_s + lane_addr + 32u, r1);
-      tmem_wait_ld();
-      const int key0 = j * kFwKeys;
-      const bool masked_tile = key0 + kFwKeys - 1 > ib * kTile;  // tile reaches past this block's first query
-      float sc[kFwKeys];
-      float m_tile = -INFINITY;
-#pragma unroll
-      for (int c2 = 0; c2 < kFwKeys; ++c2) {
-        float x = __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]) * scale2;
-        if (masked_tile && key0 + c2 > qi) x = -INFINITY;  // causal: key <= query
-        sc[c2] = x;
-        m_tile = fmaxf(m_tile, x);
-      }
-      const bool need = m_tile > m_used + kRescaleThreshold;
-      if (j == 0) {
-        m_used = m_tile;  // key 0 is visible to every row, so this is finite
-      } else if (__any_sync(0xffffffffu, need)) {
-        // rescale this warp's O rows (the previous P V product has completed: s_full follows it)
-        const float m_new = need ? m_tile : m_used;
-        const float alpha = ex2(m_used - m_new);
-        l *= alpha;
-        m_used = m_new;
-#pragma unroll
-        for (int cc = 0; cc < kD / 32; ++cc) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c2 = 0; c2 < 32; ++c2) o[c2] = __float_as_uint(__uint_as_float(o[c2]) * alpha);
-          tmem_st32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
-        }
-        tmem_wait_st();
-      }
-      // probabilities relative to the reference maximum; bf16 copy for the P V product
-      unsigned char* prow = p_tile + row * 128;
-#pragma unroll
-      for (int c16 = 0; c16 < 8; ++c16) {
-        float pv[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          pv[e] = ex2(sc[c16 * 8 + e] - m_used);
-          l += pv[e];
-        }
-        // P = hi + lo with both parts bf16: the product with V then carries ~16 significant bits
-        uint4 w, wl;
-        uint32_t* wp = &w.x;
-        uint32_t* wlp = &wl.x;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pv[2 * e], pv[2 * e + 1]);
-          const float2 hf = __bfloat1622float2(hi2);
-          wp[e] = *reinterpret_cast<const uint32_t*>(&hi2);
-          wlp[e] = Vec16<__nv_bfloat16>::pack2(pv[2 * e] - hf.x, pv[2 * e + 1] - hf.y);
-        }
-        *reinterpret_cast<uint4*>(prow + ((c16 ^ (row & 7)) << 4)) = w;
-        *reinterpret_cast<uint4*>(prow + kTile * 128 + ((c16 ^ (row & 7)) << 4)) = wl;
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.p_full);
-    }
-    if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.o_done, 0, abort_flag));
-    if (ok) {
-      tc_fence_after();
-      const float inv_l = 1.0f / l;
-      OutT* orow = out + ((int64_t)(lo + qi) * n_heads + h) * kD;
-#pragma unroll
-      for (int cc = 0; cc < kD / 32; ++cc) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + lane_addr + (uint32_t)cc * 32u, o);
-        tmem_wait_ld();
-        if (qi < n) {
-#pragma unroll
-          for (int c8 = 0; c8 < 4; ++c8) {
-            float f[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[c8 * 8 + e]) * inv_l;
-            Vec16<__nv_bfloat16>::store(orow + cc * 32 + c8 * 8, f);
+              for (int ks = 0; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
+                const uint32_t kk = (uint32_t)(ks & 3);
+                mma_ts(tmem + kFwColO + (uint32_t)g * 128u, tmem + kFwColP + (uint32_t)g * 64u + (uint32_t)ks * 8u,
+                       smem_desc_sw128(v0 + kk * 2048u, kFwKvSlotBytes / 2, 1024), idesc_o, j > 0 || ks > 0);
+              }
+              mma_commit(&sh.pv_done[g]);
+              const int other = g ^ 1;
+              if (j >= ntg[other] || next_pv[other] > j) mma_commit(&sh.kv_empty[slot_of(2 * j + 1)]);
+            }
+            __syncwarp();
+            next_pv[g] = j + 1;
+            progressed = true;
           }
         }
       }
-      if (qi < n) s.rowstat[(int64_t)h * s.total_tokens + lo + qi] = make_float2(m_used, inv_l);
+      if (progressed) {
+        idle = 0;
+      } else if (++idle > kFwLoopLimit || ((idle & 1023u) == 0 && *abort_flag)) {
+        *abort_flag = 1;
+        ok = false;
+      }
+    }
+  } else {
+    // ---------------- softmax groups: one thread per query row ----------------
+    const int g = (warp - 2) >> 2;             // 0: group A, 1: group B
+    const int ib = g == 0 ? ibA : ibB;
+    const int ntg = g == 0 ? ntA : ntB;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int qi = ib * kTile + row;           // query position inside the sequence
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tmem_o = tmem + kFwColO + (uint32_t)g * 128u + lane_addr;
+    const uint32_t tmem_s = tmem + kFwColS + (uint32_t)g * 64u + lane_addr;
+    const uint32_t tmem_p = tmem + kFwColP + (uint32_t)g * 64u + lane_addr;
+    bool ok = true;
+    float m_used = -INFINITY, l = 0.f;
+#ifdef H2O_PHASE_TIMERS
+    long long prof_[5] = {0, 0, 0, 0, 0};
+#endif
+    for (int j = 0; j < ntg && ok; ++j) {
+      FWD_CLK(c0_);
+      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[g], j & 1, abort_flag));  // collectives below
+      if (!ok) break;
+      tc_fence_after();
+      FWD_CLK(c1_);
+      uint32_t r0[32], r1[32];
+      tmem_ld32(tmem_s, r0);
+      tmem_ld32(tmem_s + 32u, r1);
+      tmem_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.s_free[g]);  // the next S may be computed while we work on this one
+      FWD_CLK(c2_);
+      const int key0 = j * kFwKeys;
+      const bool masked_tile = key0 + kFwKeys - 1 > ib * kTile;  // tile reaches past this block's first query
+      // raw scores stay unscaled: the scale is positive, so the maximum commutes with it and the
+      // multiplication is folded into the exponent's fused multiply-add below
+      float m_raw = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < kFwKeys; ++c2) {
+        uint32_t& word = c2 < 32 ? r0[c2] : r1[c2 - 32];
+        if (masked_tile && key0 + c2 > qi) word = 0xff800000u;  // -inf, causal: key <= query
+        m_raw = fmaxf(m_raw, __uint_as_float(word));
+      }
+      const float m_tile = m_raw * scale2;
+      const bool need = m_tile > m_used + kRescaleThreshold;
+      if (j == 0) {
+        m_used = m_tile;  // key 0 is visible to every row, so this is finite
+      } else {
+        const bool rescale = __any_sync(0xffffffffu, need);
+        // O_g must include tile j-1 before it is rescaled, and P_g(j-1) must have been consumed before
+        // it is overwritten below; both are signalled by pv_done (normally long since complete)
+        ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(j - 1) & 1u, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (rescale) {
+          const float m_new = need ? m_tile : m_used;
+          const float alpha = ex2(m_used - m_new);
+          l *= alpha;
+          m_used = m_new;
+#pragma unroll
+          for (int cc = 0; cc < kD / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + (uint32_t)cc * 32u, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c2 = 0; c2 < 32; ++c2) o[c2] = __float_as_uint(__uint_as_float(o[c2]) * alpha);
+            tmem_st32(tmem_o + (uint32_t)cc * 32u, o);
+          }
+          tmem_wait_st();
+        }
+      }
+      const float neg_m = -m_used;
+      FWD_CLK(c3_);
+      // probabilities relative to the reference maximum as bf16 hi (columns 0..31) and bf16 lo
+      // (columns 32..63): column c holds keys 2c and 2c+1
+      uint32_t hw[32], lw[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
+        const float s1 = __uint_as_float(c < 16 ? r0[2 * c + 1] : r1[2 * c - 31]);
+        const float p0 = ex2(fmaf(s0, scale2, neg_m));
+        const float p1 = ex2(fmaf(s1, scale2, neg_m));
+        l += p0 + p1;
+        const __nv_bfloat162 hi2 = __floats2bfloat162_rn(p0, p1);
+        const float2 hf = __bfloat1622float2(hi2);
+        hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
+        lw[c] = Vec16<__nv_bfloat16>::pack2(p0 - hf.x, p1 - hf.y);
+      }
+      tmem_st32(tmem_p, hw);
+      tmem_st32(tmem_p + 32u, lw);
+      tmem_wait_st();
+      FWD_CLK(c4_);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.p_full[g]);
+      FWD_ADD(0, c0_, c1_);
+      FWD_ADD(1, c1_, c2_);
+      FWD_ADD(2, c2_, c3_);
+      FWD_ADD(3, c3_, c4_);
+    }
+#ifdef H2O_PHASE_TIMERS
+    if (lane == 0 && quarter == 0) {
+      for (int i = 0; i < 4; ++i) atomicAdd(&g_fwd_prof[i], (unsigned long long)prof_[i]);
+      atomicAdd(&g_fwd_prof[5], (unsigned long long)ntg);
+    }
+#endif
+    if (ntg > 0) {
+      if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(ntg - 1) & 1u, abort_flag));
+      if (ok) {
+        tc_fence_after();
+        const float inv_l = 1.0f / l;
+        __nv_bfloat16* orow = out + ((int64_t)(lo + qi) * n_heads + h) * kD;
+#pragma unroll
+        for (int cc = 0; cc < kD / 32; ++cc) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + (uint32_t)cc * 32u, o);
+          tmem_wait_ld();
+          if (qi < n) {
+#pragma unroll
+            for (int c8 = 0; c8 < 4; ++c8) {
+              float f[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[c8 * 8 + e]) * inv_l;
+              Vec16<__nv_bfloat16>::store(orow + cc * 32 + c8 * 8, f);
+            }
+          }
+        }
+        if (qi < n) s.rowstat[(int64_t)h * s.total_tokens + lo + qi] = make_float2(m_used, inv_l);
+      }
     }
   }
   tc_fence_before();
@@ -523,23 +625,33 @@ float make_scale2(float c) { return (float)((double)c * kLog2eD); }
 
 }  // namespace
 
+#ifdef H2O_PHASE_TIMERS
+extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
+  if (reset) {
+    unsigned long long z[8] = {};
+    return (int)cudaMemcpyToSymbol(g_fwd_prof, z, sizeof(z));
+  }
+  return (int)cudaMemcpyFromSymbol(host, g_fwd_prof, sizeof(unsigned long long) * 8);
+}
+#endif
+
 cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                           const void* v, void* out, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
   if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
       !make_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
-  const int smem = kTileBytes + kFwKvSlots * kFwKvSlotBytes + 2 * kTile * 128 + 1024;
+  const int smem = 2 * kTileBytes + kFwKvSlots * kFwKvSlotBytes + 1024;
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   const int nb = (max_seqlen + kTile - 1) / kTile;
-  dim3 grid((unsigned)nb, (unsigned)c.units);
-  fwd_tc_kernel<__nv_bfloat16><<<grid, kFwThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
-                                                                  static_cast<__nv_bfloat16*>(out), c.status);
+  dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
+  fwd_tc_kernel<<<grid, kFwThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
+                                                   static_cast<__nv_bfloat16*>(out), c.status);
   return cudaGetLastError();
 }
 
