@@ -478,7 +478,12 @@ cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, boo
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   using C = Cfg<T, D>;
   // ring depth: the whole chunk if it is short, otherwise enough to keep ~64 KB in flight per block
-  const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : kDefaultStages;
+  // Ring depth.  With few blocks (at most two per SM) each block needs a deep ring to keep enough
+  // bytes in flight; with many blocks a shallow ring lets more of them be resident, which hides each
+  // block's serial prologue and epilogue behind the others' streams.
+  const int blocks = c.units * split;
+  const int auto_stages = blocks > 4 * 148 ? 2 : kDefaultStages;
+  const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : auto_stages;
   int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
   stages = stages < 1 ? 1 : (stages > want ? want : stages);
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
