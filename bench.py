@@ -339,11 +339,21 @@ def main():
         h2d = L * 3 * prompts[0][0].numel() * esize + S * L * 3 * wl.batch * H * d * esize
         d2h = L * prompts[0][0].numel() * esize + S * L * (wl.batch * H * d * esize + wl.batch * H * 4)
 
+        # one stream per layer cache for the prompt phase: the device-to-host copy of one layer's output
+        # overlaps the host-to-device copies of the next layer's prompt
+        lstreams = [torch.cuda.Stream(device=dev) for _ in range(L)]
+
         def one_step_host():
+            start = torch.cuda.Event()
+            start.record(stream)
             for l in range(L):
                 q, k, v, o = hp[l]
-                caches[l].reset(stream)
-                caches[l].prefill_select_host(q, k, v, cu, o, stream)
+                lstreams[l].wait_event(start)
+                caches[l].reset(lstreams[l])
+                caches[l].prefill_select_host(q, k, v, cu, o, lstreams[l])
+                done = torch.cuda.Event()
+                done.record(lstreams[l])
+                stream.wait_event(done)
             for s in range(S):
                 for l in range(L):
                     dq, dk, dv, do, de = hd[l]
