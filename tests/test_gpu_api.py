@@ -1,0 +1,150 @@
+"""Behaviour of the C ABI on a device: call order, host-buffer variants, reset, determinism."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from workloads import Workload, make_decode_inputs, make_prompt_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    import paper_2306_14048_b200 as p
+
+    assert torch.cuda.is_available(), "these tests need a CUDA device; there is no CPU fallback"
+    return p
+
+
+WL = Workload("api", 3, 4, 128, "bf16", (260, 97, 513), 6, (16, 8, 20), (16, 8, 20), 1, 909)
+
+
+def _full_run(pkg, wl, host=False, reset_first=False):
+    cache = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    if reset_first:  # dirty the cache with another prompt, then reset it
+        cache.prefill_select(v, q, k, cu, torch.empty_like(q))
+        cache.reset()
+    outs = []
+    if host:
+        hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
+        ho = torch.empty_like(hq).pin_memory()
+        cache.prefill_select_host(hq, hk, hv, cu, ho)
+        torch.cuda.synchronize()
+        outs.append(ho.float().numpy().copy())
+    else:
+        o = torch.empty_like(q)
+        cache.prefill_select(q, k, v, cu, o)
+        outs.append(o.float().cpu().numpy())
+    evs = []
+    for step in range(wl.decode_steps):
+        dq, dk, dv = make_decode_inputs(wl, step, device="cuda")
+        if host:
+            hq, hk, hv = (x.cpu().pin_memory() for x in (dq, dk, dv))
+            ho = torch.empty_like(hq).pin_memory()
+            he = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32).pin_memory()
+            cache.decode_step_host(hq, hk, hv, ho, he)
+            torch.cuda.synchronize()
+            outs.append(ho.float().numpy().copy())
+            evs.append(he.numpy().copy())
+        else:
+            do = torch.empty_like(dq)
+            de = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32, device="cuda")
+            cache.decode_step(dq, dk, dv, do, de)
+            outs.append(do.float().cpu().numpy())
+            evs.append(de.cpu().numpy())
+    state = cache.export()
+    assert cache.status() == 0
+    cache.close()
+    return outs, evs, state
+
+
+def _identical(a, b):
+    for x, y in zip(a[0], b[0]):
+        assert np.array_equal(x, y)
+    for x, y in zip(a[1], b[1]):
+        assert np.array_equal(x, y)
+    for x, y in zip(a[2], b[2]):
+        assert np.array_equal(x, y)
+
+
+def test_two_runs_are_bit_identical(pkg):
+    """No float atomics anywhere on the path: the same inputs give the same bits."""
+    _identical(_full_run(pkg, WL), _full_run(pkg, WL))
+
+
+def test_host_buffer_calls_equal_device_calls(pkg):
+    _identical(_full_run(pkg, WL, host=True), _full_run(pkg, WL))
+
+
+def test_reset_returns_the_cache_to_empty(pkg):
+    _identical(_full_run(pkg, WL, reset_first=True), _full_run(pkg, WL))
+
+
+def test_call_order_and_argument_errors(pkg):
+    wl = WL
+    cache = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    o = torch.empty_like(q)
+    with pytest.raises(pkg.H2OError) as e:  # out aliases an input
+        cache.prefill_select(q, k, v, cu, q)
+    assert e.value.code == pkg.H2O_ERR_INVALID_ARG
+    bad_cu = np.array(cu)
+    bad_cu[1] = 0  # an empty sequence
+    with pytest.raises(pkg.H2OError) as e:
+        cache.prefill_select(q, k, v, bad_cu, o)
+    assert e.value.code == pkg.H2O_ERR_INVALID_ARG
+    cache.prefill_select(q, k, v, cu, o)
+    with pytest.raises(pkg.H2OError) as e:  # only once per cache
+        cache.prefill_select(q, k, v, cu, o)
+    assert e.value.code == pkg.H2O_ERR_STATE
+    dq, dk, dv = make_decode_inputs(wl, 0, device="cuda")
+    cache.decode_step(dq, dk, dv, torch.empty_like(dq), None)  # evicted_pos is optional
+    with pytest.raises(pkg.H2OError) as e:  # and not after decoding has started
+        cache.prefill_select(q, k, v, cu, o)
+    assert e.value.code == pkg.H2O_ERR_STATE
+    # undersized scratch
+    need = pkg.h2o_prefill_scratch_bytes(cache.cfg, int(cu[-1]))
+    cache.reset()
+    small = torch.empty(need // 2 + 256, dtype=torch.uint8, device="cuda")
+    sp = (small.data_ptr() + 255) // 256 * 256
+    rc = pkg.lib.h2o_prefill_select(cache._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                    np.ascontiguousarray(cu, dtype=np.int32).ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                    o.data_ptr(), sp, need // 2, None)
+    assert rc == pkg.H2O_ERR_WORKSPACE
+    assert cache.status() == 0
+    _, _, count, t = cache.export()
+    assert not count.any() and not t.any()  # refused calls launch nothing
+    cache.close()
+
+
+def test_caches_on_different_streams(pkg):
+    """Two caches driven from two streams at once give the same results as one after the other."""
+    wl = WL
+    ref = _full_run(pkg, wl)
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    caches = [pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent) for _ in range(2)]
+    q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    outs = [[], []]
+    torch.cuda.synchronize()
+    for i, (c, st) in enumerate(zip(caches, streams)):
+        o = torch.empty_like(q)
+        c.prefill_select(q, k, v, cu, o, st)
+        outs[i].append(o)
+    ins = [make_decode_inputs(wl, s, device="cuda") for s in range(wl.decode_steps)]
+    torch.cuda.synchronize()
+    for s in range(wl.decode_steps):
+        for i, (c, st) in enumerate(zip(caches, streams)):
+            dq, dk, dv = ins[s]
+            do = torch.empty_like(dq)
+            c.decode_step(dq, dk, dv, do, None, st)
+            outs[i].append(do)
+    torch.cuda.synchronize()
+    for i, c in enumerate(caches):
+        for got, want in zip(outs[i], ref[0]):
+            assert np.array_equal(got.float().cpu().numpy(), want)
+        for x, y in zip(c.export(), ref[2]):
+            assert np.array_equal(x, y)
+        c.close()
