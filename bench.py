@@ -208,6 +208,8 @@ def main():
     ap.add_argument("--config", default="c2_opt6p7b", choices=sorted(CONFIGS))
     ap.add_argument("--layers", type=int, default=8, help="independent layer caches rotated per decode step")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the config's decode step count")
+    ap.add_argument("--batch-limit", type=int, default=0,
+                    help="keep only the first N sequences of the configuration (for small profiler captures)")
     ap.add_argument("--ref-units", type=int, default=4)
     ap.add_argument("--split", type=int, default=0, help="decode thread blocks per unit (0 = library default)")
     ap.add_argument("--stages", type=int, default=0, help="decode ring depth (0 = library default)")
@@ -220,6 +222,10 @@ def main():
     wl = CONFIGS[args.config]
     if args.decode_steps:
         wl = wl.scaled(decode_steps=args.decode_steps)
+    if args.batch_limit and args.batch_limit < wl.batch:
+        n = args.batch_limit
+        wl = wl.scaled(name="%s[:%d]" % (wl.name, n), batch=n, prompt_lens=wl.prompt_lens[:n], heavy=wl.heavy[:n],
+                       recent=wl.recent[:n])
     if args.impl == "reference":
         run_reference(args, wl)
         return
