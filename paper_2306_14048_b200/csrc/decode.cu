@@ -487,11 +487,10 @@ cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, boo
   int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
   stages = stages < 1 ? 1 : (stages > want ? want : stages);
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
-  static bool attr_done = false;  // one flag per template instance; setting it twice is harmless
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
+  static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D>), kMaxDynSmem, &attr_flags);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};

@@ -48,6 +48,19 @@ struct PrefillScratch {
 // Read-only view of a handle's configuration (budget arrays are the handle's own copies).
 const h2o_config_t* cache_config(const h2o_cache_t* cache);
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) is a per-device setting: remember per kernel and
+// device whether it has been raised already.  `flags` is a zero-initialised static of the caller.
+inline cudaError_t ensure_dynamic_smem(const void* func, int bytes, unsigned long long* flags) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (*flags & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) *flags |= bit;
+  return e;
+}
+
 // Launchers (each returns the cudaError_t of its launch).
 // `split` thread blocks (one cluster) share a unit, each owning `chunk` consecutive slots.
 // `stages` is the depth of the shared-memory ring (0 = default).  `quiescent`: nothing this library

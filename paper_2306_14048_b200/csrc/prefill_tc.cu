@@ -642,11 +642,10 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
       !make_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
   const int smem = 2 * kTileBytes + kFwKvSlots * kFwKvSlotBytes + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static unsigned long long attr_flags = 0;
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fwd_tc_kernel), smem, &attr_flags);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   const int nb = (max_seqlen + kTile - 1) / kTile;
   dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
@@ -663,11 +662,10 @@ cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int ma
   if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
     return cudaErrorInvalidValue;
   const int smem = kTileBytes * (1 + kCsQStages) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  static unsigned long long attr_flags = 0;
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(colsum_tc_kernel), smem, &attr_flags);
     if (e != cudaSuccess) return e;
-    attr_done = true;
   }
   const int nb = (max_seqlen + kTile - 1) / kTile;
   dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
