@@ -161,3 +161,12 @@ def test_rotating_caches_early_prefetch_equals_waiting_first(H2OCache):
     for sa, sb in zip(a[2], b[2]):
         for x, y in zip(sa, sb):
             assert np.array_equal(x, y)
+
+
+def test_large_budget_per_unit(H2OCache):
+    """A unit with thousands of slots: forced cluster split with large per-block chunks and deep score rows."""
+    from parity_harness import run_parity
+
+    wl = _wl("bigB", 1, 2, 128, "bf16", [9500], 12, [4600], [4400], seed=61)
+    st = run_parity(wl, H2OCache, export_every=6)
+    print(st)
