@@ -158,8 +158,12 @@ struct Shared {
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kThreads + 32)
+// MINB is the number of blocks per SM the register allocation must leave room for.  A launch with at
+// most two blocks per SM runs fastest with all the registers the compiler wants (MINB 1: no spills, more
+// loads in flight per thread); a launch with many blocks per SM is bound by how many of them are
+// resident to hide one another's serial prologue and epilogue (MINB 4).
+template <typename T, int D, int MINB>
+__global__ void __launch_bounds__(kThreads + 32, MINB)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
               T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
               int cache_is_quiescent) {
@@ -333,14 +337,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       sh.gl[g] = lg;
     }
     consumer_sync();
-#ifdef H2O_EPI_REPS
-    for (int rep_ = 0; rep_ < H2O_EPI_REPS; ++rep_) {  // debug: run the epilogue again to time a warm pass
-    const bool last_rep_ = rep_ == H2O_EPI_REPS - 1;
-    if (!last_rep_) consumer_sync();
-#else
     {
-    const bool last_rep_ = true;
-#endif
     H2O_STAMP(8);
 
     // ---- block statistics, computed by every warp alike (fixed order, same result) -------
@@ -430,7 +427,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
           b = warp_argmin(o2);
         }
       }
-      if (rank == 0 && last_rep_) {  // replace the victim in place (or append while the cache is filling)
+      if (rank == 0) {  // replace the victim in place (or append while the cache is filling)
         int slot, ev;
         if (!full) {
           slot = cnt;
@@ -473,8 +470,8 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   H2O_STAMP(6);
 }
 
-template <typename T, int D>
-cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
+template <typename T, int D, int MINB>
+cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   using C = Cfg<T, D>;
   // ring depth: the whole chunk if it is short, otherwise enough to keep ~64 KB in flight per block
@@ -489,7 +486,7 @@ cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, boo
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
   {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D>), kMaxDynSmem, &attr_flags);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB>), kMaxDynSmem, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
@@ -507,9 +504,17 @@ cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, boo
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D>, c, static_cast<const T*>(q), static_cast<const T*>(k_new),
+  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB>, c, static_cast<const T*>(q), static_cast<const T*>(k_new),
                             static_cast<const T*>(v_new), static_cast<T*>(out), evicted_pos, split, chunk, stages,
                             quiescent ? 1 : 0);
+}
+
+template <typename T, int D>
+cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
+                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  if (c.units * split > 2 * 148)
+    return launch_minb<T, D, 4>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_minb<T, D, 1>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace
