@@ -124,6 +124,24 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
                     int32_t* evicted_pos, void* stream);
 
 /*
+ * n_tokens consecutive decoding steps for every unit in one call: Algorithm 1 applied
+ * token by token (the paper's sequential generation; with an empty cache and the prompt
+ * as input it is the token-by-token eviction of Algorithm 1 over the prompt, the
+ * mechanics of the streaming experiment of Section 5.3).  The result — outputs, cache
+ * contents, accumulated scores, evicted positions — is that of n_tokens calls of
+ * h2o_decode_step on the rows of the inputs in order.
+ * q, k, v, out : dev [n_tokens, batch, n_heads, head_dim] (step-major), 16-byte aligned.
+ * evicted_pos  : dev [n_tokens, batch, n_heads] int32 or NULL.
+ * n_tokens     : >= 1.
+ * For bf16, head_dim 128 and budgets with max_s(k_s + r_s) + 32 <= 512 the steps run 32
+ * at a time inside one kernel (scores and outputs on the tensor cores, the sequential
+ * part in registers); every other configuration is served by one decode-step kernel per
+ * token.  Both are asynchronous on `stream`.
+ */
+int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const void* v, int32_t n_tokens,
+                     void* out, int32_t* evicted_pos, void* stream);
+
+/*
  * h2o_prefill_select for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a deployment convenience).  Some hosts of this library may not call
  * cudaMalloc at all: a plugin inside a serving process whose memory pool is owned by someone
@@ -210,6 +228,8 @@ int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages
  *   once the stream has finished the call.
  */
 int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
+/* h2o_decode_chunk: 0 = automatic (chunk kernel where it applies), 1 = one decode-step kernel per token. */
+int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path);
 /*
  * Process-wide diagnostic switch (no counterpart in the paper).  A decode kernel launched right
  * after a decode / prefill / reset of a DIFFERENT cache on the same stream starts copying its own

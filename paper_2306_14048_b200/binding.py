@@ -85,6 +85,10 @@ def _load() -> ctypes.CDLL:
     lib.h2o_decode_step.restype = c.c_int
     lib.h2o_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.h2o_cache_reset.restype = c.c_int
+    lib.h2o_decode_chunk.argtypes = [vp, vp, vp, vp, c.c_int32, vp, vp, vp]
+    lib.h2o_decode_chunk.restype = c.c_int
+    lib.h2o_cache_set_chunk_path.argtypes = [vp, c.c_int32]
+    lib.h2o_cache_set_chunk_path.restype = c.c_int
     lib.h2o_cache_reset.argtypes = [vp, vp]
     lib.h2o_host_staging_bytes.restype = c.c_size_t
     lib.h2o_host_staging_bytes.argtypes = [cfgp, c.c_int64]
@@ -194,6 +198,15 @@ class H2OCache:
         _check(lib.h2o_decode_step(self._h, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                    None if evicted_pos is None else evicted_pos.data_ptr(), _stream_ptr(stream)),
                "h2o_decode_step")
+
+    def decode_chunk(self, q, k, v, out, evicted_pos=None, stream=None):
+        """h2o_decode_chunk: q, k, v, out are [n_tokens, batch, n_heads, head_dim]; evicted_pos [n_tokens, batch, n_heads]."""
+        _check(lib.h2o_decode_chunk(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), int(q.shape[0]), out.data_ptr(),
+                                    None if evicted_pos is None else evicted_pos.data_ptr(), _stream_ptr(stream)),
+               "h2o_decode_chunk")
+
+    def set_chunk_path(self, path: int):
+        _check(lib.h2o_cache_set_chunk_path(self._h, int(path)), "h2o_cache_set_chunk_path")
 
     def reset(self, stream=None):
         _check(lib.h2o_cache_reset(self._h, _stream_ptr(stream)), "h2o_cache_reset")

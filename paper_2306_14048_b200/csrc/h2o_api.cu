@@ -107,6 +107,7 @@ struct h2o_cache {
   std::vector<h2o::UnitMeta> meta;  // launch order
   int split, chunk, stages;
   int prefill_path;  // 0 = automatic, 1 = force the ALU kernels
+  int chunk_path;    // 0 = automatic, 1 = force one decode-step kernel per token in h2o_decode_chunk
   Layout layout;
   h2o::CacheView view;
   Phase phase;
@@ -235,6 +236,7 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
   c->split = split;
   c->stages = 0;
   c->prefill_path = 0;
+  c->chunk_path = 0;
   c->chunk = (((L.max_B + split - 1) / split) + 3) & ~3;
 
   char* ws = static_cast<char*>(dev_workspace);
@@ -338,6 +340,43 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
     return H2O_ERR_CUDA;
   }
   cache->phase = Phase::Decoding;
+  return H2O_OK;
+}
+
+int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const void* v, int32_t n_tokens, void* out,
+                     int32_t* evicted_pos, void* stream) {
+  if (!cache || !q || !k || !v || !out || n_tokens < 1) return H2O_ERR_INVALID_ARG;
+  for (const void* p : {q, k, v, (const void*)out})
+    if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  g_last_writer.note_and_check(st, cache->view.K);
+  cudaError_t e = cudaSuccess;
+  if (cache->chunk_path == 0 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+                                                          cache->layout.total_slots)) {
+    e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, q, k, v, n_tokens, out, evicted_pos, st);
+  } else {
+    const size_t step = (size_t)cache->view.units * cache->cfg.head_dim * elem_size(cache->cfg.dtype);
+    for (int32_t i = 0; i < n_tokens && e == cudaSuccess; ++i) {
+      const size_t off = (size_t)i * step;
+      e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, false,
+                             static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
+                             static_cast<const char*>(v) + off, static_cast<char*>(out) + off,
+                             evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr, st);
+    }
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  cache->phase = Phase::Decoding;
+  return H2O_OK;
+}
+
+int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path) {
+  if (!cache || (path != 0 && path != 1)) return H2O_ERR_INVALID_ARG;
+  cache->chunk_path = path;
   return H2O_OK;
 }
 

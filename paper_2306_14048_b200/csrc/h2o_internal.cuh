@@ -8,6 +8,8 @@
 
 #include "h2o.h"
 
+struct CUtensorMap_st;  // <cuda.h>
+
 namespace h2o {
 
 // Static description of one unit, stored in launch order (largest budget first).
@@ -78,6 +80,14 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
                           const void* v, void* out, cudaStream_t stream);
 cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                              cudaStream_t stream);
+// Tensor map over a [rows][n_heads][128] bf16 array: box = box_rows x 1 head x 64 elements, 128-byte swizzle.
+bool make_tile_map(CUtensorMap_st* map, const void* base, int64_t rows, int n_heads, int box_rows);
+// Up to kDecodeChunkTokens consecutive decode steps per launch (bf16, head_dim 128, small budgets);
+// inputs and outputs are [n_tokens][units][head_dim], evicted_pos [n_tokens][units] (nullable).
+constexpr int kDecodeChunkTokens = 32;
+bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots);
+cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const void* q, const void* k, const void* v,
+                                int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream);
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
                                  const void* v, cudaStream_t stream);
 

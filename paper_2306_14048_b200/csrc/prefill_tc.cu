@@ -606,8 +606,14 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Softmax scale times log2(e), rounded once.  The forward and the column-sum kernel use the same
+// value, so a row's probabilities sum to one exactly as the forward pass normalised them.
+float make_scale2(float c) { return (float)((double)c * kLog2eD); }
+
+}  // namespace
+
 // [total_tokens, n_heads, 128] bf16, box = rows x 1 head x 64 elements (128 bytes), 128-byte swizzle
-bool make_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_heads, int box_rows) {
+bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_heads, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)n_heads, (cuuint64_t)total_tokens};
@@ -618,12 +624,6 @@ bool make_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_he
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-// Softmax scale times log2(e), rounded once.  The forward and the column-sum kernel use the same
-// value, so a row's probabilities sum to one exactly as the forward pass normalised them.
-float make_scale2(float c) { return (float)((double)c * kLog2eD); }
-
-}  // namespace
 
 #ifdef H2O_PHASE_TIMERS
 extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
@@ -638,8 +638,8 @@ extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
 cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                           const void* v, void* out, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
-  if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
-      !make_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
+  if (!make_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
+      !make_tile_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
   const int smem = 2 * kTileBytes + kFwKvSlots * kFwKvSlotBytes + 1024;
   static unsigned long long attr_flags = 0;
@@ -659,7 +659,7 @@ bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 &&
 cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                              cudaStream_t stream) {
   CUtensorMap map_q, map_k;
-  if (!make_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
+  if (!make_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_tile_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
     return cudaErrorInvalidValue;
   const int smem = kTileBytes * (1 + kCsQStages) + 1024;
   static unsigned long long attr_flags = 0;

@@ -77,12 +77,13 @@ def _gather_units(x, cu, units, H):
 
 def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
-               device: str = "cuda", prefill_path: int = 0) -> ParityStats:
+               device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
     (all of them by default) as a batch of single-head sequences, which is exact because units never
-    interact.
+    interact.  With ``chunk`` > 0 the CUDA path advances ``chunk`` tokens per call (h2o_decode_chunk)
+    while the oracle still takes them one decode step at a time.
     """
     stats = ParityStats()
     H, d = wl.n_heads, wl.head_dim
@@ -131,24 +132,38 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     def pick(x):  # [batch, H, d] -> the sampled units as [len(units), 1, d] float32 on the host
         return x.reshape(wl.units, d)[uidx].float().cpu().numpy()[:, None, :]
 
-    for step in range(steps):
-        q, k, v = make_decode_inputs(wl, step, layer=layer, device=device)
-        out = torch.empty_like(q)
-        ev.fill_(-7)
-        gpu.decode_step(q, k, v, out, ev)
-        g_ev = ev.reshape(-1)[uidx].cpu().numpy()
-        g_out = out.reshape(wl.units, d)[uidx].float().cpu().numpy()
-        res = ora.decode_step(pick(q), pick(k), pick(v), hint=g_ev, tie_rel=TIE_REL)
-        for x, u in enumerate(units):
-            st = int(res["status"][x])
-            if st == 2:
-                raise AssertionError("step %d unit %d: evicted %d, oracle %d (gap %.3g)" % (
-                    step, u, g_ev[x], res["evicted"][x], res["gap"][x]))
-            stats.near_ties_decode += st == 1
-        stats.decisions += len(units)
-        stats.max_out_err = max(stats.max_out_err, assert_close(g_out, res["out"], wl.dtype, "decode out step %d" % step))
-        if (step + 1) % export_every == 0 or step == steps - 1:
-            compare_state(gpu, ora, units, wl.dtype, stats, "after step %d" % step)
+    step = 0
+    while step < steps:
+        nt = min(chunk, steps - step) if chunk > 0 else 1
+        qs, ks, vs = zip(*[make_decode_inputs(wl, step + i, layer=layer, device=device) for i in range(nt)])
+        if chunk > 0:
+            q, k, v = (torch.stack(x).contiguous() for x in (qs, ks, vs))  # [nt, batch, H, d]
+            out = torch.empty_like(q)
+            evs = torch.full((nt, wl.batch, H), -7, dtype=torch.int32, device=device)
+            gpu.set_chunk_path(chunk_path)
+            gpu.decode_chunk(q, k, v, out, evs)
+        else:
+            out = torch.empty_like(qs[0])[None]
+            ev.fill_(-7)
+            gpu.decode_step(qs[0], ks[0], vs[0], out[0], ev)
+            evs = ev[None]
+        for i in range(nt):
+            g_ev = evs[i].reshape(-1)[uidx].cpu().numpy()
+            g_out = out[i].reshape(wl.units, d)[uidx].float().cpu().numpy()
+            res = ora.decode_step(pick(qs[i]), pick(ks[i]), pick(vs[i]), hint=g_ev, tie_rel=TIE_REL)
+            for x, u in enumerate(units):
+                st = int(res["status"][x])
+                if st == 2:
+                    raise AssertionError("step %d unit %d: evicted %d, oracle %d (gap %.3g)" % (
+                        step + i, u, g_ev[x], res["evicted"][x], res["gap"][x]))
+                stats.near_ties_decode += st == 1
+            stats.decisions += len(units)
+            stats.max_out_err = max(stats.max_out_err,
+                                    assert_close(g_out, res["out"], wl.dtype, "decode out step %d" % (step + i)))
+        last = step + nt - 1
+        if (last + 1) % export_every < nt or last == steps - 1:
+            compare_state(gpu, ora, units, wl.dtype, stats, "after step %d" % last)
+        step += nt
     assert gpu.status() == 0
     stats.steps = steps
     gpu.close()
