@@ -7,13 +7,17 @@
 //   1. computes S^T = K Q^T for ALL keys in play (the cached entries and the chunk's own keys) on
 //      the tensor cores, accumulators in tensor memory: one TMEM lane = one key, one column = one
 //      token of the chunk;
-//   2. walks the tokens in order with ONE THREAD PER KEY holding that key's scores, its accumulated
-//      score (fp64), position, slot and an alive flag in registers: softmax over the live set, score
-//      accumulation, eviction of the minimum under (score, position) — two block-wide reductions per
-//      token, no global memory traffic;
-//   3. writes the probabilities (bf16 hi + lo, zero for dead or unborn keys) to shared memory and
+//   2. turns them into exponentials relative to a per-token reference maximum (any reference gives
+//      the same softmax), all tokens at once;
+//   3. walks the tokens in order.  Four warps; a thread owns up to four keys (one per 128-key tile:
+//      a warp can only read its own quarter of the TMEM lanes) with their exponentials, accumulated
+//      scores (fp64), positions, slots and alive flags in registers.  Per token ONE exchange between
+//      the warps carries both the eviction candidates of this token and the partial sums of the next
+//      token's normaliser (taken over the set before the eviction; the victim's own term is then
+//      subtracted, or the sum redone if that term is large enough for cancellation to matter);
+//   4. writes the probabilities (bf16 hi + lo, zero for dead or unborn keys) to shared memory and
 //      computes O^T = V^T P^T on the tensor cores;
-//   4. writes the surviving chunk entries into the slots they inherited from their victims.
+//   5. writes the surviving chunk entries into the slots they inherited from their victims.
 // The result equals that of the same number of single decode steps (same set semantics, same order).
 //
 // Paper: Algorithm 1 / Algorithm 2 (token-by-token eviction), Section 4.2 (greedy eviction policy).
@@ -30,46 +34,50 @@ using namespace ptx;
 
 constexpr int kD = 128;
 constexpr int kC = kDecodeChunkTokens;      // tokens per launch
-constexpr int kKeyThreads = 512;            // one thread per key row
-constexpr int kKeyWarps = kKeyThreads / 32;
+constexpr int kKeyWarps = 4;                // one per quarter of the TMEM lanes
+constexpr int kKeyThreads = kKeyWarps * 32;
 constexpr int kThreads = kKeyThreads + 32;  // + control warp (TMA and MMA issue)
 constexpr int kTileRows = 128;
+constexpr int kMaxTiles = 4;                // keys per thread
+constexpr int kMaxKeys = kMaxTiles * kTileRows;
+constexpr int kBatchTiles = 2;              // key / value tiles resident in shared memory at a time
+constexpr int kMaxBatches = kMaxTiles / kBatchTiles;
 constexpr int kHalfBytes = kTileRows * 128;  // 128 rows x 64 bf16
 constexpr int kTileBytes = 2 * kHalfBytes;   // two halves cover head_dim 128
-constexpr int kMaxTiles = kKeyThreads / kTileRows;
 constexpr int kQHalfBytes = kC * 128;
-constexpr int kPBlockBytes = kC * 128;               // 64 keys x kC tokens of bf16
-constexpr int kPBufBytes = (kKeyThreads / 64) * kPBlockBytes;
-constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;    // S^T of key tile m: columns [m * kC, (m + 1) * kC)
-constexpr uint32_t kColO = 128;  // O^T: kC columns
-constexpr int kDynSmem = kMaxTiles * kTileBytes + 2 * kPBufBytes + 2 * kQHalfBytes + 1024;
-static_assert(kMaxTiles * kC <= (int)kColO && kColO + kC <= kTmemCols, "tensor memory columns");
+constexpr int kPBlockBytes = kC * 128;       // 64 keys x kC tokens of bf16
+constexpr uint32_t kColS = 0;                // key tile m: columns [m * kC, (m + 1) * kC); O^T behind the last tile
 
-struct KeyCand {
-  unsigned long long key;  // bit pattern of the accumulated score (>= 0, so it orders like the value)
-  int pos;
-  int slot;
-  int x;  // key index inside the block; -1: none
-  int pad_;
-};
+// Shared memory holds one batch of tiles (keys first, values later), the probabilities of that batch
+// as bf16 hi and lo, and the chunk's queries; tensor memory is sized by the tiles of the largest unit.
+__host__ __device__ constexpr int dyn_smem_bytes(int tiles) {
+  return (tiles < kBatchTiles ? tiles : kBatchTiles) * (kTileBytes + 4 * kPBlockBytes) + 2 * kQHalfBytes + 1024;
+}
+__host__ __device__ constexpr uint32_t tmem_cols(int tiles) { return tiles <= 1 ? 64u : tiles <= 3 ? 128u : 256u; }
 
 struct Shared {
-  uint64_t k_full, k_ready, s_full, v_full, p_ready, o_full;
+  uint64_t k_full[kMaxBatches], k_ready[kMaxBatches], s_done[kMaxBatches];
+  uint64_t v_full[kMaxBatches], p_ready[kMaxBatches], o_done[kMaxBatches];
   uint32_t tmem_base;
   int abort_flag;
   float wmax[kKeyWarps][kC];
   float m_row[kC];
-  float red_sum[2][kKeyWarps];
-  float red_max[kKeyWarps];
-  KeyCand red_cand[2][kKeyWarps];
+  // what each warp posts per token (two buffers, by token parity): its eviction candidate for this
+  // token and its share of the next token's normaliser
+  __align__(16) unsigned long long post_key[2][kKeyWarps];  // bit pattern of the candidate's score (>= 0: orders like the value); ~0: none
+  __align__(16) int post_pos[2][kKeyWarps];                 // INT_MAX: none
+  __align__(16) float post_sum[2][kKeyWarps];               // next row's exponentials over the warp's live keys (before the eviction)
+  int post_slot[2][kKeyWarps];
+  int post_x[2][kKeyWarps];       // candidate's key index inside the block; -1: none
+  float post_enext[2][kKeyWarps]; // the candidate's exponential in the next row
+  float redo[kKeyWarps];
   int evicted[kC];
   int wb_slot[kC];
 };
 
 // Optional cycle stamps of block 0 (compile with -DH2O_PHASE_TIMERS).
 #ifdef H2O_PHASE_TIMERS
-__device__ long long g_chunk_prof[16];
+__device__ long long g_chunk_prof[32];
 #define DC_STAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) g_chunk_prof[i] = clock64(); } while (0)
 #else
 #define DC_STAMP(i) do { } while (0)
@@ -84,6 +92,12 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ void key_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kKeyThreads) : "memory"); }
 
 // Byte offset of 16-byte piece `c16` (0..7) of row `row` inside a 128-byte-swizzled block of 128-byte rows.
@@ -91,52 +105,32 @@ __device__ __forceinline__ uint32_t swz(int row, int c16) {
   return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((c16 ^ (row & 7)) << 4));
 }
 
-// Sum over the 16 per-warp values held by lanes 0..15 (and mirrored in 16..31); same order in every warp.
-__device__ __forceinline__ float sum16(float v) {
-  v += __shfl_xor_sync(0xffffffffu, v, 8);
-  v += __shfl_xor_sync(0xffffffffu, v, 4);
-  v += __shfl_xor_sync(0xffffffffu, v, 2);
-  v += __shfl_xor_sync(0xffffffffu, v, 1);
-  return v;
+// Eviction candidate; "none" is the largest value of the order, so plain comparisons suffice.
+struct Cand {
+  unsigned long long key;
+  int pos, slot, x;
+  float e_next;
+};
+__device__ __forceinline__ bool cand_before(unsigned long long ka, int pa, unsigned long long kb, int pb) {
+  return (ka < kb) | ((ka == kb) & (pa < pb));  // no short-circuit: branch-free
 }
+__device__ __forceinline__ Cand cand_min(const Cand& a, const Cand& b) { return cand_before(b.key, b.pos, a.key, a.pos) ? b : a; }
 
-// Warp-wide minimum under (score, position); every lane gets the winner.
-__device__ __forceinline__ KeyCand warp_argmin(const KeyCand& a) {
-  const bool valid = a.x >= 0;
-  const unsigned long long bits = valid ? a.key : ~0ull;
-  const unsigned hi = (unsigned)(bits >> 32), lo = (unsigned)bits;
-  const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
-  const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
-  const bool tie = valid && hi == mh && lo == ml;
-  const unsigned mp = __reduce_min_sync(0xffffffffu, tie ? (unsigned)a.pos : 0xffffffffu);
-  const unsigned who = __ballot_sync(0xffffffffu, tie && (unsigned)a.pos == mp);
-  KeyCand b;
-  b.key = ((unsigned long long)mh << 32) | ml;
-  b.pos = (int)mp;
-  b.pad_ = 0;
-  if (who == 0) {
-    b.slot = -1;
-    b.x = -1;
-    return b;
-  }
-  const int src = __ffs(who) - 1;
-  b.slot = __shfl_sync(0xffffffffu, a.slot, src);
-  b.x = __shfl_sync(0xffffffffu, a.x, src);
-  return b;
-}
-
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, CacheView c, const __nv_bfloat16* __restrict__ k_in,
                     const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out,
-                    int32_t* __restrict__ evicted_pos, int tok0, int n_tok) {
+                    int32_t* __restrict__ evicted_pos, int tok0, int n_tok, int tiles_cap) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ Shared sh;
+  const int res_tiles = min(tiles_cap, kBatchTiles);
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
-  unsigned char* kv = dyn;                                   // key tiles, later value tiles
-  unsigned char* p_hi = dyn + kMaxTiles * kTileBytes;        // [8 blocks of 64 keys][kC tokens][128 B]
-  unsigned char* p_lo = p_hi + kPBufBytes;
-  unsigned char* q_s = p_lo + kPBufBytes;                    // [2 halves][kC tokens][128 B]
+  unsigned char* kv = dyn;                                        // one batch of key tiles, later of value tiles
+  unsigned char* p_hi = kv + res_tiles * kTileBytes;              // [2 blocks of 64 keys per tile][kC tokens][128 B]
+  unsigned char* p_lo = p_hi + res_tiles * 2 * kPBlockBytes;
+  unsigned char* q_s = p_lo + res_tiles * 2 * kPBlockBytes;       // [2 halves][kC tokens][128 B]
+  const uint32_t col_o = (uint32_t)(tiles_cap * kC);              // O^T: kC columns behind the scores
+  const uint32_t ncols = tmem_cols(tiles_cap);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int su = blockIdx.x;
@@ -146,7 +140,8 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int ceff = min(kC, n_tok - tok0);
   const int nk = cnt0 + ceff;                          // keys in play: cached entries, then the chunk's own
   const int ntiles = (nk + kTileRows - 1) / kTileRows;
-  if (nk > kKeyThreads || ceff < 1) {                  // the host never launches this; leave before any barrier exists
+  const int nbatch = (ntiles + kBatchTiles - 1) / kBatchTiles;
+  if (ntiles > tiles_cap || ceff < 1) {                // the host never launches this; leave before any barrier exists
     if (tid == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
     return;
   }
@@ -155,16 +150,18 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const __nv_bfloat16* v_u = v_in + ((int64_t)tok0 * c.units + u) * kD;
 
   if (tid == 0) {
-    mbar_init(&sh.k_full, 1);
-    mbar_init(&sh.k_ready, kKeyThreads);
-    mbar_init(&sh.s_full, 1);
-    mbar_init(&sh.v_full, 1);
-    mbar_init(&sh.p_ready, kKeyThreads);
-    mbar_init(&sh.o_full, 1);
+    for (int b = 0; b < kMaxBatches; ++b) {
+      mbar_init(&sh.k_full[b], 1);
+      mbar_init(&sh.k_ready[b], kKeyThreads);
+      mbar_init(&sh.s_done[b], 1);
+      mbar_init(&sh.v_full[b], 1);
+      mbar_init(&sh.p_ready[b], kKeyThreads);
+      mbar_init(&sh.o_done[b], 1);
+    }
     sh.abort_flag = 0;
     fence_barrier_init();
   }
-  if (warp == kKeyWarps) tmem_alloc(&sh.tmem_base, kTmemCols);
+  if (warp == kKeyWarps) tmem_alloc(&sh.tmem_base, ncols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -178,239 +175,376 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      mbar_expect_tx(&sh.k_full, (uint32_t)(ntiles * kTileBytes + 2 * kQHalfBytes));
-      tma_load_3d(q_s, &map_q, 0, u, tok0, &sh.k_full);
-      tma_load_3d(q_s + kQHalfBytes, &map_q, 64, u, tok0, &sh.k_full);
-      for (int m = 0; m < ntiles; ++m) {
-        const int row = (int)mt.slot_off + m * kTileRows;
-        tma_load_3d(kv + m * kTileBytes, &map_k, 0, 0, row, &sh.k_full);
-        tma_load_3d(kv + m * kTileBytes + kHalfBytes, &map_k, 64, 0, row, &sh.k_full);
-      }
     }
-    // S^T = K Q^T once the key threads have put the chunk's own keys behind the cached ones
-    ok = wait_or_abort(&sh.k_ready, 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    if (ok && elect_one()) {
-      constexpr uint32_t idesc_s = instr_desc_f16(kTileRows, kC, kFmtBF16, kFmtBF16, false, false);
-      const uint32_t a0 = smem_u32(kv), b0 = smem_u32(q_s);
-      for (int m = 0; m < ntiles; ++m) {
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t offa = (uint32_t)m * kTileBytes + (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-          const uint32_t offb = (uint32_t)(ks >> 2) * kQHalfBytes + (uint32_t)(ks & 3) * 32u;
-          mma_ss(tmem + kColS + (uint32_t)(m * kC), smem_desc_sw128(a0 + offa, 16, 1024),
-                 smem_desc_sw128(b0 + offb, 16, 1024), idesc_s, ks > 0);
+    // S^T = K Q^T, one batch of key tiles at a time
+    for (int b = 0; b < nbatch; ++b) {
+      const int tb = min(kBatchTiles, ntiles - b * kBatchTiles);
+      if (b > 0) ok = ok && wait_or_abort(&sh.s_done[b - 1], 0, abort_flag);  // the previous batch has been read
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok && lane == 0) {
+        mbar_expect_tx(&sh.k_full[b], (uint32_t)(tb * kTileBytes + (b == 0 ? 2 * kQHalfBytes : 0)));
+        if (b == 0) {
+          tma_load_3d(q_s, &map_q, 0, u, tok0, &sh.k_full[0]);
+          tma_load_3d(q_s + kQHalfBytes, &map_q, 64, u, tok0, &sh.k_full[0]);
+        }
+        for (int ml = 0; ml < tb; ++ml) {
+          const int row = (int)mt.slot_off + (b * kBatchTiles + ml) * kTileRows;
+          tma_load_3d(kv + ml * kTileBytes, &map_k, 0, 0, row, &sh.k_full[b]);
+          tma_load_3d(kv + ml * kTileBytes + kHalfBytes, &map_k, 64, 0, row, &sh.k_full[b]);
         }
       }
-      mma_commit(&sh.s_full);
-    }
-    __syncwarp();
-    // the key tiles are dead once the scores exist: the values take their place
-    ok = ok && wait_or_abort(&sh.s_full, 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok && lane == 0) {
-      mbar_expect_tx(&sh.v_full, (uint32_t)(ntiles * kTileBytes));
-      for (int m = 0; m < ntiles; ++m) {
-        const int row = (int)mt.slot_off + m * kTileRows;
-        tma_load_3d(kv + m * kTileBytes, &map_v, 0, 0, row, &sh.v_full);
-        tma_load_3d(kv + m * kTileBytes + kHalfBytes, &map_v, 64, 0, row, &sh.v_full);
-      }
-    }
-    __syncwarp();
-    // O^T = V^T P^T (hi and lo halves of P) once every token's probabilities are in shared memory
-    ok = ok && wait_or_abort(&sh.p_ready, 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    if (ok && elect_one()) {
-      constexpr uint32_t idesc_o = instr_desc_f16(kD, kC, kFmtBF16, kFmtBF16, true, false);
-      const uint32_t v0 = smem_u32(kv), ph = smem_u32(p_hi), pl = smem_u32(p_lo);
-      bool first = true;
-      for (int kb = 0; kb < 2 * ntiles; ++kb) {
+      // ... once the key threads have put the chunk's own keys behind the cached ones
+      ok = ok && wait_or_abort(&sh.k_ready[b], 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      if (ok && elect_one()) {
+        constexpr uint32_t idesc_s = instr_desc_f16(kTileRows, kC, kFmtBF16, kFmtBF16, false, false);
+        const uint32_t a0 = smem_u32(kv), b0 = smem_u32(q_s);
+        for (int ml = 0; ml < tb; ++ml) {
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint32_t offv = (uint32_t)(kb >> 1) * kTileBytes + (uint32_t)(((kb & 1) * 64 + ks * 16) * 128);
-          const uint32_t offp = (uint32_t)kb * kPBlockBytes + (uint32_t)ks * 32u;
-          const uint64_t da = smem_desc_sw128(v0 + offv, kHalfBytes, 1024);
-          mma_ss(tmem + kColO, da, smem_desc_sw128(ph + offp, 16, 1024), idesc_o, !first);
-          mma_ss(tmem + kColO, da, smem_desc_sw128(pl + offp, 16, 1024), idesc_o, true);
-          first = false;
+          for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t offa = (uint32_t)ml * kTileBytes + (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+            const uint32_t offb = (uint32_t)(ks >> 2) * kQHalfBytes + (uint32_t)(ks & 3) * 32u;
+            mma_ss(tmem + kColS + (uint32_t)((b * kBatchTiles + ml) * kC), smem_desc_sw128(a0 + offa, 16, 1024),
+                   smem_desc_sw128(b0 + offb, 16, 1024), idesc_s, ks > 0);
+          }
+        }
+        mma_commit(&sh.s_done[b]);
+      }
+      __syncwarp();
+    }
+    // the key tiles are dead once the scores exist: the values take their place, batch by batch;
+    // O^T += V^T P^T (hi and lo halves of P) for each batch once its probabilities are staged
+    for (int b = 0; b < nbatch; ++b) {
+      const int tb = min(kBatchTiles, ntiles - b * kBatchTiles);
+      ok = ok && wait_or_abort(b == 0 ? &sh.s_done[nbatch - 1] : &sh.o_done[b - 1], 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok && lane == 0) {
+        mbar_expect_tx(&sh.v_full[b], (uint32_t)(tb * kTileBytes));
+        for (int ml = 0; ml < tb; ++ml) {
+          const int row = (int)mt.slot_off + (b * kBatchTiles + ml) * kTileRows;
+          tma_load_3d(kv + ml * kTileBytes, &map_v, 0, 0, row, &sh.v_full[b]);
+          tma_load_3d(kv + ml * kTileBytes + kHalfBytes, &map_v, 64, 0, row, &sh.v_full[b]);
         }
       }
-      mma_commit(&sh.o_full);
+      ok = ok && wait_or_abort(&sh.p_ready[b], 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      if (ok && elect_one()) {
+        constexpr uint32_t idesc_o = instr_desc_f16(kD, kC, kFmtBF16, kFmtBF16, true, false);
+        const uint32_t v0 = smem_u32(kv), ph = smem_u32(p_hi), pl = smem_u32(p_lo);
+        for (int kb = 0; kb < 2 * tb; ++kb) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint32_t offv = (uint32_t)(kb >> 1) * kTileBytes + (uint32_t)(((kb & 1) * 64 + ks * 16) * 128);
+            const uint32_t offp = (uint32_t)kb * kPBlockBytes + (uint32_t)ks * 32u;
+            const uint64_t da = smem_desc_sw128(v0 + offv, kHalfBytes, 1024);
+            mma_ss(tmem + col_o, da, smem_desc_sw128(ph + offp, 16, 1024), idesc_o, b > 0 || kb > 0 || ks > 0);
+            mma_ss(tmem + col_o, da, smem_desc_sw128(pl + offp, 16, 1024), idesc_o, true);
+          }
+        }
+        mma_commit(&sh.o_done[b]);
+      }
+      __syncwarp();
     }
-    __syncwarp();
   } else {
-    // ---------------- key threads ----------------
-    const int x = tid;  // key index: tile x / 128, TMEM lane x % 128
+    // ---------------- key threads: thread (warp, lane) owns keys 128 m + 32 warp + lane ----------------
+    const int x0 = tid;  // key of tile 0; also this thread's TMEM lane
     bool ok = true;
-    bool alive = x < cnt0;
-    double acc = 0.0;
-    int pos = 0, slot = x;
-    if (alive) {
-      acc = c.acc[mt.slot_off + x];
-      pos = c.pos[mt.slot_off + x];
-    }
-    // the chunk's own key rows go behind the cached ones (row cnt0 + j), in the layout the TMA wrote
-    DC_STAMP(0);
-    ok = wait_or_abort(&sh.k_full, 0, abort_flag);
-    DC_STAMP(1);
-    {
-      const int j = tid >> 4, c16 = tid & 15;
-      if (j < ceff) {
-        const uint4 val = *reinterpret_cast<const uint4*>(k_u + (int64_t)j * in_stride + c16 * 8);
-        const int row = cnt0 + j;
-        unsigned char* dst = kv + (row >> 7) * kTileBytes + (c16 >> 3) * kHalfBytes + swz(row & 127, c16 & 7);
-        *reinterpret_cast<uint4*>(dst) = val;
+    bool alive[kMaxTiles];
+    double acc[kMaxTiles];
+    int pos[kMaxTiles], slot[kMaxTiles], jx[kMaxTiles];
+#pragma unroll
+    for (int m = 0; m < kMaxTiles; ++m) {
+      const int x = m * kTileRows + x0;
+      alive[m] = x < cnt0;
+      acc[m] = 0.0;
+      pos[m] = 0;
+      slot[m] = x;
+      jx[m] = x - cnt0;  // index inside the chunk (if 0 <= jx < ceff)
+      if (alive[m]) {
+        acc[m] = c.acc[mt.slot_off + x];
+        pos[m] = c.pos[mt.slot_off + x];
+      } else if (jx[m] < ceff) {  // one of the chunk's own keys: enters the set at token jx with an empty score
+        pos[m] = t0 + jx[m];
+        slot[m] = -1;
       }
     }
-    fence_proxy_async();
-    mbar_arrive(&sh.k_ready);
+    // rows [cnt0, cnt0 + ceff) of the key / value matrices are the chunk's own: written behind the
+    // cached rows in the layout the TMA produced; rows no key owns are zeroed (values only)
+    auto patch_rows = [&](const __nv_bfloat16* src_u, int b, bool zero_tail) {
+      const int row_lo = b * kBatchTiles * kTileRows, row_hi = row_lo + kBatchTiles * kTileRows;
+      for (int idx = tid; idx < ceff * 16; idx += kKeyThreads) {
+        const int j = idx >> 4, c16 = idx & 15;
+        const int row = cnt0 + j;
+        if (row >= row_lo && row < row_hi) {
+          const uint4 val = *reinterpret_cast<const uint4*>(src_u + (int64_t)j * in_stride + c16 * 8);
+          const int rl = row - row_lo;
+          unsigned char* dst = kv + (rl >> 7) * kTileBytes + (c16 >> 3) * kHalfBytes + swz(rl & 127, c16 & 7);
+          *reinterpret_cast<uint4*>(dst) = val;
+        }
+      }
+      if (zero_tail) {
+        const int z_lo = max(nk, row_lo), z_hi = min(ntiles * kTileRows, row_hi);
+        for (int idx = tid; idx < (z_hi - z_lo) * 16; idx += kKeyThreads) {
+          const int rl = z_lo + (idx >> 4) - row_lo, z16 = idx & 15;
+          unsigned char* dst = kv + (rl >> 7) * kTileBytes + (z16 >> 3) * kHalfBytes + swz(rl & 127, z16 & 7);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    };
+    DC_STAMP(0);
+    for (int b = 0; b < nbatch; ++b) {
+      ok = wait_or_abort(&sh.k_full[b], 0, abort_flag) && ok;
+      patch_rows(k_u, b, false);
+      fence_proxy_async();
+      mbar_arrive(&sh.k_ready[b]);
+    }
+    DC_STAMP(1);
 
-    // this key's raw scores against the chunk's tokens
-    float s[kC];
-#pragma unroll
-    for (int i = 0; i < kC; ++i) s[i] = 0.f;
-    ok = wait_or_abort(&sh.s_full, 0, abort_flag) && ok;
+    // ---- scores -> exponentials, in place in tensor memory ----
+    // Everything that walks the tokens below is a ROLLED loop over tensor-memory columns: straight-line
+    // code that runs once per token would be bound by instruction fetch, not by the arithmetic.
+    ok = wait_or_abort(&sh.s_done[nbatch - 1], 0, abort_flag) && ok;
     ok = __all_sync(0xffffffffu, ok);
     DC_STAMP(2);
     tc_fence_after();
-    if (ok && (warp >> 2) < ntiles) {
-      uint32_t raw[32];
-      tmem_ld32(tmem + kColS + (uint32_t)((warp >> 2) * kC) + ((uint32_t)((warp & 3) * 32) << 16), raw);
-      tmem_wait_ld();
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    // reference maximum of every token's row: over all keys of that row, alive or not (any reference
+    // works for a softmax, and this one needs no reduction inside the sequential loop)
+    // Exponentials are taken in the base-2 domain, scores times c log2(e) (rounded once, as in the
+    // prefill kernels): exp2(fma(raw, scale2, -m2)) rounds the difference once, so the absolute error
+    // of an exponential stays near 1e-8 whatever its size.
+    const float scale2 = c.scale * 1.4426950408889634f;
+    if (ok) {
+      float mx[kC];
 #pragma unroll
-      for (int i = 0; i < kC; ++i) s[i] = c.scale * __uint_as_float(raw[i]);
-    }
-    // reference maximum of every token's row: over all keys that exist at that token (alive or not;
-    // any reference works for a softmax, and this one needs no reduction inside the sequential loop)
-    const int jx = x - cnt0;  // index of this key inside the chunk (if >= 0)
-    {
+      for (int i = 0; i < kC; ++i) mx[i] = -INFINITY;
+      for (int m = 0; m < ntiles; ++m) {
+        uint32_t raw[32];
+        tmem_ld32(tmem + kColS + (uint32_t)(m * kC) + lane_base, raw);
+        tmem_wait_ld();
+        const int jxm = m * kTileRows + x0 - cnt0;
+        // a key takes part in token i's row if it is cached or one of the chunk's keys 0..i
+        const int first = jxm < 0 ? 0 : (jxm < ceff ? jxm : kC);
+#pragma unroll
+        for (int i = 0; i < kC; ++i) mx[i] = fmaxf(mx[i], i >= first ? __uint_as_float(raw[i]) : -INFINITY);
+      }
       float mine = -INFINITY;
 #pragma unroll
       for (int i = 0; i < kC; ++i) {
-        const bool valid = x < cnt0 || (jx < ceff && jx <= i);
-        const float v = warp_max(valid ? s[i] : -INFINITY);
+        const float v = warp_max(mx[i]);
         if (lane == i) mine = v;
       }
       sh.wmax[warp][lane] = mine;
-      key_sync();
-      if (tid < kC) {
-        float m = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kKeyWarps; ++w) m = fmaxf(m, sh.wmax[w][tid]);
-        sh.m_row[tid] = m;
-      }
-      key_sync();
     }
-
+    key_sync();
+    if (tid < kC)  // the scale is positive, so the largest scaled score is the scaled largest raw score
+      sh.m_row[tid] = scale2 * fmaxf(fmaxf(sh.wmax[0][tid], sh.wmax[1][tid]), fmaxf(sh.wmax[2][tid], sh.wmax[3][tid]));
+    key_sync();
+    if (ok) {
+      for (int m = 0; m < ntiles; ++m) {
+        uint32_t raw[32];
+        tmem_ld32(tmem + kColS + (uint32_t)(m * kC) + lane_base, raw);
+        tmem_wait_ld();
+        const int jxm = m * kTileRows + x0 - cnt0;
+        const int first = jxm < 0 ? 0 : (jxm < ceff ? jxm : kC);
+#pragma unroll
+        for (int i = 0; i < kC; ++i)
+          raw[i] = __float_as_uint(i >= first ? ex2(fmaf(__uint_as_float(raw[i]), scale2, -sh.m_row[i])) : 0.f);
+        tmem_st32(tmem + kColS + (uint32_t)(m * kC) + lane_base, raw);
+      }
+      tmem_wait_st();
+    }
     DC_STAMP(3);
+
     // ---- the tokens, in order (Algorithm 1) ----
     int live = cnt0;  // entries in the cache before the current token
-    const uint32_t pcol = (uint32_t)((x >> 6) * kPBlockBytes + (x & 7) * 2);
-    const int pc16 = (x & 63) >> 3;
+    // exponentials of this thread's keys in the current token's row and in the next one
+    uint32_t cur[kMaxTiles], nxt[kMaxTiles], nn[kMaxTiles];
 #pragma unroll
-    for (int i = 0; i < kC; ++i) {
-      if (i < ceff) {
-        const int t = t0 + i;
-        const bool is_new = jx == i;
-        if (is_new) {  // the token's own key enters the set with an empty score
-          alive = true;
-          acc = 0.0;
-          pos = t;
-          slot = -1;
+    for (int m = 0; m < kMaxTiles; ++m) {
+      cur[m] = 0u;
+      nxt[m] = 0u;
+      if (ok && m < ntiles) {
+        tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + lane_base, cur[m]);
+        if (ceff > 1) tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + 1u + lane_base, nxt[m]);
+      }
+    }
+    tmem_wait_ld8(cur[0], cur[1], cur[2], cur[3], nxt[0], nxt[1], nxt[2], nxt[3]);
+    float l;
+    {  // normaliser of the first token: nothing has been evicted yet
+      float sm = 0.f;
+#pragma unroll
+      for (int m = 0; m < kMaxTiles; ++m)
+        if (alive[m] || jx[m] == 0) sm += __uint_as_float(cur[m]);
+      sm = warp_sum(sm);
+      if (lane == 0) sh.post_sum[1][warp] = sm;
+      key_sync();
+      const float4 s4 = *reinterpret_cast<const float4*>(sh.post_sum[1]);
+      l = (s4.x + s4.y) + (s4.z + s4.w);
+    }
+#pragma unroll 1
+    for (int i = 0; i < ceff; ++i) {
+#pragma unroll
+      for (int m = 0; m < kMaxTiles; ++m) {  // the row after next, in flight while this token is worked on
+        nn[m] = 0u;
+        if (ok && m < ntiles && i + 2 < ceff) tmem_ld1(tmem + kColS + (uint32_t)(m * kC + i + 2) + lane_base, nn[m]);
+      }
+      const int t = t0 + i, par = i & 1;
+      const float inv_l = __frcp_rn(l);
+      const bool full = live >= B;
+      Cand cm[kMaxTiles];
+      float sm = 0.f;
+#pragma unroll
+      for (int m = 0; m < kMaxTiles; ++m) {
+        alive[m] = alive[m] | (jx[m] == i);  // the token's own key enters the set
+        const float p = alive[m] ? __uint_as_float(cur[m]) * inv_l : 0.f;
+        if (alive[m]) acc[m] += (double)p;  // Algorithm 2: accumulated score
+        // the probability replaces the exponential in tensor memory (zero for dead or unborn keys)
+        if (ok && m < ntiles) tmem_st1(tmem + kColS + (uint32_t)(m * kC + i) + lane_base, __float_as_uint(p));
+        const float en = __uint_as_float(nxt[m]);
+        const bool elig = alive[m] & (pos[m] <= t - r);  // outside the recent window: may be evicted (used when full)
+        cm[m].key = elig ? (unsigned long long)__double_as_longlong(acc[m]) : ~0ull;
+        cm[m].pos = elig ? pos[m] : INT_MAX;
+        cm[m].slot = slot[m];
+        cm[m].x = elig ? m * kTileRows + x0 : -1;
+        cm[m].e_next = en;
+        sm += (alive[m] | (jx[m] == i + 1)) ? en : 0.f;  // next row, over the set before this token's eviction
+      }
+      if (full) {
+        // warp minimum under (score, position) and warp sum, interleaved: two independent chains
+        const Cand cd = cand_min(cand_min(cm[0], cm[1]), cand_min(cm[2], cm[3]));
+        const unsigned hi = (unsigned)(cd.key >> 32), lo = (unsigned)cd.key;
+        const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
+        sm += __shfl_xor_sync(0xffffffffu, sm, 16);
+        const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+        sm += __shfl_xor_sync(0xffffffffu, sm, 8);
+        const bool tie = (cd.x >= 0) & (hi == mh) & (lo == ml);
+        const unsigned mp = __reduce_min_sync(0xffffffffu, tie ? (unsigned)cd.pos : 0xffffffffu);
+        sm += __shfl_xor_sync(0xffffffffu, sm, 4);
+        const unsigned who = __ballot_sync(0xffffffffu, tie & ((unsigned)cd.pos == mp));
+        sm += __shfl_xor_sync(0xffffffffu, sm, 2);
+        sm += __shfl_xor_sync(0xffffffffu, sm, 1);
+        const int src = who ? __ffs(who) - 1 : 0;
+        const int w_slot = __shfl_sync(0xffffffffu, cd.slot, src);
+        const int w_x = __shfl_sync(0xffffffffu, cd.x, src);
+        const float w_en = __shfl_sync(0xffffffffu, cd.e_next, src);
+        if (lane == 0) {
+          sh.post_key[par][warp] = who ? (((unsigned long long)mh << 32) | ml) : ~0ull;
+          sh.post_pos[par][warp] = who ? (int)mp : INT_MAX;
+          sh.post_slot[par][warp] = w_slot;
+          sh.post_x[par][warp] = who ? w_x : -1;
+          sh.post_enext[par][warp] = w_en;
+          sh.post_sum[par][warp] = sm;
         }
-        float e = alive ? expf(s[i] - sh.m_row[i]) : 0.f;
-        {
-          const float ws = warp_sum(e);
-          if (lane == 0) sh.red_sum[i & 1][warp] = ws;
+      } else {
+        sm = warp_sum(sm);
+        if (lane == 0) sh.post_sum[par][warp] = sm;
+      }
+      key_sync();
+      const float4 s4 = *reinterpret_cast<const float4*>(sh.post_sum[par]);
+      const float lsum = (s4.x + s4.y) + (s4.z + s4.w);
+      tmem_wait_ld4(nn[0], nn[1], nn[2], nn[3]);
+      if (full) {
+        const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(&sh.post_key[par][0]);
+        const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(&sh.post_key[par][2]);
+        const int4 p4 = *reinterpret_cast<const int4*>(sh.post_pos[par]);
+        const bool b01 = cand_before(k01.y, p4.y, k01.x, p4.x), b23 = cand_before(k23.y, p4.w, k23.x, p4.z);
+        const unsigned long long ka = b01 ? k01.y : k01.x, kb = b23 ? k23.y : k23.x;
+        const int pa = b01 ? p4.y : p4.x, pb = b23 ? p4.w : p4.z;
+        const int wa = b01 ? 1 : 0, wbi = b23 ? 3 : 2;
+        const bool bb = cand_before(kb, pb, ka, pa);
+        const int wv = bb ? wbi : wa;
+        const int vx = sh.post_x[par][wv];
+        float v_en = 0.f;
+        if (vx >= 0) {
+          const int vslot = sh.post_slot[par][wv];
+          v_en = sh.post_enext[par][wv];
+#pragma unroll
+          for (int m = 0; m < kMaxTiles; ++m) {
+            const bool is_victim = m * kTileRows + x0 == vx;
+            alive[m] = alive[m] & !is_victim;
+            slot[m] = (!is_victim & (jx[m] == i)) ? vslot : slot[m];  // in-place replacement of the victim
+          }
+          if (tid == 0) sh.evicted[i] = bb ? pb : pa;
+        } else {  // a full cache always has a candidate; record instead of corrupting
+#pragma unroll
+          for (int m = 0; m < kMaxTiles; ++m)
+            if (jx[m] == i) alive[m] = false;
+          if (tid == 0) {
+            sh.evicted[i] = -1;
+            atomicCAS(c.status, 0, H2O_ERR_STATE);
+          }
         }
-        key_sync();
-        float l = sum16(sh.red_sum[i & 1][lane & 15]);
-        if (!(l > 1e-30f)) {  // every live score sits far below a dead key's: use the live maximum instead
-          const float wm = warp_max(alive ? s[i] : -INFINITY);
-          if (lane == 0) sh.red_max[warp] = wm;
+        l = lsum - v_en;
+        if (i + 1 < ceff && v_en > 0.25f * lsum) {  // cancellation would cost digits: sum again without the victim
+          float s2 = 0.f;
+#pragma unroll
+          for (int m = 0; m < kMaxTiles; ++m)
+            if (alive[m] || jx[m] == i + 1) s2 += __uint_as_float(nxt[m]);
+          s2 = warp_sum(s2);
+          if (lane == 0) sh.redo[warp] = s2;
           key_sync();
-          float m = sh.red_max[lane & 15];
-          m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
-          m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
-          m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-          m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-          e = alive ? expf(s[i] - m) : 0.f;
-          const float ws = warp_sum(e);
-          key_sync();  // everyone has read red_sum and red_max
-          if (lane == 0) sh.red_sum[i & 1][warp] = ws;
-          key_sync();
-          l = sum16(sh.red_sum[i & 1][lane & 15]);
+          l = (sh.redo[0] + sh.redo[1]) + (sh.redo[2] + sh.redo[3]);
         }
-        const float p = e / l;
-        if (alive) acc += (double)p;  // Algorithm 2: accumulated score
-        {
+      } else {
+#pragma unroll
+        for (int m = 0; m < kMaxTiles; ++m)
+          if (jx[m] == i) slot[m] = live;
+        live += 1;
+        if (tid == 0) sh.evicted[i] = -1;
+        l = lsum;
+      }
+#pragma unroll
+      for (int m = 0; m < kMaxTiles; ++m) {
+        cur[m] = nxt[m];
+        nxt[m] = nn[m];
+      }
+    }
+    tmem_wait_st();
+    DC_STAMP(4);
+
+    // ---- per batch of tiles: probabilities to shared memory as bf16 hi + lo, values patched ----
+    for (int b = 0; b < nbatch; ++b) {
+      const int tb = min(kBatchTiles, ntiles - b * kBatchTiles);
+      if (b > 0) ok = wait_or_abort(&sh.o_done[b - 1], 0, abort_flag) && ok;  // staging and value tiles are free again
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      for (int ml = 0; ml < tb; ++ml) {
+        uint32_t pr[32];
+        if (ok) {
+          tmem_ld32(tmem + kColS + (uint32_t)((b * kBatchTiles + ml) * kC) + lane_base, pr);
+          tmem_wait_ld();
+        }
+        const uint32_t pcol = (uint32_t)((ml * 2 + (x0 >> 6)) * kPBlockBytes + (x0 & 7) * 2);
+        const int pc16 = (x0 & 63) >> 3;
+#pragma unroll
+        for (int i = 0; i < kC; ++i) {
+          const float p = (ok && i < ceff) ? __uint_as_float(pr[i]) : 0.f;
           const __nv_bfloat16 hi = __float2bfloat16_rn(p);
           const __nv_bfloat16 lo = __float2bfloat16_rn(p - __bfloat162float(hi));
           const uint32_t off = pcol + (uint32_t)((i >> 3) * 1024 + (i & 7) * 128 + ((pc16 ^ (i & 7)) << 4));
           *reinterpret_cast<__nv_bfloat16*>(p_hi + off) = hi;
           *reinterpret_cast<__nv_bfloat16*>(p_lo + off) = lo;
         }
-        if (live >= B) {  // full: evict the minimum among the entries outside the recent window
-          KeyCand cd;
-          cd.key = (unsigned long long)__double_as_longlong(acc);
-          cd.pos = pos;
-          cd.slot = slot;
-          cd.x = (alive && pos <= t - r) ? x : -1;
-          cd.pad_ = 0;
-          const KeyCand wb = warp_argmin(cd);
-          if (lane == 0) sh.red_cand[i & 1][warp] = wb;
-          key_sync();
-          const KeyCand vic = warp_argmin(sh.red_cand[i & 1][lane & 15]);
-          if (vic.x >= 0) {
-            if (x == vic.x) alive = false;
-            else if (is_new) slot = vic.slot;  // in-place replacement of the victim
-            if (tid == 0) sh.evicted[i] = vic.pos;
-          } else {  // a full cache always has a candidate; record instead of corrupting
-            if (is_new) alive = false;
-            if (tid == 0) {
-              sh.evicted[i] = -1;
-              atomicCAS(c.status, 0, H2O_ERR_STATE);
-            }
-          }
-        } else {
-          if (is_new) slot = live;
-          live += 1;
-          if (tid == 0) sh.evicted[i] = -1;
-        }
       }
+      ok = wait_or_abort(&sh.v_full[b], 0, abort_flag) && ok;
+      patch_rows(v_u, b, true);
+      fence_proxy_async();
+      mbar_arrive(&sh.p_ready[b]);
     }
-
-    // ---- values: the chunk's own rows behind the cached ones, zeros in the rows no key owns ----
-    DC_STAMP(4);
-    ok = wait_or_abort(&sh.v_full, 0, abort_flag) && ok;
-    DC_STAMP(5);
-    {
-      const int j = tid >> 4, c16 = tid & 15;
-      if (j < ceff) {
-        const uint4 val = *reinterpret_cast<const uint4*>(v_u + (int64_t)j * in_stride + c16 * 8);
-        const int row = cnt0 + j;
-        unsigned char* dst = kv + (row >> 7) * kTileBytes + (c16 >> 3) * kHalfBytes + swz(row & 127, c16 & 7);
-        *reinterpret_cast<uint4*>(dst) = val;
-      }
-      const int nzero = (ntiles * kTileRows - nk) * 16;
-      for (int idx = tid; idx < nzero; idx += kKeyThreads) {
-        const int row = nk + (idx >> 4), z16 = idx & 15;
-        unsigned char* dst = kv + (row >> 7) * kTileBytes + (z16 >> 3) * kHalfBytes + swz(row & 127, z16 & 7);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-    fence_proxy_async();
-    mbar_arrive(&sh.p_ready);
-
     DC_STAMP(6);
+
     // ---- write the state back: scores of the survivors, the chunk's surviving rows into their slots ----
-    if (alive) {
-      c.acc[mt.slot_off + slot] = acc;
-      if (jx >= 0) c.pos[mt.slot_off + slot] = pos;
+#pragma unroll
+    for (int m = 0; m < kMaxTiles; ++m) {
+      if (alive[m]) {
+        c.acc[mt.slot_off + slot[m]] = acc[m];
+        if (jx[m] >= 0) c.pos[mt.slot_off + slot[m]] = pos[m];
+      }
+      if (jx[m] >= 0 && jx[m] < ceff) sh.wb_slot[jx[m]] = alive[m] ? slot[m] : -1;
     }
-    if (jx >= 0 && jx < ceff) sh.wb_slot[jx] = alive ? slot : -1;
     key_sync();
     for (int idx = tid; idx < ceff * 32; idx += kKeyThreads) {
       const int j = idx >> 5, pc = idx & 31, c16 = pc & 15;
@@ -429,20 +563,18 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
     // ---- outputs: lane = head dimension, column = token ----
     DC_STAMP(7);
-    if (warp < 4) {
-      ok = wait_or_abort(&sh.o_full, 0, abort_flag) && ok;
-      DC_STAMP(8);
-      ok = __all_sync(0xffffffffu, ok);
-      tc_fence_after();
-      if (ok) {
-        uint32_t o[32];
-        tmem_ld32(tmem + kColO + ((uint32_t)(warp * 32) << 16), o);
-        tmem_wait_ld();
-        __nv_bfloat16* out_u = out + ((int64_t)tok0 * c.units + u) * kD + tid;
+    ok = wait_or_abort(&sh.o_done[nbatch - 1], 0, abort_flag) && ok;
+    ok = __all_sync(0xffffffffu, ok);
+    DC_STAMP(8);
+    tc_fence_after();
+    if (ok) {
+      uint32_t o[32];
+      tmem_ld32(tmem + col_o + lane_base, o);
+      tmem_wait_ld();
+      __nv_bfloat16* out_u = out + ((int64_t)tok0 * c.units + u) * kD + tid;
 #pragma unroll
-        for (int i = 0; i < kC; ++i)
-          if (i < ceff) out_u[(int64_t)i * in_stride] = __float2bfloat16_rn(__uint_as_float(o[i]));
-      }
+      for (int i = 0; i < kC; ++i)
+        if (i < ceff) out_u[(int64_t)i * in_stride] = __float2bfloat16_rn(__uint_as_float(o[i]));
     }
   }
   DC_STAMP(9);
@@ -452,7 +584,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
   if (warp == kKeyWarps) {
     tc_fence_after();
-    tmem_dealloc(tmem, kTmemCols);
+    tmem_dealloc(tmem, ncols);
   }
 }
 
@@ -460,29 +592,32 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
 #ifdef H2O_PHASE_TIMERS
 extern "C" int h2o_debug_chunk_prof(long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_chunk_prof, sizeof(long long) * 16);
+  return (int)cudaMemcpyFromSymbol(host, g_chunk_prof, sizeof(long long) * 32);
 }
 #endif
 
 bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots) {
-  return prefill_tc_supported(dtype, head_dim) && max_B + kC <= kKeyThreads && total_slots < INT_MAX - kTileRows;
+  return prefill_tc_supported(dtype, head_dim) && max_B + kC <= kMaxKeys && total_slots < INT_MAX - kTileRows;
 }
 
-cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const void* q, const void* k, const void* v,
-                                int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, int max_B, const void* q, const void* k,
+                                const void* v, int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
   if (!make_tile_map(&map_q, q, n_tokens, c.units, kC) || !make_tile_map(&map_k, c.K, total_slots, 1, kTileRows) ||
       !make_tile_map(&map_v, c.V, total_slots, 1, kTileRows))
     return cudaErrorInvalidValue;
+  const int tiles_cap = (max_B + kC + kTileRows - 1) / kTileRows;
+  if (tiles_cap > kMaxTiles) return cudaErrorInvalidValue;
   static unsigned long long attr_flags = 0;
   {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_chunk_kernel), kDynSmem, &attr_flags);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_chunk_kernel), dyn_smem_bytes(kMaxTiles),
+                                        &attr_flags);
     if (e != cudaSuccess) return e;
   }
   for (int tok0 = 0; tok0 < n_tokens; tok0 += kC) {
-    decode_chunk_kernel<<<(unsigned)c.units, kThreads, kDynSmem, stream>>>(
+    decode_chunk_kernel<<<(unsigned)c.units, kThreads, dyn_smem_bytes(tiles_cap), stream>>>(
         map_q, map_k, map_v, c, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
-        static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens);
+        static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens, tiles_cap);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
