@@ -133,7 +133,7 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
  * q, k, v, out : dev [n_tokens, batch, n_heads, head_dim] (step-major), 16-byte aligned.
  * evicted_pos  : dev [n_tokens, batch, n_heads] int32 or NULL.
  * n_tokens     : >= 1.
- * For bf16, head_dim 128 and budgets with max_s(k_s + r_s) + 32 <= 512 the steps run 32
+ * For bf16, head_dim 128 and budgets with max_s(k_s + r_s) + 32 <= 1024 the steps run 32
  * at a time inside one kernel (scores and outputs on the tensor cores, the sequential
  * part in registers); every other configuration is served by one decode-step kernel per
  * token.  Both are asynchronous on `stream`.

@@ -1,4 +1,4 @@
-// Several consecutive decode steps in one launch (bf16, head_dim 128, budget + 32 <= 512 slots).
+// Several consecutive decode steps in one launch (bf16, head_dim 128, budget + 32 <= 1024 slots).
 //
 // Algorithm 1 of the paper runs token by token: token i attends over S_{i-1} and itself, the scores
 // are accumulated, one entry is evicted.  Each eviction depends on every earlier row, so the steps
@@ -9,7 +9,7 @@
 //      token of the chunk;
 //   2. turns them into exponentials relative to a per-token reference maximum (any reference gives
 //      the same softmax), all tokens at once;
-//   3. walks the tokens in order.  Four warps; a thread owns up to four keys (one per 128-key tile:
+//   3. walks the tokens in order.  Four warps; a thread owns up to 2, 4 or 8 keys (one per 128-key tile:
 //      a warp can only read its own quarter of the TMEM lanes) with their exponentials, accumulated
 //      scores (fp64), positions, slots and alive flags in registers.  Per token ONE exchange between
 //      the warps carries both the eviction candidates of this token and the partial sums of the next
@@ -38,10 +38,11 @@ constexpr int kKeyWarps = 4;                // one per quarter of the TMEM lanes
 constexpr int kKeyThreads = kKeyWarps * 32;
 constexpr int kThreads = kKeyThreads + 32;  // + control warp (TMA and MMA issue)
 constexpr int kTileRows = 128;
-constexpr int kMaxTiles = 4;                // keys per thread
+constexpr int kMaxTiles = 8;                // most keys per thread (the kernel is compiled for 2, 4 and 8)
 constexpr int kMaxKeys = kMaxTiles * kTileRows;
-constexpr int kBatchTiles = 2;              // key / value tiles resident in shared memory at a time
-constexpr int kMaxBatches = kMaxTiles / kBatchTiles;
+constexpr int kMaxBatches = 4;
+// key / value tiles resident in shared memory at a time, by keys per thread
+__host__ __device__ constexpr int batch_tiles(int kt) { return kt <= 2 ? 1 : 2; }
 constexpr int kHalfBytes = kTileRows * 128;  // 128 rows x 64 bf16
 constexpr int kTileBytes = 2 * kHalfBytes;   // two halves cover head_dim 128
 constexpr int kQHalfBytes = kC * 128;
@@ -50,10 +51,12 @@ constexpr uint32_t kColS = 0;                // key tile m: columns [m * kC, (m 
 
 // Shared memory holds one batch of tiles (keys first, values later), the probabilities of that batch
 // as bf16 hi and lo, and the chunk's queries; tensor memory is sized by the tiles of the largest unit.
-__host__ __device__ constexpr int dyn_smem_bytes(int tiles) {
-  return (tiles < kBatchTiles ? tiles : kBatchTiles) * (kTileBytes + 4 * kPBlockBytes) + 2 * kQHalfBytes + 1024;
+__host__ __device__ constexpr int dyn_smem_bytes(int kt) {
+  return batch_tiles(kt) * (kTileBytes + 4 * kPBlockBytes) + 2 * kQHalfBytes + 1024;
 }
-__host__ __device__ constexpr uint32_t tmem_cols(int tiles) { return tiles <= 1 ? 64u : tiles <= 3 ? 128u : 256u; }
+__host__ __device__ constexpr uint32_t tmem_cols(int tiles) {
+  return tiles <= 1 ? 64u : tiles <= 3 ? 128u : tiles <= 7 ? 256u : 512u;
+}
 
 struct Shared {
   uint64_t k_full[kMaxBatches], k_ready[kMaxBatches], s_done[kMaxBatches];
@@ -116,14 +119,43 @@ __device__ __forceinline__ bool cand_before(unsigned long long ka, int pa, unsig
 }
 __device__ __forceinline__ Cand cand_min(const Cand& a, const Cand& b) { return cand_before(b.key, b.pos, a.key, a.pos) ? b : a; }
 
-__global__ void __launch_bounds__(kThreads, 2)
+template <int N>
+__device__ __forceinline__ Cand cand_min_of(const Cand (&c)[N]) {  // balanced tree: short dependency chain
+  if constexpr (N == 2) {
+    return cand_min(c[0], c[1]);
+  } else if constexpr (N == 4) {
+    return cand_min(cand_min(c[0], c[1]), cand_min(c[2], c[3]));
+  } else {
+    static_assert(N == 8, "keys per thread");
+    return cand_min(cand_min(cand_min(c[0], c[1]), cand_min(c[2], c[3])),
+                    cand_min(cand_min(c[4], c[5]), cand_min(c[6], c[7])));
+  }
+}
+
+// Wait for the tensor-memory loads in flight; the registers are named so that no use moves above the wait.
+template <int N>
+__device__ __forceinline__ void tmem_wait_ld_regs(uint32_t (&r)[N]) {
+  if constexpr (N == 2) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(r[0]), "+r"(r[1])::"memory");
+  } else if constexpr (N == 4) {
+    tmem_wait_ld4(r[0], r[1], r[2], r[3]);
+  } else {
+    static_assert(N == 8, "keys per thread");
+    tmem_wait_ld8(r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7]);
+  }
+}
+
+// KT = keys per thread = most 128-key tiles a unit of this cache can need.
+template <int KT>
+__global__ void __launch_bounds__(kThreads, KT <= 2 ? 3 : KT <= 4 ? 2 : 1)
 decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, CacheView c, const __nv_bfloat16* __restrict__ k_in,
                     const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out,
                     int32_t* __restrict__ evicted_pos, int tok0, int n_tok, int tiles_cap) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ Shared sh;
-  const int res_tiles = min(tiles_cap, kBatchTiles);
+  constexpr int kBatchTiles = batch_tiles(KT);
+  constexpr int res_tiles = kBatchTiles;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
   unsigned char* kv = dyn;                                        // one batch of key tiles, later of value tiles
   unsigned char* p_hi = kv + res_tiles * kTileBytes;              // [2 blocks of 64 keys per tile][kC tokens][128 B]
@@ -141,7 +173,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const int nk = cnt0 + ceff;                          // keys in play: cached entries, then the chunk's own
   const int ntiles = (nk + kTileRows - 1) / kTileRows;
   const int nbatch = (ntiles + kBatchTiles - 1) / kBatchTiles;
-  if (ntiles > tiles_cap || ceff < 1) {                // the host never launches this; leave before any barrier exists
+  if (ntiles > tiles_cap || tiles_cap > KT || ceff < 1) {                // the host never launches this; leave before any barrier exists
     if (tid == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
     return;
   }
@@ -251,11 +283,11 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ---------------- key threads: thread (warp, lane) owns keys 128 m + 32 warp + lane ----------------
     const int x0 = tid;  // key of tile 0; also this thread's TMEM lane
     bool ok = true;
-    bool alive[kMaxTiles];
-    double acc[kMaxTiles];
-    int pos[kMaxTiles], slot[kMaxTiles], jx[kMaxTiles];
+    bool alive[KT];
+    double acc[KT];
+    int pos[KT], slot[KT], jx[KT];
 #pragma unroll
-    for (int m = 0; m < kMaxTiles; ++m) {
+    for (int m = 0; m < KT; ++m) {
       const int x = m * kTileRows + x0;
       alive[m] = x < cnt0;
       acc[m] = 0.0;
@@ -361,9 +393,9 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ---- the tokens, in order (Algorithm 1) ----
     int live = cnt0;  // entries in the cache before the current token
     // exponentials of this thread's keys in the current token's row and in the next one
-    uint32_t cur[kMaxTiles], nxt[kMaxTiles], nn[kMaxTiles];
+    uint32_t cur[KT], nxt[KT], nn[KT];
 #pragma unroll
-    for (int m = 0; m < kMaxTiles; ++m) {
+    for (int m = 0; m < KT; ++m) {
       cur[m] = 0u;
       nxt[m] = 0u;
       if (ok && m < ntiles) {
@@ -371,12 +403,13 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (ceff > 1) tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + 1u + lane_base, nxt[m]);
       }
     }
-    tmem_wait_ld8(cur[0], cur[1], cur[2], cur[3], nxt[0], nxt[1], nxt[2], nxt[3]);
+    tmem_wait_ld_regs(cur);
+    tmem_wait_ld_regs(nxt);
     float l;
     {  // normaliser of the first token: nothing has been evicted yet
       float sm = 0.f;
 #pragma unroll
-      for (int m = 0; m < kMaxTiles; ++m)
+      for (int m = 0; m < KT; ++m)
         if (alive[m] || jx[m] == 0) sm += __uint_as_float(cur[m]);
       sm = warp_sum(sm);
       if (lane == 0) sh.post_sum[1][warp] = sm;
@@ -387,17 +420,17 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll 1
     for (int i = 0; i < ceff; ++i) {
 #pragma unroll
-      for (int m = 0; m < kMaxTiles; ++m) {  // the row after next, in flight while this token is worked on
+      for (int m = 0; m < KT; ++m) {  // the row after next, in flight while this token is worked on
         nn[m] = 0u;
         if (ok && m < ntiles && i + 2 < ceff) tmem_ld1(tmem + kColS + (uint32_t)(m * kC + i + 2) + lane_base, nn[m]);
       }
       const int t = t0 + i, par = i & 1;
       const float inv_l = __frcp_rn(l);
       const bool full = live >= B;
-      Cand cm[kMaxTiles];
+      Cand cm[KT];
       float sm = 0.f;
 #pragma unroll
-      for (int m = 0; m < kMaxTiles; ++m) {
+      for (int m = 0; m < KT; ++m) {
         alive[m] = alive[m] | (jx[m] == i);  // the token's own key enters the set
         const float p = alive[m] ? __uint_as_float(cur[m]) * inv_l : 0.f;
         if (alive[m]) acc[m] += (double)p;  // Algorithm 2: accumulated score
@@ -414,7 +447,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       }
       if (full) {
         // warp minimum under (score, position) and warp sum, interleaved: two independent chains
-        const Cand cd = cand_min(cand_min(cm[0], cm[1]), cand_min(cm[2], cm[3]));
+        const Cand cd = cand_min_of(cm);
         const unsigned hi = (unsigned)(cd.key >> 32), lo = (unsigned)cd.key;
         const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
         sm += __shfl_xor_sync(0xffffffffu, sm, 16);
@@ -445,7 +478,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       key_sync();
       const float4 s4 = *reinterpret_cast<const float4*>(sh.post_sum[par]);
       const float lsum = (s4.x + s4.y) + (s4.z + s4.w);
-      tmem_wait_ld4(nn[0], nn[1], nn[2], nn[3]);
+      tmem_wait_ld_regs(nn);
       if (full) {
         const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(&sh.post_key[par][0]);
         const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(&sh.post_key[par][2]);
@@ -462,7 +495,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           const int vslot = sh.post_slot[par][wv];
           v_en = sh.post_enext[par][wv];
 #pragma unroll
-          for (int m = 0; m < kMaxTiles; ++m) {
+          for (int m = 0; m < KT; ++m) {
             const bool is_victim = m * kTileRows + x0 == vx;
             alive[m] = alive[m] & !is_victim;
             slot[m] = (!is_victim & (jx[m] == i)) ? vslot : slot[m];  // in-place replacement of the victim
@@ -470,7 +503,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           if (tid == 0) sh.evicted[i] = bb ? pb : pa;
         } else {  // a full cache always has a candidate; record instead of corrupting
 #pragma unroll
-          for (int m = 0; m < kMaxTiles; ++m)
+          for (int m = 0; m < KT; ++m)
             if (jx[m] == i) alive[m] = false;
           if (tid == 0) {
             sh.evicted[i] = -1;
@@ -481,7 +514,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (i + 1 < ceff && v_en > 0.25f * lsum) {  // cancellation would cost digits: sum again without the victim
           float s2 = 0.f;
 #pragma unroll
-          for (int m = 0; m < kMaxTiles; ++m)
+          for (int m = 0; m < KT; ++m)
             if (alive[m] || jx[m] == i + 1) s2 += __uint_as_float(nxt[m]);
           s2 = warp_sum(s2);
           if (lane == 0) sh.redo[warp] = s2;
@@ -490,14 +523,14 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       } else {
 #pragma unroll
-        for (int m = 0; m < kMaxTiles; ++m)
+        for (int m = 0; m < KT; ++m)
           if (jx[m] == i) slot[m] = live;
         live += 1;
         if (tid == 0) sh.evicted[i] = -1;
         l = lsum;
       }
 #pragma unroll
-      for (int m = 0; m < kMaxTiles; ++m) {
+      for (int m = 0; m < KT; ++m) {
         cur[m] = nxt[m];
         nxt[m] = nn[m];
       }
@@ -538,7 +571,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
     // ---- write the state back: scores of the survivors, the chunk's surviving rows into their slots ----
 #pragma unroll
-    for (int m = 0; m < kMaxTiles; ++m) {
+    for (int m = 0; m < KT; ++m) {
       if (alive[m]) {
         c.acc[mt.slot_off + slot[m]] = acc[m];
         if (jx[m] >= 0) c.pos[mt.slot_off + slot[m]] = pos[m];
@@ -600,6 +633,30 @@ bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_sl
   return prefill_tc_supported(dtype, head_dim) && max_B + kC <= kMaxKeys && total_slots < INT_MAX - kTileRows;
 }
 
+namespace {
+
+template <int KT>
+cudaError_t launch_kt(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v, const CacheView& c,
+                      const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos, int tiles_cap,
+                      cudaStream_t stream) {
+  static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_chunk_kernel<KT>), dyn_smem_bytes(KT),
+                                        &attr_flags);
+    if (e != cudaSuccess) return e;
+  }
+  for (int tok0 = 0; tok0 < n_tokens; tok0 += kC) {
+    decode_chunk_kernel<KT><<<(unsigned)c.units, kThreads, dyn_smem_bytes(KT), stream>>>(
+        map_q, map_k, map_v, c, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
+        static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens, tiles_cap);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace
+
 cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, int max_B, const void* q, const void* k,
                                 const void* v, int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
@@ -607,21 +664,10 @@ cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, int max
       !make_tile_map(&map_v, c.V, total_slots, 1, kTileRows))
     return cudaErrorInvalidValue;
   const int tiles_cap = (max_B + kC + kTileRows - 1) / kTileRows;
-  if (tiles_cap > kMaxTiles) return cudaErrorInvalidValue;
-  static unsigned long long attr_flags = 0;
-  {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_chunk_kernel), dyn_smem_bytes(kMaxTiles),
-                                        &attr_flags);
-    if (e != cudaSuccess) return e;
-  }
-  for (int tok0 = 0; tok0 < n_tokens; tok0 += kC) {
-    decode_chunk_kernel<<<(unsigned)c.units, kThreads, dyn_smem_bytes(tiles_cap), stream>>>(
-        map_q, map_k, map_v, c, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
-        static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens, tiles_cap);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
-  return cudaSuccess;
+  if (tiles_cap <= 2) return launch_kt<2>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
+  if (tiles_cap <= 4) return launch_kt<4>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
+  if (tiles_cap <= 8) return launch_kt<8>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace h2o

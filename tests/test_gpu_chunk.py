@@ -57,8 +57,8 @@ def test_chunk_edge_budgets(H2OCache, heavy, recent):
     print(st)
 
 
-def test_chunk_largest_supported_budget_and_peaky_softmax(H2OCache):
-    """Budget 480 (= 512 key threads - 32 tokens): all four key tiles in use; four times the default scale."""
+def test_chunk_four_tiles_and_peaky_softmax(H2OCache):
+    """Budget 480 (four keys per thread, all four key tiles in use); four times the default scale."""
     from parity_harness import run_parity
 
     wl = _wl("chunkmax", 2, 2, 128, "bf16", [700, 600], 64, [240, 200], [240, 200], seed=104)
@@ -66,15 +66,34 @@ def test_chunk_largest_supported_budget_and_peaky_softmax(H2OCache):
     print(st)
 
 
+def test_chunk_largest_supported_budget(H2OCache):
+    """Budget 992 (= 1024 keys - 32 tokens): eight keys per thread, four batches of tiles; the short
+    sequence of the batch uses a single tile of the same kernel."""
+    from parity_harness import run_parity
+
+    wl = _wl("chunk8", 2, 2, 128, "bf16", [1500, 90], 64, [496, 20], [496, 30], seed=107)
+    st = run_parity(wl, H2OCache, chunk=32, export_every=32)
+    print(st)
+
+
+def test_chunk_one_tile_budgets(H2OCache):
+    """Small budgets (two keys per thread, one tile resident at a time), several blocks per SM."""
+    from parity_harness import run_parity
+
+    wl = _wl("chunk2", 6, 8, 128, "bf16", [200, 90, 150, 300, 64, 222], 64, [20, 10, 50, 100, 6, 60], [20, 20, 46, 100, 6, 64], seed=108)
+    st = run_parity(wl, H2OCache, chunk=32, export_every=32)
+    print(st)
+
+
 @pytest.mark.parametrize("dtype,d,heavy,recent", [
     ("f32", 64, [20, 9], [24, 5]),          # no tensor-core path for this dtype
-    ("bf16", 128, [300, 100], [300, 100]),  # budget too large for the chunk kernel
+    ("bf16", 128, [600, 100], [600, 100]),  # budget too large for the chunk kernel
 ])
 def test_chunk_served_by_single_step_kernels(H2OCache, dtype, d, heavy, recent):
     """Configurations outside the chunk kernel's range take one decode-step kernel per token, same results."""
     from parity_harness import run_parity
 
-    wl = _wl("chunkfb", 2, 2, d, dtype, [900, 400], 40, heavy, recent, seed=105)
+    wl = _wl("chunkfb", 2, 2, d, dtype, [1500, 400], 40, heavy, recent, seed=105)
     st = run_parity(wl, H2OCache, chunk=20, export_every=20)
     print(st)
 
@@ -113,9 +132,10 @@ def test_chunk_kernel_and_single_steps_leave_the_same_cache(H2OCache):
     np.testing.assert_allclose(o1, o2, rtol=1e-2, atol=2e-3)
 
 
-@pytest.mark.parametrize("name,units", [("c2_opt6p7b", [0, 77, 255]), ("c3_opt30b", [5, 2000, 3583])])
+@pytest.mark.parametrize("name,units", [("c2_opt6p7b", [0, 77, 255]), ("c3_opt30b", [5, 2000, 3583]),
+                                        ("c5_ragged_32layer", [3, 1234, 4095])])
 def test_chunk_full_size_sampled(H2OCache, name, units):
-    """Configs 2 and 3 at full size: 64 tokens in two chunk launches, sampled units against the oracle."""
+    """Configs 2, 3 and 5 (one layer) at full size: 64 tokens in two chunk launches, sampled units against the oracle."""
     from parity_harness import run_parity
 
     wl = CONFIGS[name]
