@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(kThreads, KT <= 2 ? 3 : KT <= 4 ? 2 : 1)
 decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, CacheView c, const __nv_bfloat16* __restrict__ k_in,
                     const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out,
-                    int32_t* __restrict__ evicted_pos, int tok0, int n_tok, int tiles_cap) {
+                    int32_t* __restrict__ evicted_pos, int tok0, int n_tok, int tiles_cap, int unit_base) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ Shared sh;
   constexpr int kBatchTiles = batch_tiles(KT);
@@ -165,7 +165,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   const uint32_t ncols = tmem_cols(tiles_cap);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int su = blockIdx.x;
+  const int su = unit_base + (int)blockIdx.x;  // launch position of the unit
   const UnitMeta mt = c.meta[su];
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
   const int cnt0 = c.count[su], t0 = c.tpos[su];
@@ -637,37 +637,56 @@ namespace {
 
 template <int KT>
 cudaError_t launch_kt(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v, const CacheView& c,
-                      const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos, int tiles_cap,
-                      cudaStream_t stream) {
+                      const void* k, const void* v, int tok0, int n_tokens, void* out, int32_t* evicted_pos,
+                      int tiles_cap, int unit_base, int n_units, cudaStream_t stream) {
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
   {
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_chunk_kernel<KT>), dyn_smem_bytes(KT),
                                         &attr_flags);
     if (e != cudaSuccess) return e;
   }
-  for (int tok0 = 0; tok0 < n_tokens; tok0 += kC) {
-    decode_chunk_kernel<KT><<<(unsigned)c.units, kThreads, dyn_smem_bytes(KT), stream>>>(
-        map_q, map_k, map_v, c, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
-        static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens, tiles_cap);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
-  return cudaSuccess;
+  decode_chunk_kernel<KT><<<(unsigned)n_units, kThreads, dyn_smem_bytes(KT), stream>>>(
+      map_q, map_k, map_v, c, static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v),
+      static_cast<__nv_bfloat16*>(out), evicted_pos, tok0, n_tokens, tiles_cap, unit_base);
+  return cudaGetLastError();
 }
+
+int tiles_for(int B) { return (B + kC + kTileRows - 1) / kTileRows; }
 
 }  // namespace
 
-cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, int max_B, const void* q, const void* k,
-                                const void* v, int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+// `meta` is the host copy of the unit table, in launch order (largest budget first).  Units are
+// grouped by the keys per thread their budget needs, one grid per group and chunk: a unit with a
+// small budget then neither pays for eight keys per thread nor for one block per SM.
+cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const UnitMeta* meta, const void* q,
+                                const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos,
+                                cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
   if (!make_tile_map(&map_q, q, n_tokens, c.units, kC) || !make_tile_map(&map_k, c.K, total_slots, 1, kTileRows) ||
       !make_tile_map(&map_v, c.V, total_slots, 1, kTileRows))
     return cudaErrorInvalidValue;
-  const int tiles_cap = (max_B + kC + kTileRows - 1) / kTileRows;
-  if (tiles_cap <= 2) return launch_kt<2>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
-  if (tiles_cap <= 4) return launch_kt<4>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
-  if (tiles_cap <= 8) return launch_kt<8>(map_q, map_k, map_v, c, k, v, n_tokens, out, evicted_pos, tiles_cap, stream);
-  return cudaErrorInvalidValue;
+  int n8 = 0, n4 = 0;  // units needing more than 4 tiles, then more than 2
+  for (int su = 0; su < c.units; ++su) {
+    const int t = tiles_for(meta[su].kbud + meta[su].rwin);
+    if (t > kMaxTiles) return cudaErrorInvalidValue;
+    n8 += t > 4;
+    n4 += t > 2 && t <= 4;
+  }
+  const int n2 = c.units - n8 - n4;
+  for (int tok0 = 0; tok0 < n_tokens; tok0 += kC) {
+    cudaError_t e = cudaSuccess;
+    if (n8 > 0)
+      e = launch_kt<8>(map_q, map_k, map_v, c, k, v, tok0, n_tokens, out, evicted_pos,
+                       tiles_for(meta[0].kbud + meta[0].rwin), 0, n8, stream);
+    if (e == cudaSuccess && n4 > 0)
+      e = launch_kt<4>(map_q, map_k, map_v, c, k, v, tok0, n_tokens, out, evicted_pos,
+                       tiles_for(meta[n8].kbud + meta[n8].rwin), n8, n4, stream);
+    if (e == cudaSuccess && n2 > 0)
+      e = launch_kt<2>(map_q, map_k, map_v, c, k, v, tok0, n_tokens, out, evicted_pos,
+                       tiles_for(meta[n8 + n4].kbud + meta[n8 + n4].rwin), n8 + n4, n2, stream);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace h2o

@@ -355,7 +355,7 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   cudaError_t e = cudaSuccess;
   if (cache->chunk_path == 0 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
-    e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->layout.max_B, q, k, v, n_tokens, out,
+    e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
   } else {
     const size_t step = (size_t)cache->view.units * cache->cfg.head_dim * elem_size(cache->cfg.dtype);

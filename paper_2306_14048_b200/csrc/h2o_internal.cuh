@@ -86,8 +86,10 @@ bool make_tile_map(CUtensorMap_st* map, const void* base, int64_t rows, int n_he
 // inputs and outputs are [n_tokens][units][head_dim], evicted_pos [n_tokens][units] (nullable).
 constexpr int kDecodeChunkTokens = 32;
 bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots);
-cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, int max_B, const void* q, const void* k,
-                                const void* v, int n_tokens, void* out, int32_t* evicted_pos, cudaStream_t stream);
+// `meta`: host copy of the unit table in launch order.
+cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const UnitMeta* meta, const void* q,
+                                const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos,
+                                cudaStream_t stream);
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
                                  const void* v, cudaStream_t stream);
 
