@@ -364,6 +364,27 @@ def main():
         torch.cuda.synchronize()
         warm_us = w0.elapsed_time(w1) * 1e3 / n_warm
 
+    # context figure: the same decode steps of layer 0 through h2o_decode_chunk (several tokens per
+    # launch, the token-by-token mode of Algorithm 1), from a freshly prefilled cache
+    chunk_fig = None
+    if rank == 0:
+        n_tok = min(256, S)
+        q, k, v, o = prompts[0]
+        ms = []
+        for _ in range(3):
+            caches[0].reset(stream)
+            caches[0].prefill_select(q, k, v, cu, o, stream)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            caches[0].decode_chunk(dec[0][0][:n_tok], dec[0][1][:n_tok], dec[0][2][:n_tok], dec[0][3][:n_tok],
+                                   dec[0][4][:n_tok], stream)
+            c1.record(stream)
+            torch.cuda.synchronize()
+            ms.append(c0.elapsed_time(c1))
+        assert caches[0].status() == 0, "device status word set"
+        chunk_fig = {"tokens": n_tok, "ms": float(np.median(ms)), "us_per_token_step": float(np.median(ms)) * 1e3 / n_tok,
+                     "seq_heads_per_s": wl.units * n_tok / (float(np.median(ms)) * 1e-3)}
+
     # ---- end to end: pinned host tensors through the host-buffer C calls -----------------
     e2e = None
     if not args.no_e2e:
@@ -437,6 +458,7 @@ def main():
             "prefill_tflops_executed_mma": 2.0 * flops / (prefill_ms * 1e-3) / 1e12,
             "gpu_launches": args.steps * L * (3 + S),
             "decode_one_layer_back_to_back_us": warm_us,
+            "decode_chunk_one_layer": chunk_fig,
             "clocks": clocks,
             "roofline": {
                 "kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
