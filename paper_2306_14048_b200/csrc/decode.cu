@@ -297,8 +297,11 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
           float kf[VEC];
           Vec16<T>::load(kt + row * D + ch * VEC, kf);
           Vec16<T>::load(vt + row * D + ch * VEC, vf[ps]);
+          float2 d2 = make_float2(0.f, 0.f);  // two fp32 FMAs per instruction (packed fp32x2 of this architecture)
 #pragma unroll
-          for (int v = 0; v < VEC; ++v) part = fmaf(qf[v], kf[v], part);
+          for (int v = 0; v < VEC; v += 2)
+            d2 = __ffma2_rn(make_float2(qf[v], qf[v + 1]), make_float2(kf[v], kf[v + 1]), d2);
+          part = d2.x + d2.y;
         } else {
 #pragma unroll
           for (int v = 0; v < VEC; ++v) vf[ps][v] = 0.f;
@@ -315,13 +318,21 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
         const float f = expf(mg - mnew);  // expf(-inf) = 0 for the group's first rows
         lg *= f;
 #pragma unroll
-        for (int v = 0; v < VEC; ++v) o[v] *= f;
+        for (int v = 0; v < VEC; v += 2) {
+          const float2 t2 = __fmul2_rn(make_float2(o[v], o[v + 1]), make_float2(f, f));
+          o[v] = t2.x;
+          o[v + 1] = t2.y;
+        }
 #pragma unroll
         for (int ps = 0; ps < C::PASSES; ++ps) {
           const float e = expf(sc[ps] - mnew);  // 0 for rows past the end
           lg += e;
 #pragma unroll
-          for (int v = 0; v < VEC; ++v) o[v] = fmaf(e, vf[ps][v], o[v]);
+          for (int v = 0; v < VEC; v += 2) {
+            const float2 t2 = __ffma2_rn(make_float2(e, e), make_float2(vf[ps][v], vf[ps][v + 1]), make_float2(o[v], o[v + 1]));
+            o[v] = t2.x;
+            o[v + 1] = t2.y;
+          }
         }
         mg = mnew;
       }

@@ -33,6 +33,7 @@ def _declared_functions():
 def test_library_exports_every_declared_symbol(pkg):
     declared = _declared_functions()
     assert "h2o_cache_create" in declared and "h2o_decode_step" in declared and "h2o_prefill_select" in declared
+    assert "h2o_decode_chunk" in declared
     raw = ctypes.CDLL(pkg.binding.LIB_PATH)
     for name in declared:
         assert hasattr(raw, name), "missing export: " + name
@@ -84,6 +85,8 @@ def test_create_argument_checks_and_no_fallback(pkg):
     for code in range(-7, 1):
         assert pkg.lib.h2o_strerror(code)
     assert pkg.lib.h2o_decode_step(None, None, None, None, None, None, None) == pkg.H2O_ERR_INVALID_ARG
+    assert pkg.lib.h2o_decode_chunk(None, None, None, None, 4, None, None, None) == pkg.H2O_ERR_INVALID_ARG
+    assert pkg.lib.h2o_cache_set_chunk_path(None, 0) == pkg.H2O_ERR_INVALID_ARG
     assert pkg.lib.h2o_prefill_select(None, None, None, None, None, None, None, 0, None) == pkg.H2O_ERR_INVALID_ARG
 
 
