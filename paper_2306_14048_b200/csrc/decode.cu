@@ -151,9 +151,12 @@ struct Shared {
   float red[GROUPS][D];  // per-group partial outputs (unnormalised, relative to the group's maximum)
   float gm[GROUPS], gl[GROUPS];
   Cand wbest[kWarps];
-  float m_c, l_c;      // block statistics, also read by the other blocks of the cluster
-  float x_out[D];      // block partial output relative to m_c (read by rank 0)
-  Cand x_cand;
+  // Cluster exchange: every block PUSHES its values into its peers' shared memory (remote stores are
+  // fire-and-forget, remote loads a round trip), then one cluster barrier makes them visible.
+  float x_m[kMaxSplit], x_l[kMaxSplit];  // block statistics of every rank (written by that rank)
+  Cand x_cand[kMaxSplit];                // rank 0 only: every rank's eviction candidate
+  // (the partial outputs pushed to rank 0, [kMaxSplit][D] floats, live in dynamic shared memory and
+  //  exist only in launches that split a unit, so that unsplit launches keep their blocks per SM)
 };
 
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
@@ -176,12 +179,16 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   double* acc_s = reinterpret_cast<double*>(dyn + (size_t)stages * 2 * kTileBytes);
   int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
   float* p = reinterpret_cast<float*>(pos_s + chunk);
+  float* x_out = p + chunk;  // [kMaxSplit][D], only when split > 1
 
   H2O_STAMP(1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, ch = lane % LPR;
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = split > 1 ? (int)cluster.block_rank() : 0;
+  // Early arrival on the cluster barrier; the matching wait comes right before the first remote
+  // store, by which time every block of the cluster has long started (its shared memory exists).
+  if (split > 1) cluster.barrier_arrive();
   const int su = blockIdx.x / split;  // launch position of the unit
   const UnitMeta mt = c.meta[su];     // static table, written once at create time
   // Programmatic dependent launch: this grid may have been started while the previous kernel of
@@ -264,6 +271,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     __syncwarp();
     if (split > 1) {  // the producer warp only keeps the cluster barriers balanced
+      cluster.barrier_wait();
       cluster.sync();
       cluster.sync();
     }
@@ -369,21 +377,22 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
     part_o = fmaf(w_self, vself, part_o);
     if (split > 1) {
-      if (tid == 0) {
-        sh.m_c = mc;
-        sh.l_c = lc;
+      cluster.barrier_wait();  // every peer is running: its shared memory may be written
+      if (tid < split) {       // my statistics into every block of the cluster (my own included)
+        *cluster.map_shared_rank(&sh.x_m[rank], tid) = mc;
+        *cluster.map_shared_rank(&sh.x_l[rank], tid) = lc;
       }
-      if (tid < D) sh.x_out[tid] = part_o;
+      if (tid < D) *cluster.map_shared_rank(x_out + rank * D + tid, 0) = part_o;
       cluster.sync();
-      const float mr = lane < split ? *cluster.map_shared_rank(&sh.m_c, lane) : -INFINITY;
-      const float lr = lane < split ? *cluster.map_shared_rank(&sh.l_c, lane) : 0.f;
+      const float mr = lane < split ? sh.x_m[lane] : -INFINITY;
+      const float lr = lane < split ? sh.x_l[lane] : 0.f;
       m = warp_max(mr);
       l = warp_sum(mr > -INFINITY ? lr * expf(mr - m) : 0.f);
       if (rank == 0 && tid < D) {
         part_o *= expf(mc - m);
         for (int rk = 1; rk < split; ++rk) {
-          const float mrk = *cluster.map_shared_rank(&sh.m_c, rk);
-          if (mrk > -INFINITY) part_o = fmaf(cluster.map_shared_rank(sh.x_out, rk)[tid], expf(mrk - m), part_o);
+          const float mrk = sh.x_m[rk];
+          if (mrk > -INFINITY) part_o = fmaf(x_out[rk * D + tid], expf(mrk - m), part_o);
         }
       }
     } else {
@@ -429,14 +438,9 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
       H2O_STAMP(7);
       if (split > 1) {
-        if (lane == 0) sh.x_cand = b;
-      }
-      if (split > 1) {
-        cluster.sync();
-        if (rank == 0) {
-          Cand o2 = lane < split ? *cluster.map_shared_rank(&sh.x_cand, lane) : cand_none();
-          b = warp_argmin(o2);
-        }
+        if (lane == 0) *cluster.map_shared_rank(&sh.x_cand[rank], 0) = b;
+        cluster.sync();  // the last cluster barrier: afterwards rank 0 works on its own memory only
+        if (rank == 0) b = warp_argmin(lane < split ? sh.x_cand[lane] : cand_none());
       }
       if (rank == 0) {  // replace the victim in place (or append while the cache is filling)
         int slot, ev;
@@ -477,7 +481,6 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
     }  // epilogue scope
   }
-  if (split > 1) cluster.sync();  // nobody leaves while rank 0 still reads its peers' shared memory
   H2O_STAMP(6);
 }
 
@@ -494,7 +497,8 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : auto_stages;
   int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
   stages = stages < 1 ? 1 : (stages > want ? want : stages);
-  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
+  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16 +
+                      (split > 1 ? (size_t)kMaxSplit * D * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
   {
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB>), kMaxDynSmem, &attr_flags);
