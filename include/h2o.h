@@ -178,6 +178,10 @@ int h2o_prefill_select_static(h2o_cache_t* cache, const void* q, const void* k, 
  *                            (each rounded up to 256 bytes); scratch as above.
  *   h2o_decode_step_host   : staging >= 4 tensors of [batch, n_heads, head_dim] plus
  *                            [batch, n_heads] int32 (each rounded up to 256 bytes).
+ * When every buffer of h2o_decode_step_host is pinned or registered host memory (which the
+ * device can address) and 16-byte aligned, the kernel reads and writes it directly and no
+ * copy is enqueued; the buffers must then not be touched by the host until the stream has
+ * finished the call, and `staging` is unused.
  * h2o_host_staging_bytes(cfg, tokens) gives the size for `tokens` rows per tensor
  * (tokens = total_tokens for prefill, batch for decode); 0 for invalid arguments.
  * No counterpart in the paper; the semantics are those of the device calls.
