@@ -68,7 +68,8 @@ struct CsShared {
   uint64_t ps_full, ps_empty;  // hand-over of the second query half's partial sums
   uint32_t tmem_base;
   int abort_flag;
-  __align__(16) float2 rstat[2][kTile];  // per query of the tile: {minus reference maximum (log2 domain), 1 / row sum}
+  // per query of the tile: -(reference maximum + log2 of the row sum), log2 domain
+  __align__(16) float rstat[2][kTile];
   double psum[kTile];
 };
 
@@ -179,14 +180,16 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = quarter * 32 + lane;     // key row inside the tile = TMEM lane
     const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
     double total_sum = 0.0;
-    auto fetch_nlse = [&](int t) -> float2 {
+    // P[i][j] = 2^(c2 s - m_i) / l_i = 2^(c2 s - (m_i + log2 l_i)): the normaliser is folded into the
+    // exponent's offset, one float per query and no multiplication per score
+    auto fetch_nlse = [&](int t) -> float {
       const int ib = t < t0 ? jb0 + t : jb1 + (t - t0);
       const int qi = ib * kTile + e;
-      if (e >= kTile || qi >= n) return make_float2(-INFINITY, 0.f);  // rows past the end: exp2(-inf) * 0 = 0
+      if (e >= kTile || qi >= n) return -INFINITY;  // rows past the end: exp2(-inf) = 0
       const float2 v2 = rowstat[qi];
-      return make_float2(-v2.x, v2.y);
+      return log2f(v2.y) - v2.x;  // v2 = {m, 1 / l}
     };
-    float2 nl_next = fetch_nlse(0);
+    float nl_next = fetch_nlse(0);
     bool ok = true;
     for (int t = 0; t < total && ok; ++t) {
       const int cb = t < t0 ? 0 : 1;
@@ -203,24 +206,29 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem + (uint32_t)b * kTile + (uint32_t)half * 64u + ((uint32_t)(quarter * 32) << 16);
-      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b][half * 64]);  // {-m, 1/l} of two queries
+      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b][half * 64]);  // four queries per entry
       uint32_t r0[32], r1[32];
       tmem_ld32(taddr, r0);
       tmem_wait_ld();
       tmem_ld32(taddr + 32u, r1);  // in flight while the first 32 columns are processed
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       auto chunk = [&](const uint32_t (&r)[32], int c0, bool masked) {
 #pragma unroll
-        for (int c2 = 0; c2 < 32; c2 += 2) {
-          const float4 st = st4[(c0 + c2) >> 1];
-          float pa = ex2(fmaf(__uint_as_float(r[c2]), scale2, st.x)) * st.y;
-          float pb = ex2(fmaf(__uint_as_float(r[c2 + 1]), scale2, st.z)) * st.w;
+        for (int c4 = 0; c4 < 32; c4 += 4) {
+          const float4 st = st4[(c0 + c4) >> 2];
+          const float2 xa = __ffma2_rn(make_float2(__uint_as_float(r[c4]), __uint_as_float(r[c4 + 1])),
+                                       make_float2(scale2, scale2), make_float2(st.x, st.y));
+          const float2 xb = __ffma2_rn(make_float2(__uint_as_float(r[c4 + 2]), __uint_as_float(r[c4 + 3])),
+                                       make_float2(scale2, scale2), make_float2(st.z, st.w));
+          float2 pa = make_float2(ex2(xa.x), ex2(xa.y)), pb = make_float2(ex2(xb.x), ex2(xb.y));
           if (masked) {  // causal: query >= key (diagonal tile only)
-            const int ql = half * 64 + c0 + c2;
-            if (ql < row) pa = 0.f;
-            if (ql + 1 < row) pb = 0.f;
+            const int ql = half * 64 + c0 + c4;
+            if (ql < row) pa.x = 0.f;
+            if (ql + 1 < row) pa.y = 0.f;
+            if (ql + 2 < row) pb.x = 0.f;
+            if (ql + 3 < row) pb.y = 0.f;
           }
-          sum4[(c2 >> 1) & 3] += pa + pb;
+          sum2[(c4 >> 2) & 3] = __fadd2_rn(sum2[(c4 >> 2) & 3], __fadd2_rn(pa, pb));
         }
       };
       if (ib == jb) {
@@ -235,7 +243,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
-      total_sum += (double)((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
+      total_sum += (double)(((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y)) +
+                            ((sum2[2].x + sum2[2].y) + (sum2[3].x + sum2[3].y)));
       if (t == t0 - 1 || t == total - 1) {  // last tile of this key block: add the two query halves
         if (half == 1) {
           sh.psum[row] = total_sum;
@@ -461,7 +470,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const uint32_t tmem_s = tmem + kFwColS + (uint32_t)g * 64u + lane_addr;
     const uint32_t tmem_p = tmem + kFwColP + (uint32_t)g * 64u + lane_addr;
     bool ok = true;
-    float m_used = -INFINITY, l = 0.f;
+    float m_used = -INFINITY;
+    float2 l2 = make_float2(0.f, 0.f);  // row sum, even and odd keys apart (packed fp32x2 adds)
 #ifdef H2O_PHASE_TIMERS
     long long prof_[5] = {0, 0, 0, 0, 0};
 #endif
@@ -504,7 +514,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         if (rescale) {
           const float m_new = need ? m_tile : m_used;
           const float alpha = ex2(m_used - m_new);
-          l *= alpha;
+          l2 = __fmul2_rn(l2, make_float2(alpha, alpha));
           m_used = m_new;
 #pragma unroll
           for (int cc = 0; cc < kD / 32; ++cc) {
@@ -527,13 +537,13 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       for (int c = 0; c < 32; ++c) {
         const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
         const float s1 = __uint_as_float(c < 16 ? r0[2 * c + 1] : r1[2 * c - 31]);
-        const float p0 = ex2(fmaf(s0, scale2, neg_m));
-        const float p1 = ex2(fmaf(s1, scale2, neg_m));
-        l += p0 + p1;
-        const __nv_bfloat162 hi2 = __floats2bfloat162_rn(p0, p1);
-        const float2 hf = __bfloat1622float2(hi2);
+        const float2 x = __ffma2_rn(make_float2(s0, s1), make_float2(scale2, scale2), make_float2(neg_m, neg_m));
+        const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+        l2 = __fadd2_rn(l2, pp);
+        const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pp.x, pp.y);
+        const float2 lo = __ffma2_rn(__bfloat1622float2(hi2), make_float2(-1.f, -1.f), pp);  // exact remainder
         hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
-        lw[c] = Vec16<__nv_bfloat16>::pack2(p0 - hf.x, p1 - hf.y);
+        lw[c] = Vec16<__nv_bfloat16>::pack2(lo.x, lo.y);
       }
       tmem_st32(tmem_p, hw);
       tmem_st32(tmem_p + 32u, lw);
@@ -557,7 +567,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(ntg - 1) & 1u, abort_flag));
       if (ok) {
         tc_fence_after();
-        const float inv_l = 1.0f / l;
+        const float inv_l = 1.0f / (l2.x + l2.y);
         __nv_bfloat16* orow = out + ((int64_t)(lo + qi) * n_heads + h) * kD;
 #pragma unroll
         for (int cc = 0; cc < kD / 32; ++cc) {
