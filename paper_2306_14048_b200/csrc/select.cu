@@ -8,7 +8,7 @@
 //
 // The k-th largest score is found with a most-significant-digit radix select on the
 // 64-bit pattern of the (non-negative) double scores: 8 passes of 8 bits, one shared
-// histogram per pass.  Everything is integer work after the column sums exist, so
+// histogram per pass, the histogram searched by a block-wide scan.  Everything is integer work after the column sums exist, so
 // the result is exact.
 //
 // Paper: Appendix A pseudocode, prefill branch ("select K heavy hitters and K recent
@@ -93,16 +93,17 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
           if ((key & himask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (tid == 0) {
-          int rem = remaining_sh;  // rank (from the top) still to be located inside this prefix
-          int bin = 255;
-          for (; bin > 0; --bin) {
-            const int cbin = (int)hist[bin];
-            if (cbin >= rem) break;
-            rem -= cbin;
+        {
+          // the bin holding the rank still to be located: scan the histogram from the top bin down, one
+          // bin per thread (thread t owns bin 255 - t), instead of a serial walk by one thread
+          const int rem = remaining_sh;
+          const int mine = (int)hist[255 - tid];
+          int tot_unused;
+          const int above = block_exclusive_scan(mine, warp_tot, tot_unused);  // candidates in higher bins
+          if (above < rem && above + mine >= rem) {  // exactly one thread
+            prefix_sh = prefix | ((uint64_t)(255 - tid) << shift);
+            remaining_sh = rem - above;
           }
-          prefix_sh = prefix | ((uint64_t)bin << shift);
-          remaining_sh = rem;
         }
         __syncthreads();
       }
@@ -149,6 +150,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
     c.acc[s0 + x] = acc0[j];
     c.pos[s0 + x] = j;
   }
+#pragma unroll 4
   for (int x = tid; x < m * LPR; x += kSelThreads) {
     const int slot = x / LPR, ch = x % LPR;
     const int64_t src = base + (int64_t)kept[slot] * stride + ch * VEC;
