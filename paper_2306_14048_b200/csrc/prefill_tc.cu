@@ -30,11 +30,17 @@ constexpr double kLog2eD = 1.4426950408889634074;
 // Optional cycle accounting of the forward kernel's softmax loop (compile with -DH2O_PHASE_TIMERS).
 #ifdef H2O_PHASE_TIMERS
 __device__ unsigned long long g_fwd_prof[8];
+__device__ long long g_fwd_tl[2][40][6];  // block (0, units-1): per group and tile, clock64 at six events
+#define FWD_TL(g, j, e) do { if (tl_on_ && (j) < 40) g_fwd_tl[g][j][e] = clock64(); } while (0)
+__device__ long long g_fwd_w[4][40][3];
+#define FWD_W(q, j, e) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (j) < 40) g_fwd_w[q][j][e] = clock64(); } while (0)
 #define FWD_CLK(v) const long long v = clock64()
 #define FWD_ADD(i, a, b) prof_[i] += (b) - (a)
 #else
 #define FWD_CLK(v) do { } while (0)
 #define FWD_ADD(i, a, b) do { } while (0)
+#define FWD_TL(g, j, e) do { } while (0)
+#define FWD_W(q, j, e) do { } while (0)
 #endif
 
 // ---- abortable waits: the first role that times out raises a flag every other wait observes ----
@@ -309,7 +315,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // The softmax keeps one thread per query row (row max / sum need no shuffles) and updates the
 // reference maximum lazily: O rows in TMEM are rescaled only when the maximum grows by more than
 // 8 in the log2 domain.  One block per SM: all 512 TMEM columns, 161 KB of shared memory.
-constexpr int kFwThreads = 320;                   // warp 0: TMA, warp 1: MMA, warps 2..5: group A, 6..9: group B
+constexpr int kFwThreads = 352;                   // warp 0: TMA, warp 1: MMA of group A, warps 2..5: group A, 6..9: group B, warp 10: MMA of group B
+constexpr int kFwMmaWarpB = 10;
 constexpr int kFwKeys = 64;                       // keys per tile
 constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
 constexpr int kFwKvSlots = 6;                     // K_j, V_j, K_j+1, V_j+1, K_j+2, V_j+2
@@ -342,6 +349,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   unsigned char* kv_ring = dyn + 2 * kTileBytes;      // 6 x 16 KB
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef H2O_PHASE_TIMERS
+  const bool tl_on_ = blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) == 1 || ((threadIdx.x >> 5) & 3) == 2);
+#endif
   const int u = blockIdx.y;
   const int seq = u / n_heads, h = u % n_heads;
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
@@ -366,7 +376,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     }
     for (int i = 0; i < kFwKvSlots; ++i) {
       mbar_init(&sh.kv_full[i], 1);
-      mbar_init(&sh.kv_empty[i], 1);
+      mbar_init(&sh.kv_empty[i], 2);  // one arrival per group
     }
     sh.abort_flag = 0;
     fence_barrier_init();
@@ -401,75 +411,95 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         tma_load_3d(dst + kFwKvSlotBytes / 2, map, 64, h, row0, &sh.kv_full[slot]);
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer: the whole warp runs an event loop, one elected lane issues ----------
+  } else if (warp == 1 || warp == kFwMmaWarpB) {
+    // ---------------- MMA issuers: one warp per softmax group ----------------------------------------
+    // A single thread's instruction stream is what bounds the issue of these small matrix instructions
+    // (a warp needs ~750 cycles per action: barrier tests, eight instructions, commits), so each group
+    // has its own issuing warp; the tensor core takes instructions from both.  The whole warp runs the
+    // loop (warp-uniform descriptors), one elected lane issues.
     constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
     // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
     // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
     constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
-    auto slot_of = [&](int r) { return r % kFwKvSlots; };
-    auto par_of = [&](int r) { return (uint32_t)(r / kFwKvSlots) & 1u; };
-    const int ntg[2] = {ntA, ntB};
-    int next_s[2] = {0, 0};    // next S tile to issue per group
-    int next_pv[2] = {0, 0};   // next P V tile to issue per group
-    bool ok = wait_or_abort(&sh.q_full[0], 0, abort_flag) && (!hasB || wait_or_abort(&sh.q_full[1], 0, abort_flag));
+    const int g = warp == 1 ? 0 : 1;
+    const int ntg = g == 0 ? ntA : ntB;
+    int next_s = 0, next_pv = 0;        // next S tile / next P V tile to issue
+    int s_slot = 0, pv_slot = 1;        // ring slots of K_next_s and V_next_pv (tile j: slots 2 (j % 3), + 1)
+    uint32_t s_par = 0, pv_par = 0;     // their barrier phases
+    bool ok = ntg == 0 || wait_or_abort(&sh.q_full[g], 0, abort_flag);
     ok = __all_sync(0xffffffffu, ok) != 0;
     if (ok) tc_fence_after();
+    const uint32_t q_base = smem_u32(q_tiles + g * kTileBytes);
+    const uint32_t d_s = tmem + kFwColS + (uint32_t)g * 64u;
+    const uint32_t d_o = tmem + kFwColO + (uint32_t)g * 128u, a_p = tmem + kFwColP + (uint32_t)g * 64u;
     uint32_t idle = 0;
-    while (ok && (next_pv[0] < ntg[0] || next_pv[1] < ntg[1])) {
+    while (ok && next_pv < ntg) {
       bool progressed = false;
+      // ---- S_g(j): needs K_j in shared memory and the previous S_g read out by the softmax ----
+      if (next_s < ntg) {
+        const int j = next_s;
+        bool ready = mbar_test_wait(&sh.kv_full[s_slot], s_par);
+        if (ready && j > 0) ready = mbar_test_wait(&sh.s_free[g], (uint32_t)(j - 1) & 1u);
+        if (__all_sync(0xffffffffu, ready)) {
+          tc_fence_after();
+          FWD_TL(g, j, 5);
+          // descriptors once per tile; a K step only moves the start-address field of the low word
+          const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
+          const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + s_slot * kFwKvSlotBytes), 16, 1024);
+          if (elect_one()) {
 #pragma unroll
-      for (int g = 0; g < 2; ++g) {
-        // ---- S_g(j): needs K_j in shared memory and the previous S_g read out by the softmax ----
-        int j = next_s[g];
-        if (j < ntg[g]) {
-          bool ready = mbar_test_wait(&sh.kv_full[slot_of(2 * j)], par_of(2 * j));
-          if (ready && j > 0) ready = mbar_test_wait(&sh.s_free[g], (uint32_t)(j - 1) & 1u);
-          if (__all_sync(0xffffffffu, ready)) {
-            tc_fence_after();
-            const uint32_t q0 = smem_u32(q_tiles + g * kTileBytes);
-            const uint32_t k0 = smem_u32(kv_ring + slot_of(2 * j) * kFwKvSlotBytes);
-            if (elect_one()) {
-#pragma unroll
-              for (int ks = 0; ks < kD / 16; ++ks) {
-                const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
-                const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
-                mma_ss(tmem + kFwColS + (uint32_t)g * 64u, smem_desc_sw128(q0 + qoff, 16, 1024),
-                       smem_desc_sw128(k0 + koff, 16, 1024), idesc_s, ks > 0);
-              }
-              mma_commit(&sh.s_full[g]);
-              // K_j may be refilled once both groups' scores have read it
-              const int other = g ^ 1;
-              if (j >= ntg[other] || next_s[other] > j) mma_commit(&sh.kv_empty[slot_of(2 * j)]);
+            for (int ks = 0; ks < kD / 16; ++ks) {
+              const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+              const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
+              if (ks == 0)
+                mma_ss_lohi<false>(d_s, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
+              else
+                mma_ss_lohi<true>(d_s, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk),
+                                  idesc_s);
             }
-            __syncwarp();
-            next_s[g] = j + 1;
-            progressed = true;
+            mma_commit(&sh.s_full[g]);
+            FWD_TL(g, j, 0);
+            mma_commit(&sh.kv_empty[s_slot]);  // K_j may be refilled once BOTH groups' scores have read it (two arrivals)
           }
+          __syncwarp();
+          next_s = j + 1;
+          s_slot += 2;
+          if (s_slot >= kFwKvSlots) {
+            s_slot -= kFwKvSlots;
+            s_par ^= 1u;
+          }
+          progressed = true;
         }
-        // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
-        j = next_pv[g];
-        if (j < ntg[g]) {
-          bool ready = mbar_test_wait(&sh.p_full[g], (uint32_t)j & 1u);
-          if (ready) ready = mbar_test_wait(&sh.kv_full[slot_of(2 * j + 1)], par_of(2 * j + 1));
-          if (__all_sync(0xffffffffu, ready)) {
-            tc_fence_after();
-            const uint32_t v0 = smem_u32(kv_ring + slot_of(2 * j + 1) * kFwKvSlotBytes);
-            if (elect_one()) {
+      }
+      // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
+      {
+        const int j = next_pv;
+        bool ready = mbar_test_wait(&sh.p_full[g], (uint32_t)j & 1u);
+        if (ready) ready = mbar_test_wait(&sh.kv_full[pv_slot], pv_par);
+        if (__all_sync(0xffffffffu, ready)) {
+          tc_fence_after();
+          FWD_TL(g, j, 2);
+          const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + pv_slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+          if (elect_one()) {
+            if (j == 0) mma_ts_lohi<false>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
+            else mma_ts_lohi<true>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
 #pragma unroll
-              for (int ks = 0; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
-                const uint32_t kk = (uint32_t)(ks & 3);
-                mma_ts(tmem + kFwColO + (uint32_t)g * 128u, tmem + kFwColP + (uint32_t)g * 64u + (uint32_t)ks * 8u,
-                       smem_desc_sw128(v0 + kk * 2048u, kFwKvSlotBytes / 2, 1024), idesc_o, j > 0 || ks > 0);
-              }
-              mma_commit(&sh.pv_done[g]);
-              const int other = g ^ 1;
-              if (j >= ntg[other] || next_pv[other] > j) mma_commit(&sh.kv_empty[slot_of(2 * j + 1)]);
+            for (int ks = 1; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
+              const uint32_t kk = (uint32_t)(ks & 3);
+              mma_ts_lohi<true>(d_o, a_p + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
             }
-            __syncwarp();
-            next_pv[g] = j + 1;
-            progressed = true;
+            mma_commit(&sh.pv_done[g]);
+            FWD_TL(g, j, 4);
+            mma_commit(&sh.kv_empty[pv_slot]);
           }
+          __syncwarp();
+          next_pv = j + 1;
+          pv_slot += 2;
+          if (pv_slot >= kFwKvSlots) {
+            pv_slot -= kFwKvSlots;
+            pv_par ^= 1u;
+          }
+          progressed = true;
         }
       }
       if (progressed) {
@@ -477,6 +507,20 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       } else if (++idle > kFwLoopLimit || ((idle & 1023u) == 0 && *abort_flag)) {
         *abort_flag = 1;
         ok = false;
+      }
+    }
+    // Tiles this group never uses (its query block ends earlier, or it does not exist): the ring still
+    // expects two arrivals per slot, given here as soon as the tile has landed.
+    for (int j = ntg; j < nt && ok; ++j) {
+      ok = wait_or_abort(&sh.kv_full[s_slot], s_par, abort_flag);
+      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[s_slot]);
+      ok = ok && wait_or_abort(&sh.kv_full[s_slot + 1], s_par, abort_flag);
+      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[s_slot + 1]);
+      ok = __all_sync(0xffffffffu, ok) != 0;
+      s_slot += 2;
+      if (s_slot >= kFwKvSlots) {
+        s_slot -= kFwKvSlots;
+        s_par ^= 1u;
       }
     }
   } else {
@@ -503,6 +547,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       FWD_CLK(c1_);
+      FWD_TL(g, j, 1);
+      if (g == 0) FWD_W(quarter, j, 0);
       uint32_t r0[32], r1[32];
       tmem_ld32(tmem_s, r0);
       tmem_ld32(tmem_s + 32u, r1);
@@ -552,6 +598,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       }
       const float neg_m = -m_used;
       FWD_CLK(c3_);
+      if (g == 0) FWD_W(quarter, j, 1);
       // probabilities relative to the reference maximum as bf16 hi (columns 0..31) and bf16 lo
       // (columns 32..63): column c holds keys 2c and 2c+1
       uint32_t hw[32], lw[32];
@@ -571,6 +618,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       tmem_st32(tmem_p + 32u, lw);
       tmem_wait_st();
       FWD_CLK(c4_);
+      FWD_TL(g, j, 3);
+      if (g == 0) FWD_W(quarter, j, 2);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.p_full[g]);
@@ -658,6 +707,12 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int
 }
 
 #ifdef H2O_PHASE_TIMERS
+extern "C" int h2o_debug_fwd_warps(long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_fwd_w, sizeof(long long) * 4 * 40 * 3);
+}
+extern "C" int h2o_debug_fwd_timeline(long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(long long) * 2 * 40 * 6);
+}
 extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
   if (reset) {
     unsigned long long z[8] = {};
