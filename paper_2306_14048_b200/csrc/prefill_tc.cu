@@ -325,7 +325,6 @@ constexpr uint32_t kFwColO = 0;                   // O_g : 128 columns each
 constexpr uint32_t kFwColS = 256;                 // S_g : 64 columns each
 constexpr uint32_t kFwColP = 384;                 // P_g : 64 columns each (hi 0..31, lo 32..63)
 constexpr float kRescaleThreshold = 8.0f;
-constexpr uint32_t kFwLoopLimit = 1u << 26;       // passes of the MMA event loop before it gives up
 
 struct FwShared {
   uint64_t q_full[2];
@@ -414,17 +413,16 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   } else if (warp == 1 || warp == kFwMmaWarpB) {
     // ---------------- MMA issuers: one warp per softmax group ----------------------------------------
     // A single thread's instruction stream is what bounds the issue of these small matrix instructions
-    // (a warp needs ~750 cycles per action: barrier tests, eight instructions, commits), so each group
-    // has its own issuing warp; the tensor core takes instructions from both.  The whole warp runs the
-    // loop (warp-uniform descriptors), one elected lane issues.
+    // (a warp needs several hundred cycles per action: barrier waits, eight instructions, commits), so
+    // each group has its own issuing warp; the tensor core takes instructions from both.  The whole warp
+    // runs the loop (warp-uniform descriptors), one elected lane issues.
     constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
     // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
     // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
     constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
     const int g = warp == 1 ? 0 : 1;
     const int ntg = g == 0 ? ntA : ntB;
-    int next_s = 0, next_pv = 0;        // next S tile / next P V tile to issue
-    int s_slot = 0, pv_slot = 1;        // ring slots of K_next_s and V_next_pv (tile j: slots 2 (j % 3), + 1)
+    int s_slot = 0, pv_slot = 1;        // ring slots of the next K tile / V tile (tile j: slots 2 (j % 3), + 1)
     uint32_t s_par = 0, pv_par = 0;     // their barrier phases
     bool ok = ntg == 0 || wait_or_abort(&sh.q_full[g], 0, abort_flag);
     ok = __all_sync(0xffffffffu, ok) != 0;
@@ -432,81 +430,71 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const uint32_t q_base = smem_u32(q_tiles + g * kTileBytes);
     const uint32_t d_s = tmem + kFwColS + (uint32_t)g * 64u;
     const uint32_t d_o = tmem + kFwColO + (uint32_t)g * 128u, a_p = tmem + kFwColP + (uint32_t)g * 64u;
-    uint32_t idle = 0;
-    while (ok && next_pv < ntg) {
-      bool progressed = false;
-      // ---- S_g(j): needs K_j in shared memory and the previous S_g read out by the softmax ----
-      if (next_s < ntg) {
-        const int j = next_s;
-        bool ready = mbar_test_wait(&sh.kv_full[s_slot], s_par);
-        if (ready && j > 0) ready = mbar_test_wait(&sh.s_free[g], (uint32_t)(j - 1) & 1u);
-        if (__all_sync(0xffffffffu, ready)) {
-          tc_fence_after();
-          FWD_TL(g, j, 5);
-          // descriptors once per tile; a K step only moves the start-address field of the low word
-          const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
-          const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + s_slot * kFwKvSlotBytes), 16, 1024);
-          if (elect_one()) {
+    // S_g(js) = Q_g K_js^T: needs K_js in shared memory (and, checked by the caller, S_g(js-1) read out)
+    auto issue_s = [&](int js) {
+      ok = ok && wait_or_abort(&sh.kv_full[s_slot], s_par, abort_flag);
+      ok = __all_sync(0xffffffffu, ok) != 0;
+      if (!ok) return;
+      tc_fence_after();
+      FWD_TL(g, js, 5);
+      // descriptors once per tile; a K step only moves the start-address field of the low word
+      const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
+      const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + s_slot * kFwKvSlotBytes), 16, 1024);
+      if (elect_one()) {
 #pragma unroll
-            for (int ks = 0; ks < kD / 16; ++ks) {
-              const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
-              const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
-              if (ks == 0)
-                mma_ss_lohi<false>(d_s, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
-              else
-                mma_ss_lohi<true>(d_s, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk),
-                                  idesc_s);
-            }
-            mma_commit(&sh.s_full[g]);
-            FWD_TL(g, j, 0);
-            mma_commit(&sh.kv_empty[s_slot]);  // K_j may be refilled once BOTH groups' scores have read it (two arrivals)
-          }
-          __syncwarp();
-          next_s = j + 1;
-          s_slot += 2;
-          if (s_slot >= kFwKvSlots) {
-            s_slot -= kFwKvSlots;
-            s_par ^= 1u;
-          }
-          progressed = true;
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+          const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
+          if (ks == 0)
+            mma_ss_lohi<false>(d_s, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
+          else
+            mma_ss_lohi<true>(d_s, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk), idesc_s);
         }
+        mma_commit(&sh.s_full[g]);
+        FWD_TL(g, js, 0);
+        mma_commit(&sh.kv_empty[s_slot]);  // K_js may be refilled once BOTH groups' scores have read it (two arrivals)
+      }
+      __syncwarp();
+      s_slot += 2;
+      if (s_slot >= kFwKvSlots) {
+        s_slot -= kFwKvSlots;
+        s_par ^= 1u;
+      }
+    };
+    // Per group the events come in a fixed order — S(j) read out, then P(j) stored — so the warp simply
+    // waits for them in turn (blocking waits: no polling next to the softmax warps of its scheduler).
+    if (ntg > 0) issue_s(0);
+    for (int j = 0; j < ntg && ok; ++j) {
+      if (j + 1 < ntg) {  // S(j+1) runs under the softmax of tile j
+        ok = wait_or_abort(&sh.s_free[g], (uint32_t)j & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok) != 0;
+        issue_s(j + 1);
       }
       // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
-      {
-        const int j = next_pv;
-        bool ready = mbar_test_wait(&sh.p_full[g], (uint32_t)j & 1u);
-        if (ready) ready = mbar_test_wait(&sh.kv_full[pv_slot], pv_par);
-        if (__all_sync(0xffffffffu, ready)) {
-          tc_fence_after();
-          FWD_TL(g, j, 2);
-          const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + pv_slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
-          if (elect_one()) {
-            if (j == 0) mma_ts_lohi<false>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
-            else mma_ts_lohi<true>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
+      ok = ok && wait_or_abort(&sh.p_full[g], (uint32_t)j & 1u, abort_flag);
+      ok = ok && wait_or_abort(&sh.kv_full[pv_slot], pv_par, abort_flag);
+      ok = __all_sync(0xffffffffu, ok) != 0;
+      if (!ok) break;
+      tc_fence_after();
+      FWD_TL(g, j, 2);
+      const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + pv_slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+      if (elect_one()) {
+        if (j == 0) mma_ts_lohi<false>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
+        else mma_ts_lohi<true>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
 #pragma unroll
-            for (int ks = 1; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
-              const uint32_t kk = (uint32_t)(ks & 3);
-              mma_ts_lohi<true>(d_o, a_p + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
-            }
-            mma_commit(&sh.pv_done[g]);
-            FWD_TL(g, j, 4);
-            mma_commit(&sh.kv_empty[pv_slot]);
-          }
-          __syncwarp();
-          next_pv = j + 1;
-          pv_slot += 2;
-          if (pv_slot >= kFwKvSlots) {
-            pv_slot -= kFwKvSlots;
-            pv_par ^= 1u;
-          }
-          progressed = true;
+        for (int ks = 1; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
+          const uint32_t kk = (uint32_t)(ks & 3);
+          mma_ts_lohi<true>(d_o, a_p + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
         }
+        mma_commit(&sh.pv_done[g]);
+        FWD_TL(g, j, 4);
+        mma_commit(&sh.kv_empty[pv_slot]);
       }
-      if (progressed) {
-        idle = 0;
-      } else if (++idle > kFwLoopLimit || ((idle & 1023u) == 0 && *abort_flag)) {
-        *abort_flag = 1;
-        ok = false;
+      __syncwarp();
+      pv_slot += 2;
+      if (pv_slot >= kFwKvSlots) {
+        pv_slot -= kFwKvSlots;
+        pv_par ^= 1u;
       }
     }
     // Tiles this group never uses (its query block ends earlier, or it does not exist): the ring still
