@@ -32,15 +32,12 @@ constexpr double kLog2eD = 1.4426950408889634074;
 __device__ unsigned long long g_fwd_prof[8];
 __device__ long long g_fwd_tl[2][40][6];  // block (0, units-1): per group and tile, clock64 at six events
 #define FWD_TL(g, j, e) do { if (tl_on_ && (j) < 40) g_fwd_tl[g][j][e] = clock64(); } while (0)
-__device__ long long g_fwd_w[4][40][3];
-#define FWD_W(q, j, e) do { if (blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (j) < 40) g_fwd_w[q][j][e] = clock64(); } while (0)
 #define FWD_CLK(v) const long long v = clock64()
 #define FWD_ADD(i, a, b) prof_[i] += (b) - (a)
 #else
 #define FWD_CLK(v) do { } while (0)
 #define FWD_ADD(i, a, b) do { } while (0)
 #define FWD_TL(g, j, e) do { } while (0)
-#define FWD_W(q, j, e) do { } while (0)
 #endif
 
 // ---- abortable waits: the first role that times out raises a flag every other wait observes ----
@@ -51,6 +48,12 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   }
   *abort_flag = 1;
   return false;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 
 __device__ __forceinline__ float ex2(float x) {
@@ -322,17 +325,20 @@ constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B]
 constexpr int kFwKvSlots = 6;                     // K_j, V_j, K_j+1, V_j+1, K_j+2, V_j+2
 constexpr int kFwTmemCols = 512;
 constexpr uint32_t kFwColO = 0;                   // O_g : 128 columns each
-constexpr uint32_t kFwColS = 256;                 // S_g : 64 columns each
-constexpr uint32_t kFwColP = 384;                 // P_g : 64 columns each (hi 0..31, lo 32..63)
+// S and P share two 64-column buffers per group: S_g(j) lands in buffer j % 2, the softmax reads it into
+// registers and writes P_g(j) (bf16 hi in columns 0..31, lo in 32..63) over it, S_g(j+1) meanwhile uses
+// the other buffer.  P is thereby double-buffered: the exponentials of tile j+1 need not wait for P V of tile j.
+constexpr uint32_t kFwColSP = 256;                // group g, buffer b: columns 256 + 128 g + 64 b
 constexpr float kRescaleThreshold = 8.0f;
 
 struct FwShared {
   uint64_t q_full[2];
   uint64_t kv_full[kFwKvSlots], kv_empty[kFwKvSlots];
-  uint64_t s_full[2];   // MMA -> softmax: S_g(j) complete
-  uint64_t s_free[2];   // softmax -> MMA: S_g(j) is in registers, the columns may be overwritten
-  uint64_t p_full[2];   // softmax -> MMA: P_g(j) is in tensor memory
-  uint64_t pv_done[2];  // MMA -> softmax: O_g includes tile j (P_g may be overwritten, O_g may be rescaled)
+  uint64_t s_full[2][2];  // [group][buffer] MMA -> softmax: S_g(j) complete (one barrier per buffer: two S tiles can be ahead)
+  uint64_t p_full[2][2];  // [group][buffer] softmax -> MMA: P_g(j) is in tensor memory
+  uint64_t pv_done[2];    // MMA -> softmax: O_g includes tile j (O_g may be rescaled)
+  uint64_t o_final[2];    // MMA -> softmax: O_g includes the group's last tile (a barrier of its own: the softmax
+                          // does not wait on every phase of pv_done, so a parity wait for the last one could alias)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -368,10 +374,12 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (threadIdx.x == 0) {
     for (int g = 0; g < 2; ++g) {
       mbar_init(&sh.q_full[g], 1);
-      mbar_init(&sh.s_full[g], 1);
-      mbar_init(&sh.s_free[g], 4);
-      mbar_init(&sh.p_full[g], 4);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(&sh.s_full[g][b], 1);
+        mbar_init(&sh.p_full[g][b], 4);
+      }
       mbar_init(&sh.pv_done[g], 1);
+      mbar_init(&sh.o_final[g], 1);
     }
     for (int i = 0; i < kFwKvSlots; ++i) {
       mbar_init(&sh.kv_full[i], 1);
@@ -428,9 +436,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     ok = __all_sync(0xffffffffu, ok) != 0;
     if (ok) tc_fence_after();
     const uint32_t q_base = smem_u32(q_tiles + g * kTileBytes);
-    const uint32_t d_s = tmem + kFwColS + (uint32_t)g * 64u;
-    const uint32_t d_o = tmem + kFwColO + (uint32_t)g * 128u, a_p = tmem + kFwColP + (uint32_t)g * 64u;
-    // S_g(js) = Q_g K_js^T: needs K_js in shared memory (and, checked by the caller, S_g(js-1) read out)
+    const uint32_t sp_base = tmem + kFwColSP + (uint32_t)g * 128u;  // + 64 (j & 1)
+    const uint32_t d_o = tmem + kFwColO + (uint32_t)g * 128u;
+    // S_g(js) = Q_g K_js^T into buffer js % 2: needs K_js in shared memory.  The buffer's previous content,
+    // P_g(js-2), is read by P V of tile js-2, which this thread issued earlier: the tensor core runs one
+    // thread's instructions in order.
     auto issue_s = [&](int js) {
       ok = ok && wait_or_abort(&sh.kv_full[s_slot], s_par, abort_flag);
       ok = __all_sync(0xffffffffu, ok) != 0;
@@ -440,6 +450,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // descriptors once per tile; a K step only moves the start-address field of the low word
       const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + s_slot * kFwKvSlotBytes), 16, 1024);
+      const uint32_t d_s = sp_base + (uint32_t)(js & 1) * 64u;
       if (elect_one()) {
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks) {
@@ -450,7 +461,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           else
             mma_ss_lohi<true>(d_s, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk), idesc_s);
         }
-        mma_commit(&sh.s_full[g]);
+        mma_commit(&sh.s_full[g][js & 1]);
         FWD_TL(g, js, 0);
         mma_commit(&sh.kv_empty[s_slot]);  // K_js may be refilled once BOTH groups' scores have read it (two arrivals)
       }
@@ -461,23 +472,21 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         s_par ^= 1u;
       }
     };
-    // Per group the events come in a fixed order — S(j) read out, then P(j) stored — so the warp simply
-    // waits for them in turn (blocking waits: no polling next to the softmax warps of its scheduler).
+    // Two score tiles ahead of the softmax, then per tile: P V as soon as the probabilities are stored,
+    // and the score tile after next into the buffer that P V just read (blocking waits: per group the
+    // events come in a fixed order, and nothing polls next to the softmax warps of this scheduler).
     if (ntg > 0) issue_s(0);
+    if (ntg > 1) issue_s(1);
     for (int j = 0; j < ntg && ok; ++j) {
-      if (j + 1 < ntg) {  // S(j+1) runs under the softmax of tile j
-        ok = wait_or_abort(&sh.s_free[g], (uint32_t)j & 1u, abort_flag);
-        ok = __all_sync(0xffffffffu, ok) != 0;
-        issue_s(j + 1);
-      }
       // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
-      ok = ok && wait_or_abort(&sh.p_full[g], (uint32_t)j & 1u, abort_flag);
+      ok = ok && wait_or_abort(&sh.p_full[g][j & 1], (uint32_t)(j >> 1) & 1u, abort_flag);
       ok = ok && wait_or_abort(&sh.kv_full[pv_slot], pv_par, abort_flag);
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) break;
       tc_fence_after();
       FWD_TL(g, j, 2);
       const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + pv_slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+      const uint32_t a_p = sp_base + (uint32_t)(j & 1) * 64u;
       if (elect_one()) {
         if (j == 0) mma_ts_lohi<false>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
         else mma_ts_lohi<true>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
@@ -487,6 +496,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           mma_ts_lohi<true>(d_o, a_p + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
         }
         mma_commit(&sh.pv_done[g]);
+        if (j == ntg - 1) mma_commit(&sh.o_final[g]);
         FWD_TL(g, j, 4);
         mma_commit(&sh.kv_empty[pv_slot]);
       }
@@ -496,6 +506,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         pv_slot -= kFwKvSlots;
         pv_par ^= 1u;
       }
+      if (j + 2 < ntg) issue_s(j + 2);
     }
     // Tiles this group never uses (its query block ends earlier, or it does not exist): the ring still
     // expects two arrivals per slot, given here as soon as the tile has landed.
@@ -521,8 +532,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     const int qi = ib * kTile + row;           // query position inside the sequence
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
     const uint32_t tmem_o = tmem + kFwColO + (uint32_t)g * 128u + lane_addr;
-    const uint32_t tmem_s = tmem + kFwColS + (uint32_t)g * 64u + lane_addr;
-    const uint32_t tmem_p = tmem + kFwColP + (uint32_t)g * 64u + lane_addr;
+    const uint32_t tmem_sp = tmem + kFwColSP + (uint32_t)g * 128u + lane_addr;  // + 64 (j & 1)
     bool ok = true;
     float m_used = -INFINITY;
     float2 l2 = make_float2(0.f, 0.f);  // row sum, even and odd keys apart (packed fp32x2 adds)
@@ -531,43 +541,43 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #endif
     for (int j = 0; j < ntg && ok; ++j) {
       FWD_CLK(c0_);
-      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[g], j & 1, abort_flag));  // collectives below
+      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[g][j & 1], (uint32_t)(j >> 1) & 1u, abort_flag));  // collectives below
       if (!ok) break;
       tc_fence_after();
       FWD_CLK(c1_);
       FWD_TL(g, j, 1);
-      if (g == 0) FWD_W(quarter, j, 0);
+      const uint32_t buf = tmem_sp + (uint32_t)(j & 1) * 64u;
       uint32_t r0[32], r1[32];
-      tmem_ld32(tmem_s, r0);
-      tmem_ld32(tmem_s + 32u, r1);
+      tmem_ld32(buf, r0);
+      tmem_ld32(buf + 32u, r1);
       tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.s_free[g]);  // the next S may be computed while we work on this one
       FWD_CLK(c2_);
       const int key0 = j * kFwKeys;
       const bool masked_tile = key0 + kFwKeys - 1 > ib * kTile;  // tile reaches past this block's first query
       // raw scores stay unscaled: the scale is positive, so the maximum commutes with it and the
       // multiplication is folded into the exponent's fused multiply-add below
+      if (masked_tile) {
+#pragma unroll
+        for (int c2 = 0; c2 < kFwKeys; ++c2)
+          if (key0 + c2 > qi) (c2 < 32 ? r0[c2] : r1[c2 - 32]) = 0xff800000u;  // -inf, causal: key <= query
+      }
       float m_raw = -INFINITY;
 #pragma unroll
-      for (int c2 = 0; c2 < kFwKeys; ++c2) {
-        uint32_t& word = c2 < 32 ? r0[c2] : r1[c2 - 32];
-        if (masked_tile && key0 + c2 > qi) word = 0xff800000u;  // -inf, causal: key <= query
-        m_raw = fmaxf(m_raw, __uint_as_float(word));
-      }
+      for (int c2 = 0; c2 < kFwKeys; c2 += 2)  // three-input maximum: half the instructions on the ALU pipe
+        m_raw = max3(m_raw, __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]),
+                     __uint_as_float(c2 < 32 ? r0[c2 + 1] : r1[c2 - 31]));
       const float m_tile = m_raw * scale2;
       const bool need = m_tile > m_used + kRescaleThreshold;
       if (j == 0) {
         m_used = m_tile;  // key 0 is visible to every row, so this is finite
       } else {
         const bool rescale = __any_sync(0xffffffffu, need);
-        // O_g must include tile j-1 before it is rescaled, and P_g(j-1) must have been consumed before
-        // it is overwritten below; both are signalled by pv_done (normally long since complete)
-        ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(j - 1) & 1u, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
         if (rescale) {
+          // O_g must include tile j-1 before it is rescaled (P V of tile j is issued only after this
+          // tile's probabilities, so it sees the rescaled rows)
+          ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(j - 1) & 1u, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
           const float m_new = need ? m_tile : m_used;
           const float alpha = ex2(m_used - m_new);
           l2 = __fmul2_rn(l2, make_float2(alpha, alpha));
@@ -586,7 +596,6 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       }
       const float neg_m = -m_used;
       FWD_CLK(c3_);
-      if (g == 0) FWD_W(quarter, j, 1);
       // probabilities relative to the reference maximum as bf16 hi (columns 0..31) and bf16 lo
       // (columns 32..63): column c holds keys 2c and 2c+1
       uint32_t hw[32], lw[32];
@@ -602,15 +611,14 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
         lw[c] = Vec16<__nv_bfloat16>::pack2(lo.x, lo.y);
       }
-      tmem_st32(tmem_p, hw);
-      tmem_st32(tmem_p + 32u, lw);
+      tmem_st32(buf, hw);        // over the scores, which are in registers by now
+      tmem_st32(buf + 32u, lw);
       tmem_wait_st();
       FWD_CLK(c4_);
       FWD_TL(g, j, 3);
-      if (g == 0) FWD_W(quarter, j, 2);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.p_full[g]);
+      if (lane == 0) mbar_arrive(&sh.p_full[g][j & 1]);
       FWD_ADD(0, c0_, c1_);
       FWD_ADD(1, c1_, c2_);
       FWD_ADD(2, c2_, c3_);
@@ -623,7 +631,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     }
 #endif
     if (ntg > 0) {
-      if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(ntg - 1) & 1u, abort_flag));
+      if (ok) ok = __all_sync(0xffffffffu, wait_or_abort(&sh.o_final[g], 0, abort_flag));
       if (ok) {
         tc_fence_after();
         const float inv_l = 1.0f / (l2.x + l2.y);
@@ -695,9 +703,6 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int
 }
 
 #ifdef H2O_PHASE_TIMERS
-extern "C" int h2o_debug_fwd_warps(long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_fwd_w, sizeof(long long) * 4 * 40 * 3);
-}
 extern "C" int h2o_debug_fwd_timeline(long long* host) {
   return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(long long) * 2 * 40 * 6);
 }
