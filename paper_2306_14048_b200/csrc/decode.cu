@@ -32,8 +32,10 @@ namespace h2o {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+// Consumer warps per block: 8 by default; 4 for launches of many small units (more blocks resident per
+// SM hide one another's serial prologue and epilogue, which dominate a unit of a few tiles).
+constexpr int kMaxWarps = 8;
+constexpr int kSmallUnitRows = 160;  // largest block share (slots) served by the 4-warp variant
 constexpr int kTileBytes = 8192;
 constexpr int kMaxStages = 8;
 constexpr int kDefaultStages = 4;
@@ -129,13 +131,13 @@ __device__ unsigned long long g_phase[8192 * 16];
 #define H2O_STAMP(i) do { } while (0)
 #endif
 
-template <typename T, int D>
+template <typename T, int D, int NW>
 struct Cfg {
   static constexpr int VEC = Vec16<T>::N;
   static constexpr int LPR = D / VEC;                  // lanes per row
   static constexpr int RPW = 32 / LPR;                 // rows per warp pass (= row groups per warp)
-  static constexpr int RPC = kWarps * RPW;             // rows per block pass
-  static constexpr int GROUPS = kWarps * RPW;          // independent online-softmax streams per block
+  static constexpr int RPC = NW * RPW;                 // rows per block pass
+  static constexpr int GROUPS = NW * RPW;              // independent online-softmax streams per block
   static constexpr int ROW_BYTES = D * (int)sizeof(T);
   static constexpr int TILE_ROWS = kTileBytes / ROW_BYTES;
   static constexpr int PASSES = TILE_ROWS / RPC;
@@ -150,7 +152,7 @@ struct Shared {
   uint64_t aux;
   float red[GROUPS][D];  // per-group partial outputs (unnormalised, relative to the group's maximum)
   float gm[GROUPS], gl[GROUPS];
-  Cand wbest[kWarps];
+  Cand wbest[kMaxWarps];
   // Cluster exchange: every block PUSHES its values into its peers' shared memory (remote stores are
   // fire-and-forget, remote loads a round trip), then one cluster barrier makes them visible.
   float x_m[kMaxSplit], x_l[kMaxSplit];  // block statistics of every rank (written by that rank)
@@ -159,18 +161,20 @@ struct Shared {
   //  exist only in launches that split a unit, so that unsplit launches keep their blocks per SM)
 };
 
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+template <int THREADS>
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 
 // MINB is the number of blocks per SM the register allocation must leave room for.  A launch with at
 // most two blocks per SM runs fastest with all the registers the compiler wants (MINB 1: no spills, more
 // loads in flight per thread); a launch with many blocks per SM is bound by how many of them are
 // resident to hide one another's serial prologue and epilogue (MINB 4).
-template <typename T, int D, int MINB>
-__global__ void __launch_bounds__(kThreads + 32, MINB)
+template <typename T, int D, int MINB, int NW>
+__global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
               T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
               int cache_is_quiescent) {
-  using C = Cfg<T, D>;
+  using C = Cfg<T, D, NW>;
+  constexpr int kWarps = NW, kThreads = NW * 32;
   constexpr int VEC = C::VEC, LPR = C::LPR, RPW = C::RPW, RPC = C::RPC, TILE_ROWS = C::TILE_ROWS, GROUPS = C::GROUPS;
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared<GROUPS, D> sh;
@@ -179,7 +183,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   double* acc_s = reinterpret_cast<double*>(dyn + (size_t)stages * 2 * kTileBytes);
   int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
   float* p = reinterpret_cast<float*>(pos_s + chunk);
-  float* x_out = p + chunk;  // [kMaxSplit][D], only when split > 1
+  float* x_out = p + chunk + 4;  // [kMaxSplit][D], only when split > 1 (behind the 16 spare bytes of p)
 
   H2O_STAMP(1);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -355,7 +359,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       sh.gm[g] = mg;
       sh.gl[g] = lg;
     }
-    consumer_sync();
+    consumer_sync<kThreads>();
     {
     H2O_STAMP(8);
 
@@ -432,7 +436,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     H2O_STAMP(11);
     if (lane == 0) sh.wbest[warp] = best;
     if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
-    consumer_sync();
+    consumer_sync<kThreads>();
     H2O_STAMP(5);
     if (warp == 0) {
       Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
@@ -484,11 +488,10 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   H2O_STAMP(6);
 }
 
-template <typename T, int D, int MINB>
+template <typename T, int D, int MINB, int NW>
 cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
-                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  using C = Cfg<T, D>;
-  // ring depth: the whole chunk if it is short, otherwise enough to keep ~64 KB in flight per block
+                        const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  using C = Cfg<T, D, NW>;
   // Ring depth.  With few blocks (at most two per SM) each block needs a deep ring to keep enough
   // bytes in flight; with many blocks a shallow ring lets more of them be resident, which hides each
   // block's serial prologue and epilogue behind the others' streams.
@@ -501,13 +504,14 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
                       (split > 1 ? (size_t)kMaxSplit * D * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
   {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB>), kMaxDynSmem, &attr_flags);
+    cudaError_t e =
+        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB, NW>), kMaxDynSmem, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(c.units * split));
-  cfg.blockDim = dim3(kThreads + 32);
+  cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute at[2];
@@ -519,17 +523,20 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB>, c, static_cast<const T*>(q), static_cast<const T*>(k_new),
-                            static_cast<const T*>(v_new), static_cast<T*>(out), evicted_pos, split, chunk, stages,
-                            quiescent ? 1 : 0);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW>, c, static_cast<const T*>(q),
+                            static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
+                            evicted_pos, split, chunk, stages, quiescent ? 1 : 0);
 }
 
 template <typename T, int D>
 cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  if (c.units * split > 2 * 148)
-    return launch_minb<T, D, 4>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
-  return launch_minb<T, D, 1>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+  const int blocks = c.units * split;
+  if (blocks > 4 * 148 && chunk <= kSmallUnitRows)  // many small units: half-size blocks, five per SM
+    return launch_minb<T, D, 5, 4>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+  if (blocks > 2 * 148)
+    return launch_minb<T, D, 4, 8>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_minb<T, D, 1, 8>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace
