@@ -77,13 +77,15 @@ def _gather_units(x, cu, units, H):
 
 def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
-               device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0) -> ParityStats:
+               device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
+               pattern: Optional[Sequence[int]] = None) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
     (all of them by default) as a batch of single-head sequences, which is exact because units never
     interact.  With ``chunk`` > 0 the CUDA path advances ``chunk`` tokens per call (h2o_decode_chunk)
-    while the oracle still takes them one decode step at a time.
+    while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
+    sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
     """
     stats = ParityStats()
     H, d = wl.n_heads, wl.head_dim
@@ -132,8 +134,11 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     def pick(x):  # [batch, H, d] -> the sampled units as [len(units), 1, d] float32 on the host
         return x.reshape(wl.units, d)[uidx].float().cpu().numpy()[:, None, :]
 
-    step = 0
+    step, call = 0, 0
     while step < steps:
+        if pattern:
+            chunk = int(pattern[call % len(pattern)])
+            call += 1
         nt = min(chunk, steps - step) if chunk > 0 else 1
         qs, ks, vs = zip(*[make_decode_inputs(wl, step + i, layer=layer, device=device) for i in range(nt)])
         if chunk > 0:

@@ -85,6 +85,16 @@ def test_chunk_one_tile_budgets(H2OCache):
     print(st)
 
 
+def test_chunk_and_single_step_calls_interleaved(H2OCache):
+    """The two kernels hand the cache to one another: chunk calls of several sizes mixed with single steps."""
+    from parity_harness import run_parity
+
+    wl = _wl("chunkmix", 3, 4, 128, "bf16", [200, 64, 333], 120, [30, 8, 60], [30, 8, 40], seed=109)
+    st = run_parity(wl, H2OCache, pattern=[32, 0, 0, 5, 1, 0, 40, 3], export_every=1)
+    assert st.decisions == 12 + 12 * 120
+    print(st)
+
+
 @pytest.mark.parametrize("dtype,d,heavy,recent", [
     ("f32", 64, [20, 9], [24, 5]),          # no tensor-core path for this dtype
     ("bf16", 128, [600, 100], [600, 100]),  # budget too large for the chunk kernel
