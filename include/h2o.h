@@ -84,6 +84,18 @@ size_t h2o_prefill_scratch_bytes(const h2o_config_t* cfg, int64_t total_tokens);
 int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes);
 
 /*
+ * Attach a handle to a workspace that ALREADY holds a cache of the same configuration —
+ * a byte copy of another handle's workspace, taken while no work on it was in flight and
+ * possibly restored from a file: the whole state of a cache (K/V slots, scores, positions,
+ * counters) lives in its workspace, so copying the bytes is the snapshot and this call is
+ * the resume.  Nothing in the workspace is modified; its unit table is compared with the
+ * one `cfg` produces (H2O_ERR_STATE if they differ).  The handle accepts decode calls;
+ * h2o_prefill_select is refused (H2O_ERR_STATE) until h2o_cache_reset.
+ * No counterpart in the paper (its cache is transient state of one generation).
+ */
+int h2o_cache_attach(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes);
+
+/*
  * Prefill selection (Appendix A pseudocode, prefill branch: attention over the
  * whole prompt, then "select K heavy hitters and K recent tokens", all tokens
  * if the prompt is not longer than the budget).  For every unit:

@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_create.restype = c.c_int
     lib.h2o_cache_create.argtypes = [c.POINTER(vp), cfgp, vp, c.c_size_t]
     lib.h2o_prefill_select.restype = c.c_int
+    lib.h2o_cache_attach.argtypes = [c.POINTER(vp), cfgp, vp, c.c_size_t]
+    lib.h2o_cache_attach.restype = c.c_int
     lib.h2o_prefill_select.argtypes = [vp, vp, vp, vp, i32p, vp, vp, c.c_size_t, vp]
     lib.h2o_prefill_select_static.restype = c.c_int
     lib.h2o_prefill_select_static.argtypes = [vp, vp, vp, vp, i32p, vp, vp]
@@ -160,7 +162,8 @@ class H2OCache:
     ``status`` -> h2o_cache_status, ``close`` -> h2o_cache_destroy.
     """
 
-    def __init__(self, batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale=0.0, device=0):
+    def __init__(self, batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale=0.0, device=0, snapshot=None):
+        """``snapshot``: bytes of another handle's workspace (``snapshot()``) to resume from (h2o_cache_attach)."""
         self.cfg, self._keep = make_config(batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale, device)
         self.batch, self.n_heads, self.head_dim = int(batch), int(n_heads), int(head_dim)
         self.units = self.batch * self.n_heads
@@ -173,9 +176,21 @@ class H2OCache:
         self._ws_ptr = (self.workspace.data_ptr() + 255) // 256 * 256
         self.workspace_bytes = nbytes
         handle = ctypes.c_void_p()
-        _check(lib.h2o_cache_create(ctypes.byref(handle), ctypes.byref(self.cfg), self._ws_ptr, nbytes), "h2o_cache_create")
+        if snapshot is None:
+            _check(lib.h2o_cache_create(ctypes.byref(handle), ctypes.byref(self.cfg), self._ws_ptr, nbytes), "h2o_cache_create")
+        else:
+            off = self._ws_ptr - self.workspace.data_ptr()
+            self.workspace[off:off + nbytes].copy_(snapshot.to(self.device))
+            torch.cuda.synchronize(self.device)
+            _check(lib.h2o_cache_attach(ctypes.byref(handle), ctypes.byref(self.cfg), self._ws_ptr, nbytes), "h2o_cache_attach")
         self._h = handle
         self._scratch = None
+
+    def snapshot(self):
+        """The workspace bytes (a copy): the complete state of the cache.  Synchronises the device first."""
+        torch.cuda.synchronize(self.device)
+        off = self._ws_ptr - self.workspace.data_ptr()
+        return self.workspace[off:off + self.workspace_bytes].clone()
 
     def prefill_select(self, q, k, v, cu_seqlens, out, stream=None):
         cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)

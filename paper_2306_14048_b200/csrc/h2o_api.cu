@@ -198,7 +198,8 @@ size_t h2o_prefill_scratch_bytes(const h2o_config_t* cfg, int64_t total_tokens) 
   return make_scratch_layout(cfg, total_tokens).total;
 }
 
-int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes) {
+static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes,
+                       bool attach) {
   if (!out) return H2O_ERR_INVALID_ARG;
   const int rc = check_config(cfg);
   if (rc != H2O_OK) return rc;
@@ -268,9 +269,20 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
   v.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
 
   bool ok = true;
-  ok = ok && cudaMemset(ws + L.acc, 0, L.meta - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
-  ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
-  ok = ok && cudaMemcpy(ws + L.meta, meta.data(), units * sizeof(h2o::UnitMeta), cudaMemcpyHostToDevice) == cudaSuccess;
+  if (attach) {
+    // the workspace already holds a cache: its unit table must be the one this configuration produces
+    std::vector<h2o::UnitMeta> have(units);
+    ok = cudaMemcpy(have.data(), ws + L.meta, units * sizeof(h2o::UnitMeta), cudaMemcpyDeviceToHost) == cudaSuccess;
+    if (ok && std::memcmp(have.data(), meta.data(), units * sizeof(h2o::UnitMeta)) != 0) {
+      delete c;
+      return H2O_ERR_STATE;
+    }
+    c->phase = Phase::Decoding;  // whatever it holds, it is not to be prefilled again
+  } else {
+    ok = ok && cudaMemset(ws + L.acc, 0, L.meta - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
+    ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
+    ok = ok && cudaMemcpy(ws + L.meta, meta.data(), units * sizeof(h2o::UnitMeta), cudaMemcpyHostToDevice) == cudaSuccess;
+  }
   if (!ok) {
     cudaGetLastError();
     delete c;
@@ -278,6 +290,14 @@ int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
   }
   *out = c;
   return H2O_OK;
+}
+
+int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes) {
+  return create_impl(out, cfg, dev_workspace, workspace_bytes, false);
+}
+
+int h2o_cache_attach(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes) {
+  return create_impl(out, cfg, dev_workspace, workspace_bytes, true);
 }
 
 int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,

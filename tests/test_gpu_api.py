@@ -151,3 +151,44 @@ def test_caches_on_different_streams(pkg):
         for x, y in zip(c.export(), ref[2]):
             assert np.array_equal(x, y)
         c.close()
+
+
+def test_snapshot_and_attach_resume_bit_identically(pkg):
+    """The workspace bytes are the whole state: a handle attached to a copy continues exactly like the original,
+    also through a file-like round trip on the host; a different configuration is refused."""
+    wl = WL
+    q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    a = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    a.prefill_select(q, k, v, cu, torch.empty_like(q))
+    steps = [make_decode_inputs(wl, s, device="cuda") for s in range(wl.decode_steps)]
+
+    def step(c, s):
+        dq, dk, dv = steps[s]
+        o = torch.empty_like(dq)
+        e = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32, device="cuda")
+        c.decode_step(dq, dk, dv, o, e)
+        return o.float().cpu().numpy(), e.cpu().numpy()
+
+    for s in range(2):
+        step(a, s)
+    snap = a.snapshot().cpu()  # as if written to and read back from a file
+    b = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent, snapshot=snap)
+    for s in range(2, wl.decode_steps):
+        oa, ea = step(a, s)
+        ob, eb = step(b, s)
+        assert np.array_equal(oa, ob) and np.array_equal(ea, eb)
+    for x, y in zip(a.export(), b.export()):
+        assert np.array_equal(x, y)
+    assert a.status() == 0 and b.status() == 0
+    # an attached cache is not prefilled again
+    with pytest.raises(pkg.H2OError) as err:
+        b.prefill_select(q, k, v, cu, torch.empty_like(q))
+    assert err.value.code == pkg.H2O_ERR_STATE
+    # the unit table of another configuration does not match
+    heavy2 = tuple(x + 4 for x in wl.heavy)
+    snap2 = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, heavy2, wl.recent).snapshot()
+    with pytest.raises(pkg.H2OError) as err:
+        pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent, snapshot=snap2[:a.workspace_bytes])
+    assert err.value.code == pkg.H2O_ERR_STATE
+    a.close()
+    b.close()
