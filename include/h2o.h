@@ -254,6 +254,14 @@ int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path);
  * identical either way.  Returns the previous setting.
  */
 int h2o_debug_set_early_prefetch(int32_t enabled);
+/*
+ * Diagnostic (no counterpart in the paper): enqueue a one-warp kernel that polls `polls` times
+ * (1 .. 2^20, i.e. at most a few milliseconds) on a barrier nobody ever arrives at and then, like
+ * every bounded wait of this library that gives up, records H2O_ERR_TIMEOUT in the cache's status
+ * word and returns normally.  h2o_cache_status then reports the code; h2o_cache_reset clears it.
+ * Shows that a timed-out wait costs a status code, not the context.
+ */
+int h2o_debug_wait_probe(h2o_cache_t* cache, int32_t polls, void* stream);
 int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, size_t* acc0_offset);
 const char* h2o_strerror(int code);
 

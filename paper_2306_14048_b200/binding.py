@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_create.restype = c.c_int
     lib.h2o_cache_create.argtypes = [c.POINTER(vp), cfgp, vp, c.c_size_t]
     lib.h2o_prefill_select.restype = c.c_int
+    lib.h2o_debug_wait_probe.argtypes = [vp, c.c_int32, vp]
+    lib.h2o_debug_wait_probe.restype = c.c_int
     lib.h2o_cache_attach.argtypes = [c.POINTER(vp), cfgp, vp, c.c_size_t]
     lib.h2o_cache_attach.restype = c.c_int
     lib.h2o_prefill_select.argtypes = [vp, vp, vp, vp, i32p, vp, vp, c.c_size_t, vp]

@@ -602,6 +602,17 @@ int h2o_cache_status(h2o_cache_t* cache, void* stream) {
   return word;
 }
 
+int h2o_debug_wait_probe(h2o_cache_t* cache, int32_t polls, void* stream) {
+  if (!cache || polls < 1 || polls > (1 << 20)) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  if (h2o::launch_wait_probe(cache->view, (uint32_t)polls, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
+  return H2O_OK;
+}
+
 const char* h2o_strerror(int code) {
   switch (code) {
     case H2O_OK: return "ok";

@@ -90,6 +90,8 @@ bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_sl
 cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const UnitMeta* meta, const void* q,
                                 const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos,
                                 cudaStream_t stream);
+// One warp waits `polls` times on a barrier nobody arrives at, then records H2O_ERR_TIMEOUT (diagnostic).
+cudaError_t launch_wait_probe(const CacheView& c, uint32_t polls, cudaStream_t stream);
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
                                  const void* v, cudaStream_t stream);
 

@@ -192,3 +192,18 @@ def test_snapshot_and_attach_resume_bit_identically(pkg):
     assert err.value.code == pkg.H2O_ERR_STATE
     a.close()
     b.close()
+
+
+def test_a_wait_that_gives_up_costs_a_status_code_not_the_context(pkg):
+    """A bounded wait that runs out records H2O_ERR_TIMEOUT; the kernel returns, reset clears the word and
+    the cache works as before."""
+    wl = WL
+    c = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    assert c.status() == 0
+    assert pkg.lib.h2o_debug_wait_probe(c._h, 2000, None) == 0
+    assert c.status() == pkg.H2O_ERR_TIMEOUT
+    assert pkg.lib.h2o_debug_wait_probe(c._h, 0, None) == pkg.H2O_ERR_INVALID_ARG
+    c.reset()
+    assert c.status() == 0
+    c.close()
+    _identical(_full_run(pkg, wl), _full_run(pkg, wl))  # the device is as usable as before
