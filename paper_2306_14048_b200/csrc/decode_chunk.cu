@@ -73,7 +73,7 @@ struct Shared {
   int post_slot[2][kKeyWarps];
   int post_x[2][kKeyWarps];       // candidate's key index inside the block; -1: none
   float post_enext[2][kKeyWarps]; // the candidate's exponential in the next row
-  float redo[kKeyWarps];
+  float redo[kKeyWarps], redo2[kKeyWarps];
   int evicted[kC];
   int wb_slot[kC];
 };
@@ -342,11 +342,11 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     DC_STAMP(2);
     tc_fence_after();
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    // reference maximum of every token's row: over all keys of that row, alive or not (any reference
-    // works for a softmax, and this one needs no reduction inside the sequential loop)
-    // Exponentials are taken in the base-2 domain, scores times c log2(e) (rounded once, as in the
-    // prefill kernels): exp2(fma(raw, scale2, -m2)) rounds the difference once, so the absolute error
-    // of an exponential stays near 1e-8 whatever its size.
+    // Reference maximum of every token's row: over all keys of that row, alive or not — any reference
+    // gives the same softmax, and this one needs no reduction inside the sequential loop.  Should a key
+    // that died earlier in the chunk tower so far above the live ones that their exponentials vanish,
+    // the row falls back to the live maximum (two extra exchanges, see `rescue` below).
+    // Scores are kept in the base-2 domain, times c log2(e) rounded once as in the prefill kernels.
     const float scale2 = c.scale * 1.4426950408889634f;
     if (ok) {
       float mx[kC];
@@ -382,8 +382,8 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int jxm = m * kTileRows + x0 - cnt0;
         const int first = jxm < 0 ? 0 : (jxm < ceff ? jxm : kC);
 #pragma unroll
-        for (int i = 0; i < kC; ++i)
-          raw[i] = __float_as_uint(i >= first ? ex2(fmaf(__uint_as_float(raw[i]), scale2, -sh.m_row[i])) : 0.f);
+        for (int i = 0; i < kC; ++i)  // scaled score; -inf where the key is not part of the row
+          raw[i] = __float_as_uint(i >= first ? __uint_as_float(raw[i]) * scale2 : -INFINITY);
         tmem_st32(tmem + kColS + (uint32_t)(m * kC) + lane_base, raw);
       }
       tmem_wait_st();
@@ -392,58 +392,91 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 
     // ---- the tokens, in order (Algorithm 1) ----
     int live = cnt0;  // entries in the cache before the current token
-    // exponentials of this thread's keys in the current token's row and in the next one
-    uint32_t cur[KT], nxt[KT], nn[KT];
-#pragma unroll
-    for (int m = 0; m < KT; ++m) {
-      cur[m] = 0u;
-      nxt[m] = 0u;
-      if (ok && m < ntiles) {
-        tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + lane_base, cur[m]);
-        if (ceff > 1) tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + 1u + lane_base, nxt[m]);
-      }
-    }
-    tmem_wait_ld_regs(cur);
-    tmem_wait_ld_regs(nxt);
     float l;
-    {  // normaliser of the first token: nothing has been evicted yet
+    // this thread's keys: exponentials in the current token's row, scaled scores of the next row and of
+    // the row after next (in flight)
+    float e_cur[KT];
+    uint32_t nxt[KT], nn[KT];
+    // Live-maximum fallback for row `row` (scores `tv`): exponentials `ev` relative to the largest score
+    // among the entries alive in that row, and their sum.  Reached by all key threads together.
+    auto rescue = [&](const uint32_t (&tv)[KT], float (&ev)[KT], int row) -> float {
+      float mx = -INFINITY;
+#pragma unroll
+      for (int m = 0; m < KT; ++m)
+        if (alive[m] | (jx[m] == row)) mx = fmaxf(mx, __uint_as_float(tv[m]));
+      mx = warp_max(mx);
+      if (lane == 0) sh.redo[warp] = mx;
+      key_sync();
+      const float ml = fmaxf(fmaxf(sh.redo[0], sh.redo[1]), fmaxf(sh.redo[2], sh.redo[3]));
+      float s2 = 0.f;
+#pragma unroll
+      for (int m = 0; m < KT; ++m) {
+        ev[m] = ex2(__uint_as_float(tv[m]) - ml);
+        if (alive[m] | (jx[m] == row)) s2 += ev[m];
+      }
+      s2 = warp_sum(s2);
+      if (lane == 0) sh.redo2[warp] = s2;
+      key_sync();
+      return (sh.redo2[0] + sh.redo2[1]) + (sh.redo2[2] + sh.redo2[3]);
+    };
+    constexpr float kTinySum = 1e-30f;  // below this the live exponentials have (nearly) underflowed
+    {
+      uint32_t t0v[KT];
+#pragma unroll
+      for (int m = 0; m < KT; ++m) {
+        t0v[m] = 0xff800000u;  // -inf
+        nxt[m] = 0xff800000u;
+        if (ok && m < ntiles) {
+          tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + lane_base, t0v[m]);
+          if (ceff > 1) tmem_ld1(tmem + kColS + (uint32_t)(m * kC) + 1u + lane_base, nxt[m]);
+        }
+      }
+      tmem_wait_ld_regs(t0v);
+      tmem_wait_ld_regs(nxt);
+      const float m0 = sh.m_row[0];
+#pragma unroll
+      for (int m = 0; m < KT; ++m) e_cur[m] = ex2(__uint_as_float(t0v[m]) - m0);
+      // normaliser of the first token: nothing has been evicted yet
       float sm = 0.f;
 #pragma unroll
       for (int m = 0; m < KT; ++m)
-        if (alive[m] || jx[m] == 0) sm += __uint_as_float(cur[m]);
+        if (alive[m] | (jx[m] == 0)) sm += e_cur[m];
       sm = warp_sum(sm);
       if (lane == 0) sh.post_sum[1][warp] = sm;
       key_sync();
       const float4 s4 = *reinterpret_cast<const float4*>(sh.post_sum[1]);
       l = (s4.x + s4.y) + (s4.z + s4.w);
+      if (!(l > kTinySum)) l = rescue(t0v, e_cur, 0);
     }
 #pragma unroll 1
     for (int i = 0; i < ceff; ++i) {
 #pragma unroll
       for (int m = 0; m < KT; ++m) {  // the row after next, in flight while this token is worked on
-        nn[m] = 0u;
+        nn[m] = 0xff800000u;  // -inf: no such row
         if (ok && m < ntiles && i + 2 < ceff) tmem_ld1(tmem + kColS + (uint32_t)(m * kC + i + 2) + lane_base, nn[m]);
       }
       const int t = t0 + i, par = i & 1;
       const float inv_l = __frcp_rn(l);
       const bool full = live >= B;
       Cand cm[KT];
+      float en[KT];  // exponentials of the next row
+      const float m_next = i + 1 < ceff ? sh.m_row[i + 1] : 0.f;
       float sm = 0.f;
 #pragma unroll
       for (int m = 0; m < KT; ++m) {
+        en[m] = ex2(__uint_as_float(nxt[m]) - m_next);  // 0 where the key is not part of that row
         alive[m] = alive[m] | (jx[m] == i);  // the token's own key enters the set
-        const float p = alive[m] ? __uint_as_float(cur[m]) * inv_l : 0.f;
+        const float p = alive[m] ? e_cur[m] * inv_l : 0.f;
         if (alive[m]) acc[m] += (double)p;  // Algorithm 2: accumulated score
-        // the probability replaces the exponential in tensor memory (zero for dead or unborn keys)
+        // the probability replaces the score in tensor memory (zero for dead or unborn keys)
         if (ok && m < ntiles) tmem_st1(tmem + kColS + (uint32_t)(m * kC + i) + lane_base, __float_as_uint(p));
-        const float en = __uint_as_float(nxt[m]);
         const bool elig = alive[m] & (pos[m] <= t - r);  // outside the recent window: may be evicted (used when full)
         cm[m].key = elig ? (unsigned long long)__double_as_longlong(acc[m]) : ~0ull;
         cm[m].pos = elig ? pos[m] : INT_MAX;
         cm[m].slot = slot[m];
         cm[m].x = elig ? m * kTileRows + x0 : -1;
-        cm[m].e_next = en;
-        sm += (alive[m] | (jx[m] == i + 1)) ? en : 0.f;  // next row, over the set before this token's eviction
+        cm[m].e_next = en[m];
+        sm += (alive[m] | (jx[m] == i + 1)) ? en[m] : 0.f;  // next row, over the set before this token's eviction
       }
       if (full) {
         // warp minimum under (score, position) and warp sum, interleaved: two independent chains
@@ -515,7 +548,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           float s2 = 0.f;
 #pragma unroll
           for (int m = 0; m < KT; ++m)
-            if (alive[m] || jx[m] == i + 1) s2 += __uint_as_float(nxt[m]);
+            if (alive[m] | (jx[m] == i + 1)) s2 += en[m];
           s2 = warp_sum(s2);
           if (lane == 0) sh.redo[warp] = s2;
           key_sync();
@@ -529,9 +562,10 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (tid == 0) sh.evicted[i] = -1;
         l = lsum;
       }
+      if (i + 1 < ceff && !(l > kTinySum)) l = rescue(nxt, en, i + 1);
 #pragma unroll
       for (int m = 0; m < KT; ++m) {
-        cur[m] = nxt[m];
+        e_cur[m] = en[m];
         nxt[m] = nn[m];
       }
     }

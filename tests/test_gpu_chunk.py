@@ -151,3 +151,46 @@ def test_chunk_full_size_sampled(H2OCache, name, units):
     wl = CONFIGS[name]
     st = run_parity(wl, H2OCache, units=units, steps=64, chunk=64, export_every=64)
     print(st)
+
+
+def test_chunk_dead_key_towers_over_the_live_ones(H2OCache):
+    """A key that is evicted early in a chunk and would dominate the later rows by ~100 nats: the
+    kernel's per-row reference maximum includes it, so the live exponentials underflow and the row has
+    to fall back to the live maximum.  Outputs and evictions must still match the oracle's single steps."""
+    from oracle import h2o_oracle
+    from parity_harness import assert_close
+
+    d, nt, heads = 128, 32, 2
+    g = torch.Generator().manual_seed(4321)
+    a = torch.zeros(d); a[0] = 1.0
+    b = torch.zeros(d); b[1] = 1.0
+    q = 0.3 * torch.randn(nt, 1, heads, d, generator=g)
+    k = 0.3 * torch.randn(nt, 1, heads, d, generator=g)
+    v = torch.randn(nt, 1, heads, d, generator=g)
+    q[:16] += 3.0 * a
+    q[16:] += 3.0 * b
+    k[1] = 384.0 * (b - a)  # score about -100 under the first queries (never attended, evicted), +100 under the later ones
+    q, k, v = (x.to(torch.bfloat16).cuda().contiguous() for x in (q, k, v))
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    heavy, recent = [2], [2]
+    gpu = H2OCache(1, heads, d, "bf16", heavy, recent, softmax_scale=scale)
+    out = torch.empty_like(q)
+    ev = torch.full((nt, 1, heads), -7, dtype=torch.int32, device="cuda")
+    gpu.decode_chunk(q, k, v, out, ev)
+    assert gpu.status() == 0
+    ora = h2o_oracle.OracleCache(1, heads, d, heavy, recent, scale=scale)
+    g_out, g_ev = out.float().cpu().numpy(), ev.cpu().numpy()
+    assert np.isfinite(g_out).all()
+    for i in range(nt):
+        res = ora.decode_step(q[i].float().cpu().numpy(), k[i].float().cpu().numpy(), v[i].float().cpu().numpy(),
+                              hint=g_ev[i].reshape(-1), tie_rel=1e-6)
+        assert (res["status"] != 2).all(), "token %d: evicted %s, oracle %s" % (i, g_ev[i].reshape(-1), res["evicted"])
+        assert_close(g_out[i].reshape(heads, d), res["out"], "bf16", "token %d" % i)
+    assert (g_ev[3].reshape(-1) == 1).all() or (g_ev[:16] == 1).any(), "the planted key was meant to be evicted early"
+    pos, acc, count, t = gpu.export()
+    for u in range(heads):
+        opos, oacc = ora.export(u)
+        order = np.argsort(pos[u, :count[u]])
+        assert np.array_equal(pos[u, :count[u]][order], opos)
+        assert_close(acc[u, :count[u]][order], oacc, "bf16", "acc unit %d" % u)
+    gpu.close()
