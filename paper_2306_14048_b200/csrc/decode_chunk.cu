@@ -147,7 +147,7 @@ __device__ __forceinline__ void tmem_wait_ld_regs(uint32_t (&r)[N]) {
 
 // KT = keys per thread = most 128-key tiles a unit of this cache can need.
 template <int KT>
-__global__ void __launch_bounds__(kThreads, KT <= 2 ? 3 : KT <= 4 ? 2 : 1)
+__global__ void __launch_bounds__(kThreads, KT <= 2 ? 3 : 2)
 decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, CacheView c, const __nv_bfloat16* __restrict__ k_in,
                     const __nv_bfloat16* __restrict__ v_in, __nv_bfloat16* __restrict__ out,
