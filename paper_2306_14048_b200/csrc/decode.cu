@@ -172,7 +172,7 @@ template <typename T, int D, int MINB, int NW>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
               T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
-              int cache_is_quiescent) {
+              int launch_flags) {
   using C = Cfg<T, D, NW>;
   constexpr int kWarps = NW, kThreads = NW * 32;
   constexpr int VEC = C::VEC, LPR = C::LPR, RPW = C::RPW, RPC = C::RPC, TILE_ROWS = C::TILE_ROWS, GROUPS = C::GROUPS;
@@ -194,7 +194,19 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   // store, by which time every block of the cluster has long started (its shared memory exists).
   if (split > 1) cluster.barrier_arrive();
   const int su = blockIdx.x / split;  // launch position of the unit
-  const UnitMeta mt = c.meta[su];     // static table, written once at create time
+  const bool cache_is_quiescent = (launch_flags & 1) != 0, all_full = (launch_flags & 2) != 0;
+  // the unit's static description: arithmetic when all budgets are equal, else one load from the table
+  // written at create time
+  UnitMeta mt;
+  if (c.uni_pad >= 0) {
+    mt.slot_off = (int64_t)su * c.uni_pad;
+    mt.unit = su;
+    mt.kbud = c.uni_k;
+    mt.rwin = c.uni_r;
+    mt.pad_ = 0;
+  } else {
+    mt = c.meta[su];
+  }
   // Programmatic dependent launch: this grid may have been started while the previous kernel of
   // the stream was still running.  What it may touch before that kernel has finished
   // (griddepcontrol.wait) depends on who wrote what:
@@ -208,12 +220,17 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
-  const int cnt = c.count[su];
-  const int t = c.tpos[su];
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
   const int lo = rank * chunk;                            // first slot of this block
-  const int nloc = max(0, min(cnt - lo, chunk));          // occupied slots of this block
-  const int ntile = (nloc + TILE_ROWS - 1) / TILE_ROWS;   // stages to stream (one K tile + one V tile each)
+  // How many slots to stream.  Normally the occupied ones, which takes the counter from memory first.
+  // When the host expects every unit to be full (`all_full`) the block streams its whole share of the
+  // budget at once and reads the counter meanwhile: with equal budgets the first copies then depend on
+  // no load at all.  The expectation only decides WHAT IS FETCHED — rows beyond the real count are
+  // never used — so a stale flag (say, in a replayed CUDA graph) costs bandwidth, not correctness.
+  int cnt = 0;
+  if (!all_full) cnt = c.count[su];
+  const int nstr = all_full ? max(0, min(B - lo, chunk)) : max(0, min(cnt - lo, chunk));
+  const int ntile = (nstr + TILE_ROWS - 1) / TILE_ROWS;   // stages to stream (one K tile + one V tile each)
   T* Kb = reinterpret_cast<T*>(c.K) + (mt.slot_off + lo) * D;
   T* Vb = reinterpret_cast<T*>(c.V) + (mt.slot_off + lo) * D;
   double* acc_g = c.acc + mt.slot_off + lo;
@@ -225,7 +242,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
 
   auto issue_stage = [&](int j) {  // producer lane only
     const int s = j % stages;
-    const int rows = min(TILE_ROWS, nloc - j * TILE_ROWS);
+    const int rows = min(TILE_ROWS, nstr - j * TILE_ROWS);
     const uint32_t bytes = (uint32_t)rows * C::ROW_BYTES;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
     mbar_expect_tx(&sh.full[s], 2 * bytes);
@@ -241,13 +258,16 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     for (int j = 0; j < min(stages, ntile); ++j) issue_stage(j);
-    if (nloc > 0) {
-      const int npad = (nloc + 3) & ~3;  // stays inside the unit's padded slot range
+    if (nstr > 0) {
+      const int npad = (nstr + 3) & ~3;  // stays inside the unit's padded slot range
       mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
       bulk_g2s(acc_s, acc_g, (uint32_t)npad * 8u, &sh.aux);
       bulk_g2s(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
     }
   }
+  if (all_full) cnt = c.count[su];
+  const int t = c.tpos[su];
+  const int nloc = max(0, min(min(cnt - lo, chunk), nstr));  // occupied slots of this block
   __syncthreads();  // barriers are initialised before any consumer polls them
   if (cache_is_quiescent) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -489,7 +509,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
 }
 
 template <typename T, int D, int MINB, int NW>
-cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
+cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req, int launch_flags, const void* q,
                         const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   using C = Cfg<T, D, NW>;
   // Ring depth.  With few blocks (at most two per SM) each block needs a deep ring to keep enough
@@ -525,11 +545,11 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW>, c, static_cast<const T*>(q),
                             static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
-                            evicted_pos, split, chunk, stages, quiescent ? 1 : 0);
+                            evicted_pos, split, chunk, stages, launch_flags);
 }
 
 template <typename T, int D>
-cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, bool quiescent, const void* q,
+cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, int quiescent, const void* q,
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   const int blocks = c.units * split;
   if (blocks > 4 * 148 && chunk <= kSmallUnitRows)  // many small units: half-size blocks, five per SM
@@ -547,10 +567,11 @@ extern "C" int h2o_debug_phase_timers(unsigned long long* host, int n) {
 }
 #endif
 
-cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent,
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent_b, bool all_full,
                           const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                           cudaStream_t stream) {
   if (split < 1 || split > kMaxSplit) return cudaErrorInvalidValue;
+  const int quiescent = (quiescent_b ? 1 : 0) | (all_full ? 2 : 0);  // launch flags
   if (dtype == H2O_F32) {
     if (c.head_dim == 64)
       return launch<float, 64>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);

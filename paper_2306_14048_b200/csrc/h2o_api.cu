@@ -108,6 +108,8 @@ struct h2o_cache {
   int split, chunk, stages;
   int prefill_path;  // 0 = automatic, 1 = force the ALU kernels
   int chunk_path;    // 0 = automatic, 1 = force one decode-step kernel per token in h2o_decode_chunk
+  // tokens every unit of sequence s has been given (prompt + decode steps); < 0: unknown (attached cache)
+  std::vector<int64_t> seen;
   Layout layout;
   h2o::CacheView view;
   Phase phase;
@@ -163,6 +165,17 @@ void* device_alias(const void* host_ptr) {
   if (attr.type != cudaMemoryTypeHost || !attr.devicePointer) return nullptr;
   if (reinterpret_cast<uintptr_t>(attr.devicePointer) % 16 != 0) return nullptr;
   return attr.devicePointer;
+}
+
+// Does the host know that every unit holds exactly its budget of entries?
+bool all_units_full(const h2o_cache* c) {
+  for (int s = 0; s < c->cfg.batch; ++s)
+    if (c->seen[s] < (int64_t)c->heavy[s] + c->recent[s]) return false;  // also when unknown (-1)
+  return true;
+}
+void advance_seen(h2o_cache* c, int64_t tokens) {
+  for (auto& x : c->seen)
+    if (x >= 0) x += tokens;
 }
 
 struct DeviceGuard {
@@ -267,6 +280,15 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   v.n_heads = cfg->n_heads;
   v.head_dim = cfg->head_dim;
   v.scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  {
+    bool uniform = true;
+    for (int s = 1; s < cfg->batch; ++s)
+      uniform = uniform && c->heavy[s] == c->heavy[0] && c->recent[s] == c->recent[0];
+    v.uni_pad = uniform ? ((c->heavy[0] + c->recent[0] + 3) & ~3) : -1;
+    v.uni_k = c->heavy[0];
+    v.uni_r = c->recent[0];
+  }
+  c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
   if (attach) {
@@ -352,6 +374,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
     return H2O_ERR_CUDA;
   }
   g_last_writer.note_and_check(st, cache->view.K);  // select/gather wrote this cache
+  for (int s = 0; s < cfg.batch; ++s) cache->seen[s] = (int64_t)cu_seqlens[s + 1] - cu_seqlens[s];
   cache->phase = Phase::Prefilled;
   return H2O_OK;
 }
@@ -366,12 +389,13 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   // the cache workspace is the identity: two handles on one workspace must count as the same cache
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
   const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages,
-                                           quiescent, q, k_new, v_new, out, evicted_pos,
+                                           quiescent, all_units_full(cache), q, k_new, v_new, out, evicted_pos,
                                            static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
+  advance_seen(cache, 1);
   cache->phase = Phase::Decoding;
   return H2O_OK;
 }
@@ -390,14 +414,16 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
+    if (e == cudaSuccess) advance_seen(cache, n_tokens);
   } else {
     const size_t step = (size_t)cache->view.units * cache->cfg.head_dim * elem_size(cache->cfg.dtype);
     for (int32_t i = 0; i < n_tokens && e == cudaSuccess; ++i) {
       const size_t off = (size_t)i * step;
       e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, false,
-                             static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
+                             all_units_full(cache), static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
                              static_cast<const char*>(v) + off, static_cast<char*>(out) + off,
                              evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr, st);
+      if (e == cudaSuccess) advance_seen(cache, 1);
     }
   }
   if (e != cudaSuccess) {
@@ -513,6 +539,7 @@ int h2o_cache_reset(h2o_cache_t* cache, void* stream) {
     return H2O_ERR_CUDA;
   }
   g_last_writer.note_and_check(st, cache->view.K);  // the memsets wrote this cache
+  cache->seen.assign(cache->cfg.batch, 0);
   cache->phase = Phase::Empty;
   return H2O_OK;
 }

@@ -34,6 +34,10 @@ struct CacheView {
   const UnitMeta* meta;  // [units]
   int32_t units, n_heads, head_dim;
   float scale;           // softmax scale c
+  // When every sequence has the same budgets the unit table is arithmetic (unit = launch position,
+  // slot_off = position * uni_pad) and a block need not load it: uni_pad = slots per unit rounded up
+  // to 4, uni_k / uni_r the budgets; uni_pad < 0 otherwise.
+  int32_t uni_pad, uni_k, uni_r;
 };
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
@@ -68,7 +72,9 @@ inline cudaError_t ensure_dynamic_smem(const void* func, int bytes, unsigned lon
 // `stages` is the depth of the shared-memory ring (0 = default).  `quiescent`: nothing this library
 // launched immediately before on the stream can have written this cache, so the kernel may read the
 // cache before the previous kernel of the stream has finished (it still waits before reading q/k/v).
-cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent,
+// `all_full`: the host knows that every unit holds exactly its budget of entries, so blocks need not
+// load the counters before they start streaming.
+cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent, bool all_full,
                           const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                           cudaStream_t stream);
 // ALU path; `rows` = attention rows + row statistics, `colsum` = column sums.
