@@ -55,7 +55,10 @@ def decode_bytes_per_unit_step(cnt: int, d: int, esize: int) -> int:
 
 # DRAM bytes (read + write) of one decode launch, from the ncu capture summarised in
 # profiles/decode_kernel__c2_opt6p7b.md (55.26 MB read + 0.07 MB written for config 2).
-NCU_DECODE_TRAFFIC_PER_LAUNCH = {"c2_opt6p7b": 55.33e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (ncu, see profiles/).  c2 was captured at
+# full size; c3 on the first 32 of 64 sequences (102.5 MB) and scaled by the units, which the traffic is
+# proportional to (every unit's slots are read once).
+NCU_DECODE_TRAFFIC_PER_LAUNCH = {"c2_opt6p7b": 55.33e6, "c3_opt30b": 2 * 102.5e6}
 
 
 def aggregate_over_ranks(values, world: int, device, dist=None):
