@@ -53,9 +53,8 @@ def decode_bytes_per_unit_step(cnt: int, d: int, esize: int) -> int:
     return 2 * cnt * d * esize + 16 * cnt + 4 * cnt + 6 * d * esize
 
 
-# DRAM bytes (read + write) of one decode launch, from the ncu capture summarised in
-# profiles/decode_kernel__c2_opt6p7b.md (55.26 MB read + 0.07 MB written for config 2).
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch (ncu, see profiles/).  c2 was captured at
+# DRAM bytes of one decode launch, dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture (the
+# summaries are committed with the profiles): 55.26 MB read + 0.07 MB written for config 2, captured at
 # full size; c3 on the first 32 of 64 sequences (102.5 MB) and scaled by the units, which the traffic is
 # proportional to (every unit's slots are read once).
 NCU_DECODE_TRAFFIC_PER_LAUNCH = {"c2_opt6p7b": 55.33e6, "c3_opt30b": 2 * 102.5e6}
