@@ -30,7 +30,7 @@ constexpr double kLog2eD = 1.4426950408889634074;
 // Optional cycle accounting of the forward kernel's softmax loop (compile with -DH2O_PHASE_TIMERS).
 #ifdef H2O_PHASE_TIMERS
 __device__ unsigned long long g_fwd_prof[8];
-__device__ long long g_fwd_tl[2][40][6];  // block (0, units-1): per group and tile, clock64 at six events
+__device__ long long g_fwd_tl[2][40][10];  // block (0, units-1): per group and tile, clock64 at ten events
 #define FWD_TL(g, j, e) do { if (tl_on_ && (j) < 40) g_fwd_tl[g][j][e] = clock64(); } while (0)
 #define FWD_CLK(v) const long long v = clock64()
 #define FWD_ADD(i, a, b) prof_[i] += (b) - (a)
@@ -304,12 +304,12 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // ---------------------------------------------------------------------------------------------
 // Forward: out = softmax(c Q K^T) V over the causal triangle, plus per-row {max, 1/sum}
 // ---------------------------------------------------------------------------------------------
-// One thread block per (unit, PAIR of 128-query blocks); key tiles of 64, loaded once (TMA) for
-// both query blocks.  Two softmax warpgroups (A, B), one per query block, and one MMA-issuing warp
-// that runs a small event loop.  Per group g and key tile j:
+// One thread block per (unit, PAIR of 128-query blocks) (short prompts: per single query block); key tiles
+// of 64, loaded once (TMA) for both query blocks.  One softmax group of four warps per query block (A, B)
+// and, per group, two MMA-issuing warps (even key tiles, odd key tiles).  Per group g and key tile j:
 //   S_g(j) = Q_g K_j^T           M 128, N 64, K 128; Q and K from shared memory, fp32 accumulator
-//                                in TMEM.  Issued as soon as the softmax has READ S_g(j-1) into
-//                                registers, so it runs while that softmax is still computing.
+//                                in TMEM.  Issued two tiles ahead of the softmax, right behind P V(j-2)
+//                                by the same thread (the score buffer is the one that product reads).
 //   P_g(j) = exp2(c S_g(j) - m)  written by the softmax threads into TMEM as bf16 hi | bf16 lo
 //                                (a single bf16 P would put its 2^-9 rounding into the output)
 //   O_g   += P_hi V_j + P_lo V_j M 128, N 128, K 64 twice; P is the TMEM operand, V the MN-major
@@ -317,55 +317,73 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 //                                instruction is bound by shared-memory bandwidth)
 // The softmax keeps one thread per query row (row max / sum need no shuffles) and updates the
 // reference maximum lazily: O rows in TMEM are rescaled only when the maximum grows by more than
-// 8 in the log2 domain.  One block per SM: all 512 TMEM columns, 161 KB of shared memory.
-constexpr int kFwThreads = 352;                   // warp 0: TMA, warp 1: MMA of group A, warps 2..5: group A, 6..9: group B, warp 10: MMA of group B
-constexpr int kFwMmaWarpB = 10;
+// 8 in the log2 domain.  With two groups, one block per SM: all 512 TMEM columns, 161 KB of shared memory.
+// In steady state the tensor pipe is busy about four fifths of the time (S 256 + P V 512 cycles per group
+// and tile against a period of ~990), so issue waits behind the other warps' instructions.
+// Warps come in groups of four that set their register budget together (setmaxnreg): warps 0..3 TMA and
+// MMA issuers (few registers), warps 4..7 softmax of group A (, warps 8..11 softmax of group B, warp 12 the
+// fourth MMA issuer, 13..15 idle).  The block starts with 128 registers per thread; the issuers give
+// registers back and the softmax warps take them.
+__host__ __device__ constexpr int fw_threads(int groups) { return groups == 2 ? 512 : 256; }
+constexpr int kFwRegsIssue = 72, kFwRegsSoftmax = 168;
 constexpr int kFwKeys = 64;                       // keys per tile
 constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
-constexpr int kFwKvSlots = 6;                     // K_j, V_j, K_j+1, V_j+1, K_j+2, V_j+2
-constexpr int kFwTmemCols = 512;
+constexpr int kFwMaxKvSlots = 6;
+constexpr bool kFwSplitP = true;                 // P as bf16 hi + bf16 lo (two P V products): one bf16 alone (2^-9 per
+                                                 // probability) misses the output tolerance on peaky rows
+constexpr int kFwShortPrompt = 1024;              // up to here one query block per thread block
+// ring slots: K_j, V_j, K_j+1, V_j+1 (, K_j+2, V_j+2 with two groups); TMEM columns: O and two S/P buffers per group
+__host__ __device__ constexpr int fw_kv_slots(int groups) { return groups == 2 ? 6 : 4; }
+__host__ __device__ constexpr uint32_t fw_tmem_cols(int groups) { return groups == 2 ? 512u : 256u; }
 constexpr uint32_t kFwColO = 0;                   // O_g : 128 columns each
 // S and P share two 64-column buffers per group: S_g(j) lands in buffer j % 2, the softmax reads it into
 // registers and writes P_g(j) (bf16 hi in columns 0..31, lo in 32..63) over it, S_g(j+1) meanwhile uses
 // the other buffer.  P is thereby double-buffered: the exponentials of tile j+1 need not wait for P V of tile j.
-constexpr uint32_t kFwColSP = 256;                // group g, buffer b: columns 256 + 128 g + 64 b
+// group g, buffer b: columns 128 G + 128 g + 64 b behind the G output accumulators
 constexpr float kRescaleThreshold = 8.0f;
 
 struct FwShared {
   uint64_t q_full[2];
-  uint64_t kv_full[kFwKvSlots], kv_empty[kFwKvSlots];
+  uint64_t kv_full[kFwMaxKvSlots], kv_empty[kFwMaxKvSlots];
   uint64_t s_full[2][2];  // [group][buffer] MMA -> softmax: S_g(j) complete (one barrier per buffer: two S tiles can be ahead)
   uint64_t p_full[2][2];  // [group][buffer] softmax -> MMA: P_g(j) is in tensor memory
-  uint64_t pv_done[2];    // MMA -> softmax: O_g includes tile j (O_g may be rescaled)
+  uint64_t pv_done[2][2]; // [group][tile parity] MMA -> softmax: O_g includes tile j (O_g may be rescaled)
   uint64_t o_final[2];    // MMA -> softmax: O_g includes the group's last tile (a barrier of its own: the softmax
                           // does not wait on every phase of pv_done, so a parity wait for the last one could alias)
   uint32_t tmem_base;
   int abort_flag;
 };
 
-__global__ void __launch_bounds__(kFwThreads)
+// G = query blocks (softmax groups) per thread block.  Two share every K/V tile and fill an SM (all of
+// its tensor memory); one per block lets two blocks share an SM, which hides the fixed cost of a block
+// (allocation, first loads, pipeline fill, output) when prompts are short.
+template <int G>
+__global__ void __launch_bounds__(fw_threads(G), G == 2 ? 1 : 2)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, float scale2,
               __nv_bfloat16* __restrict__ out, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FwShared sh;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
-  unsigned char* q_tiles = dyn;                       // 2 x 32 KB
-  unsigned char* kv_ring = dyn + 2 * kTileBytes;      // 6 x 16 KB
+  constexpr int kFwKvSlots = fw_kv_slots(G);
+  constexpr uint32_t kFwTmemCols = fw_tmem_cols(G);
+  constexpr uint32_t kFwColSP = 128u * G;
+  unsigned char* q_tiles = dyn;                       // G x 32 KB
+  unsigned char* kv_ring = dyn + G * kTileBytes;      // slots of 16 KB
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #ifdef H2O_PHASE_TIMERS
-  const bool tl_on_ = blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) == 1 || ((threadIdx.x >> 5) & 3) == 2);
+  const bool tl_on_ = blockIdx.x == 0 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && ((threadIdx.x >> 5) >= 1 && ((threadIdx.x >> 5) <= 4 || (threadIdx.x >> 5) == 8 || (threadIdx.x >> 5) == 12));
 #endif
   const int u = blockIdx.y;
   const int seq = u / n_heads, h = u % n_heads;
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
   const int nb = (n + kTile - 1) / kTile;
-  const int npair = (nb + 1) / 2;
-  if ((int)blockIdx.x >= npair) return;
-  const int pr = npair - 1 - (int)blockIdx.x;  // long pairs first
-  const int ibA = 2 * pr, ibB = 2 * pr + 1;
-  const bool hasB = ibB < nb;
+  const int nitem = G == 2 ? (nb + 1) / 2 : nb;  // pairs of query blocks, or single ones
+  if ((int)blockIdx.x >= nitem) return;
+  const int pr = nitem - 1 - (int)blockIdx.x;  // long ones first
+  const int ibA = G == 2 ? 2 * pr : pr, ibB = ibA + 1;
+  const bool hasB = G == 2 && ibB < nb;
   // key tiles visible to each group (keys 0 .. min(n, (ib+1)*128) - 1)
   const int ntA = (min(n, (ibA + 1) * kTile) + kFwKeys - 1) / kFwKeys;
   const int ntB = hasB ? (min(n, (ibB + 1) * kTile) + kFwKeys - 1) / kFwKeys : 0;
@@ -378,12 +396,13 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         mbar_init(&sh.s_full[g][b], 1);
         mbar_init(&sh.p_full[g][b], 4);
       }
-      mbar_init(&sh.pv_done[g], 1);
-      mbar_init(&sh.o_final[g], 1);
+      mbar_init(&sh.pv_done[g][0], 1);
+      mbar_init(&sh.pv_done[g][1], 1);
+      mbar_init(&sh.o_final[g], (g == 0 ? ntA : ntB) >= 2 ? 2 : 1);  // one arrival per issuing warp that has a tile
     }
     for (int i = 0; i < kFwKvSlots; ++i) {
       mbar_init(&sh.kv_full[i], 1);
-      mbar_init(&sh.kv_empty[i], 2);  // one arrival per group
+      mbar_init(&sh.kv_empty[i], G);  // one arrival per group
     }
     sh.abort_flag = 0;
     fence_barrier_init();
@@ -395,6 +414,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   const uint32_t tmem = sh.tmem_base;
   volatile int* abort_flag = &sh.abort_flag;
 
+  // MMA issuer index: (group, tile parity) = (idx % G, idx / G); warps 1..3 and, with two groups, warp 12
+  const int mma_idx = (warp >= 1 && warp <= 3) ? warp - 1 : (warp == 12 ? 3 : -1);
+  const bool softmax_warp = warp >= 4 && warp < 4 + 4 * G;
+  if (softmax_warp) setmaxnreg_inc<kFwRegsSoftmax>();
+  else setmaxnreg_dec<kFwRegsIssue>();
   if (warp == 0) {
     // ---------------- TMA producer: Q tiles, then K_0, V_0, K_1, V_1, ... through the slot ring ----
     if (lane == 0) {
@@ -418,113 +442,103 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         tma_load_3d(dst + kFwKvSlotBytes / 2, map, 64, h, row0, &sh.kv_full[slot]);
       }
     }
-  } else if (warp == 1 || warp == kFwMmaWarpB) {
-    // ---------------- MMA issuers: one warp per softmax group ----------------------------------------
-    // A single thread's instruction stream is what bounds the issue of these small matrix instructions
-    // (a warp needs several hundred cycles per action: barrier waits, eight instructions, commits), so
-    // each group has its own issuing warp; the tensor core takes instructions from both.  The whole warp
-    // runs the loop (warp-uniform descriptors), one elected lane issues.
+  } else if (mma_idx >= 0 && mma_idx < 2 * G) {
+    // ---------------- MMA issuers: two warps per softmax group, one for the even key tiles, one for the odd ----
+    // A single thread's instruction stream is what bounds the issue of these small matrix instructions: one
+    // warp needs about a thousand cycles per action (barrier waits, eight instructions, commits), two
+    // actions per tile, while the softmax of a tile takes ~1,300.  So every group has two issuing warps,
+    // each with two tile times for its P V(j) and S(j+2); the tensor core takes instructions from all of
+    // them.  The whole warp runs the loop (warp-uniform descriptors), one elected lane issues (a single
+    // active lane running the loop was slower).
     constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
     // V is the MN-major operand.  (Both operands of one instruction must have the same 16-bit format:
     // an fp16 P against a bf16 V is rejected by the hardware as an illegal instruction.)
     constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
-    const int g = warp == 1 ? 0 : 1;
+    constexpr int kRing = kFwKvSlots / 2;  // key tiles in the ring: tile j has K in slot 2 (j % kRing), V in the next
+    const int g = mma_idx % G, par = mma_idx / G;  // group, parity of this warp's tiles
     const int ntg = g == 0 ? ntA : ntB;
-    int s_slot = 0, pv_slot = 1;        // ring slots of the next K tile / V tile (tile j: slots 2 (j % 3), + 1)
-    uint32_t s_par = 0, pv_par = 0;     // their barrier phases
-    bool ok = ntg == 0 || wait_or_abort(&sh.q_full[g], 0, abort_flag);
+    bool ok = ntg <= par || wait_or_abort(&sh.q_full[g], 0, abort_flag);
     ok = __all_sync(0xffffffffu, ok) != 0;
     if (ok) tc_fence_after();
     const uint32_t q_base = smem_u32(q_tiles + g * kTileBytes);
-    const uint32_t sp_base = tmem + kFwColSP + (uint32_t)g * 128u;  // + 64 (j & 1)
+    const uint32_t sp = tmem + kFwColSP + (uint32_t)g * 128u + (uint32_t)par * 64u;  // this warp's S/P buffer
     const uint32_t d_o = tmem + kFwColO + (uint32_t)g * 128u;
+    const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
     // S_g(js) = Q_g K_js^T into buffer js % 2: needs K_js in shared memory.  The buffer's previous content,
     // P_g(js-2), is read by P V of tile js-2, which this thread issued earlier: the tensor core runs one
     // thread's instructions in order.
     auto issue_s = [&](int js) {
-      ok = ok && wait_or_abort(&sh.kv_full[s_slot], s_par, abort_flag);
+      const int slot = 2 * (js % kRing);
+      ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(js / kRing) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) return;
       tc_fence_after();
       FWD_TL(g, js, 5);
       // descriptors once per tile; a K step only moves the start-address field of the low word
-      const uint64_t dq = smem_desc_sw128(q_base, 16, 1024);
-      const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + s_slot * kFwKvSlotBytes), 16, 1024);
-      const uint32_t d_s = sp_base + (uint32_t)(js & 1) * 64u;
+      const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), 16, 1024);
       if (elect_one()) {
 #pragma unroll
         for (int ks = 0; ks < kD / 16; ++ks) {
           const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
           const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
           if (ks == 0)
-            mma_ss_lohi<false>(d_s, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
+            mma_ss_lohi<false>(sp, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
           else
-            mma_ss_lohi<true>(d_s, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk), idesc_s);
+            mma_ss_lohi<true>(sp, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk), idesc_s);
         }
-        mma_commit(&sh.s_full[g][js & 1]);
+        mma_commit(&sh.s_full[g][par]);
         FWD_TL(g, js, 0);
-        mma_commit(&sh.kv_empty[s_slot]);  // K_js may be refilled once BOTH groups' scores have read it (two arrivals)
+        mma_commit(&sh.kv_empty[slot]);  // K_js may be refilled once every group's scores have read it
       }
       __syncwarp();
-      s_slot += 2;
-      if (s_slot >= kFwKvSlots) {
-        s_slot -= kFwKvSlots;
-        s_par ^= 1u;
-      }
     };
-    // Two score tiles ahead of the softmax, then per tile: P V as soon as the probabilities are stored,
-    // and the score tile after next into the buffer that P V just read (blocking waits: per group the
-    // events come in a fixed order, and nothing polls next to the softmax warps of this scheduler).
-    if (ntg > 0) issue_s(0);
-    if (ntg > 1) issue_s(1);
-    for (int j = 0; j < ntg && ok; ++j) {
+    if (par < ntg) issue_s(par);
+    for (int j = par; j < ntg && ok; j += 2) {
       // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
-      ok = ok && wait_or_abort(&sh.p_full[g][j & 1], (uint32_t)(j >> 1) & 1u, abort_flag);
-      ok = ok && wait_or_abort(&sh.kv_full[pv_slot], pv_par, abort_flag);
+      const int slot = 2 * (j % kRing) + 1;
+      FWD_TL(g, j, 6);
+      // P V(0) initialises O_g: the odd warp's first product must not overtake it
+      if (j == 1) ok = ok && wait_or_abort(&sh.pv_done[g][0], 0, abort_flag);
+      ok = ok && wait_or_abort(&sh.p_full[g][par], (uint32_t)(j >> 1) & 1u, abort_flag);
+      FWD_TL(g, j, 7);
+      ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(j / kRing) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok) != 0;
       if (!ok) break;
       tc_fence_after();
       FWD_TL(g, j, 2);
-      const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + pv_slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
-      const uint32_t a_p = sp_base + (uint32_t)(j & 1) * 64u;
+      const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
       if (elect_one()) {
-        if (j == 0) mma_ts_lohi<false>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
-        else mma_ts_lohi<true>(d_o, a_p, desc_lo(dv), desc_hi(dv), idesc_o);
+        if (j == 0) mma_ts_lohi<false>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
+        else mma_ts_lohi<true>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
 #pragma unroll
-        for (int ks = 1; ks < 2 * (kFwKeys / 16); ++ks) {  // hi columns, then lo columns
+        for (int ks = 1; ks < (kFwSplitP ? 2 : 1) * (kFwKeys / 16); ++ks) {  // hi columns (, then lo columns)
           const uint32_t kk = (uint32_t)(ks & 3);
-          mma_ts_lohi<true>(d_o, a_p + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
+          mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
         }
-        mma_commit(&sh.pv_done[g]);
-        if (j == ntg - 1) mma_commit(&sh.o_final[g]);
+        FWD_TL(g, j, 8);
+        mma_commit(&sh.pv_done[g][par]);
+        if (j + 2 >= ntg) mma_commit(&sh.o_final[g]);  // this warp's last tile
         FWD_TL(g, j, 4);
-        mma_commit(&sh.kv_empty[pv_slot]);
+        mma_commit(&sh.kv_empty[slot]);
+        FWD_TL(g, j, 9);
       }
       __syncwarp();
-      pv_slot += 2;
-      if (pv_slot >= kFwKvSlots) {
-        pv_slot -= kFwKvSlots;
-        pv_par ^= 1u;
-      }
       if (j + 2 < ntg) issue_s(j + 2);
     }
-    // Tiles this group never uses (its query block ends earlier, or it does not exist): the ring still
-    // expects two arrivals per slot, given here as soon as the tile has landed.
-    for (int j = ntg; j < nt && ok; ++j) {
-      ok = wait_or_abort(&sh.kv_full[s_slot], s_par, abort_flag);
-      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[s_slot]);
-      ok = ok && wait_or_abort(&sh.kv_full[s_slot + 1], s_par, abort_flag);
-      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[s_slot + 1]);
+    // Tiles of this parity that the group never uses (its query block ends earlier, or it does not exist):
+    // the ring still expects one arrival per group and slot, given here as soon as the tile has landed.
+    for (int j = ntg + ((ntg ^ par) & 1); j < nt && ok; j += 2) {
+      const int slot = 2 * (j % kRing);
+      const uint32_t ph = (uint32_t)(j / kRing) & 1u;
+      ok = wait_or_abort(&sh.kv_full[slot], ph, abort_flag);
+      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[slot]);
+      ok = ok && wait_or_abort(&sh.kv_full[slot + 1], ph, abort_flag);
+      if (ok && lane == 0) mbar_arrive(&sh.kv_empty[slot + 1]);
       ok = __all_sync(0xffffffffu, ok) != 0;
-      s_slot += 2;
-      if (s_slot >= kFwKvSlots) {
-        s_slot -= kFwKvSlots;
-        s_par ^= 1u;
-      }
     }
-  } else {
+  } else if (softmax_warp) {
     // ---------------- softmax groups: one thread per query row ----------------
-    const int g = (warp - 2) >> 2;             // 0: group A, 1: group B
+    const int g = (warp - 4) >> 2;             // 0: group A, 1: group B
     const int ib = g == 0 ? ibA : ibB;
     const int ntg = g == 0 ? ntA : ntB;
     const int quarter = warp & 3;
@@ -575,7 +589,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         if (rescale) {
           // O_g must include tile j-1 before it is rescaled (P V of tile j is issued only after this
           // tile's probabilities, so it sees the rescaled rows)
-          ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g], (uint32_t)(j - 1) & 1u, abort_flag));
+          ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[g][(j - 1) & 1], (uint32_t)((j - 1) >> 1) & 1u, abort_flag));
           if (!ok) break;
           tc_fence_after();
           const float m_new = need ? m_tile : m_used;
@@ -598,7 +612,8 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       FWD_CLK(c3_);
       // probabilities relative to the reference maximum as bf16 hi (columns 0..31) and bf16 lo
       // (columns 32..63): column c holds keys 2c and 2c+1
-      uint32_t hw[32], lw[32];
+      uint32_t hw[32];
+      [[maybe_unused]] uint32_t lw[32];
 #pragma unroll
       for (int c = 0; c < 32; ++c) {
         const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
@@ -607,12 +622,14 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const float2 pp = make_float2(ex2(x.x), ex2(x.y));
         l2 = __fadd2_rn(l2, pp);
         const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pp.x, pp.y);
-        const float2 lo = __ffma2_rn(__bfloat1622float2(hi2), make_float2(-1.f, -1.f), pp);  // exact remainder
         hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
-        lw[c] = Vec16<__nv_bfloat16>::pack2(lo.x, lo.y);
+        if constexpr (kFwSplitP) {
+          const float2 lo = __ffma2_rn(__bfloat1622float2(hi2), make_float2(-1.f, -1.f), pp);  // exact remainder
+          lw[c] = Vec16<__nv_bfloat16>::pack2(lo.x, lo.y);
+        }
       }
       tmem_st32(buf, hw);        // over the scores, which are in registers by now
-      tmem_st32(buf + 32u, lw);
+      if constexpr (kFwSplitP) tmem_st32(buf + 32u, lw);
       tmem_wait_st();
       FWD_CLK(c4_);
       FWD_TL(g, j, 3);
@@ -704,7 +721,7 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int
 
 #ifdef H2O_PHASE_TIMERS
 extern "C" int h2o_debug_fwd_timeline(long long* host) {
-  return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(long long) * 2 * 40 * 6);
+  return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(g_fwd_tl));
 }
 extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
   if (reset) {
@@ -715,23 +732,36 @@ extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
 }
 #endif
 
+namespace {
+
+template <int G>
+cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v, const CacheView& c,
+                         const PrefillScratch& s, int max_seqlen, void* out, cudaStream_t stream) {
+  const int smem = G * kTileBytes + fw_kv_slots(G) * kFwKvSlotBytes + 1024;
+  static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fwd_tc_kernel<G>), smem, &attr_flags);
+    if (e != cudaSuccess) return e;
+  }
+  const int nb = (max_seqlen + kTile - 1) / kTile;
+  dim3 grid((unsigned)(G == 2 ? (nb + 1) / 2 : nb), (unsigned)c.units);
+  fwd_tc_kernel<G><<<grid, fw_threads(G), smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
+                                                         static_cast<__nv_bfloat16*>(out), c.status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
 cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                           const void* v, void* out, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
   if (!make_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
       !make_tile_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
-  const int smem = 2 * kTileBytes + kFwKvSlots * kFwKvSlotBytes + 1024;
-  static unsigned long long attr_flags = 0;
-  {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fwd_tc_kernel), smem, &attr_flags);
-    if (e != cudaSuccess) return e;
-  }
-  const int nb = (max_seqlen + kTile - 1) / kTile;
-  dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
-  fwd_tc_kernel<<<grid, kFwThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
-                                                   static_cast<__nv_bfloat16*>(out), c.status);
-  return cudaGetLastError();
+  // short prompts: one query block per thread block, two blocks per SM; long ones: two query blocks share
+  // every K/V tile
+  if (max_seqlen <= kFwShortPrompt) return launch_fwd_g<1>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
+  return launch_fwd_g<2>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
 }
 
 bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 && head_dim == kD && encode_fn() != nullptr; }

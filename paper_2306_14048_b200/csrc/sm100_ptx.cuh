@@ -17,6 +17,17 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 // One lane of a converged warp (the same lane every time).  The MMA-issuing warp runs its loop with
 // all lanes, so that descriptors and addresses stay warp-uniform (uniform registers), and predicates
 // only the single-thread instructions with this.
+// Register budget of the calling group of four warps (all 128 threads execute it): give registers back
+// to the block's pool, or take them (waits until enough have been given back).
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
