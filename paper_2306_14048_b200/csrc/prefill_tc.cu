@@ -30,6 +30,8 @@ constexpr double kLog2eD = 1.4426950408889634074;
 // Optional cycle accounting of the forward kernel's softmax loop (compile with -DH2O_PHASE_TIMERS).
 #ifdef H2O_PHASE_TIMERS
 __device__ unsigned long long g_fwd_prof[8];
+__device__ unsigned long long g_cs_prof[8];
+__device__ unsigned long long g_cs_blk[8];
 __device__ long long g_fwd_tl[2][40][10];  // block (0, units-1): per group and tile, clock64 at ten events
 #define FWD_TL(g, j, e) do { if (tl_on_ && (j) < 40) g_fwd_tl[g][j][e] = clock64(); } while (0)
 #define FWD_CLK(v) const long long v = clock64()
@@ -89,25 +91,35 @@ __device__ __forceinline__ float2 ex2_fma2(float2 x) {
 constexpr int kCsThreads = 320;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..9: epilogue
 constexpr int kCsQStages = 2;
 constexpr int kCsTmemCols = 256;  // two accumulator buffers of 128 columns
+constexpr int kCsStatBufs = 8;    // buffers of per-query statistics (at least five, see CsShared)
 
 struct CsShared {
   uint64_t k_full, k_empty;
   uint64_t q_full[kCsQStages], q_empty[kCsQStages];
   uint64_t acc_full[2], acc_empty[2];
-  uint64_t nl_full[2];  // 128 epilogue threads have staged the tile's row statistics
+  uint64_t nl_full[kCsStatBufs];  // the producer warp has staged a tile's row statistics
   uint64_t ps_full, ps_empty;  // hand-over of the second query half's partial sums
   uint32_t tmem_base;
   int abort_flag;
   // per query of the tile: -(reference maximum + log2 of the row sum), log2 domain
-  __align__(16) float rstat[2][kTile];
+  // Filled by the producer warp ahead of the epilogue.  No barrier guards the reuse of a buffer: the producer
+  // writes tile t's statistics after Q(t) could be loaded, i.e. after the MMA of tile t-2 completed, which
+  // was issued after every epilogue warp had loaded the scores of tile t-4, i.e. finished summing tile t-5.
+  __align__(16) float rstat[kCsStatBufs][kTile];
   double psum[kTile];
 };
 
-__global__ void __launch_bounds__(kCsThreads)
+__global__ void __launch_bounds__(kCsThreads, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  PrefillScratch s, int n_heads, float scale2, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ CsShared sh;
+  FWD_CLK(e0_);
+#ifdef H2O_PHASE_TIMERS
+  long long e1e_ = 0, e2e_ = 0;
+  unsigned long long gt0_;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0_));
+#endif
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
   unsigned char* k_tile = dyn;                       // [2 boxes][128 rows][128 B]
   unsigned char* q_ring = dyn + kTileBytes;          // [stages][2 boxes][128 rows][128 B]
@@ -135,8 +147,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.acc_full[i], 1);
       mbar_init(&sh.acc_empty[i], 8);  // one arrival per epilogue warp
-      mbar_init(&sh.nl_full[i], 128);
     }
+    for (int i = 0; i < kCsStatBufs; ++i) mbar_init(&sh.nl_full[i], 1);
     mbar_init(&sh.ps_full, 128);
     mbar_init(&sh.ps_empty, 128);
     sh.abort_flag = 0;
@@ -150,27 +162,55 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   volatile int* abort_flag = &sh.abort_flag;
 
   if (warp == 0) {
-    // ---------------- TMA producer ----------------
+    // ---------------- producer: row statistics of each query tile (whole warp), TMA loads (lane 0) ----------------
+    // P[i][j] = 2^(c2 s - m_i) / l_i = 2^(c2 s - (m_i + log2 l_i)): the normaliser is folded into the
+    // exponent's offset, one float per query and no multiplication per score
+    const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
     if (lane == 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
-      for (int t = 0; t < total; ++t) {
+    }
+    bool ok = true;
+    auto tile_ib = [&](int t) { return t < t0 ? jb0 + t : jb1 + (t - t0); };
+    auto fetch = [&](int t, float2 (&raw)[4]) {  // {m, 1 / l} of the tile's 128 queries, four per lane
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int qi = tile_ib(t) * kTile + i * 32 + lane;
+        raw[i] = qi < n ? rowstat[qi] : make_float2(INFINITY, 1.f);  // rows past the end: exp2(-inf) = 0
+      }
+    };
+    float2 raw[4];
+    fetch(0, raw);
+    for (int t = 0; t < total && ok; ++t) {
+      if (lane == 0) {
         const int cb = t < t0 ? 0 : 1;
         const int jb = cb == 0 ? jb0 : jb1;
-        const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
         if (t == 0 || t == t0) {
-          if (cb == 1 && !wait_or_abort(&sh.k_empty, 0, abort_flag)) break;
-          mbar_expect_tx(&sh.k_full, kTileBytes);
-          tma_load_3d(k_tile, &map_k, 0, h, lo + jb * kTile, &sh.k_full);
-          tma_load_3d(k_tile + kBoxBytes, &map_k, 64, h, lo + jb * kTile, &sh.k_full);
+          if (cb == 1) ok = wait_or_abort(&sh.k_empty, 0, abort_flag);
+          if (ok) {
+            mbar_expect_tx(&sh.k_full, kTileBytes);
+            tma_load_3d(k_tile, &map_k, 0, h, lo + jb * kTile, &sh.k_full);
+            tma_load_3d(k_tile + kBoxBytes, &map_k, 64, h, lo + jb * kTile, &sh.k_full);
+          }
         }
         const int st = t % kCsQStages;
-        if (!wait_or_abort(&sh.q_empty[st], ((t / kCsQStages) & 1) ^ 1, abort_flag)) break;
-        unsigned char* dst = q_ring + st * kTileBytes;
-        mbar_expect_tx(&sh.q_full[st], kTileBytes);
-        tma_load_3d(dst, &map_q, 0, h, lo + ib * kTile, &sh.q_full[st]);
-        tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + ib * kTile, &sh.q_full[st]);
+        ok = ok && wait_or_abort(&sh.q_empty[st], ((t / kCsQStages) & 1) ^ 1, abort_flag);
+        if (ok) {
+          unsigned char* dst = q_ring + st * kTileBytes;
+          mbar_expect_tx(&sh.q_full[st], kTileBytes);
+          tma_load_3d(dst, &map_q, 0, h, lo + tile_ib(t) * kTile, &sh.q_full[st]);
+          tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + tile_ib(t) * kTile, &sh.q_full[st]);
+        }
       }
+      // row statistics of tile t (fetched one iteration ago)
+      const int b4 = t % kCsStatBufs;
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) sh.rstat[b4][i * 32 + lane] = log2f(raw[i].y) - raw[i].x;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.nl_full[b4]);
+      if (t + 1 < total) fetch(t + 1, raw);
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
@@ -181,8 +221,14 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         bool ok = true;
         if (t == 0 || t == t0) ok = wait_or_abort(&sh.k_full, cb, abort_flag);
         const int st = t % kCsQStages, b = t & 1;
+        FWD_CLK(m0_);
+        // the tile's row statistics must be staged before its scores are handed to the epilogue: the
+        // epilogue waits for acc_full only (each wait stalls its warps ~200 cycles behind the exponentials)
+        ok = ok && wait_or_abort(&sh.nl_full[t % kCsStatBufs], (uint32_t)(t / kCsStatBufs) & 1u, abort_flag);
         ok = ok && wait_or_abort(&sh.q_full[st], (t / kCsQStages) & 1, abort_flag);
+        FWD_CLK(m1_);
         ok = ok && wait_or_abort(&sh.acc_empty[b], ((t >> 1) & 1) ^ 1, abort_flag);
+        FWD_CLK(m2_);
         if (!__all_sync(0xffffffffu, ok)) break;
         tc_fence_after();
         const uint32_t a0 = smem_u32(k_tile), b0 = smem_u32(q_ring + st * kTileBytes);
@@ -198,6 +244,14 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (t == t0 - 1 && ncb == 2) mma_commit(&sh.k_empty);
         }
         __syncwarp();
+#ifdef H2O_PHASE_TIMERS
+        if (lane == 0) {
+          const long long m3_ = clock64();
+          atomicAdd(&g_cs_prof[5], (unsigned long long)(m1_ - m0_));
+          atomicAdd(&g_cs_prof[6], (unsigned long long)(m2_ - m1_));
+          atomicAdd(&g_cs_prof[7], (unsigned long long)(m3_ - m2_));
+        }
+#endif
       }
     }
   } else {
@@ -208,39 +262,44 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int quarter = warp & 3;            // TMEM lane quarter this warp may access
     const int half = e >> 7;                 // which 64 queries of the tile
     const int row = quarter * 32 + lane;     // key row inside the tile = TMEM lane
-    const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
     double total_sum = 0.0;
-    // P[i][j] = 2^(c2 s - m_i) / l_i = 2^(c2 s - (m_i + log2 l_i)): the normaliser is folded into the
-    // exponent's offset, one float per query and no multiplication per score
-    auto fetch_nlse = [&](int t) -> float {
-      const int ib = t < t0 ? jb0 + t : jb1 + (t - t0);
-      const int qi = ib * kTile + e;
-      if (e >= kTile || qi >= n) return -INFINITY;  // rows past the end: exp2(-inf) = 0
-      const float2 v2 = rowstat[qi];
-      return log2f(v2.y) - v2.x;  // v2 = {m, 1 / l}
-    };
-    float nl_next = fetch_nlse(0);
     bool ok = true;
+#ifdef H2O_PHASE_TIMERS
+    e1e_ = clock64();
+#endif
     for (int t = 0; t < total && ok; ++t) {
+#ifdef H2O_PHASE_TIMERS
+      if (t == 1) e2e_ = clock64();
+#endif
+      const int b3 = t % kCsStatBufs;                // buffer of the row statistics
       const int cb = t < t0 ? 0 : 1;
       const int jb = cb == 0 ? jb0 : jb1;
       const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
       const int b = t & 1;
-      if (e < kTile) {
-        sh.rstat[b][e] = nl_next;
-        mbar_arrive(&sh.nl_full[b]);
-      }
-      if (t + 1 < total) nl_next = fetch_nlse(t + 1);
-      ok = wait_or_abort(&sh.nl_full[b], (t >> 1) & 1, abort_flag) && wait_or_abort(&sh.acc_full[b], (t >> 1) & 1, abort_flag);
+      FWD_CLK(k0_);
+      // One wait per tile: it costs ~200 cycles even when the phase is complete (barrier operations queue
+      // behind the exponentials), and testing the barrier early, in the middle of the arithmetic, only moves
+      // that stall (the warp issues in order and stops at the first use of the answer).  The row statistics
+      // are covered by this wait: the MMA warp saw them staged before it issued the tile.
+      FWD_CLK(k05_);
+      ok = wait_or_abort(&sh.acc_full[b], (t >> 1) & 1, abort_flag);
+
       ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
       if (!ok) break;
       tc_fence_after();
+      FWD_CLK(k1_);
       const uint32_t taddr = tmem + (uint32_t)b * kTile + (uint32_t)half * 64u + ((uint32_t)(quarter * 32) << 16);
-      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b][half * 64]);  // four queries per entry
+      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b3][half * 64]);  // four queries per entry
       uint32_t r0[32], r1[32];
       tmem_ld32(taddr, r0);
+      tmem_ld32(taddr + 32u, r1);
       tmem_wait_ld();
-      tmem_ld32(taddr + 32u, r1);  // in flight while the first 32 columns are processed
+      // the scores are in registers: hand the accumulator back before the arithmetic, so that the tile
+      // after next is computed (issue latency, 512 tensor cycles, commit) while this one is summed
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
+      FWD_CLK(k2_);
       float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       auto chunk = [&](const uint32_t (&r)[32], int c0, bool masked) {
 #pragma unroll
@@ -264,16 +323,21 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       };
       if (ib == jb) {
         chunk(r0, 0, true);
-        tmem_wait_ld();
         chunk(r1, 32, true);
       } else {
         chunk(r0, 0, false);
-        tmem_wait_ld();
         chunk(r1, 32, false);
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
+      FWD_CLK(k3_);
+#ifdef H2O_PHASE_TIMERS
+      if (lane == 0 && warp == 2) {
+        atomicAdd(&g_cs_prof[0], (unsigned long long)(k1_ - k0_));
+        atomicAdd(&g_cs_prof[4], (unsigned long long)(k05_ - k0_));
+        atomicAdd(&g_cs_prof[1], (unsigned long long)(k2_ - k1_));
+        atomicAdd(&g_cs_prof[2], (unsigned long long)(k3_ - k2_));
+        atomicAdd(&g_cs_prof[3], 1ull);
+      }
+#endif
       total_sum += (double)(((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y)) +
                             ((sum2[2].x + sum2[2].y) + (sum2[3].x + sum2[3].y)));
       if (t == t0 - 1 || t == total - 1) {  // last tile of this key block: add the two query halves
@@ -292,6 +356,9 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
   }
+#ifdef H2O_PHASE_TIMERS
+  const long long e3_ = clock64();
+#endif
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(status, 0, H2O_ERR_TIMEOUT);
@@ -299,6 +366,21 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tc_fence_after();
     tmem_dealloc(tmem, kCsTmemCols);
   }
+#ifdef H2O_PHASE_TIMERS
+  if (threadIdx.x == 64) {
+    const long long e4_ = clock64();
+    atomicAdd(&g_cs_blk[0], (unsigned long long)(e1e_ - e0_));
+    atomicAdd(&g_cs_blk[1], (unsigned long long)(e2e_ - e1e_));
+    atomicAdd(&g_cs_blk[2], (unsigned long long)(e3_ - e2e_));
+    atomicAdd(&g_cs_blk[3], (unsigned long long)(e4_ - e3_));
+    atomicAdd(&g_cs_blk[4], 1ull);
+    unsigned long long gt1_;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1_));
+    atomicAdd(&g_cs_blk[5], gt1_ - gt0_);
+    atomicMin(&g_cs_blk[6], gt0_);
+    atomicMax(&g_cs_blk[7], gt1_);
+  }
+#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -722,6 +804,16 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int
 #ifdef H2O_PHASE_TIMERS
 extern "C" int h2o_debug_fwd_timeline(long long* host) {
   return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(g_fwd_tl));
+}
+extern "C" int h2o_debug_cs_prof(unsigned long long* host, int reset) {
+  if (reset) {
+    unsigned long long z[8] = {};
+    unsigned long long zb[8] = {0, 0, 0, 0, 0, 0, ~0ull, 0};
+    cudaMemcpyToSymbol(g_cs_blk, zb, sizeof(zb));
+    return (int)cudaMemcpyToSymbol(g_cs_prof, z, sizeof(z));
+  }
+  cudaMemcpyFromSymbol(host + 8, g_cs_blk, sizeof(unsigned long long) * 8);
+  return (int)cudaMemcpyFromSymbol(host, g_cs_prof, sizeof(unsigned long long) * 8);
 }
 extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
   if (reset) {
