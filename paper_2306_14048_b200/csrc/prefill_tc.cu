@@ -30,8 +30,6 @@ constexpr double kLog2eD = 1.4426950408889634074;
 // Optional cycle accounting of the forward kernel's softmax loop (compile with -DH2O_PHASE_TIMERS).
 #ifdef H2O_PHASE_TIMERS
 __device__ unsigned long long g_fwd_prof[8];
-__device__ unsigned long long g_cs_prof[8];
-__device__ unsigned long long g_cs_blk[8];
 __device__ long long g_fwd_tl[2][40][10];  // block (0, units-1): per group and tile, clock64 at ten events
 #define FWD_TL(g, j, e) do { if (tl_on_ && (j) < 40) g_fwd_tl[g][j][e] = clock64(); } while (0)
 #define FWD_CLK(v) const long long v = clock64()
@@ -92,6 +90,7 @@ constexpr int kCsThreads = 320;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps
 constexpr int kCsQStages = 2;
 constexpr int kCsTmemCols = 256;  // two accumulator buffers of 128 columns
 constexpr int kCsStatBufs = 8;    // buffers of per-query statistics (at least five, see CsShared)
+constexpr int kCsPersistentTiles = 8;  // items of at most this many tiles are walked by persistent blocks
 
 struct CsShared {
   uint64_t k_full, k_empty;
@@ -109,33 +108,62 @@ struct CsShared {
   double psum[kTile];
 };
 
+// Work item: one (unit, pair of key blocks {pi, nb-1-pi}); all items of a unit have nb+1 tiles.  A block
+// walks over items blockIdx.x, blockIdx.x + gridDim.x, ...: barriers, tensor memory and the pipeline stay
+// up from one item to the next, so an item's first loads overlap the previous item's last tiles.
+struct CsItem {
+  int h, lo, n;   // head, first token and length of the sequence
+  int jb0, jb1;   // the two key blocks (jb1 == jb0: one)
+  int t0, total;  // tiles of the first key block, tiles of the item
+};
+struct CsWalk {
+  int w, t;  // item, tile inside the item
+  CsItem it;
+  __device__ __forceinline__ int jb() const { return t < it.t0 ? it.jb0 : it.jb1; }                       // key block
+  __device__ __forceinline__ int ib() const { return t < it.t0 ? it.jb0 + t : it.jb1 + (t - it.t0); }     // query block
+  __device__ __forceinline__ bool first_of_cb() const { return t == 0 || t == it.t0; }
+  __device__ __forceinline__ bool last_of_cb() const { return t == it.t0 - 1 || t == it.total - 1; }
+};
+__device__ __forceinline__ bool cs_item(const PrefillScratch& s, int n_heads, int max_pairs, int w, CsItem& it) {
+  const int u = w / max_pairs, pi = w % max_pairs;
+  const int seq = u / n_heads;
+  it.h = u % n_heads;
+  it.lo = s.cu[seq];
+  it.n = s.cu[seq + 1] - it.lo;
+  const int nb = (it.n + kTile - 1) / kTile;
+  if (pi >= (nb + 1) / 2) return false;
+  it.jb0 = pi;
+  it.jb1 = nb - 1 - pi;
+  it.t0 = nb - it.jb0;  // tiles of key block jb: query blocks jb .. nb-1
+  it.total = it.t0 + (it.jb1 > it.jb0 ? nb - it.jb1 : 0);
+  return true;
+}
+__device__ __forceinline__ bool cs_seek(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
+  while (k.w < n_items && !cs_item(s, n_heads, max_pairs, k.w, k.it)) k.w += (int)gridDim.x;
+  return k.w < n_items;
+}
+__device__ __forceinline__ bool cs_first(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
+  k.w = (int)blockIdx.x;
+  k.t = 0;
+  return cs_seek(s, n_heads, max_pairs, n_items, k);
+}
+__device__ __forceinline__ bool cs_next(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
+  if (++k.t < k.it.total) return true;
+  k.t = 0;
+  k.w += (int)gridDim.x;
+  return cs_seek(s, n_heads, max_pairs, n_items, k);
+}
+
 __global__ void __launch_bounds__(kCsThreads, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 PrefillScratch s, int n_heads, float scale2, int32_t* status) {
+                 PrefillScratch s, int n_heads, int max_pairs, int n_items, float scale2, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ CsShared sh;
-  FWD_CLK(e0_);
-#ifdef H2O_PHASE_TIMERS
-  long long e1e_ = 0, e2e_ = 0;
-  unsigned long long gt0_;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt0_));
-#endif
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
   unsigned char* k_tile = dyn;                       // [2 boxes][128 rows][128 B]
   unsigned char* q_ring = dyn + kTileBytes;          // [stages][2 boxes][128 rows][128 B]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u = blockIdx.y;
-  const int seq = u / n_heads, h = u % n_heads;
-  const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
-  const int nb = (n + kTile - 1) / kTile;
-  const int pi = blockIdx.x;
-  if (pi >= (nb + 1) / 2) return;  // whole block leaves before any barrier or TMEM exists
-  const int jb0 = pi, jb1 = nb - 1 - pi;
-  const int ncb = jb1 > jb0 ? 2 : 1;
-  // tiles of column block jb: row blocks jb .. nb-1
-  const int t0 = nb - jb0;                        // tiles of the first column block
-  const int total = t0 + (ncb == 2 ? nb - jb1 : 0);
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.k_full, 1);
@@ -160,99 +188,95 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
   volatile int* abort_flag = &sh.abort_flag;
+  // every role walks over the same tiles; g counts them (ring stages, buffers and barrier phases follow g)
 
   if (warp == 0) {
     // ---------------- producer: row statistics of each query tile (whole warp), TMA loads (lane 0) ----------------
     // P[i][j] = 2^(c2 s - m_i) / l_i = 2^(c2 s - (m_i + log2 l_i)): the normaliser is folded into the
     // exponent's offset, one float per query and no multiplication per score
-    const float2* rowstat = s.rowstat + (int64_t)h * s.total_tokens + lo;
     if (lane == 0) {
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
     }
-    bool ok = true;
-    auto tile_ib = [&](int t) { return t < t0 ? jb0 + t : jb1 + (t - t0); };
-    auto fetch = [&](int t, float2 (&raw)[4]) {  // {m, 1 / l} of the tile's 128 queries, four per lane
+    auto fetch = [&](const CsWalk& k, float2 (&raw)[4]) {  // {m, 1 / l} of the tile's 128 queries, four per lane
+      const float2* rowstat = s.rowstat + (int64_t)k.it.h * s.total_tokens + k.it.lo;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int qi = tile_ib(t) * kTile + i * 32 + lane;
-        raw[i] = qi < n ? rowstat[qi] : make_float2(INFINITY, 1.f);  // rows past the end: exp2(-inf) = 0
+        const int qi = k.ib() * kTile + i * 32 + lane;
+        raw[i] = qi < k.it.n ? rowstat[qi] : make_float2(INFINITY, 1.f);  // rows past the end: exp2(-inf) = 0
       }
     };
+    CsWalk cur;
+    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
     float2 raw[4];
-    fetch(0, raw);
-    for (int t = 0; t < total && ok; ++t) {
+    if (have) fetch(cur, raw);
+    bool ok = true;
+    for (int g = 0, kc = 0; have && ok; ++g) {
+      const bool new_k = cur.first_of_cb();
       if (lane == 0) {
-        const int cb = t < t0 ? 0 : 1;
-        const int jb = cb == 0 ? jb0 : jb1;
-        if (t == 0 || t == t0) {
-          if (cb == 1) ok = wait_or_abort(&sh.k_empty, 0, abort_flag);
+        if (new_k) {
+          // the single K buffer: the previous key block's last MMA must have read it
+          if (kc >= 1) ok = wait_or_abort(&sh.k_empty, (uint32_t)(kc - 1) & 1u, abort_flag);
           if (ok) {
             mbar_expect_tx(&sh.k_full, kTileBytes);
-            tma_load_3d(k_tile, &map_k, 0, h, lo + jb * kTile, &sh.k_full);
-            tma_load_3d(k_tile + kBoxBytes, &map_k, 64, h, lo + jb * kTile, &sh.k_full);
+            tma_load_3d(k_tile, &map_k, 0, cur.it.h, cur.it.lo + cur.jb() * kTile, &sh.k_full);
+            tma_load_3d(k_tile + kBoxBytes, &map_k, 64, cur.it.h, cur.it.lo + cur.jb() * kTile, &sh.k_full);
           }
         }
-        const int st = t % kCsQStages;
-        ok = ok && wait_or_abort(&sh.q_empty[st], ((t / kCsQStages) & 1) ^ 1, abort_flag);
+        const int st = g % kCsQStages;
+        ok = ok && wait_or_abort(&sh.q_empty[st], ((uint32_t)(g / kCsQStages) & 1u) ^ 1u, abort_flag);
         if (ok) {
           unsigned char* dst = q_ring + st * kTileBytes;
           mbar_expect_tx(&sh.q_full[st], kTileBytes);
-          tma_load_3d(dst, &map_q, 0, h, lo + tile_ib(t) * kTile, &sh.q_full[st]);
-          tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + tile_ib(t) * kTile, &sh.q_full[st]);
+          tma_load_3d(dst, &map_q, 0, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
+          tma_load_3d(dst + kBoxBytes, &map_q, 64, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
         }
       }
-      // row statistics of tile t (fetched one iteration ago)
-      const int b4 = t % kCsStatBufs;
+      if (new_k) ++kc;
+      // row statistics of this tile (fetched one iteration ago)
+      const int b8 = g % kCsStatBufs;
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) sh.rstat[b4][i * 32 + lane] = log2f(raw[i].y) - raw[i].x;
+      for (int i = 0; i < 4; ++i) sh.rstat[b8][i * 32 + lane] = log2f(raw[i].y) - raw[i].x;
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.nl_full[b4]);
-      if (t + 1 < total) fetch(t + 1, raw);
+      if (lane == 0) mbar_arrive(&sh.nl_full[b8]);
+      have = cs_next(s, n_heads, max_pairs, n_items, cur);
+      if (have) fetch(cur, raw);
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
-    {
-      constexpr uint32_t idesc = instr_desc_f16(kTile, kTile, kFmtBF16, kFmtBF16, false, false);
-      for (int t = 0; t < total; ++t) {
-        const int cb = t < t0 ? 0 : 1;
-        bool ok = true;
-        if (t == 0 || t == t0) ok = wait_or_abort(&sh.k_full, cb, abort_flag);
-        const int st = t % kCsQStages, b = t & 1;
-        FWD_CLK(m0_);
-        // the tile's row statistics must be staged before its scores are handed to the epilogue: the
-        // epilogue waits for acc_full only (each wait stalls its warps ~200 cycles behind the exponentials)
-        ok = ok && wait_or_abort(&sh.nl_full[t % kCsStatBufs], (uint32_t)(t / kCsStatBufs) & 1u, abort_flag);
-        ok = ok && wait_or_abort(&sh.q_full[st], (t / kCsQStages) & 1, abort_flag);
-        FWD_CLK(m1_);
-        ok = ok && wait_or_abort(&sh.acc_empty[b], ((t >> 1) & 1) ^ 1, abort_flag);
-        FWD_CLK(m2_);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        tc_fence_after();
-        const uint32_t a0 = smem_u32(k_tile), b0 = smem_u32(q_ring + st * kTileBytes);
-        if (elect_one()) {
-#pragma unroll
-          for (int ks = 0; ks < kD / 16; ++ks) {
-            const uint32_t off = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
-            mma_ss(tmem + (uint32_t)b * kTile, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
-                   idesc, ks > 0);
-          }
-          mma_commit(&sh.q_empty[st]);   // the Q stage may be refilled once these MMAs have read it
-          mma_commit(&sh.acc_full[b]);   // and the accumulator is ready for the epilogue
-          if (t == t0 - 1 && ncb == 2) mma_commit(&sh.k_empty);
-        }
-        __syncwarp();
-#ifdef H2O_PHASE_TIMERS
-        if (lane == 0) {
-          const long long m3_ = clock64();
-          atomicAdd(&g_cs_prof[5], (unsigned long long)(m1_ - m0_));
-          atomicAdd(&g_cs_prof[6], (unsigned long long)(m2_ - m1_));
-          atomicAdd(&g_cs_prof[7], (unsigned long long)(m3_ - m2_));
-        }
-#endif
+    constexpr uint32_t idesc = instr_desc_f16(kTile, kTile, kFmtBF16, kFmtBF16, false, false);
+    CsWalk cur;
+    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
+    for (int g = 0, kc = 0; have; ++g) {
+      bool ok = true;
+      if (cur.first_of_cb()) {
+        ok = wait_or_abort(&sh.k_full, (uint32_t)kc & 1u, abort_flag);
+        ++kc;
       }
+      const int st = g % kCsQStages, b = g & 1;
+      // the tile's row statistics must be staged before its scores are handed to the epilogue: the
+      // epilogue waits for acc_full only (each wait stalls its warps ~200 cycles behind the exponentials)
+      ok = ok && wait_or_abort(&sh.nl_full[g % kCsStatBufs], (uint32_t)(g / kCsStatBufs) & 1u, abort_flag);
+      ok = ok && wait_or_abort(&sh.q_full[st], (uint32_t)(g / kCsQStages) & 1u, abort_flag);
+      ok = ok && wait_or_abort(&sh.acc_empty[b], ((uint32_t)(g >> 1) & 1u) ^ 1u, abort_flag);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tc_fence_after();
+      const uint32_t a0 = smem_u32(k_tile), b0 = smem_u32(q_ring + st * kTileBytes);
+      if (elect_one()) {
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t off = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+          mma_ss(tmem + (uint32_t)b * kTile, smem_desc_sw128(a0 + off, 16, 1024), smem_desc_sw128(b0 + off, 16, 1024),
+                 idesc, ks > 0);
+        }
+        mma_commit(&sh.q_empty[st]);   // the Q stage may be refilled once these MMAs have read it
+        mma_commit(&sh.acc_full[b]);   // and the accumulator is ready for the epilogue
+        if (cur.last_of_cb()) mma_commit(&sh.k_empty);
+      }
+      __syncwarp();
+      have = cs_next(s, n_heads, max_pairs, n_items, cur);
     }
   } else {
     // ---------------- epilogue: exp and in-thread column sums ----------------
@@ -264,32 +288,21 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = quarter * 32 + lane;     // key row inside the tile = TMEM lane
     double total_sum = 0.0;
     bool ok = true;
-#ifdef H2O_PHASE_TIMERS
-    e1e_ = clock64();
-#endif
-    for (int t = 0; t < total && ok; ++t) {
-#ifdef H2O_PHASE_TIMERS
-      if (t == 1) e2e_ = clock64();
-#endif
-      const int b3 = t % kCsStatBufs;                // buffer of the row statistics
-      const int cb = t < t0 ? 0 : 1;
-      const int jb = cb == 0 ? jb0 : jb1;
-      const int ib = cb == 0 ? jb0 + t : jb1 + (t - t0);
-      const int b = t & 1;
-      FWD_CLK(k0_);
+    CsWalk cur;
+    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
+    for (int g = 0, cbc = 0; have && ok; ++g) {  // cbc: key blocks finished so far
+      const int b = g & 1;
+      const int b8 = g % kCsStatBufs;                // buffer of the row statistics
       // One wait per tile: it costs ~200 cycles even when the phase is complete (barrier operations queue
       // behind the exponentials), and testing the barrier early, in the middle of the arithmetic, only moves
       // that stall (the warp issues in order and stops at the first use of the answer).  The row statistics
       // are covered by this wait: the MMA warp saw them staged before it issued the tile.
-      FWD_CLK(k05_);
-      ok = wait_or_abort(&sh.acc_full[b], (t >> 1) & 1, abort_flag);
-
+      ok = wait_or_abort(&sh.acc_full[b], (uint32_t)(g >> 1) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);  // the TMEM loads below are warp-collective
       if (!ok) break;
       tc_fence_after();
-      FWD_CLK(k1_);
       const uint32_t taddr = tmem + (uint32_t)b * kTile + (uint32_t)half * 64u + ((uint32_t)(quarter * 32) << 16);
-      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b3][half * 64]);  // four queries per entry
+      const float4* st4 = reinterpret_cast<const float4*>(&sh.rstat[b8][half * 64]);  // four queries per entry
       uint32_t r0[32], r1[32];
       tmem_ld32(taddr, r0);
       tmem_ld32(taddr + 32u, r1);
@@ -299,7 +312,6 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[b]);
-      FWD_CLK(k2_);
       float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
       auto chunk = [&](const uint32_t (&r)[32], int c0, bool masked) {
 #pragma unroll
@@ -321,44 +333,36 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           sum2[(c4 >> 2) & 3] = __fadd2_rn(sum2[(c4 >> 2) & 3], __fadd2_rn(pa, pb));
         }
       };
-      if (ib == jb) {
+      if (cur.ib() == cur.jb()) {
         chunk(r0, 0, true);
         chunk(r1, 32, true);
       } else {
         chunk(r0, 0, false);
         chunk(r1, 32, false);
       }
-      FWD_CLK(k3_);
-#ifdef H2O_PHASE_TIMERS
-      if (lane == 0 && warp == 2) {
-        atomicAdd(&g_cs_prof[0], (unsigned long long)(k1_ - k0_));
-        atomicAdd(&g_cs_prof[4], (unsigned long long)(k05_ - k0_));
-        atomicAdd(&g_cs_prof[1], (unsigned long long)(k2_ - k1_));
-        atomicAdd(&g_cs_prof[2], (unsigned long long)(k3_ - k2_));
-        atomicAdd(&g_cs_prof[3], 1ull);
-      }
-#endif
       total_sum += (double)(((sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y)) +
                             ((sum2[2].x + sum2[2].y) + (sum2[3].x + sum2[3].y)));
-      if (t == t0 - 1 || t == total - 1) {  // last tile of this key block: add the two query halves
+      if (cur.last_of_cb()) {  // last tile of this key block: add the two query halves
         if (half == 1) {
-          sh.psum[row] = total_sum;
-          mbar_arrive(&sh.ps_full);
+          // the previous key block's partial sums must have been taken
+          if (cbc >= 1) ok = wait_or_abort(&sh.ps_empty, (uint32_t)(cbc - 1) & 1u, abort_flag);
+          if (ok) {
+            sh.psum[row] = total_sum;
+            mbar_arrive(&sh.ps_full);
+          }
         } else {
-          ok = wait_or_abort(&sh.ps_full, cb, abort_flag);
-          const int key = jb * kTile + row;
-          if (ok && key < n) s.acc0[(int64_t)h * s.total_tokens + lo + key] = total_sum + sh.psum[row];
+          ok = wait_or_abort(&sh.ps_full, (uint32_t)cbc & 1u, abort_flag);
+          const int key = cur.jb() * kTile + row;
+          if (ok && key < cur.it.n) s.acc0[(int64_t)cur.it.h * s.total_tokens + cur.it.lo + key] = total_sum + sh.psum[row];
           if (ok) mbar_arrive(&sh.ps_empty);
         }
-        if (half == 1 && cb == 0 && ncb == 2) ok = wait_or_abort(&sh.ps_empty, 0, abort_flag);
         ok = __all_sync(0xffffffffu, ok);  // keep the warp together for the next tile's collectives
         total_sum = 0.0;
+        ++cbc;
       }
+      have = cs_next(s, n_heads, max_pairs, n_items, cur);
     }
   }
-#ifdef H2O_PHASE_TIMERS
-  const long long e3_ = clock64();
-#endif
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(status, 0, H2O_ERR_TIMEOUT);
@@ -366,21 +370,6 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     tc_fence_after();
     tmem_dealloc(tmem, kCsTmemCols);
   }
-#ifdef H2O_PHASE_TIMERS
-  if (threadIdx.x == 64) {
-    const long long e4_ = clock64();
-    atomicAdd(&g_cs_blk[0], (unsigned long long)(e1e_ - e0_));
-    atomicAdd(&g_cs_blk[1], (unsigned long long)(e2e_ - e1e_));
-    atomicAdd(&g_cs_blk[2], (unsigned long long)(e3_ - e2e_));
-    atomicAdd(&g_cs_blk[3], (unsigned long long)(e4_ - e3_));
-    atomicAdd(&g_cs_blk[4], 1ull);
-    unsigned long long gt1_;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt1_));
-    atomicAdd(&g_cs_blk[5], gt1_ - gt0_);
-    atomicMin(&g_cs_blk[6], gt0_);
-    atomicMax(&g_cs_blk[7], gt1_);
-  }
-#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -805,16 +794,6 @@ bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int
 extern "C" int h2o_debug_fwd_timeline(long long* host) {
   return (int)cudaMemcpyFromSymbol(host, g_fwd_tl, sizeof(g_fwd_tl));
 }
-extern "C" int h2o_debug_cs_prof(unsigned long long* host, int reset) {
-  if (reset) {
-    unsigned long long z[8] = {};
-    unsigned long long zb[8] = {0, 0, 0, 0, 0, 0, ~0ull, 0};
-    cudaMemcpyToSymbol(g_cs_blk, zb, sizeof(zb));
-    return (int)cudaMemcpyToSymbol(g_cs_prof, z, sizeof(z));
-  }
-  cudaMemcpyFromSymbol(host + 8, g_cs_blk, sizeof(unsigned long long) * 8);
-  return (int)cudaMemcpyFromSymbol(host, g_cs_prof, sizeof(unsigned long long) * 8);
-}
 extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
   if (reset) {
     unsigned long long z[8] = {};
@@ -856,6 +835,21 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
   return launch_fwd_g<2>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
 }
 
+namespace {
+// SMs of the current device (asked once per device)
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+}  // namespace
+
 bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 && head_dim == kD && encode_fn() != nullptr; }
 
 cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
@@ -870,8 +864,16 @@ cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int ma
     if (e != cudaSuccess) return e;
   }
   const int nb = (max_seqlen + kTile - 1) / kTile;
-  dim3 grid((unsigned)((nb + 1) / 2), (unsigned)c.units);
-  colsum_tc_kernel<<<grid, kCsThreads, smem, stream>>>(map_q, map_k, s, c.n_heads, make_scale2(c.scale), c.status);
+  const int max_pairs = (nb + 1) / 2, n_items = max_pairs * c.units;
+  if (n_items == 0) return cudaSuccess;
+  // Short prompts (few tiles per item): persistent blocks, two per SM (256 TMEM columns, 97 KB of shared
+  // memory each), so that an item's fixed cost (first loads, pipeline fill) overlaps the previous item's
+  // last tiles: config 3 (five tiles per item) 273 -> 250 us.  Long items run one per block and leave the
+  // balancing to the hardware scheduler (config 2, 17 tiles per item: 212 us against 216 us persistent).
+  const bool persistent = nb + 1 <= kCsPersistentTiles && n_items > 2 * sm_count();
+  const int blocks = persistent ? 2 * sm_count() : n_items;
+  colsum_tc_kernel<<<blocks, kCsThreads, smem, stream>>>(map_q, map_k, s, c.n_heads, max_pairs, n_items,
+                                                         make_scale2(c.scale), c.status);
   return cudaGetLastError();
 }
 
