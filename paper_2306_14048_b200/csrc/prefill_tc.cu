@@ -40,6 +40,31 @@ __device__ long long g_fwd_tl[2][40][10];  // block (0, units-1): per group and 
 #define FWD_TL(g, j, e) do { } while (0)
 #endif
 
+// 32 output columns of one query row: accumulator values times 1 / row sum, as bf16.  A thread owns a row, so
+// a warp's store instruction touches 32 different rows; 32-byte stores (whole sectors) halve the number of
+// instructions and transactions against 16-byte ones.  `wide` = the output base is 32-byte aligned.
+__device__ __forceinline__ void store_out_32(__nv_bfloat16* dst, const uint32_t (&o)[32], float inv_l, bool wide) {
+  if (wide) {
+#pragma unroll
+    for (int c16 = 0; c16 < 2; ++c16) {
+      uint32_t w[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        w[e] = Vec16<__nv_bfloat16>::pack2(__uint_as_float(o[c16 * 16 + 2 * e]) * inv_l,
+                                           __uint_as_float(o[c16 * 16 + 2 * e + 1]) * inv_l);
+      st_global_256(dst + c16 * 16, w);
+    }
+  } else {
+#pragma unroll
+    for (int c8 = 0; c8 < 4; ++c8) {
+      float f[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[c8 * 8 + e]) * inv_l;
+      Vec16<__nv_bfloat16>::store(dst + c8 * 8, f);
+    }
+  }
+}
+
 // ---- abortable waits: the first role that times out raises a flag every other wait observes ----
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
@@ -219,8 +244,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           if (kc >= 1) ok = wait_or_abort(&sh.k_empty, (uint32_t)(kc - 1) & 1u, abort_flag);
           if (ok) {
             mbar_expect_tx(&sh.k_full, kTileBytes);
-            tma_load_3d(k_tile, &map_k, 0, cur.it.h, cur.it.lo + cur.jb() * kTile, &sh.k_full);
-            tma_load_3d(k_tile + kBoxBytes, &map_k, 64, cur.it.h, cur.it.lo + cur.jb() * kTile, &sh.k_full);
+            tma_load_tile(k_tile, &map_k, cur.it.h, cur.it.lo + cur.jb() * kTile, &sh.k_full);
           }
         }
         const int st = g % kCsQStages;
@@ -228,8 +252,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (ok) {
           unsigned char* dst = q_ring + st * kTileBytes;
           mbar_expect_tx(&sh.q_full[st], kTileBytes);
-          tma_load_3d(dst, &map_q, 0, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
-          tma_load_3d(dst + kBoxBytes, &map_q, 64, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
+          tma_load_tile(dst, &map_q, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
         }
       }
       if (new_k) ++kc;
@@ -433,6 +456,7 @@ __global__ void __launch_bounds__(fw_threads(G), G == 2 ? 1 : 2)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, float scale2,
               __nv_bfloat16* __restrict__ out, int32_t* status) {
+  const bool wide_out = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FwShared sh;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
@@ -499,8 +523,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       for (int g = 0; g < (hasB ? 2 : 1); ++g) {
         unsigned char* dst = q_tiles + g * kTileBytes;
         mbar_expect_tx(&sh.q_full[g], kTileBytes);
-        tma_load_3d(dst, &map_q, 0, h, lo + (ibA + g) * kTile, &sh.q_full[g]);
-        tma_load_3d(dst + kBoxBytes, &map_q, 64, h, lo + (ibA + g) * kTile, &sh.q_full[g]);
+        tma_load_tile(dst, &map_q, h, lo + (ibA + g) * kTile, &sh.q_full[g]);
       }
       for (int r = 0; r < 2 * nt; ++r) {
         const int slot = r % kFwKvSlots;
@@ -509,8 +532,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         unsigned char* dst = kv_ring + slot * kFwKvSlotBytes;
         const int row0 = lo + (r >> 1) * kFwKeys;
         mbar_expect_tx(&sh.kv_full[slot], kFwKvSlotBytes);
-        tma_load_3d(dst, map, 0, h, row0, &sh.kv_full[slot]);
-        tma_load_3d(dst + kFwKvSlotBytes / 2, map, 64, h, row0, &sh.kv_full[slot]);
+        tma_load_tile(dst, map, h, row0, &sh.kv_full[slot]);
       }
     }
   } else if (mma_idx >= 0 && mma_idx < 2 * G) {
@@ -729,15 +751,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
           uint32_t o[32];
           tmem_ld32(tmem_o + (uint32_t)cc * 32u, o);
           tmem_wait_ld();
-          if (qi < n) {
-#pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              float f[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(o[c8 * 8 + e]) * inv_l;
-              Vec16<__nv_bfloat16>::store(orow + cc * 32 + c8 * 8, f);
-            }
-          }
+          if (qi < n) store_out_32(orow + cc * 32, o, inv_l, wide_out);
         }
         if (qi < n) s.rowstat[(int64_t)h * s.total_tokens + lo + qi] = make_float2(m_used, inv_l);
       }
@@ -749,6 +763,393 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, kFwTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward for short prompts: persistent blocks, one softmax group, two blocks per SM
+// ---------------------------------------------------------------------------------------------
+// Same arithmetic, tiles and tensor-memory layout as the one-group instance of the kernel above, but a
+// block walks over work items (unit, query block) instead of ending after one: barriers, tensor memory
+// and the K/V ring stay up, so an item's first loads and score tiles overlap the previous item's last
+// tiles and its output.  With 512-token prompts a block of the kernel above spends more time on its fixed
+// cost (allocation, first loads, pipeline fill, output, exit and relaunch) than on its five tiles.
+// All counters run over the block's whole sequence of key tiles: tile T uses ring slots 2 (T % 2) and
+// + 1, score buffer T % 2 and the issuing warp T % 2; a warp issues P V(T), then S(T + 2), which may
+// belong to the next item.
+constexpr int kFsThreads = 256;  // warp 0 TMA, warps 1, 2 MMA (even, odd tiles), warp 3 idle, warps 4..7 softmax
+constexpr int kFsKvSlots = 4;
+constexpr uint32_t kFsTmemCols = 256;  // O 128 columns, two score / probability buffers of 64
+// register budgets after the block's start with 128 per thread (the issuers keep two tile walkers)
+constexpr int kFsRegsIssue = 88, kFsRegsSoftmax = 168;
+
+struct FsShared {
+  uint64_t q_full, q_empty;  // Q of the item is in shared memory / both issuing warps are done with it
+  uint64_t kv_full[kFsKvSlots], kv_empty[kFsKvSlots];
+  uint64_t s_full[2], p_full[2], pv_done[2];
+  uint64_t o_final;          // both issuing warps' last products of the item are complete
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct FsItem {
+  int h, lo, n;  // head, first token and length of the sequence
+  int ib, nt;    // query block, key tiles
+};
+struct FsWalk {
+  int w;   // item index
+  int j;   // key tile inside the item
+  int T;   // key tiles before this one, over all items of the block
+  int ic;  // items before this one
+  FsItem it;
+};
+__device__ __forceinline__ bool fs_item(const PrefillScratch& s, int n_heads, int nb_max, int w, FsItem& it) {
+  const int u = w / nb_max, x = w % nb_max;
+  const int seq = u / n_heads;
+  it.h = u % n_heads;
+  it.lo = s.cu[seq];
+  it.n = s.cu[seq + 1] - it.lo;
+  const int nb = (it.n + kTile - 1) / kTile;
+  if (x >= nb) return false;
+  it.ib = nb - 1 - x;
+  it.nt = (min(it.n, (it.ib + 1) * kTile) + kFwKeys - 1) / kFwKeys;  // keys 0 .. min(n, (ib+1)*128) - 1
+  return true;
+}
+__device__ __forceinline__ bool fs_seek(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
+  while (k.w < n_items && !fs_item(s, n_heads, nb_max, k.w, k.it)) k.w += (int)gridDim.x;
+  return k.w < n_items;
+}
+__device__ __forceinline__ bool fs_first(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
+  k.w = (int)blockIdx.x;
+  k.j = k.T = k.ic = 0;
+  return fs_seek(s, n_heads, nb_max, n_items, k);
+}
+// next key tile; false after the block's last one
+__device__ __forceinline__ bool fs_next(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
+  ++k.T;
+  if (++k.j < k.it.nt) return true;
+  k.j = 0;
+  ++k.ic;
+  k.w += (int)gridDim.x;
+  return fs_seek(s, n_heads, nb_max, n_items, k);
+}
+
+__global__ void __launch_bounds__(kFsThreads, 2)
+fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, int nb_max, int n_items,
+                    float scale2, __nv_bfloat16* __restrict__ out, int32_t* status) {
+  extern __shared__ unsigned char dyn_raw[];
+  __shared__ FsShared sh;
+  const bool wide_out = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
+  unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
+  unsigned char* q_tile = dyn;                // 32 KB
+  unsigned char* kv_ring = dyn + kTileBytes;  // four slots of 16 KB
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef H2O_PHASE_TIMERS
+  const bool tl_on_ = blockIdx.x == 0 && lane == 0 && (warp == 1 || warp == 2 || warp == 4);
+#endif
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sh.q_full, 1);
+    mbar_init(&sh.q_empty, 2);
+    for (int i = 0; i < kFsKvSlots; ++i) {
+      mbar_init(&sh.kv_full[i], 1);
+      mbar_init(&sh.kv_empty[i], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sh.s_full[b], 1);
+      mbar_init(&sh.p_full[b], 4);
+      mbar_init(&sh.pv_done[b], 1);
+    }
+    mbar_init(&sh.o_final, 2);
+    sh.abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sh.tmem_base, kFsTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  volatile int* abort_flag = &sh.abort_flag;
+  const bool softmax_warp = warp >= 4;
+
+  // One branch per register budget (the groups of four warps change theirs right at its top, so that
+  // the compiler sees which code runs under which budget).
+  if (!softmax_warp) {
+  setmaxnreg_dec<kFsRegsIssue>();
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      prefetch_tensormap(&map_v);
+      FsWalk k;
+      bool have = fs_first(s, n_heads, nb_max, n_items, k);
+      bool ok = true;
+      while (have && ok) {
+        if (k.j == 0) {  // new item: its Q tile, once both issuing warps are done with the previous one
+          if (k.ic >= 1) ok = wait_or_abort(&sh.q_empty, (uint32_t)(k.ic - 1) & 1u, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(&sh.q_full, kTileBytes);
+          tma_load_tile(q_tile, &map_q, k.it.h, k.it.lo + k.it.ib * kTile, &sh.q_full);
+        }
+        const int slot = 2 * (k.T & 1);
+        const uint32_t par = ((uint32_t)(k.T >> 1) & 1u) ^ 1u;
+        const int row0 = k.it.lo + k.j * kFwKeys;
+#pragma unroll
+        for (int r = 0; r < 2 && ok; ++r) {
+          ok = wait_or_abort(&sh.kv_empty[slot + r], par, abort_flag);
+          if (!ok) break;
+          const CUtensorMap* map = r ? &map_v : &map_k;
+          unsigned char* dst = kv_ring + (slot + r) * kFwKvSlotBytes;
+          mbar_expect_tx(&sh.kv_full[slot + r], kFwKvSlotBytes);
+          tma_load_tile(dst, map, k.it.h, row0, &sh.kv_full[slot + r]);
+        }
+        have = fs_next(s, n_heads, nb_max, n_items, k);
+      }
+    }
+  } else if (warp == 1 || warp == 2) {
+    // ---------------- MMA issuers: warp 1 the even key tiles, warp 2 the odd ones ----------------
+    constexpr uint32_t idesc_s = instr_desc_f16(kTile, kFwKeys, kFmtBF16, kFmtBF16, false, false);
+    constexpr uint32_t idesc_o = instr_desc_f16(kTile, kD, kFmtBF16, kFmtBF16, false, true);
+    const int par = warp - 1;
+    const uint32_t sp = tmem + 128u + (uint32_t)par * 64u;  // this warp's score / probability buffer
+    const uint32_t d_o = tmem;
+    const uint64_t dq = smem_desc_sw128(smem_u32(q_tile), 16, 1024);
+    bool ok = true;
+    // This warp's tiles are T = par, par + 2, ...  It needs only the position inside the item (first,
+    // second, last own tile) and the item count; items in which it has no tile (a single tile, of the
+    // other parity) still get its arrival on the per-item barriers (q_empty from the S walker, o_final
+    // from the P V walker).
+    struct Lean {
+      int w, j, T, ic, nt;
+    };
+    auto lean_seek = [&](Lean& k) {
+      while (k.w < n_items) {
+        const int u = k.w / nb_max, x = k.w - u * nb_max;
+        const int seq = u / n_heads;
+        const int lo_ = s.cu[seq], n_ = s.cu[seq + 1] - lo_;
+        const int nb_ = (n_ + kTile - 1) / kTile;
+        if (x < nb_) {
+          k.nt = (min(n_, (nb_ - x) * kTile) + kFwKeys - 1) / kFwKeys;
+          return true;
+        }
+        k.w += (int)gridDim.x;
+      }
+      return false;
+    };
+    auto lean_next = [&](Lean& k) {
+      ++k.T;
+      if (++k.j < k.nt) return true;
+      k.j = 0;
+      ++k.ic;
+      k.w += (int)gridDim.x;
+      return lean_seek(k);
+    };
+    // from a tile of the other parity (an item of one tile gets the direct arrival) to the next own tile
+    auto skip_other = [&](Lean& k, bool& have, uint64_t* item_bar) {
+      if (k.nt == 1 && lane == 0) mbar_arrive(item_bar);
+      have = lean_next(k);
+    };
+    Lean ks_{(int)blockIdx.x, 0, 0, 0, 0}, kp_{(int)blockIdx.x, 0, 0, 0, 0};
+    bool have_s = lean_seek(ks_);
+    if (have_s && par == 1) skip_other(ks_, have_s, &sh.q_empty);
+    bool have_p = lean_seek(kp_);
+    if (have_p && par == 1) skip_other(kp_, have_p, &sh.o_final);
+    int q_seen = -1;  // last item whose Q this warp has waited for
+    // The S walker runs one own tile ahead of the P V walker: S(T + 2) is issued right behind P V(T) by
+    // the same thread, and its buffer is the one that product reads (the tensor core runs one thread's
+    // instructions in order).
+    for (bool first = true; ok; first = false) {
+      if (!first) {
+        if (!have_p) break;
+        // ---- O += P(T) V_T ----
+        const int T = kp_.T, j = kp_.j;
+        const int slot = 2 * (T & 1) + 1;
+        // the item's first product initialises O: the other warp's product of tile 1 must not overtake it
+        if (j == 1) ok = ok && wait_or_abort(&sh.pv_done[par ^ 1], (uint32_t)((T - 1) >> 1) & 1u, abort_flag);
+        ok = ok && wait_or_abort(&sh.p_full[par], (uint32_t)(T >> 1) & 1u, abort_flag);
+        ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(T >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok) != 0;
+        if (!ok) break;
+        tc_fence_after();
+        FWD_TL(0, T, 2);
+        const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+        if (elect_one()) {
+          // (P(0) of an item is stored only after the softmax warps have read the previous item's O)
+          if (j == 0) mma_ts_lohi<false>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
+          else mma_ts_lohi<true>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
+#pragma unroll
+          for (int ks = 1; ks < (kFwSplitP ? 2 : 1) * (kFwKeys / 16); ++ks) {  // hi columns (, then lo columns)
+            const uint32_t kk = (uint32_t)(ks & 3);
+            mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
+          }
+          mma_commit(&sh.pv_done[par]);
+          if (j + 2 >= kp_.nt) mma_commit(&sh.o_final);  // this warp's last product of the item
+          mma_commit(&sh.kv_empty[slot]);
+          FWD_TL(0, T, 4);
+        }
+        __syncwarp();
+        have_p = lean_next(kp_);
+        if (have_p) skip_other(kp_, have_p, &sh.o_final);
+      }
+      if (have_s) {
+        // ---- S(T) = Q K_T^T ----
+        const int T = ks_.T;
+        if (ks_.ic != q_seen) {
+          ok = ok && wait_or_abort(&sh.q_full, (uint32_t)ks_.ic & 1u, abort_flag);
+          q_seen = ks_.ic;
+        }
+        const int slot = 2 * (T & 1);
+        ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(T >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok) != 0;
+        if (!ok) break;
+        tc_fence_after();
+        FWD_TL(0, T, 5);
+        const uint64_t dk = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), 16, 1024);
+        if (elect_one()) {
+#pragma unroll
+          for (int ks = 0; ks < kD / 16; ++ks) {
+            const uint32_t qoff = (uint32_t)(ks >> 2) * kBoxBytes + (uint32_t)(ks & 3) * 32u;
+            const uint32_t koff = (uint32_t)(ks >> 2) * (kFwKvSlotBytes / 2) + (uint32_t)(ks & 3) * 32u;
+            if (ks == 0)
+              mma_ss_lohi<false>(sp, desc_lo(dq), desc_hi(dq), desc_lo(dk), desc_hi(dk), idesc_s);
+            else
+              mma_ss_lohi<true>(sp, desc_lo(dq) + (qoff >> 4), desc_hi(dq), desc_lo(dk) + (koff >> 4), desc_hi(dk), idesc_s);
+          }
+          mma_commit(&sh.s_full[par]);
+          mma_commit(&sh.kv_empty[slot]);
+          if (ks_.j + 2 >= ks_.nt) mma_commit(&sh.q_empty);  // this warp's last score tile of the item
+          FWD_TL(0, T, 0);
+        }
+        __syncwarp();
+        have_s = lean_next(ks_);
+        if (have_s) skip_other(ks_, have_s, &sh.q_empty);
+      } else if (first) {
+        break;
+      }
+    }
+  }
+  } else {
+    setmaxnreg_inc<kFsRegsSoftmax>();
+    // ---------------- softmax: one thread per query row ----------------
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tmem_o = tmem + lane_addr;
+    const uint32_t tmem_sp = tmem + 128u + lane_addr;  // + 64 (T & 1)
+    bool ok = true;
+    float m_used = -INFINITY;
+    float2 l2 = make_float2(0.f, 0.f);  // row sum, even and odd keys apart (packed fp32x2 adds)
+    FsItem it;
+    int T = 0;  // key tiles so far, over all items
+    for (int w = (int)blockIdx.x, ic = 0; ok; w += (int)gridDim.x, ++ic) {
+      while (w < n_items && !fs_item(s, n_heads, nb_max, w, it)) w += (int)gridDim.x;
+      if (w >= n_items) break;
+      const int qi = it.ib * kTile + row;  // query position inside the sequence
+      for (int j = 0; j < it.nt && ok; ++j, ++T) {
+      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[T & 1], (uint32_t)(T >> 1) & 1u, abort_flag));  // collectives below
+      if (!ok) break;
+      tc_fence_after();
+      FWD_TL(0, T, 1);
+      const uint32_t buf = tmem_sp + (uint32_t)(T & 1) * 64u;
+      uint32_t r0[32], r1[32];
+      tmem_ld32(buf, r0);
+      tmem_ld32(buf + 32u, r1);
+      tmem_wait_ld();
+      const int key0 = j * kFwKeys;
+      const bool masked_tile = key0 + kFwKeys - 1 > it.ib * kTile;  // tile reaches past this block's first query
+      if (masked_tile) {
+#pragma unroll
+        for (int c2 = 0; c2 < kFwKeys; ++c2)
+          if (key0 + c2 > qi) (c2 < 32 ? r0[c2] : r1[c2 - 32]) = 0xff800000u;  // -inf, causal: key <= query
+      }
+      float m_raw = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < kFwKeys; c2 += 2)
+        m_raw = max3(m_raw, __uint_as_float(c2 < 32 ? r0[c2] : r1[c2 - 32]),
+                     __uint_as_float(c2 < 32 ? r0[c2 + 1] : r1[c2 - 31]));
+      const float m_tile = m_raw * scale2;
+      const bool need = m_tile > m_used + kRescaleThreshold;
+      if (j == 0) {
+        m_used = m_tile;  // key 0 is visible to every row, so this is finite
+        l2 = make_float2(0.f, 0.f);
+      } else {
+        const bool rescale = __any_sync(0xffffffffu, need);
+        if (rescale) {
+          // O must include tile T-1 before it is rescaled
+          ok = __all_sync(0xffffffffu, wait_or_abort(&sh.pv_done[(T - 1) & 1], (uint32_t)((T - 1) >> 1) & 1u, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          const float m_new = need ? m_tile : m_used;
+          const float alpha = ex2(m_used - m_new);
+          l2 = __fmul2_rn(l2, make_float2(alpha, alpha));
+          m_used = m_new;
+#pragma unroll
+          for (int cc = 0; cc < kD / 32; ++cc) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + (uint32_t)cc * 32u, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c2 = 0; c2 < 32; ++c2) o[c2] = __float_as_uint(__uint_as_float(o[c2]) * alpha);
+            tmem_st32(tmem_o + (uint32_t)cc * 32u, o);
+          }
+          tmem_wait_st();
+        }
+      }
+      const float neg_m = -m_used;
+      uint32_t hw[32];
+      [[maybe_unused]] uint32_t lw[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
+        const float s1 = __uint_as_float(c < 16 ? r0[2 * c + 1] : r1[2 * c - 31]);
+        const float2 x = __ffma2_rn(make_float2(s0, s1), make_float2(scale2, scale2), make_float2(neg_m, neg_m));
+        const float2 pp = make_float2(ex2(x.x), ex2(x.y));
+        l2 = __fadd2_rn(l2, pp);
+        const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pp.x, pp.y);
+        hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
+        if constexpr (kFwSplitP) {
+          const float2 lo = __ffma2_rn(__bfloat1622float2(hi2), make_float2(-1.f, -1.f), pp);  // exact remainder
+          lw[c] = Vec16<__nv_bfloat16>::pack2(lo.x, lo.y);
+        }
+      }
+      tmem_st32(buf, hw);  // over the scores, which are in registers by now
+      if constexpr (kFwSplitP) tmem_st32(buf + 32u, lw);
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.p_full[T & 1]);
+      FWD_TL(0, T, 3);
+      }
+      if (ok) {  // the item's output
+        ok = __all_sync(0xffffffffu, wait_or_abort(&sh.o_final, (uint32_t)ic & 1u, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        FWD_TL(0, T - 1, 6);
+        const float inv_l = 1.0f / (l2.x + l2.y);
+        __nv_bfloat16* orow = out + ((int64_t)(it.lo + qi) * n_heads + it.h) * kD;
+#pragma unroll
+        for (int cc = 0; cc < kD / 32; ++cc) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + (uint32_t)cc * 32u, o);
+          tmem_wait_ld();
+          if (qi < it.n) store_out_32(orow + cc * 32, o, inv_l, wide_out);
+        }
+        if (qi < it.n) s.rowstat[(int64_t)it.h * s.total_tokens + it.lo + qi] = make_float2(m_used, inv_l);
+        // (the next item's first probabilities, which release its first P V and with it the overwrite
+        //  of O, are stored by these same warps after this point)
+        tc_fence_before();
+        FWD_TL(0, T - 1, 7);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && sh.abort_flag) atomicCAS(status, 0, H2O_ERR_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kFsTmemCols);
   }
 }
 
@@ -778,6 +1179,20 @@ float make_scale2(float c) { return (float)((double)c * kLog2eD); }
 }  // namespace
 
 // [total_tokens, n_heads, 128] bf16, box = rows x 1 head x 64 elements (128 bytes), 128-byte swizzle
+// [total_tokens, n_heads, 128] bf16 as {64 elements, tokens, 2 halves, heads}: one box = rows x both halves
+// of one head, 128-byte swizzle, landing as [half][row][128 bytes]
+bool make_whole_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_heads, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {64, (cuuint64_t)total_tokens, 2, (cuuint64_t)n_heads};
+  const cuuint64_t strides[3] = {(cuuint64_t)n_heads * kD * 2, 128, (cuuint64_t)kD * 2};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 2, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_tile_map(CUtensorMap* map, const void* base, int64_t total_tokens, int n_heads, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -804,6 +1219,21 @@ extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
 #endif
 
 namespace {
+// SMs of the current device (asked once per device)
+int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+}  // namespace
+
+namespace {
 
 template <int G>
 cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v, const CacheView& c,
@@ -826,36 +1256,38 @@ cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, con
 cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                           const void* v, void* out, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
-  if (!make_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
-      !make_tile_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
+  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
+      !make_whole_tile_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
   // short prompts: one query block per thread block, two blocks per SM; long ones: two query blocks share
   // every K/V tile
-  if (max_seqlen <= kFwShortPrompt) return launch_fwd_g<1>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
+  if (max_seqlen <= kFwShortPrompt) {
+    const int nb_max = (max_seqlen + kTile - 1) / kTile, n_items = nb_max * c.units;
+    if (n_items == 0) return cudaSuccess;
+    const int smem = kTileBytes + kFsKvSlots * kFwKvSlotBytes + 1024;
+    static unsigned long long attr_flags = 0;
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fwd_tc_short_kernel), smem, &attr_flags);
+    if (e != cudaSuccess) return e;
+    // Items of one unit differ in length (query block ib has 2 (ib + 1) key tiles) and follow one another
+    // in the item order, so the stride with which a block walks over the items must not share a factor
+    // with the number of query blocks, or a block would see the same ib every time.
+    int blocks = n_items < 2 * sm_count() ? n_items : 2 * sm_count();
+    auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
+    while (blocks > 1 && blocks < n_items && gcd(blocks, nb_max) != 1) --blocks;
+    fwd_tc_short_kernel<<<blocks, kFsThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, nb_max, n_items,
+                                                              make_scale2(c.scale), static_cast<__nv_bfloat16*>(out),
+                                                              c.status);
+    return cudaGetLastError();
+  }
   return launch_fwd_g<2>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
 }
-
-namespace {
-// SMs of the current device (asked once per device)
-int sm_count() {
-  static int cached[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (cached[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
-}  // namespace
 
 bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 && head_dim == kD && encode_fn() != nullptr; }
 
 cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                              cudaStream_t stream) {
   CUtensorMap map_q, map_k;
-  if (!make_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_tile_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
+  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
     return cudaErrorInvalidValue;
   const int smem = kTileBytes * (1 + kCsQStages) + 1024;
   static unsigned long long attr_flags = 0;

@@ -17,6 +17,13 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 // One lane of a converged warp (the same lane every time).  The MMA-issuing warp runs its loop with
 // all lanes, so that descriptors and addresses stay warp-uniform (uniform registers), and predicates
 // only the single-thread instructions with this.
+// 32-byte global store (this architecture has 256-bit loads and stores); the address must be 32-byte aligned
+__device__ __forceinline__ void st_global_256(void* p, const uint32_t (&v)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+               "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+               : "memory");
+}
+
 // Register budget of the calling group of four warps (all 128 threads execute it): give registers back
 // to the block's pool, or take them (waits until enough have been given back).
 template <int N>
@@ -92,6 +99,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, i
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
           "r"(smem_u32(dst)),
       "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+      : "memory");
+}
+// One copy for a whole tile of head_dim 128: the map's dimensions are {64 elements, rows, 2 halves of the
+// head dimension, heads}, the box {64, rows, 2, 1}, so shared memory receives [half][row][128 bytes] (each
+// half a 128-byte-swizzled K-major operand block).  The TMA unit takes about as long per copy as per
+// box of half the size, so this doubles what one producer thread can stream.
+__device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int head, int row, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::
+          "r"(smem_u32(dst)),
+      "l"(map), "r"(0), "r"(row), "r"(0), "r"(head), "r"(smem_u32(bar))
       : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
