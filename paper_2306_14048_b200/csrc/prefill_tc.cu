@@ -398,8 +398,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // ---------------------------------------------------------------------------------------------
 // Forward: out = softmax(c Q K^T) V over the causal triangle, plus per-row {max, 1/sum}
 // ---------------------------------------------------------------------------------------------
-// One thread block per (unit, PAIR of 128-query blocks) (short prompts: per single query block); key tiles
-// of 64, loaded once (TMA) for both query blocks.  One softmax group of four warps per query block (A, B)
+// One thread block per (unit, PAIR of 128-query blocks) (short prompts take the persistent kernel further
+// down); key tiles of 64, loaded once (TMA) for both query blocks.  One softmax group of four warps per query block (A, B)
 // and, per group, two MMA-issuing warps (even key tiles, odd key tiles).  Per group g and key tile j:
 //   S_g(j) = Q_g K_j^T           M 128, N 64, K 128; Q and K from shared memory, fp32 accumulator
 //                                in TMEM.  Issued two tiles ahead of the softmax, right behind P V(j-2)
@@ -419,7 +419,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // fourth MMA issuer, 13..15 idle).  The block starts with 128 registers per thread; the issuers give
 // registers back and the softmax warps take them.
 __host__ __device__ constexpr int fw_threads(int groups) { return groups == 2 ? 512 : 256; }
-constexpr int kFwRegsIssue = 72, kFwRegsSoftmax = 168;
+constexpr int kFwRegsIssue = 80, kFwRegsSoftmax = 168;
 constexpr int kFwKeys = 64;                       // keys per tile
 constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
 constexpr int kFwMaxKvSlots = 6;
@@ -449,8 +449,8 @@ struct FwShared {
 };
 
 // G = query blocks (softmax groups) per thread block.  Two share every K/V tile and fill an SM (all of
-// its tensor memory); one per block lets two blocks share an SM, which hides the fixed cost of a block
-// (allocation, first loads, pipeline fill, output) when prompts are short.
+// its tensor memory): the instance that is launched.  (One per block works too, two blocks per SM; for
+// short prompts the persistent kernel below replaced it.)
 template <int G>
 __global__ void __launch_bounds__(fw_threads(G), G == 2 ? 1 : 2)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -512,8 +512,10 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
   // MMA issuer index: (group, tile parity) = (idx % G, idx / G); warps 1..3 and, with two groups, warp 12
   const int mma_idx = (warp >= 1 && warp <= 3) ? warp - 1 : (warp == 12 ? 3 : -1);
   const bool softmax_warp = warp >= 4 && warp < 4 + 4 * G;
-  if (softmax_warp) setmaxnreg_inc<kFwRegsSoftmax>();
-  else setmaxnreg_dec<kFwRegsIssue>();
+  // One branch per register budget (the groups of four warps change theirs right at its top, so that
+  // the compiler sees which code runs under which budget).
+  if (!softmax_warp) {
+  setmaxnreg_dec<kFwRegsIssue>();
   if (warp == 0) {
     // ---------------- TMA producer: Q tiles, then K_0, V_0, K_1, V_1, ... through the slot ring ----
     if (lane == 0) {
@@ -590,8 +592,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // ---- O_g += P_g(j) V_j: needs P_g(j) in tensor memory and V_j in shared memory ----
       const int slot = 2 * (j % kRing) + 1;
       FWD_TL(g, j, 6);
-      // P V(0) initialises O_g: the odd warp's first product must not overtake it
-      if (j == 1) ok = ok && wait_or_abort(&sh.pv_done[g][0], 0, abort_flag);
+      // The products of a group accumulate into O_g in tile order: this one is issued when the previous
+      // tile's (the other warp's) is complete.  That fixes the order of the fp32 additions, so every bit of
+      // the output is the same in every run, and keeps P V(0), which initialises O_g, first.  (In steady
+      // state that product completed a tile time ago: the wait costs its own latency only.)
+      if (j >= 1) ok = ok && wait_or_abort(&sh.pv_done[g][par ^ 1], (uint32_t)((j - 1) >> 1) & 1u, abort_flag);
       ok = ok && wait_or_abort(&sh.p_full[g][par], (uint32_t)(j >> 1) & 1u, abort_flag);
       FWD_TL(g, j, 7);
       ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(j / kRing) & 1u, abort_flag);
@@ -629,7 +634,9 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       if (ok && lane == 0) mbar_arrive(&sh.kv_empty[slot + 1]);
       ok = __all_sync(0xffffffffu, ok) != 0;
     }
-  } else if (softmax_warp) {
+  }
+  } else {
+    setmaxnreg_inc<kFwRegsSoftmax>();
     // ---------------- softmax groups: one thread per query row ----------------
     const int g = (warp - 4) >> 2;             // 0: group A, 1: group B
     const int ib = g == 0 ? ibA : ibB;
@@ -779,6 +786,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 // belong to the next item.
 constexpr int kFsThreads = 256;  // warp 0 TMA, warps 1, 2 MMA (even, odd tiles), warp 3 idle, warps 4..7 softmax
 constexpr int kFsKvSlots = 4;
+constexpr int kFsDescs = 8;
 constexpr uint32_t kFsTmemCols = 256;  // O 128 columns, two score / probability buffers of 64
 // register budgets after the block's start with 128 per thread (the issuers keep two tile walkers)
 constexpr int kFsRegsIssue = 88, kFsRegsSoftmax = 168;
@@ -790,50 +798,52 @@ struct FsShared {
   uint64_t o_final;          // both issuing warps' last products of the item are complete
   uint32_t tmem_base;
   int abort_flag;
+  // The producer thread alone looks items up (two dependent loads and divisions per item); it leaves each
+  // item's description here before it loads the item's Q.  The S walkers wait for q_full of every item
+  // in order and read entry ic % 8 then; the same threads' P V walkers come later; the softmax warps read
+  // it after they have seen the item's first score tile (issued behind that wait).  `last` ends the walk;
+  // a block without items gets nt == 0 in entry 0.  `start` (used once) tells the softmax warps that
+  // entry 0 is there.  (The producer is never more than three items ahead of the slowest reader: Q of
+  // item ic+1 waits for the last scores of item ic.)
+  uint64_t start;
+  struct Desc {
+    int h, lo, n, ib, nt, last;
+  } desc[kFsDescs];
 };
 
 struct FsItem {
   int h, lo, n;  // head, first token and length of the sequence
   int ib, nt;    // query block, key tiles
 };
-struct FsWalk {
-  int w;   // item index
-  int j;   // key tile inside the item
-  int T;   // key tiles before this one, over all items of the block
-  int ic;  // items before this one
-  FsItem it;
+// sequence bounds of item w, loaded ahead of their use (plain loads: nothing branches on them here)
+struct FsAhead {
+  int w, lo, end;
 };
-__device__ __forceinline__ bool fs_item(const PrefillScratch& s, int n_heads, int nb_max, int w, FsItem& it) {
-  const int u = w / nb_max, x = w % nb_max;
-  const int seq = u / n_heads;
+__device__ __forceinline__ FsAhead fs_look(const PrefillScratch& s, int n_heads, int nb_max, int n_items, int w) {
+  FsAhead a{w, 0, 0};
+  if (w < n_items) {
+    const int seq = (w / nb_max) / n_heads;
+    a.lo = s.cu[seq];
+    a.end = s.cu[seq + 1];
+  }
+  return a;
+}
+__device__ __forceinline__ bool fs_make(int n_heads, int nb_max, const FsAhead& a, FsItem& it) {
+  const int u = a.w / nb_max, x = a.w % nb_max;
   it.h = u % n_heads;
-  it.lo = s.cu[seq];
-  it.n = s.cu[seq + 1] - it.lo;
+  it.lo = a.lo;
+  it.n = a.end - a.lo;
   const int nb = (it.n + kTile - 1) / kTile;
   if (x >= nb) return false;
   it.ib = nb - 1 - x;
   it.nt = (min(it.n, (it.ib + 1) * kTile) + kFwKeys - 1) / kFwKeys;  // keys 0 .. min(n, (ib+1)*128) - 1
   return true;
 }
-__device__ __forceinline__ bool fs_seek(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
-  while (k.w < n_items && !fs_item(s, n_heads, nb_max, k.w, k.it)) k.w += (int)gridDim.x;
-  return k.w < n_items;
+// first item at or after a.w (stride gridDim.x) that exists; returns its index (>= n_items: none)
+__device__ __forceinline__ int fs_seek(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsAhead a, FsItem& it) {
+  while (a.w < n_items && !fs_make(n_heads, nb_max, a, it)) a = fs_look(s, n_heads, nb_max, n_items, a.w + (int)gridDim.x);
+  return a.w;
 }
-__device__ __forceinline__ bool fs_first(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
-  k.w = (int)blockIdx.x;
-  k.j = k.T = k.ic = 0;
-  return fs_seek(s, n_heads, nb_max, n_items, k);
-}
-// next key tile; false after the block's last one
-__device__ __forceinline__ bool fs_next(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsWalk& k) {
-  ++k.T;
-  if (++k.j < k.it.nt) return true;
-  k.j = 0;
-  ++k.ic;
-  k.w += (int)gridDim.x;
-  return fs_seek(s, n_heads, nb_max, n_items, k);
-}
-
 __global__ void __launch_bounds__(kFsThreads, 2)
 fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, int nb_max, int n_items,
@@ -862,6 +872,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(&sh.pv_done[b], 1);
     }
     mbar_init(&sh.o_final, 2);
+    mbar_init(&sh.start, 1);
     sh.abort_flag = 0;
     fence_barrier_init();
   }
@@ -883,29 +894,47 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      FsWalk k;
-      bool have = fs_first(s, n_heads, nb_max, n_items, k);
+      // the item being loaded and, resolved one item ahead (so that `last` is known), the one after it
+      FsItem it, nx;
+      int w = fs_seek(s, n_heads, nb_max, n_items, fs_look(s, n_heads, nb_max, n_items, (int)blockIdx.x), it);
       bool ok = true;
-      while (have && ok) {
-        if (k.j == 0) {  // new item: its Q tile, once both issuing warps are done with the previous one
-          if (k.ic >= 1) ok = wait_or_abort(&sh.q_empty, (uint32_t)(k.ic - 1) & 1u, abort_flag);
-          if (!ok) break;
-          mbar_expect_tx(&sh.q_full, kTileBytes);
-          tma_load_tile(q_tile, &map_q, k.it.h, k.it.lo + k.it.ib * kTile, &sh.q_full);
-        }
-        const int slot = 2 * (k.T & 1);
-        const uint32_t par = ((uint32_t)(k.T >> 1) & 1u) ^ 1u;
-        const int row0 = k.it.lo + k.j * kFwKeys;
+      if (w >= n_items) {  // nothing for this block
+        sh.desc[0].nt = 0;
+        sh.desc[0].last = 1;
+        mbar_arrive(&sh.start);
+        mbar_arrive(&sh.q_full);
+      }
+      for (int ic = 0, T = 0; ok && w < n_items; ++ic) {
+        const int wn = fs_seek(s, n_heads, nb_max, n_items, fs_look(s, n_heads, nb_max, n_items, w + (int)gridDim.x), nx);
+        // the item's Q tile, once both issuing warps are done with the previous one
+        if (ic >= 1) ok = wait_or_abort(&sh.q_empty, (uint32_t)(ic - 1) & 1u, abort_flag);
+        if (!ok) break;
+        FsShared::Desc& d = sh.desc[ic % kFsDescs];
+        d.h = it.h;
+        d.lo = it.lo;
+        d.n = it.n;
+        d.ib = it.ib;
+        d.nt = it.nt;
+        d.last = wn >= n_items;
+        if (ic == 0) mbar_arrive(&sh.start);
+        mbar_expect_tx(&sh.q_full, kTileBytes);  // (release: the description is written before)
+        tma_load_tile(q_tile, &map_q, it.h, it.lo + it.ib * kTile, &sh.q_full);
+        for (int j = 0; j < it.nt && ok; ++j, ++T) {
+          const int slot = 2 * (T & 1);
+          const uint32_t par = ((uint32_t)(T >> 1) & 1u) ^ 1u;
+          const int row0 = it.lo + j * kFwKeys;
 #pragma unroll
-        for (int r = 0; r < 2 && ok; ++r) {
-          ok = wait_or_abort(&sh.kv_empty[slot + r], par, abort_flag);
-          if (!ok) break;
-          const CUtensorMap* map = r ? &map_v : &map_k;
-          unsigned char* dst = kv_ring + (slot + r) * kFwKvSlotBytes;
-          mbar_expect_tx(&sh.kv_full[slot + r], kFwKvSlotBytes);
-          tma_load_tile(dst, map, k.it.h, row0, &sh.kv_full[slot + r]);
+          for (int r = 0; r < 2 && ok; ++r) {
+            ok = wait_or_abort(&sh.kv_empty[slot + r], par, abort_flag);
+            if (!ok) break;
+            const CUtensorMap* map = r ? &map_v : &map_k;
+            unsigned char* dst = kv_ring + (slot + r) * kFwKvSlotBytes;
+            mbar_expect_tx(&sh.kv_full[slot + r], kFwKvSlotBytes);
+            tma_load_tile(dst, map, it.h, row0, &sh.kv_full[slot + r]);
+          }
         }
-        have = fs_next(s, n_heads, nb_max, n_items, k);
+        w = wn;
+        it = nx;
       }
     }
   } else if (warp == 1 || warp == 2) {
@@ -922,52 +951,63 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // other parity) still get its arrival on the per-item barriers (q_empty from the S walker, o_final
     // from the P V walker).
     struct Lean {
-      int w, j, T, ic, nt;
+      int j, T, ic, nt, last;
     };
-    auto lean_seek = [&](Lean& k) {
-      while (k.w < n_items) {
-        const int u = k.w / nb_max, x = k.w - u * nb_max;
-        const int seq = u / n_heads;
-        const int lo_ = s.cu[seq], n_ = s.cu[seq + 1] - lo_;
-        const int nb_ = (n_ + kTile - 1) / kTile;
-        if (x < nb_) {
-          k.nt = (min(n_, (nb_ - x) * kTile) + kFwKeys - 1) / kFwKeys;
-          return true;
-        }
-        k.w += (int)gridDim.x;
-      }
-      return false;
+    // enter item k.ic: the S walker waits for its Q (and with it for its description), the P V walker of
+    // the same thread comes later; false for a block without items
+    auto lean_enter = [&](Lean& k, bool wait_q) {
+      if (wait_q) ok = ok && wait_or_abort(&sh.q_full, (uint32_t)k.ic & 1u, abort_flag);
+      if (!ok) return false;
+      const volatile FsShared::Desc& d = sh.desc[k.ic % kFsDescs];
+      k.nt = d.nt;
+      k.last = d.last;
+      return k.nt > 0;
     };
-    auto lean_next = [&](Lean& k) {
+    auto lean_first = [&](Lean& k, bool wait_q) {
+      k.j = k.T = k.ic = 0;
+      return lean_enter(k, wait_q);
+    };
+    auto lean_next = [&](Lean& k, bool wait_q) {
       ++k.T;
       if (++k.j < k.nt) return true;
+      if (k.last) return false;
       k.j = 0;
       ++k.ic;
-      k.w += (int)gridDim.x;
-      return lean_seek(k);
+      return lean_enter(k, wait_q);
     };
     // from a tile of the other parity (an item of one tile gets the direct arrival) to the next own tile
-    auto skip_other = [&](Lean& k, bool& have, uint64_t* item_bar) {
+    auto skip_other = [&](Lean& k, bool& have, uint64_t* item_bar, bool wait_q) {
       if (k.nt == 1 && lane == 0) mbar_arrive(item_bar);
-      have = lean_next(k);
+      have = lean_next(k, wait_q);
     };
-    Lean ks_{(int)blockIdx.x, 0, 0, 0, 0}, kp_{(int)blockIdx.x, 0, 0, 0, 0};
-    bool have_s = lean_seek(ks_);
-    if (have_s && par == 1) skip_other(ks_, have_s, &sh.q_empty);
-    bool have_p = lean_seek(kp_);
-    if (have_p && par == 1) skip_other(kp_, have_p, &sh.o_final);
-    int q_seen = -1;  // last item whose Q this warp has waited for
+    Lean ks_, kp_;
+    bool have_s = lean_first(ks_, true);
+    if (have_s && par == 1) skip_other(ks_, have_s, &sh.q_empty, true);
+    bool have_p = lean_first(kp_, false);
+    if (have_p && par == 1) skip_other(kp_, have_p, &sh.o_final, false);
     // The S walker runs one own tile ahead of the P V walker: S(T + 2) is issued right behind P V(T) by
     // the same thread, and its buffer is the one that product reads (the tensor core runs one thread's
     // instructions in order).
+    // Both walkers move on at the START of their next step.  For the S walker this keeps the wait for the
+    // next item's Q behind the product that may be ready; the P V walker then enters an item only after the
+    // S walker has (it reads the item's description without a wait of its own).
+    bool s_advance = false, p_advance = false;
     for (bool first = true; ok; first = false) {
       if (!first) {
+        if (p_advance) {
+          have_p = lean_next(kp_, false);
+          if (have_p) skip_other(kp_, have_p, &sh.o_final, false);
+          p_advance = false;
+        }
         if (!have_p) break;
         // ---- O += P(T) V_T ----
         const int T = kp_.T, j = kp_.j;
         const int slot = 2 * (T & 1) + 1;
-        // the item's first product initialises O: the other warp's product of tile 1 must not overtake it
-        if (j == 1) ok = ok && wait_or_abort(&sh.pv_done[par ^ 1], (uint32_t)((T - 1) >> 1) & 1u, abort_flag);
+        // The products of one item accumulate into O in tile order: this one is issued when the previous
+        // tile's (the other warp's) is complete.  That fixes the order of the fp32 additions, so every bit
+        // of the output is the same in every run, and keeps the first product, which initialises O, first.
+        // (In steady state that product completed a tile time ago: the wait costs its own latency only.)
+        if (j >= 1) ok = ok && wait_or_abort(&sh.pv_done[par ^ 1], (uint32_t)((T - 1) >> 1) & 1u, abort_flag);
         ok = ok && wait_or_abort(&sh.p_full[par], (uint32_t)(T >> 1) & 1u, abort_flag);
         ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(T >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok) != 0;
@@ -990,16 +1030,18 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           FWD_TL(0, T, 4);
         }
         __syncwarp();
-        have_p = lean_next(kp_);
-        if (have_p) skip_other(kp_, have_p, &sh.o_final);
+        p_advance = true;
+      }
+      if (s_advance) {
+        // (only now, behind the product above: entering the next item waits for its Q, and a product that
+        //  is ready must not wait behind that)
+        have_s = lean_next(ks_, true);
+        if (have_s) skip_other(ks_, have_s, &sh.q_empty, true);
+        s_advance = false;
       }
       if (have_s) {
         // ---- S(T) = Q K_T^T ----
         const int T = ks_.T;
-        if (ks_.ic != q_seen) {
-          ok = ok && wait_or_abort(&sh.q_full, (uint32_t)ks_.ic & 1u, abort_flag);
-          q_seen = ks_.ic;
-        }
         const int slot = 2 * (T & 1);
         ok = ok && wait_or_abort(&sh.kv_full[slot], (uint32_t)(T >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok) != 0;
@@ -1023,8 +1065,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           FWD_TL(0, T, 0);
         }
         __syncwarp();
-        have_s = lean_next(ks_);
-        if (have_s) skip_other(ks_, have_s, &sh.q_empty);
+        s_advance = true;
       } else if (first) {
         break;
       }
@@ -1043,12 +1084,29 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     float2 l2 = make_float2(0.f, 0.f);  // row sum, even and odd keys apart (packed fp32x2 adds)
     FsItem it;
     int T = 0;  // key tiles so far, over all items
-    for (int w = (int)blockIdx.x, ic = 0; ok; w += (int)gridDim.x, ++ic) {
-      while (w < n_items && !fs_item(s, n_heads, nb_max, w, it)) w += (int)gridDim.x;
-      if (w >= n_items) break;
+    ok = __all_sync(0xffffffffu, wait_or_abort(&sh.start, 0, abort_flag));  // entry 0 of the descriptions is there
+    for (int ic = 0, last = 0; ok && !last; ++ic) {
+      // the item's description: readable once the item's first score tile has been seen
+      bool first_seen = false;
+      if (ic > 0) {
+        ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[T & 1], (uint32_t)(T >> 1) & 1u, abort_flag));
+        if (!ok) break;
+        first_seen = true;
+      }
+      {
+        const volatile FsShared::Desc& d = sh.desc[ic % kFsDescs];
+        it.h = d.h;
+        it.lo = d.lo;
+        it.n = d.n;
+        it.ib = d.ib;
+        it.nt = d.nt;
+        last = d.last;
+      }
+      if (it.nt == 0) break;
       const int qi = it.ib * kTile + row;  // query position inside the sequence
       for (int j = 0; j < it.nt && ok; ++j, ++T) {
-      ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[T & 1], (uint32_t)(T >> 1) & 1u, abort_flag));  // collectives below
+      if (!(j == 0 && first_seen))
+        ok = __all_sync(0xffffffffu, wait_or_abort(&sh.s_full[T & 1], (uint32_t)(T >> 1) & 1u, abort_flag));  // collectives below
       if (!ok) break;
       tc_fence_after();
       FWD_TL(0, T, 1);

@@ -17,6 +17,13 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 // One lane of a converged warp (the same lane every time).  The MMA-issuing warp runs its loop with
 // all lanes, so that descriptors and addresses stay warp-uniform (uniform registers), and predicates
 // only the single-thread instructions with this.
+// Same box as tma_load_tile, fetched into L2 only.
+__device__ __forceinline__ void tma_prefetch_tile(const CUtensorMap* map, int head, int row) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(0), "r"(row), "r"(0),
+               "r"(head)
+               : "memory");
+}
+
 // 32-byte global store (this architecture has 256-bit loads and stores); the address must be 32-byte aligned
 __device__ __forceinline__ void st_global_256(void* p, const uint32_t (&v)[8]) {
   asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]),

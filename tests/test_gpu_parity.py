@@ -116,6 +116,49 @@ def test_tensor_core_prefill_tile_edges(H2OCache):
     print(st)
 
 
+def test_tensor_core_prefill_long_and_short_kernels_mixed_lengths(H2OCache):
+    """Both forward kernels of the tensor-core path: prompts up to 1024 tokens take the persistent
+    one-query-block kernel (blocks walk over several (unit, query block) items, single-tile items included),
+    longer ones the two-query-block kernel; the column-sum kernel runs persistent in the first case."""
+    from parity_harness import run_parity
+
+    short = [1024, 1, 130, 512, 64, 1000, 129, 700, 3, 256, 900, 65] * 3  # more items than resident blocks need
+    wl = _wl("short", len(short), 8, 128, "bf16", short, 4, [6] * len(short), [5] * len(short), seed=45)
+    st = run_parity(wl, H2OCache, units=[0, 9, 17, 100, 287], export_every=2)
+    print(st)
+    long_ = [1025, 300, 1500]
+    wl = _wl("long", len(long_), 2, 128, "bf16", long_, 4, [6] * 3, [5] * 3, seed=46)
+    st = run_parity(wl, H2OCache, export_every=2)
+    print(st)
+
+
+@pytest.mark.parametrize("lens,heads", [([512] * 12, 16), ([2048, 1100], 4), ([700, 33, 1024, 129, 5], 6)])
+def test_tensor_core_prefill_is_bit_reproducible(H2OCache, lens, heads):
+    """Two issuing warps per query block add their products into the same accumulator; they are chained so
+    that the order of those additions is fixed.  The same prompt twice: every bit of the outputs and of the
+    column sums must agree (also with the output tensor at an address that is only 16-byte aligned, which
+    takes the narrow stores)."""
+    from workloads import make_prompt_inputs
+
+    wl = _wl("repro", len(lens), heads, 128, "bf16", lens, 2, [4] * len(lens), [4] * len(lens), seed=47)
+    q, k, v, cu = make_prompt_inputs(wl, layer=0, device="cuda")
+    c = H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    res = []
+    backing = torch.empty(q.numel() + 8, dtype=q.dtype, device="cuda")
+    for rep in range(6):
+        out = torch.full_like(q, float("nan")) if rep < 5 else backing[8:].view_as(q)
+        if rep == 5:
+            assert out.data_ptr() % 32 == 16
+        c.reset()
+        c.prefill_select(q, k, v, cu, out)
+        assert c.status() == 0
+        res.append((out.clone().view(torch.int16), c.prefill_column_sums(wl.total_tokens).clone()))
+    for o, a in res[1:]:
+        assert torch.equal(o, res[0][0])
+        assert torch.equal(a, res[0][1])
+    c.close()
+
+
 def test_rotating_caches_early_prefetch_equals_waiting_first(H2OCache):
     """Several caches stepped in rotation on one stream (the benchmark's pattern).  The kernels then
     prefetch their cache before the previous launch has finished; everything observable must be
