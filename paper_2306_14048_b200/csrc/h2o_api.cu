@@ -92,7 +92,7 @@ ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens)
   };
   S.rowstat = take(cells * 2 * sizeof(float));  // row maximum and row sum (planar or interleaved)
   S.acc0 = take(cells * sizeof(double));
-  S.cu = take(((size_t)cfg->batch + 1) * sizeof(int32_t));
+  S.cu = take(((size_t)cfg->batch + 1 + 2) * sizeof(int32_t));  // cu_seqlens, then two work counters
   S.total = off;
   return S;
 }
@@ -352,8 +352,10 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   ps.rowstat = reinterpret_cast<float2*>(sc + S.rowstat);
   ps.acc0 = reinterpret_cast<double*>(sc + S.acc0);
   ps.cu = reinterpret_cast<int32_t*>(sc + S.cu);
+  ps.work = ps.cu + cfg.batch + 1;
   ps.total_tokens = total;
   cache->cu.assign(cu_seqlens, cu_seqlens + cfg.batch + 1);  // pageable source: staged before the call returns
+  cache->cu.resize((size_t)cfg.batch + 3, 0);  // the work counters travel with it: zero at every launch
   if (cudaMemcpyAsync(ps.cu, cache->cu.data(), cache->cu.size() * sizeof(int32_t), cudaMemcpyHostToDevice, st) !=
       cudaSuccess) {
     cudaGetLastError();

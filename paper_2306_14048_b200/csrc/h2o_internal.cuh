@@ -48,6 +48,7 @@ struct PrefillScratch {
   float2* rowstat; // tensor-core path: {reference maximum (log2 domain), 1 / row sum}; aliases rowmax/rowsum
   double* acc0;    // column sums
   int32_t* cu;     // [batch + 1] device copy of cu_seqlens
+  int32_t* work;   // two work counters of the persistent prefill kernels, zero when the launch starts
   int64_t total_tokens;
 };
 

@@ -10,6 +10,7 @@
 //
 // Paper: accumulated attention score of Algorithm 2 evaluated over all prompt rows (the prefill
 // branch of the Appendix A pseudocode).
+#include <algorithm>
 #include <cstring>
 
 #include "h2o_internal.cuh"
@@ -425,7 +426,11 @@ constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B]
 constexpr int kFwMaxKvSlots = 6;
 constexpr bool kFwSplitP = true;                 // P as bf16 hi + bf16 lo (two P V products): one bf16 alone (2^-9 per
                                                  // probability) misses the output tolerance on peaky rows
-constexpr int kFwShortPrompt = 1024;              // up to here one query block per thread block
+// Up to this prompt length the persistent one-query-block kernel runs the forward pass (measured: 512-token
+// prompts 621 -> 480 us, 2048-token prompts 399 -> 378 us, ragged up to 4096: 13.1 -> 12.4 ms per layer of
+// prefill-select); beyond, every block streaming its own K and V through L2 costs more than the fixed costs
+// it saves (32768 tokens: 17.2 against 16.0 ms), and two query blocks per thread block share every tile.
+constexpr int kFwShortPrompt = 4096;
 // ring slots: K_j, V_j, K_j+1, V_j+1 (, K_j+2, V_j+2 with two groups); TMEM columns: O and two S/P buffers per group
 __host__ __device__ constexpr int fw_kv_slots(int groups) { return groups == 2 ? 6 : 4; }
 __host__ __device__ constexpr uint32_t fw_tmem_cols(int groups) { return groups == 2 ? 512u : 256u; }
@@ -774,13 +779,14 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------------
-// Forward for short prompts: persistent blocks, one softmax group, two blocks per SM
+// Forward for prompts of up to kFwShortPrompt tokens: persistent blocks, one softmax group, two blocks per SM
 // ---------------------------------------------------------------------------------------------
 // Same arithmetic, tiles and tensor-memory layout as the one-group instance of the kernel above, but a
 // block walks over work items (unit, query block) instead of ending after one: barriers, tensor memory
 // and the K/V ring stay up, so an item's first loads and score tiles overlap the previous item's last
 // tiles and its output.  With 512-token prompts a block of the kernel above spends more time on its fixed
-// cost (allocation, first loads, pipeline fill, output, exit and relaunch) than on its five tiles.
+// cost (allocation, first loads, pipeline fill, output, exit and relaunch) than on its five tiles; with
+// 2048-token prompts that cost is still a quarter of a block's time.
 // All counters run over the block's whole sequence of key tiles: tile T uses ring slots 2 (T % 2) and
 // + 1, score buffer T % 2 and the issuing warp T % 2; a warp issues P V(T), then S(T + 2), which may
 // belong to the next item.
@@ -815,39 +821,35 @@ struct FsItem {
   int h, lo, n;  // head, first token and length of the sequence
   int ib, nt;    // query block, key tiles
 };
-// sequence bounds of item w, loaded ahead of their use (plain loads: nothing branches on them here)
-struct FsAhead {
-  int w, lo, end;
+// Item order: units in groups of `grp` (small enough for their K and V to stay in L2 while the group is
+// being worked on); inside a group every unit's longest query block first, then every unit's second
+// longest, ...: long items start early, the ones claimed last are short.
+struct FsOrder {
+  int n_heads, units, nb_max, grp, n_items;
 };
-__device__ __forceinline__ FsAhead fs_look(const PrefillScratch& s, int n_heads, int nb_max, int n_items, int w) {
-  FsAhead a{w, 0, 0};
-  if (w < n_items) {
-    const int seq = (w / nb_max) / n_heads;
-    a.lo = s.cu[seq];
-    a.end = s.cu[seq + 1];
-  }
-  return a;
-}
-__device__ __forceinline__ bool fs_make(int n_heads, int nb_max, const FsAhead& a, FsItem& it) {
-  const int u = a.w / nb_max, x = a.w % nb_max;
-  it.h = u % n_heads;
-  it.lo = a.lo;
-  it.n = a.end - a.lo;
+__device__ __forceinline__ bool fs_item(const PrefillScratch& s, const FsOrder& o, int w, FsItem& it) {
+  const int per_group = o.grp * o.nb_max;
+  const int g = w / per_group, r = w - g * per_group;
+  const int in_group = min(o.grp, o.units - g * o.grp);
+  const int x = r / in_group, uu = r - x * in_group;
+  if (x >= o.nb_max) return false;  // the last group may be smaller
+  const int u = g * o.grp + uu;
+  const int seq = u / o.n_heads;
+  it.h = u - seq * o.n_heads;
+  it.lo = s.cu[seq];
+  it.n = s.cu[seq + 1] - it.lo;
   const int nb = (it.n + kTile - 1) / kTile;
   if (x >= nb) return false;
   it.ib = nb - 1 - x;
   it.nt = (min(it.n, (it.ib + 1) * kTile) + kFwKeys - 1) / kFwKeys;  // keys 0 .. min(n, (ib+1)*128) - 1
   return true;
 }
-// first item at or after a.w (stride gridDim.x) that exists; returns its index (>= n_items: none)
-__device__ __forceinline__ int fs_seek(const PrefillScratch& s, int n_heads, int nb_max, int n_items, FsAhead a, FsItem& it) {
-  while (a.w < n_items && !fs_make(n_heads, nb_max, a, it)) a = fs_look(s, n_heads, nb_max, n_items, a.w + (int)gridDim.x);
-  return a.w;
-}
+
 __global__ void __launch_bounds__(kFsThreads, 2)
 fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                    const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, int nb_max, int n_items,
-                    float scale2, __nv_bfloat16* __restrict__ out, int32_t* status) {
+                    const __grid_constant__ CUtensorMap map_v, PrefillScratch s, FsOrder order, float scale2,
+                    __nv_bfloat16* __restrict__ out, int32_t* status) {
+  const int n_heads = order.n_heads, n_items = order.n_items;
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FsShared sh;
   const bool wide_out = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
@@ -894,9 +896,21 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       prefetch_tensormap(&map_q);
       prefetch_tensormap(&map_k);
       prefetch_tensormap(&map_v);
-      // the item being loaded and, resolved one item ahead (so that `last` is known), the one after it
-      FsItem it, nx;
-      int w = fs_seek(s, n_heads, nb_max, n_items, fs_look(s, n_heads, nb_max, n_items, (int)blockIdx.x), it);
+      // Items are claimed from a counter in the order of the item index (unit by unit, a unit's longest
+      // query block first): blocks that finish early take more, and the items of a unit run close together
+      // in time, so its K and V are read from memory once.  The claim (an atomic and two dependent loads)
+      // is made two items ahead: `last` of an item needs to know whether another one follows, and the
+      // lookup must not sit between an item's end and the next one's first loads.
+      auto claim = [&](FsItem& it) {  // next existing item; n_items: none left
+        int w;
+        do {
+          w = atomicAdd(s.work, 1);
+        } while (w < n_items && !fs_item(s, order, w, it));
+        return w < n_items ? w : n_items;
+      };
+      FsItem it, nx, nx2;
+      int w = claim(it);
+      int wn = w < n_items ? claim(nx) : n_items;
       bool ok = true;
       if (w >= n_items) {  // nothing for this block
         sh.desc[0].nt = 0;
@@ -905,7 +919,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_arrive(&sh.q_full);
       }
       for (int ic = 0, T = 0; ok && w < n_items; ++ic) {
-        const int wn = fs_seek(s, n_heads, nb_max, n_items, fs_look(s, n_heads, nb_max, n_items, w + (int)gridDim.x), nx);
+        int wn2 = n_items;
         // the item's Q tile, once both issuing warps are done with the previous one
         if (ic >= 1) ok = wait_or_abort(&sh.q_empty, (uint32_t)(ic - 1) & 1u, abort_flag);
         if (!ok) break;
@@ -932,9 +946,13 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             mbar_expect_tx(&sh.kv_full[slot + r], kFwKvSlotBytes);
             tma_load_tile(dst, map, it.h, row0, &sh.kv_full[slot + r]);
           }
+          // the ring is full after the item's first tiles: time for the lookup two items ahead
+          if (j == min(1, it.nt - 1) && wn < n_items) wn2 = claim(nx2);
         }
         w = wn;
         it = nx;
+        wn = wn2;
+        nx = nx2;
       }
     }
   } else if (warp == 1 || warp == 2) {
@@ -1320,21 +1338,23 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
   // short prompts: one query block per thread block, two blocks per SM; long ones: two query blocks share
   // every K/V tile
   if (max_seqlen <= kFwShortPrompt) {
-    const int nb_max = (max_seqlen + kTile - 1) / kTile, n_items = nb_max * c.units;
+    FsOrder o;
+    o.n_heads = c.n_heads;
+    o.units = c.units;
+    o.nb_max = (max_seqlen + kTile - 1) / kTile;
+    // K and V of a group: at most ~48 MB, well inside the L2
+    const int64_t unit_bytes = (int64_t)o.nb_max * kTile * kD * 2 * 2;
+    o.grp = (int)std::max<int64_t>(1, std::min<int64_t>(c.units, (48ll << 20) / unit_bytes));
+    o.n_items = (c.units + o.grp - 1) / o.grp * o.grp * o.nb_max;
+    const int n_items = o.n_items;
     if (n_items == 0) return cudaSuccess;
     const int smem = kTileBytes + kFsKvSlots * kFwKvSlotBytes + 1024;
     static unsigned long long attr_flags = 0;
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(fwd_tc_short_kernel), smem, &attr_flags);
     if (e != cudaSuccess) return e;
-    // Items of one unit differ in length (query block ib has 2 (ib + 1) key tiles) and follow one another
-    // in the item order, so the stride with which a block walks over the items must not share a factor
-    // with the number of query blocks, or a block would see the same ib every time.
-    int blocks = n_items < 2 * sm_count() ? n_items : 2 * sm_count();
-    auto gcd = [](int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; };
-    while (blocks > 1 && blocks < n_items && gcd(blocks, nb_max) != 1) --blocks;
-    fwd_tc_short_kernel<<<blocks, kFsThreads, smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, nb_max, n_items,
-                                                              make_scale2(c.scale), static_cast<__nv_bfloat16*>(out),
-                                                              c.status);
+    const int blocks = n_items < 2 * sm_count() ? n_items : 2 * sm_count();
+    fwd_tc_short_kernel<<<blocks, kFsThreads, smem, stream>>>(map_q, map_k, map_v, s, o, make_scale2(c.scale),
+                                                              static_cast<__nv_bfloat16*>(out), c.status);
     return cudaGetLastError();
   }
   return launch_fwd_g<2>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
