@@ -456,6 +456,18 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     H2O_STAMP(11);
     if (lane == 0) sh.wbest[warp] = best;
     if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    // The new token's K/V row in 16-byte chunks, for the write into the freed slot at the very end: fetched
+    // here (they are in L2 since the start of the kernel) so that the round trip overlaps the barrier and
+    // the final reduction instead of following them.
+    constexpr int kNewChunks = (2 * LPR + 31) / 32;
+    uint4 new_row[kNewChunks];
+    if (warp == 0 && rank == 0) {
+#pragma unroll
+      for (int i2 = 0; i2 < kNewChunks; ++i2) {
+        const int i = lane + 32 * i2;
+        if (i < 2 * LPR) new_row[i2] = *reinterpret_cast<const uint4*>((i < LPR ? ku : vu) + (i % LPR) * VEC);
+      }
+    }
     consumer_sync<kThreads>();
     H2O_STAMP(5);
     if (warp == 0) {
@@ -492,11 +504,13 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
           c.tpos[su] = t + 1;
         }
         if (slot >= 0) {
-          for (int i = lane; i < 2 * LPR; i += 32) {  // the new K/V row goes straight into the freed slot
-            const int c16 = i % LPR;
-            const uint4 val = *reinterpret_cast<const uint4*>((i < LPR ? ku : vu) + c16 * VEC);
-            T* base = reinterpret_cast<T*>(i < LPR ? c.K : c.V) + (mt.slot_off + slot) * D;
-            *reinterpret_cast<uint4*>(base + c16 * VEC) = val;
+#pragma unroll
+          for (int i2 = 0; i2 < kNewChunks; ++i2) {  // the new K/V row goes straight into the freed slot
+            const int i = lane + 32 * i2;
+            if (i < 2 * LPR) {
+              T* base = reinterpret_cast<T*>(i < LPR ? c.K : c.V) + (mt.slot_off + slot) * D;
+              *reinterpret_cast<uint4*>(base + (i % LPR) * VEC) = new_row[i2];
+            }
           }
         }
       }
