@@ -125,7 +125,37 @@ int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const flo
   return failed ? -2 : 0;
 }
 
-/* Eviction order: x before y iff acc_x < acc_y, or equal and pos_x < pos_y. */
+/*
+ * Score variant (Section "Discussions and Limitations", paragraph on previous attempts): the authors also
+ * ranked by the AVERAGED attention score, i.e. the accumulated score divided by the number of attention
+ * rows that contributed to it.  A key at position p has been attended by the queries p .. tnow, so
+ *   rank score = acc / (tnow - p + 1)        (mode 1)
+ *   rank score = acc                         (mode 0, Algorithm 2 as printed)
+ * The accumulated score itself is stored unchanged in both modes.
+ */
+static int g_score_mode = 0;
+int h2o_oracle_set_score_mode(int mode) {
+  if (mode != 0 && mode != 1) return -1;
+  g_score_mode = mode;
+  return 0;
+}
+static double rank_score(double acc, long pos, long tnow) {
+  return g_score_mode == 1 ? acc / (double)(tnow - pos + 1) : acc;
+}
+
+/*
+ * F_score(S) = sum over the kept keys of h(accumulated score) (Definition of the score function and the
+ * remark on h: identity in Algorithm 1/2, sqrt(z + 1) and log(z + 1) as concave choices).  Reporting
+ * only: for increasing h the victim, the key whose removal keeps F_score largest, is the same.
+ *   hkind 0: h(z) = z, 1: sqrt(z + 1), 2: log(z + 1)
+ */
+double h2o_oracle_fscore(const double* acc, long m, int hkind) {
+  double f = 0.0;
+  for (long j = 0; j < m; ++j) f += hkind == 1 ? sqrt(acc[j] + 1.0) : hkind == 2 ? log(acc[j] + 1.0) : acc[j];
+  return f;
+}
+
+/* Eviction order: x before y iff score_x < score_y, or equal and pos_x < pos_y. */
 static int precedes(double acc_x, long pos_x, double acc_y, long pos_y) {
   if (acc_x < acc_y) return 1;
   if (acc_x > acc_y) return 0;
@@ -169,7 +199,7 @@ long h2o_oracle_select(const double* acc0, long n, long k, long r, int32_t* kept
   scored_t* c = (scored_t*)malloc(sizeof(scored_t) * (size_t)nc);
   if (!c) return -1;
   for (long j = 0; j < nc; ++j) {
-    c[j].acc = acc0[j];
+    c[j].acc = rank_score(acc0[j], j, n - 1); /* the last prompt token is the latest query */
     c[j].pos = j;
   }
   qsort(c, (size_t)nc, sizeof(scored_t), scored_cmp); /* weakest first */
@@ -269,10 +299,11 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
       long second = -1;
       for (long j = 0; j < m; ++j) {
         if ((long)up[j] > tt - r) continue; /* protected recent window */
-        if (victim < 0 || precedes(ua[j], up[j], ua[victim], up[victim])) {
+        if (victim < 0 || precedes(rank_score(ua[j], up[j], tt), up[j], rank_score(ua[victim], up[victim], tt), up[victim])) {
           second = victim;
           victim = j;
-        } else if (second < 0 || precedes(ua[j], up[j], ua[second], up[second])) {
+        } else if (second < 0 ||
+                   precedes(rank_score(ua[j], up[j], tt), up[j], rank_score(ua[second], up[second], tt), up[second])) {
           second = j;
         }
       }
@@ -281,13 +312,13 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
         bad = 1;
         continue;
       }
-      if (second >= 0) gap[u] = rel_gap(ua[victim], ua[second]);
+      if (second >= 0) gap[u] = rel_gap(rank_score(ua[victim], up[victim], tt), rank_score(ua[second], up[second], tt));
       evicted[u] = up[victim];
       if (hint && hint[u] != -2 && hint[u] != evicted[u]) {
         long alt = -1;
         for (long j = 0; j < m; ++j)
           if (up[j] == hint[u] && (long)up[j] <= tt - r) alt = j;
-        if (alt >= 0 && rel_gap(ua[alt], ua[victim]) < tie_rel) {
+        if (alt >= 0 && rel_gap(rank_score(ua[alt], up[alt], tt), rank_score(ua[victim], up[victim], tt)) < tie_rel) {
           status[u] = 1;
           victim = alt;
         } else {

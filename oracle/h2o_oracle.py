@@ -48,6 +48,10 @@ def _load():
         lib.h2o_oracle_decode_step.restype = c.c_int
         lib.h2o_oracle_decode_step.argtypes = [c.c_long, c.c_long, c.c_long, ip, ip, ip, ip, ip, dp, dp, dp, fp, fp, fp,
                                                c.c_double, ip, c.c_double, dp, ip, ip, dp, dp]
+        lib.h2o_oracle_set_score_mode.restype = c.c_int
+        lib.h2o_oracle_set_score_mode.argtypes = [c.c_int]
+        lib.h2o_oracle_fscore.restype = c.c_double
+        lib.h2o_oracle_fscore.argtypes = [dp, c.c_long, c.c_int]
         _lib = lib
     return _lib
 
@@ -85,6 +89,20 @@ def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False):
     if rc != 0:
         raise RuntimeError("oracle attention failed: %d" % rc)
     return (O, acc0, P) if want_p else (O, acc0)
+
+
+def set_score_mode(mode: int) -> None:
+    """0: rank by the accumulated score (Algorithm 2); 1: by the averaged score (accumulated score over the
+    number of queries that attended the key; the variant named in "Discussions and Limitations").
+    Process-wide: the tests that use mode 1 set it back to 0 when they are done."""
+    if _load().h2o_oracle_set_score_mode(int(mode)) != 0:
+        raise ValueError("score mode must be 0 or 1")
+
+
+def fscore(acc: np.ndarray, hkind: int = 0) -> float:
+    """F_score = sum of h(accumulated score) over the kept keys; h: 0 identity, 1 sqrt(z+1), 2 log(z+1)."""
+    acc = np.ascontiguousarray(acc, dtype=np.float64)
+    return float(_load().h2o_oracle_fscore(_p(acc, ctypes.c_double), acc.shape[0], int(hkind)))
 
 
 def select(acc0: np.ndarray, k: int, r: int):

@@ -404,3 +404,82 @@ def test_heads_and_sequences_are_independent(oracle):
     np.testing.assert_array_equal(r_sub["out"], r_all["out"][[1, 4]])
     np.testing.assert_array_equal(r_sub["evicted"], r_all["evicted"][[1, 4]])
     assert full.t[1] == lens[0] + 1 and full.t[0] == lens[0]
+
+
+# ---------------------------------------------------------------------------------------------------
+# Score variants ("Discussions and Limitations": averaged attention score; remark on h: F_score reporting)
+# ---------------------------------------------------------------------------------------------------
+@pytest.fixture()
+def averaged_mode(oracle):
+    oracle.set_score_mode(1)
+    yield oracle
+    oracle.set_score_mode(0)
+
+
+@pytest.mark.parametrize("k,r", [(3, 0), (2, 2), (4, 1), (1, 3)])
+def test_averaged_score_variant_matches_a_literal_simulation(averaged_mode, k, r):
+    """Rank by accumulated score / number of queries that attended the key (positions p .. t: t - p + 1),
+    simulated literally in Python with explicit column sums; the accumulated scores themselves are
+    unchanged.  The run must also differ somewhere from the accumulated-score policy, or it pins nothing."""
+    oracle = averaged_mode
+    T, d, scale = 20, 4, 0.7
+    rng = np.random.default_rng(500 + 10 * k + r)
+    q, kk, v = _rand_qkv(rng, T, d)
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    S, rows, Kd = [], [], {}
+    evictions = []
+    for t in range(T):
+        Kd[t] = kk[t]
+        G = S + [t]
+        logits = [scale * math.fsum(float(a) * float(b) for a, b in zip(q[t], Kd[j])) for j in G]
+        mx = max(logits)
+        w = [math.exp(x - mx) for x in logits]
+        tot = math.fsum(w)
+        rows.append({j: x / tot for j, x in zip(G, w)})
+        ev = -1
+        if len(G) > k + r:
+            cand = [j for j in G if j <= t - r]
+            avg = {j: math.fsum(row.get(j, 0.0) for row in rows) / (t - j + 1) for j in cand}
+            ev = min(sorted(cand), key=lambda j: avg[j])  # first minimum in ascending position
+            vals = sorted(avg.values())
+            if len(vals) > 1 and (vals[1] - vals[0]) / max(vals[1], 1e-300) < 1e-9:
+                pytest.skip("tiny accidental near-tie in random data")
+            G.remove(ev)
+        S = G
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        assert res["evicted"][0] == ev
+        evictions.append(ev)
+        pos, acc = cache.export(0)
+        assert set(pos.tolist()) == set(S)
+        np.testing.assert_allclose(acc, [math.fsum(row.get(j, 0.0) for row in rows) for j in pos], rtol=1e-12)
+    oracle.set_score_mode(0)
+    plain = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    plain_ev = [int(plain.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])["evicted"][0]) for t in range(T)]
+    if r < 3:  # with a long recent window and few candidates the two policies may coincide
+        assert plain_ev != evictions
+
+
+def test_averaged_score_prefill_selection_is_top_k_of_column_sum_over_age(averaged_mode):
+    oracle = averaged_mode
+    rng = np.random.default_rng(77)
+    n, k, r = 40, 6, 5
+    acc0 = rng.random(n) * np.linspace(3.0, 0.2, n)  # older keys have collected more, as in a real prompt
+    kept, _ = oracle.select(acc0, k, r)
+    avg = acc0[: n - r] / (n - np.arange(n - r))
+    want = sorted(np.argsort(-avg, kind="stable")[:k].tolist() + list(range(n - r, n)))
+    assert kept.tolist() == want
+    oracle.set_score_mode(0)
+    kept0, _ = oracle.select(acc0, k, r)
+    assert kept0.tolist() != want  # the plain policy favours the old keys here
+
+
+def test_fscore_reports_sum_of_h_of_accumulated_scores(oracle):
+    acc = np.array([0.0, 3.0, 8.0, 0.25])
+    assert oracle.fscore(acc, 0) == pytest.approx(11.25, rel=1e-15)
+    assert oracle.fscore(acc, 1) == pytest.approx(1.0 + 2.0 + 3.0 + math.sqrt(1.25), rel=1e-15)
+    assert oracle.fscore(acc, 2) == pytest.approx(0.0 + math.log(4.0) + math.log(9.0) + math.log(1.25), rel=1e-15)
+    # removing the key with the smallest accumulated score keeps F_score largest, for every h (the reason
+    # why h does not change the decisions)
+    for hk in (0, 1, 2):
+        drops = [oracle.fscore(np.delete(acc, j), hk) for j in range(len(acc))]
+        assert int(np.argmax(drops)) == int(np.argmin(acc))
