@@ -247,6 +247,30 @@ int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
 /* h2o_decode_chunk: 0 = automatic (chunk kernel where it applies), 1 = one decode-step kernel per token. */
 int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path);
 /*
+ * Score variants.
+ *
+ * h2o_cache_set_score_mode: how candidates are RANKED when heavy hitters are selected after the prompt
+ *   and when a victim is chosen in a decode step.
+ *     0 (default)  by the accumulated attention score (Algorithm 1 / Algorithm 2, h(z) = z);
+ *     1            by the averaged attention score — the accumulated score divided by the number of queries
+ *                  that attended the key (a key at position p, current query position t: t - p + 1; after a
+ *                  prompt of n tokens: n - p) — the variant the paper's "Discussions and Limitations" reports
+ *                  as an experiment against the bias towards old tokens.
+ *   The stored scores are the accumulated ones in both modes; ties still go to the lowest position.
+ *   Only on an empty cache (after create or reset, before the first prefill or decode call): H2O_ERR_STATE
+ *   otherwise.  The mode survives h2o_cache_reset.  With mode 1, h2o_decode_chunk takes one decode-step
+ *   kernel per token.
+ *
+ * h2o_cache_fscore: F_score of every unit, the sum of h(accumulated score) over the unit's kept keys (the
+ *   score function in the paper's definition of the eviction policy; remark on h).
+ *     hkind 0: h(z) = z,  1: h(z) = sqrt(z + 1),  2: h(z) = log(z + 1).
+ *   Reporting only: for an increasing h the victim is the same.  out_dev: DEVICE pointer, [batch * n_heads]
+ *   doubles in (sequence, head) order, written on `stream`; owned by the caller.
+ *   Errors: H2O_ERR_INVALID_ARG (null pointer, hkind outside 0..2), H2O_ERR_CUDA.
+ */
+int h2o_cache_set_score_mode(h2o_cache_t* cache, int32_t mode);
+int h2o_cache_fscore(h2o_cache_t* cache, int32_t hkind, double* out_dev, void* stream);
+/*
  * Process-wide diagnostic switch (no counterpart in the paper).  A decode kernel launched right
  * after a decode / prefill / reset of a DIFFERENT cache on the same stream starts copying its own
  * cache tiles into shared memory before the preceding kernel has finished (inputs q/k/v are still

@@ -93,6 +93,10 @@ def _load() -> ctypes.CDLL:
     lib.h2o_decode_chunk.restype = c.c_int
     lib.h2o_cache_set_chunk_path.argtypes = [vp, c.c_int32]
     lib.h2o_cache_set_chunk_path.restype = c.c_int
+    lib.h2o_cache_set_score_mode.argtypes = [vp, c.c_int32]
+    lib.h2o_cache_set_score_mode.restype = c.c_int
+    lib.h2o_cache_fscore.argtypes = [vp, c.c_int32, vp, vp]
+    lib.h2o_cache_fscore.restype = c.c_int
     lib.h2o_cache_reset.argtypes = [vp, vp]
     lib.h2o_host_staging_bytes.restype = c.c_size_t
     lib.h2o_host_staging_bytes.argtypes = [cfgp, c.c_int64]
@@ -224,6 +228,16 @@ class H2OCache:
 
     def set_chunk_path(self, path: int):
         _check(lib.h2o_cache_set_chunk_path(self._h, int(path)), "h2o_cache_set_chunk_path")
+
+    def set_score_mode(self, mode: int):
+        """0: rank by the accumulated score, 1: by the averaged score (empty cache only)."""
+        _check(lib.h2o_cache_set_score_mode(self._h, int(mode)), "h2o_cache_set_score_mode")
+
+    def fscore(self, hkind: int = 0, stream=None):
+        """F_score per (sequence, head): sum of h(accumulated score); h: 0 identity, 1 sqrt(z+1), 2 log(z+1)."""
+        out = torch.empty(self.cfg.batch * self.cfg.n_heads, dtype=torch.float64, device=self.device)
+        _check(lib.h2o_cache_fscore(self._h, int(hkind), out.data_ptr(), _stream_ptr(stream)), "h2o_cache_fscore")
+        return out.view(self.cfg.batch, self.cfg.n_heads)
 
     def reset(self, stream=None):
         _check(lib.h2o_cache_reset(self._h, _stream_ptr(stream)), "h2o_cache_reset")

@@ -443,12 +443,13 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       acc_g[x] = a;
       const int ps = pos_s[x];
       if (full && ps <= t - r) {
-        const Cand cx = cand_make(a, ps, lo + x);
+        // averaged variant: the key has been attended by the queries at positions ps .. t
+        const Cand cx = cand_make(c.score_mode == 1 ? a / (double)(t - ps + 1) : a, ps, lo + x);
         if (cand_before(cx, best)) best = cx;
       }
     }
     if (rank == 0 && tid == 0 && full && r == 0) {  // without a recent window the new token competes too
-      const Cand cs = cand_make((double)p_self, t, -2);
+      const Cand cs = cand_make((double)p_self, t, -2);  // attended once: its average is its score
       if (cand_before(cs, best)) best = cs;
     }
     H2O_STAMP(10);

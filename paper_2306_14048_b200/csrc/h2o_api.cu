@@ -288,6 +288,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
     v.uni_k = c->heavy[0];
     v.uni_r = c->recent[0];
   }
+  v.score_mode = 0;
   c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
@@ -412,7 +413,8 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   g_last_writer.note_and_check(st, cache->view.K);
   cudaError_t e = cudaSuccess;
-  if (cache->chunk_path == 0 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+  // (the chunk kernel ranks by the accumulated score only)
+  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
@@ -433,6 +435,24 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
     return H2O_ERR_CUDA;
   }
   cache->phase = Phase::Decoding;
+  return H2O_OK;
+}
+
+int h2o_cache_set_score_mode(h2o_cache_t* cache, int32_t mode) {
+  if (!cache || (mode != 0 && mode != 1)) return H2O_ERR_INVALID_ARG;
+  if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one ranking rule per generation
+  cache->view.score_mode = mode;
+  return H2O_OK;
+}
+
+int h2o_cache_fscore(h2o_cache_t* cache, int32_t hkind, double* out_dev, void* stream) {
+  if (!cache || !out_dev || hkind < 0 || hkind > 2) return H2O_ERR_INVALID_ARG;
+  DeviceGuard guard(cache->cfg.device);
+  if (!guard.ok) return H2O_ERR_CUDA;
+  if (h2o::launch_fscore(cache->view, hkind, out_dev, static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return H2O_ERR_CUDA;
+  }
   return H2O_OK;
 }
 

@@ -38,6 +38,10 @@ struct CacheView {
   // slot_off = position * uni_pad) and a block need not load it: uni_pad = slots per unit rounded up
   // to 4, uni_k / uni_r the budgets; uni_pad < 0 otherwise.
   int32_t uni_pad, uni_k, uni_r;
+  // 0: candidates are ranked by the accumulated score (Algorithm 2); 1: by the averaged score, accumulated
+  // score / number of queries that attended the key ("Discussions and Limitations").  Stored scores are the
+  // accumulated ones in both modes.
+  int32_t score_mode;
 };
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
@@ -93,6 +97,7 @@ bool make_tile_map(CUtensorMap_st* map, const void* base, int64_t rows, int n_he
 // inputs and outputs are [n_tokens][units][head_dim], evicted_pos [n_tokens][units] (nullable).
 constexpr int kDecodeChunkTokens = 32;
 bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots);
+cudaError_t launch_fscore(const CacheView& c, int hkind, double* out, cudaStream_t stream);
 // `meta`: host copy of the unit table in launch order.
 cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const UnitMeta* meta, const void* q,
                                 const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos,

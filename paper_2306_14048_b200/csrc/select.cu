@@ -21,8 +21,10 @@ namespace {
 
 constexpr int kSelThreads = 256;
 
-__device__ __forceinline__ uint64_t score_key(double a) {
-  // column sums of probabilities are >= 0, for which the bit pattern is monotone
+// Ranking key of key j of a prompt of n tokens: its column sum, or (averaged variant) the column sum over
+// the number of queries that attended it, n - j.  Both are >= 0, for which the bit pattern is monotone.
+__device__ __forceinline__ uint64_t score_key(double a, int j, int n, int mode) {
+  if (mode == 1) a = a / (double)(n - j);
   return (uint64_t)__double_as_longlong(a < 0.0 ? 0.0 : a);
 }
 
@@ -89,7 +91,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
         const uint64_t prefix = prefix_sh;
         const uint64_t himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
         for (int j = tid; j < nc; j += kSelThreads) {
-          const uint64_t key = score_key(acc0[j]);
+          const uint64_t key = score_key(acc0[j], j, n, c.score_mode);
           if ((key & himask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
         }
         __syncthreads();
@@ -110,7 +112,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
       thr = prefix_sh;
       need_eq = remaining_sh;  // 1 <= need_eq <= number of candidates equal to thr
       int eq = 0;
-      for (int j = tid; j < nc; j += kSelThreads) eq += score_key(acc0[j]) == thr ? 1 : 0;
+      for (int j = tid; j < nc; j += kSelThreads) eq += score_key(acc0[j], j, n, c.score_mode) == thr ? 1 : 0;
       int tot;
       block_exclusive_scan(eq, warp_tot, tot);
       total_eq = tot;
@@ -121,7 +123,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
       const int j = j0 + tid;
       int is_eq = 0, gt = 0;
       if (j < nc && kb > 0) {
-        const uint64_t key = score_key(acc0[j]);
+        const uint64_t key = score_key(acc0[j], j, n, c.score_mode);
         is_eq = key == thr;
         gt = key > thr;
       }
@@ -176,6 +178,29 @@ cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_B, const
   return cudaGetLastError();
 }
 
+// F_score of every unit: the sum of h(accumulated score) over its occupied slots (the score function of
+// the eviction policy's definition; h: 0 identity, 1 sqrt(z + 1), 2 log(z + 1), see the remark on h).
+// Reporting only.  fp64, fixed summation order.
+constexpr int kFsThreads = 128;
+__global__ void __launch_bounds__(kFsThreads) fscore_kernel(CacheView c, int hkind, double* __restrict__ out) {
+  __shared__ double part[kFsThreads];
+  const UnitMeta mt = c.meta[blockIdx.x];
+  const int cnt = c.count[blockIdx.x];
+  const double* acc = c.acc + mt.slot_off;
+  double f = 0.0;
+  for (int x = threadIdx.x; x < cnt; x += kFsThreads) {
+    const double a = acc[x];
+    f += hkind == 1 ? sqrt(a + 1.0) : hkind == 2 ? log(a + 1.0) : a;
+  }
+  part[threadIdx.x] = f;
+  __syncthreads();
+  for (int w = kFsThreads / 2; w > 0; w >>= 1) {
+    if ((int)threadIdx.x < w) part[threadIdx.x] += part[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[mt.unit] = part[0];
+}
+
 }  // namespace
 
 cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
@@ -188,4 +213,11 @@ cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, in
   return launch<__nv_bfloat16, 128>(c, s, max_B, k, v, stream);
 }
 
+}  // namespace h2o
+
+namespace h2o {
+cudaError_t launch_fscore(const CacheView& c, int hkind, double* out, cudaStream_t stream) {
+  fscore_kernel<<<c.units, kFsThreads, 0, stream>>>(c, hkind, out);
+  return cudaGetLastError();
+}
 }  // namespace h2o

@@ -78,7 +78,7 @@ def _gather_units(x, cu, units, H):
 def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
                device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
-               pattern: Optional[Sequence[int]] = None) -> ParityStats:
+               pattern: Optional[Sequence[int]] = None, score_mode: int = 0) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
@@ -87,6 +87,14 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
     sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
     """
+    if score_mode > 0:  # the oracle's ranking rule is process-wide: always put it back
+        h2o_oracle.set_score_mode(score_mode)
+        try:
+            return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
+                              chunk, chunk_path, pattern, score_mode=0 - score_mode)
+        finally:
+            h2o_oracle.set_score_mode(0)
+    score_mode = -score_mode  # (negative: the oracle is already in that mode)
     stats = ParityStats()
     H, d = wl.n_heads, wl.head_dim
     units = list(range(wl.units)) if units is None else sorted(set(int(u) for u in units))
@@ -96,6 +104,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     scale = float(np.float32(scale if scale > 0 else 1.0 / np.sqrt(float(d))))
     gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
     gpu.set_prefill_path(prefill_path)
+    gpu.set_score_mode(score_mode)
     ora = h2o_oracle.OracleCache(len(units), 1, d, [wl.heavy[u // H] for u in units], [wl.recent[u // H] for u in units],
                                  scale=scale)
     uidx = torch.as_tensor(units, dtype=torch.long, device=device)
@@ -120,8 +129,9 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
                 acc0, (b_keep, b_drop) = ora.last_acc0[x], ora.last_boundary[x]
                 diff = set(gkept.tolist()) ^ set(o_kept[x].tolist())
                 assert len(gkept) == len(o_kept[x]), "prefill unit %d: kept count" % u
+                rank = (lambda j: acc0[j] / (hi - lo - j)) if score_mode == 1 else (lambda j: acc0[j])
                 for j in diff:  # every disputed position must sit on the k-th / (k+1)-th boundary
-                    assert _rel(acc0[j], b_keep) < TIE_REL and _rel(acc0[j], b_drop) < TIE_REL, (
+                    assert _rel(rank(j), b_keep) < TIE_REL and _rel(rank(j), b_drop) < TIE_REL, (
                         "prefill unit %d: position %d (score %.17g) kept/dropped against the oracle "
                         "(boundary %.17g / %.17g)" % (u, j, acc0[j], b_keep, b_drop))
                 stats.near_ties_prefill += 1

@@ -213,3 +213,62 @@ def test_large_budget_per_unit(H2OCache):
     wl = _wl("bigB", 1, 2, 128, "bf16", [9500], 12, [4600], [4400], seed=61)
     st = run_parity(wl, H2OCache, export_every=6)
     print(st)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_averaged_score_variant(H2OCache, dtype, d):
+    """Ranking by accumulated score / number of attending queries ("Discussions and Limitations"): prefill
+    selection, decode steps, a split unit, and h2o_decode_chunk (served by the step kernels in this mode)."""
+    from parity_harness import run_parity
+
+    wl = _wl("avg", 3, 3, d, dtype, [300, 77, 513], 48, [20, 9, 33], [24, 5, 31], seed=201)
+    st = run_parity(wl, H2OCache, export_every=8, score_mode=1)
+    assert st.decisions == 9 + 9 * 48
+    print(st)
+    st = run_parity(wl, H2OCache, export_every=16, score_mode=1, chunk=16)
+    print(st)
+    wl = _wl("avg0", 2, 2, d, dtype, [200, 150], 40, [12, 30], [0, 0], seed=202)  # no recent window
+    st = run_parity(wl, H2OCache, export_every=8, score_mode=1)
+    print(st)
+
+
+def test_averaged_score_differs_from_accumulated_and_needs_an_empty_cache(H2OCache):
+    """The two ranking rules keep different sets on the same inputs (old keys collect more), and the rule
+    cannot change in the middle of a generation."""
+    import paper_2306_14048_b200 as pkg
+    from workloads import make_decode_inputs, make_prompt_inputs
+
+    wl = _wl("avgdiff", 2, 4, 128, "bf16", [400, 380], 8, [16, 16], [8, 8], seed=203)
+    q, k, v, cu = make_prompt_inputs(wl, layer=0, device="cuda")
+    kept = []
+    for mode in (0, 1):
+        c = H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+        c.set_score_mode(mode)
+        c.prefill_select(q, k, v, cu, torch.empty_like(q))
+        with pytest.raises(pkg.H2OError):
+            c.set_score_mode(1 - mode)
+        pos, acc, count, t = c.export()
+        kept.append([np.sort(pos[u, :count[u]]) for u in range(wl.units)])
+        c.close()
+    assert any(not np.array_equal(a, b) for a, b in zip(*kept))
+    assert np.mean([a.mean() for a in kept[1]]) > np.mean([a.mean() for a in kept[0]])  # younger keys on average
+
+
+def test_fscore_report(H2OCache):
+    """Sum of h(accumulated score) per unit against the oracle's, for the three h of the paper's remark."""
+    from oracle import h2o_oracle
+    from workloads import make_decode_inputs, make_prompt_inputs
+
+    wl = _wl("fs", 2, 3, 128, "bf16", [260, 90], 5, [10, 200], [6, 100], seed=204)  # the second sequence is not full
+    q, k, v, cu = make_prompt_inputs(wl, layer=0, device="cuda")
+    c = H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    c.prefill_select(q, k, v, cu, torch.empty_like(q))
+    for s_ in range(5):
+        qs, ks, vs = make_decode_inputs(wl, s_, layer=0, device="cuda")
+        c.decode_step(qs, ks, vs, torch.empty_like(qs), None)
+    pos, acc, count, t = c.export()
+    for hk in (0, 1, 2):
+        f = c.fscore(hk).cpu().numpy().reshape(-1)
+        for u in range(wl.units):
+            assert f[u] == pytest.approx(h2o_oracle.fscore(acc[u, :count[u]], hk), rel=1e-12)
+    c.close()
