@@ -371,7 +371,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   } else {
     e = h2o::launch_prefill_naive(cache->view, ps, cfg.dtype, max_seqlen, q, k, v, out, true, true, st);
   }
-  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, cfg.dtype, cache->layout.max_B, k, v, st);
+  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, cfg.dtype, cache->layout.max_B, max_seqlen, k, v, st);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;

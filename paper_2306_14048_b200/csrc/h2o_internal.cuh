@@ -104,7 +104,7 @@ cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const U
                                 cudaStream_t stream);
 // One warp waits `polls` times on a barrier nobody arrives at, then records H2O_ERR_TIMEOUT (diagnostic).
 cudaError_t launch_wait_probe(const CacheView& c, uint32_t polls, cudaStream_t stream);
-cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
+cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, int max_seqlen, const void* k,
                                  const void* v, cudaStream_t stream);
 
 // ---------------------------------------------------------------------------

@@ -51,7 +51,8 @@ __device__ __forceinline__ int block_exclusive_scan(int x, int* warp_tot, int& t
   return before + incl - x;
 }
 
-template <typename T, int D>
+// KPT: candidates' keys a thread holds in registers (0: none, every pass reads them from memory)
+template <typename T, int D, int KPT>
 __global__ void __launch_bounds__(kSelThreads)
 select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, const T* __restrict__ v) {
   constexpr int VEC = Vec16<T>::N, LPR = D / VEC;
@@ -78,6 +79,27 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
     uint64_t thr = 0;      // key of the kb-th largest candidate
     int need_eq = 0;       // how many candidates with key == thr are kept
     int total_eq = 0;
+    // The eight radix passes and the count of equal keys all read every candidate's key: up to KPT * 256
+    // candidates they are kept in registers (one trip to memory, one division in the averaged mode);
+    // longer prompts read them again in every pass.  (KPT follows the longest prompt of the call.)
+    const bool cached = KPT > 0 && nc <= kSelThreads * KPT;
+    uint64_t keys[KPT > 0 ? KPT : 1];
+    if (cached && kb > 0) {
+#pragma unroll
+      for (int i = 0; i < KPT; ++i) {
+        const int j = tid + i * kSelThreads;
+        keys[i] = j < nc ? score_key(acc0[j], j, n, c.score_mode) : 0ull;
+      }
+    }
+    auto for_each_key = [&](auto&& f) {
+      if (cached) {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i)
+          if (tid + i * kSelThreads < nc) f(keys[i]);
+      } else {
+        for (int j = tid; j < nc; j += kSelThreads) f(score_key(acc0[j], j, n, c.score_mode));
+      }
+    };
     if (kb > 0) {
       if (tid == 0) {
         prefix_sh = 0;
@@ -90,10 +112,9 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
         __syncthreads();
         const uint64_t prefix = prefix_sh;
         const uint64_t himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
-        for (int j = tid; j < nc; j += kSelThreads) {
-          const uint64_t key = score_key(acc0[j], j, n, c.score_mode);
+        for_each_key([&](uint64_t key) {
           if ((key & himask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
-        }
+        });
         __syncthreads();
         {
           // the bin holding the rank still to be located: scan the histogram from the top bin down, one
@@ -112,7 +133,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
       thr = prefix_sh;
       need_eq = remaining_sh;  // 1 <= need_eq <= number of candidates equal to thr
       int eq = 0;
-      for (int j = tid; j < nc; j += kSelThreads) eq += score_key(acc0[j], j, n, c.score_mode) == thr ? 1 : 0;
+      for_each_key([&](uint64_t key) { eq += key == thr ? 1 : 0; });
       int tot;
       block_exclusive_scan(eq, warp_tot, tot);
       total_eq = tot;
@@ -165,17 +186,27 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
   }
 }
 
-template <typename T, int D>
-cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_B, const void* k, const void* v,
-                   cudaStream_t stream) {
+template <typename T, int D, int KPT>
+cudaError_t launch_kpt(const CacheView& c, const PrefillScratch& s, int max_B, const void* k, const void* v,
+                       cudaStream_t stream) {
   const size_t smem = sizeof(int32_t) * (size_t)(max_B > 0 ? max_B : 1);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(select_gather_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e =
+        cudaFuncSetAttribute(select_gather_kernel<T, D, KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  select_gather_kernel<T, D><<<c.units, kSelThreads, smem, stream>>>(c, s, static_cast<const T*>(k),
-                                                                    static_cast<const T*>(v));
+  select_gather_kernel<T, D, KPT><<<c.units, kSelThreads, smem, stream>>>(c, s, static_cast<const T*>(k),
+                                                                         static_cast<const T*>(v));
   return cudaGetLastError();
+}
+
+template <typename T, int D>
+cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_B, int max_seqlen, const void* k, const void* v,
+                   cudaStream_t stream) {
+  if (max_seqlen <= 2 * kSelThreads) return launch_kpt<T, D, 2>(c, s, max_B, k, v, stream);
+  if (max_seqlen <= 8 * kSelThreads) return launch_kpt<T, D, 8>(c, s, max_B, k, v, stream);
+  if (max_seqlen <= 16 * kSelThreads) return launch_kpt<T, D, 16>(c, s, max_B, k, v, stream);
+  return launch_kpt<T, D, 0>(c, s, max_B, k, v, stream);
 }
 
 // F_score of every unit: the sum of h(accumulated score) over its occupied slots (the score function of
@@ -203,14 +234,14 @@ __global__ void __launch_bounds__(kFsThreads) fscore_kernel(CacheView c, int hki
 
 }  // namespace
 
-cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, const void* k,
-                                 const void* v, cudaStream_t stream) {
+cudaError_t launch_select_gather(const CacheView& c, const PrefillScratch& s, int dtype, int max_B, int max_seqlen,
+                                 const void* k, const void* v, cudaStream_t stream) {
   if (dtype == H2O_F32) {
-    if (c.head_dim == 64) return launch<float, 64>(c, s, max_B, k, v, stream);
-    return launch<float, 128>(c, s, max_B, k, v, stream);
+    if (c.head_dim == 64) return launch<float, 64>(c, s, max_B, max_seqlen, k, v, stream);
+    return launch<float, 128>(c, s, max_B, max_seqlen, k, v, stream);
   }
-  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, s, max_B, k, v, stream);
-  return launch<__nv_bfloat16, 128>(c, s, max_B, k, v, stream);
+  if (c.head_dim == 64) return launch<__nv_bfloat16, 64>(c, s, max_B, max_seqlen, k, v, stream);
+  return launch<__nv_bfloat16, 128>(c, s, max_B, max_seqlen, k, v, stream);
 }
 
 }  // namespace h2o
