@@ -120,8 +120,13 @@ def select(acc0: np.ndarray, k: int, r: int):
 class OracleCache:
     """State of ``batch * n_heads`` independent units; unit index = sequence * n_heads + head."""
 
-    def __init__(self, batch: int, n_heads: int, head_dim: int, heavy: Sequence[int], recent: Sequence[int], scale: Optional[float] = None):
+    def __init__(self, batch: int, n_heads: int, head_dim: int, heavy: Sequence[int], recent: Sequence[int], scale: Optional[float] = None,
+                 kv4: bool = False):
+        """kv4: stored K/V rows are 4-bit group-quantised (oracle/kv_quant.py): a row is quantised when it
+        enters the cache — the kept prompt rows after selection, a new token's row after its own step, in
+        which it still takes part at full precision."""
         assert len(heavy) == batch and len(recent) == batch
+        self.kv4 = bool(kv4)
         self.batch, self.n_heads, self.d = batch, n_heads, head_dim
         self.units = batch * n_heads
         self.scale = float(scale) if scale and scale > 0 else 1.0 / float(np.sqrt(head_dim))
@@ -171,6 +176,9 @@ class OracleCache:
         self.t[u] = t
         self.pos[u, :m] = positions
         self.acc[u, :m] = acc
+        if self.kv4 and m > 0:
+            from oracle import kv_quant
+            k_rows, v_rows = kv_quant.qdq(_f32(k_rows)), kv_quant.qdq(_f32(v_rows))
         self.K[u, :m] = k_rows
         self.V[u, :m] = v_rows
 
@@ -184,9 +192,21 @@ class OracleCache:
         qf = _f32(q).reshape(self.units, self.d)
         kf = _f32(k_new).reshape(self.units, self.d)
         vf = _f32(v_new).reshape(self.units, self.d)
+        t_before = self.t.copy()
         if units is not None:
-            return self._decode_subset(qf, kf, vf, hint, tie_rel, want_p, list(units))
-        return self._decode(self, qf, kf, vf, hint, tie_rel, want_p)
+            res = self._decode_subset(qf, kf, vf, hint, tie_rel, want_p, list(units))
+        else:
+            res = self._decode(self, qf, kf, vf, hint, tie_rel, want_p)
+        if self.kv4:  # the new token's row, if it was kept, is stored quantised from now on
+            from oracle import kv_quant
+            kq, vq = kv_quant.qdq(kf), kv_quant.qdq(vf)
+            for u in (range(self.units) if units is None else units):
+                m = int(self.cnt[u])
+                hit = np.nonzero(self.pos[u, :m] == t_before[u])[0]
+                if hit.size:
+                    self.K[u, hit[0]] = kq[u]
+                    self.V[u, hit[0]] = vq[u]
+        return res
 
     @staticmethod
     def _decode(st, qf, kf, vf, hint, tie_rel, want_p):

@@ -483,3 +483,66 @@ def test_fscore_reports_sum_of_h_of_accumulated_scores(oracle):
     for hk in (0, 1, 2):
         drops = [oracle.fscore(np.delete(acc, j), hk) for j in range(len(acc))]
         assert int(np.argmax(drops)) == int(np.argmin(acc))
+
+
+# ---------------------------------------------------------------------------------------------------
+# 4-bit group quantisation of stored rows (the paper names the combination, not a quantiser: these pins
+# are mathematical)
+# ---------------------------------------------------------------------------------------------------
+def test_kv4_quantiser_error_bound_end_points_and_idempotence():
+    from oracle import kv_quant
+
+    rng = np.random.default_rng(9)
+    x = kv_quant.bf16_round(rng.standard_normal((64, 128)).astype(np.float32) * np.float32(3.0))
+    x[5, 32:64] = np.float32(0.75)  # a constant group
+    x[6, :32] = np.linspace(-4, 4, 32, dtype=np.float32)
+    codes, scale, zero = kv_quant.quantize_rows(x)
+    assert codes.dtype == np.uint8 and codes.max() <= 15
+    xh = kv_quant.dequantize_rows(codes, scale, zero)
+    g = x.reshape(64, 4, 32)
+    # every value within half a step (+ one bf16 rounding of the step); the minimum is reproduced exactly
+    step = scale[..., None]
+    assert np.all(np.abs(xh.reshape(64, 4, 32) - g) <= 0.5 * step * (1 + 2.0 ** -7) + 1e-6)
+    assert np.array_equal(xh.reshape(64, 4, 32).min(axis=-1), g.min(axis=-1))
+    assert np.all(codes.reshape(64, 4, 32).min(axis=-1) == 0)
+    nonconst = g.max(axis=-1) > g.min(axis=-1)
+    assert np.all(codes.reshape(64, 4, 32).max(axis=-1)[nonconst] >= 14)  # the maximum lands on the last step or next to it
+    assert np.array_equal(xh[5, 32:64], x[5, 32:64])  # constant group: exact
+    # reading back and storing again changes nothing
+    codes2, scale2, zero2 = kv_quant.quantize_rows(xh)
+    assert np.array_equal(kv_quant.dequantize_rows(codes2, scale2, zero2), xh)
+    # scale and zero are bf16 values
+    assert np.array_equal(kv_quant.bf16_round(scale), scale) and np.array_equal(kv_quant.bf16_round(zero), zero)
+
+
+def test_kv4_bf16_rounding_helper_matches_torch():
+    import torch
+    from oracle import kv_quant
+
+    x = np.random.default_rng(3).standard_normal(10000).astype(np.float32) * np.float32(100.0)
+    x[:4] = [1.00390625, 1.01171875, -1.00390625, 0.0]  # ties to even on both sides
+    want = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+    assert np.array_equal(kv_quant.bf16_round(x), want)
+
+
+def test_kv4_cache_stores_quantised_rows_but_attends_the_new_token_exactly(oracle):
+    from oracle import kv_quant
+
+    rng = np.random.default_rng(12)
+    d, k, r, T = 32, 2, 2, 9
+    q, kk, v = _rand_qkv(rng, T, d)
+    c4 = oracle.OracleCache(1, 1, d, [k], [r], scale=0.5, kv4=True)
+    ref = oracle.OracleCache(1, 1, d, [k], [r], scale=0.5)
+    for t in range(T):
+        # a plain cache that is FED quantised rows for everything but the current token must behave the same
+        res4 = c4.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        resr = ref.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        m = int(ref.cnt[0])
+        hit = np.nonzero(ref.pos[0, :m] == t)[0]
+        if hit.size:
+            ref.K[0, hit[0]] = kv_quant.qdq(kk[t][None].astype(np.float32))[0]
+            ref.V[0, hit[0]] = kv_quant.qdq(v[t][None].astype(np.float32))[0]
+        assert res4["evicted"][0] == resr["evicted"][0]
+        np.testing.assert_array_equal(res4["out"], resr["out"])
+    m = int(c4.cnt[0])
+    np.testing.assert_array_equal(c4.K[0, :m], kv_quant.qdq(c4.K[0, :m].astype(np.float32)))  # stored rows are on the grid
