@@ -53,6 +53,12 @@ def decode_bytes_per_unit_step(cnt: int, d: int, esize: int) -> int:
     return 2 * cnt * d * esize + 16 * cnt + 4 * cnt + 6 * d * esize
 
 
+def decode_bytes_per_unit_step_kv4(cnt: int, d: int) -> int:
+    """The same with 4-bit group-quantised slots (80-byte rows for d = 128), bf16 q/k/v/out."""
+    row = d // 2 + (d // 32) * 4
+    return 2 * cnt * row + 16 * cnt + 4 * cnt + 4 * d * 2 + 2 * row
+
+
 # DRAM bytes of one decode launch, dram__bytes_read.sum + dram__bytes_write.sum of an ncu capture (the
 # summaries are committed with the profiles): 55.26 MB read + 0.07 MB written for config 2, captured at
 # full size; c3 on the first 32 of 64 sequences (102.5 MB) and scaled by the units, which the traffic is
@@ -387,6 +393,44 @@ def main():
         chunk_fig = {"tokens": n_tok, "ms": float(np.median(ms)), "us_per_token_step": float(np.median(ms)) * 1e3 / n_tok,
                      "seq_heads_per_s": wl.units * n_tok / (float(np.median(ms)) * 1e-3)}
 
+    # context figure: the same decode steps with 4-bit group-quantised K/V slots (dtype bf16_kv4), rotating
+    # over the layer caches like the main loop
+    kv4_fig = None
+    if rank == 0 and wl.dtype == "bf16" and d == 128 and max(k_ + r_ for k_, r_ in zip(wl.heavy, wl.recent)) <= 8192:
+        kcaches = [pkg.H2OCache(wl.batch, H, d, "bf16_kv4", wl.heavy, wl.recent, device=local) for _ in range(L)]
+        for l in range(L):
+            q, k, v, o = prompts[l]
+            kcaches[l].prefill_select(q, k, v, cu, o, stream)
+        n_k = min(64, S)
+
+        def kv4_loop():
+            for s_ in range(n_k):
+                for l in range(L):
+                    kcaches[l].decode_step(dec[l][0][s_], dec[l][1][s_], dec[l][2][s_], dec[l][3][s_], dec[l][4][s_], stream)
+
+        kv4_loop()
+        torch.cuda.synchronize()
+        kgraph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(kgraph, stream=stream):
+            kv4_loop()
+        k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            kgraph.replay()
+            k0.record(stream)
+            kgraph.replay()
+            k1.record(stream)
+        torch.cuda.synchronize()
+        for c_ in kcaches:
+            assert c_.status() == 0, "device status word set"
+        k_us = k0.elapsed_time(k1) * 1e3 / (n_k * L)
+        k_cnt = [min(n, kk + rr) for n, kk, rr in zip(wl.prompt_lens, wl.heavy, wl.recent)]
+        k_bytes = sum(decode_bytes_per_unit_step_kv4(c_, d) for c_ in k_cnt) * H
+        kv4_fig = {"us_per_launch": k_us, "bytes_per_launch": k_bytes, "achieved_gbs": k_bytes / (k_us * 1e-6) / 1e9,
+                   "speedup_vs_bf16_slots": None}
+        for c_ in kcaches:
+            c_.close()
+        del kcaches
+
     # ---- end to end: pinned host tensors through the host-buffer C calls -----------------
     e2e = None
     if not args.no_e2e:
@@ -439,6 +483,8 @@ def main():
         cnt = [min(n, kk + rr) for n, kk, rr in zip(wl.prompt_lens, wl.heavy, wl.recent)]
         bytes_launch = sum(decode_bytes_per_unit_step(c, d, esize) for c in cnt) * H
         launch_us = decode_ms * 1e3 / (S * L)
+        if kv4_fig:
+            kv4_fig["speedup_vs_bf16_slots"] = launch_us / kv4_fig["us_per_launch"]
         achieved = bytes_launch / (launch_us * 1e-6) / 1e9
         flops = sum(prefill_flops(n, d) for n in wl.prompt_lens) * H * L
         out = {
@@ -461,6 +507,7 @@ def main():
             "gpu_launches": args.steps * L * (3 + S),
             "decode_one_layer_back_to_back_us": warm_us,
             "decode_chunk_one_layer": chunk_fig,
+            "decode_kv4_slots": kv4_fig,
             "clocks": clocks,
             "roofline": {
                 "kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",

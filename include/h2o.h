@@ -43,7 +43,17 @@ extern "C" {
 #define H2O_ERR_CUDA (-5)        /* a CUDA runtime call or kernel launch failed                 */
 #define H2O_ERR_TIMEOUT (-6)     /* a bounded device-side wait gave up (seen by h2o_cache_status) */
 
-typedef enum { H2O_F32 = 0, H2O_BF16 = 1 } h2o_dtype_t;
+/*
+ * H2O_BF16_KV4: q / k / v / out are bf16 (head_dim 128 only); the stored K/V slots are 4-bit group-quantised
+ * (the paper's Q3 "compatible with quantization": it names the combination, not a quantiser; this library's
+ * own: groups of 32 channels, zero = group minimum, scale = bf16((max - min) / 15), code =
+ * clamp(rint((x - zero) / scale), 0, 15), all in fp32; 80 bytes per row instead of 256).  A row is
+ * quantised when it enters the cache: kept prompt rows at selection, a new token's row after its own
+ * decode step, in which it takes part at full precision.  Prompt attention itself is unquantised.
+ * h2o_decode_chunk takes one decode-step kernel per token in this format; units are not split over
+ * thread-block clusters.
+ */
+typedef enum { H2O_F32 = 0, H2O_BF16 = 1, H2O_BF16_KV4 = 2 } h2o_dtype_t;
 
 typedef struct h2o_cache h2o_cache_t; /* opaque, host-side */
 

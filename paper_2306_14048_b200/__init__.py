@@ -6,6 +6,7 @@ Python binding used by the tests and the benchmark.
 from .binding import (  # noqa: F401
     EXPORTED,
     H2O_BF16,
+    H2O_BF16_KV4,
     H2O_ERR_CUDA,
     H2O_ERR_INVALID_ARG,
     H2O_ERR_STATE,

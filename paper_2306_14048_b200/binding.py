@@ -25,6 +25,7 @@ H2O_ERR_CUDA = -5
 H2O_ERR_TIMEOUT = -6
 H2O_F32 = 0
 H2O_BF16 = 1
+H2O_BF16_KV4 = 2  # bf16 inputs, 4-bit group-quantised K/V slots
 
 EXPORTED = (
     "h2o_cache_workspace_bytes",
@@ -141,7 +142,8 @@ def make_config(batch, n_heads, head_dim, dtype, heavy: Sequence[int], recent: S
     """Returns (h2o_config_t, keepalive) — the budget arrays must outlive the struct."""
     hv = (ctypes.c_int32 * len(heavy))(*[int(x) for x in heavy])
     rc = (ctypes.c_int32 * len(recent))(*[int(x) for x in recent])
-    code = {torch.float32: H2O_F32, torch.bfloat16: H2O_BF16, "f32": H2O_F32, "bf16": H2O_BF16}.get(dtype, dtype)
+    code = {torch.float32: H2O_F32, torch.bfloat16: H2O_BF16, "f32": H2O_F32, "bf16": H2O_BF16,
+            "bf16_kv4": H2O_BF16_KV4}.get(dtype, dtype)
     cfg = h2o_config_t(int(batch), int(n_heads), int(head_dim), int(code), hv, rc, float(softmax_scale), int(device))
     return cfg, (hv, rc)
 

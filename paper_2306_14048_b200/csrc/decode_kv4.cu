@@ -1,0 +1,493 @@
+// Decode step and slot gather for caches whose K/V slots are stored 4-bit group-quantised
+// (dtype H2O_BF16_KV4: q / k / v / out are bf16, head_dim 128).
+//
+// The paper states that the eviction policy combines with 4-bit quantisation (Q3 of its question section,
+// appendix on throughput with quantisation) without giving a quantiser; the one used here is this library's
+// own.  A stored row of 128 channels is 80 bytes:
+//   bytes  0..63   codes, channel c in byte c / 2 (even channel: low nibble); group g = channels 32 g .. 32 g + 31
+//                  = bytes 16 g .. 16 g + 15
+//   bytes 64..79   per group g: scale (bf16), zero (bf16)
+// and, in fp32 with round-to-nearest-even throughout,
+//   zero  = min of the group (an input value)          scale = bf16((max - zero) / 15), 1 for a constant group
+//   code  = clamp(rint((x - zero) / scale), 0, 15)      x_hat = zero + code * scale
+// A row is quantised when it enters the cache: the kept prompt rows at the gather, a new token's row after
+// its own step, in which it still takes part at full precision.
+//
+// The decode step is the same fused step as decode.cu (scores over the occupied slots, softmax, P V,
+// fp64 score accumulation, victim search, in-place write), with the dequantisation folded into the
+// arithmetic: per group  q . x_hat = zero * sum(q) + scale * sum(q_i code_i)  and
+// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <climits>
+#include <cmath>
+#include <cstdint>
+
+#include "../../include/h2o.h"
+#include "h2o_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace h2o {
+namespace {
+
+using namespace ptx;
+
+constexpr int kD = 128;
+constexpr int kRowBytes = 80;
+constexpr int kWarps = 8;                 // consumer warps; one more warp streams the tiles
+constexpr int kThreads = kWarps * 32;
+constexpr int kTileRows = 64;             // rows per tile: eight per consumer warp
+constexpr int kTileBytes = kTileRows * kRowBytes;  // 5120
+constexpr int kStages = 4;
+constexpr uint32_t kSpin = 1u << 22;
+
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpin; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Nibble i (0..7) of a 32-bit word as the float 1 + n / 16: the nibble goes to the top four mantissa bits
+// of 1.0 (one shift, one logic operation; no integer-to-float conversion).  Sums over these are turned
+// back into sums over the codes once per group: sum(w_i n_i) = 16 (sum(w_i f_i) - sum(w_i)); the constant
+// is small enough (16 against codes up to 15) for that to cost four bits of the fp32 accumulation.
+__device__ __forceinline__ float nibf(uint32_t w, int i) {
+  const uint32_t sh = i <= 4 ? (w << (19 - 4 * i)) : (w >> (4 * i - 19));
+  return __uint_as_float((sh & 0x00780000u) | 0x3F800000u);
+}
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+
+struct Cand {
+  unsigned long long key;  // bit pattern of the (non-negative) ranking score
+  int pos, slot;           // slot -1: none, -2: the new token itself
+};
+__device__ __forceinline__ Cand cand_none() { return Cand{~0ull, INT_MAX, -1}; }
+__device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {
+  if (a.slot == -1) return false;
+  if (b.slot == -1) return true;
+  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
+}
+__device__ __forceinline__ Cand warp_argmin(Cand a) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    Cand b;
+    b.key = __shfl_xor_sync(0xffffffffu, a.key, off);
+    b.pos = __shfl_xor_sync(0xffffffffu, a.pos, off);
+    b.slot = __shfl_xor_sync(0xffffffffu, a.slot, off);
+    if (cand_before(b, a)) a = b;
+  }
+  return a;
+}
+
+// Quantise one group of 32 channels (bf16 inputs); codes: 16 bytes, meta = scale | zero << 16 (bf16 bits).
+__device__ __forceinline__ void quantise_group(const __nv_bfloat16* src, uint4& codes, uint32_t& meta) {
+  float x[32];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * i);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      x[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+      x[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+    }
+  }
+  float mn = x[0], mx = x[0];
+#pragma unroll
+  for (int i = 1; i < 32; ++i) {
+    mn = fminf(mn, x[i]);
+    mx = fmaxf(mx, x[i]);
+  }
+  float scale = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(__fsub_rn(mx, mn), 15.0f)));
+  if (!(scale > 0.f)) scale = 1.0f;
+  uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    float t = rintf(__fdiv_rn(__fsub_rn(x[i], mn), scale));
+    t = fminf(fmaxf(t, 0.f), 15.f);
+    w[i >> 3] |= (uint32_t)t << (4 * (i & 7));
+  }
+  codes = make_uint4(w[0], w[1], w[2], w[3]);
+  meta = (__float_as_uint(scale) >> 16) | (__float_as_uint(mn) & 0xffff0000u);
+}
+
+struct Shared {
+  uint64_t full[kStages], empty[kStages], aux;
+  uint64_t nr;  // the producer warp has quantised the new token's row
+  float red[kWarps][kD];  // per-warp partial outputs (unnormalised, relative to the warp's maximum)
+  float gm[kWarps], gl[kWarps];
+  Cand wbest[kWarps];
+  __align__(16) unsigned char newrow[2][kRowBytes];  // the new token's K and V row, quantised
+};
+
+__global__ void __launch_bounds__(kThreads + 32, 2)
+decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
+                  const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
+                  int32_t* __restrict__ evicted_pos, int chunk) {
+  extern __shared__ __align__(128) unsigned char dyn[];
+  __shared__ Shared sh;
+  // dynamic layout: ring[kStages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk] f32
+  unsigned char* ring = dyn;
+  double* acc_s = reinterpret_cast<double*>(dyn + (size_t)kStages * 2 * kTileBytes);
+  int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
+  float* p = reinterpret_cast<float*>(pos_s + chunk);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int su = blockIdx.x;
+  const UnitMeta mt = c.meta[su];
+  // the previous kernel of the stream may have written this cache or produced q / k_new / v_new
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
+  const int cnt = c.count[su];
+  const int t = c.tpos[su];
+  const int ntile = (cnt + kTileRows - 1) / kTileRows;
+  unsigned char* Kb = static_cast<unsigned char*>(c.K) + mt.slot_off * kRowBytes;
+  unsigned char* Vb = static_cast<unsigned char*>(c.V) + mt.slot_off * kRowBytes;
+  double* acc_g = c.acc + mt.slot_off;
+  int32_t* pos_g = c.pos + mt.slot_off;
+  const __nv_bfloat16* qu = q + (int64_t)u * kD;
+  const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
+  const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
+  bool timed_out = false;
+
+  auto issue_stage = [&](int j) {  // producer lane only
+    const int s = j % kStages;
+    const int rows = min(kTileRows, cnt - j * kTileRows);
+    const uint32_t bytes = (uint32_t)rows * kRowBytes;
+    unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
+    mbar_expect_tx(&sh.full[s], 2 * bytes);
+    bulk_load(dst, Kb + (size_t)j * kTileBytes, bytes, &sh.full[s]);
+    bulk_load(dst + kTileBytes, Vb + (size_t)j * kTileBytes, bytes, &sh.full[s]);
+  };
+  if (tid == kThreads) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], kWarps);
+    }
+    mbar_init(&sh.aux, 1);
+    mbar_init(&sh.nr, 1);
+    fence_barrier_init();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int j = 0; j < min(kStages, ntile); ++j) issue_stage(j);
+    if (cnt > 0) {
+      const int npad = (cnt + 3) & ~3;  // stays inside the unit's padded slot range
+      mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
+      bulk_load(acc_s, acc_g, (uint32_t)npad * 8u, &sh.aux);
+      bulk_load(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
+    }
+  }
+  __syncthreads();
+
+  if (warp == kWarps) {
+    // ---- producer warp: one lane streams the tiles; lanes 0..7 quantise the new token's row meanwhile ----
+    if (lane < 8) {
+      uint4 codes;
+      uint32_t meta;
+      quantise_group((lane < 4 ? ku : vu) + 32 * (lane & 3), codes, meta);
+      unsigned char* row = sh.newrow[lane >> 2];
+      *reinterpret_cast<uint4*>(row + 16 * (lane & 3)) = codes;
+      *reinterpret_cast<uint32_t*>(row + 64 + 4 * (lane & 3)) = meta;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.nr);
+    if (lane == 0) {
+      for (int j = kStages; j < ntile; ++j) {
+        if (!bar_wait(&sh.empty[j % kStages], (uint32_t)(j / kStages - 1) & 1u)) timed_out = true;
+        issue_stage(j);
+      }
+      if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    }
+  } else {
+    // ---- consumer warps --------------------------------------------------------------------------
+    // score phase: lane = (row sub of the warp's eight rows, group g of 32 channels);
+    // output phase: lane owns channels 4 lane .. 4 lane + 3 (group lane / 8) of every row
+    const int sub = lane >> 2, g = lane & 3;
+    float qf[32];
+    float qsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(qu + 32 * g + 8 * i);
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        qf[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+        qf[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) qsum += qf[i];
+    // the new token against itself, at full precision (every warp computes the same value)
+    float s_self;
+    {
+      float part = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(ku + 32 * g + 8 * i);
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          part = fmaf(qf[8 * i + 2 * j], __uint_as_float(w[j] << 16), part);
+          part = fmaf(qf[8 * i + 2 * j + 1], __uint_as_float(w[j] & 0xffff0000u), part);
+        }
+      }
+      part += __shfl_xor_sync(0xffffffffu, part, 1);
+      part += __shfl_xor_sync(0xffffffffu, part, 2);
+      s_self = c.scale * part;
+    }
+    // Both phases use the same mapping: lane = (row sub of the warp's eight rows, group g of 32 channels),
+    // one 16-byte load of codes per row and matrix.  Every (row sub, group) keeps 32 output accumulators;
+    // the eight rows of a warp share one softmax state and are added up once, after the stream.
+    float o[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) o[i] = 0.f;
+    float zacc = 0.f;  // sum of p * (zero - 16 scale) of this lane's rows and group
+    float mg = -INFINITY, lg = 0.f;
+    for (int j = 0; j < ntile; ++j) {
+      const int s = j % kStages;
+      if (!bar_wait(&sh.full[s], (uint32_t)(j / kStages) & 1u)) timed_out = true;
+      const unsigned char* kt = ring + (size_t)s * 2 * kTileBytes;
+      const unsigned char* vt = kt + kTileBytes;
+      const int rows = min(kTileRows, cnt - j * kTileRows);
+      const int row = warp * 8 + sub;
+      float sc = -INFINITY;
+      uint4 vw = make_uint4(0, 0, 0, 0);
+      uint32_t vmeta = 0;
+      {
+        float part = 0.f;
+        if (row < rows) {
+          const uint4 cw = *reinterpret_cast<const uint4*>(kt + row * kRowBytes + 16 * g);
+          const uint32_t meta = *reinterpret_cast<const uint32_t*>(kt + row * kRowBytes + 64 + 4 * g);
+          vw = *reinterpret_cast<const uint4*>(vt + row * kRowBytes + 16 * g);
+          vmeta = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * g);
+          const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
+          float d0 = 0.f, d1 = 0.f;  // two chains
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            d0 = fmaf(qf[i], nibf(w[i >> 3], i & 7), d0);
+            d1 = fmaf(qf[i + 1], nibf(w[(i + 1) >> 3], (i + 1) & 7), d1);
+          }
+          // q . x_hat = (zero - 16 scale) sum(q) + 16 scale sum(q_i f_i)
+          const float sc16 = 16.0f * bf16_bits_to_float(meta & 0xffffu);
+          part = fmaf(sc16, d0 + d1, (bf16_bits_to_float(meta >> 16) - sc16) * qsum);
+        }
+        part += __shfl_xor_sync(0xffffffffu, part, 1);
+        part += __shfl_xor_sync(0xffffffffu, part, 2);
+        if (row < rows) {
+          sc = c.scale * part;
+          if (g == 0) p[j * kTileRows + row] = sc;  // raw score, finalised after the stream
+        }
+      }
+      // one softmax state per warp: maximum over its eight rows
+      float mnew = fmaxf(mg, sc);
+      mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 4));
+      mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 8));
+      mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 16));
+      if (mnew > -INFINITY) {  // warp-uniform
+        const float f = expf(mg - mnew);  // expf(-inf) = 0 for the warp's first rows
+        const float e = expf(sc - mnew);  // 0 for rows past the end
+        float esum = e;                   // over the warp's rows (the four lanes of a row hold the same e)
+        esum += __shfl_xor_sync(0xffffffffu, esum, 4);
+        esum += __shfl_xor_sync(0xffffffffu, esum, 8);
+        esum += __shfl_xor_sync(0xffffffffu, esum, 16);
+        lg = fmaf(lg, f, esum);
+        // p * x_hat_i = p (zero - 16 scale) + (16 p scale) f_i
+        const float sc16 = 16.0f * bf16_bits_to_float(vmeta & 0xffffu);
+        const float es = e * sc16;
+        zacc = fmaf(zacc, f, e * (bf16_bits_to_float(vmeta >> 16) - sc16));
+        const uint32_t w[4] = {vw.x, vw.y, vw.z, vw.w};
+        if (f == 1.0f) {  // (warp-uniform) the reference maximum did not move: the usual case
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = fmaf(es, nibf(w[i >> 3], i & 7), o[i]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = fmaf(es, nibf(w[i >> 3], i & 7), o[i] * f);
+        }
+        mg = mnew;
+      }
+      __syncwarp();
+      if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.empty[s])) : "memory");
+    }
+    // add up the warp's eight rows (same softmax reference), then this lane's group goes to shared memory
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      float v = o[i] + zacc;
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      o[i] = v;
+    }
+    if (sub == 0) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) sh.red[warp][32 * g + i] = o[i];
+    }
+    if (lane == 0) {
+      sh.gm[warp] = mg;
+      sh.gl[warp] = lg;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+
+    // ---- block statistics, computed by every warp alike -------------------------------------------
+    const float m_i = lane < kWarps ? sh.gm[lane] : -INFINITY;
+    float m = m_i;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    m = fmaxf(m, s_self);
+    const float w_i = (lane < kWarps && m_i > -INFINITY) ? expf(m_i - m) : 0.f;
+    float l = lane < kWarps ? sh.gl[lane] * w_i : 0.f;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    const float w_self = expf(s_self - m);
+    l += w_self;
+    const float inv_l = 1.0f / l;
+    if (warp == 0) {  // output: this lane's four channels
+      float res[4];
+      {
+        const uint2 raw = *reinterpret_cast<const uint2*>(vu + 4 * lane);  // the new token's value
+        res[0] = w_self * __uint_as_float(raw.x << 16);
+        res[1] = w_self * __uint_as_float(raw.x & 0xffff0000u);
+        res[2] = w_self * __uint_as_float(raw.y << 16);
+        res[3] = w_self * __uint_as_float(raw.y & 0xffff0000u);
+      }
+#pragma unroll
+      for (int g2 = 0; g2 < kWarps; ++g2) {
+        const float w = __shfl_sync(0xffffffffu, w_i, g2);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) res[i] = fmaf(sh.red[g2][4 * lane + i], w, res[i]);
+      }
+      uint2 pk;
+      pk.x = Vec16<__nv_bfloat16>::pack2(res[0] * inv_l, res[1] * inv_l);
+      pk.y = Vec16<__nv_bfloat16>::pack2(res[2] * inv_l, res[3] * inv_l);
+      *reinterpret_cast<uint2*>(out + (int64_t)u * kD + 4 * lane) = pk;
+    }
+
+    // ---- final probabilities, accumulation (Algorithm 2: accumulated score += probability), victim search ----
+    if (cnt > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
+    const bool full = cnt >= B;
+    const float p_self = w_self * inv_l;
+    Cand best = cand_none();
+    for (int x = tid; x < cnt; x += kThreads) {
+      const float px = expf(p[x] - m) * inv_l;
+      const double a = acc_s[x] + (double)px;
+      acc_g[x] = a;
+      const int ps = pos_s[x];
+      if (full && ps <= t - r) {
+        const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
+        const Cand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
+        if (cand_before(cx, best)) best = cx;
+      }
+    }
+    if (tid == 0 && full && r == 0) {  // without a recent window the new token competes too
+      const Cand cs{(unsigned long long)__double_as_longlong((double)p_self), t, -2};
+      if (cand_before(cs, best)) best = cs;
+    }
+    best = warp_argmin(best);
+    if (lane == 0) sh.wbest[warp] = best;
+    if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    if (warp == 0) {
+      const Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+      int slot, ev;
+      if (!full) {
+        slot = cnt;
+        ev = -1;
+      } else if (b.slot == -2) {
+        slot = -1;
+        ev = t;
+      } else if (b.slot >= 0) {
+        slot = b.slot;
+        ev = b.pos;
+      } else {  // a full cache always has a candidate; record instead of corrupting
+        slot = -1;
+        ev = -1;
+        if (lane == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
+      }
+      if (lane == 0) {
+        if (!full) c.count[su] = cnt + 1;
+        if (slot >= 0) {
+          c.acc[mt.slot_off + slot] = (double)p_self;
+          c.pos[mt.slot_off + slot] = t;
+        }
+        if (evicted_pos) evicted_pos[u] = ev;
+        c.tpos[su] = t + 1;
+      }
+      const bool nr_ok = bar_wait(&sh.nr, 0);  // (long complete: the row was quantised during the stream)
+      if (!nr_ok && lane == 0) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+      if (nr_ok && slot >= 0 && lane < 10) {  // the quantised new row goes straight into the freed slot
+        const int which = lane / 5, part = lane % 5;  // K: five 16-byte pieces, V: five
+        unsigned char* dst = (which == 0 ? Kb : Vb) + (size_t)slot * kRowBytes + 16 * part;
+        *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(sh.newrow[which] + 16 * part);
+      }
+    }
+  }
+}
+
+// Gather of the kept prompt rows into 4-bit slots: one thread per (slot, K or V, group).
+__global__ void __launch_bounds__(256)
+gather_kv4_kernel(CacheView c, PrefillScratch s, const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v) {
+  const int su = blockIdx.x;
+  const UnitMeta mt = c.meta[su];
+  const int u = mt.unit;
+  const int seq = u / c.n_heads, h = u % c.n_heads;
+  const int lo = s.cu[seq];
+  const int m = c.count[su];
+  const int64_t stride = (int64_t)c.n_heads * kD;
+  const int64_t base = ((int64_t)lo * c.n_heads + h) * kD;
+  unsigned char* Kb = static_cast<unsigned char*>(c.K) + mt.slot_off * kRowBytes;
+  unsigned char* Vb = static_cast<unsigned char*>(c.V) + mt.slot_off * kRowBytes;
+  for (int x = threadIdx.x; x < m * 8; x += blockDim.x) {
+    const int slot = x >> 3, part = x & 7, grp = part & 3;
+    const int j = c.pos[mt.slot_off + slot];
+    const __nv_bfloat16* src = (part < 4 ? k : v) + base + (int64_t)j * stride + 32 * grp;
+    uint4 codes;
+    uint32_t meta;
+    quantise_group(src, codes, meta);
+    unsigned char* row = (part < 4 ? Kb : Vb) + (size_t)slot * kRowBytes;
+    *reinterpret_cast<uint4*>(row + 16 * grp) = codes;
+    *reinterpret_cast<uint32_t*>(row + 64 + 4 * grp) = meta;
+  }
+}
+
+}  // namespace
+
+size_t kv4_row_bytes() { return kRowBytes; }
+
+cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
+                              int32_t* evicted_pos, cudaStream_t stream) {
+  const int chunk = (max_B + 3) & ~3;
+  const size_t smem = (size_t)kStages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
+  static unsigned long long attr_flags = 0;
+  {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel), 200 * 1024, &attr_flags);
+    if (e != cudaSuccess) return e;
+  }
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)c.units);
+  cfg.blockDim = dim3(kThreads + 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel, c, static_cast<const __nv_bfloat16*>(q),
+                            static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk);
+}
+
+// after the selection kernel has written positions, scores and counts (its own row gather is skipped)
+cudaError_t launch_gather_kv4(const CacheView& c, const PrefillScratch& s, const void* k, const void* v, cudaStream_t stream) {
+  gather_kv4_kernel<<<c.units, 256, 0, stream>>>(c, s, static_cast<const __nv_bfloat16*>(k),
+                                                 static_cast<const __nv_bfloat16*>(v));
+  return cudaGetLastError();
+}
+
+}  // namespace h2o

@@ -16,13 +16,19 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxSlotsPerUnit = 65536;  // bounded by the decode kernel's shared-memory score rows
+constexpr int kMaxSlotsPerUnitKv4 = 8192;  // 4-bit slots: one thread block per unit, its scores and staging in shared memory
 constexpr int kMaxPromptLen = 49151;     // the ALU prefill keeps one score row in shared memory
 constexpr int kMaxChunk = 8192;          // slots per decode thread block
 constexpr int kMaxUnits = 65535;
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-size_t elem_size(int dtype) { return dtype == H2O_F32 ? 4 : 2; }
+size_t elem_size(int dtype) { return dtype == H2O_F32 ? 4 : 2; }  // of q / k / v / out
+// dtype of the inputs as the kernels' template selectors know it
+int input_dtype(int dtype) { return dtype == H2O_BF16_KV4 ? H2O_BF16 : dtype; }
+size_t slot_row_bytes(const h2o_config_t* cfg) {
+  return cfg->dtype == H2O_BF16_KV4 ? h2o::kv4_row_bytes() : (size_t)cfg->head_dim * elem_size(cfg->dtype);
+}
 
 struct Layout {
   size_t K, V, acc, pos, count, tpos, status, meta, total;
@@ -34,13 +40,15 @@ struct Layout {
 int check_config(const h2o_config_t* cfg) {
   if (!cfg || !cfg->heavy_budget || !cfg->recent_window) return H2O_ERR_INVALID_ARG;
   if (cfg->batch < 1 || cfg->n_heads < 1 || cfg->device < 0) return H2O_ERR_INVALID_ARG;
-  if (cfg->dtype != H2O_F32 && cfg->dtype != H2O_BF16) return H2O_ERR_UNSUPPORTED;
+  if (cfg->dtype != H2O_F32 && cfg->dtype != H2O_BF16 && cfg->dtype != H2O_BF16_KV4) return H2O_ERR_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return H2O_ERR_UNSUPPORTED;
+  if (cfg->dtype == H2O_BF16_KV4 && cfg->head_dim != 128) return H2O_ERR_UNSUPPORTED;
   if ((int64_t)cfg->batch * cfg->n_heads > kMaxUnits) return H2O_ERR_UNSUPPORTED;
   for (int s = 0; s < cfg->batch; ++s) {
     const int64_t k = cfg->heavy_budget[s], r = cfg->recent_window[s];
     if (k < 0 || r < 0 || k + r < 1) return H2O_ERR_INVALID_ARG;
     if (k + r > kMaxSlotsPerUnit) return H2O_ERR_UNSUPPORTED;
+    if (cfg->dtype == H2O_BF16_KV4 && k + r > kMaxSlotsPerUnitKv4) return H2O_ERR_UNSUPPORTED;
   }
   if (std::isnan(cfg->softmax_scale) || std::isinf(cfg->softmax_scale)) return H2O_ERR_INVALID_ARG;
   return H2O_OK;
@@ -56,7 +64,7 @@ Layout make_layout(const h2o_config_t* cfg) {
     max_B = std::max(max_B, B);
   }
   const size_t units = (size_t)cfg->batch * cfg->n_heads;
-  const size_t row = (size_t)cfg->head_dim * elem_size(cfg->dtype);
+  const size_t row = slot_row_bytes(cfg);
   size_t off = 0;
   auto take = [&](size_t bytes) {
     const size_t at = off;
@@ -289,6 +297,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
     v.uni_r = c->recent[0];
   }
   v.score_mode = 0;
+  v.kv4 = cfg->dtype == H2O_BF16_KV4 ? 1 : 0;
   c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
@@ -363,15 +372,17 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
     return H2O_ERR_CUDA;
   }
   // bf16 / head_dim 128 runs on the tensor cores; every other combination on the fp32 FMA pipe
-  const bool tc = cache->prefill_path != 1 && h2o::prefill_tc_supported(cfg.dtype, cfg.head_dim);
+  const int in_dtype = input_dtype(cfg.dtype);
+  const bool tc = cache->prefill_path != 1 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
   cudaError_t e = cudaSuccess;
   if (tc) {
     e = h2o::launch_fwd_tc(cache->view, ps, max_seqlen, q, k, v, out, st);
     if (e == cudaSuccess) e = h2o::launch_colsum_tc(cache->view, ps, max_seqlen, q, k, st);
   } else {
-    e = h2o::launch_prefill_naive(cache->view, ps, cfg.dtype, max_seqlen, q, k, v, out, true, true, st);
+    e = h2o::launch_prefill_naive(cache->view, ps, in_dtype, max_seqlen, q, k, v, out, true, true, st);
   }
-  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, cfg.dtype, cache->layout.max_B, max_seqlen, k, v, st);
+  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, in_dtype, cache->layout.max_B, max_seqlen, k, v, st);
+  if (e == cudaSuccess && cache->view.kv4) e = h2o::launch_gather_kv4(cache->view, ps, k, v, st);
   if (e != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
@@ -391,8 +402,11 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   if (!guard.ok) return H2O_ERR_CUDA;
   // the cache workspace is the identity: two handles on one workspace must count as the same cache
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
-  const cudaError_t e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages,
-                                           quiescent, all_units_full(cache), q, k_new, v_new, out, evicted_pos,
+  const cudaError_t e =
+      cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, q, k_new, v_new, out, evicted_pos,
+                                               static_cast<cudaStream_t>(stream))
+                      : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, quiescent,
+                                           all_units_full(cache), q, k_new, v_new, out, evicted_pos,
                                            static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) {
     cudaGetLastError();
@@ -414,7 +428,7 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   g_last_writer.note_and_check(st, cache->view.K);
   cudaError_t e = cudaSuccess;
   // (the chunk kernel ranks by the accumulated score only)
-  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
@@ -423,10 +437,14 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
     const size_t step = (size_t)cache->view.units * cache->cfg.head_dim * elem_size(cache->cfg.dtype);
     for (int32_t i = 0; i < n_tokens && e == cudaSuccess; ++i) {
       const size_t off = (size_t)i * step;
-      e = h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, false,
-                             all_units_full(cache), static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
-                             static_cast<const char*>(v) + off, static_cast<char*>(out) + off,
-                             evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr, st);
+      int32_t* ev_i = evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr;
+      e = cache->view.kv4
+              ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, static_cast<const char*>(q) + off,
+                                       static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
+                                       static_cast<char*>(out) + off, ev_i, st)
+              : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, false,
+                                   all_units_full(cache), static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
+                                   static_cast<const char*>(v) + off, static_cast<char*>(out) + off, ev_i, st);
       if (e == cudaSuccess) advance_seen(cache, 1);
     }
   }

@@ -42,6 +42,7 @@ struct CacheView {
   // score / number of queries that attended the key ("Discussions and Limitations").  Stored scores are the
   // accumulated ones in both modes.
   int32_t score_mode;
+  int32_t kv4;  // 1: K/V slots are 80-byte 4-bit rows (written by the kernels of decode_kv4.cu)
 };
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
@@ -98,6 +99,10 @@ bool make_tile_map(CUtensorMap_st* map, const void* base, int64_t rows, int n_he
 constexpr int kDecodeChunkTokens = 32;
 bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots);
 cudaError_t launch_fscore(const CacheView& c, int hkind, double* out, cudaStream_t stream);
+size_t kv4_row_bytes();
+cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
+                              int32_t* evicted_pos, cudaStream_t stream);
+cudaError_t launch_gather_kv4(const CacheView& c, const PrefillScratch& s, const void* k, const void* v, cudaStream_t stream);
 // `meta`: host copy of the unit table in launch order.
 cudaError_t launch_decode_chunk(const CacheView& c, int64_t total_slots, const UnitMeta* meta, const void* q,
                                 const void* k, const void* v, int n_tokens, void* out, int32_t* evicted_pos,

@@ -173,6 +173,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
     c.acc[s0 + x] = acc0[j];
     c.pos[s0 + x] = j;
   }
+  if (c.kv4 == 0)  // (4-bit slots are filled by their own gather kernel, from the positions written above)
 #pragma unroll 4
   for (int x = tid; x < m * LPR; x += kSelThreads) {
     const int slot = x / LPR, ch = x % LPR;

@@ -19,7 +19,7 @@ from oracle import h2o_oracle
 from workloads import Workload, make_decode_inputs, make_prompt_inputs
 
 TIE_REL = 1e-6
-TOL = {"bf16": (2e-3, 1e-2), "f32": (1e-5, 1e-4)}  # |gpu - oracle| <= abs + rel * |oracle|
+TOL = {"bf16": (2e-3, 1e-2), "f32": (1e-5, 1e-4), "bf16_kv4": (2e-3, 1e-2)}  # |gpu - oracle| <= abs + rel * |oracle|
 
 
 @dataclasses.dataclass
@@ -106,7 +106,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     gpu.set_prefill_path(prefill_path)
     gpu.set_score_mode(score_mode)
     ora = h2o_oracle.OracleCache(len(units), 1, d, [wl.heavy[u // H] for u in units], [wl.recent[u // H] for u in units],
-                                 scale=scale)
+                                 scale=scale, kv4=(wl.dtype == "bf16_kv4"))
     uidx = torch.as_tensor(units, dtype=torch.long, device=device)
     if prefill:
         q, k, v, cu = make_prompt_inputs(wl, layer=layer, device=device)

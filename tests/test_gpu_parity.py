@@ -272,3 +272,47 @@ def test_fscore_report(H2OCache):
         for u in range(wl.units):
             assert f[u] == pytest.approx(h2o_oracle.fscore(acc[u, :count[u]], hk), rel=1e-12)
     c.close()
+
+
+def test_kv4_slots_ragged(H2OCache):
+    """4-bit group-quantised K/V slots (bf16 inputs): prefill selection quantises the kept rows, every decode
+    step attends the new token at full precision and stores it quantised; against the oracle's quantiser."""
+    from parity_harness import run_parity
+
+    wl = _wl("kv4", 3, 3, 128, "bf16_kv4", [300, 77, 513], 80, [20, 9, 33], [24, 5, 31], seed=301)
+    st = run_parity(wl, H2OCache, export_every=8)
+    assert st.decisions == 9 + 9 * 80
+    print(st)
+
+
+@pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([1, 0], [0, 1])])
+def test_kv4_edge_budgets_and_fill_phase(H2OCache, heavy, recent):
+    from parity_harness import run_parity
+
+    wl = _wl("kv4edge", 2, 2, 128, "bf16_kv4", [37, 21], 40, heavy, recent, seed=302)
+    st = run_parity(wl, H2OCache, export_every=4)
+    print(st)
+    wl = _wl("kv4fill", 2, 2, 128, "bf16_kv4", [1, 1], 90, [10, 40], [6, 50], seed=303)
+    st = run_parity(wl, H2OCache, prefill=False, export_every=8)  # Algorithm 1 from an empty cache, tiles fill up
+    print(st)
+
+
+def test_kv4_large_budget_chunk_call_and_averaged_score(H2OCache):
+    """Several tiles per unit (budget 700), h2o_decode_chunk (step kernels in this format), averaged ranking."""
+    from parity_harness import run_parity
+
+    wl = _wl("kv4big", 2, 2, 128, "bf16_kv4", [1500, 900], 40, [350, 100], [350, 100], seed=304)
+    st = run_parity(wl, H2OCache, export_every=8, chunk=8)
+    print(st)
+    wl = _wl("kv4avg", 2, 2, 128, "bf16_kv4", [300, 200], 40, [20, 12], [10, 0], seed=305)
+    st = run_parity(wl, H2OCache, export_every=8, score_mode=1)
+    print(st)
+
+
+def test_kv4_rejects_what_it_does_not_support(H2OCache):
+    import paper_2306_14048_b200 as pkg
+
+    with pytest.raises(pkg.H2OError):
+        H2OCache(1, 1, 64, "bf16_kv4", [4], [4])  # head_dim 128 only
+    with pytest.raises(pkg.H2OError):
+        H2OCache(1, 1, 128, "bf16_kv4", [8000], [8000])  # more slots than one thread block stages
