@@ -16,7 +16,7 @@
 // The decode step is the same fused step as decode.cu (scores over the occupied slots, softmax, P V,
 // fp64 score accumulation, victim search, in-place write), with the dequantisation folded into the
 // arithmetic: per group  q . x_hat = zero * sum(q) + scale * sum(q_i code_i)  and
-// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.
+// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs half a packed FMA on its code.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -53,13 +53,21 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// Nibble i (0..7) of a 32-bit word as the float 1 + n / 16: the nibble goes to the top four mantissa bits
-// of 1.0 (one shift, one logic operation; no integer-to-float conversion).  Sums over these are turned
-// back into sums over the codes once per group: sum(w_i n_i) = 16 (sum(w_i f_i) - sum(w_i)); the constant
-// is small enough (16 against codes up to 15) for that to cost four bits of the fp32 accumulation.
-__device__ __forceinline__ float nibf(uint32_t w, int i) {
-  const uint32_t sh = i <= 4 ? (w << (19 - 4 * i)) : (w >> (4 * i - 19));
-  return __uint_as_float((sh & 0x00780000u) | 0x3F800000u);
+// The eight codes of a 32-bit word as four float pairs, without integer-to-float conversions.  A nibble at
+// bits 4i .. 4i+3 (i <= 4) of a float's mantissa, under the exponent of 2^(23-4i), reads as 2^(23-4i) + n:
+// one logic operation per code (mask and exponent in one), one packed subtraction per pair (exact), and for
+// the three top nibbles one shift of the word.  1.6 instructions per code instead of a shift, a mask and a
+// conversion each.
+__device__ __forceinline__ void codes8(uint32_t w, float2 (&n)[4]) {
+  const uint32_t h = w >> 12;  // nibbles 5, 6, 7 at bits 8, 12, 16
+  const float2 a = make_float2(__uint_as_float((w & 0x0000000Fu) | 0x4B000000u), __uint_as_float((w & 0x000000F0u) | 0x49000000u));
+  const float2 b = make_float2(__uint_as_float((w & 0x00000F00u) | 0x47000000u), __uint_as_float((w & 0x0000F000u) | 0x45000000u));
+  const float2 c = make_float2(__uint_as_float((w & 0x000F0000u) | 0x43000000u), __uint_as_float((h & 0x00000F00u) | 0x47000000u));
+  const float2 d = make_float2(__uint_as_float((h & 0x0000F000u) | 0x45000000u), __uint_as_float((h & 0x000F0000u) | 0x43000000u));
+  n[0] = __fadd2_rn(a, make_float2(-8388608.0f, -524288.0f));
+  n[1] = __fadd2_rn(b, make_float2(-32768.0f, -2048.0f));
+  n[2] = __fadd2_rn(c, make_float2(-128.0f, -32768.0f));
+  n[3] = __fadd2_rn(d, make_float2(-2048.0f, -128.0f));
 }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 
@@ -126,15 +134,15 @@ struct Shared {
   __align__(16) unsigned char newrow[2][kRowBytes];  // the new token's K and V row, quantised
 };
 
-__global__ void __launch_bounds__(kThreads + 32, 2)
+__global__ void __launch_bounds__(kThreads + 32, 4)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                  int32_t* __restrict__ evicted_pos, int chunk) {
+                  int32_t* __restrict__ evicted_pos, int chunk, int stages) {
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
-  // dynamic layout: ring[kStages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk] f32
+  // dynamic layout: ring[stages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk] f32
   unsigned char* ring = dyn;
-  double* acc_s = reinterpret_cast<double*>(dyn + (size_t)kStages * 2 * kTileBytes);
+  double* acc_s = reinterpret_cast<double*>(dyn + (size_t)stages * 2 * kTileBytes);
   int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
   float* p = reinterpret_cast<float*>(pos_s + chunk);
 
@@ -158,7 +166,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   bool timed_out = false;
 
   auto issue_stage = [&](int j) {  // producer lane only
-    const int s = j % kStages;
+    const int s = j % stages;
     const int rows = min(kTileRows, cnt - j * kTileRows);
     const uint32_t bytes = (uint32_t)rows * kRowBytes;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
@@ -167,7 +175,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     bulk_load(dst + kTileBytes, Vb + (size_t)j * kTileBytes, bytes, &sh.full[s]);
   };
   if (tid == kThreads) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < stages; ++s) {
       mbar_init(&sh.full[s], 1);
       mbar_init(&sh.empty[s], kWarps);
     }
@@ -175,7 +183,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     mbar_init(&sh.nr, 1);
     fence_barrier_init();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    for (int j = 0; j < min(kStages, ntile); ++j) issue_stage(j);
+    for (int j = 0; j < min(stages, ntile); ++j) issue_stage(j);
     if (cnt > 0) {
       const int npad = (cnt + 3) & ~3;  // stays inside the unit's padded slot range
       mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
@@ -198,22 +206,23 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh.nr);
     if (lane == 0) {
-      for (int j = kStages; j < ntile; ++j) {
-        if (!bar_wait(&sh.empty[j % kStages], (uint32_t)(j / kStages - 1) & 1u)) timed_out = true;
+      for (int j = stages; j < ntile; ++j) {
+        if (!bar_wait(&sh.empty[j % stages], (uint32_t)(j / stages - 1) & 1u)) timed_out = true;
         issue_stage(j);
       }
       if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     }
   } else {
     // ---- consumer warps --------------------------------------------------------------------------
-    // score phase: lane = (row sub of the warp's eight rows, group g of 32 channels);
-    // output phase: lane owns channels 4 lane .. 4 lane + 3 (group lane / 8) of every row
-    const int sub = lane >> 2, g = lane & 3;
-    float qf[32];
+    // lane = (row sub of the warp's four rows per pass, eighth h8 of the row: 16 channels, half a group);
+    // a 64-row tile is two passes.  16 query values and 16 output accumulators per lane keep the kernel at
+    // four blocks per SM, which is what hides a block's serial start and end behind other blocks' streams.
+    const int sub = lane >> 3, h8 = lane & 7;
+    float qf[16];
     float qsum = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(qu + 32 * g + 8 * i);
+    for (int i = 0; i < 2; ++i) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(qu + 16 * h8 + 8 * i);
       const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -222,14 +231,14 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       }
     }
 #pragma unroll
-    for (int i = 0; i < 32; ++i) qsum += qf[i];
+    for (int i = 0; i < 16; ++i) qsum += qf[i];
     // the new token against itself, at full precision (every warp computes the same value)
     float s_self;
     {
       float part = 0.f;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(ku + 32 * g + 8 * i);
+      for (int i = 0; i < 2; ++i) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(ku + 16 * h8 + 8 * i);
         const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -239,93 +248,108 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       }
       part += __shfl_xor_sync(0xffffffffu, part, 1);
       part += __shfl_xor_sync(0xffffffffu, part, 2);
+      part += __shfl_xor_sync(0xffffffffu, part, 4);
       s_self = c.scale * part;
     }
-    // Both phases use the same mapping: lane = (row sub of the warp's eight rows, group g of 32 channels),
-    // one 16-byte load of codes per row and matrix.  Every (row sub, group) keeps 32 output accumulators;
-    // the eight rows of a warp share one softmax state and are added up once, after the stream.
-    float o[32];
+    float o[16];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) o[i] = 0.f;
-    float zacc = 0.f;  // sum of p * (zero - 16 scale) of this lane's rows and group
+    for (int i = 0; i < 16; ++i) o[i] = 0.f;
+    float zacc = 0.f;  // sum of p * zero of this lane's rows and group
     float mg = -INFINITY, lg = 0.f;
     for (int j = 0; j < ntile; ++j) {
-      const int s = j % kStages;
-      if (!bar_wait(&sh.full[s], (uint32_t)(j / kStages) & 1u)) timed_out = true;
+      const int s = j % stages;
+      if (!bar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
       const unsigned char* kt = ring + (size_t)s * 2 * kTileBytes;
       const unsigned char* vt = kt + kTileBytes;
       const int rows = min(kTileRows, cnt - j * kTileRows);
-      const int row = warp * 8 + sub;
-      float sc = -INFINITY;
-      uint4 vw = make_uint4(0, 0, 0, 0);
-      uint32_t vmeta = 0;
-      {
-        float part = 0.f;
-        if (row < rows) {
-          const uint4 cw = *reinterpret_cast<const uint4*>(kt + row * kRowBytes + 16 * g);
-          const uint32_t meta = *reinterpret_cast<const uint32_t*>(kt + row * kRowBytes + 64 + 4 * g);
-          vw = *reinterpret_cast<const uint4*>(vt + row * kRowBytes + 16 * g);
-          vmeta = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * g);
-          const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
-          float d0 = 0.f, d1 = 0.f;  // two chains
+      float sc[2];
+      uint2 vw[2];
+      uint32_t vmeta[2];
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            d0 = fmaf(qf[i], nibf(w[i >> 3], i & 7), d0);
-            d1 = fmaf(qf[i + 1], nibf(w[(i + 1) >> 3], (i + 1) & 7), d1);
+      for (int ps = 0; ps < 2; ++ps) {
+        const int row = ps * 32 + warp * 4 + sub;
+        float part = 0.f;
+        vw[ps] = make_uint2(0, 0);
+        vmeta[ps] = 0;
+        if (row < rows) {
+          const uint2 cw = *reinterpret_cast<const uint2*>(kt + row * kRowBytes + 8 * h8);
+          const uint32_t meta = *reinterpret_cast<const uint32_t*>(kt + row * kRowBytes + 64 + 4 * (h8 >> 1));
+          vw[ps] = *reinterpret_cast<const uint2*>(vt + row * kRowBytes + 8 * h8);
+          vmeta[ps] = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * (h8 >> 1));
+          const uint32_t w[2] = {cw.x, cw.y};
+          float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);  // two chains of packed fp32x2 FMAs
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            float2 n[4];
+            codes8(w[k], n);
+            d0 = __ffma2_rn(make_float2(qf[8 * k], qf[8 * k + 1]), n[0], d0);
+            d1 = __ffma2_rn(make_float2(qf[8 * k + 2], qf[8 * k + 3]), n[1], d1);
+            d0 = __ffma2_rn(make_float2(qf[8 * k + 4], qf[8 * k + 5]), n[2], d0);
+            d1 = __ffma2_rn(make_float2(qf[8 * k + 6], qf[8 * k + 7]), n[3], d1);
           }
-          // q . x_hat = (zero - 16 scale) sum(q) + 16 scale sum(q_i f_i)
-          const float sc16 = 16.0f * bf16_bits_to_float(meta & 0xffffu);
-          part = fmaf(sc16, d0 + d1, (bf16_bits_to_float(meta >> 16) - sc16) * qsum);
+          // q . x_hat = zero sum(q) + scale sum(q_i code_i)
+          part = fmaf(bf16_bits_to_float(meta & 0xffffu), (d0.x + d0.y) + (d1.x + d1.y), bf16_bits_to_float(meta >> 16) * qsum);
         }
         part += __shfl_xor_sync(0xffffffffu, part, 1);
         part += __shfl_xor_sync(0xffffffffu, part, 2);
+        part += __shfl_xor_sync(0xffffffffu, part, 4);
+        sc[ps] = -INFINITY;
         if (row < rows) {
-          sc = c.scale * part;
-          if (g == 0) p[j * kTileRows + row] = sc;  // raw score, finalised after the stream
+          sc[ps] = c.scale * part;
+          if (h8 == 0) p[j * kTileRows + row] = sc[ps];  // raw score, finalised after the stream
         }
       }
-      // one softmax state per warp: maximum over its eight rows
-      float mnew = fmaxf(mg, sc);
-      mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 4));
+      // one softmax state per warp: maximum over its eight rows of this tile
+      float mnew = fmaxf(mg, fmaxf(sc[0], sc[1]));
       mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 8));
       mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 16));
       if (mnew > -INFINITY) {  // warp-uniform
         const float f = expf(mg - mnew);  // expf(-inf) = 0 for the warp's first rows
-        const float e = expf(sc - mnew);  // 0 for rows past the end
-        float esum = e;                   // over the warp's rows (the four lanes of a row hold the same e)
-        esum += __shfl_xor_sync(0xffffffffu, esum, 4);
+        const float e[2] = {expf(sc[0] - mnew), expf(sc[1] - mnew)};  // 0 for rows past the end
+        float esum = e[0] + e[1];  // over the warp's rows (the eight lanes of a row hold the same e)
         esum += __shfl_xor_sync(0xffffffffu, esum, 8);
         esum += __shfl_xor_sync(0xffffffffu, esum, 16);
         lg = fmaf(lg, f, esum);
-        // p * x_hat_i = p (zero - 16 scale) + (16 p scale) f_i
-        const float sc16 = 16.0f * bf16_bits_to_float(vmeta & 0xffffu);
-        const float es = e * sc16;
-        zacc = fmaf(zacc, f, e * (bf16_bits_to_float(vmeta >> 16) - sc16));
-        const uint32_t w[4] = {vw.x, vw.y, vw.z, vw.w};
-        if (f == 1.0f) {  // (warp-uniform) the reference maximum did not move: the usual case
+        zacc *= f;
+        if (f != 1.0f) {  // (warp-uniform) the reference maximum moved
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = fmaf(es, nibf(w[i >> 3], i & 7), o[i]);
-        } else {
+          for (int i = 0; i < 16; ++i) o[i] *= f;
+        }
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = fmaf(es, nibf(w[i >> 3], i & 7), o[i] * f);
+        for (int ps = 0; ps < 2; ++ps) {
+          // p * x_hat_i = p zero + (p scale) code_i
+          const float es = e[ps] * bf16_bits_to_float(vmeta[ps] & 0xffffu);
+          zacc = fmaf(e[ps], bf16_bits_to_float(vmeta[ps] >> 16), zacc);
+          const uint32_t w[2] = {vw[ps].x, vw[ps].y};
+          const float2 es2 = make_float2(es, es);
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            float2 n[4];
+            codes8(w[k], n);
+#pragma unroll
+            for (int t2 = 0; t2 < 4; ++t2) {
+              const float2 r2 = __ffma2_rn(es2, n[t2], make_float2(o[8 * k + 2 * t2], o[8 * k + 2 * t2 + 1]));
+              o[8 * k + 2 * t2] = r2.x;
+              o[8 * k + 2 * t2 + 1] = r2.y;
+            }
+          }
         }
         mg = mnew;
       }
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.empty[s])) : "memory");
     }
-    // add up the warp's eight rows (same softmax reference), then this lane's group goes to shared memory
+    // add up the warp's rows (same softmax reference), then this lane's channels go to shared memory
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
+    for (int i = 0; i < 16; ++i) {
       float v = o[i] + zacc;
-      v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 16);
       o[i] = v;
     }
     if (sub == 0) {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) sh.red[warp][32 * g + i] = o[i];
+      for (int i = 0; i < 16; ++i) sh.red[warp][16 * h8 + i] = o[i];
     }
     if (lane == 0) {
       sh.gm[warp] = mg;
@@ -461,7 +485,9 @@ size_t kv4_row_bytes() { return kRowBytes; }
 cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
                               int32_t* evicted_pos, cudaStream_t stream) {
   const int chunk = (max_B + 3) & ~3;
-  const size_t smem = (size_t)kStages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
+  // many units: a shallow ring lets four blocks share an SM, which hides each block's serial start and end
+  const int stages = c.units > 4 * 148 ? 2 : kStages;
+  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
   static unsigned long long attr_flags = 0;
   {
     cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel), 200 * 1024, &attr_flags);
@@ -480,7 +506,7 @@ cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, cons
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, decode_kv4_kernel, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk);
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stages);
 }
 
 // after the selection kernel has written positions, scores and counts (its own row gather is skipped)
