@@ -16,7 +16,7 @@
 // The decode step is the same fused step as decode.cu (scores over the occupied slots, softmax, P V,
 // fp64 score accumulation, victim search, in-place write), with the dequantisation folded into the
 // arithmetic: per group  q . x_hat = zero * sum(q) + scale * sum(q_i code_i)  and
-// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs half a packed FMA on its code.
+// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -53,21 +53,21 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// The eight codes of a 32-bit word as four float pairs, without integer-to-float conversions.  A nibble at
-// bits 4i .. 4i+3 (i <= 4) of a float's mantissa, under the exponent of 2^(23-4i), reads as 2^(23-4i) + n:
-// one logic operation per code (mask and exponent in one), one packed subtraction per pair (exact), and for
-// the three top nibbles one shift of the word.  1.6 instructions per code instead of a shift, a mask and a
-// conversion each.
-__device__ __forceinline__ void codes8(uint32_t w, float2 (&n)[4]) {
+// The eight codes of a 32-bit word as floats, without integer-to-float conversions.  A nibble at bits
+// 4i .. 4i+3 (i <= 4) of a float's mantissa, under the exponent of 2^(23-4i), reads as 2^(23-4i) + n: one logic
+// operation per code (mask and exponent in one), one subtraction (exact), and for the three top nibbles
+// one shift of the word.  (Packed fp32x2 subtractions and FMAs on pairs were slower: 173 against 158 us
+// on the large ragged workload.)
+__device__ __forceinline__ void codes8(uint32_t w, float (&n)[8]) {
   const uint32_t h = w >> 12;  // nibbles 5, 6, 7 at bits 8, 12, 16
-  const float2 a = make_float2(__uint_as_float((w & 0x0000000Fu) | 0x4B000000u), __uint_as_float((w & 0x000000F0u) | 0x49000000u));
-  const float2 b = make_float2(__uint_as_float((w & 0x00000F00u) | 0x47000000u), __uint_as_float((w & 0x0000F000u) | 0x45000000u));
-  const float2 c = make_float2(__uint_as_float((w & 0x000F0000u) | 0x43000000u), __uint_as_float((h & 0x00000F00u) | 0x47000000u));
-  const float2 d = make_float2(__uint_as_float((h & 0x0000F000u) | 0x45000000u), __uint_as_float((h & 0x000F0000u) | 0x43000000u));
-  n[0] = __fadd2_rn(a, make_float2(-8388608.0f, -524288.0f));
-  n[1] = __fadd2_rn(b, make_float2(-32768.0f, -2048.0f));
-  n[2] = __fadd2_rn(c, make_float2(-128.0f, -32768.0f));
-  n[3] = __fadd2_rn(d, make_float2(-2048.0f, -128.0f));
+  n[0] = __uint_as_float((w & 0x0000000Fu) | 0x4B000000u) - 8388608.0f;
+  n[1] = __uint_as_float((w & 0x000000F0u) | 0x49000000u) - 524288.0f;
+  n[2] = __uint_as_float((w & 0x00000F00u) | 0x47000000u) - 32768.0f;
+  n[3] = __uint_as_float((w & 0x0000F000u) | 0x45000000u) - 2048.0f;
+  n[4] = __uint_as_float((w & 0x000F0000u) | 0x43000000u) - 128.0f;
+  n[5] = __uint_as_float((h & 0x00000F00u) | 0x47000000u) - 32768.0f;
+  n[6] = __uint_as_float((h & 0x0000F000u) | 0x45000000u) - 2048.0f;
+  n[7] = __uint_as_float((h & 0x000F0000u) | 0x43000000u) - 128.0f;
 }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 
@@ -277,18 +277,22 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
           vw[ps] = *reinterpret_cast<const uint2*>(vt + row * kRowBytes + 8 * h8);
           vmeta[ps] = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * (h8 >> 1));
           const uint32_t w[2] = {cw.x, cw.y};
-          float2 d0 = make_float2(0.f, 0.f), d1 = make_float2(0.f, 0.f);  // two chains of packed fp32x2 FMAs
+          float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;  // four chains
 #pragma unroll
           for (int k = 0; k < 2; ++k) {
-            float2 n[4];
+            float n[8];
             codes8(w[k], n);
-            d0 = __ffma2_rn(make_float2(qf[8 * k], qf[8 * k + 1]), n[0], d0);
-            d1 = __ffma2_rn(make_float2(qf[8 * k + 2], qf[8 * k + 3]), n[1], d1);
-            d0 = __ffma2_rn(make_float2(qf[8 * k + 4], qf[8 * k + 5]), n[2], d0);
-            d1 = __ffma2_rn(make_float2(qf[8 * k + 6], qf[8 * k + 7]), n[3], d1);
+            d0 = fmaf(qf[8 * k], n[0], d0);
+            d1 = fmaf(qf[8 * k + 1], n[1], d1);
+            d2 = fmaf(qf[8 * k + 2], n[2], d2);
+            d3 = fmaf(qf[8 * k + 3], n[3], d3);
+            d0 = fmaf(qf[8 * k + 4], n[4], d0);
+            d1 = fmaf(qf[8 * k + 5], n[5], d1);
+            d2 = fmaf(qf[8 * k + 6], n[6], d2);
+            d3 = fmaf(qf[8 * k + 7], n[7], d3);
           }
           // q . x_hat = zero sum(q) + scale sum(q_i code_i)
-          part = fmaf(bf16_bits_to_float(meta & 0xffffu), (d0.x + d0.y) + (d1.x + d1.y), bf16_bits_to_float(meta >> 16) * qsum);
+          part = fmaf(bf16_bits_to_float(meta & 0xffffu), (d0 + d1) + (d2 + d3), bf16_bits_to_float(meta >> 16) * qsum);
         }
         part += __shfl_xor_sync(0xffffffffu, part, 1);
         part += __shfl_xor_sync(0xffffffffu, part, 2);
@@ -321,17 +325,12 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
           const float es = e[ps] * bf16_bits_to_float(vmeta[ps] & 0xffffu);
           zacc = fmaf(e[ps], bf16_bits_to_float(vmeta[ps] >> 16), zacc);
           const uint32_t w[2] = {vw[ps].x, vw[ps].y};
-          const float2 es2 = make_float2(es, es);
 #pragma unroll
           for (int k = 0; k < 2; ++k) {
-            float2 n[4];
+            float n[8];
             codes8(w[k], n);
 #pragma unroll
-            for (int t2 = 0; t2 < 4; ++t2) {
-              const float2 r2 = __ffma2_rn(es2, n[t2], make_float2(o[8 * k + 2 * t2], o[8 * k + 2 * t2 + 1]));
-              o[8 * k + 2 * t2] = r2.x;
-              o[8 * k + 2 * t2 + 1] = r2.y;
-            }
+            for (int i = 0; i < 8; ++i) o[8 * k + i] = fmaf(es, n[i], o[8 * k + i]);
           }
         }
         mg = mnew;
