@@ -82,6 +82,39 @@ def test_host_buffer_calls_equal_device_calls(pkg, mode):
     _identical(_full_run(pkg, WL, host=mode), _full_run(pkg, WL))
 
 
+def test_kv4_slots_host_calls_snapshots_and_reproducibility(pkg):
+    """The 4-bit slot format through the same API surface: host-buffer calls equal device calls, two runs are
+    bit-identical, and a snapshot of its (smaller) workspace resumes exactly."""
+    wl = Workload("kv4api", 3, 4, 128, "bf16_kv4", (260, 97, 513), 6, (16, 8, 20), (16, 8, 20), 1, 909)
+    _identical(_full_run(pkg, wl), _full_run(pkg, wl))
+    _identical(_full_run(pkg, wl, host="pinned"), _full_run(pkg, wl))
+    q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    a = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+    full = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, "bf16", wl.heavy, wl.recent)
+    assert a.workspace_bytes < 0.5 * full.workspace_bytes
+    full.close()
+    a.prefill_select(q, k, v, cu, torch.empty_like(q))
+    steps = [make_decode_inputs(wl, s, device="cuda") for s in range(wl.decode_steps)]
+
+    def step(c, s):
+        dq, dk, dv = steps[s]
+        o = torch.empty_like(dq)
+        e = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32, device="cuda")
+        c.decode_step(dq, dk, dv, o, e)
+        return o.float().cpu().numpy(), e.cpu().numpy()
+
+    for s in range(3):
+        step(a, s)
+    b = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent, snapshot=a.snapshot().cpu())
+    for s in range(3, wl.decode_steps):
+        oa, ea = step(a, s)
+        ob, eb = step(b, s)
+        assert np.array_equal(oa, ob) and np.array_equal(ea, eb)
+    assert a.status() == 0 and b.status() == 0
+    a.close()
+    b.close()
+
+
 def test_reset_returns_the_cache_to_empty(pkg):
     _identical(_full_run(pkg, WL, reset_first=True), _full_run(pkg, WL))
 
