@@ -373,6 +373,9 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
     H2O_STAMP(3);
     const int g = warp * RPW + sub;
+    // (the staged scores and positions arrived long ago; looking at their barrier here instead of after the
+    //  statistics takes the barrier operation's latency out of the serial tail)
+    if (nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
 #pragma unroll
     for (int v = 0; v < VEC; ++v) sh.red[g][ch * VEC + v] = o[v];
     if (ch == 0) {
@@ -424,16 +427,15 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       l = lc;
     }
     H2O_STAMP(4);
+    const float inv_l = 1.0f / l;
     if (rank == 0 && tid < D) {
-      const float res = part_o / l;  // (kept as a division: one per output element)
+      const float res = part_o * inv_l;
       if constexpr (sizeof(T) == 4) reinterpret_cast<float*>(out)[(int64_t)u * D + tid] = res;
       else reinterpret_cast<__nv_bfloat16*>(out)[(int64_t)u * D + tid] = __float2bfloat16_rn(res);
     }
 
     // ---- final probabilities, accumulation (Algorithm 2: o~_i = o~_{i-1} + o_i), victim search ----
-    if (nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
     const bool full = cnt >= B;
-    const float inv_l = 1.0f / l;
     const float p_self = expf(s_self - m) * inv_l;
     Cand best = cand_none();
 #pragma unroll 2
