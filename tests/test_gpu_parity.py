@@ -130,6 +130,11 @@ def test_tensor_core_prefill_long_and_short_kernels_mixed_lengths(H2OCache):
     wl = _wl("long", len(long_), 2, 128, "bf16", long_, 4, [6] * 3, [5] * 3, seed=46)
     st = run_parity(wl, H2OCache, export_every=2)
     print(st)
+    # beyond 4096 tokens the two-query-block kernel runs the forward pass of the whole (ragged) batch
+    longer = [4200, 130, 700]
+    wl = _wl("longer", len(longer), 2, 128, "bf16", longer, 2, [6] * 3, [5] * 3, seed=48)
+    st = run_parity(wl, H2OCache, units=[0, 3, 5], export_every=2)
+    print(st)
 
 
 @pytest.mark.parametrize("lens,heads", [([512] * 12, 16), ([2048, 1100], 4), ([700, 33, 1024, 129, 5], 6)])
