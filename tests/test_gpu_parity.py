@@ -137,7 +137,7 @@ def test_tensor_core_prefill_long_and_short_kernels_mixed_lengths(H2OCache):
     print(st)
 
 
-@pytest.mark.parametrize("lens,heads", [([512] * 12, 16), ([2048, 1100], 4), ([700, 33, 1024, 129, 5], 6)])
+@pytest.mark.parametrize("lens,heads", [([512] * 12, 16), ([2048, 1100], 4), ([700, 33, 1024, 129, 5], 6), ([4300, 900], 4)])
 def test_tensor_core_prefill_is_bit_reproducible(H2OCache, lens, heads):
     """Two issuing warps per query block add their products into the same accumulator; they are chained so
     that the order of those additions is fixed.  The same prompt twice: every bit of the outputs and of the
