@@ -54,6 +54,9 @@ struct PrefillScratch {
   double* acc0;    // column sums
   int32_t* cu;     // [batch + 1] device copy of cu_seqlens
   int32_t* work;   // two work counters of the persistent prefill kernels, zero when the launch starts
+  // item order of the persistent forward kernel (host-built): first item index of every group of units
+  const int32_t* item_base;  // [fs_groups + 1]
+  int32_t fs_grp, fs_groups, fs_items;
   int64_t total_tokens;
 };
 
@@ -100,6 +103,7 @@ constexpr int kDecodeChunkTokens = 32;
 bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_slots);
 cudaError_t launch_fscore(const CacheView& c, int hkind, double* out, cudaStream_t stream);
 size_t kv4_row_bytes();
+int fwd_group_units(int units, int max_seqlen);
 cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
                               int32_t* evicted_pos, cudaStream_t stream);
 cudaError_t launch_gather_kv4(const CacheView& c, const PrefillScratch& s, const void* k, const void* v, cudaStream_t stream);

@@ -825,21 +825,24 @@ struct FsItem {
 // being worked on); inside a group every unit's longest query block first, then every unit's second
 // longest, ...: long items start early, the ones claimed last are short.
 struct FsOrder {
-  int n_heads, units, nb_max, grp, n_items;
+  int n_heads, units, grp, n_groups, n_items;
+  const int32_t* item_base;  // [n_groups + 1] first item index of every group (host-built from the prompt lengths:
+                             // a group has as many levels x as its longest sequence has query blocks, so that
+                             // a ragged batch does not make most indices name blocks that do not exist)
 };
-__device__ __forceinline__ bool fs_item(const PrefillScratch& s, const FsOrder& o, int w, FsItem& it) {
-  const int per_group = o.grp * o.nb_max;
-  const int g = w / per_group, r = w - g * per_group;
+// g: group of the previous item this thread looked up (item indices only grow)
+__device__ __forceinline__ bool fs_item(const PrefillScratch& s, const FsOrder& o, int w, int& g, FsItem& it) {
+  while (g + 1 < o.n_groups && w >= o.item_base[g + 1]) ++g;
+  const int r = w - o.item_base[g];
   const int in_group = min(o.grp, o.units - g * o.grp);
   const int x = r / in_group, uu = r - x * in_group;
-  if (x >= o.nb_max) return false;  // the last group may be smaller
   const int u = g * o.grp + uu;
   const int seq = u / o.n_heads;
   it.h = u - seq * o.n_heads;
   it.lo = s.cu[seq];
   it.n = s.cu[seq + 1] - it.lo;
   const int nb = (it.n + kTile - 1) / kTile;
-  if (x >= nb) return false;
+  if (x >= nb) return false;  // a shorter sequence of the group
   it.ib = nb - 1 - x;
   it.nt = (min(it.n, (it.ib + 1) * kTile) + kFwKeys - 1) / kFwKeys;  // keys 0 .. min(n, (ib+1)*128) - 1
   return true;
@@ -901,11 +904,12 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // in time, so its K and V are read from memory once.  The claim (an atomic and two dependent loads)
       // is made two items ahead: `last` of an item needs to know whether another one follows, and the
       // lookup must not sit between an item's end and the next one's first loads.
+      int g_at = 0;
       auto claim = [&](FsItem& it) {  // next existing item; n_items: none left
         int w;
         do {
           w = atomicAdd(s.work, 1);
-        } while (w < n_items && !fs_item(s, order, w, it));
+        } while (w < n_items && !fs_item(s, order, w, g_at, it));
         return w < n_items ? w : n_items;
       };
       FsItem it, nx, nx2;
@@ -1341,11 +1345,10 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
     FsOrder o;
     o.n_heads = c.n_heads;
     o.units = c.units;
-    o.nb_max = (max_seqlen + kTile - 1) / kTile;
-    // K and V of a group: at most ~48 MB, well inside the L2
-    const int64_t unit_bytes = (int64_t)o.nb_max * kTile * kD * 2 * 2;
-    o.grp = (int)std::max<int64_t>(1, std::min<int64_t>(c.units, (48ll << 20) / unit_bytes));
-    o.n_items = (c.units + o.grp - 1) / o.grp * o.grp * o.nb_max;
+    o.grp = s.fs_grp;
+    o.n_groups = s.fs_groups;
+    o.n_items = s.fs_items;
+    o.item_base = s.item_base;
     const int n_items = o.n_items;
     if (n_items == 0) return cudaSuccess;
     const int smem = kTileBytes + kFsKvSlots * kFwKvSlotBytes + 1024;
@@ -1358,6 +1361,15 @@ cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_s
     return cudaGetLastError();
   }
   return launch_fwd_g<2>(map_q, map_k, map_v, c, s, max_seqlen, out, stream);
+}
+
+// Units per group of the persistent forward kernel's item order (K and V of a group: at most ~48 MB, well
+// inside the L2); 0: this prompt length does not use that kernel.
+int fwd_group_units(int units, int max_seqlen) {
+  if (max_seqlen > kFwShortPrompt) return 0;
+  const int nb_max = (max_seqlen + kTile - 1) / kTile;
+  const int64_t unit_bytes = (int64_t)nb_max * kTile * kD * 2 * 2;
+  return (int)std::max<int64_t>(1, std::min<int64_t>(units, (48ll << 20) / unit_bytes));
 }
 
 bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 && head_dim == kD && encode_fn() != nullptr; }
