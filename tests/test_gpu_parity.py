@@ -137,6 +137,18 @@ def test_tensor_core_prefill_long_and_short_kernels_mixed_lengths(H2OCache):
     print(st)
 
 
+def test_tensor_core_prefill_item_order_over_several_groups_of_units(H2OCache):
+    """The persistent forward kernel orders its (unit, query block) items by groups of units whose K/V fit
+    the L2 and gives a group as many levels as its longest sequence has query blocks: a very ragged batch
+    whose groups end inside a sequence (5 heads, 24 units per group at this length)."""
+    from parity_harness import run_parity
+
+    lens = [4000, 1, 129, 64, 2500, 3, 700, 128, 33, 1024, 5, 3100]
+    wl = _wl("groups", len(lens), 5, 128, "bf16", lens, 3, [6] * len(lens), [5] * len(lens), seed=47)
+    st = run_parity(wl, H2OCache, units=[0, 4, 7, 21, 23, 24, 26, 39, 47, 48, 55, 59], export_every=2)
+    print(st)
+
+
 @pytest.mark.parametrize("lens,heads", [([512] * 12, 16), ([2048, 1100], 4), ([700, 33, 1024, 129, 5], 6), ([4300, 900], 4)])
 def test_tensor_core_prefill_is_bit_reproducible(H2OCache, lens, heads):
     """Two issuing warps per query block add their products into the same accumulator; they are chained so
