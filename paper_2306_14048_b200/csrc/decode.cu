@@ -10,13 +10,15 @@
 //   - A unit's slots are split over `split` thread blocks that form one cluster; each
 //     block owns `chunk` consecutive slots.  split = 1 for many small units, up to 8
 //     for few long ones, so that every SM has several blocks resident.
-//   - K tiles, then V tiles, of 8 KB each are streamed into a shared-memory ring with
-//     cp.async.bulk (the TMA engine, one elected thread issues, completion counted on
-//     an mbarrier).  The first STAGES tiles are issued before anything else happens, so
-//     V tiles are already in flight while the softmax of the K pass is computed.
-//   - Raw scores stay in shared memory; the softmax is exact (two passes over on-chip
-//     scores, no online rescaling).  Blocks of a cluster exchange (max, sum), partial
-//     outputs and victim candidates through distributed shared memory.
+//   - The slots are streamed as pairs of an 8 KB K tile and the matching 8 KB V tile into a
+//     shared-memory ring with cp.async.bulk (the TMA engine, one elected thread issues,
+//     completion counted on an mbarrier).  The first STAGES pairs are issued before anything
+//     else happens.
+//   - Every row group of a warp keeps its own online softmax (running maximum, sum and partial
+//     output); the groups are merged once after the stream.  Raw scores stay in shared memory:
+//     the final probabilities that are accumulated use the exact maximum and sum.  Blocks of a
+//     cluster exchange (max, sum), partial outputs and victim candidates through distributed
+//     shared memory.
 //   - Accumulated scores are fp64 in memory: eviction decisions compare sums of
 //     hundreds of probabilities and must not depend on fp32 rounding of the sum.
 // Every wait on an mbarrier is bounded; a wait that gives up records H2O_ERR_TIMEOUT in
