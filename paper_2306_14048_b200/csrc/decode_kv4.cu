@@ -69,6 +69,25 @@ __device__ __forceinline__ void codes8(uint32_t w, float (&n)[8]) {
   n[6] = __uint_as_float((h & 0x0000F000u) | 0x45000000u) - 2048.0f;
   n[7] = __uint_as_float((h & 0x000F0000u) | 0x43000000u) - 128.0f;
 }
+// The eight codes of a 32-bit word as four pairs of exact bf16 values, r[k] = (code k, code k + 4): a nibble in
+// the low mantissa bits of 128.0 reads as 128 + code; the subtraction is exact.
+__device__ __forceinline__ void codes_bf16x2(uint32_t w, uint32_t (&r)[4]) {
+  const __nv_bfloat162 c128 = __floats2bfloat162_rn(128.f, 128.f);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    uint32_t x = ((w >> (4 * k)) & 0x000F000Fu) | 0x43004300u;
+    __nv_bfloat162 v = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), c128);
+    r[k] = *reinterpret_cast<uint32_t*>(&v);
+  }
+}
+// D (16 x 8, fp32) += A (16 x 16, bf16, row) * B (16 x 8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 
 struct Cand {
@@ -132,6 +151,9 @@ struct Shared {
   float gm[kWarps], gl[kWarps];
   Cand wbest[kWarps];
   __align__(16) unsigned char newrow[2][kRowBytes];  // the new token's K and V row, quantised
+  // the query as the B operand of the score products, per lane 16 words (rows padded to 20 words: 16-byte
+  // reads of eight consecutive lanes then fall into different banks)
+  __align__(16) uint32_t qb[32][20];
 };
 
 __global__ void __launch_bounds__(kThreads + 32, 4)
@@ -177,7 +199,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   if (tid == kThreads) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&sh.full[s], 1);
-      mbar_init(&sh.empty[s], kWarps);
+      mbar_init(&sh.empty[s], kWarps / 2);  // a tile is consumed by four warps
     }
     mbar_init(&sh.aux, 1);
     mbar_init(&sh.nr, 1);
@@ -214,36 +236,28 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     }
   } else {
     // ---- consumer warps --------------------------------------------------------------------------
-    // lane = (row sub of the warp's four rows per pass, eighth h8 of the row: 16 channels, half a group);
-    // a 64-row tile is two passes.  16 query values and 16 output accumulators per lane keep the kernel at
-    // four blocks per SM, which is what hides a block's serial start and end behind other blocks' streams.
+    // A warp takes 16 rows of a tile (warps 0..3 the even tiles, warps 4..7 the odd ones).
+    // Scores on the tensor cores (mma.sync m16n8k16, bf16 x bf16 -> fp32; codes 0..15 are exact in bf16):
+    // A = the codes of 16 rows x 16 channels, B = the query with column n = quantisation group (zero outside
+    // the group), so that one accumulator tile holds, per row, the four group sums  sum(q_i code_i);
+    // scale and zero are applied once per group.  Lane (g, c4) = (lane / 4, lane % 4) loads the 16 bytes of
+    // group c4 of rows g and g + 8; which channel sits at which k index is free as long as B agrees.
+    // Values stay on the FMA pipe: lane = (row sub of four rows per pass, eighth h8 of the row: 16 channels).
     const int sub = lane >> 3, h8 = lane & 7;
-    float qf[16];
-    float qsum = 0.f;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(qu + 16 * h8 + 8 * i);
-      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        qf[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
-        qf[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-      }
-    }
-#pragma unroll
-    for (int i = 0; i < 16; ++i) qsum += qf[i];
+    const int g = lane >> 2, c4 = lane & 3;
     // the new token against itself, at full precision (every warp computes the same value)
     float s_self;
     {
       float part = 0.f;
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(ku + 16 * h8 + 8 * i);
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        const uint4 rq = *reinterpret_cast<const uint4*>(qu + 16 * h8 + 8 * i);
+        const uint4 rk = *reinterpret_cast<const uint4*>(ku + 16 * h8 + 8 * i);
+        const uint32_t wq[4] = {rq.x, rq.y, rq.z, rq.w}, wk[4] = {rk.x, rk.y, rk.z, rk.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          part = fmaf(qf[8 * i + 2 * j], __uint_as_float(w[j] << 16), part);
-          part = fmaf(qf[8 * i + 2 * j + 1], __uint_as_float(w[j] & 0xffff0000u), part);
+          part = fmaf(__uint_as_float(wq[j] << 16), __uint_as_float(wk[j] << 16), part);
+          part = fmaf(__uint_as_float(wq[j] & 0xffff0000u), __uint_as_float(wk[j] & 0xffff0000u), part);
         }
       }
       part += __shfl_xor_sync(0xffffffffu, part, 1);
@@ -251,66 +265,102 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       part += __shfl_xor_sync(0xffffffffu, part, 4);
       s_self = c.scale * part;
     }
+    // the query of group c4: its sum, and (warp 0) its words as B operands.  For the word w of a row
+    // (channels 8 w .. 8 w + 7 of the group) the two products use k index pairs (code 0, code 4 | code 1,
+    // code 5) and (code 2, code 6 | code 3, code 7), see codes_bf16x2.
+    float qsA, qsB;  // query sums of groups 2 c4 and 2 c4 + 1 (used by c4 < 2)
+    {
+      uint32_t raw[16];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 r4 = *reinterpret_cast<const uint4*>(qu + 32 * c4 + 8 * i);
+        raw[4 * i] = r4.x;
+        raw[4 * i + 1] = r4.y;
+        raw[4 * i + 2] = r4.z;
+        raw[4 * i + 3] = r4.w;
+      }
+      float qs = 0.f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) qs += __uint_as_float(raw[i] << 16) + __uint_as_float(raw[i] & 0xffff0000u);
+      qsA = __shfl_sync(0xffffffffu, qs, (lane & ~3) | ((2 * c4) & 3));
+      qsB = __shfl_sync(0xffffffffu, qs, (lane & ~3) | ((2 * c4 + 1) & 3));
+      if (warp == 0) {
+        const bool mine = g == c4;  // column n = g of B is group g: only the lanes that hold that group's channels
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          uint4 b;
+          b.x = mine ? __byte_perm(raw[4 * w], raw[4 * w + 2], 0x5410) : 0u;
+          b.y = mine ? __byte_perm(raw[4 * w], raw[4 * w + 2], 0x7632) : 0u;
+          b.z = mine ? __byte_perm(raw[4 * w + 1], raw[4 * w + 3], 0x5410) : 0u;
+          b.w = mine ? __byte_perm(raw[4 * w + 1], raw[4 * w + 3], 0x7632) : 0u;
+          *reinterpret_cast<uint4*>(&sh.qb[lane][4 * w]) = b;
+        }
+      }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
     float o[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) o[i] = 0.f;
     float zacc = 0.f;  // sum of p * zero of this lane's rows and group
     float mg = -INFINITY, lg = 0.f;
-    for (int j = 0; j < ntile; ++j) {
+    const int cb = (warp & 3) * 16;  // the warp's rows of a tile
+    for (int j = warp >> 2; j < ntile; j += 2) {
       const int s = j % stages;
       if (!bar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
       const unsigned char* kt = ring + (size_t)s * 2 * kTileBytes;
       const unsigned char* vt = kt + kTileBytes;
       const int rows = min(kTileRows, cnt - j * kTileRows);
-      float sc[2];
-      uint2 vw[2];
-      uint32_t vmeta[2];
+      // ---- scores of rows cb + g and cb + g + 8 ----
+      const int rowA = cb + g, rowB = rowA + 8;
+      float sA, sB;
+      {
+        const uint4 ka = *reinterpret_cast<const uint4*>(kt + rowA * kRowBytes + 16 * c4);
+        const uint4 kb = *reinterpret_cast<const uint4*>(kt + rowB * kRowBytes + 16 * c4);
+        const uint32_t wa[4] = {ka.x, ka.y, ka.z, ka.w}, wb[4] = {kb.x, kb.y, kb.z, kb.w};
+        float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};  // two chains
 #pragma unroll
-      for (int ps = 0; ps < 2; ++ps) {
-        const int row = ps * 32 + warp * 4 + sub;
-        float part = 0.f;
-        vw[ps] = make_uint2(0, 0);
-        vmeta[ps] = 0;
-        if (row < rows) {
-          const uint2 cw = *reinterpret_cast<const uint2*>(kt + row * kRowBytes + 8 * h8);
-          const uint32_t meta = *reinterpret_cast<const uint32_t*>(kt + row * kRowBytes + 64 + 4 * (h8 >> 1));
-          vw[ps] = *reinterpret_cast<const uint2*>(vt + row * kRowBytes + 8 * h8);
-          vmeta[ps] = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * (h8 >> 1));
-          const uint32_t w[2] = {cw.x, cw.y};
-          float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;  // four chains
-#pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            float n[8];
-            codes8(w[k], n);
-            d0 = fmaf(qf[8 * k], n[0], d0);
-            d1 = fmaf(qf[8 * k + 1], n[1], d1);
-            d2 = fmaf(qf[8 * k + 2], n[2], d2);
-            d3 = fmaf(qf[8 * k + 3], n[3], d3);
-            d0 = fmaf(qf[8 * k + 4], n[4], d0);
-            d1 = fmaf(qf[8 * k + 5], n[5], d1);
-            d2 = fmaf(qf[8 * k + 6], n[6], d2);
-            d3 = fmaf(qf[8 * k + 7], n[7], d3);
-          }
-          // q . x_hat = zero sum(q) + scale sum(q_i code_i)
-          part = fmaf(bf16_bits_to_float(meta & 0xffffu), (d0 + d1) + (d2 + d3), bf16_bits_to_float(meta >> 16) * qsum);
+        for (int w = 0; w < 4; ++w) {
+          uint32_t ra[4], rb[4];
+          codes_bf16x2(wa[w], ra);
+          codes_bf16x2(wb[w], rb);
+          const uint4 b = *reinterpret_cast<const uint4*>(&sh.qb[lane][4 * w]);
+          mma_bf16_16816(d0, ra[0], rb[0], ra[1], rb[1], b.x, b.y);
+          mma_bf16_16816(d1, ra[2], rb[2], ra[3], rb[3], b.z, b.w);
         }
-        part += __shfl_xor_sync(0xffffffffu, part, 1);
-        part += __shfl_xor_sync(0xffffffffu, part, 2);
-        part += __shfl_xor_sync(0xffffffffu, part, 4);
-        sc[ps] = -INFINITY;
-        if (row < rows) {
-          sc[ps] = c.scale * part;
-          if (h8 == 0) p[j * kTileRows + row] = sc[ps];  // raw score, finalised after the stream
+        // lanes c4 < 2 hold the sums of groups 2 c4 and 2 c4 + 1 (columns 4..7 of the tile are zero)
+        const uint2 ma = *reinterpret_cast<const uint2*>(kt + rowA * kRowBytes + 64 + 8 * (c4 & 1));
+        const uint2 mb = *reinterpret_cast<const uint2*>(kt + rowB * kRowBytes + 64 + 8 * (c4 & 1));
+        // q . x_hat = zero sum(q) + scale sum(q_i code_i), per group
+        float pa = fmaf(bf16_bits_to_float(ma.x & 0xffffu), d0[0] + d1[0], bf16_bits_to_float(ma.x >> 16) * qsA);
+        pa += fmaf(bf16_bits_to_float(ma.y & 0xffffu), d0[1] + d1[1], bf16_bits_to_float(ma.y >> 16) * qsB);
+        float pb = fmaf(bf16_bits_to_float(mb.x & 0xffffu), d0[2] + d1[2], bf16_bits_to_float(mb.x >> 16) * qsA);
+        pb += fmaf(bf16_bits_to_float(mb.y & 0xffffu), d0[3] + d1[3], bf16_bits_to_float(mb.y >> 16) * qsB);
+        if (c4 >= 2) {
+          pa = 0.f;
+          pb = 0.f;
+        }
+        pa += __shfl_xor_sync(0xffffffffu, pa, 1);
+        pb += __shfl_xor_sync(0xffffffffu, pb, 1);
+        pa += __shfl_xor_sync(0xffffffffu, pa, 2);
+        pb += __shfl_xor_sync(0xffffffffu, pb, 2);
+        // (rows past the end hold stale bytes: whatever they gave is dropped here)
+        sA = rowA < rows ? c.scale * pa : -INFINITY;
+        sB = rowB < rows ? c.scale * pb : -INFINITY;
+        if (c4 == 0) {  // raw scores, finalised after the stream
+          if (rowA < rows) p[j * kTileRows + rowA] = sA;
+          if (rowB < rows) p[j * kTileRows + rowB] = sB;
         }
       }
-      // one softmax state per warp: maximum over its eight rows of this tile
-      float mnew = fmaxf(mg, fmaxf(sc[0], sc[1]));
+      // one softmax state per warp: maximum over its sixteen rows of this tile
+      float mnew = fmaxf(mg, fmaxf(sA, sB));
+      mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 4));
       mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 8));
       mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 16));
       if (mnew > -INFINITY) {  // warp-uniform
         const float f = expf(mg - mnew);  // expf(-inf) = 0 for the warp's first rows
-        const float e[2] = {expf(sc[0] - mnew), expf(sc[1] - mnew)};  // 0 for rows past the end
-        float esum = e[0] + e[1];  // over the warp's rows (the eight lanes of a row hold the same e)
+        const float eA = expf(sA - mnew), eB = expf(sB - mnew);  // 0 for rows past the end
+        float esum = eA + eB;  // over the warp's rows (the four lanes of a group hold the same values)
+        esum += __shfl_xor_sync(0xffffffffu, esum, 4);
         esum += __shfl_xor_sync(0xffffffffu, esum, 8);
         esum += __shfl_xor_sync(0xffffffffu, esum, 16);
         lg = fmaf(lg, f, esum);
@@ -319,12 +369,21 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
 #pragma unroll
           for (int i = 0; i < 16; ++i) o[i] *= f;
         }
+        // ---- values: four passes of four rows; row cb + 4 ps + sub has its weight in lane group (4 ps + sub) % 8 ----
 #pragma unroll
-        for (int ps = 0; ps < 2; ++ps) {
+        for (int ps = 0; ps < 4; ++ps) {
+          const int row = cb + 4 * ps + sub;
+          const float e = __shfl_sync(0xffffffffu, ps < 2 ? eA : eB, 4 * (4 * (ps & 1) + sub));
+          uint2 vw = make_uint2(0, 0);
+          uint32_t vmeta = 0;
+          if (row < rows) {
+            vw = *reinterpret_cast<const uint2*>(vt + row * kRowBytes + 8 * h8);
+            vmeta = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * (h8 >> 1));
+          }
           // p * x_hat_i = p zero + (p scale) code_i
-          const float es = e[ps] * bf16_bits_to_float(vmeta[ps] & 0xffffu);
-          zacc = fmaf(e[ps], bf16_bits_to_float(vmeta[ps] >> 16), zacc);
-          const uint32_t w[2] = {vw[ps].x, vw[ps].y};
+          const float es = e * bf16_bits_to_float(vmeta & 0xffffu);
+          zacc = fmaf(e, bf16_bits_to_float(vmeta >> 16), zacc);
+          const uint32_t w[2] = {vw.x, vw.y};
 #pragma unroll
           for (int k = 0; k < 2; ++k) {
             float n[8];
