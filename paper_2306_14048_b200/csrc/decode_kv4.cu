@@ -16,7 +16,8 @@
 // The decode step is the same fused step as decode.cu (scores over the occupied slots, softmax, P V,
 // fp64 score accumulation, victim search, in-place write), with the dequantisation folded into the
 // arithmetic: per group  q . x_hat = zero * sum(q) + scale * sum(q_i code_i)  and
-// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.
+// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.  The group sums
+// sum(q_i code_i) of the scores come from mma.sync m16n8k16 on the codes as exact bf16 values.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
