@@ -157,7 +157,10 @@ struct Shared {
   __align__(16) uint32_t qb[32][20];
 };
 
-__global__ void __launch_bounds__(kThreads + 32, 4)
+// MINB: blocks per SM the register allocation leaves room for.  A launch with at most two blocks per SM runs
+// faster with the registers the compiler wants (96, nothing spilled); many units need four resident blocks.
+template <int MINB>
+__global__ void __launch_bounds__(kThreads + 32, MINB)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted_pos, int chunk, int stages) {
@@ -541,18 +544,15 @@ gather_kv4_kernel(CacheView c, PrefillScratch s, const __nv_bfloat16* __restrict
 
 size_t kv4_row_bytes() { return kRowBytes; }
 
-cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
-                              int32_t* evicted_pos, cudaStream_t stream) {
-  const int chunk = (max_B + 3) & ~3;
-  // many units: a shallow ring lets four blocks share an SM, which hides each block's serial start and end
-  const int stages = c.units > 4 * 148 ? 2 : kStages;
-  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
-  static unsigned long long attr_flags = 0;
+template <int MINB>
+static cudaError_t launch_kv4(const CacheView& c, int chunk, int stages, size_t smem, const void* q, const void* k_new,
+                              const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  static unsigned long long attr_flags = 0;  // one word per instance, one bit per device
   {
-    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel), 200 * 1024, &attr_flags);
+    cudaError_t e =
+        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB>), 200 * 1024, &attr_flags);
     if (e != cudaSuccess) return e;
   }
-  if (smem > 200 * 1024) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)c.units);
   cfg.blockDim = dim3(kThreads + 32);
@@ -563,9 +563,20 @@ cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, cons
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stages);
+}
+
+cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
+                              int32_t* evicted_pos, cudaStream_t stream) {
+  const int chunk = (max_B + 3) & ~3;
+  // many units: a shallow ring lets four blocks share an SM, which hides each block's serial start and end
+  const int stages = c.units > 4 * 148 ? 2 : kStages;
+  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
+  if (smem > 200 * 1024) return cudaErrorInvalidValue;
+  if (c.units <= 2 * 148) return launch_kv4<2>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_kv4<4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 // after the selection kernel has written positions, scores and counts (its own row gather is skipped)
