@@ -36,8 +36,8 @@ using namespace ptx;
 
 constexpr int kD = 128;
 constexpr int kRowBytes = 80;
-constexpr int kWarps = 8;                 // consumer warps; one more warp streams the tiles
-constexpr int kThreads = kWarps * 32;
+constexpr int kMaxWarps = 8;              // consumer warps: 8, or 4 for launches of many units (twice the blocks per SM
+                                          // hide one another's serial start and end); one more warp streams the tiles
 constexpr int kTileRows = 64;             // rows per tile: eight per consumer warp
 constexpr int kTileBytes = kTileRows * kRowBytes;  // 5120
 constexpr int kStages = 4;
@@ -148,9 +148,9 @@ __device__ __forceinline__ void quantise_group(const __nv_bfloat16* src, uint4& 
 struct Shared {
   uint64_t full[kStages], empty[kStages], aux;
   uint64_t nr;  // the producer warp has quantised the new token's row
-  float red[kWarps][kD];  // per-warp partial outputs (unnormalised, relative to the warp's maximum)
-  float gm[kWarps], gl[kWarps];
-  Cand wbest[kWarps];
+  float red[kMaxWarps][kD];  // per-warp partial outputs (unnormalised, relative to the warp's maximum)
+  float gm[kMaxWarps], gl[kMaxWarps];
+  Cand wbest[kMaxWarps];
   __align__(16) unsigned char newrow[2][kRowBytes];  // the new token's K and V row, quantised
   // the query as the B operand of the score products, per lane 16 words (rows padded to 20 words: 16-byte
   // reads of eight consecutive lanes then fall into different banks)
@@ -159,11 +159,12 @@ struct Shared {
 
 // MINB: blocks per SM the register allocation leaves room for.  A launch with at most two blocks per SM runs
 // faster with the registers the compiler wants (96, nothing spilled); many units need four resident blocks.
-template <int MINB>
-__global__ void __launch_bounds__(kThreads + 32, MINB)
+template <int MINB, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32 + 32, MINB)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted_pos, int chunk, int stages) {
+  constexpr int kThreads = kWarps * 32;
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
   // dynamic layout: ring[stages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk] f32
@@ -203,7 +204,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   if (tid == kThreads) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&sh.full[s], 1);
-      mbar_init(&sh.empty[s], kWarps / 2);  // a tile is consumed by four warps
+      mbar_init(&sh.empty[s], 4);  // a tile is consumed by four warps
     }
     mbar_init(&sh.aux, 1);
     mbar_init(&sh.nr, 1);
@@ -240,7 +241,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     }
   } else {
     // ---- consumer warps --------------------------------------------------------------------------
-    // A warp takes 16 rows of a tile (warps 0..3 the even tiles, warps 4..7 the odd ones).
+    // A warp takes 16 rows of a tile (with eight warps: warps 0..3 the even tiles, warps 4..7 the odd ones).
     // Scores on the tensor cores (mma.sync m16n8k16, bf16 x bf16 -> fp32; codes 0..15 are exact in bf16):
     // A = the codes of 16 rows x 16 channels, B = the query with column n = quantisation group (zero outside
     // the group), so that one accumulator tile holds, per row, the four group sums  sum(q_i code_i);
@@ -308,7 +309,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     float zacc = 0.f;  // sum of p * zero of this lane's rows and group
     float mg = -INFINITY, lg = 0.f;
     const int cb = (warp & 3) * 16;  // the warp's rows of a tile
-    for (int j = warp >> 2; j < ntile; j += 2) {
+    for (int j = warp >> 2; j < ntile; j += kWarps / 4) {
       const int s = j % stages;
       if (!bar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
       const unsigned char* kt = ring + (size_t)s * 2 * kTileBytes;
@@ -544,18 +545,18 @@ gather_kv4_kernel(CacheView c, PrefillScratch s, const __nv_bfloat16* __restrict
 
 size_t kv4_row_bytes() { return kRowBytes; }
 
-template <int MINB>
+template <int MINB, int NW>
 static cudaError_t launch_kv4(const CacheView& c, int chunk, int stages, size_t smem, const void* q, const void* k_new,
                               const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   static unsigned long long attr_flags = 0;  // one word per instance, one bit per device
   {
     cudaError_t e =
-        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB>), 200 * 1024, &attr_flags);
+        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB, NW>), 200 * 1024, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)c.units);
-  cfg.blockDim = dim3(kThreads + 32);
+  cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute at[1];
@@ -563,7 +564,7 @@ static cudaError_t launch_kv4(const CacheView& c, int chunk, int stages, size_t 
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stages);
 }
@@ -575,8 +576,12 @@ cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, cons
   const int stages = c.units > 4 * 148 ? 2 : kStages;
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  if (c.units <= 2 * 148) return launch_kv4<2>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
-  return launch_kv4<4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  if (c.units <= 2 * 148) return launch_kv4<2, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  if (c.units > 8 * 148) {  // four consumer warps per block: five blocks per SM (no spills), six when the units are small
+    if (chunk <= 256) return launch_kv4<6, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+    return launch_kv4<5, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  }
+  return launch_kv4<4, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 // after the selection kernel has written positions, scores and counts (its own row gather is skipped)

@@ -326,6 +326,18 @@ def test_kv4_large_budget_chunk_call_and_averaged_score(H2OCache):
     print(st)
 
 
+@pytest.mark.parametrize("plen,budget", [(60, 6), (330, 150)])
+def test_kv4_many_units_four_warp_blocks(H2OCache, plen, budget):
+    """More than 8 x 148 units: the decode step runs its four-warp instances (small and large block share)."""
+    from parity_harness import run_parity
+
+    batch, heads = 38, 32
+    lens = [plen + (7 * i) % 23 for i in range(batch)]
+    wl = _wl("kv4many", batch, heads, 128, "bf16_kv4", lens, 6, [budget] * batch, [budget] * batch, seed=305)
+    st = run_parity(wl, H2OCache, units=[0, 31, 32, 500, 777, 1215], export_every=3)
+    print(st)
+
+
 def test_kv4_rejects_what_it_does_not_support(H2OCache):
     import paper_2306_14048_b200 as pkg
 
