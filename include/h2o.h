@@ -4,15 +4,19 @@
  * kept or evicted by accumulated attention score.
  *
  * Vocabulary.  A *unit* is one (sequence, head); units never interact (the
- * paper evicts "for each head", Appendix A).  Per sequence s the cache holds
+ * paper evicts per head, Appendix A).  Per sequence s the cache holds
  * B_s = k_s + r_s *slots* per head: k_s heavy hitters and the r_s most recent
- * tokens (Section 5 "evenly assigns the caching budget", Appendix A "first K
- * entries heavy hitters, last K entries most recent").  Slot order carries no
- * meaning; each slot records the token position it holds.
+ * tokens (the even split of the budget of Section 5; the heavy and recent regions
+ * of Appendix A).  Slot order carries no meaning; each slot records the token
+ * position it holds.
  *
  * Conventions common to every call
  *   - Returns 0 (H2O_OK) or a negative H2O_ERR_* code; nothing is printed, thrown
- *     or aborted.  On error no kernel has been launched by that call.
+ *     or aborted.  Argument, size and call-order errors are found before anything is
+ *     enqueued.  H2O_ERR_CUDA can come from a launch in the middle of a call that
+ *     enqueues several kernels (h2o_prefill_select, h2o_decode_chunk); the cache is
+ *     then partly written, every later prefill or decode call on it returns
+ *     H2O_ERR_STATE, and h2o_cache_reset makes it usable again.
  *   - "dev" pointers are CUDA device pointers on the cache's device, "host"
  *     pointers are ordinary host memory.  The library never allocates or frees
  *     device memory and keeps no caller pointer after a call returns, except the
@@ -45,7 +49,7 @@ extern "C" {
 
 /*
  * H2O_BF16_KV4: q / k / v / out are bf16 (head_dim 128 only); the stored K/V slots are 4-bit group-quantised
- * (the paper's Q3 "compatible with quantization": it names the combination, not a quantiser; this library's
+ * (the paper's third question, on quantisation: it names the combination, not a quantiser; this library's
  * own: groups of 32 channels, zero = group minimum, scale = bf16((max - min) / 15), code =
  * clamp(rint((x - zero) / scale), 0, 15), all in fp32; 80 bytes per row instead of 256).  A row is
  * quantised when it enters the cache: kept prompt rows at selection, a new token's row after its own
@@ -88,8 +92,8 @@ size_t h2o_prefill_scratch_bytes(const h2o_config_t* cfg, int64_t total_tokens);
  * h2o_cache_workspace_bytes(cfg) bytes).  The budget arrays are copied.  Small
  * tables are copied to the device synchronously; no kernel state survives a
  * failed create.  *out is set only on success.
- * Pre-allocated storage that is overwritten in place follows Section 4.2
- * ("do not swap memory ... directly fill with newly-added KV") and Appendix A.
+ * Pre-allocated storage whose evicted entry is overwritten by the new one, without
+ * moving any other row, follows Section 4.2 (implementation details) and Appendix A.
  */
 int h2o_cache_create(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_workspace, size_t workspace_bytes);
 
@@ -107,8 +111,8 @@ int h2o_cache_attach(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_works
 
 /*
  * Prefill selection (Appendix A pseudocode, prefill branch: attention over the
- * whole prompt, then "select K heavy hitters and K recent tokens", all tokens
- * if the prompt is not longer than the budget).  For every unit:
+ * whole prompt, then the heavy hitters and the most recent tokens are kept, all
+ * tokens if the prompt is not longer than the budget).  For every unit:
  *   P[i][j] = softmax_j(c q_i.k_j), j <= i          causal attention, n_s rows
  *   out_i   = sum_j P[i][j] v_j
  *   acc0[j] = sum_{i >= j} P[i][j]                   accumulated score (Algorithm 2, accumulation line)

@@ -21,7 +21,7 @@
  *     K heavy + K recent (all if the prompt is shorter); eviction is skipped
  *     while the cache is not full (Appendix A, system details and pseudocode).
  *
- * Readings taken where the paper leaves a choice (each is listed in the design notes):
+ * Readings taken where the paper leaves a choice:
  *   - token t attends to the kept set plus itself, then one entry is evicted;
  *   - scores are accumulated at every step, also while the cache is filling, and
  *     the prompt's column sums are carried into decoding;

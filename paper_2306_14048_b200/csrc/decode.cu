@@ -535,7 +535,7 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   // bytes in flight; with many blocks a shallow ring lets more of them be resident, which hides each
   // block's serial prologue and epilogue behind the others' streams.
   const int blocks = c.units * split;
-  const int auto_stages = blocks > 4 * 148 ? 2 : kDefaultStages;
+  const int auto_stages = blocks > 4 * sm_count() ? 2 : kDefaultStages;
   const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : auto_stages;
   int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
   stages = stages < 1 ? 1 : (stages > want ? want : stages);
@@ -571,9 +571,9 @@ template <typename T, int D>
 cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, int quiescent, const void* q,
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   const int blocks = c.units * split;
-  if (blocks > 4 * 148 && chunk <= kSmallUnitRows)  // many small units: half-size blocks, five per SM
+  if (blocks > 4 * sm_count() && chunk <= kSmallUnitRows)  // many small units: half-size blocks, five per SM
     return launch_minb<T, D, 5, 4>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
-  if (blocks > 2 * 148)
+  if (blocks > 2 * sm_count())
     return launch_minb<T, D, 4, 8>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
   return launch_minb<T, D, 1, 8>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
 }

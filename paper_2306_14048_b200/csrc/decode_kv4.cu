@@ -25,7 +25,7 @@
 #include <cmath>
 #include <cstdint>
 
-#include "../../include/h2o.h"
+#include "h2o.h"
 #include "h2o_internal.cuh"
 #include "sm100_ptx.cuh"
 
@@ -573,11 +573,11 @@ cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, cons
                               int32_t* evicted_pos, cudaStream_t stream) {
   const int chunk = (max_B + 3) & ~3;
   // many units: a shallow ring lets four blocks share an SM, which hides each block's serial start and end
-  const int stages = c.units > 4 * 148 ? 2 : kStages;
+  const int stages = c.units > 4 * sm_count() ? 2 : kStages;
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  if (c.units <= 2 * 148) return launch_kv4<2, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
-  if (c.units > 8 * 148) {  // four consumer warps per block: five blocks per SM (no spills), six when the units are small
+  if (c.units <= 2 * sm_count()) return launch_kv4<2, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  if (c.units > 8 * sm_count()) {  // four consumer warps per block: five blocks per SM (no spills), six when the units are small
     if (chunk <= 256) return launch_kv4<6, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
     return launch_kv4<5, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
   }

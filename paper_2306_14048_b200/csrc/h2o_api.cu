@@ -106,7 +106,9 @@ ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens)
   return S;
 }
 
-enum class Phase { Empty, Prefilled, Decoding };
+// Failed: a launch of a multi-kernel call was refused after earlier work of the same call had been enqueued; the
+// workspace is then partly written and only h2o_cache_reset (or destroy) is accepted.
+enum class Phase { Empty, Prefilled, Decoding, Failed };
 
 }  // namespace
 
@@ -266,7 +268,8 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   // Thread blocks per unit.  One block per unit unless there are fewer units than SMs: sharing a
   // unit costs three cluster barriers per step, which only pays when SMs would otherwise idle.
   int split = 1;
-  while (split < 8 && (((int64_t)units * split < 148 && L.max_B / (2 * split) >= 64) ||
+  const int sms = h2o::sm_count();
+  while (split < 8 && (((int64_t)units * split < sms && L.max_B / (2 * split) >= 64) ||
                        (L.max_B + split - 1) / split > kMaxChunk))
     split *= 2;
   c->split = split;
@@ -315,6 +318,10 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
     ok = ok && cudaMemset(ws + L.acc, 0, L.meta - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
     ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
     ok = ok && cudaMemcpy(ws + L.meta, meta.data(), units * sizeof(h2o::UnitMeta), cudaMemcpyHostToDevice) == cudaSuccess;
+    // The memsets are asynchronous and a pageable copy returns once the data is staged, all on the legacy default
+    // stream, which a non-blocking stream is not ordered behind: wait here, so that the tables are on the device
+    // whatever stream the caller uses next.
+    ok = ok && cudaStreamSynchronize(0) == cudaSuccess;
   }
   if (!ok) {
     cudaGetLastError();
@@ -403,10 +410,13 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   } else {
     e = h2o::launch_prefill_naive(cache->view, ps, in_dtype, max_seqlen, q, k, v, out, true, true, st);
   }
-  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, in_dtype, cache->layout.max_B, max_seqlen, k, v, st);
+  if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, in_dtype, std::min(cache->layout.max_B, max_seqlen), max_seqlen, k, v, st);
   if (e == cudaSuccess && cache->view.kv4) e = h2o::launch_gather_kv4(cache->view, ps, k, v, st);
   if (e != cudaSuccess) {
+    // earlier kernels of this call may already be enqueued and have written part of the workspace
     cudaGetLastError();
+    g_last_writer.note_and_check(st, cache->view.K);
+    cache->phase = Phase::Failed;
     return H2O_ERR_CUDA;
   }
   g_last_writer.note_and_check(st, cache->view.K);  // select/gather wrote this cache
@@ -418,6 +428,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
 int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const void* v_new, void* out,
                     int32_t* evicted_pos, void* stream) {
   if (!cache || !q || !k_new || !v_new || !out) return H2O_ERR_INVALID_ARG;
+  if (cache->phase == Phase::Failed) return H2O_ERR_STATE;
   for (const void* p : {q, k_new, v_new, (const void*)out})
     if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
   DeviceGuard guard(cache->cfg.device);
@@ -442,6 +453,7 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
 int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const void* v, int32_t n_tokens, void* out,
                      int32_t* evicted_pos, void* stream) {
   if (!cache || !q || !k || !v || !out || n_tokens < 1) return H2O_ERR_INVALID_ARG;
+  if (cache->phase == Phase::Failed) return H2O_ERR_STATE;
   for (const void* p : {q, k, v, (const void*)out})
     if (reinterpret_cast<uintptr_t>(p) % 16 != 0) return H2O_ERR_INVALID_ARG;
   DeviceGuard guard(cache->cfg.device);
@@ -471,7 +483,9 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
     }
   }
   if (e != cudaSuccess) {
+    // some of the tokens may already have been enqueued: the cache no longer matches what the caller knows
     cudaGetLastError();
+    cache->phase = Phase::Failed;
     return H2O_ERR_CUDA;
   }
   cache->phase = Phase::Decoding;

@@ -76,6 +76,19 @@ inline cudaError_t ensure_dynamic_smem(const void* func, int bytes, unsigned lon
   return e;
 }
 
+// SMs of the current device (asked once per device; the dispatch thresholds of the launchers scale with it).
+inline int sm_count() {
+  static int cached[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
 // Launchers (each returns the cudaError_t of its launch).
 // `split` thread blocks (one cluster) share a unit, each owning `chunk` consecutive slots.
 // `stages` is the depth of the shared-memory ring (0 = default).  `quiescent`: nothing this library

@@ -1299,21 +1299,6 @@ extern "C" int h2o_debug_fwd_prof(unsigned long long* host, int reset) {
 #endif
 
 namespace {
-// SMs of the current device (asked once per device)
-int sm_count() {
-  static int cached[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (cached[dev] == 0) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    cached[dev] = n;
-  }
-  return cached[dev];
-}
-}  // namespace
-
-namespace {
 
 template <int G>
 cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_v, const CacheView& c,

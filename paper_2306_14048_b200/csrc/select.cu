@@ -11,8 +11,8 @@
 // histogram per pass, the histogram searched by a block-wide scan.  Everything is integer work after the column sums exist, so
 // the result is exact.
 //
-// Paper: Appendix A pseudocode, prefill branch ("select K heavy hitters and K recent
-// tokens"; all tokens when the prompt is not longer than 2K).
+// Paper: Appendix A pseudocode, prefill branch (K heavy hitters and K recent tokens are
+// kept; all tokens when the prompt is not longer than 2K).
 #include "h2o_internal.cuh"
 
 namespace h2o {
@@ -56,7 +56,7 @@ template <typename T, int D, int KPT>
 __global__ void __launch_bounds__(kSelThreads)
 select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, const T* __restrict__ v) {
   constexpr int VEC = Vec16<T>::N, LPR = D / VEC;
-  extern __shared__ int32_t kept[];  // [B]
+  extern __shared__ int32_t kept[];  // [min(B, longest prompt)]
   __shared__ unsigned int hist[256];
   __shared__ int warp_tot[kSelThreads / 32];
   __shared__ uint64_t prefix_sh;

@@ -14,9 +14,6 @@ constexpr uint32_t kSpinLimit = 1u << 24;  // polls before a wait gives up
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// One lane of a converged warp (the same lane every time).  The MMA-issuing warp runs its loop with
-// all lanes, so that descriptors and addresses stay warp-uniform (uniform registers), and predicates
-// only the single-thread instructions with this.
 // Same box as tma_load_tile, fetched into L2 only.
 __device__ __forceinline__ void tma_prefetch_tile(const CUtensorMap* map, int head, int row) {
   asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(0), "r"(row), "r"(0),

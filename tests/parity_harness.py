@@ -10,6 +10,8 @@ scores must agree within the stated tolerance.
 from __future__ import annotations
 
 import dataclasses
+import json
+import os
 from typing import Optional, Sequence
 
 import numpy as np
@@ -31,6 +33,16 @@ class ParityStats:
     near_ties_prefill: int = 0
     max_out_err: float = 0.0
     max_acc_err: float = 0.0
+
+
+def record(stats: ParityStats, case: str) -> None:
+    """One JSON line per parity case: printed, and appended to the file named by H2O_PARITY_LOG when that is set."""
+    line = json.dumps({"case": case, **dataclasses.asdict(stats)})
+    print(line)
+    path = os.environ.get("H2O_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
 
 
 def assert_close(got, want, dtype: str, what: str):
@@ -78,7 +90,7 @@ def _gather_units(x, cu, units, H):
 def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = None, steps: Optional[int] = None,
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
                device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
-               pattern: Optional[Sequence[int]] = None, score_mode: int = 0) -> ParityStats:
+               pattern: Optional[Sequence[int]] = None, score_mode: int = 0, static_scratch: bool = False) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
@@ -86,12 +98,13 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     interact.  With ``chunk`` > 0 the CUDA path advances ``chunk`` tokens per call (h2o_decode_chunk)
     while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
     sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
+    ``scale`` > 0 replaces the default softmax scale 1/sqrt(d) (4/sqrt(d) is the peaky-softmax stress run).
     """
     if score_mode > 0:  # the oracle's ranking rule is process-wide: always put it back
         h2o_oracle.set_score_mode(score_mode)
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
-                              chunk, chunk_path, pattern, score_mode=0 - score_mode)
+                              chunk, chunk_path, pattern, score_mode=0 - score_mode, static_scratch=static_scratch)
         finally:
             h2o_oracle.set_score_mode(0)
     score_mode = -score_mode  # (negative: the oracle is already in that mode)
@@ -111,7 +124,10 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     if prefill:
         q, k, v, cu = make_prompt_inputs(wl, layer=layer, device=device)
         out = torch.empty_like(q)
-        gpu.prefill_select(q, k, v, cu, out)
+        if static_scratch:  # the entry point that takes no scratch buffer
+            gpu.prefill_select_static(q, k, v, cu, out)
+        else:
+            gpu.prefill_select(q, k, v, cu, out)
         assert gpu.status() == 0
         qh, ocu = _gather_units(q, cu, units, H)
         kh, _ = _gather_units(k, cu, units, H)

@@ -186,6 +186,38 @@ def test_caches_on_different_streams(pkg):
         c.close()
 
 
+def test_create_then_decode_at_once_on_a_non_blocking_stream(pkg):
+    """h2o_cache_create returns with its tables on the device: a stream that is not ordered behind the legacy
+    default stream (every torch side stream is non-blocking) may be used right away, with no synchronisation
+    between create and the first call."""
+    wl = Workload("fresh", 4, 8, 128, "bf16", (1, 1, 1, 1), 24, (6, 8, 4, 10), (6, 8, 4, 10), 1, 910)
+    ins = [make_decode_inputs(wl, s, device="cuda") for s in range(wl.decode_steps)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    runs = []
+    for rep in range(6):
+        # dirty a block of memory the allocator will hand to the next workspace
+        junk = torch.full((pkg.h2o_cache_workspace_bytes(pkg.make_config(
+            wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)[0]) + 256,), 0x5A, dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()
+        del junk
+        cache = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+        outs, evs = [], []
+        for dq, dk, dv in ins:  # token-by-token from the empty cache, nothing in between
+            do = torch.empty_like(dq)
+            de = torch.empty(wl.batch, wl.n_heads, dtype=torch.int32, device="cuda")
+            cache.decode_step(dq, dk, dv, do, de, side)
+            outs.append(do)
+            evs.append(de)
+        side.synchronize()
+        assert cache.status(side) == 0
+        runs.append(([o.float().cpu().numpy() for o in outs], [e.cpu().numpy() for e in evs], cache.export(side)))
+        cache.close()
+    for r in runs[1:]:
+        _identical(runs[0], r)
+    assert (runs[0][2][3] == wl.decode_steps).all()  # every unit advanced from t = 0
+
+
 def test_snapshot_and_attach_resume_bit_identically(pkg):
     """The workspace bytes are the whole state: a handle attached to a copy continues exactly like the original,
     also through a file-like round trip on the host; a different configuration is refused."""
