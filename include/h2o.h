@@ -301,6 +301,15 @@ int h2o_debug_set_early_prefetch(int32_t enabled);
  */
 int h2o_debug_wait_probe(h2o_cache_t* cache, int32_t polls, void* stream);
 int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, size_t* acc0_offset);
+/*
+ * Diagnostic (no counterpart in the paper): per-kernel timing of the NEXT h2o_prefill_select call on this
+ * cache.  `events`: host array of four cudaEvent_t (created by the caller with timing enabled; NULL entries
+ * are skipped), recorded on that call's stream before the attention kernel (P1-P3 of the path), after it,
+ * after the column-sum kernel (P4) and after selection and gather (P5-P6).  The handles are used by that one
+ * call only; `events` == NULL cancels.  Recording between the kernels orders them strictly, so a timed call
+ * can be a little slower than an untimed one.
+ */
+int h2o_debug_set_prefill_events(h2o_cache_t* cache, void* const* events);
 const char* h2o_strerror(int code);
 
 #ifdef __cplusplus

@@ -119,6 +119,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_prefill_scratch_layout.argtypes = [cfgp, c.c_int64, c.POINTER(c.c_size_t)]
     lib.h2o_debug_set_early_prefetch.restype = c.c_int
     lib.h2o_debug_set_early_prefetch.argtypes = [c.c_int32]
+    lib.h2o_debug_set_prefill_events.restype = c.c_int
+    lib.h2o_debug_set_prefill_events.argtypes = [vp, c.POINTER(vp)]
     lib.h2o_strerror.restype = c.c_char_p
     lib.h2o_strerror.argtypes = [c.c_int]
     return lib
@@ -288,6 +290,12 @@ class H2OCache:
 
     def set_decode_shape(self, split: int = 0, stages: int = 0):
         _check(lib.h2o_cache_set_decode_shape(self._h, int(split), int(stages)), "h2o_cache_set_decode_shape")
+
+    def set_prefill_events(self, events):
+        """h2o_debug_set_prefill_events: four torch.cuda.Event(enable_timing=True), already recorded once (torch
+        creates the CUDA handle lazily), for the next prefill_select call."""
+        arr = (ctypes.c_void_p * 4)(*[int(e.cuda_event) for e in events])
+        _check(lib.h2o_debug_set_prefill_events(self._h, arr), "h2o_debug_set_prefill_events")
 
     def set_prefill_path(self, path: int):
         _check(lib.h2o_cache_set_prefill_path(self._h, int(path)), "h2o_cache_set_prefill_path")

@@ -124,6 +124,7 @@ struct h2o_cache {
   Layout layout;
   h2o::CacheView view;
   Phase phase;
+  cudaEvent_t prefill_events[4] = {nullptr, nullptr, nullptr, nullptr};  // see h2o_debug_set_prefill_events
 };
 
 namespace {
@@ -404,14 +405,31 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   const int in_dtype = input_dtype(cfg.dtype);
   const bool tc = cache->prefill_path != 1 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
   cudaError_t e = cudaSuccess;
+  // optional phase events of this one call (diagnostic): before the forward kernel, after it, after the column
+  // sums, after selection and gather
+  cudaEvent_t pev[4];
+  for (int i = 0; i < 4; ++i) {
+    pev[i] = cache->prefill_events[i];
+    cache->prefill_events[i] = nullptr;
+  }
+  auto stamp = [&](int i) {
+    if (e == cudaSuccess && pev[i]) e = cudaEventRecord(pev[i], st);
+  };
+  stamp(0);
   if (tc) {
-    e = h2o::launch_fwd_tc(cache->view, ps, max_seqlen, q, k, v, out, st);
+    if (e == cudaSuccess) e = h2o::launch_fwd_tc(cache->view, ps, max_seqlen, q, k, v, out, st);
+    stamp(1);
     if (e == cudaSuccess) e = h2o::launch_colsum_tc(cache->view, ps, max_seqlen, q, k, st);
+    stamp(2);
   } else {
-    e = h2o::launch_prefill_naive(cache->view, ps, in_dtype, max_seqlen, q, k, v, out, true, true, st);
+    if (e == cudaSuccess) e = h2o::launch_prefill_naive(cache->view, ps, in_dtype, max_seqlen, q, k, v, out, true, false, st);
+    stamp(1);
+    if (e == cudaSuccess) e = h2o::launch_prefill_naive(cache->view, ps, in_dtype, max_seqlen, q, k, v, out, false, true, st);
+    stamp(2);
   }
   if (e == cudaSuccess) e = h2o::launch_select_gather(cache->view, ps, in_dtype, std::min(cache->layout.max_B, max_seqlen), max_seqlen, k, v, st);
   if (e == cudaSuccess && cache->view.kv4) e = h2o::launch_gather_kv4(cache->view, ps, k, v, st);
+  stamp(3);
   if (e != cudaSuccess) {
     // earlier kernels of this call may already be enqueued and have written part of the workspace
     cudaGetLastError();
@@ -643,6 +661,12 @@ int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, si
   if (check_config(cfg) != H2O_OK || total_tokens < 1 || total_tokens > INT32_MAX) return H2O_ERR_INVALID_ARG;
   const ScratchLayout S = make_scratch_layout(cfg, total_tokens);
   if (acc0_offset) *acc0_offset = S.acc0;
+  return H2O_OK;
+}
+
+int h2o_debug_set_prefill_events(h2o_cache_t* cache, void* const* events) {
+  if (!cache) return H2O_ERR_INVALID_ARG;
+  for (int i = 0; i < 4; ++i) cache->prefill_events[i] = events ? static_cast<cudaEvent_t>(events[i]) : nullptr;
   return H2O_OK;
 }
 
