@@ -60,6 +60,37 @@ int h2o_oracle_num_threads(void) {
 }
 
 /*
+ * Sparse attention patterns combined with the heavy hitters (the table of Section 5.1 that lists the strided
+ * and fixed Sparse Transformer patterns with and without H2).  The paper reports the combination but gives no
+ * formula; the reading taken here: the cache keeps exactly what it keeps without a pattern (k heavy hitters by
+ * accumulated score, the r most recent positions); the pattern decides which entries of the RECENT region a
+ * query attends.  For the query at position t and a key at position p:
+ *   p == t          : attended (the token itself);
+ *   p <= t - r      : attended (older than the window: a heavy hitter, or the candidate that has just left it);
+ *   t - r < p < t   : attended iff the pattern allows (p, t):
+ *       kind 1, strided(l, w): t - p < w (local) or (t - p) mod l == 0 (every l-th position back);
+ *       kind 2, fixed(l, c)  : floor(p / l) == floor(t / l) (same block) or p mod l >= l - c (summary columns).
+ * An entry that is not attended is absent from numerator and normaliser of that row and receives no score from
+ * it.  "Without H2" is k = 0.  kind 0 = no pattern (everything in the window attended).
+ */
+static int g_mask_kind = 0;
+static long g_mask_a = 1, g_mask_b = 1;
+int h2o_oracle_set_mask(int kind, long a, long b) {
+  if (kind < 0 || kind > 2) return -1;
+  if (kind != 0 && (a < 1 || b < 0)) return -1;
+  if (kind == 2 && b > a) return -1;
+  g_mask_kind = kind;
+  g_mask_a = a;
+  g_mask_b = b;
+  return 0;
+}
+static int attended(long p, long t, long r) {
+  if (p == t || p <= t - r || g_mask_kind == 0) return 1;
+  if (g_mask_kind == 1) return (t - p) < g_mask_b || (t - p) % g_mask_a == 0;
+  return p / g_mask_a == t / g_mask_a || p % g_mask_a >= g_mask_a - g_mask_b;
+}
+
+/*
  * Causal softmax attention of one (sequence, head) and the column sums of its
  * probability matrix.
  *   Q, K, V : n rows of d floats, consecutive rows `stride` floats apart.
@@ -69,9 +100,11 @@ int h2o_oracle_num_threads(void) {
  *   acc0    : [n]     acc0[j] = sum_{i>=j} P[i][j]   (summed for increasing i)
  *   P_out   : optional [n][n] (NULL to skip), zero above the diagonal.
  * P[i][j] = exp(s_ij - m_i) / l_i with s_ij = c <Q_i, K_j>, j <= i.
+ * With a sparse pattern set (h2o_oracle_set_mask) row i leaves out the keys j of its recent window
+ * (i - r < j < i, r = `window`) that the pattern does not allow: P[i][j] = 0 there.
  */
 int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const float* V, long n, long d, long stride,
-                                       double c, double* O, double* rowmax, double* rowsum, double* acc0,
+                                       double c, long window, double* O, double* rowmax, double* rowsum, double* acc0,
                                        double* P_out) {
   if (n < 0 || d <= 0 || stride < d) return -1;
   int failed = 0;
@@ -88,12 +121,13 @@ int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const flo
       const float* qi = Q + i * stride;
       double m = -INFINITY;
       for (long j = 0; j <= i; ++j) {
+        if (!attended(j, i, window)) continue;
         e[j] = c * dot_fd(qi, K + j * stride, d);
         if (e[j] > m) m = e[j];
       }
       double l = 0.0;
       for (long j = 0; j <= i; ++j) {
-        e[j] = exp(e[j] - m);
+        e[j] = attended(j, i, window) ? exp(e[j] - m) : 0.0;
         l += e[j];
       }
       rowmax[i] = m;
@@ -116,6 +150,7 @@ int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const flo
       const float* kj = K + j * stride;
       double a = 0.0;
       for (long i = j; i < n; ++i) {
+        if (!attended(j, i, window)) continue;
         const double s = c * dot_fd(Q + i * stride, kj, d);
         a += exp(s - rowmax[i]) / rowsum[i];
       }
@@ -271,6 +306,7 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
     double* e = (double*)malloc(sizeof(double) * (size_t)m);
     double mx = -INFINITY;
     for (long j = 0; j < m; ++j) {
+      if (!attended(up[j], tt, r)) continue; /* left out by the sparse pattern (none by default) */
       double s = 0.0;
       for (long x = 0; x < d; ++x) s += (double)q[u * d + x] * uk[j * d + x];
       e[j] = c * s;
@@ -278,7 +314,7 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
     }
     double l = 0.0;
     for (long j = 0; j < m; ++j) {
-      e[j] = exp(e[j] - mx);
+      e[j] = attended(up[j], tt, r) ? exp(e[j] - mx) : 0.0;
       l += e[j];
     }
     double* o = out + u * d;

@@ -42,7 +42,7 @@ def _load():
         dp, fp, ip = c.POINTER(c.c_double), c.POINTER(c.c_float), c.POINTER(c.c_int32)
         lib.h2o_oracle_num_threads.restype = c.c_int
         lib.h2o_oracle_causal_attention_colsum.restype = c.c_int
-        lib.h2o_oracle_causal_attention_colsum.argtypes = [fp, fp, fp, c.c_long, c.c_long, c.c_long, c.c_double, dp, dp, dp, dp, dp]
+        lib.h2o_oracle_causal_attention_colsum.argtypes = [fp, fp, fp, c.c_long, c.c_long, c.c_long, c.c_double, c.c_long, dp, dp, dp, dp, dp]
         lib.h2o_oracle_select.restype = c.c_long
         lib.h2o_oracle_select.argtypes = [dp, c.c_long, c.c_long, c.c_long, ip, dp]
         lib.h2o_oracle_decode_step.restype = c.c_int
@@ -50,6 +50,8 @@ def _load():
                                                c.c_double, ip, c.c_double, dp, ip, ip, dp, dp]
         lib.h2o_oracle_set_score_mode.restype = c.c_int
         lib.h2o_oracle_set_score_mode.argtypes = [c.c_int]
+        lib.h2o_oracle_set_mask.restype = c.c_int
+        lib.h2o_oracle_set_mask.argtypes = [c.c_int, c.c_long, c.c_long]
         lib.h2o_oracle_fscore.restype = c.c_double
         lib.h2o_oracle_fscore.argtypes = [dp, c.c_long, c.c_int]
         _lib = lib
@@ -71,8 +73,9 @@ def _f32(x) -> np.ndarray:
     return np.ascontiguousarray(x, dtype=np.float32)
 
 
-def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False):
-    """One unit: q, k, v ``[n, d]`` views (row stride may exceed d).  Returns O, acc0, (P)."""
+def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False, window: int = 0):
+    """One unit: q, k, v ``[n, d]`` views (row stride may exceed d).  Returns O, acc0, (P).
+    ``window``: the unit's recent window r; only read when a sparse pattern is set (``set_mask``)."""
     n, d = q.shape
     assert q.dtype == np.float32 and k.dtype == np.float32 and v.dtype == np.float32
     stride = q.strides[0] // 4
@@ -83,7 +86,7 @@ def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False):
     acc0 = np.empty(n, dtype=np.float64)
     P = np.empty((n, n), dtype=np.float64) if want_p else None
     rc = _load().h2o_oracle_causal_attention_colsum(
-        _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), n, d, stride, float(scale),
+        _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), n, d, stride, float(scale), int(window),
         _p(O, ctypes.c_double), _p(rowmax, ctypes.c_double), _p(rowsum, ctypes.c_double), _p(acc0, ctypes.c_double),
         _p(P, ctypes.c_double))
     if rc != 0:
@@ -97,6 +100,17 @@ def set_score_mode(mode: int) -> None:
     Process-wide: the tests that use mode 1 set it back to 0 when they are done."""
     if _load().h2o_oracle_set_score_mode(int(mode)) != 0:
         raise ValueError("score mode must be 0 or 1")
+
+
+MASK_NONE, MASK_STRIDED, MASK_FIXED = 0, 1, 2
+
+
+def set_mask(kind: int, a: int = 1, b: int = 1) -> None:
+    """Sparse pattern applied inside the recent window (combination of the heavy hitters with the strided / fixed
+    Sparse Transformer patterns): 0 none; 1 strided(stride a, local window b); 2 fixed(block a, b summary columns).
+    Process-wide, like the score mode: tests that set it put it back to 0."""
+    if _load().h2o_oracle_set_mask(int(kind), int(a), int(b)) != 0:
+        raise ValueError("bad mask parameters")
 
 
 def fscore(acc: np.ndarray, hkind: int = 0) -> float:
@@ -160,7 +174,7 @@ class OracleCache:
         for u in todo:
             s, h = divmod(u, self.n_heads)
             lo, hi = int(cu[s]), int(cu[s + 1])
-            O, acc0 = causal_attention_colsum(q[lo:hi, h], k[lo:hi, h], v[lo:hi, h], self.scale)
+            O, acc0 = causal_attention_colsum(q[lo:hi, h], k[lo:hi, h], v[lo:hi, h], self.scale, window=int(self.rwin[u]))
             out[lo:hi, h] = O
             kept, boundary = select(acc0, int(self.kbud[u]), int(self.rwin[u]))
             self.last_acc0[u], self.last_boundary[u] = acc0, boundary

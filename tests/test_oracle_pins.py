@@ -102,8 +102,9 @@ class LiteralH2O:
     candidate v, taking the argmax.
     """
 
-    def __init__(self, k, r, scale, h):
+    def __init__(self, k, r, scale, h, attend=None):
         self.k, self.r, self.c, self.h = k, r, scale, h
+        self.attend = attend  # optional predicate (key position, query position, r) -> attended?
         self.S = []  # kept positions
         self.rows = []  # rows[i][j] = probability token i gave token j
         self.K, self.V = {}, {}
@@ -119,12 +120,14 @@ class LiteralH2O:
         t = self.t
         self.K[t], self.V[t] = k_new, v_new
         G = self.S + [t]
-        logits = [self.c * math.fsum(float(a) * float(b) for a, b in zip(q, self.K[j])) for j in G]
+        seen = [j for j in G if self.attend is None or self.attend(j, t, self.r)]
+        logits = [self.c * math.fsum(float(a) * float(b) for a, b in zip(q, self.K[j])) for j in seen]
         mx = max(logits)
         w = [math.exp(x - mx) for x in logits]
         tot = math.fsum(w)
-        probs = [x / tot for x in w]
-        self.rows.append({j: p for j, p in zip(G, probs)})
+        row = {j: x / tot for j, x in zip(seen, w)}
+        probs = [row.get(j, 0.0) for j in G]
+        self.rows.append(row)
         out = [math.fsum(p * float(self.V[j][x]) for j, p in zip(G, probs)) for x in range(len(q))]
         evicted = -1
         min_gap = math.inf
@@ -546,3 +549,149 @@ def test_kv4_cache_stores_quantised_rows_but_attends_the_new_token_exactly(oracl
         np.testing.assert_array_equal(res4["out"], resr["out"])
     m = int(c4.cnt[0])
     np.testing.assert_array_equal(c4.K[0, :m], kv_quant.qdq(c4.K[0, :m].astype(np.float32)))  # stored rows are on the grid
+
+
+# --------------------------------------------------------------------------
+# sparse patterns inside the recent window (heavy hitters combined with the strided / fixed masks)
+# --------------------------------------------------------------------------
+def _pattern(kind, a, b):
+    """(key position p, query position t) -> allowed by the pattern, written on arrays."""
+    if kind == "strided":
+        return lambda p, t: ((t - p) < b) | ((t - p) % a == 0)
+    return lambda p, t: ((p // a) == (t // a)) | ((p % a) >= a - b)
+
+
+def _mask_matrix(T, r, pat):
+    """M[t][j]: key j attended by query t under the reading: itself, everything older than the window,
+    and of the window what the pattern allows."""
+    t, j = np.indices((T, T))
+    return (j <= t) & ((j == t) | (j <= t - r) | pat(j, t))
+
+
+def _textbook_masked(q, k, v, scale, M):
+    s = scale * (q.astype(np.float64) @ k.astype(np.float64).T)
+    p = scipy_softmax(np.where(M, s, -np.inf), axis=1)
+    return p @ v.astype(np.float64), p
+
+
+MASKS = [("strided", 1, 4, 2), ("strided", 1, 3, 1), ("fixed", 2, 4, 1), ("fixed", 2, 5, 2)]  # (name, kind, a, b)
+
+
+@pytest.fixture
+def masked(oracle):
+    def use(kind, a, b):
+        oracle.set_mask(kind, a, b)
+
+    yield use
+    oracle.set_mask(0)
+
+
+def test_a_pattern_that_allows_the_whole_window_changes_nothing(oracle, masked):
+    n, steps, d, k, r, scale = 40, 30, 8, 5, 6, 0.5
+    rng = np.random.default_rng(31)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+
+    def run():
+        cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+        out, kept = cache.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+        res = [cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None]) for t in range(n, n + steps)]
+        return out, kept[0], [x["out"] for x in res], [int(x["evicted"][0]) for x in res], cache.export(0)
+
+    ref = run()
+    for kind, a, b in ((1, 3, r), (1, 1, 0), (2, 4, 4), (2, 1000, 0)):  # local window >= r; stride 1; all columns summary; one block
+        masked(kind, a, b)
+        got = run()
+        np.testing.assert_array_equal(got[0], ref[0])
+        np.testing.assert_array_equal(got[1], ref[1])
+        assert got[3] == ref[3]
+        for x, y in zip(got[2], ref[2]):
+            np.testing.assert_array_equal(x, y)
+        np.testing.assert_array_equal(got[4][0], ref[4][0])
+        np.testing.assert_array_equal(got[4][1], ref[4][1])
+
+
+@pytest.mark.parametrize("name,kind,a,b", MASKS)
+def test_masked_prompt_attention_is_textbook_masked_attention(oracle, masked, name, kind, a, b):
+    n, d, r, scale = 48, 8, 9, 0.4
+    rng = np.random.default_rng(32 + a)
+    q, kk, v = _rand_qkv(rng, n, d)
+    M = _mask_matrix(n, r, _pattern(name, a, b))
+    assert not M[np.tril_indices(n)].all()  # the pattern really removes something
+    ref_out, ref_p = _textbook_masked(q, kk, v, scale, M)
+    masked(kind, a, b)
+    O, acc0, P = oracle.causal_attention_colsum(q, kk, v, scale, want_p=True, window=r)
+    np.testing.assert_allclose(O, ref_out, rtol=1e-11, atol=1e-13)
+    np.testing.assert_allclose(P, ref_p, rtol=1e-11, atol=1e-300)
+    np.testing.assert_allclose(acc0, ref_p.sum(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(P.sum(axis=1), 1.0, rtol=1e-14)
+
+
+@pytest.mark.parametrize("name,kind,a,b", MASKS)
+def test_masked_zero_heavy_budget_is_the_pattern_alone(oracle, masked, name, kind, a, b):
+    """Without heavy hitters (k = 0) the token-by-token policy is plain masked attention: the window entries the
+    pattern allows, the token that is just leaving the window, and the token itself."""
+    T, d, r, scale = 40, 8, 7, 0.5
+    rng = np.random.default_rng(33 + b)
+    q, kk, v = _rand_qkv(rng, T, d)
+    t, j = np.indices((T, T))
+    M = (j <= t) & (j >= t - r) & _mask_matrix(T, r, _pattern(name, a, b))
+    ref_out, _ = _textbook_masked(q, kk, v, scale, M)
+    masked(kind, a, b)
+    cache = oracle.OracleCache(1, 1, d, [0], [r], scale=scale)
+    for step in range(T):
+        res = cache.decode_step(q[step][None, None], kk[step][None, None], v[step][None, None])
+        np.testing.assert_allclose(res["out"][0], ref_out[step], rtol=1e-11, atol=1e-13)
+        assert res["evicted"][0] == (step - r if step >= r else -1)
+
+
+@pytest.mark.parametrize("name,kind,a,b", MASKS)
+def test_masked_cache_that_never_evicts_is_textbook_masked_attention(oracle, masked, name, kind, a, b):
+    n, steps, d, r, scale = 30, 14, 8, 8, 0.35
+    rng = np.random.default_rng(34 + a + b)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+    M = _mask_matrix(n + steps, r, _pattern(name, a, b))
+    ref_out, ref_p = _textbook_masked(q, kk, v, scale, M)
+    masked(kind, a, b)
+    one_shot = oracle.OracleCache(1, 1, d, [n + steps], [r], scale=scale)
+    token_by_token = oracle.OracleCache(1, 1, d, [n + steps], [r], scale=scale)
+    out, kept = one_shot.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    np.testing.assert_allclose(out[:, 0], ref_out[:n], rtol=1e-11, atol=1e-13)
+    for t in range(n + steps):
+        rb = token_by_token.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        np.testing.assert_allclose(rb["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+        if t >= n:
+            ra = one_shot.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+            np.testing.assert_allclose(ra["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+    for cache in (one_shot, token_by_token):
+        pos, acc = cache.export(0)
+        assert pos.tolist() == list(range(n + steps))
+        np.testing.assert_allclose(acc, ref_p.sum(axis=0), rtol=1e-12, atol=1e-300)
+
+
+@pytest.mark.parametrize("name,kind,a,b", MASKS)
+@pytest.mark.parametrize("k,r", [(3, 4), (2, 6), (5, 3)])
+def test_masked_policy_matches_the_literal_simulation(oracle, masked, name, kind, a, b, k, r):
+    """Evictions under a pattern: the literal argmax over explicit column sums of the masked probability matrix."""
+    T, d, scale = 22, 4, 0.6
+    rng = np.random.default_rng(500 + 7 * k + r + a)
+    q, kk, v = _rand_qkv(rng, T, d)
+    pat = _pattern(name, a, b)
+    lit = LiteralH2O(k, r, scale, lambda z: z, attend=lambda p, t, r_: p == t or p <= t - r_ or bool(pat(p, t)))
+    masked(kind, a, b)
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    decided = 0
+    for t in range(T):
+        out_l, ev_l, probs, gap = lit.step(q[t], kk[t], v[t])
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        np.testing.assert_allclose(np.sort(res["p"][0, :len(probs)]), np.sort(probs), rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(res["out"][0], out_l, rtol=1e-11, atol=1e-13)
+        if gap > 1e-9:
+            assert res["evicted"][0] == ev_l
+            decided += 1
+        else:  # follow the simulation through an accidental near-tie so that later steps stay comparable
+            cache = None
+            break
+        pos, acc = cache.export(0)
+        assert set(pos.tolist()) == set(lit.S)
+        np.testing.assert_allclose(acc, [lit.column_sum(j) for j in pos], rtol=1e-12, atol=1e-300)
+    assert decided >= 8
