@@ -283,6 +283,27 @@ int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path);
  *   Errors: H2O_ERR_INVALID_ARG (null pointer, hkind outside 0..2), H2O_ERR_CUDA.
  */
 int h2o_cache_set_score_mode(h2o_cache_t* cache, int32_t mode);
+/*
+ * Heavy hitters combined with a sparse attention pattern (Section 5.1, the table that lists the strided and
+ * the fixed Sparse Transformer patterns with and without H2; the paper gives the results, not the rule).  This
+ * library's reading: the cache keeps what it keeps without a pattern — k_s heavy hitters by accumulated score
+ * and the r_s most recent positions — and the pattern decides which entries of the RECENT region a query
+ * attends.  For the query at position t and a key at position p:
+ *     p == t         attended (the token itself);
+ *     p <= t - r_s   attended (a heavy hitter, or the entry that has just left the window);
+ *     t - r_s < p < t attended iff the pattern allows it:
+ *       kind 1, strided(a = stride, b = local window): t - p < b or (t - p) mod a == 0;
+ *       kind 2, fixed(a = block length, b = summary columns, b <= a): floor(p / a) == floor(t / a) or
+ *                                                                    p mod a >= a - b.
+ *   An entry that is not attended is absent from the softmax of that step and its score does not grow.  The
+ *   prompt rows of h2o_prefill_select follow the same rule.  "Without H2" is k_s = 0; kind 0 switches the
+ *   pattern off.
+ * Only on an empty cache (H2O_ERR_STATE otherwise); the pattern survives h2o_cache_reset.  With a pattern,
+ * h2o_prefill_select uses the fp32-FMA kernels and h2o_decode_chunk one decode-step kernel per token.
+ * Errors: H2O_ERR_INVALID_ARG (kind outside 0..2, a < 1, b < 0, b > a for kind 2), H2O_ERR_UNSUPPORTED
+ * (4-bit slots).
+ */
+int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b);
 int h2o_cache_fscore(h2o_cache_t* cache, int32_t hkind, double* out_dev, void* stream);
 /*
  * Process-wide diagnostic switch (no counterpart in the paper).  A decode kernel launched right

@@ -96,6 +96,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_set_chunk_path.restype = c.c_int
     lib.h2o_cache_set_score_mode.argtypes = [vp, c.c_int32]
     lib.h2o_cache_set_score_mode.restype = c.c_int
+    lib.h2o_cache_set_mask.argtypes = [vp, c.c_int32, c.c_int32, c.c_int32]
+    lib.h2o_cache_set_mask.restype = c.c_int
     lib.h2o_cache_fscore.argtypes = [vp, c.c_int32, vp, vp]
     lib.h2o_cache_fscore.restype = c.c_int
     lib.h2o_cache_reset.argtypes = [vp, vp]
@@ -236,6 +238,10 @@ class H2OCache:
     def set_score_mode(self, mode: int):
         """0: rank by the accumulated score, 1: by the averaged score (empty cache only)."""
         _check(lib.h2o_cache_set_score_mode(self._h, int(mode)), "h2o_cache_set_score_mode")
+
+    def set_mask(self, kind: int, a: int = 1, b: int = 0):
+        """h2o_cache_set_mask: 0 none, 1 strided(stride a, local window b), 2 fixed(block a, b summary columns)."""
+        _check(lib.h2o_cache_set_mask(self._h, int(kind), int(a), int(b)), "h2o_cache_set_mask")
 
     def fscore(self, hkind: int = 0, stream=None):
         """F_score per (sequence, head): sum of h(accumulated score); h: 0 identity, 1 sqrt(z+1), 2 log(z+1)."""

@@ -57,10 +57,13 @@ struct Attend {
   // On return p[0 .. cnt + has_self) holds the softmax probabilities (the query's own
   // token last), m / l the row maximum and the sum of exp(s - m), and the threads with
   // threadIdx.x < LPR hold, in o[], chunk threadIdx.x of the output row.
+  // Row x holds the key of position x; with a sparse pattern (mask_kind != 0) the query, at position t_query
+  // with recent window r_win, leaves out the rows key_attended() rejects (probability 0).
   __device__ static void run(const T* __restrict__ q, const T* __restrict__ Kb, const T* __restrict__ Vb,
                              int64_t row_stride, int cnt, const T* __restrict__ k_self,
                              const T* __restrict__ v_self, float c, float* __restrict__ p, Smem& sm,
-                             float (&o)[VEC], float& m_out, float& l_out) {
+                             float (&o)[VEC], float& m_out, float& l_out, int mask_kind = 0, int mask_a = 1,
+                             int mask_b = 0, int t_query = 0, int r_win = 0) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane / LPR, ch = lane % LPR;
     const bool has_self = k_self != nullptr;
@@ -90,7 +93,8 @@ struct Attend {
         for (int v = 0; v < VEC; ++v) part = fmaf(qf[v], kf[u][v], part);
 #pragma unroll
         for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
-        if (ch == 0 && row < cnt) p[row] = c * part;
+        if (ch == 0 && row < cnt)
+          p[row] = key_attended(mask_kind, mask_a, mask_b, row, t_query, r_win) ? c * part : -INFINITY;
       }
     }
     if (has_self && warp == 0) {

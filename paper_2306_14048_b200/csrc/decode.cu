@@ -315,6 +315,9 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
       s_self = c.scale * __shfl_sync(0xffffffffu, part, 0);
     }
+    // a sparse pattern needs the slots' positions during the stream (they are staged with the scores)
+    const int mask_kind = c.mask_kind;
+    if (mask_kind != 0 && nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
     for (int j = 0; j < ntile; ++j) {
       const int s = j % stages;
       if (!mbar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
@@ -343,6 +346,8 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
 #pragma unroll
         for (int off = LPR / 2; off > 0; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
         sc[ps] = row < rows ? c.scale * part : -INFINITY;
+        if (mask_kind != 0 && row < rows && !key_attended(mask_kind, c.mask_a, c.mask_b, pos_s[j * TILE_ROWS + row], t, r))
+          sc[ps] = -INFINITY;  // left out by the pattern: probability 0, no score from this step
         if (ch == 0 && row < rows) p[j * TILE_ROWS + row] = sc[ps];  // raw score, finalised after the stream
       }
       float mnew = mg;

@@ -31,7 +31,7 @@ size_t slot_row_bytes(const h2o_config_t* cfg) {
 }
 
 struct Layout {
-  size_t K, V, acc, pos, count, tpos, status, meta, total;
+  size_t K, V, acc, pos, count, tpos, status, meta, seq_rwin, total;
   int64_t total_slots;
   int max_B;
 };
@@ -79,6 +79,7 @@ Layout make_layout(const h2o_config_t* cfg) {
   L.tpos = take(units * sizeof(int32_t));
   L.status = take(sizeof(int32_t));
   L.meta = take(units * sizeof(h2o::UnitMeta));
+  L.seq_rwin = take((size_t)cfg->batch * sizeof(int32_t));
   L.total = off;
   L.total_slots = slots;
   L.max_B = max_B;
@@ -303,6 +304,10 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   }
   v.score_mode = 0;
   v.kv4 = cfg->dtype == H2O_BF16_KV4 ? 1 : 0;
+  v.mask_kind = 0;
+  v.mask_a = 1;
+  v.mask_b = 0;
+  v.seq_rwin = reinterpret_cast<const int32_t*>(ws + L.seq_rwin);
   c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
@@ -319,6 +324,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
     ok = ok && cudaMemset(ws + L.acc, 0, L.meta - L.acc) == cudaSuccess;  // acc, pos, count, tpos, status
     ok = ok && cudaMemset(ws + L.pos, 0xff, (size_t)L.total_slots * sizeof(int32_t)) == cudaSuccess;  // pos = -1
     ok = ok && cudaMemcpy(ws + L.meta, meta.data(), units * sizeof(h2o::UnitMeta), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(ws + L.seq_rwin, c->recent.data(), (size_t)cfg->batch * sizeof(int32_t), cudaMemcpyHostToDevice) == cudaSuccess;
     // The memsets are asynchronous and a pageable copy returns once the data is staged, all on the legacy default
     // stream, which a non-blocking stream is not ordered behind: wait here, so that the tables are on the device
     // whatever stream the caller uses next.
@@ -403,7 +409,8 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   }
   // bf16 / head_dim 128 runs on the tensor cores; every other combination on the fp32 FMA pipe
   const int in_dtype = input_dtype(cfg.dtype);
-  const bool tc = cache->prefill_path != 1 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
+  // (a sparse pattern is applied by the fp32-FMA kernels only)
+  const bool tc = cache->prefill_path != 1 && cache->view.mask_kind == 0 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
   cudaError_t e = cudaSuccess;
   // optional phase events of this one call (diagnostic): before the forward kernel, after it, after the column
   // sums, after selection and gather
@@ -480,7 +487,7 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   g_last_writer.note_and_check(st, cache->view.K);
   cudaError_t e = cudaSuccess;
   // (the chunk kernel ranks by the accumulated score only)
-  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && cache->view.mask_kind == 0 && !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
@@ -514,6 +521,17 @@ int h2o_cache_set_score_mode(h2o_cache_t* cache, int32_t mode) {
   if (!cache || (mode != 0 && mode != 1)) return H2O_ERR_INVALID_ARG;
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one ranking rule per generation
   cache->view.score_mode = mode;
+  return H2O_OK;
+}
+
+int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b) {
+  if (!cache || kind < 0 || kind > 2) return H2O_ERR_INVALID_ARG;
+  if (kind != 0 && (a < 1 || b < 0 || (kind == 2 && b > a))) return H2O_ERR_INVALID_ARG;
+  if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one attention rule per generation
+  if (kind != 0 && cache->view.kv4) return H2O_ERR_UNSUPPORTED;
+  cache->view.mask_kind = kind;
+  cache->view.mask_a = kind ? a : 1;
+  cache->view.mask_b = kind ? b : 0;
   return H2O_OK;
 }
 

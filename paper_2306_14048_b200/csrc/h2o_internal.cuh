@@ -43,7 +43,21 @@ struct CacheView {
   // accumulated ones in both modes.
   int32_t score_mode;
   int32_t kv4;  // 1: K/V slots are 80-byte 4-bit rows (written by the kernels of decode_kv4.cu)
+  // Sparse pattern inside the recent window (heavy hitters combined with the strided / fixed Sparse Transformer
+  // patterns, Section 5.1): 0 none, 1 strided(stride mask_a, local window mask_b), 2 fixed(block mask_a, mask_b
+  // summary columns).  See key_attended().
+  int32_t mask_kind, mask_a, mask_b;
+  const int32_t* seq_rwin;  // [batch] recent window of every sequence (the prompt kernels index by unit, not by launch position)
 };
+
+// Does the query at position t attend the key at position p (r = the unit's recent window)?  The token itself and
+// everything older than the window (heavy hitters, and the entry that has just left the window) always; of the
+// window what the pattern allows.
+__device__ __forceinline__ bool key_attended(int kind, int a, int b, int p, int t, int r) {
+  if (kind == 0 || p == t || p <= t - r) return true;
+  if (kind == 1) return (t - p) < b || (t - p) % a == 0;
+  return p / a == t / a || p % a >= a - b;
+}
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
 // index = h * total_tokens + token.

@@ -32,7 +32,9 @@ prefill_rows_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, cons
   const int64_t stride = (int64_t)c.n_heads * D;
   const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
   float o[VEC], m, l;
-  A::run(q + base + i * stride, k + base, v + base, stride, i + 1, nullptr, nullptr, c.scale, p, sm, o, m, l);
+  const int r = c.mask_kind ? c.seq_rwin[seq] : 0;
+  A::run(q + base + i * stride, k + base, v + base, stride, i + 1, nullptr, nullptr, c.scale, p, sm, o, m, l, c.mask_kind,
+         c.mask_a, c.mask_b, i, r);
   if (threadIdx.x < LPR) Vec16<T>::store(out + base + i * stride + threadIdx.x * VEC, o);
   if (threadIdx.x == 0) {
     s.rowmax[(int64_t)h * s.total_tokens + lo + i] = m;
@@ -68,6 +70,7 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
 #pragma unroll
     for (int x = 0; x < D; ++x) kf[x] = 0.f;
   }
+  const int r = c.mask_kind ? c.seq_rwin[seq] : 0;
   double a = 0.0;
   for (int i = j0; i < n; ++i) {  // every thread of the block reads the same query row (broadcast)
     const T* qi = q + base + i * stride;
@@ -79,7 +82,8 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
 #pragma unroll
       for (int e = 0; e < VEC; ++e) dot = fmaf(t[e], kf[x + e], dot);
     }
-    if (i >= j) a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
+    if (i >= j && key_attended(c.mask_kind, c.mask_a, c.mask_b, j, i, r))
+      a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
   }
   if (j < n) s.acc0[(int64_t)h * s.total_tokens + lo + j] = a;
 }

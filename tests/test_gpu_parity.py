@@ -345,3 +345,63 @@ def test_kv4_rejects_what_it_does_not_support(H2OCache):
         H2OCache(1, 1, 64, "bf16_kv4", [4], [4])  # head_dim 128 only
     with pytest.raises(pkg.H2OError):
         H2OCache(1, 1, 128, "bf16_kv4", [8000], [8000])  # more slots than one thread block stages
+
+
+# ---------------------------------------------------------------------------------------------------------
+# heavy hitters combined with a sparse pattern inside the recent window (h2o_cache_set_mask)
+# ---------------------------------------------------------------------------------------------------------
+MASKS = [(1, 8, 3), (1, 5, 1), (2, 16, 2), (2, 7, 3)]  # strided(stride, local window), fixed(block, summary columns)
+
+
+@pytest.mark.parametrize("mask", MASKS)
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_sparse_pattern_ragged(H2OCache, mask, dtype, d):
+    """Prompt rows and decode steps under a pattern: ragged batch, several tiles, one prompt shorter than its budget."""
+    from parity_harness import run_parity
+
+    wl = _wl("mask", 4, 3, d, dtype, [300, 77, 513, 40], 48, [20, 9, 33, 30], [24, 5, 31, 30], seed=177 + d)
+    st = run_parity(wl, H2OCache, export_every=8, mask=mask)
+    print(st)
+
+
+@pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([3, 2], [1, 2]), ([6, 1], [12, 9])])
+def test_sparse_pattern_edge_budgets_token_by_token(H2OCache, heavy, recent):
+    """No heavy hitters (the pattern alone), tiny windows, and the fill phase from an empty cache."""
+    from parity_harness import run_parity
+
+    wl = _wl("maskedge", 2, 2, 64, "f32", [1, 1], 60, heavy, recent, seed=15)
+    for mask in ((1, 4, 2), (2, 5, 1)):
+        st = run_parity(wl, H2OCache, prefill=False, export_every=5, mask=mask)
+        print(st)
+
+
+def test_sparse_pattern_units_split_over_a_cluster_and_chunk_call(H2OCache):
+    """Long budgets (a unit shared by the blocks of a cluster) and the multi-token call, which takes one
+    decode-step kernel per token when a pattern is set."""
+    from parity_harness import run_parity
+
+    wl = _wl("maskcluster", 2, 2, 128, "bf16", [1500, 1300], 40, [150, 30], [150, 40], seed=131)
+    st = run_parity(wl, H2OCache, export_every=8, mask=(1, 16, 4))
+    print(st)
+    wl = _wl("maskchunk", 2, 3, 128, "bf16", [400, 300], 40, [20, 30], [24, 16], seed=132)
+    st = run_parity(wl, H2OCache, export_every=8, mask=(2, 12, 2), chunk=16)
+    print(st)
+
+
+def test_sparse_pattern_argument_and_state_errors(H2OCache):
+    import paper_2306_14048_b200 as pkg
+
+    cache = H2OCache(1, 2, 64, "f32", [4], [4])
+    for bad in ((3, 1, 0), (-1, 1, 0), (1, 0, 1), (1, 4, -1), (2, 4, 5)):
+        assert pkg.lib.h2o_cache_set_mask(cache._h, *bad) == pkg.H2O_ERR_INVALID_ARG
+    assert pkg.lib.h2o_cache_set_mask(None, 0, 1, 0) == pkg.H2O_ERR_INVALID_ARG
+    cache.set_mask(1, 4, 2)
+    x = torch.zeros(1, 2, 64, device="cuda")
+    cache.decode_step(x, x, x, torch.empty_like(x))
+    assert pkg.lib.h2o_cache_set_mask(cache._h, 0, 1, 0) == pkg.H2O_ERR_STATE  # one rule per generation
+    cache.reset()
+    cache.set_mask(0)
+    cache.close()
+    kv4 = H2OCache(1, 2, 128, "bf16_kv4", [4], [4])
+    assert pkg.lib.h2o_cache_set_mask(kv4._h, 1, 4, 2) == pkg.H2O_ERR_UNSUPPORTED
+    kv4.close()
