@@ -117,17 +117,19 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                : "memory");
 }
 
-// Optional phase timers (compile with -DH2O_PHASE_TIMERS): thread 0 of every block records
-// %globaltimer at a few points; h2o_debug_phase_timers copies them out.  Off in normal builds.
+// Optional phase timers (compile with -DH2O_PHASE_TIMERS): thread 0 of every block records %globaltimer (ns,
+// common to all SMs) at a few points, for the last eight launches (the host numbers the launches in the upper bits
+// of launch_flags), and its SM in entry 0; h2o_debug_phase_timers copies them out.  Off in normal builds.
 #ifdef H2O_PHASE_TIMERS
-__device__ unsigned long long g_phase[8192 * 16];
-#define H2O_STAMP(i)                                                                   \
-  do {                                                                                 \
-    if (threadIdx.x == 0 && blockIdx.x < 8192) {                                       \
-      unsigned long long ts_;                                                          \
-      asm volatile("mov.u64 %0, %%clock64;" : "=l"(ts_));                             \
-      g_phase[blockIdx.x * 16 + (i)] = ts_;                                             \
-    }                                                                                  \
+constexpr int kPhaseBlocks = 4096, kPhaseLaunches = 8;
+__device__ unsigned long long g_phase[kPhaseLaunches * kPhaseBlocks * 16];
+#define H2O_STAMP(i)                                                                                        \
+  do {                                                                                                      \
+    if (threadIdx.x == 0 && blockIdx.x < kPhaseBlocks) {                                                    \
+      unsigned long long ts_;                                                                               \
+      asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ts_));                                             \
+      g_phase[((((unsigned)launch_flags >> 8) % kPhaseLaunches) * kPhaseBlocks + blockIdx.x) * 16 + (i)] = ts_; \
+    }                                                                                                       \
   } while (0)
 #else
 #define H2O_STAMP(i) do { } while (0)
@@ -188,6 +190,13 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   float* x_out = p + chunk + 4;  // [kMaxSplit][D], only when split > 1 (behind the 16 spare bytes of p)
 
   H2O_STAMP(1);
+#ifdef H2O_PHASE_TIMERS
+  if (threadIdx.x == 0 && blockIdx.x < kPhaseBlocks) {
+    unsigned smid_;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid_));
+    g_phase[((((unsigned)launch_flags >> 8) % kPhaseLaunches) * kPhaseBlocks + blockIdx.x) * 16 + 0] = smid_;
+  }
+#endif
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, ch = lane % LPR;
   cg::cluster_group cluster = cg::this_cluster();
@@ -271,10 +280,12 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   const int t = c.tpos[su];
   const int nloc = max(0, min(min(cnt - lo, chunk), nstr));  // occupied slots of this block
   __syncthreads();  // barriers are initialised before any consumer polls them
+  H2O_STAMP(12);
   if (cache_is_quiescent) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
+  H2O_STAMP(13);
 
   // the new token's own key/value: loaded now, used after the stream
   float qf[VEC], ksf[VEC], vself = 0.f;
@@ -595,7 +606,11 @@ cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, i
                           const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                           cudaStream_t stream) {
   if (split < 1 || split > kMaxSplit) return cudaErrorInvalidValue;
-  const int quiescent = (quiescent_b ? 1 : 0) | (all_full ? 2 : 0);  // launch flags
+  int quiescent = (quiescent_b ? 1 : 0) | (all_full ? 2 : 0);  // launch flags
+#ifdef H2O_PHASE_TIMERS
+  static int launch_no = 0;
+  quiescent |= (launch_no++ & 0xffff) << 8;
+#endif
   if (dtype == H2O_F32) {
     if (c.head_dim == 64)
       return launch<float, 64>(c, split, chunk, stages, quiescent, q, k_new, v_new, out, evicted_pos, stream);

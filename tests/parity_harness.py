@@ -91,7 +91,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
                device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
                pattern: Optional[Sequence[int]] = None, score_mode: int = 0, static_scratch: bool = False,
-               mask: Optional[Sequence[int]] = None) -> ParityStats:
+               mask: Optional[Sequence[int]] = None, split: int = 0) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
@@ -99,6 +99,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     interact.  With ``chunk`` > 0 the CUDA path advances ``chunk`` tokens per call (h2o_decode_chunk)
     while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
     sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
+    ``split``: thread blocks (one cluster) per unit in the decode kernel, 0 = the library's choice.
     ``mask`` = (kind, a, b): sparse pattern inside the recent window (h2o_cache_set_mask) on both sides.
     ``scale`` > 0 replaces the default softmax scale 1/sqrt(d) (4/sqrt(d) is the peaky-softmax stress run).
     """
@@ -108,14 +109,15 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         h2o_oracle.set_mask(*mask)
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
-                              chunk, chunk_path, pattern, score_mode, static_scratch, mask=(0,) + tuple(mask))
+                              chunk, chunk_path, pattern, score_mode, static_scratch, mask=(0,) + tuple(mask), split=split)
         finally:
             h2o_oracle.set_mask(0)
     if score_mode > 0:  # the oracle's ranking rule is process-wide: always put it back
         h2o_oracle.set_score_mode(score_mode)
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
-                              chunk, chunk_path, pattern, score_mode=0 - score_mode, static_scratch=static_scratch, mask=mask)
+                              chunk, chunk_path, pattern, score_mode=0 - score_mode, static_scratch=static_scratch, mask=mask,
+                              split=split)
         finally:
             h2o_oracle.set_score_mode(0)
     score_mode = -score_mode  # (negative: the oracle is already in that mode)
@@ -128,6 +130,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     scale = float(np.float32(scale if scale > 0 else 1.0 / np.sqrt(float(d))))
     gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
     gpu.set_prefill_path(prefill_path)
+    gpu.set_decode_shape(split, 0)
     gpu.set_score_mode(score_mode)
     if mask is not None:  # (0, kind, a, b): the oracle already has it
         gpu.set_mask(*mask[1:])
