@@ -424,6 +424,11 @@ constexpr int kFwRegsIssue = 80, kFwRegsSoftmax = 168;
 constexpr int kFwKeys = 64;                       // keys per tile
 constexpr int kFwKvSlotBytes = 2 * kFwKeys * 128;   // [2 boxes][64 rows][128 B] = 16 KB
 constexpr int kFwMaxKvSlots = 6;
+// The low halves matter only where a probability is large: a tile whose probabilities all stay below
+// kFwLoThreshold of their row's running sum (an upper bound of the final probability) contributes at most
+// 2^-9 of them to the output, far inside its tolerance, and its second product is skipped.  The softmax warps
+// vote per tile; the decision depends on the data alone, so results stay the same from run to run.
+constexpr float kFwLoThreshold = 1.0f / 32.0f;
 constexpr bool kFwSplitP = true;                 // P as bf16 hi + bf16 lo (two P V products): one bf16 alone (2^-9 per
                                                  // probability) misses the output tolerance on peaky rows
 // Up to this prompt length the persistent one-query-block kernel runs the forward pass (measured: 512-token
@@ -451,6 +456,8 @@ struct FwShared {
                           // does not wait on every phase of pv_done, so a parity wait for the last one could alias)
   uint32_t tmem_base;
   int abort_flag;
+  uint32_t lo_need[2][2][4];  // [group][buffer][softmax warp]: some probability of the tile is large (kFwLoThreshold);
+                              // written before the warp's arrival on p_full, read by the issuing warp after its wait
 };
 
 // G = query blocks (softmax groups) per thread block.  Two share every K/V tile and fill an SM (all of
@@ -610,13 +617,18 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       tc_fence_after();
       FWD_TL(g, j, 2);
       const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+      const volatile uint32_t* ln = sh.lo_need[g][par];  // (tile j uses buffer j % 2 == par)
+      const bool need_lo = kFwSplitP && (ln[0] | ln[1] | ln[2] | ln[3]) != 0u;
       if (elect_one()) {
         if (j == 0) mma_ts_lohi<false>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
         else mma_ts_lohi<true>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
 #pragma unroll
-        for (int ks = 1; ks < (kFwSplitP ? 2 : 1) * (kFwKeys / 16); ++ks) {  // hi columns (, then lo columns)
-          const uint32_t kk = (uint32_t)(ks & 3);
-          mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
+        for (int ks = 1; ks < kFwKeys / 16; ++ks)  // hi columns
+          mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + (((uint32_t)ks * 2048u) >> 4), desc_hi(dv), idesc_o);
+        if (need_lo) {
+#pragma unroll
+          for (int ks = 0; ks < kFwKeys / 16; ++ks)  // lo columns, same V rows
+            mma_ts_lohi<true>(d_o, sp + 32u + (uint32_t)ks * 8u, desc_lo(dv) + (((uint32_t)ks * 2048u) >> 4), desc_hi(dv), idesc_o);
         }
         FWD_TL(g, j, 8);
         mma_commit(&sh.pv_done[g][par]);
@@ -719,6 +731,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       // (columns 32..63): column c holds keys 2c and 2c+1
       uint32_t hw[32];
       [[maybe_unused]] uint32_t lw[32];
+      float p_max = 0.f;
 #pragma unroll
       for (int c = 0; c < 32; ++c) {
         const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
@@ -726,6 +739,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         const float2 x = __ffma2_rn(make_float2(s0, s1), make_float2(scale2, scale2), make_float2(neg_m, neg_m));
         const float2 pp = make_float2(ex2(x.x), ex2(x.y));
         l2 = __fadd2_rn(l2, pp);
+        p_max = max3(p_max, pp.x, pp.y);
         const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pp.x, pp.y);
         hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
         if constexpr (kFwSplitP) {
@@ -739,8 +753,11 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
       FWD_CLK(c4_);
       FWD_TL(g, j, 3);
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.p_full[g][j & 1]);
+      const bool lo_vote = __any_sync(0xffffffffu, p_max > kFwLoThreshold * (l2.x + l2.y));
+      if (lane == 0) {
+        sh.lo_need[g][j & 1][quarter] = lo_vote ? 1u : 0u;
+        mbar_arrive(&sh.p_full[g][j & 1]);
+      }
       FWD_ADD(0, c0_, c1_);
       FWD_ADD(1, c1_, c2_);
       FWD_ADD(2, c2_, c3_);
@@ -804,6 +821,7 @@ struct FsShared {
   uint64_t o_final;          // both issuing warps' last products of the item are complete
   uint32_t tmem_base;
   int abort_flag;
+  uint32_t lo_need[2][4];    // [buffer][softmax warp], as in FwShared
   // The producer thread alone looks items up (two dependent loads and divisions per item); it leaves each
   // item's description here before it loads the item's Q.  The S walkers wait for q_full of every item
   // in order and read entry ic % 8 then; the same threads' P V walkers come later; the softmax warps read
@@ -1037,14 +1055,19 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         tc_fence_after();
         FWD_TL(0, T, 2);
         const uint64_t dv = smem_desc_sw128(smem_u32(kv_ring + slot * kFwKvSlotBytes), kFwKvSlotBytes / 2, 1024);
+        const volatile uint32_t* ln = sh.lo_need[par];  // (tile T uses buffer T % 2 == par)
+        const bool need_lo = kFwSplitP && (ln[0] | ln[1] | ln[2] | ln[3]) != 0u;
         if (elect_one()) {
           // (P(0) of an item is stored only after the softmax warps have read the previous item's O)
           if (j == 0) mma_ts_lohi<false>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
           else mma_ts_lohi<true>(d_o, sp, desc_lo(dv), desc_hi(dv), idesc_o);
 #pragma unroll
-          for (int ks = 1; ks < (kFwSplitP ? 2 : 1) * (kFwKeys / 16); ++ks) {  // hi columns (, then lo columns)
-            const uint32_t kk = (uint32_t)(ks & 3);
-            mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + ((kk * 2048u) >> 4), desc_hi(dv), idesc_o);
+          for (int ks = 1; ks < kFwKeys / 16; ++ks)  // hi columns
+            mma_ts_lohi<true>(d_o, sp + (uint32_t)ks * 8u, desc_lo(dv) + (((uint32_t)ks * 2048u) >> 4), desc_hi(dv), idesc_o);
+          if (need_lo) {
+#pragma unroll
+            for (int ks = 0; ks < kFwKeys / 16; ++ks)  // lo columns, same V rows
+              mma_ts_lohi<true>(d_o, sp + 32u + (uint32_t)ks * 8u, desc_lo(dv) + (((uint32_t)ks * 2048u) >> 4), desc_hi(dv), idesc_o);
           }
           mma_commit(&sh.pv_done[par]);
           if (j + 2 >= kp_.nt) mma_commit(&sh.o_final);  // this warp's last product of the item
@@ -1180,6 +1203,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const float neg_m = -m_used;
       uint32_t hw[32];
       [[maybe_unused]] uint32_t lw[32];
+      float p_max = 0.f;
 #pragma unroll
       for (int c = 0; c < 32; ++c) {
         const float s0 = __uint_as_float(c < 16 ? r0[2 * c] : r1[2 * c - 32]);
@@ -1187,6 +1211,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const float2 x = __ffma2_rn(make_float2(s0, s1), make_float2(scale2, scale2), make_float2(neg_m, neg_m));
         const float2 pp = make_float2(ex2(x.x), ex2(x.y));
         l2 = __fadd2_rn(l2, pp);
+        p_max = max3(p_max, pp.x, pp.y);
         const __nv_bfloat162 hi2 = __floats2bfloat162_rn(pp.x, pp.y);
         hw[c] = *reinterpret_cast<const uint32_t*>(&hi2);
         if constexpr (kFwSplitP) {
@@ -1198,8 +1223,11 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       if constexpr (kFwSplitP) tmem_st32(buf + 32u, lw);
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.p_full[T & 1]);
+      const bool lo_vote = __any_sync(0xffffffffu, p_max > kFwLoThreshold * (l2.x + l2.y));
+      if (lane == 0) {
+        sh.lo_need[T & 1][quarter] = lo_vote ? 1u : 0u;
+        mbar_arrive(&sh.p_full[T & 1]);
+      }
       FWD_TL(0, T, 3);
       }
       if (ok) {  // the item's output
