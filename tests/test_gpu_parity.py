@@ -30,9 +30,11 @@ def _wl(name, batch, heads, d, dtype, lens, steps, heavy, recent, seed=1234):
 def test_config1_tiny_fp32_full(H2OCache):
     from parity_harness import run_parity
 
+    from parity_harness import record
+
     st = run_parity(CONFIGS["c1_tiny"], H2OCache, export_every=8)
     assert st.decisions == 4 + 4 * 64
-    print(st)
+    record(st, "c1 full")
 
 
 @pytest.mark.parametrize("dtype,d", [("bf16", 128), ("bf16", 64), ("f32", 128), ("f32", 64)])
