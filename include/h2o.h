@@ -331,6 +331,13 @@ int h2o_prefill_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens, si
  * can be a little slower than an untimed one.
  */
 int h2o_debug_set_prefill_events(h2o_cache_t* cache, void* const* events);
+/*
+ * Diagnostic (no counterpart in the paper): 1 if this library was built with -DH2O_BOUNDS — every slot, unit and
+ * prompt-row index of the kernels checked before use, a violation recorded as H2O_ERR_STATE in the status word
+ * and the access skipped (the build the parity tests are also run against, in place of a memory checker) —
+ * 0 for the normal build.
+ */
+int h2o_debug_bounds_checked(void);
 const char* h2o_strerror(int code);
 
 #ifdef __cplusplus

@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libh2o_b200.so")
+# H2O_B200_LIB names another build of the same library (the checked variant libh2o_b200_bounds.so of build.py)
+LIB_PATH = os.environ.get("H2O_B200_LIB") or os.path.join(_PKG, "libh2o_b200.so")
 
 H2O_OK = 0
 H2O_ERR_INVALID_ARG = -1
@@ -123,6 +124,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_debug_set_early_prefetch.argtypes = [c.c_int32]
     lib.h2o_debug_set_prefill_events.restype = c.c_int
     lib.h2o_debug_set_prefill_events.argtypes = [vp, c.POINTER(vp)]
+    lib.h2o_debug_bounds_checked.restype = c.c_int
+    lib.h2o_debug_bounds_checked.argtypes = []
     lib.h2o_strerror.restype = c.c_char_p
     lib.h2o_strerror.argtypes = [c.c_int]
     return lib

@@ -240,7 +240,11 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   // never used — so a stale flag (say, in a replayed CUDA graph) costs bandwidth, not correctness.
   int cnt = 0;
   if (!all_full) cnt = c.count[su];
-  const int nstr = all_full ? max(0, min(B - lo, chunk)) : max(0, min(cnt - lo, chunk));
+  int nstr = all_full ? max(0, min(B - lo, chunk)) : max(0, min(cnt - lo, chunk));
+  // (checked build: the unit and the whole range of rows this block streams must lie inside the cache)
+  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) ||
+      (nstr > 0 && !H2O_IN_RANGE(mt.slot_off + lo + ((nstr + 3) & ~3) - 1, c.total_slots, c.status)))
+    nstr = 0;
   const int ntile = (nstr + TILE_ROWS - 1) / TILE_ROWS;   // stages to stream (one K tile + one V tile each)
   T* Kb = reinterpret_cast<T*>(c.K) + (mt.slot_off + lo) * D;
   T* Vb = reinterpret_cast<T*>(c.V) + (mt.slot_off + lo) * D;
@@ -277,6 +281,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
   }
   if (all_full) cnt = c.count[su];
+  if (!H2O_IN_RANGE(cnt, B + 1, c.status)) cnt = 0;  // (checked build) a unit never holds more than its budget
   const int t = c.tpos[su];
   const int nloc = max(0, min(min(cnt - lo, chunk), nstr));  // occupied slots of this block
   __syncthreads();  // barriers are initialised before any consumer polls them
@@ -460,7 +465,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     for (int x = tid; x < nloc; x += kThreads) {
       const float px = expf(p[x] - m) * inv_l;
       const double a = acc_s[x] + (double)px;
-      acc_g[x] = a;
+      if (H2O_IN_RANGE(mt.slot_off + lo + x, c.total_slots, c.status)) acc_g[x] = a;
       const int ps = pos_s[x];
       if (full && ps <= t - r) {
         // averaged variant: the key has been attended by the queries at positions ps .. t
@@ -515,6 +520,8 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
           ev = -1;
           if (lane == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
         }
+        if (slot >= 0 && (!H2O_IN_RANGE(slot, B, c.status) || !H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status)))
+          slot = -1;  // (checked build) never write outside the unit's slots
         if (lane == 0) {
           if (!full) c.count[su] = cnt + 1;
           if (slot >= 0) {

@@ -606,7 +606,8 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // ---- write the state back: scores of the survivors, the chunk's surviving rows into their slots ----
 #pragma unroll
     for (int m = 0; m < KT; ++m) {
-      if (alive[m]) {
+      if (alive[m] && H2O_IN_RANGE(slot[m], mt.kbud + mt.rwin, c.status) &&
+          H2O_IN_RANGE(mt.slot_off + slot[m], c.total_slots, c.status)) {
         c.acc[mt.slot_off + slot[m]] = acc[m];
         if (jx[m] >= 0) c.pos[mt.slot_off + slot[m]] = pos[m];
       }
@@ -616,7 +617,7 @@ decode_chunk_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     for (int idx = tid; idx < ceff * 32; idx += kKeyThreads) {
       const int j = idx >> 5, pc = idx & 31, c16 = pc & 15;
       const int sl = sh.wb_slot[j];
-      if (sl >= 0) {
+      if (sl >= 0 && H2O_IN_RANGE(sl, mt.kbud + mt.rwin, c.status) && H2O_IN_RANGE(mt.slot_off + sl, c.total_slots, c.status)) {
         const __nv_bfloat16* src = (pc < 16 ? k_u : v_u) + (int64_t)j * in_stride + c16 * 8;
         __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(pc < 16 ? c.K : c.V) + (mt.slot_off + sl) * kD + c16 * 8;
         *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);

@@ -180,7 +180,11 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
-  const int cnt = c.count[su];
+  int cnt = c.count[su];
+  // (checked build: the unit and the rows this block streams must lie inside the cache)
+  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) || !H2O_IN_RANGE(cnt, B + 1, c.status) ||
+      !H2O_IN_RANGE(mt.slot_off + (cnt > 0 ? cnt - 1 : 0), c.total_slots, c.status))
+    cnt = 0;
   const int t = c.tpos[su];
   const int ntile = (cnt + kTileRows - 1) / kTileRows;
   unsigned char* Kb = static_cast<unsigned char*>(c.K) + mt.slot_off * kRowBytes;
@@ -462,7 +466,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     for (int x = tid; x < cnt; x += kThreads) {
       const float px = expf(p[x] - m) * inv_l;
       const double a = acc_s[x] + (double)px;
-      acc_g[x] = a;
+      if (H2O_IN_RANGE(mt.slot_off + x, c.total_slots, c.status)) acc_g[x] = a;
       const int ps = pos_s[x];
       if (full && ps <= t - r) {
         const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
@@ -495,6 +499,8 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
         ev = -1;
         if (lane == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
       }
+      if (slot >= 0 && (!H2O_IN_RANGE(slot, B, c.status) || !H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status)))
+        slot = -1;  // (checked build) never write outside the unit's slots
       if (lane == 0) {
         if (!full) c.count[su] = cnt + 1;
         if (slot >= 0) {
@@ -530,7 +536,9 @@ gather_kv4_kernel(CacheView c, PrefillScratch s, const __nv_bfloat16* __restrict
   unsigned char* Vb = static_cast<unsigned char*>(c.V) + mt.slot_off * kRowBytes;
   for (int x = threadIdx.x; x < m * 8; x += blockDim.x) {
     const int slot = x >> 3, part = x & 7, grp = part & 3;
+    if (!H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status)) continue;
     const int j = c.pos[mt.slot_off + slot];
+    if (!H2O_IN_RANGE(j, s.cu[seq + 1] - lo, c.status)) continue;  // a kept position is a prompt row of this sequence
     const __nv_bfloat16* src = (part < 4 ? k : v) + base + (int64_t)j * stride + 32 * grp;
     uint4 codes;
     uint32_t meta;

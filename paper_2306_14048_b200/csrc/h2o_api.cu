@@ -308,6 +308,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   v.mask_a = 1;
   v.mask_b = 0;
   v.seq_rwin = reinterpret_cast<const int32_t*>(ws + L.seq_rwin);
+  v.total_slots = L.total_slots;
   c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
@@ -756,6 +757,14 @@ int h2o_debug_wait_probe(h2o_cache_t* cache, int32_t polls, void* stream) {
     return H2O_ERR_CUDA;
   }
   return H2O_OK;
+}
+
+int h2o_debug_bounds_checked(void) {
+#ifdef H2O_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 const char* h2o_strerror(int code) {

@@ -48,7 +48,23 @@ struct CacheView {
   // summary columns).  See key_attended().
   int32_t mask_kind, mask_a, mask_b;
   const int32_t* seq_rwin;  // [batch] recent window of every sequence (the prompt kernels index by unit, not by launch position)
+  int64_t total_slots;      // slots of all units together (the limit of every slot index)
 };
+
+// Debug build (-DH2O_BOUNDS, the stand-in for a memory checker): every slot, unit and prompt-row index that
+// addresses the cache, the prompt tensors or the per-unit arrays is checked right before it is used; a violation
+// records H2O_ERR_STATE in the cache's status word and the access is skipped.  In normal builds the checks
+// compile to nothing.
+#ifdef H2O_BOUNDS
+__device__ __forceinline__ bool index_in_range(long long idx, long long limit, int32_t* status) {
+  if (idx >= 0 && idx < limit) return true;
+  atomicCAS(status, 0, H2O_ERR_STATE);
+  return false;
+}
+#define H2O_IN_RANGE(idx, limit, status) ::h2o::index_in_range((long long)(idx), (long long)(limit), (status))
+#else
+#define H2O_IN_RANGE(idx, limit, status) true
+#endif
 
 // Does the query at position t attend the key at position p (r = the unit's recent window)?  The token itself and
 // everything older than the window (heavy hitters, and the entry that has just left the window) always; of the

@@ -29,6 +29,7 @@ prefill_rows_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, cons
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
   const int i = blockIdx.x;
   if (i >= n) return;
+  if (!H2O_IN_RANGE(u, c.units, c.status) || !H2O_IN_RANGE((int64_t)lo + i, s.total_tokens, c.status)) return;
   const int64_t stride = (int64_t)c.n_heads * D;
   const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
   float o[VEC], m, l;
@@ -85,7 +86,7 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
     if (i >= j && key_attended(c.mask_kind, c.mask_a, c.mask_b, j, i, r))
       a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
   }
-  if (j < n) s.acc0[(int64_t)h * s.total_tokens + lo + j] = a;
+  if (j < n && H2O_IN_RANGE((int64_t)lo + j, s.total_tokens, c.status)) s.acc0[(int64_t)h * s.total_tokens + lo + j] = a;
 }
 
 template <typename T, int D>

@@ -154,7 +154,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
       const int keep = (j < n) && (j >= nc || gt || (is_eq && eq_rank >= total_eq - need_eq));
       int tot_keep;
       const int dst = kept_base + block_exclusive_scan(keep, warp_tot, tot_keep);
-      if (keep && dst < B) kept[dst] = j;
+      if (keep && dst < B && H2O_IN_RANGE(dst, m, c.status)) kept[dst] = j;
       kept_base += tot_keep;
       eq_base += tot_eq_chunk;
     }
@@ -170,6 +170,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
   T* Vb = reinterpret_cast<T*>(c.V) + s0 * D;
   for (int x = tid; x < m; x += kSelThreads) {
     const int j = kept[x];
+    if (!H2O_IN_RANGE(j, n, c.status) || !H2O_IN_RANGE(s0 + x, c.total_slots, c.status)) continue;
     c.acc[s0 + x] = acc0[j];
     c.pos[s0 + x] = j;
   }
@@ -177,6 +178,7 @@ select_gather_kernel(CacheView c, PrefillScratch s, const T* __restrict__ k, con
 #pragma unroll 4
   for (int x = tid; x < m * LPR; x += kSelThreads) {
     const int slot = x / LPR, ch = x % LPR;
+    if (!H2O_IN_RANGE(kept[slot], n, c.status) || !H2O_IN_RANGE(s0 + slot, c.total_slots, c.status)) continue;
     const int64_t src = base + (int64_t)kept[slot] * stride + ch * VEC;
     *reinterpret_cast<uint4*>(Kb + (int64_t)slot * D + ch * VEC) = *reinterpret_cast<const uint4*>(k + src);
     *reinterpret_cast<uint4*>(Vb + (int64_t)slot * D + ch * VEC) = *reinterpret_cast<const uint4*>(v + src);
