@@ -660,7 +660,7 @@ def main():
                     help="launch every decode step from the host instead of replaying a CUDA graph of the decode loop")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-all", action="store_true", help="end-to-end figure for the per_config workloads too")
-    ap.add_argument("--e2e-pinned-gb", type=float, default=12.0, help="pinned host memory the end-to-end leg may use for prompts")
+    ap.add_argument("--e2e-pinned-gb", type=float, default=28.0, help="pinned host memory the end-to-end leg may use for prompts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="only the selected configuration")
     ap.add_argument("--context", action="store_true", help="chunk-call context figure for every configuration")

@@ -91,6 +91,32 @@ static int attended(long p, long t, long r) {
 }
 
 /*
+ * "Top-K" attention combined with the heavy hitters (appendix "Enhancing the Top-K baseline": each query keeps
+ * only its largest attention logits; the paper reports it with and without H2 and gives no rule for the
+ * combination).  Reading: in a decode step the query attends, of everything it would otherwise attend (the kept
+ * entries the sparse pattern allows, and itself), only the m entries with the largest scaled logits — equal
+ * logits: the higher position first; the others get probability 0 and no score from that step.  The cache policy
+ * is unchanged.  m = 0 switches it off; the prompt rows of the one-shot prefill stay dense.
+ */
+static long g_topk = 0;
+int h2o_oracle_set_topk(long m) {
+  if (m < 0) return -1;
+  g_topk = m;
+  return 0;
+}
+typedef struct {
+  double s;
+  long pos, idx;
+} logit_t;
+static int logit_cmp(const void* a, const void* b) { /* strongest first: larger logit, then higher position */
+  const logit_t* x = (const logit_t*)a;
+  const logit_t* y = (const logit_t*)b;
+  if (x->s != y->s) return x->s > y->s ? -1 : 1;
+  if (x->pos != y->pos) return x->pos > y->pos ? -1 : 1;
+  return 0;
+}
+
+/*
  * Causal softmax attention of one (sequence, head) and the column sums of its
  * probability matrix.
  *   Q, K, V : n rows of d floats, consecutive rows `stride` floats apart.
@@ -272,12 +298,14 @@ long h2o_oracle_select(const double* acc0, long n, long k, long r, int32_t* kept
  * Outputs: out [units][d]; evicted [units] = oracle's own decision (-1 none);
  *          status [units]; gap [units] = relative gap between the two smallest
  *          candidate scores (inf when fewer than two); p_out optional [units][cap]
- *          = probabilities of the entries in state order, the new token last.
+ *          = probabilities of the entries in state order, the new token last; tgap optional [units] = with
+ *          "Top-K" attention on, the relative gap between the weakest kept and the strongest dropped logit
+ *          (inf when nothing was dropped).
  */
 int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, const int32_t* rwin, int32_t* t,
                            int32_t* cnt, int32_t* pos, double* acc, double* Kc, double* Vc, const float* q,
                            const float* knew, const float* vnew, double c, const int32_t* hint, double tie_rel,
-                           double* out, int32_t* evicted, int32_t* status, double* gap, double* p_out) {
+                           double* out, int32_t* evicted, int32_t* status, double* gap, double* p_out, double* tgap) {
   int bad = 0;
 #pragma omp parallel for schedule(dynamic, 8)
   for (long u = 0; u < units; ++u) {
@@ -304,19 +332,41 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
     m += 1;
     /* scores, softmax, output */
     double* e = (double*)malloc(sizeof(double) * (size_t)m);
-    double mx = -INFINITY;
+    char* att = (char*)malloc((size_t)m);
+    long natt = 0;
     for (long j = 0; j < m; ++j) {
-      if (!attended(up[j], tt, r)) continue; /* left out by the sparse pattern (none by default) */
+      att[j] = (char)attended(up[j], tt, r); /* 0: left out by the sparse pattern (none by default) */
+      if (!att[j]) continue;
       double s = 0.0;
       for (long x = 0; x < d; ++x) s += (double)q[u * d + x] * uk[j * d + x];
       e[j] = c * s;
-      if (e[j] > mx) mx = e[j];
+      natt += 1;
     }
+    if (tgap) tgap[u] = INFINITY;
+    if (g_topk > 0 && natt > g_topk) { /* keep the g_topk strongest logits only */
+      logit_t* lg = (logit_t*)malloc(sizeof(logit_t) * (size_t)natt);
+      long n2 = 0;
+      for (long j = 0; j < m; ++j)
+        if (att[j]) {
+          lg[n2].s = e[j];
+          lg[n2].pos = up[j];
+          lg[n2].idx = j;
+          n2 += 1;
+        }
+      qsort(lg, (size_t)natt, sizeof(logit_t), logit_cmp);
+      for (long x = g_topk; x < natt; ++x) att[lg[x].idx] = 0;
+      if (tgap) tgap[u] = rel_gap(lg[g_topk - 1].s, lg[g_topk].s); /* weakest kept against strongest dropped */
+      free(lg);
+    }
+    double mx = -INFINITY;
+    for (long j = 0; j < m; ++j)
+      if (att[j] && e[j] > mx) mx = e[j];
     double l = 0.0;
     for (long j = 0; j < m; ++j) {
-      e[j] = attended(up[j], tt, r) ? exp(e[j] - mx) : 0.0;
+      e[j] = att[j] ? exp(e[j] - mx) : 0.0;
       l += e[j];
     }
+    free(att);
     double* o = out + u * d;
     for (long x = 0; x < d; ++x) o[x] = 0.0;
     for (long j = 0; j < m; ++j) {

@@ -47,9 +47,11 @@ def _load():
         lib.h2o_oracle_select.argtypes = [dp, c.c_long, c.c_long, c.c_long, ip, dp]
         lib.h2o_oracle_decode_step.restype = c.c_int
         lib.h2o_oracle_decode_step.argtypes = [c.c_long, c.c_long, c.c_long, ip, ip, ip, ip, ip, dp, dp, dp, fp, fp, fp,
-                                               c.c_double, ip, c.c_double, dp, ip, ip, dp, dp]
+                                               c.c_double, ip, c.c_double, dp, ip, ip, dp, dp, dp]
         lib.h2o_oracle_set_score_mode.restype = c.c_int
         lib.h2o_oracle_set_score_mode.argtypes = [c.c_int]
+        lib.h2o_oracle_set_topk.restype = c.c_int
+        lib.h2o_oracle_set_topk.argtypes = [c.c_long]
         lib.h2o_oracle_set_mask.restype = c.c_int
         lib.h2o_oracle_set_mask.argtypes = [c.c_int, c.c_long, c.c_long]
         lib.h2o_oracle_fscore.restype = c.c_double
@@ -111,6 +113,12 @@ def set_mask(kind: int, a: int = 1, b: int = 1) -> None:
     Process-wide, like the score mode: tests that set it put it back to 0."""
     if _load().h2o_oracle_set_mask(int(kind), int(a), int(b)) != 0:
         raise ValueError("bad mask parameters")
+
+
+def set_topk(m: int) -> None:
+    """"Top-K" attention in decode steps: each query attends only its m largest logits (0 = off).  Process-wide."""
+    if _load().h2o_oracle_set_topk(int(m)) != 0:
+        raise ValueError("m must be >= 0")
 
 
 def fscore(acc: np.ndarray, hkind: int = 0) -> float:
@@ -230,16 +238,17 @@ class OracleCache:
         status = np.empty(n, dtype=np.int32)
         gap = np.empty(n, dtype=np.float64)
         p = np.zeros((n, st.cap), dtype=np.float64) if want_p else None
+        tgap = np.empty(n, dtype=np.float64)
         h = None if hint is None else np.ascontiguousarray(hint, dtype=np.int32)
         rc = _load().h2o_oracle_decode_step(
             n, st.d, st.cap, _p(st.kbud, ctypes.c_int32), _p(st.rwin, ctypes.c_int32), _p(st.t, ctypes.c_int32),
             _p(st.cnt, ctypes.c_int32), _p(st.pos, ctypes.c_int32), _p(st.acc, ctypes.c_double), _p(st.K, ctypes.c_double),
             _p(st.V, ctypes.c_double), _p(qf, ctypes.c_float), _p(kf, ctypes.c_float), _p(vf, ctypes.c_float), st.scale,
             _p(h, ctypes.c_int32), float(tie_rel), _p(out, ctypes.c_double), _p(evicted, ctypes.c_int32),
-            _p(status, ctypes.c_int32), _p(gap, ctypes.c_double), _p(p, ctypes.c_double))
+            _p(status, ctypes.c_int32), _p(gap, ctypes.c_double), _p(p, ctypes.c_double), _p(tgap, ctypes.c_double))
         if rc != 0:
             raise RuntimeError("oracle decode step failed: inconsistent state (%d)" % rc)
-        return dict(out=out, evicted=evicted, status=status, gap=gap, p=p)
+        return dict(out=out, evicted=evicted, status=status, gap=gap, p=p, topk_gap=tgap)
 
     def _decode_subset(self, qf, kf, vf, hint, tie_rel, want_p, units):
         """Step only some units: copy their state out, step, copy back (units are independent)."""

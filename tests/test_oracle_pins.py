@@ -105,6 +105,7 @@ class LiteralH2O:
     def __init__(self, k, r, scale, h, attend=None):
         self.k, self.r, self.c, self.h = k, r, scale, h
         self.attend = attend  # optional predicate (key position, query position, r) -> attended?
+        self.topk = 0  # > 0: a query attends only its topk largest logits (equal logits: the higher position)
         self.S = []  # kept positions
         self.rows = []  # rows[i][j] = probability token i gave token j
         self.K, self.V = {}, {}
@@ -122,6 +123,10 @@ class LiteralH2O:
         G = self.S + [t]
         seen = [j for j in G if self.attend is None or self.attend(j, t, self.r)]
         logits = [self.c * math.fsum(float(a) * float(b) for a, b in zip(q, self.K[j])) for j in seen]
+        if self.topk and len(seen) > self.topk:
+            order = sorted(range(len(seen)), key=lambda i: (logits[i], seen[i]), reverse=True)[:self.topk]
+            seen = [seen[i] for i in sorted(order)]
+            logits = [self.c * math.fsum(float(a) * float(b) for a, b in zip(q, self.K[j])) for j in seen]
         mx = max(logits)
         w = [math.exp(x - mx) for x in logits]
         tot = math.fsum(w)
@@ -695,3 +700,106 @@ def test_masked_policy_matches_the_literal_simulation(oracle, masked, name, kind
         assert set(pos.tolist()) == set(lit.S)
         np.testing.assert_allclose(acc, [lit.column_sum(j) for j in pos], rtol=1e-12, atol=1e-300)
     assert decided >= 8
+
+
+# --------------------------------------------------------------------------
+# "Top-K" attention in decode steps (each query keeps only its m largest logits)
+# --------------------------------------------------------------------------
+@pytest.fixture
+def topk(oracle):
+    def use(m):
+        oracle.set_topk(m)
+
+    yield use
+    oracle.set_topk(0)
+
+
+def _textbook_topk(q, k, v, scale, m):
+    """Causal attention in which every row keeps its m largest logits (numpy argsort; ties cannot occur in random data)."""
+    n = q.shape[0]
+    s = scale * (q.astype(np.float64) @ k.astype(np.float64).T)
+    s = np.where(np.tril(np.ones((n, n), dtype=bool)), s, -np.inf)
+    keep = np.zeros((n, n), dtype=bool)
+    for i in range(n):
+        keep[i, np.argsort(-s[i, :i + 1], kind="stable")[:m]] = True
+    p = scipy_softmax(np.where(keep, s, -np.inf), axis=1)
+    return p @ v.astype(np.float64), p
+
+
+@pytest.mark.parametrize("m", [1, 3, 8])
+def test_topk_with_a_cache_that_never_evicts_is_textbook_top_m_attention(oracle, topk, m):
+    T, d, scale = 36, 8, 0.45
+    rng = np.random.default_rng(700 + m)
+    q, kk, v = _rand_qkv(rng, T, d)
+    ref_out, ref_p = _textbook_topk(q, kk, v, scale, m)
+    topk(m)
+    cache = oracle.OracleCache(1, 1, d, [T], [4], scale=scale)
+    for t in range(T):
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        np.testing.assert_allclose(res["out"][0], ref_out[t], rtol=1e-11, atol=1e-13)
+        assert int((res["p"][0, :t + 1] > 0).sum()) == min(m, t + 1)
+        assert math.fsum(res["p"][0, :t + 1]) == pytest.approx(1.0, abs=1e-14)
+    pos, acc = cache.export(0)
+    np.testing.assert_allclose(acc, ref_p.sum(axis=0), rtol=1e-12, atol=1e-300)  # scores: column sums of what was attended
+
+
+def test_topk_not_smaller_than_the_cache_changes_nothing(oracle, topk):
+    n, steps, d, k, r, scale = 30, 25, 8, 4, 5, 0.5
+    rng = np.random.default_rng(710)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+
+    def run():
+        cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+        cache.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+        res = [cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None]) for t in range(n, n + steps)]
+        return [x["out"] for x in res], [int(x["evicted"][0]) for x in res], cache.export(0)
+
+    ref = run()
+    topk(k + r + 1)  # the kept entries and the token itself
+    got = run()
+    assert got[1] == ref[1]
+    for x, y in zip(got[0], ref[0]):
+        np.testing.assert_array_equal(x, y)
+    np.testing.assert_array_equal(got[2][1], ref[2][1])
+
+
+@pytest.mark.parametrize("k,r,m", [(3, 3, 2), (4, 2, 4), (2, 5, 3), (5, 0, 2)])
+def test_topk_policy_matches_the_literal_simulation(oracle, topk, k, r, m):
+    """Evictions under Top-K attention: explicit column sums of the probability matrix that has zeros for the logits a
+    query dropped, literal argmax of F_score."""
+    T, d, scale = 22, 4, 0.6
+    rng = np.random.default_rng(720 + 10 * k + r + m)
+    q, kk, v = _rand_qkv(rng, T, d)
+    lit = LiteralH2O(k, r, scale, lambda z: z)
+    lit.topk = m
+    topk(m)
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    decided = 0
+    for t in range(T):
+        out_l, ev_l, probs, gap = lit.step(q[t], kk[t], v[t])
+        res = cache.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None], want_p=True)
+        np.testing.assert_allclose(np.sort(res["p"][0, :len(probs)]), np.sort(probs), rtol=1e-12, atol=1e-300)
+        np.testing.assert_allclose(res["out"][0], out_l, rtol=1e-11, atol=1e-13)
+        if 0.0 < gap <= 1e-9:
+            break  # an accidental near-tie: the two would drift apart from here
+        # (an exact tie — two entries no query has attended yet both have score 0 — is decided by position on both sides)
+        assert res["evicted"][0] == ev_l
+        decided += 1
+        pos, acc = cache.export(0)
+        assert set(pos.tolist()) == set(lit.S)
+        np.testing.assert_allclose(acc, [lit.column_sum(j) for j in pos], rtol=1e-12, atol=1e-300)
+    assert decided >= 8
+
+
+def test_topk_tie_keeps_the_higher_position_and_reports_the_gap(oracle, topk):
+    d, scale = 4, 1.0
+    key = np.array([[1.0, 0.0, 0.0, 0.0]], dtype=np.float32)
+    cache = oracle.OracleCache(1, 1, d, [8], [2], scale=scale)
+    zero = np.zeros((1, d), dtype=np.float32)
+    for _ in range(3):  # three identical keys at positions 0, 1, 2
+        cache.decode_step(zero[None], key[None], key[None])
+    topk(2)
+    res = cache.decode_step(key[None], (0.5 * key)[None], key[None], want_p=True)  # logits 1, 1, 1 and 0.5 for itself
+    p = res["p"][0, :4]
+    assert p[0] == 0.0 and p[3] == 0.0 and p[1] == pytest.approx(0.5) and p[2] == pytest.approx(0.5)
+    assert res["topk_gap"][0] == 0.0  # weakest kept and strongest dropped logit are equal
