@@ -304,6 +304,20 @@ int h2o_cache_set_score_mode(h2o_cache_t* cache, int32_t mode);
  * (4-bit slots).
  */
 int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b);
+/*
+ * Heavy hitters combined with "Top-K" attention (appendix "Enhancing the Top-K baseline", the table with and
+ * without H2; results only, no rule).  This library's reading: in a decode step the query attends, of everything it
+ * would otherwise attend (the kept entries, minus what a sparse pattern leaves out, and the token itself), only the
+ * m entries with the largest scaled logits; equal logits: the higher position first.  The others get probability 0
+ * and their accumulated score does not grow in that step; the cache policy itself is unchanged.  The kernel
+ * streams the keys only and reads just the value rows of the attended entries.  m = 0 switches it off.
+ * The prompt rows of h2o_prefill_select stay dense.
+ * Only on an empty cache (H2O_ERR_STATE otherwise); the setting survives h2o_cache_reset.  A unit stays in one
+ * thread block (budgets up to 8192 slots; H2O_ERR_UNSUPPORTED beyond, and for 4-bit slots); h2o_decode_chunk takes
+ * one decode-step kernel per token.  Which of two logits closer than fp32 resolves is the larger one is decided in
+ * fp32 here.
+ */
+int h2o_cache_set_topk(h2o_cache_t* cache, int32_t m);
 int h2o_cache_fscore(h2o_cache_t* cache, int32_t hkind, double* out_dev, void* stream);
 /*
  * Process-wide diagnostic switch (no counterpart in the paper).  A decode kernel launched right

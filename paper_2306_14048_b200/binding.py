@@ -97,6 +97,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_set_chunk_path.restype = c.c_int
     lib.h2o_cache_set_score_mode.argtypes = [vp, c.c_int32]
     lib.h2o_cache_set_score_mode.restype = c.c_int
+    lib.h2o_cache_set_topk.argtypes = [vp, c.c_int32]
+    lib.h2o_cache_set_topk.restype = c.c_int
     lib.h2o_cache_set_mask.argtypes = [vp, c.c_int32, c.c_int32, c.c_int32]
     lib.h2o_cache_set_mask.restype = c.c_int
     lib.h2o_cache_fscore.argtypes = [vp, c.c_int32, vp, vp]
@@ -245,6 +247,10 @@ class H2OCache:
     def set_mask(self, kind: int, a: int = 1, b: int = 0):
         """h2o_cache_set_mask: 0 none, 1 strided(stride a, local window b), 2 fixed(block a, b summary columns)."""
         _check(lib.h2o_cache_set_mask(self._h, int(kind), int(a), int(b)), "h2o_cache_set_mask")
+
+    def set_topk(self, m: int):
+        """h2o_cache_set_topk: in decode steps a query attends only its m largest logits (0 = off)."""
+        _check(lib.h2o_cache_set_topk(self._h, int(m)), "h2o_cache_set_topk")
 
     def fscore(self, hkind: int = 0, stream=None):
         """F_score per (sequence, head): sum of h(accumulated score); h: 0 identity, 1 sqrt(z+1), 2 log(z+1)."""

@@ -157,6 +157,10 @@ struct Shared {
   float red[GROUPS][D];  // per-group partial outputs (unnormalised, relative to the group's maximum)
   float gm[GROUPS], gl[GROUPS];
   Cand wbest[kMaxWarps];
+  // "Top-K" attention: histogram and state of the radix select over the step's logits
+  unsigned int hist[256];
+  unsigned long long tk_prefix;
+  unsigned int tk_remaining, tk_count;
   // Cluster exchange: every block PUSHES its values into its peers' shared memory (remote stores are
   // fire-and-forget, remote loads a round trip), then one cluster barrier makes them visible.
   float x_m[kMaxSplit], x_l[kMaxSplit];  // block statistics of every rank (written by that rank)
@@ -172,7 +176,8 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 // most two blocks per SM runs fastest with all the registers the compiler wants (MINB 1: no spills, more
 // loads in flight per thread); a launch with many blocks per SM is bound by how many of them are
 // resident to hide one another's serial prologue and epilogue (MINB 4).
-template <typename T, int D, int MINB, int NW>
+// TOPK: the instance with "Top-K" attention (its selection code costs registers the plain step must not pay for).
+template <typename T, int D, int MINB, int NW, bool TOPK>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
               T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
@@ -260,9 +265,10 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     const int rows = min(TILE_ROWS, nstr - j * TILE_ROWS);
     const uint32_t bytes = (uint32_t)rows * C::ROW_BYTES;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
-    mbar_expect_tx(&sh.full[s], 2 * bytes);
+    // ("Top-K" attention streams the keys only: which value rows are needed is known after the last score)
+    mbar_expect_tx(&sh.full[s], TOPK ? bytes : 2 * bytes);
     bulk_g2s(dst, Kb + (int64_t)j * TILE_ROWS * D, bytes, &sh.full[s]);
-    bulk_g2s(dst + kTileBytes, Vb + (int64_t)j * TILE_ROWS * D, bytes, &sh.full[s]);
+    if (!TOPK) bulk_g2s(dst + kTileBytes, Vb + (int64_t)j * TILE_ROWS * D, bytes, &sh.full[s]);
   };
   if (tid == kThreads) {  // producer lane: set up the barriers and get the first tiles moving at once
     for (int s = 0; s < stages; ++s) {
@@ -333,6 +339,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     }
     // a sparse pattern needs the slots' positions during the stream (they are staged with the scores)
     const int mask_kind = c.mask_kind;
+    constexpr bool topk_mode = TOPK;  // (the host launches one block per unit then: split == 1)
     if (mask_kind != 0 && nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
     for (int j = 0; j < ntile; ++j) {
       const int s = j % stages;
@@ -349,7 +356,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
         if (row < rows) {
           float kf[VEC];
           Vec16<T>::load(kt + row * D + ch * VEC, kf);
-          Vec16<T>::load(vt + row * D + ch * VEC, vf[ps]);
+          if (!topk_mode) Vec16<T>::load(vt + row * D + ch * VEC, vf[ps]);
           float2 d2 = make_float2(0.f, 0.f);  // two fp32 FMAs per instruction (packed fp32x2 of this architecture)
 #pragma unroll
           for (int v = 0; v < VEC; v += 2)
@@ -369,6 +376,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       float mnew = mg;
 #pragma unroll
       for (int ps = 0; ps < C::PASSES; ++ps) mnew = fmaxf(mnew, sc[ps]);
+      if (topk_mode) mnew = -INFINITY;  // scores only: softmax and values follow the selection
       if (mnew > -INFINITY) {  // at least one real row so far in this group
         const float f = expf(mg - mnew);  // expf(-inf) = 0 for the group's first rows
         lg *= f;
@@ -409,6 +417,124 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     {
     H2O_STAMP(8);
 
+    float part_o = 0.f;  // block partial output relative to the block maximum
+    if constexpr (TOPK) {
+      // ---- "Top-K" attention: keep the c.topk largest logits of the step (the kept entries the pattern allows,
+      // and the token itself; equal logits: the higher position first).  All raw scores are in shared memory.
+      // The key of an entry is (order-preserving bits of its logit, position): keys are distinct, so the
+      // topk-th largest one is a threshold; it is found by a most-significant-digit radix select, 8 bits a pass.
+      auto key_of = [&](int x) -> unsigned long long {  // x < nloc: cached row x; x == nloc: the token itself
+        const float sx = x < nloc ? p[x] : s_self;
+        if (!(sx > -INFINITY)) return 0ull;  // left out by the pattern: below every real key
+        unsigned int ub = __float_as_uint(sx);
+        ub = (ub & 0x80000000u) ? ~ub : (ub | 0x80000000u);
+        return ((unsigned long long)ub << 32) | (unsigned int)(x < nloc ? pos_s[x] : t);
+      };
+      const int ncand = nloc + 1;
+      if (tid == 0) {
+        sh.tk_prefix = 0ull;
+        sh.tk_remaining = (unsigned int)c.topk;
+        sh.tk_count = 0u;
+      }
+      consumer_sync<kThreads>();
+      {
+        unsigned int real = 0;
+        for (int x = tid; x < ncand; x += kThreads) real += key_of(x) != 0ull ? 1u : 0u;
+        real = (unsigned int)warp_sum((float)real);  // (at most 8193 per unit: exact in fp32)
+        if (lane == 0) atomicAdd(&sh.tk_count, real);
+      }
+      consumer_sync<kThreads>();
+      unsigned long long thr = 1ull;  // every real key
+      if (sh.tk_count > (unsigned int)c.topk) {
+        for (int pass = 0; pass < 8; ++pass) {
+          const int shift = 56 - 8 * pass;
+          for (int i = tid; i < 256; i += kThreads) sh.hist[i] = 0u;
+          consumer_sync<kThreads>();
+          const unsigned long long prefix = sh.tk_prefix;
+          const unsigned long long himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
+          for (int x = tid; x < ncand; x += kThreads) {
+            const unsigned long long key = key_of(x);
+            if (key != 0ull && (key & himask) == prefix) atomicAdd(&sh.hist[(unsigned int)(key >> shift) & 255u], 1u);
+          }
+          consumer_sync<kThreads>();
+          if (warp == 0) {  // the bin that holds the rank still looked for, scanning from the top bin down
+            const int rem = (int)sh.tk_remaining;
+            int cnts[8], tot = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              cnts[i] = (int)sh.hist[255 - 8 * lane - i];
+              tot += cnts[i];
+            }
+            int incl = tot;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+              const int y = __shfl_up_sync(0xffffffffu, incl, off);
+              if (lane >= off) incl += y;
+            }
+            int before = incl - tot;
+            if (before < rem && incl >= rem) {  // exactly one lane
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                if (before < rem && before + cnts[i] >= rem) {
+                  sh.tk_prefix = prefix | ((unsigned long long)(255 - 8 * lane - i) << shift);
+                  sh.tk_remaining = (unsigned int)(rem - before);
+                  before = rem;  // done
+                } else {
+                  before += cnts[i];
+                }
+              }
+            }
+          }
+          consumer_sync<kThreads>();
+        }
+        thr = sh.tk_prefix;
+      }
+      // drop what is below the threshold; block statistics over what is left
+      if (key_of(nloc) < thr) s_self = -INFINITY;  // (every thread alike)
+      float mx = -INFINITY;
+      for (int x = tid; x < nloc; x += kThreads) {
+        if (key_of(x) < thr) p[x] = -INFINITY;
+        mx = fmaxf(mx, p[x]);
+      }
+      mx = warp_max(mx);
+      if (lane == 0) sh.gm[warp] = mx;
+      consumer_sync<kThreads>();
+      float mc = s_self;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) mc = fmaxf(mc, sh.gm[w]);
+      float sum = 0.f;
+      for (int x = tid; x < nloc; x += kThreads) sum += p[x] > -INFINITY ? expf(p[x] - mc) : 0.f;
+      sum = warp_sum(sum);
+      if (lane == 0) sh.gl[warp] = sum;
+      // the value rows of the attended entries, straight from memory (row group g takes rows g, g + GROUPS, ...)
+      float ov[VEC];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) ov[v] = 0.f;
+      for (int x = g; x < nloc; x += GROUPS) {
+        const float sx = p[x];
+        if (sx > -INFINITY) {
+          const float ex = expf(sx - mc);
+          float vrow[VEC];
+          Vec16<T>::load(Vb + (int64_t)x * D + ch * VEC, vrow);
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) ov[v] = fmaf(ex, vrow[v], ov[v]);
+        }
+      }
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) sh.red[g][ch * VEC + v] = ov[v];
+      consumer_sync<kThreads>();
+      const float w_self = s_self > -INFINITY ? expf(s_self - mc) : 0.f;
+      float lc = w_self;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) lc += sh.gl[w];
+      if (tid < D) {
+#pragma unroll
+        for (int g2 = 0; g2 < GROUPS; ++g2) part_o += sh.red[g2][tid];
+        part_o = fmaf(w_self, vself, part_o);
+      }
+      m = mc;
+      l = lc;
+    } else {
     // ---- block statistics, computed by every warp alike (fixed order, same result) -------
     const float m_i = lane < GROUPS ? sh.gm[lane] : -INFINITY;
     float mc = warp_max(m_i);
@@ -419,7 +545,6 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     const float w_self = rank == 0 ? expf(s_self - mc) : 0.f;
     lc += w_self;
     H2O_STAMP(9);
-    float part_o = 0.f;  // block partial output relative to mc
 #pragma unroll
     for (int g2 = 0; g2 < GROUPS; ++g2) {
       const float w = __shfl_sync(0xffffffffu, w_i, g2);
@@ -449,6 +574,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
       m = mc;
       l = lc;
     }
+    }  // (not "Top-K")
     H2O_STAMP(4);
     const float inv_l = 1.0f / l;
     if (rank == 0 && tid < D) {
@@ -550,7 +676,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   H2O_STAMP(6);
 }
 
-template <typename T, int D, int MINB, int NW>
+template <typename T, int D, int MINB, int NW, bool TOPK = false>
 cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req, int launch_flags, const void* q,
                         const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   using C = Cfg<T, D, NW>;
@@ -567,7 +693,7 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
   {
     cudaError_t e =
-        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB, NW>), kMaxDynSmem, &attr_flags);
+        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kernel<T, D, MINB, NW, TOPK>), kMaxDynSmem, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   if (smem > (size_t)kMaxDynSmem) return cudaErrorInvalidValue;
@@ -585,7 +711,7 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW>, c, static_cast<const T*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW, TOPK>, c, static_cast<const T*>(q),
                             static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
                             evicted_pos, split, chunk, stages, launch_flags);
 }
@@ -594,6 +720,8 @@ template <typename T, int D>
 cudaError_t launch(const CacheView& c, int split, int chunk, int stages_req, int quiescent, const void* q,
                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   const int blocks = c.units * split;
+  if (c.topk > 0)  // "Top-K" attention: its own instance (four blocks per SM; one block per unit)
+    return launch_minb<T, D, 4, 8, true>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
   if (blocks > 4 * sm_count() && chunk <= kSmallUnitRows)  // many small units: half-size blocks, five per SM
     return launch_minb<T, D, 5, 4>(c, split, chunk, stages_req, quiescent, q, k_new, v_new, out, evicted_pos, stream);
   if (blocks > 2 * sm_count())
@@ -613,6 +741,7 @@ cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, i
                           const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                           cudaStream_t stream) {
   if (split < 1 || split > kMaxSplit) return cudaErrorInvalidValue;
+  if (c.topk > 0 && split != 1) return cudaErrorInvalidValue;  // the selection runs over one block's scores
   int quiescent = (quiescent_b ? 1 : 0) | (all_full ? 2 : 0);  // launch flags
 #ifdef H2O_PHASE_TIMERS
   static int launch_no = 0;

@@ -307,6 +307,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   v.mask_kind = 0;
   v.mask_a = 1;
   v.mask_b = 0;
+  v.topk = 0;
   v.seq_rwin = reinterpret_cast<const int32_t*>(ws + L.seq_rwin);
   v.total_slots = L.total_slots;
   c->seen.assign(cfg->batch, attach ? -1 : 0);
@@ -488,7 +489,8 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   g_last_writer.note_and_check(st, cache->view.K);
   cudaError_t e = cudaSuccess;
   // (the chunk kernel ranks by the accumulated score only)
-  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && cache->view.mask_kind == 0 && !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+  if (cache->chunk_path == 0 && cache->view.score_mode == 0 && cache->view.mask_kind == 0 && cache->view.topk == 0 &&
+      !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
@@ -533,6 +535,20 @@ int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b) {
   cache->view.mask_kind = kind;
   cache->view.mask_a = kind ? a : 1;
   cache->view.mask_b = kind ? b : 0;
+  return H2O_OK;
+}
+
+int h2o_cache_set_topk(h2o_cache_t* cache, int32_t m) {
+  if (!cache || m < 0) return H2O_ERR_INVALID_ARG;
+  if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one attention rule per generation
+  if (m > 0) {
+    if (cache->view.kv4) return H2O_ERR_UNSUPPORTED;
+    const int chunk = (cache->layout.max_B + 3) & ~3;  // one thread block per unit: the selection runs over its scores
+    if (chunk > kMaxChunk) return H2O_ERR_UNSUPPORTED;
+    cache->split = 1;
+    cache->chunk = chunk;
+  }
+  cache->view.topk = m;
   return H2O_OK;
 }
 
@@ -660,6 +676,7 @@ int h2o_cache_reset(h2o_cache_t* cache, void* stream) {
 int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages) {
   if (!cache || stages < 0 || stages > 8) return H2O_ERR_INVALID_ARG;
   if (split != 0 && split != 1 && split != 2 && split != 4 && split != 8) return H2O_ERR_INVALID_ARG;
+  if (split > 1 && cache->view.topk > 0) return H2O_ERR_UNSUPPORTED;  // "Top-K" attention keeps a unit in one block
   if (split != 0) {
     const int chunk = (((cache->layout.max_B + split - 1) / split) + 3) & ~3;
     if (chunk > kMaxChunk) return H2O_ERR_UNSUPPORTED;

@@ -47,6 +47,9 @@ struct CacheView {
   // patterns, Section 5.1): 0 none, 1 strided(stride mask_a, local window mask_b), 2 fixed(block mask_a, mask_b
   // summary columns).  See key_attended().
   int32_t mask_kind, mask_a, mask_b;
+  // "Top-K" attention in decode steps (appendix "Enhancing the Top-K baseline"): > 0: a query attends only its topk
+  // largest logits among what it would otherwise attend (equal logits: the higher position); 0: off.
+  int32_t topk;
   const int32_t* seq_rwin;  // [batch] recent window of every sequence (the prompt kernels index by unit, not by launch position)
   int64_t total_slots;      // slots of all units together (the limit of every slot index)
 };

@@ -40,6 +40,7 @@ def main():
         ("4-bit slots", wl("b8", 3, 2, 128, "bf16_kv4", [300, 77, 513], 24, [20, 9, 33], [24, 5, 31], 808), {}),
         ("chunk call", wl("b9", 2, 3, 128, "bf16", [400, 300], 40, [20, 30], [24, 16], 809), dict(chunk=16)),
         ("sparse pattern", wl("b10", 2, 3, 128, "bf16", [400, 300], 24, [20, 30], [24, 16], 810), dict(mask=(1, 8, 3))),
+        ("top-k attention", wl("b12", 2, 3, 128, "bf16", [400, 300], 24, [20, 30], [24, 16], 812), dict(topk=9)),
     ]
     for name, w, kw in cases:
         st = run_parity(w, pkg.H2OCache, export_every=8, **kw)  # asserts status == 0 at the end

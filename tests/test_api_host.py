@@ -90,6 +90,7 @@ def test_create_argument_checks_and_no_fallback(pkg):
     assert pkg.lib.h2o_cache_set_score_mode(None, 0) == pkg.H2O_ERR_INVALID_ARG
     assert pkg.lib.h2o_cache_fscore(None, 0, None, None) == pkg.H2O_ERR_INVALID_ARG
     assert pkg.lib.h2o_cache_set_mask(None, 1, 4, 2) == pkg.H2O_ERR_INVALID_ARG
+    assert pkg.lib.h2o_cache_set_topk(None, 4) == pkg.H2O_ERR_INVALID_ARG
     assert pkg.lib.h2o_prefill_select(None, None, None, None, None, None, None, 0, None) == pkg.H2O_ERR_INVALID_ARG
 
 

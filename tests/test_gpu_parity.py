@@ -407,3 +407,60 @@ def test_sparse_pattern_argument_and_state_errors(H2OCache):
     kv4 = H2OCache(1, 2, 128, "bf16_kv4", [4], [4])
     assert pkg.lib.h2o_cache_set_mask(kv4._h, 1, 4, 2) == pkg.H2O_ERR_UNSUPPORTED
     kv4.close()
+
+
+# ---------------------------------------------------------------------------------------------------------
+# heavy hitters combined with "Top-K" attention in decode steps (h2o_cache_set_topk)
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("m", [1, 7, 40, 500])
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_topk_attention_ragged(H2OCache, m, dtype, d):
+    """m below, around and above the cache size (above: everything is attended, through the same code path)."""
+    from parity_harness import run_parity
+
+    wl = _wl("topk", 4, 3, d, dtype, [300, 77, 513, 40], 48, [20, 9, 33, 30], [24, 5, 31, 30], seed=277 + d)
+    st = run_parity(wl, H2OCache, export_every=8, topk=m)
+    print(st)
+
+
+@pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([6, 1], [12, 9])])
+def test_topk_attention_edge_budgets_token_by_token(H2OCache, heavy, recent):
+    """Fill phase from an empty cache, no heavy hitters, no recent window (the new token may be the one dropped, and with
+    Top-K attention it may not even attend itself)."""
+    from parity_harness import run_parity
+
+    wl = _wl("topkedge", 2, 2, 64, "f32", [1, 1], 60, heavy, recent, seed=25)
+    for m in (1, 3):
+        st = run_parity(wl, H2OCache, prefill=False, export_every=5, topk=m)
+        print(st)
+
+
+def test_topk_attention_long_budget_pattern_and_chunk_call(H2OCache):
+    """A budget that would be split over a cluster stays in one block; Top-K on top of a sparse pattern; the
+    multi-token call falls back to one decode-step kernel per token."""
+    from parity_harness import run_parity
+
+    wl = _wl("topklong", 2, 2, 128, "bf16", [1500, 1300], 24, [600, 500], [500, 600], seed=231)
+    print(run_parity(wl, H2OCache, export_every=8, topk=64))
+    wl = _wl("topkmask", 2, 3, 128, "bf16", [400, 300], 40, [20, 30], [24, 16], seed=232)
+    print(run_parity(wl, H2OCache, export_every=8, topk=9, mask=(1, 8, 3)))
+    print(run_parity(wl, H2OCache, export_every=8, topk=9, chunk=16))
+
+
+def test_topk_argument_and_state_errors(H2OCache):
+    import paper_2306_14048_b200 as pkg
+
+    cache = H2OCache(1, 2, 64, "f32", [4], [4])
+    assert pkg.lib.h2o_cache_set_topk(cache._h, -1) == pkg.H2O_ERR_INVALID_ARG
+    cache.set_topk(3)
+    assert pkg.lib.h2o_cache_set_decode_shape(cache._h, 2, 0) == pkg.H2O_ERR_UNSUPPORTED
+    x = torch.zeros(1, 2, 64, device="cuda")
+    cache.decode_step(x, x, x, torch.empty_like(x))
+    assert pkg.lib.h2o_cache_set_topk(cache._h, 0) == pkg.H2O_ERR_STATE
+    cache.close()
+    kv4 = H2OCache(1, 2, 128, "bf16_kv4", [4], [4])
+    assert pkg.lib.h2o_cache_set_topk(kv4._h, 2) == pkg.H2O_ERR_UNSUPPORTED
+    kv4.close()
+    big = H2OCache(1, 1, 64, "f32", [6000], [6000])
+    assert pkg.lib.h2o_cache_set_topk(big._h, 2) == pkg.H2O_ERR_UNSUPPORTED
+    big.close()
