@@ -482,6 +482,35 @@ class ConfigRun:
         return {"us_per_launch": us, "bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
                 "speedup_vs_bf16_slots": bf16_launch_us / us, "layer_caches": Lk}
 
+    def topk_figure(self, m=64):
+        """The same decode steps with "Top-K" attention (each query attends its m largest logits): the kernel streams
+        the keys only and reads m value rows per unit; rotating over (up to 8) layer caches."""
+        wl, pkg = self.wl, self.pkg
+        if max(k + r for k, r in zip(wl.heavy, wl.recent)) > 8192:
+            return None
+        Lk = min(self.L, 8)
+        kc = [pkg.H2OCache(wl.batch, self.H, self.d, wl.dtype, wl.heavy, wl.recent, device=self.local) for _ in range(Lk)]
+        for l in range(Lk):
+            kc[l].set_topk(m)
+            q, k, v = self.prompts[l] if self.resident else self._draw_prompt(l)
+            kc[l].prefill_select(q, k, v, self.cu, self.outs[l if self.resident else 0], self.stream)
+        n_k = min(32, self.S)
+
+        def loop():
+            for s in range(n_k):
+                for l in range(Lk):
+                    d_ = self.dec[l]
+                    kc[l].decode_step(d_[0][s], d_[1][s], d_[2][s], d_[3][s], d_[4][s], self.stream)
+
+        us = self.graph_replay_us(loop, n_k * Lk)
+        for c in kc:
+            assert c.status() == 0, "device status word set"
+            c.close()
+        cnt = slot_counts(wl)
+        nbytes = sum(c_ * self.d * self.esize + min(m, c_) * self.d * self.esize + 20 * c_ + 6 * self.d * self.esize for c_ in cnt) * self.H
+        return {"m": m, "us_per_launch": us, "bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
+                "layer_caches": Lk}
+
     def e2e(self, n_steps):
         """The same step through the host-buffer C calls, pinned host tensors; on at most `e2e_layers` layers."""
         wl, L, S = self.wl, self.L, self.S
@@ -627,6 +656,8 @@ def measure_config(pkg, wl, layers, dev, local, rank, world, dist, args, steps, 
         if headline or args.context:
             rec["decode_chunk_one_layer"] = run.chunk_figure()
         rec["decode_kv4_slots"] = run.kv4_figure(launch_us)
+        if headline or args.context:
+            rec["decode_topk_attention"] = run.topk_figure()
     e2e = None
     if not args.no_e2e and (headline or args.e2e_all):
         e = run.e2e(max(1, min(steps, 2)))
@@ -725,7 +756,7 @@ def main():
         }
         for key in ("prefill_ms", "decode_ms", "decode_only_seq_heads_per_s", "prefill_tflops_algorithmic",
                     "wall_ms_per_step_with_input_generation", "clocks", "roofline", "roofline_prefill",
-                    "decode_chunk_one_layer", "decode_kv4_slots", "e2e"):
+                    "decode_chunk_one_layer", "decode_kv4_slots", "decode_topk_attention", "e2e"):
             if key in rec:
                 out[key] = rec[key]
         if per_config:
