@@ -160,7 +160,7 @@ struct Shared {
   // "Top-K" attention: histogram and state of the radix select over the step's logits
   unsigned int hist[256];
   unsigned long long tk_prefix;
-  unsigned int tk_remaining, tk_count;
+  unsigned int tk_remaining, tk_count, tk_bin;  // tk_bin: entries in the bin the last pass chose
   // Cluster exchange: every block PUSHES its values into its peers' shared memory (remote stores are
   // fire-and-forget, remote loads a round trip), then one cluster barrier makes them visible.
   float x_m[kMaxSplit], x_l[kMaxSplit];  // block statistics of every rank (written by that rank)
@@ -478,6 +478,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
                 if (before < rem && before + cnts[i] >= rem) {
                   sh.tk_prefix = prefix | ((unsigned long long)(255 - 8 * lane - i) << shift);
                   sh.tk_remaining = (unsigned int)(rem - before);
+                  sh.tk_bin = (unsigned int)cnts[i];
                   before = rem;  // done
                 } else {
                   before += cnts[i];
@@ -486,6 +487,9 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
             }
           }
           consumer_sync<kThreads>();
+          // after the four passes over the logit's bits: if every entry that shares the threshold logit is wanted
+          // (nearly always: it is the only one), the positions need not be looked at
+          if (pass == 3 && sh.tk_bin == sh.tk_remaining) break;
         }
         thr = sh.tk_prefix;
       }
