@@ -706,15 +706,17 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute at[2];
+  cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)split;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
+  at[2].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+  at[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
   cfg.attrs = at;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = split > 1 ? 3 : 2;
   return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW, TOPK>, c, static_cast<const T*>(q),
                             static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
                             evicted_pos, split, chunk, stages, launch_flags);
