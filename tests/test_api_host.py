@@ -52,6 +52,27 @@ def test_workspace_arithmetic(pkg):
     assert pkg.h2o_prefill_scratch_bytes(cfg, 0) == 0
 
 
+def test_full_cache_bytes_match_the_papers_example(pkg):
+    """Section 1: a 30B model, batch 128, sequence length 1024 -> 180 GB of KV cache.  With a budget equal to the
+    sequence length the library's K/V slots are that cache; its scores and positions add 12 bytes per slot."""
+    vals = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "kv_cache_size.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            vals[k] = int(v)
+    b, h, d, n = vals["batch"], vals["n_heads"], vals["head_dim"], vals["seq_len"]
+    cfg, keep = pkg.make_config(b, h, d, "bf16", [n // 2] * b, [n // 2] * b)
+    per_layer = pkg.h2o_cache_workspace_bytes(cfg)
+    slots = b * h * n
+    kv = 2 * slots * d * vals["bytes_per_element"]
+    assert abs(kv * vals["model_layers"] / 1e9 - vals["kv_cache_gb"]) < 1.0  # 180.4 GB
+    assert kv + slots * 12 <= per_layer <= kv + slots * 12 + slots * 4 + (b * h + 1024) * (d + 4) * 4 + (1 << 20)
+    import bench
+
+    one_unit_step = bench.decode_bytes_per_unit_step(n, d, vals["bytes_per_element"])
+    assert one_unit_step == 2 * n * d * 2 + 20 * n + 6 * d * 2  # the decode step reads that cache once
+
+
 @pytest.mark.parametrize("kw", [
     dict(head_dim=96), dict(dtype=7), dict(batch=0), dict(n_heads=0), dict(heavy=[-1]), dict(heavy=[0], recent=[0]),
     dict(recent=[1 << 20]),
