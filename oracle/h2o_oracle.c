@@ -119,7 +119,7 @@ static int logit_cmp(const void* a, const void* b) { /* strongest first: larger 
 /*
  * Causal softmax attention of one (sequence, head) and the column sums of its
  * probability matrix.
- *   Q, K, V : n rows of d floats, consecutive rows `stride` floats apart.
+ *   Q, K, V : n rows of d floats, consecutive rows `stride_q` (Q) and `stride` (K, V) floats apart.
  *   c       : softmax scale.
  *   O       : [n][d]  O_i = sum_{j<=i} P[i][j] V_j
  *   rowmax, rowsum : [n]  m_i = max_j s_ij,  l_i = sum_j exp(s_ij - m_i)
@@ -129,10 +129,10 @@ static int logit_cmp(const void* a, const void* b) { /* strongest first: larger 
  * With a sparse pattern set (h2o_oracle_set_mask) row i leaves out the keys j of its recent window
  * (i - r < j < i, r = `window`) that the pattern does not allow: P[i][j] = 0 there.
  */
-int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const float* V, long n, long d, long stride,
-                                       double c, long window, double* O, double* rowmax, double* rowsum, double* acc0,
-                                       double* P_out) {
-  if (n < 0 || d <= 0 || stride < d) return -1;
+int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const float* V, long n, long d, long stride_q,
+                                       long stride, double c, long window, double* O, double* rowmax, double* rowsum,
+                                       double* acc0, double* P_out) {
+  if (n < 0 || d <= 0 || stride < d || stride_q < d) return -1;
   int failed = 0;
 #pragma omp parallel
   {
@@ -144,7 +144,7 @@ int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const flo
 #pragma omp for schedule(dynamic, 4)
     for (long i = 0; i < n; ++i) {
       if (!e) continue;
-      const float* qi = Q + i * stride;
+      const float* qi = Q + i * stride_q;
       double m = -INFINITY;
       for (long j = 0; j <= i; ++j) {
         if (!attended(j, i, window)) continue;
@@ -177,7 +177,7 @@ int h2o_oracle_causal_attention_colsum(const float* Q, const float* K, const flo
       double a = 0.0;
       for (long i = j; i < n; ++i) {
         if (!attended(j, i, window)) continue;
-        const double s = c * dot_fd(Q + i * stride, kj, d);
+        const double s = c * dot_fd(Q + i * stride_q, kj, d);
         a += exp(s - rowmax[i]) / rowsum[i];
       }
       acc0[j] = a;
@@ -288,7 +288,12 @@ long h2o_oracle_select(const double* acc0, long n, long k, long r, int32_t* kept
  * State, per unit u, in rows of capacity `cap` (>= k+r+1) entries:
  *   cnt[u], t[u], pos[u][cap], acc[u][cap], Kc[u][cap][d], Vc[u][cap][d]
  * Entry order carries no meaning; only `pos` does.
- * Inputs: q, knew, vnew [units][d]; kbud, rwin [units]; scale c.
+ * Inputs: q [units][group][d], knew, vnew [units][d]; kbud, rwin [units]; scale c.
+ * group: query heads that share one unit's keys and values (grouped-query attention; 1 = every head has its own).
+ *        The paper evicts per head and has no such sharing; the nearest text is its comparison with a method that
+ *        accumulates scores across heads.  Reading: each query head of the group attends the shared entries with its
+ *        own softmax, and a key's accumulated score grows by the SUM of the probabilities the group's heads gave it;
+ *        out is [units][group][d].
  * hint  : optional [units]; a decision made elsewhere for this step (-1 none,
  *         >= 0 evicted position, -2 = no hint).  The oracle always computes its own
  *         victim first.  If the hint names a different candidate whose accumulated
@@ -302,7 +307,7 @@ long h2o_oracle_select(const double* acc0, long n, long k, long r, int32_t* kept
  *          "Top-K" attention on, the relative gap between the weakest kept and the strongest dropped logit
  *          (inf when nothing was dropped).
  */
-int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, const int32_t* rwin, int32_t* t,
+int h2o_oracle_decode_step(long units, long group, long d, long cap, const int32_t* kbud, const int32_t* rwin, int32_t* t,
                            int32_t* cnt, int32_t* pos, double* acc, double* Kc, double* Vc, const float* q,
                            const float* knew, const float* vnew, double c, const int32_t* hint, double tie_rel,
                            double* out, int32_t* evicted, int32_t* status, double* gap, double* p_out, double* tgap) {
@@ -330,19 +335,22 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
       uv[m * d + x] = (double)vnew[u * d + x];
     }
     m += 1;
-    /* scores, softmax, output */
+    /* scores, softmax, output: once per query head of the unit's group (one without grouped-query attention);
+     * every query head adds its probabilities to the shared keys' accumulated scores */
+    if (tgap) tgap[u] = INFINITY;
     double* e = (double*)malloc(sizeof(double) * (size_t)m);
     char* att = (char*)malloc((size_t)m);
+    for (long g = 0; g < group; ++g) {
+    const float* qg = q + (u * group + g) * d;
     long natt = 0;
     for (long j = 0; j < m; ++j) {
       att[j] = (char)attended(up[j], tt, r); /* 0: left out by the sparse pattern (none by default) */
       if (!att[j]) continue;
       double s = 0.0;
-      for (long x = 0; x < d; ++x) s += (double)q[u * d + x] * uk[j * d + x];
+      for (long x = 0; x < d; ++x) s += (double)qg[x] * uk[j * d + x];
       e[j] = c * s;
       natt += 1;
     }
-    if (tgap) tgap[u] = INFINITY;
     if (g_topk > 0 && natt > g_topk) { /* keep the g_topk strongest logits only */
       logit_t* lg = (logit_t*)malloc(sizeof(logit_t) * (size_t)natt);
       long n2 = 0;
@@ -355,7 +363,7 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
         }
       qsort(lg, (size_t)natt, sizeof(logit_t), logit_cmp);
       for (long x = g_topk; x < natt; ++x) att[lg[x].idx] = 0;
-      if (tgap) tgap[u] = rel_gap(lg[g_topk - 1].s, lg[g_topk].s); /* weakest kept against strongest dropped */
+      if (tgap) tgap[u] = fmin(tgap[u], rel_gap(lg[g_topk - 1].s, lg[g_topk].s)); /* weakest kept against strongest dropped */
       free(lg);
     }
     double mx = -INFINITY;
@@ -366,15 +374,16 @@ int h2o_oracle_decode_step(long units, long d, long cap, const int32_t* kbud, co
       e[j] = att[j] ? exp(e[j] - mx) : 0.0;
       l += e[j];
     }
-    free(att);
-    double* o = out + u * d;
+    double* o = out + (u * group + g) * d;
     for (long x = 0; x < d; ++x) o[x] = 0.0;
     for (long j = 0; j < m; ++j) {
       const double p = e[j] / l;
       for (long x = 0; x < d; ++x) o[x] += p * uv[j * d + x];
       ua[j] += p; /* accumulate */
-      if (p_out) p_out[u * cap + j] = p;
+      if (p_out) p_out[u * cap + j] = g == 0 ? p : p_out[u * cap + j] + p; /* (summed over the group) */
     }
+    } /* query heads of the group */
+    free(att);
     free(e);
     /* eviction */
     evicted[u] = -1;

@@ -42,11 +42,11 @@ def _load():
         dp, fp, ip = c.POINTER(c.c_double), c.POINTER(c.c_float), c.POINTER(c.c_int32)
         lib.h2o_oracle_num_threads.restype = c.c_int
         lib.h2o_oracle_causal_attention_colsum.restype = c.c_int
-        lib.h2o_oracle_causal_attention_colsum.argtypes = [fp, fp, fp, c.c_long, c.c_long, c.c_long, c.c_double, c.c_long, dp, dp, dp, dp, dp]
+        lib.h2o_oracle_causal_attention_colsum.argtypes = [fp, fp, fp, c.c_long, c.c_long, c.c_long, c.c_long, c.c_double, c.c_long, dp, dp, dp, dp, dp]
         lib.h2o_oracle_select.restype = c.c_long
         lib.h2o_oracle_select.argtypes = [dp, c.c_long, c.c_long, c.c_long, ip, dp]
         lib.h2o_oracle_decode_step.restype = c.c_int
-        lib.h2o_oracle_decode_step.argtypes = [c.c_long, c.c_long, c.c_long, ip, ip, ip, ip, ip, dp, dp, dp, fp, fp, fp,
+        lib.h2o_oracle_decode_step.argtypes = [c.c_long, c.c_long, c.c_long, c.c_long, ip, ip, ip, ip, ip, dp, dp, dp, fp, fp, fp,
                                                c.c_double, ip, c.c_double, dp, ip, ip, dp, dp, dp]
         lib.h2o_oracle_set_score_mode.restype = c.c_int
         lib.h2o_oracle_set_score_mode.argtypes = [c.c_int]
@@ -80,15 +80,15 @@ def causal_attention_colsum(q, k, v, scale: float, want_p: bool = False, window:
     ``window``: the unit's recent window r; only read when a sparse pattern is set (``set_mask``)."""
     n, d = q.shape
     assert q.dtype == np.float32 and k.dtype == np.float32 and v.dtype == np.float32
-    stride = q.strides[0] // 4
-    assert q.strides == k.strides == v.strides and q.strides[1] == 4
+    stride_q, stride = q.strides[0] // 4, k.strides[0] // 4
+    assert k.strides == v.strides and q.strides[1] == 4 and k.strides[1] == 4
     O = np.empty((n, d), dtype=np.float64)
     rowmax = np.empty(n, dtype=np.float64)
     rowsum = np.empty(n, dtype=np.float64)
     acc0 = np.empty(n, dtype=np.float64)
     P = np.empty((n, n), dtype=np.float64) if want_p else None
     rc = _load().h2o_oracle_causal_attention_colsum(
-        _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), n, d, stride, float(scale), int(window),
+        _p(q, ctypes.c_float), _p(k, ctypes.c_float), _p(v, ctypes.c_float), n, d, stride_q, stride, float(scale), int(window),
         _p(O, ctypes.c_double), _p(rowmax, ctypes.c_double), _p(rowsum, ctypes.c_double), _p(acc0, ctypes.c_double),
         _p(P, ctypes.c_double))
     if rc != 0:
@@ -143,12 +143,15 @@ class OracleCache:
     """State of ``batch * n_heads`` independent units; unit index = sequence * n_heads + head."""
 
     def __init__(self, batch: int, n_heads: int, head_dim: int, heavy: Sequence[int], recent: Sequence[int], scale: Optional[float] = None,
-                 kv4: bool = False):
+                 kv4: bool = False, group: int = 1):
         """kv4: stored K/V rows are 4-bit group-quantised (oracle/kv_quant.py): a row is quantised when it
         enters the cache — the kept prompt rows after selection, a new token's row after its own step, in
         which it still takes part at full precision."""
         assert len(heavy) == batch and len(recent) == batch
         self.kv4 = bool(kv4)
+        # grouped-query attention: `group` query heads share the keys and values of one (sequence, head) unit; q and
+        # out then have n_heads * group heads (query head = head * group + g), k and v n_heads
+        self.group = int(group)
         self.batch, self.n_heads, self.d = batch, n_heads, head_dim
         self.units = batch * n_heads
         self.scale = float(scale) if scale and scale > 0 else 1.0 / float(np.sqrt(head_dim))
@@ -175,6 +178,7 @@ class OracleCache:
         q, k, v = _f32(q), _f32(k), _f32(v)
         cu = np.asarray(cu_seqlens, dtype=np.int64)
         out = np.full(q.shape, np.nan, dtype=np.float64)
+        G = self.group
         todo = range(self.units) if units is None else units
         kept_all = {}
         self.last_acc0 = [None] * self.units
@@ -182,8 +186,12 @@ class OracleCache:
         for u in todo:
             s, h = divmod(u, self.n_heads)
             lo, hi = int(cu[s]), int(cu[s + 1])
-            O, acc0 = causal_attention_colsum(q[lo:hi, h], k[lo:hi, h], v[lo:hi, h], self.scale, window=int(self.rwin[u]))
-            out[lo:hi, h] = O
+            acc0 = 0.0
+            for g in range(G):  # every query head of the group over the shared keys; column sums add up
+                O, a_g = causal_attention_colsum(q[lo:hi, h * G + g], k[lo:hi, h], v[lo:hi, h], self.scale,
+                                                 window=int(self.rwin[u]))
+                out[lo:hi, h * G + g] = O
+                acc0 = acc0 + a_g
             kept, boundary = select(acc0, int(self.kbud[u]), int(self.rwin[u]))
             self.last_acc0[u], self.last_boundary[u] = acc0, boundary
             kept_all[u] = kept
@@ -209,9 +217,9 @@ class OracleCache:
                     units: Optional[Sequence[int]] = None):
         """One step for all units (or the listed ones).  q, k_new, v_new: ``[batch, n_heads, d]``.
 
-        Returns dict(out [units, d], evicted [units], status [units], gap [units], p [units, cap] or None).
+        Returns dict(out [units, group * d], evicted [units], status [units], gap [units], p [units, cap] or None).
         """
-        qf = _f32(q).reshape(self.units, self.d)
+        qf = _f32(q).reshape(self.units, self.group * self.d)
         kf = _f32(k_new).reshape(self.units, self.d)
         vf = _f32(v_new).reshape(self.units, self.d)
         t_before = self.t.copy()
@@ -233,7 +241,7 @@ class OracleCache:
     @staticmethod
     def _decode(st, qf, kf, vf, hint, tie_rel, want_p):
         n = st.cnt.shape[0]
-        out = np.empty((n, st.d), dtype=np.float64)
+        out = np.empty((n, st.group * st.d), dtype=np.float64)
         evicted = np.empty(n, dtype=np.int32)
         status = np.empty(n, dtype=np.int32)
         gap = np.empty(n, dtype=np.float64)
@@ -241,7 +249,7 @@ class OracleCache:
         tgap = np.empty(n, dtype=np.float64)
         h = None if hint is None else np.ascontiguousarray(hint, dtype=np.int32)
         rc = _load().h2o_oracle_decode_step(
-            n, st.d, st.cap, _p(st.kbud, ctypes.c_int32), _p(st.rwin, ctypes.c_int32), _p(st.t, ctypes.c_int32),
+            n, st.group, st.d, st.cap, _p(st.kbud, ctypes.c_int32), _p(st.rwin, ctypes.c_int32), _p(st.t, ctypes.c_int32),
             _p(st.cnt, ctypes.c_int32), _p(st.pos, ctypes.c_int32), _p(st.acc, ctypes.c_double), _p(st.K, ctypes.c_double),
             _p(st.V, ctypes.c_double), _p(qf, ctypes.c_float), _p(kf, ctypes.c_float), _p(vf, ctypes.c_float), st.scale,
             _p(h, ctypes.c_int32), float(tie_rel), _p(out, ctypes.c_double), _p(evicted, ctypes.c_int32),
@@ -258,7 +266,7 @@ class OracleCache:
             pass
 
         st = _S()
-        st.d, st.cap, st.scale = self.d, self.cap, self.scale
+        st.d, st.cap, st.scale, st.group = self.d, self.cap, self.scale, self.group
         for name in ("kbud", "rwin", "t", "cnt", "pos", "acc", "K", "V"):
             setattr(st, name, np.ascontiguousarray(getattr(self, name)[idx]))
         res = self._decode(st, np.ascontiguousarray(qf[idx]), np.ascontiguousarray(kf[idx]), np.ascontiguousarray(vf[idx]),

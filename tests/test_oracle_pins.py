@@ -803,3 +803,85 @@ def test_topk_tie_keeps_the_higher_position_and_reports_the_gap(oracle, topk):
     p = res["p"][0, :4]
     assert p[0] == 0.0 and p[3] == 0.0 and p[1] == pytest.approx(0.5) and p[2] == pytest.approx(0.5)
     assert res["topk_gap"][0] == 0.0  # weakest kept and strongest dropped logit are equal
+
+
+# --------------------------------------------------------------------------
+# grouped-query attention: several query heads share one unit's keys and values; scores add up over the group
+# --------------------------------------------------------------------------
+def test_group_of_identical_queries_is_one_head_with_scaled_scores(oracle):
+    n, steps, d, k, r, scale, G = 30, 25, 8, 4, 5, 0.5, 3
+    rng = np.random.default_rng(810)
+    q, kk, v = _rand_qkv(rng, n + steps, d)
+    one = oracle.OracleCache(1, 1, d, [k], [r], scale=scale)
+    grp = oracle.OracleCache(1, 1, d, [k], [r], scale=scale, group=G)
+    qg = np.repeat(q[:, None, :], G, axis=1)  # [tokens, G, d]: the same query in every head of the group
+    o1, kept1 = one.prefill(_as_thd(q[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    og, keptg = grp.prefill(np.ascontiguousarray(qg[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    np.testing.assert_array_equal(kept1[0], keptg[0])
+    for g in range(G):
+        np.testing.assert_array_equal(og[:, g], o1[:, 0])
+    for t in range(n, n + steps):
+        r1 = one.decode_step(q[t][None, None], kk[t][None, None], v[t][None, None])
+        rg = grp.decode_step(qg[t][None], kk[t][None, None], v[t][None, None])
+        assert r1["evicted"][0] == rg["evicted"][0]
+        for g in range(G):
+            np.testing.assert_array_equal(rg["out"][0, g * d:(g + 1) * d], r1["out"][0])
+    np.testing.assert_array_equal(one.export(0)[0], grp.export(0)[0])
+    np.testing.assert_allclose(grp.export(0)[1], G * one.export(0)[1], rtol=1e-14)
+
+
+def test_group_with_a_cache_that_never_evicts_is_textbook_attention_per_query_head(oracle):
+    n, steps, d, scale, G = 24, 10, 8, 0.4, 4
+    rng = np.random.default_rng(811)
+    kk = rng.standard_normal((n + steps, d)).astype(np.float32)
+    v = rng.standard_normal((n + steps, d)).astype(np.float32)
+    qs = rng.standard_normal((n + steps, G, d)).astype(np.float32)
+    refs = [_textbook_causal(qs[:, g], kk, v, scale) for g in range(G)]
+    cache = oracle.OracleCache(1, 1, d, [n + steps], [3], scale=scale, group=G)
+    out, kept = cache.prefill(np.ascontiguousarray(qs[:n]), _as_thd(kk[:n]), _as_thd(v[:n]), [0, n])
+    for g in range(G):
+        np.testing.assert_allclose(out[:, g], refs[g][0][:n], rtol=1e-11, atol=1e-13)
+    for t in range(n, n + steps):
+        res = cache.decode_step(qs[t][None], kk[t][None, None], v[t][None, None])
+        for g in range(G):
+            np.testing.assert_allclose(res["out"][0, g * d:(g + 1) * d], refs[g][0][t], rtol=1e-11, atol=1e-13)
+    pos, acc = cache.export(0)
+    assert pos.tolist() == list(range(n + steps))
+    np.testing.assert_allclose(acc, sum(p.sum(axis=0) for _, p in refs), rtol=1e-12)  # column sums add up over the group
+
+
+@pytest.mark.parametrize("k,r,G", [(3, 3, 2), (2, 4, 3), (4, 0, 2)])
+def test_group_policy_matches_the_literal_simulation(oracle, k, r, G):
+    """One simulation step per query head over the same kept set (the rows of all heads enter the explicit column
+    sums), the eviction after the group's last head."""
+    T, d, scale = 20, 4, 0.6
+    rng = np.random.default_rng(820 + 10 * k + r + G)
+    kk = rng.standard_normal((T, d)).astype(np.float32)
+    v = rng.standard_normal((T, d)).astype(np.float32)
+    qs = (rng.standard_normal((T, G, d)) + 0.7).astype(np.float32)
+    lit = LiteralH2O(k, r, scale, lambda z: z)
+    cache = oracle.OracleCache(1, 1, d, [k], [r], scale=scale, group=G)
+    decided = 0
+    for t in range(T):
+        # literal: the first G - 1 heads attend without evicting (their rows are recorded), the last one evicts
+        kept_before = list(lit.S)
+        outs = []
+        for g in range(G):
+            lit.S, lit.t = list(kept_before), t
+            budget = lit.k
+            if g < G - 1:
+                lit.k = 10 ** 6  # no eviction for this head
+            out_l, ev_l, probs, gap = lit.step(qs[t, g], kk[t], v[t])
+            lit.k = budget
+            outs.append(out_l)
+        res = cache.decode_step(qs[t][None], kk[t][None, None], v[t][None, None])
+        for g in range(G):
+            np.testing.assert_allclose(res["out"][0, g * d:(g + 1) * d], outs[g], rtol=1e-11, atol=1e-13)
+        if 0.0 < gap <= 1e-9:
+            break
+        assert res["evicted"][0] == ev_l
+        decided += 1
+        pos, acc = cache.export(0)
+        assert set(pos.tolist()) == set(lit.S)
+        np.testing.assert_allclose(acc, [lit.column_sum(j) for j in pos], rtol=1e-12, atol=1e-300)
+    assert decided >= 8
