@@ -74,7 +74,20 @@ typedef struct {
   const int32_t* recent_window; /* host [batch]: r_s >= 0, k_s + r_s >= 1                      */
   float softmax_scale;          /* c in exp(c q.k); <= 0 selects 1/sqrt(head_dim)              */
   int32_t device;               /* CUDA device ordinal                                         */
+  int32_t query_group;          /* grouped-query attention: query heads per (K/V) head: 0 or 1 (none), 2, 4 or 8 */
 } h2o_config_t;
+
+/*
+ * Grouped-query attention (query_group = G > 1; no counterpart in the paper, which evicts per head; its comparison
+ * with a method that accumulates scores across heads is the nearest text).  n_heads counts the K/V heads: a unit is
+ * one (sequence, K/V head) and its G query heads share its cache.  q and out then have n_heads * G heads, query
+ * head = head * G + g ([..., n_heads * G, head_dim]); k, v, k_new, v_new and evicted_pos keep n_heads.  Every query
+ * head attends the unit's entries with its own softmax, and a key's accumulated score grows by the SUM of the
+ * probabilities the group's heads gave it; selection after the prompt and eviction use that sum.  Each K and V row
+ * is read once for the whole group.  Supported: f32 / bf16 slots, budgets with G * (k_s + r_s + 1) * 4 bytes up to
+ * about 160 KB; the prompt runs on the fp32-FMA kernels; sparse patterns, "Top-K" attention, 4-bit slots and the
+ * host-buffer calls are not combined with it (H2O_ERR_UNSUPPORTED).
+ */
 
 /* Bytes of device workspace h2o_cache_create needs for this configuration
  * (K/V slots, accumulated scores, positions, counters).  Pure host arithmetic.

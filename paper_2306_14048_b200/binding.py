@@ -61,6 +61,7 @@ class h2o_config_t(ctypes.Structure):
         ("recent_window", ctypes.POINTER(ctypes.c_int32)),
         ("softmax_scale", ctypes.c_float),
         ("device", ctypes.c_int32),
+        ("query_group", ctypes.c_int32),
     ]
 
 
@@ -147,13 +148,15 @@ def _check(code: int, where: str):
         raise H2OError(code, where)
 
 
-def make_config(batch, n_heads, head_dim, dtype, heavy: Sequence[int], recent: Sequence[int], softmax_scale=0.0, device=0):
+def make_config(batch, n_heads, head_dim, dtype, heavy: Sequence[int], recent: Sequence[int], softmax_scale=0.0, device=0,
+                query_group=1):
     """Returns (h2o_config_t, keepalive) — the budget arrays must outlive the struct."""
     hv = (ctypes.c_int32 * len(heavy))(*[int(x) for x in heavy])
     rc = (ctypes.c_int32 * len(recent))(*[int(x) for x in recent])
     code = {torch.float32: H2O_F32, torch.bfloat16: H2O_BF16, "f32": H2O_F32, "bf16": H2O_BF16,
             "bf16_kv4": H2O_BF16_KV4}.get(dtype, dtype)
-    cfg = h2o_config_t(int(batch), int(n_heads), int(head_dim), int(code), hv, rc, float(softmax_scale), int(device))
+    cfg = h2o_config_t(int(batch), int(n_heads), int(head_dim), int(code), hv, rc, float(softmax_scale), int(device),
+                       int(query_group))
     return cfg, (hv, rc)
 
 
@@ -179,9 +182,12 @@ class H2OCache:
     ``status`` -> h2o_cache_status, ``close`` -> h2o_cache_destroy.
     """
 
-    def __init__(self, batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale=0.0, device=0, snapshot=None):
-        """``snapshot``: bytes of another handle's workspace (``snapshot()``) to resume from (h2o_cache_attach)."""
-        self.cfg, self._keep = make_config(batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale, device)
+    def __init__(self, batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale=0.0, device=0, snapshot=None,
+                 query_group=1):
+        """``snapshot``: bytes of another handle's workspace (``snapshot()``) to resume from (h2o_cache_attach).
+        ``query_group`` > 1: grouped-query attention, q / out carry n_heads * query_group heads."""
+        self.cfg, self._keep = make_config(batch, n_heads, head_dim, dtype, heavy, recent, softmax_scale, device,
+                                           query_group)
         self.batch, self.n_heads, self.head_dim = int(batch), int(n_heads), int(head_dim)
         self.units = self.batch * self.n_heads
         self.max_B = int(max(int(a) + int(b) for a, b in zip(heavy, recent)))

@@ -51,8 +51,18 @@ int check_config(const h2o_config_t* cfg) {
     if (cfg->dtype == H2O_BF16_KV4 && k + r > kMaxSlotsPerUnitKv4) return H2O_ERR_UNSUPPORTED;
   }
   if (std::isnan(cfg->softmax_scale) || std::isinf(cfg->softmax_scale)) return H2O_ERR_INVALID_ARG;
+  const int G = cfg->query_group;
+  if (G < 0) return H2O_ERR_INVALID_ARG;
+  if (G > 1) {  // grouped-query attention
+    if (G != 2 && G != 4 && G != 8) return H2O_ERR_UNSUPPORTED;
+    if (cfg->dtype == H2O_BF16_KV4) return H2O_ERR_UNSUPPORTED;
+    for (int s = 0; s < cfg->batch; ++s)  // the group's scores of one unit stay in shared memory
+      if (h2o::decode_gqa_smem_bytes(G, cfg->heavy_budget[s] + cfg->recent_window[s], cfg->head_dim) > 200 * 1024)
+        return H2O_ERR_UNSUPPORTED;
+  }
   return H2O_OK;
 }
+int group_of(const h2o_config_t* cfg) { return cfg->query_group > 1 ? cfg->query_group : 1; }
 
 Layout make_layout(const h2o_config_t* cfg) {
   Layout L{};
@@ -99,7 +109,7 @@ ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens)
     off = align_up(off + bytes);
     return at;
   };
-  S.rowstat = take(cells * 2 * sizeof(float));  // row maximum and row sum (planar or interleaved)
+  S.rowstat = take(cells * group_of(cfg) * 2 * sizeof(float));  // row maximum and row sum per QUERY head (planar or interleaved)
   S.acc0 = take(cells * sizeof(double));
   // cu_seqlens, two work counters, first item index of every group of units (at most one group per unit)
   S.cu = take(((size_t)cfg->batch + 1 + 2 + (size_t)cfg->batch * cfg->n_heads + 1) * sizeof(int32_t));
@@ -310,6 +320,7 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   v.topk = 0;
   v.seq_rwin = reinterpret_cast<const int32_t*>(ws + L.seq_rwin);
   v.total_slots = L.total_slots;
+  v.group = group_of(cfg);
   c->seen.assign(cfg->batch, attach ? -1 : 0);
 
   bool ok = true;
@@ -375,7 +386,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   char* sc = static_cast<char*>(scratch);
   h2o::PrefillScratch ps;
   ps.rowmax = reinterpret_cast<float*>(sc + S.rowstat);
-  ps.rowsum = ps.rowmax + (size_t)total * cfg.n_heads;
+  ps.rowsum = ps.rowmax + (size_t)total * cfg.n_heads * cache->view.group;
   ps.rowstat = reinterpret_cast<float2*>(sc + S.rowstat);
   ps.acc0 = reinterpret_cast<double*>(sc + S.acc0);
   ps.cu = reinterpret_cast<int32_t*>(sc + S.cu);
@@ -412,7 +423,8 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   // bf16 / head_dim 128 runs on the tensor cores; every other combination on the fp32 FMA pipe
   const int in_dtype = input_dtype(cfg.dtype);
   // (a sparse pattern is applied by the fp32-FMA kernels only)
-  const bool tc = cache->prefill_path != 1 && cache->view.mask_kind == 0 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
+  const bool tc = cache->prefill_path != 1 && cache->view.mask_kind == 0 && cache->view.group == 1 &&
+                  h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
   cudaError_t e = cudaSuccess;
   // optional phase events of this one call (diagnostic): before the forward kernel, after it, after the column
   // sums, after selection and gather
@@ -463,7 +475,10 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   // the cache workspace is the identity: two handles on one workspace must count as the same cache
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
   const cudaError_t e =
-      cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, q, k_new, v_new, out, evicted_pos,
+      cache->view.group > 1
+          ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, q, k_new, v_new, out, evicted_pos,
+                                   static_cast<cudaStream_t>(stream))
+      : cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, q, k_new, v_new, out, evicted_pos,
                                                static_cast<cudaStream_t>(stream))
                       : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, quiescent,
                                            all_units_full(cache), q, k_new, v_new, out, evicted_pos,
@@ -490,17 +505,22 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
   cudaError_t e = cudaSuccess;
   // (the chunk kernel ranks by the accumulated score only)
   if (cache->chunk_path == 0 && cache->view.score_mode == 0 && cache->view.mask_kind == 0 && cache->view.topk == 0 &&
-      !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
+      cache->view.group == 1 && !cache->view.kv4 && h2o::decode_chunk_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->layout.max_B,
                                                           cache->layout.total_slots)) {
     e = h2o::launch_decode_chunk(cache->view, cache->layout.total_slots, cache->meta.data(), q, k, v, n_tokens, out,
                                  evicted_pos, st);
     if (e == cudaSuccess) advance_seen(cache, n_tokens);
   } else {
     const size_t step = (size_t)cache->view.units * cache->cfg.head_dim * elem_size(cache->cfg.dtype);
+    const size_t qstep = step * cache->view.group;  // q and out carry the group's query heads
     for (int32_t i = 0; i < n_tokens && e == cudaSuccess; ++i) {
       const size_t off = (size_t)i * step;
       int32_t* ev_i = evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr;
-      e = cache->view.kv4
+      e = cache->view.group > 1
+              ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, static_cast<const char*>(q) + i * qstep,
+                                       static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
+                                       static_cast<char*>(out) + i * qstep, ev_i, st)
+          : cache->view.kv4
               ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, static_cast<const char*>(q) + off,
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
                                        static_cast<char*>(out) + off, ev_i, st)
@@ -531,7 +551,7 @@ int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b) {
   if (!cache || kind < 0 || kind > 2) return H2O_ERR_INVALID_ARG;
   if (kind != 0 && (a < 1 || b < 0 || (kind == 2 && b > a))) return H2O_ERR_INVALID_ARG;
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one attention rule per generation
-  if (kind != 0 && cache->view.kv4) return H2O_ERR_UNSUPPORTED;
+  if (kind != 0 && (cache->view.kv4 || cache->view.group > 1)) return H2O_ERR_UNSUPPORTED;
   cache->view.mask_kind = kind;
   cache->view.mask_a = kind ? a : 1;
   cache->view.mask_b = kind ? b : 0;
@@ -542,7 +562,7 @@ int h2o_cache_set_topk(h2o_cache_t* cache, int32_t m) {
   if (!cache || m < 0) return H2O_ERR_INVALID_ARG;
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one attention rule per generation
   if (m > 0) {
-    if (cache->view.kv4) return H2O_ERR_UNSUPPORTED;
+    if (cache->view.kv4 || cache->view.group > 1) return H2O_ERR_UNSUPPORTED;
     const int chunk = (cache->layout.max_B + 3) & ~3;  // one thread block per unit: the selection runs over its scores
     if (chunk > kMaxChunk) return H2O_ERR_UNSUPPORTED;
     cache->split = 1;
@@ -579,6 +599,7 @@ int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* 
                             const int32_t* cu_seqlens, void* out_host, void* staging, size_t staging_bytes,
                             void* scratch, size_t scratch_bytes, void* stream) {
   if (!cache || !q_host || !k_host || !v_host || !cu_seqlens || !out_host || !staging) return H2O_ERR_INVALID_ARG;
+  if (cache->view.group > 1) return H2O_ERR_UNSUPPORTED;  // (q / out and k / v differ in size there)
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;
   const h2o_config_t& cfg = cache->cfg;
   const int64_t total = cu_seqlens[cfg.batch];
@@ -611,6 +632,7 @@ int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* 
 int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_new_host, const void* v_new_host,
                          void* out_host, int32_t* evicted_pos_host, void* staging, size_t staging_bytes, void* stream) {
   if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !staging) return H2O_ERR_INVALID_ARG;
+  if (cache->view.group > 1) return H2O_ERR_UNSUPPORTED;
   const h2o_config_t& cfg = cache->cfg;
   if (staging_bytes < h2o_host_staging_bytes(&cfg, cfg.batch) || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0)
     return H2O_ERR_WORKSPACE;

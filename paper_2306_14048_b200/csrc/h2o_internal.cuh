@@ -52,6 +52,7 @@ struct CacheView {
   int32_t topk;
   const int32_t* seq_rwin;  // [batch] recent window of every sequence (the prompt kernels index by unit, not by launch position)
   int64_t total_slots;      // slots of all units together (the limit of every slot index)
+  int32_t group;            // query heads per unit (grouped-query attention); 1: every head has its own cache
 };
 
 // Debug build (-DH2O_BOUNDS, the stand-in for a memory checker): every slot, unit and prompt-row index that
@@ -79,7 +80,7 @@ __device__ __forceinline__ bool key_attended(int kind, int a, int b, int p, int 
 }
 
 // Scratch of one prefill call; per-head planes so that a unit's rows are contiguous:
-// index = h * total_tokens + token.
+// index = h * total_tokens + token (row statistics: h = QUERY head, n_heads * group planes; column sums: K/V head).
 struct PrefillScratch {
   float* rowmax;   // m_i
   float* rowsum;   // l_i
@@ -132,6 +133,10 @@ inline int sm_count() {
 cudaError_t launch_decode(const CacheView& c, int dtype, int split, int chunk, int stages, bool quiescent, bool all_full,
                           const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                           cudaStream_t stream);
+// Grouped-query attention (c.group query heads per unit): one block per unit, K and V rows read once for the group.
+size_t decode_gqa_smem_bytes(int group, int max_B, int head_dim);
+cudaError_t launch_decode_gqa(const CacheView& c, int dtype, int max_B, const void* q, const void* k_new, const void* v_new,
+                              void* out, int32_t* evicted_pos, cudaStream_t stream);
 // ALU path; `rows` = attention rows + row statistics, `colsum` = column sums.
 cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int max_seqlen, const void* q,
                                  const void* k, const void* v, void* out, bool rows, bool colsum, cudaStream_t stream);

@@ -24,22 +24,25 @@ prefill_rows_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, cons
   constexpr int VEC = A::VEC, LPR = A::LPR;
   extern __shared__ float p[];
   __shared__ typename A::Smem sm;
-  const int u = blockIdx.y;
-  const int seq = u / c.n_heads, h = u % c.n_heads;
+  // blockIdx.y = (sequence, QUERY head); with grouped-query attention the query heads hq = h * G + g of a group
+  // read the keys and values of head h
+  const int G = c.group, HQ = c.n_heads * G;
+  const int uq = blockIdx.y;
+  const int seq = uq / HQ, hq = uq % HQ, h = hq / G;
   const int lo = s.cu[seq], n = s.cu[seq + 1] - lo;
   const int i = blockIdx.x;
   if (i >= n) return;
-  if (!H2O_IN_RANGE(u, c.units, c.status) || !H2O_IN_RANGE((int64_t)lo + i, s.total_tokens, c.status)) return;
-  const int64_t stride = (int64_t)c.n_heads * D;
-  const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
+  if (!H2O_IN_RANGE(seq * c.n_heads + h, c.units, c.status) || !H2O_IN_RANGE((int64_t)lo + i, s.total_tokens, c.status)) return;
+  const int64_t stride = (int64_t)c.n_heads * D, stride_q = (int64_t)HQ * D;
+  const int64_t base = ((int64_t)lo * c.n_heads + h) * D, base_q = ((int64_t)lo * HQ + hq) * D;
   float o[VEC], m, l;
   const int r = c.mask_kind ? c.seq_rwin[seq] : 0;
-  A::run(q + base + i * stride, k + base, v + base, stride, i + 1, nullptr, nullptr, c.scale, p, sm, o, m, l, c.mask_kind,
+  A::run(q + base_q + i * stride_q, k + base, v + base, stride, i + 1, nullptr, nullptr, c.scale, p, sm, o, m, l, c.mask_kind,
          c.mask_a, c.mask_b, i, r);
-  if (threadIdx.x < LPR) Vec16<T>::store(out + base + i * stride + threadIdx.x * VEC, o);
+  if (threadIdx.x < LPR) Vec16<T>::store(out + base_q + i * stride_q + threadIdx.x * VEC, o);
   if (threadIdx.x == 0) {
-    s.rowmax[(int64_t)h * s.total_tokens + lo + i] = m;
-    s.rowsum[(int64_t)h * s.total_tokens + lo + i] = l;
+    s.rowmax[(int64_t)hq * s.total_tokens + lo + i] = m;
+    s.rowsum[(int64_t)hq * s.total_tokens + lo + i] = l;
   }
 }
 
@@ -53,10 +56,9 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
   const int j0 = blockIdx.x * kColThreads;
   if (j0 >= n) return;
   const int j = j0 + threadIdx.x;
-  const int64_t stride = (int64_t)c.n_heads * D;
+  const int G = c.group, HQ = c.n_heads * G;
+  const int64_t stride = (int64_t)c.n_heads * D, stride_q = (int64_t)HQ * D;
   const int64_t base = ((int64_t)lo * c.n_heads + h) * D;
-  const float* rowmax = s.rowmax + (int64_t)h * s.total_tokens + lo;
-  const float* rowsum = s.rowsum + (int64_t)h * s.total_tokens + lo;
 
   float kf[D];
   if (j < n) {
@@ -73,18 +75,23 @@ prefill_colsum_kernel(CacheView c, PrefillScratch s, const T* __restrict__ q, co
   }
   const int r = c.mask_kind ? c.seq_rwin[seq] : 0;
   double a = 0.0;
-  for (int i = j0; i < n; ++i) {  // every thread of the block reads the same query row (broadcast)
-    const T* qi = q + base + i * stride;
-    float dot = 0.f;
+  for (int g = 0; g < G; ++g) {  // the group's query heads one after the other: their column sums add up
+    const int hq = h * G + g;
+    const float* rowmax = s.rowmax + (int64_t)hq * s.total_tokens + lo;
+    const float* rowsum = s.rowsum + (int64_t)hq * s.total_tokens + lo;
+    for (int i = j0; i < n; ++i) {  // every thread of the block reads the same query row (broadcast)
+      const T* qi = q + ((int64_t)lo * HQ + hq) * D + i * stride_q;
+      float dot = 0.f;
 #pragma unroll
-    for (int x = 0; x < D; x += VEC) {
-      float t[VEC];
-      Vec16<T>::load(qi + x, t);
+      for (int x = 0; x < D; x += VEC) {
+        float t[VEC];
+        Vec16<T>::load(qi + x, t);
 #pragma unroll
-      for (int e = 0; e < VEC; ++e) dot = fmaf(t[e], kf[x + e], dot);
+        for (int e = 0; e < VEC; ++e) dot = fmaf(t[e], kf[x + e], dot);
+      }
+      if (i >= j && key_attended(c.mask_kind, c.mask_a, c.mask_b, j, i, r))
+        a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
     }
-    if (i >= j && key_attended(c.mask_kind, c.mask_a, c.mask_b, j, i, r))
-      a += (double)(expf(c.scale * dot - rowmax[i]) / rowsum[i]);
   }
   if (j < n && H2O_IN_RANGE((int64_t)lo + j, s.total_tokens, c.status)) s.acc0[(int64_t)h * s.total_tokens + lo + j] = a;
 }
@@ -99,7 +106,7 @@ cudaError_t launch(const CacheView& c, const PrefillScratch& s, int max_seqlen, 
           cudaFuncSetAttribute(prefill_rows_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return e;
     }
-    dim3 grid_rows((unsigned)max_seqlen, (unsigned)c.units);
+    dim3 grid_rows((unsigned)max_seqlen, (unsigned)(c.units * c.group));  // one block per query row of every query head
     prefill_rows_kernel<T, D><<<grid_rows, kRowThreads, smem, stream>>>(
         c, s, static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(out));
     cudaError_t e = cudaGetLastError();

@@ -81,14 +81,15 @@ def compare_state(gpu_cache, ora, units, dtype, stats: ParityStats, where: str, 
         stats.max_acc_err = max(stats.max_acc_err, assert_close(acc[u, :m][order], oacc, dtype, "%s unit %d acc" % (where, u)))
 
 
-def _gather_units(x, cu, units, H):
-    """Rows of the sampled units, packed as [sum n_u, 1, d] float32 on the host, plus their cu_seqlens."""
+def _gather_units(x, cu, units, H, G=1):
+    """Rows of the sampled units, packed as [sum n_u, G, d] float32 on the host (G = 1 for keys and values; the
+    query heads of a unit's group are heads h * G .. h * G + G - 1), plus their cu_seqlens."""
     parts, lens = [], []
     for u in units:
         s, h = divmod(u, H)
-        parts.append(x[int(cu[s]):int(cu[s + 1]), h])
+        parts.append(x[int(cu[s]):int(cu[s + 1]), h * G:(h + 1) * G])
         lens.append(int(cu[s + 1] - cu[s]))
-    packed = torch.cat(parts, dim=0).float().cpu().numpy()[:, None, :]
+    packed = torch.cat(parts, dim=0).float().cpu().numpy()
     return np.ascontiguousarray(packed), np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
 
 
@@ -96,7 +97,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
                device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
                pattern: Optional[Sequence[int]] = None, score_mode: int = 0, static_scratch: bool = False,
-               mask: Optional[Sequence[int]] = None, split: int = 0, topk: int = 0) -> ParityStats:
+               mask: Optional[Sequence[int]] = None, split: int = 0, topk: int = 0, group: int = 1) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
@@ -105,6 +106,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
     sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
     ``split``: thread blocks (one cluster) per unit in the decode kernel, 0 = the library's choice.
+    ``group`` > 1: grouped-query attention: wl.n_heads counts the K/V heads, q and out carry n_heads * group query heads
+    (drawn from the same recipe with that many heads).
     ``topk`` > 0: "Top-K" attention in decode steps on both sides (h2o_cache_set_topk); a unit whose weakest kept and
     strongest dropped logit come closer than TOPK_TIE_REL is counted and left out of every later comparison.
     ``mask`` = (kind, a, b): sparse pattern inside the recent window (h2o_cache_set_mask) on both sides.
@@ -114,7 +117,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         h2o_oracle.set_topk(topk)
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
-                              chunk, chunk_path, pattern, score_mode, static_scratch, mask, split, topk=-topk)
+                              chunk, chunk_path, pattern, score_mode, static_scratch, mask, split, topk=-topk, group=group)
         finally:
             h2o_oracle.set_topk(0)
     topk = -topk  # (negative: the oracle already has it)
@@ -125,7 +128,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
                               chunk, chunk_path, pattern, score_mode, static_scratch, mask=(0,) + tuple(mask), split=split,
-                              topk=-topk)
+                              topk=-topk, group=group)
         finally:
             h2o_oracle.set_mask(0)
     if score_mode > 0:  # the oracle's ranking rule is process-wide: always put it back
@@ -133,7 +136,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
                               chunk, chunk_path, pattern, score_mode=0 - score_mode, static_scratch=static_scratch, mask=mask,
-                              split=split, topk=-topk)
+                              split=split, topk=-topk, group=group)
         finally:
             h2o_oracle.set_score_mode(0)
     score_mode = -score_mode  # (negative: the oracle is already in that mode)
@@ -144,7 +147,10 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     steps = wl.decode_steps if steps is None else steps
     # the C ABI takes the softmax scale as a float: both sides get that same fp32 value
     scale = float(np.float32(scale if scale > 0 else 1.0 / np.sqrt(float(d))))
-    gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
+    G = int(group)
+    wl_q = wl.scaled(n_heads=H * G) if G > 1 else wl  # the query side has H * G heads
+    gpu = gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0, query_group=G) \
+        if G > 1 else gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
     gpu.set_prefill_path(prefill_path)
     gpu.set_decode_shape(split, 0)
     if topk > 0:
@@ -153,25 +159,27 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     if mask is not None:  # (0, kind, a, b): the oracle already has it
         gpu.set_mask(*mask[1:])
     ora = h2o_oracle.OracleCache(len(units), 1, d, [wl.heavy[u // H] for u in units], [wl.recent[u // H] for u in units],
-                                 scale=scale, kv4=(wl.dtype == "bf16_kv4"))
+                                 scale=scale, kv4=(wl.dtype == "bf16_kv4"), group=G)
     uidx = torch.as_tensor(units, dtype=torch.long, device=device)
     if prefill:
         q, k, v, cu = make_prompt_inputs(wl, layer=layer, device=device)
+        if G > 1:
+            q = make_prompt_inputs(wl_q, layer=layer, device=device)[0]
         out = torch.empty_like(q)
         if static_scratch:  # the entry point that takes no scratch buffer
             gpu.prefill_select_static(q, k, v, cu, out)
         else:
             gpu.prefill_select(q, k, v, cu, out)
         assert gpu.status() == 0
-        qh, ocu = _gather_units(q, cu, units, H)
+        qh, ocu = _gather_units(q, cu, units, H, G)
         kh, _ = _gather_units(k, cu, units, H)
         vh, _ = _gather_units(v, cu, units, H)
-        out_h, _ = _gather_units(out, cu, units, H)
+        out_h, _ = _gather_units(out, cu, units, H, G)
         o_out, o_kept = ora.prefill(qh, kh, vh, ocu)
         pos, acc, count, t = gpu.export()
         for x, u in enumerate(units):
             lo, hi = int(ocu[x]), int(ocu[x + 1])
-            stats.max_out_err = max(stats.max_out_err, assert_close(out_h[lo:hi, 0], o_out[lo:hi, 0], wl.dtype,
+            stats.max_out_err = max(stats.max_out_err, assert_close(out_h[lo:hi], o_out[lo:hi], wl.dtype,
                                                                     "prefill out unit %d" % u))
             m = int(count[u])
             gkept = np.sort(pos[u, :m])
@@ -191,8 +199,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         del q, k, v, out, qh, kh, vh, out_h
     ev = torch.empty(wl.batch, H, dtype=torch.int32, device=device)
 
-    def pick(x):  # [batch, H, d] -> the sampled units as [len(units), 1, d] float32 on the host
-        return x.reshape(wl.units, d)[uidx].float().cpu().numpy()[:, None, :]
+    def pick(x, g=1):  # [batch, H * g, d] -> the sampled units as [len(units), g, d] float32 on the host
+        return x.reshape(wl.units, g, d)[uidx].float().cpu().numpy()
 
     dead = set()  # oracle units left out after a "Top-K" toss-up
     step, call = 0, 0
@@ -202,6 +210,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
             call += 1
         nt = min(chunk, steps - step) if chunk > 0 else 1
         qs, ks, vs = zip(*[make_decode_inputs(wl, step + i, layer=layer, device=device) for i in range(nt)])
+        if G > 1:
+            qs = tuple(make_decode_inputs(wl_q, step + i, layer=layer, device=device)[0] for i in range(nt))
         if chunk > 0:
             q, k, v = (torch.stack(x).contiguous() for x in (qs, ks, vs))  # [nt, batch, H, d]
             out = torch.empty_like(q)
@@ -215,8 +225,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
             evs = ev[None]
         for i in range(nt):
             g_ev = evs[i].reshape(-1)[uidx].cpu().numpy()
-            g_out = out[i].reshape(wl.units, d)[uidx].float().cpu().numpy()
-            res = ora.decode_step(pick(qs[i]), pick(ks[i]), pick(vs[i]), hint=g_ev, tie_rel=TIE_REL)
+            g_out = out[i].reshape(wl.units, G * d)[uidx].float().cpu().numpy()
+            res = ora.decode_step(pick(qs[i], G), pick(ks[i]), pick(vs[i]), hint=g_ev, tie_rel=TIE_REL)
             if topk > 0:
                 for x in range(len(units)):
                     if x not in dead and res["topk_gap"][x] < TOPK_TIE_REL:

@@ -464,3 +464,56 @@ def test_topk_argument_and_state_errors(H2OCache):
     big = H2OCache(1, 1, 64, "f32", [6000], [6000])
     assert pkg.lib.h2o_cache_set_topk(big._h, 2) == pkg.H2O_ERR_UNSUPPORTED
     big.close()
+
+
+# ---------------------------------------------------------------------------------------------------------
+# grouped-query attention: G query heads share a unit's keys and values, accumulated scores add up over the group
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("group,dtype,d", [
+    (2, "bf16", 128), (4, "bf16", 128), (8, "bf16", 128), (2, "f32", 64), (4, "f32", 64), (8, "f32", 64),
+    (2, "bf16", 64), (4, "bf16", 64), (2, "f32", 128), (4, "f32", 128),
+])
+def test_grouped_query_attention_ragged(H2OCache, group, dtype, d):
+    """Prompt (fp32-FMA kernels), selection on the summed column sums, decode steps with one victim per unit."""
+    from parity_harness import run_parity
+
+    wl = _wl("gqa", 3, 2, d, dtype, [300, 77, 140], 40, [20, 9, 33], [24, 5, 31], seed=377 + d + group)
+    st = run_parity(wl, H2OCache, export_every=8, group=group)
+    print(st)
+
+
+@pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([6, 1], [12, 9])])
+def test_grouped_query_attention_edge_budgets_token_by_token(H2OCache, heavy, recent):
+    from parity_harness import run_parity
+
+    wl = _wl("gqaedge", 2, 2, 64, "f32", [1, 1], 60, heavy, recent, seed=35)
+    st = run_parity(wl, H2OCache, prefill=False, export_every=5, group=4)
+    print(st)
+
+
+def test_grouped_query_attention_long_budget_chunk_call_and_averaged_score(H2OCache):
+    from parity_harness import run_parity
+
+    wl = _wl("gqalong", 2, 2, 128, "bf16", [1500, 1300], 16, [600, 500], [500, 600], seed=331)
+    print(run_parity(wl, H2OCache, export_every=8, group=2))
+    wl = _wl("gqachunk", 2, 3, 128, "bf16", [400, 300], 40, [20, 30], [24, 16], seed=332)
+    print(run_parity(wl, H2OCache, export_every=8, group=4, chunk=16))
+    print(run_parity(wl, H2OCache, export_every=8, group=2, score_mode=1))
+
+
+def test_grouped_query_attention_argument_errors(H2OCache):
+    import ctypes
+
+    import paper_2306_14048_b200 as pkg
+
+    for bad in (3, 16, -1):
+        cfg, keep = pkg.make_config(1, 2, 64, "f32", [4], [4], query_group=bad)
+        assert pkg.h2o_cache_workspace_bytes(cfg) == 0
+    cfg, keep = pkg.make_config(1, 2, 128, "bf16_kv4", [4], [4], query_group=2)
+    assert pkg.h2o_cache_workspace_bytes(cfg) == 0
+    cfg, keep = pkg.make_config(1, 1, 64, "f32", [4000], [4000], query_group=8)  # the group's scores would not fit
+    assert pkg.h2o_cache_workspace_bytes(cfg) == 0
+    cache = H2OCache(1, 2, 64, "f32", [4], [4], query_group=2)
+    assert pkg.lib.h2o_cache_set_mask(cache._h, 1, 4, 2) == pkg.H2O_ERR_UNSUPPORTED
+    assert pkg.lib.h2o_cache_set_topk(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
+    cache.close()
