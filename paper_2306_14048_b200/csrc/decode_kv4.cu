@@ -16,8 +16,11 @@
 // The decode step is the same fused step as decode.cu (scores over the occupied slots, softmax, P V,
 // fp64 score accumulation, victim search, in-place write), with the dequantisation folded into the
 // arithmetic: per group  q . x_hat = zero * sum(q) + scale * sum(q_i code_i)  and
-// p * x_hat_i = (p * scale) * code_i + p * zero, so a channel costs one FMA on its code.  The group sums
-// sum(q_i code_i) of the scores come from mma.sync m16n8k16 on the codes as exact bf16 values.
+// sum_rows p * x_hat_i = sum_rows (p * scale) * code_i + sum_rows p * zero.  Both contractions over codes run
+// as mma.sync m16n8k16 on the codes as exact bf16 values (the unpacking, one shift and one logic operation
+// per pair of codes, is what bounds the kernel: the logic pipe, not HBM): the scores with the query as the
+// column operand, one column per group; the values with the codes transposed as the row operand and
+// p * scale, split into a bf16 head and remainder per group, as the column operand.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -36,11 +39,12 @@ using namespace ptx;
 
 constexpr int kD = 128;
 constexpr int kRowBytes = 80;
-constexpr int kMaxWarps = 8;              // consumer warps: 8, or 4 for launches of many units (twice the blocks per SM
-                                          // hide one another's serial start and end); one more warp streams the tiles
+constexpr int kMaxWarps = 16;             // consumer warps: 16 when a block has its SM to itself, 8 for two blocks per
+                                          // SM, 4 for launches of many units (more blocks per SM hide one another's
+                                          // serial start and end); one more warp streams the tiles
 constexpr int kTileRows = 64;             // rows per tile: eight per consumer warp
 constexpr int kTileBytes = kTileRows * kRowBytes;  // 5120
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;             // ring depth: 2, 4 or 8 tiles (K and V) in flight
 constexpr uint32_t kSpin = 1u << 22;
 
 __device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
@@ -54,21 +58,11 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-// The eight codes of a 32-bit word as floats, without integer-to-float conversions.  A nibble at bits
-// 4i .. 4i+3 (i <= 4) of a float's mantissa, under the exponent of 2^(23-4i), reads as 2^(23-4i) + n: one logic
-// operation per code (mask and exponent in one), one subtraction (exact), and for the three top nibbles
-// one shift of the word.  (Packed fp32x2 subtractions and FMAs on pairs were slower: 173 against 158 us
-// on the large ragged workload.)
-__device__ __forceinline__ void codes8(uint32_t w, float (&n)[8]) {
-  const uint32_t h = w >> 12;  // nibbles 5, 6, 7 at bits 8, 12, 16
-  n[0] = __uint_as_float((w & 0x0000000Fu) | 0x4B000000u) - 8388608.0f;
-  n[1] = __uint_as_float((w & 0x000000F0u) | 0x49000000u) - 524288.0f;
-  n[2] = __uint_as_float((w & 0x00000F00u) | 0x47000000u) - 32768.0f;
-  n[3] = __uint_as_float((w & 0x0000F000u) | 0x45000000u) - 2048.0f;
-  n[4] = __uint_as_float((w & 0x000F0000u) | 0x43000000u) - 128.0f;
-  n[5] = __uint_as_float((h & 0x00000F00u) | 0x47000000u) - 32768.0f;
-  n[6] = __uint_as_float((h & 0x0000F000u) | 0x45000000u) - 2048.0f;
-  n[7] = __uint_as_float((h & 0x000F0000u) | 0x43000000u) - 128.0f;
+// (a & b) | c in one logic instruction
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
 }
 // The eight codes of a 32-bit word as four pairs of exact bf16 values, r[k] = (code k, code k + 4): a nibble in
 // the low mantissa bits of 128.0 reads as 128 + code; the subtraction is exact.
@@ -76,7 +70,7 @@ __device__ __forceinline__ void codes_bf16x2(uint32_t w, uint32_t (&r)[4]) {
   const __nv_bfloat162 c128 = __floats2bfloat162_rn(128.f, 128.f);
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
-    uint32_t x = ((w >> (4 * k)) & 0x000F000Fu) | 0x43004300u;
+    uint32_t x = and_or(w >> (4 * k), 0x000F000Fu, 0x43004300u);
     __nv_bfloat162 v = __hsub2(*reinterpret_cast<__nv_bfloat162*>(&x), c128);
     r[k] = *reinterpret_cast<uint32_t*>(&v);
   }
@@ -145,8 +139,22 @@ __device__ __forceinline__ void quantise_group(const __nv_bfloat16* src, uint4& 
   meta = (__float_as_uint(scale) >> 16) | (__float_as_uint(mn) & 0xffff0000u);
 }
 
+#ifdef H2O_PHASE_TIMERS
+__device__ long long g_kvt[512 * 2 * 16];
+#define KV_STAMP(i)                                                                              \
+  do {                                                                                           \
+    if (lane == 0 && (warp == 0 || warp == 4) && blockIdx.x < 512 && (i) < 16) {                \
+      long long ts_;                                                                             \
+      asm volatile("mov.u64 %0, %%clock64;" : "=l"(ts_));                                       \
+      g_kvt[(blockIdx.x * 2 + (warp >> 2)) * 16 + (i)] = ts_;                                     \
+    }                                                                                            \
+  } while (0)
+#else
+#define KV_STAMP(i) do { } while (0)
+#endif
+
 struct Shared {
-  uint64_t full[kStages], empty[kStages], aux;
+  uint64_t full[kMaxStages], empty[kMaxStages], aux;
   uint64_t nr;  // the producer warp has quantised the new token's row
   float red[kMaxWarps][kD];  // per-warp partial outputs (unnormalised, relative to the warp's maximum)
   float gm[kMaxWarps], gl[kMaxWarps];
@@ -163,8 +171,9 @@ template <int MINB, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32 + 32, MINB)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                  int32_t* __restrict__ evicted_pos, int chunk, int stages) {
+                  int32_t* __restrict__ evicted_pos, int chunk, int stage_shift) {
   constexpr int kThreads = kWarps * 32;
+  const int stages = 1 << stage_shift;  // ring depth: a power of two
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
   // dynamic layout: ring[stages][K tile | V tile] | acc_s[chunk] f64 | pos_s[chunk] i32 | p[chunk] f32
@@ -179,6 +188,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   // the previous kernel of the stream may have written this cache or produced q / k_new / v_new
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  KV_STAMP(13);
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
   int cnt = c.count[su];
   // (checked build: the unit and the rows this block streams must lie inside the cache)
@@ -195,9 +205,21 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
   const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
   bool timed_out = false;
+  // the consumer lanes' query and new-key words, requested before the barriers are set up so that their
+  // latency overlaps the block's start: the sixteen channels 16 (lane % 8) .. (self score), the group 32 c4 .. (operands)
+  uint4 in_q[2], in_k[2], in_g[4];
+  if (warp < kWarps) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      in_q[i] = *reinterpret_cast<const uint4*>(qu + 16 * (lane & 7) + 8 * i);
+      in_k[i] = *reinterpret_cast<const uint4*>(ku + 16 * (lane & 7) + 8 * i);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) in_g[i] = *reinterpret_cast<const uint4*>(qu + 32 * (lane & 3) + 8 * i);
+  }
 
   auto issue_stage = [&](int j) {  // producer lane only
-    const int s = j % stages;
+    const int s = j & (stages - 1);
     const int rows = min(kTileRows, cnt - j * kTileRows);
     const uint32_t bytes = (uint32_t)rows * kRowBytes;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
@@ -238,7 +260,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     if (lane == 0) mbar_arrive(&sh.nr);
     if (lane == 0) {
       for (int j = stages; j < ntile; ++j) {
-        if (!bar_wait(&sh.empty[j % stages], (uint32_t)(j / stages - 1) & 1u)) timed_out = true;
+        if (!bar_wait(&sh.empty[j & (stages - 1)], (uint32_t)((j >> stage_shift) - 1) & 1u)) timed_out = true;
         issue_stage(j);
       }
       if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
@@ -251,8 +273,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     // the group), so that one accumulator tile holds, per row, the four group sums  sum(q_i code_i);
     // scale and zero are applied once per group.  Lane (g, c4) = (lane / 4, lane % 4) loads the 16 bytes of
     // group c4 of rows g and g + 8; which channel sits at which k index is free as long as B agrees.
-    // Values stay on the FMA pipe: lane = (row sub of four rows per pass, eighth h8 of the row: 16 channels).
-    const int sub = lane >> 3, h8 = lane & 7;
+    // Values on the tensor cores as well, with the codes as the row operand and the weights as the column operand.
     const int g = lane >> 2, c4 = lane & 3;
     // the new token against itself, at full precision (every warp computes the same value)
     float s_self;
@@ -260,8 +281,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       float part = 0.f;
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        const uint4 rq = *reinterpret_cast<const uint4*>(qu + 16 * h8 + 8 * i);
-        const uint4 rk = *reinterpret_cast<const uint4*>(ku + 16 * h8 + 8 * i);
+        const uint4 rq = in_q[i], rk = in_k[i];
         const uint32_t wq[4] = {rq.x, rq.y, rq.z, rq.w}, wk[4] = {rk.x, rk.y, rk.z, rk.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -282,7 +302,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       uint32_t raw[16];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint4 r4 = *reinterpret_cast<const uint4*>(qu + 32 * c4 + 8 * i);
+        const uint4 r4 = in_g[i];
         raw[4 * i] = r4.x;
         raw[4 * i + 1] = r4.y;
         raw[4 * i + 2] = r4.z;
@@ -307,15 +327,17 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       }
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
-    float o[16];
+    float o[32];  // o[4 j + i] = accumulator i of the value product j (see below)
 #pragma unroll
-    for (int i = 0; i < 16; ++i) o[i] = 0.f;
-    float zacc = 0.f;  // sum of p * zero of this lane's rows and group
+    for (int i = 0; i < 32; ++i) o[i] = 0.f;
+    float zacc = 0.f;  // sum of p * zero of this lane's rows and group, minus the code offset's share
     float mg = -INFINITY, lg = 0.f;
     const int cb = (warp & 3) * 16;  // the warp's rows of a tile
+    KV_STAMP(0);
     for (int j = warp >> 2; j < ntile; j += kWarps / 4) {
-      const int s = j % stages;
-      if (!bar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
+      const int s = j & (stages - 1);
+      if (!bar_wait(&sh.full[s], (uint32_t)(j >> stage_shift) & 1u)) timed_out = true;
+      KV_STAMP(1 + 3 * (j / (kWarps / 4)));
       const unsigned char* kt = ring + (size_t)s * 2 * kTileBytes;
       const unsigned char* vt = kt + kTileBytes;
       const int rows = min(kTileRows, cnt - j * kTileRows);
@@ -360,6 +382,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
           if (rowB < rows) p[j * kTileRows + rowB] = sB;
         }
       }
+      KV_STAMP(2 + 3 * (j / (kWarps / 4)));
       // one softmax state per warp: maximum over its sixteen rows of this tile
       float mnew = fmaxf(mg, fmaxf(sA, sB));
       mnew = fmaxf(mnew, __shfl_xor_sync(0xffffffffu, mnew, 4));
@@ -376,47 +399,76 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
         zacc *= f;
         if (f != 1.0f) {  // (warp-uniform) the reference maximum moved
 #pragma unroll
-          for (int i = 0; i < 16; ++i) o[i] *= f;
+          for (int i = 0; i < 32; ++i) o[i] *= f;
         }
-        // ---- values: four passes of four rows; row cb + 4 ps + sub has its weight in lane group (4 ps + sub) % 8 ----
+        // ---- values on the tensor cores: D[channel][column] += codes^T[channel][row] * W[row][column] ----
+        // k = the warp's sixteen rows; m = sixteen channels per product j: channel 8 g + j (word g of the
+        // row, nibble j) and 64 + 8 g + j (word g + 8); n = (group, part): column grp + 4 part holds the
+        // weight p * scale of (row, grp) split into a bf16 head (part 0) and its bf16 remainder (part 1).
+        // Codes enter as 128 + code (exact in bf16); the offset's share 128 * (sum of the weights as given)
+        // leaves through zacc together with the zeros.  Lane (g, c4) holds rows 2 c4, 2 c4 + 1, 2 c4 + 8,
+        // 2 c4 + 9 for both operands; its column of W is n = g.
+        const int grp = g & 3;
+        const bool head = g < 4;
+        float part[4];
 #pragma unroll
-        for (int ps = 0; ps < 4; ++ps) {
-          const int row = cb + 4 * ps + sub;
-          const float e = __shfl_sync(0xffffffffu, ps < 2 ? eA : eB, 4 * (4 * (ps & 1) + sub));
-          uint2 vw = make_uint2(0, 0);
-          uint32_t vmeta = 0;
-          if (row < rows) {
-            vw = *reinterpret_cast<const uint2*>(vt + row * kRowBytes + 8 * h8);
-            vmeta = *reinterpret_cast<const uint32_t*>(vt + row * kRowBytes + 64 + 4 * (h8 >> 1));
+        for (int x = 0; x < 4; ++x) {
+          const int rr = 2 * c4 + (x & 1) + 8 * (x >> 1);
+          const float e = __shfl_sync(0xffffffffu, x < 2 ? eA : eB, 4 * (2 * c4 + (x & 1)));
+          uint32_t vmeta = *reinterpret_cast<const uint32_t*>(vt + (cb + rr) * kRowBytes + 64 + 4 * grp);
+          if (cb + rr >= rows) vmeta = 0u;  // stale bytes past the end of the last tile
+          const float w = e * bf16_bits_to_float(vmeta & 0xffffu);
+          const float wh = __uint_as_float(__float_as_uint(w) & 0xffff0000u);
+          part[x] = head ? wh : w - wh;
+          if (head) zacc = fmaf(e, bf16_bits_to_float(vmeta >> 16), zacc);
+        }
+        uint32_t b0, b1;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(b0) : "f"(part[1]), "f"(part[0]));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(b1) : "f"(part[3]), "f"(part[2]));
+        // the offset's share, from the weights as rounded
+        zacc -= 128.f * ((__uint_as_float(b0 << 16) + __uint_as_float(b0 & 0xffff0000u)) +
+                         (__uint_as_float(b1 << 16) + __uint_as_float(b1 & 0xffff0000u)));
+        uint32_t a[4][8];  // [operand register][product j]
+#pragma unroll
+        for (int hp = 0; hp < 4; ++hp) {  // operand register hp: rows (2 c4, +1) or (2 c4 + 8, +9), word g or g + 8
+          const int r0 = cb + 2 * c4 + 8 * (hp >> 1);
+          const uint32_t wa = *reinterpret_cast<const uint32_t*>(vt + r0 * kRowBytes + 4 * g + 32 * (hp & 1));
+          const uint32_t wb = *reinterpret_cast<const uint32_t*>(vt + (r0 + 1) * kRowBytes + 4 * g + 32 * (hp & 1));
+          const uint32_t y0 = __byte_perm(wa, wb, 0x5410), y1 = __byte_perm(wa, wb, 0x7632);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            a[hp][i] = and_or(y0 >> (4 * i), 0x000F000Fu, 0x43004300u);
+            a[hp][4 + i] = and_or(y1 >> (4 * i), 0x000F000Fu, 0x43004300u);
           }
-          // p * x_hat_i = p zero + (p scale) code_i
-          const float es = e * bf16_bits_to_float(vmeta & 0xffffu);
-          zacc = fmaf(e, bf16_bits_to_float(vmeta >> 16), zacc);
-          const uint32_t w[2] = {vw.x, vw.y};
+        }
 #pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            float n[8];
-            codes8(w[k], n);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o[8 * k + i] = fmaf(es, n[i], o[8 * k + i]);
-          }
+        for (int j = 0; j < 8; ++j) {
+          asm volatile(
+              "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+              : "+f"(o[4 * j]), "+f"(o[4 * j + 1]), "+f"(o[4 * j + 2]), "+f"(o[4 * j + 3])
+              : "r"(a[0][j]), "r"(a[1][j]), "r"(a[2][j]), "r"(a[3][j]), "r"(b0), "r"(b1));
         }
         mg = mnew;
       }
       __syncwarp();
+      KV_STAMP(3 + 3 * (j / (kWarps / 4)));
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&sh.empty[s])) : "memory");
     }
-    // add up the warp's rows (same softmax reference), then this lane's channels go to shared memory
+    KV_STAMP(14);
+    // zeros and offset: per group, over the warp's rows (the four lanes of a row group) and over head and remainder
+    zacc += __shfl_xor_sync(0xffffffffu, zacc, 1);
+    zacc += __shfl_xor_sync(0xffffffffu, zacc, 2);
+    zacc += __shfl_xor_sync(0xffffffffu, zacc, 16);
+    // this lane's column pair is n = 2 c4, 2 c4 + 1: groups 0, 1 (c4 even: channels 8 g + j, accumulators 0 / 1)
+    // or 2, 3 (c4 odd: channels 64 + 8 g + j, accumulators 2 / 3); the one that is the channel's own group counts
+    const int own = 2 * (c4 & 1) + (g >> 2);
+    const float zg = __shfl_sync(0xffffffffu, zacc, 4 * own);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      float v = o[i] + zacc;
-      v += __shfl_xor_sync(0xffffffffu, v, 8);
-      v += __shfl_xor_sync(0xffffffffu, v, 16);
-      o[i] = v;
-    }
-    if (sub == 0) {
-#pragma unroll
-      for (int i = 0; i < 16; ++i) sh.red[warp][16 * h8 + i] = o[i];
+    for (int j = 0; j < 8; ++j) {
+      const float lo2 = (g >> 2) ? o[4 * j + 1] : o[4 * j], hi2 = (g >> 2) ? o[4 * j + 3] : o[4 * j + 2];
+      float v = (c4 & 1) ? hi2 : lo2;
+      v += __shfl_xor_sync(0xffffffffu, v, 2);  // head (c4 < 2) + remainder (c4 >= 2)
+      if (c4 < 2) sh.red[warp][64 * c4 + 8 * g + j] = v + zg;
     }
     if (lane == 0) {
       sh.gm[warp] = mg;
@@ -482,6 +534,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     if (lane == 0) sh.wbest[warp] = best;
     if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
+    KV_STAMP(15);
     if (warp == 0) {
       const Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
       int slot, ev;
@@ -551,10 +604,16 @@ gather_kv4_kernel(CacheView c, PrefillScratch s, const __nv_bfloat16* __restrict
 
 }  // namespace
 
+#ifdef H2O_PHASE_TIMERS
+extern "C" int h2o_debug_kv4_timers(long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_kvt, sizeof(long long) * (size_t)n);
+}
+#endif
+
 size_t kv4_row_bytes() { return kRowBytes; }
 
 template <int MINB, int NW>
-static cudaError_t launch_kv4(const CacheView& c, int chunk, int stages, size_t smem, const void* q, const void* k_new,
+static cudaError_t launch_kv4(const CacheView& c, int chunk, int stage_shift, size_t smem, const void* q, const void* k_new,
                               const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   static unsigned long long attr_flags = 0;  // one word per instance, one bit per device
   {
@@ -574,22 +633,34 @@ static cudaError_t launch_kv4(const CacheView& c, int chunk, int stages, size_t 
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stages);
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stage_shift);
 }
 
 cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
                               int32_t* evicted_pos, cudaStream_t stream) {
   const int chunk = (max_B + 3) & ~3;
-  // many units: a shallow ring lets four blocks share an SM, which hides each block's serial start and end
-  const int stages = c.units > 4 * sm_count() ? 2 : kStages;
-  const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16;
-  if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  if (c.units <= 2 * sm_count()) return launch_kv4<2, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
-  if (c.units > 8 * sm_count()) {  // four consumer warps per block: five blocks per SM (no spills), six when the units are small
-    if (chunk <= 256) return launch_kv4<6, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
-    return launch_kv4<5, 4>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  const int sms = sm_count();
+  const size_t fixed = (size_t)chunk * 16 + 16;
+  auto smem_for = [&](int shift) { return ((size_t)(2 * kTileBytes) << shift) + fixed; };
+  if (smem_for(1) > 200 * 1024) return cudaErrorInvalidValue;
+#define KV4_GO(M, W, SHIFT) \
+  return launch_kv4<M, W>(c, chunk, SHIFT, smem_for(SHIFT), q, k_new, v_new, out, evicted_pos, stream)
+  // Few units (at most two blocks per SM): the deepest ring that fits, since nothing else hides the load latency
+  // (eight tiles in flight against four: 13.1 -> 11.8 us per launch at 256 units of 410 slots); sixteen consumer
+  // warps when a block has the SM to itself.
+  if (c.units <= 2 * sms) {
+    const bool alone = c.units <= sms;
+    int shift = 3;
+    while (shift > 1 && (alone ? 1 : 2) * (smem_for(shift) + 12 * 1024) > 220 * 1024) --shift;
+    if (alone) KV4_GO(1, 16, shift);
+    KV4_GO(2, 8, shift);
   }
-  return launch_kv4<4, 8>(c, chunk, stages, smem, q, k_new, v_new, out, evicted_pos, stream);
+  // Many units: four consumer warps per block and four blocks per SM (96 registers a thread), whose serial
+  // starts and ends hide one another; a shallow ring once the blocks outnumber the resident slots.
+  if (c.units > 4 * sms) KV4_GO(4, 4, 1);
+  if (smem_for(2) > 200 * 1024) KV4_GO(4, 4, 1);
+  KV4_GO(4, 4, 2);
+#undef KV4_GO
 }
 
 // after the selection kernel has written positions, scores and counts (its own row gather is skipped)
