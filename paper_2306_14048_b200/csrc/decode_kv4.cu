@@ -165,13 +165,17 @@ struct Shared {
   __align__(16) uint32_t qb[32][20];
 };
 
-// MINB: blocks per SM the register allocation leaves room for.  A launch with at most two blocks per SM runs
-// faster with the registers the compiler wants (96, nothing spilled); many units need four resident blocks.
-template <int MINB, int kWarps>
+// MINB: blocks per SM the register allocation leaves room for (the kernel wants ~96 registers a thread).
+// EARLY: the instances for launches of at most two waves of blocks, where the start of a block is exposed: they
+// take the host's hints (cache untouched by the previous launch of the stream: tiles requested before the grid
+// dependency is awaited; every unit full: no counter read before the first request) and fetch the new value row
+// at the start.  In launches of many waves the same code was slower
+// (3584 units of 104 slots: 46.4 -> 48.4 us), so those instances leave it out.
+template <int MINB, int kWarps, bool EARLY>
 __global__ void __launch_bounds__(kWarps * 32 + 32, MINB)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                  int32_t* __restrict__ evicted_pos, int chunk, int stage_shift) {
+                  int32_t* __restrict__ evicted_pos, int chunk, int stage_shift, int launch_flags) {
   constexpr int kThreads = kWarps * 32;
   const int stages = 1 << stage_shift;  // ring depth: a power of two
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -185,18 +189,36 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int su = blockIdx.x;
   const UnitMeta mt = c.meta[su];
-  // the previous kernel of the stream may have written this cache or produced q / k_new / v_new
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Programmatic dependent launch, as in the step kernel of the bf16 slots: the inputs may come from the previous
+  // kernel of the stream and are read after griddepcontrol.wait; the cache is written by this library alone, and
+  // when the host knows that its previous launch on this stream wrote another cache (`cache_is_quiescent`) the
+  // tiles are requested before the wait.  When the host expects every unit to be full (`all_full`) the block
+  // streams its whole budget without reading the counter first; the expectation only decides what is fetched.
+  bool cache_is_quiescent = false, all_full = false;
+  if constexpr (EARLY) {
+    cache_is_quiescent = (launch_flags & 1) != 0;
+    all_full = (launch_flags & 2) != 0;
+  }
+  if (!cache_is_quiescent) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   KV_STAMP(13);
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
-  int cnt = c.count[su];
-  // (checked build: the unit and the rows this block streams must lie inside the cache)
-  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) || !H2O_IN_RANGE(cnt, B + 1, c.status) ||
-      !H2O_IN_RANGE(mt.slot_off + (cnt > 0 ? cnt - 1 : 0), c.total_slots, c.status))
-    cnt = 0;
+  int cnt, nstr;  // entries of the unit, rows to stream
+  if constexpr (EARLY) {
+    cnt = all_full ? 0 : c.count[su];
+    nstr = all_full ? B : cnt;
+  } else {
+    cnt = c.count[su];
+    nstr = cnt;
+  }
   const int t = c.tpos[su];
-  const int ntile = (cnt + kTileRows - 1) / kTileRows;
+  // (checked build: the unit and the rows this block streams must lie inside the cache)
+  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) || !H2O_IN_RANGE(nstr, B + 1, c.status) ||
+      !H2O_IN_RANGE(mt.slot_off + (nstr > 0 ? nstr - 1 : 0), c.total_slots, c.status))
+    nstr = 0;
+  const int ntile = (nstr + kTileRows - 1) / kTileRows;
   unsigned char* Kb = static_cast<unsigned char*>(c.K) + mt.slot_off * kRowBytes;
   unsigned char* Vb = static_cast<unsigned char*>(c.V) + mt.slot_off * kRowBytes;
   double* acc_g = c.acc + mt.slot_off;
@@ -205,22 +227,28 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
   const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
   bool timed_out = false;
-  // the consumer lanes' query and new-key words, requested before the barriers are set up so that their
-  // latency overlaps the block's start: the sixteen channels 16 (lane % 8) .. (self score), the group 32 c4 .. (operands)
+  // the consumer lanes' query and new-key words (the sixteen channels 16 (lane % 8) .. for the self score, the
+  // group 32 c4 .. for the operands) and warp 0's words of the new value: requested as early as the launch
+  // order allows, so that their latency overlaps the block's start
   uint4 in_q[2], in_k[2], in_g[4];
-  if (warp < kWarps) {
+  uint2 in_v = make_uint2(0u, 0u);
+  auto load_inputs = [&]() {
+    if (warp < kWarps) {
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      in_q[i] = *reinterpret_cast<const uint4*>(qu + 16 * (lane & 7) + 8 * i);
-      in_k[i] = *reinterpret_cast<const uint4*>(ku + 16 * (lane & 7) + 8 * i);
+      for (int i = 0; i < 2; ++i) {
+        in_q[i] = *reinterpret_cast<const uint4*>(qu + 16 * (lane & 7) + 8 * i);
+        in_k[i] = *reinterpret_cast<const uint4*>(ku + 16 * (lane & 7) + 8 * i);
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) in_g[i] = *reinterpret_cast<const uint4*>(qu + 32 * (lane & 3) + 8 * i);
+      if (EARLY && warp == 0) in_v = *reinterpret_cast<const uint2*>(vu + 4 * lane);
     }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) in_g[i] = *reinterpret_cast<const uint4*>(qu + 32 * (lane & 3) + 8 * i);
-  }
+  };
+  if (!cache_is_quiescent) load_inputs();
 
   auto issue_stage = [&](int j) {  // producer lane only
     const int s = j & (stages - 1);
-    const int rows = min(kTileRows, cnt - j * kTileRows);
+    const int rows = min(kTileRows, nstr - j * kTileRows);
     const uint32_t bytes = (uint32_t)rows * kRowBytes;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
     mbar_expect_tx(&sh.full[s], 2 * bytes);
@@ -237,14 +265,26 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     fence_barrier_init();
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     for (int j = 0; j < min(stages, ntile); ++j) issue_stage(j);
-    if (cnt > 0) {
-      const int npad = (cnt + 3) & ~3;  // stays inside the unit's padded slot range
+    if (nstr > 0) {
+      const int npad = (nstr + 3) & ~3;  // stays inside the unit's padded slot range
       mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
       bulk_load(acc_s, acc_g, (uint32_t)npad * 8u, &sh.aux);
       bulk_load(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
     }
   }
+  if constexpr (EARLY) {
+    if (all_full) cnt = c.count[su];
+  }
+  if constexpr (EARLY) cnt = min(cnt, nstr);  // (a unit never holds more than was streamed: its budget, or the counter itself)
+  else cnt = nstr;
   __syncthreads();
+  if constexpr (EARLY) {
+    if (cache_is_quiescent) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      load_inputs();
+    }
+  }
 
   if (warp == kWarps) {
     // ---- producer warp: one lane streams the tiles; lanes 0..7 quantise the new token's row meanwhile ----
@@ -492,7 +532,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     if (warp == 0) {  // output: this lane's four channels
       float res[4];
       {
-        const uint2 raw = *reinterpret_cast<const uint2*>(vu + 4 * lane);  // the new token's value
+        const uint2 raw = EARLY ? in_v : *reinterpret_cast<const uint2*>(vu + 4 * lane);  // the new token's value
         res[0] = w_self * __uint_as_float(raw.x << 16);
         res[1] = w_self * __uint_as_float(raw.x & 0xffff0000u);
         res[2] = w_self * __uint_as_float(raw.y << 16);
@@ -511,7 +551,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     }
 
     // ---- final probabilities, accumulation (Algorithm 2: accumulated score += probability), victim search ----
-    if (cnt > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
+    if (nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
     const bool full = cnt >= B;
     const float p_self = w_self * inv_l;
     Cand best = cand_none();
@@ -612,13 +652,13 @@ extern "C" int h2o_debug_kv4_timers(long long* host, int n) {
 
 size_t kv4_row_bytes() { return kRowBytes; }
 
-template <int MINB, int NW>
-static cudaError_t launch_kv4(const CacheView& c, int chunk, int stage_shift, size_t smem, const void* q, const void* k_new,
-                              const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+template <int MINB, int NW, bool EARLY>
+static cudaError_t launch_kv4(const CacheView& c, int chunk, int stage_shift, size_t smem, int launch_flags, const void* q,
+                              const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   static unsigned long long attr_flags = 0;  // one word per instance, one bit per device
   {
     cudaError_t e =
-        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB, NW>), 200 * 1024, &attr_flags);
+        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB, NW, EARLY>), 200 * 1024, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
@@ -631,20 +671,21 @@ static cudaError_t launch_kv4(const CacheView& c, int chunk, int stage_shift, si
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW, EARLY>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stage_shift);
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stage_shift, launch_flags);
 }
 
-cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, const void* k_new, const void* v_new, void* out,
-                              int32_t* evicted_pos, cudaStream_t stream) {
+cudaError_t launch_decode_kv4(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
+                              const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   const int chunk = (max_B + 3) & ~3;
+  const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
   const int sms = sm_count();
   const size_t fixed = (size_t)chunk * 16 + 16;
   auto smem_for = [&](int shift) { return ((size_t)(2 * kTileBytes) << shift) + fixed; };
   if (smem_for(1) > 200 * 1024) return cudaErrorInvalidValue;
-#define KV4_GO(M, W, SHIFT) \
-  return launch_kv4<M, W>(c, chunk, SHIFT, smem_for(SHIFT), q, k_new, v_new, out, evicted_pos, stream)
+#define KV4_GO(M, W, EARLY, SHIFT) \
+  return launch_kv4<M, W, EARLY>(c, chunk, SHIFT, smem_for(SHIFT), launch_flags, q, k_new, v_new, out, evicted_pos, stream)
   // Few units (at most two blocks per SM): the deepest ring that fits, since nothing else hides the load latency
   // (eight tiles in flight against four: 13.1 -> 11.8 us per launch at 256 units of 410 slots); sixteen consumer
   // warps when a block has the SM to itself.
@@ -652,14 +693,14 @@ cudaError_t launch_decode_kv4(const CacheView& c, int max_B, const void* q, cons
     const bool alone = c.units <= sms;
     int shift = 3;
     while (shift > 1 && (alone ? 1 : 2) * (smem_for(shift) + 12 * 1024) > 220 * 1024) --shift;
-    if (alone) KV4_GO(1, 16, shift);
-    KV4_GO(2, 8, shift);
+    if (alone) KV4_GO(1, 16, true, shift);
+    KV4_GO(2, 8, true, shift);
   }
   // Many units: four consumer warps per block and four blocks per SM (96 registers a thread), whose serial
   // starts and ends hide one another; a shallow ring once the blocks outnumber the resident slots.
-  if (c.units > 4 * sms) KV4_GO(4, 4, 1);
-  if (smem_for(2) > 200 * 1024) KV4_GO(4, 4, 1);
-  KV4_GO(4, 4, 2);
+  if (c.units > 8 * sms) KV4_GO(4, 4, false, 1);
+  if (c.units > 4 * sms || smem_for(2) > 200 * 1024) KV4_GO(4, 4, true, 1);
+  KV4_GO(4, 4, true, 2);
 #undef KV4_GO
 }
 
