@@ -258,8 +258,9 @@ int h2o_cache_status(h2o_cache_t* cache, void* stream);
  * Tuning knob (no counterpart in the paper): how the decode kernel is laid out.
  * split  = thread blocks (one cluster) sharing a unit: 1, 2, 4 or 8; 0 keeps the
  *          value chosen at create time from the number of units and the budgets.
- * stages = depth of the shared-memory ring of 16 KB (K tile + V tile) stages, 1..8;
- *          0 = default.  Results do not depend on either value beyond summation order.
+ * stages = depth of the shared-memory ring of 16 KB (K tile + V tile) stages, 1..8
+ *          (rounded down to a power of two); 0 = default.  Results do not depend on
+ *          either value beyond summation order.
  */
 int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages);
 /*

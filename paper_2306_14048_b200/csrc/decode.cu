@@ -38,7 +38,7 @@ namespace {
 // SM hide one another's serial prologue and epilogue, which dominate a unit of a few tiles).
 constexpr int kMaxWarps = 8;
 constexpr int kSmallUnitRows = 160;  // largest block share (slots) served by the 4-warp variant
-constexpr int kTileBytes = 8192;
+constexpr int kTileBytes = 8192;  // (4 KB tiles with twice the depth and 16 KB tiles with half of it were slower)
 constexpr int kMaxStages = 8;
 constexpr int kDefaultStages = 4;
 constexpr int kMaxSplit = 8;
@@ -180,8 +180,14 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 template <typename T, int D, int MINB, int NW, bool TOPK>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
-              T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages,
+              T* __restrict__ out, int32_t* __restrict__ evicted_pos, int split, int chunk, int stages, int stage_shift,
               int launch_flags) {
+  // stages = 1 << stage_shift, the ring depth: a power of two, so that slot and phase of tile j are a mask and a
+  // shift.  The register-capped instances (MINB >= 4) keep the division by the run-time depth: there the cheaper
+  // form changed the register allocation into spilling and was slower (3584 units of 104 slots: 44.2 -> 47.0 us),
+  // in the uncapped instance it is faster (256 units of 410 slots: 12.7 -> 12.2 us).
+  auto ring_slot = [&](int j) { return MINB >= 4 ? j % stages : (j & (stages - 1)); };
+  auto ring_turn = [&](int j) { return MINB >= 4 ? j / stages : (j >> stage_shift); };
   using C = Cfg<T, D, NW>;
   constexpr int kWarps = NW, kThreads = NW * 32;
   constexpr int VEC = C::VEC, LPR = C::LPR, RPW = C::RPW, RPC = C::RPC, TILE_ROWS = C::TILE_ROWS, GROUPS = C::GROUPS;
@@ -261,7 +267,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
   bool timed_out = false;
 
   auto issue_stage = [&](int j) {  // producer lane only
-    const int s = j % stages;
+    const int s = ring_slot(j);
     const int rows = min(TILE_ROWS, nstr - j * TILE_ROWS);
     const uint32_t bytes = (uint32_t)rows * C::ROW_BYTES;
     unsigned char* dst = ring + (size_t)s * 2 * kTileBytes;
@@ -312,7 +318,7 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     // ---- producer warp: one lane streams the tiles through the ring ------------------
     if (lane == 0) {
       for (int j = stages; j < ntile; ++j) {
-        if (!mbar_wait(&sh.empty[j % stages], (uint32_t)(j / stages - 1) & 1u)) timed_out = true;
+        if (!mbar_wait(&sh.empty[ring_slot(j)], (uint32_t)(ring_turn(j) - 1) & 1u)) timed_out = true;
         issue_stage(j);
       }
     }
@@ -342,8 +348,8 @@ decode_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_new,
     constexpr bool topk_mode = TOPK;  // (the host launches one block per unit then: split == 1)
     if (mask_kind != 0 && nloc > 0 && !mbar_wait(&sh.aux, 0)) timed_out = true;
     for (int j = 0; j < ntile; ++j) {
-      const int s = j % stages;
-      if (!mbar_wait(&sh.full[s], (uint32_t)(j / stages) & 1u)) timed_out = true;
+      const int s = ring_slot(j);
+      if (!mbar_wait(&sh.full[s], (uint32_t)ring_turn(j) & 1u)) timed_out = true;
       if (j == 0) H2O_STAMP(2);
       const T* kt = reinterpret_cast<const T*>(ring + (size_t)s * 2 * kTileBytes);
       const T* vt = reinterpret_cast<const T*>(ring + (size_t)s * 2 * kTileBytes + kTileBytes);
@@ -692,6 +698,9 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   const int want = stages_req > 0 ? (stages_req > kMaxStages ? kMaxStages : stages_req) : auto_stages;
   int stages = (chunk + C::TILE_ROWS - 1) / C::TILE_ROWS;
   stages = stages < 1 ? 1 : (stages > want ? want : stages);
+  int stage_shift = 0;
+  while ((2 << stage_shift) <= stages) ++stage_shift;
+  stages = 1 << stage_shift;  // the largest power of two within the wanted depth
   const size_t smem = (size_t)stages * 2 * kTileBytes + (size_t)chunk * 16 + 16 +
                       (split > 1 ? (size_t)kMaxSplit * D * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;  // one word per template instance, one bit per device
@@ -719,7 +728,7 @@ cudaError_t launch_minb(const CacheView& c, int split, int chunk, int stages_req
   cfg.numAttrs = split > 1 ? 3 : 2;
   return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, MINB, NW, TOPK>, c, static_cast<const T*>(q),
                             static_cast<const T*>(k_new), static_cast<const T*>(v_new), static_cast<T*>(out),
-                            evicted_pos, split, chunk, stages, launch_flags);
+                            evicted_pos, split, chunk, stages, stage_shift, launch_flags);
 }
 
 template <typename T, int D>
