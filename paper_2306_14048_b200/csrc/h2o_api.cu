@@ -112,7 +112,7 @@ ScratchLayout make_scratch_layout(const h2o_config_t* cfg, int64_t total_tokens)
   S.rowstat = take(cells * group_of(cfg) * 2 * sizeof(float));  // row maximum and row sum per QUERY head (planar or interleaved)
   S.acc0 = take(cells * sizeof(double));
   // cu_seqlens, two work counters, first item index of every group of units (at most one group per unit)
-  S.cu = take(((size_t)cfg->batch + 1 + 2 + (size_t)cfg->batch * cfg->n_heads + 1) * sizeof(int32_t));
+  S.cu = take(((size_t)cfg->batch + 1 + 2 + (size_t)cfg->batch * cfg->n_heads * group_of(cfg) + 1) * sizeof(int32_t));
   S.total = off;
   return S;
 }
@@ -395,19 +395,21 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   cache->cu.assign(cu_seqlens, cu_seqlens + cfg.batch + 1);  // pageable source: staged before the call returns
   cache->cu.resize((size_t)cfg.batch + 3, 0);  // the work counters travel with it: zero at every launch
   ps.item_base = ps.cu + cfg.batch + 3;
-  ps.fs_grp = h2o::fwd_group_units(cache->view.units, max_seqlen);
+  // (the forward kernels work on QUERY heads: with grouped-query attention a unit there is one query head)
+  const int q_heads = cfg.n_heads * cache->view.group, q_units = cache->view.units * cache->view.group;
+  ps.fs_grp = h2o::fwd_group_units(q_units, max_seqlen);
   ps.fs_groups = 0;
   ps.fs_items = 0;
   if (ps.fs_grp > 0) {  // item order of the persistent forward kernel: a group has as many levels as its longest
                         // sequence has query blocks of 128
-    const int units = cache->view.units, grp = ps.fs_grp;
+    const int units = q_units, grp = ps.fs_grp;
     ps.fs_groups = (units + grp - 1) / grp;
     int64_t base = 0;
     cache->cu.push_back(0);
     for (int g = 0; g < ps.fs_groups; ++g) {
       const int u0 = g * grp, u1 = std::min(units, u0 + grp);
       int nbmax = 0;
-      for (int sq = u0 / cfg.n_heads; sq <= (u1 - 1) / cfg.n_heads; ++sq)
+      for (int sq = u0 / q_heads; sq <= (u1 - 1) / q_heads; ++sq)
         nbmax = std::max(nbmax, (int)(((int64_t)cu_seqlens[sq + 1] - cu_seqlens[sq] + 127) / 128));
       base += (int64_t)(u1 - u0) * nbmax;
       if (base > INT32_MAX) return H2O_ERR_UNSUPPORTED;
@@ -423,8 +425,7 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   // bf16 / head_dim 128 runs on the tensor cores; every other combination on the fp32 FMA pipe
   const int in_dtype = input_dtype(cfg.dtype);
   // (a sparse pattern is applied by the fp32-FMA kernels only)
-  const bool tc = cache->prefill_path != 1 && cache->view.mask_kind == 0 && cache->view.group == 1 &&
-                  h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
+  const bool tc = cache->prefill_path != 1 && cache->view.mask_kind == 0 && h2o::prefill_tc_supported(in_dtype, cfg.head_dim);
   cudaError_t e = cudaSuccess;
   // optional phase events of this one call (diagnostic): before the forward kernel, after it, after the column
   // sums, after selection and gather

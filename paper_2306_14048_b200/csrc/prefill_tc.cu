@@ -137,16 +137,25 @@ struct CsShared {
 // Work item: one (unit, pair of key blocks {pi, nb-1-pi}); all items of a unit have nb+1 tiles.  A block
 // walks over items blockIdx.x, blockIdx.x + gridDim.x, ...: barriers, tensor memory and the pipeline stay
 // up from one item to the next, so an item's first loads overlap the previous item's last tiles.
+// Grouped-query attention (group > 1): a key block of K/V head h meets the query blocks of all the group's query
+// heads h * group + g, one after the other, and their probabilities add up in the same column sums; the tiles of
+// a key block are then numbered g * (query blocks) + (query block).
 struct CsItem {
-  int h, lo, n;   // head, first token and length of the sequence
+  int h, lo, n;   // K/V head, first token and length of the sequence
   int jb0, jb1;   // the two key blocks (jb1 == jb0: one)
   int t0, total;  // tiles of the first key block, tiles of the item
+  int nb, group;  // query blocks of the sequence, query heads per K/V head
 };
 struct CsWalk {
   int w, t;  // item, tile inside the item
   CsItem it;
   __device__ __forceinline__ int jb() const { return t < it.t0 ? it.jb0 : it.jb1; }                       // key block
-  __device__ __forceinline__ int ib() const { return t < it.t0 ? it.jb0 + t : it.jb1 + (t - it.t0); }     // query block
+  __device__ __forceinline__ int local() const { return t < it.t0 ? t : t - it.t0; }  // tile inside its key block
+  __device__ __forceinline__ int g() const { return it.group == 1 ? 0 : local() / (it.nb - jb()); }     // query head of the group
+  __device__ __forceinline__ int ib() const {                                                             // query block
+    return it.group == 1 ? jb() + local() : jb() + local() % (it.nb - jb());
+  }
+  __device__ __forceinline__ int qh() const { return it.h * it.group + g(); }                             // query head
   __device__ __forceinline__ bool first_of_cb() const { return t == 0 || t == it.t0; }
   __device__ __forceinline__ bool last_of_cb() const { return t == it.t0 - 1 || t == it.total - 1; }
 };
@@ -160,17 +169,20 @@ __device__ __forceinline__ bool cs_item(const PrefillScratch& s, int n_heads, in
   if (pi >= (nb + 1) / 2) return false;
   it.jb0 = pi;
   it.jb1 = nb - 1 - pi;
-  it.t0 = nb - it.jb0;  // tiles of key block jb: query blocks jb .. nb-1
-  it.total = it.t0 + (it.jb1 > it.jb0 ? nb - it.jb1 : 0);
+  it.nb = nb;
+  it.t0 = it.group * (nb - it.jb0);  // tiles of key block jb: query blocks jb .. nb-1 of every query head
+  it.total = it.t0 + (it.jb1 > it.jb0 ? it.group * (nb - it.jb1) : 0);
   return true;
 }
 __device__ __forceinline__ bool cs_seek(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
   while (k.w < n_items && !cs_item(s, n_heads, max_pairs, k.w, k.it)) k.w += (int)gridDim.x;
   return k.w < n_items;
 }
-__device__ __forceinline__ bool cs_first(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
+__device__ __forceinline__ bool cs_first(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, int group,
+                                         CsWalk& k) {
   k.w = (int)blockIdx.x;
   k.t = 0;
+  k.it.group = group;
   return cs_seek(s, n_heads, max_pairs, n_items, k);
 }
 __device__ __forceinline__ bool cs_next(const PrefillScratch& s, int n_heads, int max_pairs, int n_items, CsWalk& k) {
@@ -182,7 +194,7 @@ __device__ __forceinline__ bool cs_next(const PrefillScratch& s, int n_heads, in
 
 __global__ void __launch_bounds__(kCsThreads, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                 PrefillScratch s, int n_heads, int max_pairs, int n_items, float scale2, int32_t* status) {
+                 PrefillScratch s, int n_heads, int group, int max_pairs, int n_items, float scale2, int32_t* status) {
   extern __shared__ unsigned char dyn_raw[];
   __shared__ CsShared sh;
   unsigned char* dyn = dyn_raw + ((1024u - (smem_u32(dyn_raw) & 1023u)) & 1023u);
@@ -225,7 +237,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       prefetch_tensormap(&map_k);
     }
     auto fetch = [&](const CsWalk& k, float2 (&raw)[4]) {  // {m, 1 / l} of the tile's 128 queries, four per lane
-      const float2* rowstat = s.rowstat + (int64_t)k.it.h * s.total_tokens + k.it.lo;
+      const float2* rowstat = s.rowstat + (int64_t)k.qh() * s.total_tokens + k.it.lo;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int qi = k.ib() * kTile + i * 32 + lane;
@@ -233,7 +245,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     };
     CsWalk cur;
-    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
+    bool have = cs_first(s, n_heads, max_pairs, n_items, group, cur);
     float2 raw[4];
     if (have) fetch(cur, raw);
     bool ok = true;
@@ -253,7 +265,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (ok) {
           unsigned char* dst = q_ring + st * kTileBytes;
           mbar_expect_tx(&sh.q_full[st], kTileBytes);
-          tma_load_tile(dst, &map_q, cur.it.h, cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
+          tma_load_tile(dst, &map_q, cur.qh(), cur.it.lo + cur.ib() * kTile, &sh.q_full[st]);
         }
       }
       if (new_k) ++kc;
@@ -272,7 +284,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // ---------------- MMA issuer (whole warp runs the loop, one elected lane issues) ----------------
     constexpr uint32_t idesc = instr_desc_f16(kTile, kTile, kFmtBF16, kFmtBF16, false, false);
     CsWalk cur;
-    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
+    bool have = cs_first(s, n_heads, max_pairs, n_items, group, cur);
     for (int g = 0, kc = 0; have; ++g) {
       bool ok = true;
       if (cur.first_of_cb()) {
@@ -313,7 +325,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     double total_sum = 0.0;
     bool ok = true;
     CsWalk cur;
-    bool have = cs_first(s, n_heads, max_pairs, n_items, cur);
+    bool have = cs_first(s, n_heads, max_pairs, n_items, group, cur);
     for (int g = 0, cbc = 0; have && ok; ++g) {  // cbc: key blocks finished so far
       const int b = g & 1;
       const int b8 = g % kCsStatBufs;                // buffer of the row statistics
@@ -466,8 +478,9 @@ struct FwShared {
 template <int G>
 __global__ void __launch_bounds__(fw_threads(G), G == 2 ? 1 : 2)
 fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, float scale2,
+              const __grid_constant__ CUtensorMap map_v, PrefillScratch s, int n_heads, int kv_div, float scale2,
               __nv_bfloat16* __restrict__ out, int32_t* status) {
+  // n_heads counts QUERY heads; query head h reads K/V head h / kv_div (grouped-query attention; 1 otherwise)
   const bool wide_out = (reinterpret_cast<uintptr_t>(out) & 31u) == 0;
   extern __shared__ unsigned char dyn_raw[];
   __shared__ FwShared sh;
@@ -546,7 +559,7 @@ fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         unsigned char* dst = kv_ring + slot * kFwKvSlotBytes;
         const int row0 = lo + (r >> 1) * kFwKeys;
         mbar_expect_tx(&sh.kv_full[slot], kFwKvSlotBytes);
-        tma_load_tile(dst, map, h, row0, &sh.kv_full[slot]);
+        tma_load_tile(dst, map, h / kv_div, row0, &sh.kv_full[slot]);
       }
     }
   } else if (mma_idx >= 0 && mma_idx < 2 * G) {
@@ -843,7 +856,8 @@ struct FsItem {
 // being worked on); inside a group every unit's longest query block first, then every unit's second
 // longest, ...: long items start early, the ones claimed last are short.
 struct FsOrder {
-  int n_heads, units, grp, n_groups, n_items;
+  int n_heads, units, grp, n_groups, n_items;  // heads and units of the QUERY side
+  int kv_div;                                  // query heads per K/V head
   const int32_t* item_base;  // [n_groups + 1] first item index of every group (host-built from the prompt lengths:
                              // a group has as many levels x as its longest sequence has query blocks, so that
                              // a ragged batch does not make most indices name blocks that do not exist)
@@ -966,7 +980,7 @@ fwd_tc_short_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const CUtensorMap* map = r ? &map_v : &map_k;
             unsigned char* dst = kv_ring + (slot + r) * kFwKvSlotBytes;
             mbar_expect_tx(&sh.kv_full[slot + r], kFwKvSlotBytes);
-            tma_load_tile(dst, map, it.h, row0, &sh.kv_full[slot + r]);
+            tma_load_tile(dst, map, it.h / order.kv_div, row0, &sh.kv_full[slot + r]);
           }
           // the ring is full after the item's first tiles: time for the lookup two items ahead
           if (j == min(1, it.nt - 1) && wn < n_items) wn2 = claim(nx2);
@@ -1338,9 +1352,9 @@ cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, con
     if (e != cudaSuccess) return e;
   }
   const int nb = (max_seqlen + kTile - 1) / kTile;
-  dim3 grid((unsigned)(G == 2 ? (nb + 1) / 2 : nb), (unsigned)c.units);
-  fwd_tc_kernel<G><<<grid, fw_threads(G), smem, stream>>>(map_q, map_k, map_v, s, c.n_heads, make_scale2(c.scale),
-                                                         static_cast<__nv_bfloat16*>(out), c.status);
+  dim3 grid((unsigned)(G == 2 ? (nb + 1) / 2 : nb), (unsigned)(c.units * c.group));
+  fwd_tc_kernel<G><<<grid, fw_threads(G), smem, stream>>>(map_q, map_k, map_v, s, c.n_heads * c.group, c.group,
+                                                         make_scale2(c.scale), static_cast<__nv_bfloat16*>(out), c.status);
   return cudaGetLastError();
 }
 
@@ -1349,15 +1363,17 @@ cudaError_t launch_fwd_g(const CUtensorMap& map_q, const CUtensorMap& map_k, con
 cudaError_t launch_fwd_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                           const void* v, void* out, cudaStream_t stream) {
   CUtensorMap map_q, map_k, map_v;
-  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
+  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads * c.group, kTile) ||
+      !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kFwKeys) ||
       !make_whole_tile_map(&map_v, v, s.total_tokens, c.n_heads, kFwKeys))
     return cudaErrorInvalidValue;
   // short prompts: one query block per thread block, two blocks per SM; long ones: two query blocks share
   // every K/V tile
   if (max_seqlen <= kFwShortPrompt) {
     FsOrder o;
-    o.n_heads = c.n_heads;
-    o.units = c.units;
+    o.n_heads = c.n_heads * c.group;
+    o.units = c.units * c.group;
+    o.kv_div = c.group;
     o.grp = s.fs_grp;
     o.n_groups = s.fs_groups;
     o.n_items = s.fs_items;
@@ -1390,7 +1406,8 @@ bool prefill_tc_supported(int dtype, int head_dim) { return dtype == H2O_BF16 &&
 cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int max_seqlen, const void* q, const void* k,
                              cudaStream_t stream) {
   CUtensorMap map_q, map_k;
-  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads, kTile) || !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
+  if (!make_whole_tile_map(&map_q, q, s.total_tokens, c.n_heads * c.group, kTile) ||
+      !make_whole_tile_map(&map_k, k, s.total_tokens, c.n_heads, kTile))
     return cudaErrorInvalidValue;
   const int smem = kTileBytes * (1 + kCsQStages) + 1024;
   static unsigned long long attr_flags = 0;
@@ -1405,9 +1422,9 @@ cudaError_t launch_colsum_tc(const CacheView& c, const PrefillScratch& s, int ma
   // memory each), so that an item's fixed cost (first loads, pipeline fill) overlaps the previous item's
   // last tiles: config 3 (five tiles per item) 273 -> 250 us.  Long items run one per block and leave the
   // balancing to the hardware scheduler (config 2, 17 tiles per item: 212 us against 216 us persistent).
-  const bool persistent = nb + 1 <= kCsPersistentTiles && n_items > 2 * sm_count();
+  const bool persistent = c.group * (nb + 1) <= kCsPersistentTiles && n_items > 2 * sm_count();
   const int blocks = persistent ? 2 * sm_count() : n_items;
-  colsum_tc_kernel<<<blocks, kCsThreads, smem, stream>>>(map_q, map_k, s, c.n_heads, max_pairs, n_items,
+  colsum_tc_kernel<<<blocks, kCsThreads, smem, stream>>>(map_q, map_k, s, c.n_heads, c.group, max_pairs, n_items,
                                                          make_scale2(c.scale), c.status);
   return cudaGetLastError();
 }

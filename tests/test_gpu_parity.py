@@ -474,12 +474,26 @@ def test_topk_argument_and_state_errors(H2OCache):
     (2, "bf16", 64), (4, "bf16", 64), (2, "f32", 128), (4, "f32", 128),
 ])
 def test_grouped_query_attention_ragged(H2OCache, group, dtype, d):
-    """Prompt (fp32-FMA kernels), selection on the summed column sums, decode steps with one victim per unit."""
+    """Prompt, selection on the summed column sums, decode steps with one victim per unit."""
     from parity_harness import run_parity
 
     wl = _wl("gqa", 3, 2, d, dtype, [300, 77, 140], 40, [20, 9, 33], [24, 5, 31], seed=377 + d + group)
     st = run_parity(wl, H2OCache, export_every=8, group=group)
     print(st)
+
+
+def test_grouped_query_attention_tensor_core_prompt_kernels(H2OCache):
+    """bf16 / head_dim 128 prompts of a grouped cache run on the tensor-core kernels: the persistent forward kernel
+    (prompts up to 4096 tokens), the two-query-block one (longer), and column sums that add up over the group's
+    query heads; the fp32-FMA kernels on the same inputs give the same selection."""
+    from parity_harness import run_parity
+
+    wl = _wl("gqatc", 3, 2, 128, "bf16", [700, 129, 1025], 8, [40, 20, 60], [40, 12, 70], seed=911)
+    for group in (2, 4, 8):
+        print(run_parity(wl, H2OCache, export_every=4, group=group))
+    print(run_parity(wl, H2OCache, export_every=4, group=4, prefill_path=1))
+    wl = _wl("gqatclong", 1, 2, 128, "bf16", [4500], 4, [100], [120], seed=912)
+    print(run_parity(wl, H2OCache, export_every=2, group=2))
 
 
 @pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([6, 1], [12, 9])])
