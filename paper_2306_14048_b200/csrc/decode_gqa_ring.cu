@@ -1,0 +1,456 @@
+// Fused decode step for grouped-query attention, bf16 / head_dim 128: the streaming form of decode_gqa.cu.
+//
+// Same reading as there (own, not in the paper, which evicts per head): G query heads share the keys and values of
+// one (sequence, K/V head) unit, every query head has its own softmax over the unit's entries, a key's accumulated
+// score grows by the sum of the G probabilities (Algorithm 2's accumulation once per query head), one victim per
+// unit.
+//
+// Shape: one thread block per unit, eight consumer warps and a producer warp.  The producer streams the unit's K
+// rows and then its V rows as 8 KB tiles (32 rows) through one bulk-copy ring, so HBM stays busy across the two
+// passes.
+//   K pass: the scores of 16 rows x G heads are one mma.sync m16n8k16 chain (rows = M, heads = N, channels = K);
+//           a lane loads 16 bytes of a row and uses them as the k-slots of two products, the query operand is
+//           laid out to match (which channel sits in which k-slot is free as long as both operands agree).  The
+//           16-row blocks of the tiles go round the warps.  Raw scores to shared memory, [row][head].
+//   softmax per head over all rows (exact maximum and sum, as the accumulation needs the final probabilities),
+//           in place.
+//   V pass: a lane holds eight channels of a row (two rows per warp and pass) and G x 8 accumulators.
+// Tail as in the other step kernels: fp64 accumulation of the summed probabilities, victim by (score, position),
+// new row written into the freed slot.  Every wait on an mbarrier is bounded (H2O_ERR_TIMEOUT in the status word).
+#include <climits>
+#include <cuda_bf16.h>
+
+#include "h2o_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace h2o {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int kD = 128;
+constexpr int kWarps = 8, kThreads = kWarps * 32;
+constexpr int kTileRows = 32, kRowBytes = kD * 2, kTileBytes = kTileRows * kRowBytes;  // 8 KB
+constexpr int kStages = 8;
+constexpr uint32_t kSpin = 1u << 22;
+
+__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kSpin; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+struct Cand {
+  unsigned long long key;  // bit pattern of the (non-negative) ranking score
+  int pos, slot;           // slot -1: none, -2: the new token itself
+};
+__device__ __forceinline__ Cand cand_none() { return Cand{~0ull, INT_MAX, -1}; }
+__device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {
+  if (a.slot == -1) return false;
+  if (b.slot == -1) return true;
+  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
+}
+// Warp-wide minimum under the eviction order (scores are >= 0: their bit patterns order like the values).
+__device__ __forceinline__ Cand warp_argmin(const Cand& a) {
+  const bool valid = a.slot != -1;
+  const unsigned long long bits = valid ? a.key : ~0ull;
+  const unsigned hi = (unsigned)(bits >> 32), lo = (unsigned)bits;
+  const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
+  const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
+  const bool tie = valid && hi == mh && lo == ml;
+  const unsigned mp = __reduce_min_sync(0xffffffffu, tie ? (unsigned)a.pos : 0xffffffffu);
+  const unsigned who = __ballot_sync(0xffffffffu, tie && (unsigned)a.pos == mp);
+  if (who == 0) return cand_none();
+  Cand b;
+  b.key = ((unsigned long long)mh << 32) | ml;
+  b.pos = (int)mp;
+  b.slot = __shfl_sync(0xffffffffu, a.slot, __ffs(who) - 1);
+  return b;
+}
+
+struct Shared {
+  uint64_t full[kStages], empty[kStages], aux;
+  float part_m[kWarps][8], part_l[kWarps][8];  // per warp and head: softmax partials
+  float m[8], inv_l[8];
+  Cand wbest[kWarps];
+};
+
+// D (16 x 8, fp32) += A (16 x 16, bf16, row) * B (16 x 8, bf16, col)
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads + 32, 2)
+decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
+                       const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
+                       int32_t* __restrict__ evicted_pos, int chunk, int launch_flags) {
+  extern __shared__ __align__(128) unsigned char dyn[];
+  __shared__ Shared sh;
+  // dynamic layout: ring[kStages][tile] (reused for the warps' partial outputs after the stream) |
+  //                 acc_s[chunk] f64 | pos_s[chunk] i32 | p[(chunk + 4) * G] f32 ([row][head]; row cnt = the token itself)
+  unsigned char* ring = dyn;
+  double* acc_s = reinterpret_cast<double*>(dyn + (size_t)kStages * kTileBytes);
+  int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
+  float* p = reinterpret_cast<float*>(pos_s + chunk);
+  float* red = reinterpret_cast<float*>(ring);  // [2 * kWarps][G][kD]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int su = blockIdx.x;
+  const UnitMeta mt = c.meta[su];
+  // Programmatic dependent launch, as in the multi-head step kernel: the inputs may come from the previous kernel
+  // of the stream and are read after griddepcontrol.wait; the cache is written by this library alone, and when the
+  // host knows that its previous launch on this stream wrote another cache (`cache_is_quiescent`) the first tiles
+  // are requested before the wait.  When the host expects every unit to be full (`all_full`) the block streams its
+  // whole budget without reading the counter first; the expectation only decides what is fetched.
+  const bool cache_is_quiescent = (launch_flags & 1) != 0, all_full = (launch_flags & 2) != 0;
+  if (!cache_is_quiescent) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
+  const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
+  int cnt = all_full ? 0 : c.count[su];
+  const int t = c.tpos[su];
+  int nstr = all_full ? min(B, chunk) : cnt;  // rows to stream
+  if (!H2O_IN_RANGE(u, c.units, c.status) || !H2O_IN_RANGE(nstr, min(B, chunk) + 1, c.status) ||
+      !H2O_IN_RANGE(mt.slot_off + (nstr > 0 ? nstr - 1 : 0), c.total_slots, c.status))
+    nstr = 0;
+  const int nt = (nstr + kTileRows - 1) / kTileRows;  // tiles per matrix; the stream is K 0..nt-1, then V 0..nt-1
+  const __nv_bfloat16* Kb = reinterpret_cast<const __nv_bfloat16*>(c.K) + mt.slot_off * kD;
+  const __nv_bfloat16* Vb = reinterpret_cast<const __nv_bfloat16*>(c.V) + mt.slot_off * kD;
+  double* acc_g = c.acc + mt.slot_off;
+  int32_t* pos_g = c.pos + mt.slot_off;
+  const __nv_bfloat16* qu = q + (int64_t)u * G * kD;  // the group's query heads are consecutive
+  const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
+  const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
+  bool timed_out = false;
+
+  // the query operand of the score products: lane (n, c4) = (lane / 4, lane % 4) holds head n's channels
+  // 32 cc + 8 c4 .. + 7 for cc = 0..3 (zeros for n >= G), the same bytes a lane loads of a key row
+  const int gl = lane >> 2, c4 = lane & 3;
+  uint4 qb[4];
+  auto load_query = [&]() {
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc)
+      qb[cc] = (warp < kWarps && gl < G) ? *reinterpret_cast<const uint4*>(qu + gl * kD + 32 * cc + 8 * c4) : make_uint4(0, 0, 0, 0);
+  };
+  if (!cache_is_quiescent) load_query();
+
+  auto issue_tile = [&](int T) {  // producer lane only
+    const int s = T & (kStages - 1);
+    const int j = T < nt ? T : T - nt;
+    const int rows = min(kTileRows, nstr - j * kTileRows);
+    const uint32_t bytes = (uint32_t)rows * kRowBytes;
+    mbar_expect_tx(&sh.full[s], bytes);
+    bulk_load(ring + (size_t)s * kTileBytes, (T < nt ? Kb : Vb) + (int64_t)j * kTileRows * kD, bytes, &sh.full[s]);
+  };
+  if (tid == kThreads) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], kWarps);
+    }
+    mbar_init(&sh.aux, 1);
+    fence_barrier_init();
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    for (int T = 0; T < min(kStages, 2 * nt); ++T) issue_tile(T);
+    if (nstr > 0) {
+      const int npad = (nstr + 3) & ~3;  // stays inside the unit's padded slot range
+      mbar_expect_tx(&sh.aux, (uint32_t)npad * 12u);
+      bulk_load(acc_s, acc_g, (uint32_t)npad * 8u, &sh.aux);
+      bulk_load(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
+    }
+  }
+  if (all_full) cnt = c.count[su];
+  cnt = min(cnt, nstr);  // (a unit never holds more than was streamed: its budget, or the counter itself)
+  __syncthreads();
+  if (cache_is_quiescent) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    load_query();
+  }
+
+  if (warp == kWarps) {
+    // ---- producer warp: one lane keeps the ring full ------------------------------------------------------
+    if (lane == 0) {
+      for (int T = kStages; T < 2 * nt; ++T) {
+        if (!bar_wait(&sh.empty[T & (kStages - 1)], (uint32_t)((T >> 3) - 1) & 1u)) timed_out = true;
+        issue_tile(T);
+      }
+      if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+    }
+    return;
+  }
+
+  // ---- consumer warps -------------------------------------------------------------------------------------
+  // the new token against itself, per query head: warp g does head g with plain arithmetic
+  if (warp < G) {
+    const uint2 rq = *reinterpret_cast<const uint2*>(qu + warp * kD + 4 * lane);
+    const uint2 rk = *reinterpret_cast<const uint2*>(ku + 4 * lane);
+    float part = __uint_as_float(rq.x << 16) * __uint_as_float(rk.x << 16);
+    part = fmaf(__uint_as_float(rq.x & 0xffff0000u), __uint_as_float(rk.x & 0xffff0000u), part);
+    part = fmaf(__uint_as_float(rq.y << 16), __uint_as_float(rk.y << 16), part);
+    part = fmaf(__uint_as_float(rq.y & 0xffff0000u), __uint_as_float(rk.y & 0xffff0000u), part);
+    part = warp_sum(part);
+    if (lane == 0) p[cnt * G + warp] = c.scale * part;
+  }
+  // K pass: block b (16 rows) of the stream goes to warp b % 8; every warp steps through every tile so that
+  // the ring's barriers see all of them
+  for (int j = 0; j < nt; ++j) {
+    const int s = j & (kStages - 1);
+    if (!bar_wait(&sh.full[s], (uint32_t)(j >> 3) & 1u)) timed_out = true;
+    const int hb = ((warp - 2 * j) & 7);  // this warp's block of the tile: 0 or 1 (else none)
+    if (hb < 2) {
+      const unsigned char* kt = ring + (size_t)s * kTileBytes + (size_t)(16 * hb) * kRowBytes;
+      float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};  // two chains
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const uint4 ka = *reinterpret_cast<const uint4*>(kt + gl * kRowBytes + 64 * cc + 16 * c4);
+        const uint4 kb = *reinterpret_cast<const uint4*>(kt + (gl + 8) * kRowBytes + 64 * cc + 16 * c4);
+        mma_16816(d0, ka.x, kb.x, ka.y, kb.y, qb[cc].x, qb[cc].y);
+        mma_16816(d1, ka.z, kb.z, ka.w, kb.w, qb[cc].z, qb[cc].w);
+      }
+      // lane (gl, c4): rows gl and gl + 8 of the block, heads 2 c4 and 2 c4 + 1 (rows past the end hold stale bytes)
+      const int rowA = j * kTileRows + 16 * hb + gl, rowB = rowA + 8;
+      if (2 * c4 < G) {
+        if (rowA < cnt) *reinterpret_cast<float2*>(p + rowA * G + 2 * c4) = make_float2(c.scale * (d0[0] + d1[0]), c.scale * (d0[1] + d1[1]));
+        if (rowB < cnt) *reinterpret_cast<float2*>(p + rowB * G + 2 * c4) = make_float2(c.scale * (d0[2] + d1[2]), c.scale * (d0[3] + d1[3]));
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.empty[s]);
+  }
+  consumer_sync();
+
+  // ---- softmax per head over the cnt rows and the token itself: thread (x0, g) = (tid / G, tid % G) ----------
+  const int total = cnt + 1;
+  {
+    const int g = tid % G;
+    float mx = -INFINITY, sum = 0.f;
+    for (int x = tid / G; x < total; x += kThreads / G) {
+      const float sx = p[x * G + g];
+      if (sx > mx) {
+        sum *= expf(mx - sx);  // expf(-inf) = 0 the first time
+        mx = sx;
+      }
+      sum += expf(sx - mx);
+    }
+    // lanes of equal lane % G, then the warps
+#pragma unroll
+    for (int off = G; off < 32; off <<= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, mx, off), os = __shfl_xor_sync(0xffffffffu, sum, off);
+      const float nm = fmaxf(mx, om);
+      sum = (mx > -INFINITY ? sum * expf(mx - nm) : 0.f) + (om > -INFINITY ? os * expf(om - nm) : 0.f);
+      mx = nm;
+    }
+    if (lane < G) {
+      sh.part_m[warp][lane] = mx;
+      sh.part_l[warp][lane] = sum;
+    }
+    consumer_sync();
+    if (tid < G) {
+      float m = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) m = fmaxf(m, sh.part_m[w][tid]);
+      float l = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w)
+        if (sh.part_m[w][tid] > -INFINITY) l += sh.part_l[w][tid] * expf(sh.part_m[w][tid] - m);
+      sh.m[tid] = m;
+      sh.inv_l[tid] = 1.0f / l;
+    }
+    consumer_sync();
+    const float m = sh.m[g], inv_l = sh.inv_l[g];
+    for (int x = tid / G; x < total; x += kThreads / G) p[x * G + g] = expf(p[x * G + g] - m) * inv_l;
+  }
+  consumer_sync();
+
+  // ---- V pass: lane = (row of the warp's pair, eight channels); G x 8 accumulators ---------------------------
+  const int sub = lane >> 4, ch = lane & 15;
+  float o[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+#pragma unroll
+    for (int v = 0; v < 8; ++v) o[g][v] = 0.f;
+  for (int j = 0; j < nt; ++j) {
+    const int T = nt + j, s = T & (kStages - 1);
+    if (!bar_wait(&sh.full[s], (uint32_t)(T >> 3) & 1u)) timed_out = true;
+    const unsigned char* vt = ring + (size_t)s * kTileBytes;
+#pragma unroll
+    for (int ps = 0; ps < kTileRows / (2 * kWarps); ++ps) {
+      const int rl = ps * 2 * kWarps + 2 * warp + sub, row = j * kTileRows + rl;
+      if (row < cnt) {
+        float vf[8];
+        Vec16<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(vt + rl * kRowBytes + 16 * ch), vf);
+        float pr[G];
+        if constexpr (G == 2) {
+          const float2 p2 = *reinterpret_cast<const float2*>(p + row * G);
+          pr[0] = p2.x;
+          pr[1] = p2.y;
+        } else {
+#pragma unroll
+          for (int g4 = 0; g4 < G / 4; ++g4) {
+            const float4 p4 = *reinterpret_cast<const float4*>(p + row * G + 4 * g4);
+            pr[4 * g4] = p4.x;
+            pr[4 * g4 + 1] = p4.y;
+            pr[4 * g4 + 2] = p4.z;
+            pr[4 * g4 + 3] = p4.w;
+          }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+#pragma unroll
+          for (int v = 0; v < 8; v += 2) {
+            const float2 t2 = __ffma2_rn(make_float2(pr[g], pr[g]), make_float2(vf[v], vf[v + 1]), make_float2(o[g][v], o[g][v + 1]));
+            o[g][v] = t2.x;
+            o[g][v + 1] = t2.y;
+          }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.empty[s]);
+  }
+  // the ring is free once every warp has read its last tile: it takes the partial outputs
+  consumer_sync();
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float* dst = red + ((size_t)(2 * warp + sub) * G + g) * kD + 8 * ch;
+    *reinterpret_cast<float4*>(dst) = make_float4(o[g][0], o[g][1], o[g][2], o[g][3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(o[g][4], o[g][5], o[g][6], o[g][7]);
+  }
+  // (the staged scores and positions arrived long ago)
+  if (nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
+  consumer_sync();
+  for (int i = tid; i < G * kD; i += kThreads) {
+    const int g = i / kD, x = i % kD;
+    float acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < 2 * kWarps; ++w) acc += red[((size_t)w * G + g) * kD + x];
+    acc = fmaf(p[cnt * G + g], __bfloat162float(vu[x]), acc);
+    out[((int64_t)u * G + g) * kD + x] = __float2bfloat16_rn(acc);
+  }
+
+  // ---- accumulate (every head's probability), victim, in-place write ----------------------------------------
+  const bool full = cnt >= B;
+  Cand best = cand_none();
+  for (int x = tid; x < cnt; x += kThreads) {
+    double px = 0.0;
+#pragma unroll
+    for (int g = 0; g < G; ++g) px += (double)p[x * G + g];
+    const double a = acc_s[x] + px;
+    if (H2O_IN_RANGE(mt.slot_off + x, c.total_slots, c.status)) acc_g[x] = a;
+    const int ps = pos_s[x];
+    if (full && ps <= t - r) {
+      const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
+      const Cand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
+      if (cand_before(cx, best)) best = cx;
+    }
+  }
+  double p_self = 0.0;
+#pragma unroll
+  for (int g = 0; g < G; ++g) p_self += (double)p[cnt * G + g];
+  if (tid == 0 && full && r == 0) {  // without a recent window the new token competes too
+    const Cand cs{(unsigned long long)__double_as_longlong(p_self), t, -2};
+    if (cand_before(cs, best)) best = cs;
+  }
+  best = warp_argmin(best);
+  if (lane == 0) sh.wbest[warp] = best;
+  if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
+  // the new token's K/V row in 16-byte pieces, fetched before the barrier so that the round trip overlaps it
+  uint4 new_row = make_uint4(0, 0, 0, 0);
+  if (warp == 0) new_row = *reinterpret_cast<const uint4*>((lane < 16 ? ku : vu) + (lane & 15) * 8);
+  consumer_sync();
+  if (warp == 0) {
+    const Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+    int slot, ev;
+    if (!full) {
+      slot = cnt;
+      ev = -1;
+    } else if (b.slot == -2) {
+      slot = -1;
+      ev = t;
+    } else if (b.slot >= 0) {
+      slot = b.slot;
+      ev = b.pos;
+    } else {  // a full cache always has a candidate; record instead of corrupting
+      slot = -1;
+      ev = -1;
+      if (lane == 0) atomicCAS(c.status, 0, H2O_ERR_STATE);
+    }
+    if (slot >= 0 && (!H2O_IN_RANGE(slot, B, c.status) || !H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status))) slot = -1;
+    if (lane == 0) {
+      if (!full) c.count[su] = cnt + 1;
+      if (slot >= 0) {
+        c.acc[mt.slot_off + slot] = p_self;
+        c.pos[mt.slot_off + slot] = t;
+      }
+      if (evicted_pos) evicted_pos[u] = ev;
+      c.tpos[su] = t + 1;
+    }
+    if (slot >= 0) {  // the new K/V row goes straight into the freed slot
+      __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(lane < 16 ? c.K : c.V) + (mt.slot_off + slot) * kD + (lane & 15) * 8;
+      *reinterpret_cast<uint4*>(dst) = new_row;
+    }
+  }
+}
+
+size_t ring_smem(int group, int chunk) {
+  return (size_t)kStages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
+}
+
+template <int G>
+cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
+                        void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  static_assert((size_t)2 * kWarps * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
+  const size_t smem = ring_smem(G, chunk);
+  static unsigned long long attr_flags = 0;
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_gqa_ring_kernel<G>), 200 * 1024, &attr_flags);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)c.units);
+  cfg.blockDim = dim3(kThreads + 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_gqa_ring_kernel<G>, c, static_cast<const __nv_bfloat16*>(q),
+                            static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, launch_flags);
+}
+
+}  // namespace
+
+// Does the streaming kernel serve this cache (bf16, head_dim 128, its staging within the shared memory of a block)?
+bool decode_gqa_ring_supported(int dtype, int head_dim, int group, int max_B) {
+  if (dtype != H2O_BF16 || head_dim != kD || (group != 2 && group != 4 && group != 8)) return false;
+  return ring_smem(group, (max_B + 3) & ~3) <= 190 * 1024;
+}
+
+cudaError_t launch_decode_gqa_ring(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
+                                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+                                   cudaStream_t stream) {
+  const int chunk = (max_B + 3) & ~3;
+  const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
+  switch (c.group) {
+    case 2: return launch_ring<2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 4: return launch_ring<4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 8: return launch_ring<8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace h2o

@@ -477,8 +477,8 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
   const cudaError_t e =
       cache->view.group > 1
-          ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, q, k_new, v_new, out, evicted_pos,
-                                   static_cast<cudaStream_t>(stream))
+          ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
+                                   v_new, out, evicted_pos, static_cast<cudaStream_t>(stream))
       : cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
                                                v_new, out, evicted_pos, static_cast<cudaStream_t>(stream))
                       : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, quiescent,
@@ -518,7 +518,8 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
       const size_t off = (size_t)i * step;
       int32_t* ev_i = evicted_pos ? evicted_pos + (size_t)i * cache->view.units : nullptr;
       e = cache->view.group > 1
-              ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, static_cast<const char*>(q) + i * qstep,
+              ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, false, all_units_full(cache),
+                                       static_cast<const char*>(q) + i * qstep,
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
                                        static_cast<char*>(out) + i * qstep, ev_i, st)
           : cache->view.kv4
