@@ -30,9 +30,9 @@ namespace {
 using namespace ptx;
 
 constexpr int kD = 128;
-constexpr int kWarps = 8, kThreads = kWarps * 32;
 constexpr int kTileRows = 32, kRowBytes = kD * 2, kTileBytes = kTileRows * kRowBytes;  // 8 KB
-constexpr int kStages = 8;
+constexpr int kMaxStages = 8;  // ring depth: 8 tiles, or 4 for the four-warp instance (more blocks per SM)
+constexpr int kMaxWarps = 8;
 constexpr uint32_t kSpin = 1u << 22;
 
 __device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
@@ -46,7 +46,8 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+template <int THREADS>
+__device__ __forceinline__ void consumer_sync_n() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
 
 struct Cand {
   unsigned long long key;  // bit pattern of the (non-negative) ranking score
@@ -77,10 +78,10 @@ __device__ __forceinline__ Cand warp_argmin(const Cand& a) {
 }
 
 struct Shared {
-  uint64_t full[kStages], empty[kStages], aux;
-  float part_m[kWarps][8], part_l[kWarps][8];  // per warp and head: softmax partials
+  uint64_t full[kMaxStages], empty[kMaxStages], aux;
+  float part_m[kMaxWarps][8], part_l[kMaxWarps][8];  // per warp and head: softmax partials
   float m[8], inv_l[8];
-  Cand wbest[kWarps];
+  Cand wbest[kMaxWarps];
 };
 
 // D (16 x 8, fp32) += A (16 x 16, bf16, row) * B (16 x 8, bf16, col)
@@ -92,11 +93,15 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-template <int G>
-__global__ void __launch_bounds__(kThreads + 32, 2)
+// NW consumer warps: 8 with an 8-deep ring for launches of at most two blocks per SM, 4 with a 4-deep ring otherwise
+// (four blocks per SM hide one another's passes between the two streams and their serial ends).
+template <int G, int NW>
+__global__ void __launch_bounds__(NW * 32 + 32, NW == 8 ? 2 : 4)
 decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                        int32_t* __restrict__ evicted_pos, int chunk, int launch_flags) {
+  constexpr int kWarps = NW, kThreads = NW * 32, kStages = NW == 8 ? 8 : 4, kStageShift = NW == 8 ? 3 : 2;
+  auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
   // dynamic layout: ring[kStages][tile] (reused for the warps' partial outputs after the stream) |
@@ -185,7 +190,7 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
     // ---- producer warp: one lane keeps the ring full ------------------------------------------------------
     if (lane == 0) {
       for (int T = kStages; T < 2 * nt; ++T) {
-        if (!bar_wait(&sh.empty[T & (kStages - 1)], (uint32_t)((T >> 3) - 1) & 1u)) timed_out = true;
+        if (!bar_wait(&sh.empty[T & (kStages - 1)], (uint32_t)((T >> kStageShift) - 1) & 1u)) timed_out = true;
         issue_tile(T);
       }
       if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
@@ -194,23 +199,23 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   }
 
   // ---- consumer warps -------------------------------------------------------------------------------------
-  // the new token against itself, per query head: warp g does head g with plain arithmetic
-  if (warp < G) {
-    const uint2 rq = *reinterpret_cast<const uint2*>(qu + warp * kD + 4 * lane);
+  // the new token against itself, per query head (the heads go round the warps), with plain arithmetic
+  for (int g = warp; g < G; g += kWarps) {
+    const uint2 rq = *reinterpret_cast<const uint2*>(qu + g * kD + 4 * lane);
     const uint2 rk = *reinterpret_cast<const uint2*>(ku + 4 * lane);
     float part = __uint_as_float(rq.x << 16) * __uint_as_float(rk.x << 16);
     part = fmaf(__uint_as_float(rq.x & 0xffff0000u), __uint_as_float(rk.x & 0xffff0000u), part);
     part = fmaf(__uint_as_float(rq.y << 16), __uint_as_float(rk.y << 16), part);
     part = fmaf(__uint_as_float(rq.y & 0xffff0000u), __uint_as_float(rk.y & 0xffff0000u), part);
     part = warp_sum(part);
-    if (lane == 0) p[cnt * G + warp] = c.scale * part;
+    if (lane == 0) p[cnt * G + g] = c.scale * part;
   }
-  // K pass: block b (16 rows) of the stream goes to warp b % 8; every warp steps through every tile so that
+  // K pass: block b (16 rows) of the stream goes to warp b % NW; every warp steps through every tile so that
   // the ring's barriers see all of them
   for (int j = 0; j < nt; ++j) {
     const int s = j & (kStages - 1);
-    if (!bar_wait(&sh.full[s], (uint32_t)(j >> 3) & 1u)) timed_out = true;
-    const int hb = ((warp - 2 * j) & 7);  // this warp's block of the tile: 0 or 1 (else none)
+    if (!bar_wait(&sh.full[s], (uint32_t)(j >> kStageShift) & 1u)) timed_out = true;
+    const int hb = ((warp - 2 * j) & (kWarps - 1));  // this warp's block of the tile: 0 or 1 (else none)
     if (hb < 2) {
       const unsigned char* kt = ring + (size_t)s * kTileBytes + (size_t)(16 * hb) * kRowBytes;
       float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};  // two chains
@@ -285,7 +290,7 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
     for (int v = 0; v < 8; ++v) o[g][v] = 0.f;
   for (int j = 0; j < nt; ++j) {
     const int T = nt + j, s = T & (kStages - 1);
-    if (!bar_wait(&sh.full[s], (uint32_t)(T >> 3) & 1u)) timed_out = true;
+    if (!bar_wait(&sh.full[s], (uint32_t)(T >> kStageShift) & 1u)) timed_out = true;
     const unsigned char* vt = ring + (size_t)s * kTileBytes;
 #pragma unroll
     for (int ps = 0; ps < kTileRows / (2 * kWarps); ++ps) {
@@ -405,21 +410,22 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   }
 }
 
-size_t ring_smem(int group, int chunk) {
-  return (size_t)kStages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
+size_t ring_smem(int group, int chunk, int stages) {
+  return (size_t)stages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
 }
 
-template <int G>
+template <int G, int NW>
 cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
                         void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  static_assert((size_t)2 * kWarps * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
-  const size_t smem = ring_smem(G, chunk);
+  constexpr int kStages = NW == 8 ? 8 : 4;
+  static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
+  const size_t smem = ring_smem(G, chunk, kStages);
   static unsigned long long attr_flags = 0;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_gqa_ring_kernel<G>), 200 * 1024, &attr_flags);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_gqa_ring_kernel<G, NW>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)c.units);
-  cfg.blockDim = dim3(kThreads + 32);
+  cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute at[1];
@@ -427,9 +433,16 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_gqa_ring_kernel<G>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_gqa_ring_kernel<G, NW>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, launch_flags);
+}
+
+template <int G>
+cudaError_t launch_ring_g(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
+                          void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  if (c.units <= 2 * sm_count()) return launch_ring<G, 8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_ring<G, 4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace
@@ -437,7 +450,7 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
 // Does the streaming kernel serve this cache (bf16, head_dim 128, its staging within the shared memory of a block)?
 bool decode_gqa_ring_supported(int dtype, int head_dim, int group, int max_B) {
   if (dtype != H2O_BF16 || head_dim != kD || (group != 2 && group != 4 && group != 8)) return false;
-  return ring_smem(group, (max_B + 3) & ~3) <= 190 * 1024;
+  return ring_smem(group, (max_B + 3) & ~3, kMaxStages) <= 190 * 1024;
 }
 
 cudaError_t launch_decode_gqa_ring(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
@@ -446,9 +459,9 @@ cudaError_t launch_decode_gqa_ring(const CacheView& c, int max_B, bool cache_is_
   const int chunk = (max_B + 3) & ~3;
   const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
   switch (c.group) {
-    case 2: return launch_ring<2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-    case 4: return launch_ring<4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-    case 8: return launch_ring<8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 2: return launch_ring_g<2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 4: return launch_ring_g<4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 8: return launch_ring_g<8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
     default: return cudaErrorInvalidValue;
   }
 }
