@@ -482,6 +482,48 @@ class ConfigRun:
         return {"us_per_launch": us, "bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
                 "speedup_vs_bf16_slots": bf16_launch_us / us, "layer_caches": Lk}
 
+    def gqa_figure(self, G=4):
+        """Grouped-query attention on the same tensors: the workload's heads are the query heads, every G of them
+        share one K/V head (the first H / G heads of the K and V inputs), i.e. units = batch x H / G.  One layer's
+        prefill-select and the decode steps, rotating over (up to 8) layer caches."""
+        wl, pkg = self.wl, self.pkg
+        if not (wl.dtype == "bf16" and self.d == 128 and self.H % G == 0):
+            return None
+        Hk = self.H // G
+        Lk = min(self.L, 8)
+        kc = [pkg.H2OCache(wl.batch, Hk, self.d, "bf16", wl.heavy, wl.recent, device=self.local, query_group=G) for _ in range(Lk)]
+        pre_ms = []
+        for l in range(Lk):
+            q, k, v = self.prompts[l] if self.resident else self._draw_prompt(l)
+            kk, vv = k[:, :Hk].contiguous(), v[:, :Hk].contiguous()
+            out = self.outs[l if self.resident else 0]
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(self.stream)
+            kc[l].prefill_select(q, kk, vv, self.cu, out, self.stream)
+            b.record(self.stream)
+            torch.cuda.synchronize(self.dev)
+            pre_ms.append(a.elapsed_time(b))
+            del kk, vv
+        n_k = min(32, self.S)
+        dk = [[self.dec[l][1][s][:, :Hk].contiguous() for s in range(n_k)] for l in range(Lk)]
+        dv = [[self.dec[l][2][s][:, :Hk].contiguous() for s in range(n_k)] for l in range(Lk)]
+        ev = torch.empty(wl.batch, Hk, dtype=torch.int32, device=self.dev)
+
+        def loop():
+            for s in range(n_k):
+                for l in range(Lk):
+                    d_ = self.dec[l]
+                    kc[l].decode_step(d_[0][s], dk[l][s], dv[l][s], d_[3][s], ev, self.stream)
+
+        us = self.graph_replay_us(loop, n_k * Lk)
+        for c in kc:
+            assert c.status() == 0, "device status word set"
+            c.close()
+        nbytes = sum(decode_bytes_per_unit_step(c_, self.d, self.esize) + 2 * (G - 1) * self.d * self.esize for c_ in slot_counts(wl)) * Hk
+        return {"query_group": G, "kv_heads": Hk, "units": wl.batch * Hk, "us_per_launch": us, "bytes_per_launch": nbytes,
+                "achieved_gbs": nbytes / (us * 1e-6) / 1e9, "frac_of_measured_hbm": nbytes / (us * 1e-6) / 1e9 / _peaks()["hbm_gbs"],
+                "prefill_select_ms_per_layer": float(np.median(pre_ms)), "layer_caches": Lk}
+
     def topk_figure(self, m=64):
         """The same decode steps with "Top-K" attention (each query attends its m largest logits): the kernel streams
         the keys only and reads m value rows per unit; rotating over (up to 8) layer caches."""
@@ -659,6 +701,7 @@ def measure_config(pkg, wl, layers, dev, local, rank, world, dist, args, steps, 
         rec["decode_kv4_slots"] = run.kv4_figure(launch_us)
         if headline or args.context:
             rec["decode_topk_attention"] = run.topk_figure()
+            rec["grouped_query_attention"] = run.gqa_figure()
     e2e = None
     if not args.no_e2e and (headline or args.e2e_all):
         e = run.e2e(max(1, min(steps, 2)))
@@ -757,7 +800,7 @@ def main():
         }
         for key in ("prefill_ms", "decode_ms", "decode_only_seq_heads_per_s", "prefill_tflops_algorithmic",
                     "wall_ms_per_step_with_input_generation", "clocks", "roofline", "roofline_prefill",
-                    "decode_chunk_one_layer", "decode_kv4_slots", "decode_topk_attention", "e2e"):
+                    "decode_chunk_one_layer", "decode_kv4_slots", "decode_topk_attention", "grouped_query_attention", "e2e"):
             if key in rec:
                 out[key] = rec[key]
         if per_config:
