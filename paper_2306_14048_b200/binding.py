@@ -45,6 +45,7 @@ EXPORTED = (
     "h2o_cache_status",
     "h2o_cache_set_decode_shape",
     "h2o_cache_set_prefill_path",
+    "h2o_cache_set_decode_path",
     "h2o_debug_set_early_prefetch",
     "h2o_prefill_scratch_layout",
     "h2o_strerror",
@@ -120,6 +121,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_set_decode_shape.restype = c.c_int
     lib.h2o_cache_set_decode_shape.argtypes = [vp, c.c_int32, c.c_int32]
     lib.h2o_cache_set_prefill_path.restype = c.c_int
+    lib.h2o_cache_set_decode_path.restype = c.c_int
+    lib.h2o_cache_set_decode_path.argtypes = [vp, c.c_int32]
     lib.h2o_cache_set_prefill_path.argtypes = [vp, c.c_int32]
     lib.h2o_prefill_scratch_layout.restype = c.c_int
     lib.h2o_prefill_scratch_layout.argtypes = [cfgp, c.c_int64, c.POINTER(c.c_size_t)]
@@ -317,6 +320,9 @@ class H2OCache:
         creates the CUDA handle lazily), for the next prefill_select call."""
         arr = (ctypes.c_void_p * 4)(*[int(e.cuda_event) for e in events])
         _check(lib.h2o_debug_set_prefill_events(self._h, arr), "h2o_debug_set_prefill_events")
+
+    def set_decode_path(self, path: int):
+        _check(lib.h2o_cache_set_decode_path(self._h, int(path)), "h2o_cache_set_decode_path")
 
     def set_prefill_path(self, path: int):
         _check(lib.h2o_cache_set_prefill_path(self._h, int(path)), "h2o_cache_set_prefill_path")

@@ -11,7 +11,7 @@
 // does head g), a V pass (G weighted sums per loaded row), then the usual tail: fp64 accumulation, victim search by
 // (score, position), in-place write of the new row.  Plain 16-byte loads, four rows in flight per half warp; this
 // kernel is the plain variant of the step for every dtype and head size (no bulk-copy ring, no cluster split);
-// bf16 / head_dim 128 caches whose staging fits take the streaming kernel of decode_gqa_ring.cu instead.
+// bf16 / head_dim 128 caches whose staging fits take the streaming kernel of decode_two_pass.cu instead.
 #include <climits>
 
 #include "h2o_internal.cuh"
@@ -309,8 +309,8 @@ size_t decode_gqa_smem_bytes(int group, int max_B, int head_dim) {
 
 cudaError_t launch_decode_gqa(const CacheView& c, int dtype, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
                               const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  if (decode_gqa_ring_supported(dtype, c.head_dim, c.group, max_B))
-    return launch_decode_gqa_ring(c, max_B, cache_is_quiescent, all_full, q, k_new, v_new, out, evicted_pos, stream);
+  if (decode_two_pass_supported(dtype, c.head_dim, c.group, max_B))
+    return launch_decode_two_pass(c, max_B, cache_is_quiescent, all_full, q, k_new, v_new, out, evicted_pos, stream);
   if (dtype == H2O_F32) {
     if (c.head_dim == 64) return launch_td<float, 64>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
     return launch_td<float, 128>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);

@@ -1,9 +1,14 @@
-// Fused decode step for grouped-query attention, bf16 / head_dim 128: the streaming form of decode_gqa.cu.
+// Fused decode step in two streaming passes, bf16 / head_dim 128, for G query heads per (sequence, K/V head) unit:
+// G = 1 is plain multi-head attention (Algorithm 2's loop body, as decode.cu: scores over the occupied slots,
+// softmax, weighted values, accumulated score += probability, victim, in-place write), G = 2, 4, 8 is
+// grouped-query attention, the streaming form of decode_gqa.cu.  The grouped reading is this library's own (the
+// paper evicts per head): every query head has its own softmax over the unit's entries, a key's accumulated score
+// grows by the sum of the G probabilities (the accumulation once per query head), one victim per unit.
 //
-// Same reading as there (own, not in the paper, which evicts per head): G query heads share the keys and values of
-// one (sequence, K/V head) unit, every query head has its own softmax over the unit's entries, a key's accumulated
-// score grows by the sum of the G probabilities (Algorithm 2's accumulation once per query head), one victim per
-// unit.
+// Against the online-softmax kernel of decode.cu this one reads K completely before V: the softmax is exact when
+// the values arrive, so the V pass has no running maximum to follow and no rescaling, and the scores come from the
+// tensor cores without a shuffle; the price is the pass in between and the scores of all rows in shared memory.
+// It is the faster one for launches of many waves of mid-sized and large units; it has no cluster split.
 //
 // Shape: one thread block per unit, eight consumer warps and a producer warp.  The producer streams the unit's K
 // rows and then its V rows as 8 KB tiles (32 rows) through one bulk-copy ring, so HBM stays busy across the two
@@ -97,7 +102,7 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
 // (four blocks per SM hide one another's passes between the two streams and their serial ends).
 template <int G, int NW>
 __global__ void __launch_bounds__(NW * 32 + 32, NW == 8 ? 2 : 4)
-decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
+decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                        int32_t* __restrict__ evicted_pos, int chunk, int launch_flags) {
   constexpr int kWarps = NW, kThreads = NW * 32, kStages = NW == 8 ? 8 : 4, kStageShift = NW == 8 ? 3 : 2;
@@ -228,7 +233,12 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       }
       // lane (gl, c4): rows gl and gl + 8 of the block, heads 2 c4 and 2 c4 + 1 (rows past the end hold stale bytes)
       const int rowA = j * kTileRows + 16 * hb + gl, rowB = rowA + 8;
-      if (2 * c4 < G) {
+      if constexpr (G == 1) {
+        if (c4 == 0) {
+          if (rowA < cnt) p[rowA] = c.scale * (d0[0] + d1[0]);
+          if (rowB < cnt) p[rowB] = c.scale * (d0[2] + d1[2]);
+        }
+      } else if (2 * c4 < G) {
         if (rowA < cnt) *reinterpret_cast<float2*>(p + rowA * G + 2 * c4) = make_float2(c.scale * (d0[0] + d1[0]), c.scale * (d0[1] + d1[1]));
         if (rowB < cnt) *reinterpret_cast<float2*>(p + rowB * G + 2 * c4) = make_float2(c.scale * (d0[2] + d1[2]), c.scale * (d0[3] + d1[3]));
       }
@@ -299,7 +309,9 @@ decode_gqa_ring_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
         float vf[8];
         Vec16<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(vt + rl * kRowBytes + 16 * ch), vf);
         float pr[G];
-        if constexpr (G == 2) {
+        if constexpr (G == 1) {
+          pr[0] = p[row];
+        } else if constexpr (G == 2) {
           const float2 p2 = *reinterpret_cast<const float2*>(p + row * G);
           pr[0] = p2.x;
           pr[1] = p2.y;
@@ -421,7 +433,7 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
   static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
   const size_t smem = ring_smem(G, chunk, kStages);
   static unsigned long long attr_flags = 0;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_gqa_ring_kernel<G, NW>), 200 * 1024, &attr_flags);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)c.units);
@@ -433,7 +445,7 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_gqa_ring_kernel<G, NW>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, launch_flags);
 }
@@ -448,17 +460,18 @@ cudaError_t launch_ring_g(const CacheView& c, int chunk, int launch_flags, const
 }  // namespace
 
 // Does the streaming kernel serve this cache (bf16, head_dim 128, its staging within the shared memory of a block)?
-bool decode_gqa_ring_supported(int dtype, int head_dim, int group, int max_B) {
-  if (dtype != H2O_BF16 || head_dim != kD || (group != 2 && group != 4 && group != 8)) return false;
+bool decode_two_pass_supported(int dtype, int head_dim, int group, int max_B) {
+  if (dtype != H2O_BF16 || head_dim != kD || (group != 1 && group != 2 && group != 4 && group != 8)) return false;
   return ring_smem(group, (max_B + 3) & ~3, kMaxStages) <= 190 * 1024;
 }
 
-cudaError_t launch_decode_gqa_ring(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
+cudaError_t launch_decode_two_pass(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
                                    const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                                    cudaStream_t stream) {
   const int chunk = (max_B + 3) & ~3;
   const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
   switch (c.group) {
+    case 1: return launch_ring_g<1>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
     case 2: return launch_ring_g<2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
     case 4: return launch_ring_g<4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
     case 8: return launch_ring_g<8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);

@@ -3,7 +3,6 @@
 // allocated here; everything lives in the caller's workspace / scratch.
 #include <algorithm>
 #include <cmath>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -130,6 +129,8 @@ struct h2o_cache {
   int split, chunk, stages;
   int prefill_path;  // 0 = automatic, 1 = force the ALU kernels
   int chunk_path;    // 0 = automatic, 1 = force one decode-step kernel per token in h2o_decode_chunk
+  int decode_path;   // 0 = automatic, 1 = the online-softmax step kernel, 2 = the two-pass streaming kernel
+  double mean_budget;  // mean of k + r over the sequences
   // tokens every unit of sequence s has been given (prompt + decode steps); < 0: unknown (attached cache)
   std::vector<int64_t> seen;
   Layout layout;
@@ -288,6 +289,12 @@ static int create_impl(h2o_cache_t** out, const h2o_config_t* cfg, void* dev_wor
   c->stages = 0;
   c->prefill_path = 0;
   c->chunk_path = 0;
+  c->decode_path = 0;
+  {
+    double sum = 0.0;
+    for (int s2 = 0; s2 < cfg->batch; ++s2) sum += (double)cfg->heavy_budget[s2] + cfg->recent_window[s2];
+    c->mean_budget = sum / cfg->batch;
+  }
   c->chunk = (((L.max_B + split - 1) / split) + 3) & ~3;
 
   char* ws = static_cast<char*>(dev_workspace);
@@ -465,6 +472,23 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
   return H2O_OK;
 }
 
+namespace {
+// Which kernel serves a multi-head decode step.  The two-pass streaming kernel (K stream with the scores on
+// mma.sync, exact softmax, V stream; decode_two_pass.cu with one query head per unit) is faster than the
+// online-softmax kernel on launches of many waves of mid-sized and large units (4096 ragged units of 26..820
+// slots: 148 -> 140.5 us; 512 units of 410 slots: 28.1 -> 20.9 us) and slower on small units (3584 units of 104
+// slots: 44.2 -> 53.9 us), equal on 256 units of 410 slots; it has no cluster split, sparse pattern or "Top-K" form.
+bool two_pass_supported(const h2o_cache* cache) {
+  return cache->view.group == 1 && !cache->view.kv4 && cache->view.mask_kind == 0 && cache->view.topk == 0 &&
+         h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->layout.max_B);
+}
+bool two_pass_step(const h2o_cache* cache) {
+  if (cache->decode_path == 1 || !two_pass_supported(cache)) return false;
+  if (cache->decode_path == 2) return true;
+  return cache->split == 1 && cache->view.units > 2 * h2o::sm_count() && cache->mean_budget >= 224.0;
+}
+}  // namespace
+
 int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const void* v_new, void* out,
                     int32_t* evicted_pos, void* stream) {
   if (!cache || !q || !k_new || !v_new || !out) return H2O_ERR_INVALID_ARG;
@@ -475,8 +499,11 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   if (!guard.ok) return H2O_ERR_CUDA;
   // the cache workspace is the identity: two handles on one workspace must count as the same cache
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
+  const bool ring1 = two_pass_step(cache);
   const cudaError_t e =
-      cache->view.group > 1
+      ring1 ? h2o::launch_decode_two_pass(cache->view, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new, v_new, out,
+                                          evicted_pos, static_cast<cudaStream_t>(stream))
+      : cache->view.group > 1
           ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
                                    v_new, out, evicted_pos, static_cast<cudaStream_t>(stream))
       : cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
@@ -522,6 +549,10 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
                                        static_cast<const char*>(q) + i * qstep,
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
                                        static_cast<char*>(out) + i * qstep, ev_i, st)
+          : two_pass_step(cache)
+              ? h2o::launch_decode_two_pass(cache->view, cache->layout.max_B, false, all_units_full(cache),
+                                            static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
+                                            static_cast<const char*>(v) + off, static_cast<char*>(out) + off, ev_i, st)
           : cache->view.kv4
               ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, false, all_units_full(cache), static_cast<const char*>(q) + off,
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
@@ -582,6 +613,13 @@ int h2o_cache_fscore(h2o_cache_t* cache, int32_t hkind, double* out_dev, void* s
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
+  return H2O_OK;
+}
+
+int h2o_cache_set_decode_path(h2o_cache_t* cache, int32_t path) {
+  if (!cache || path < 0 || path > 2) return H2O_ERR_INVALID_ARG;
+  if (path == 2 && !two_pass_supported(cache)) return H2O_ERR_UNSUPPORTED;
+  cache->decode_path = path;
   return H2O_OK;
 }
 

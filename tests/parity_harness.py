@@ -97,7 +97,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
                export_every: int = 32, layer: int = 0, prefill: bool = True, scale: float = 0.0,
                device: str = "cuda", prefill_path: int = 0, chunk: int = 0, chunk_path: int = 0,
                pattern: Optional[Sequence[int]] = None, score_mode: int = 0, static_scratch: bool = False,
-               mask: Optional[Sequence[int]] = None, split: int = 0, topk: int = 0, group: int = 1) -> ParityStats:
+               mask: Optional[Sequence[int]] = None, split: int = 0, topk: int = 0, group: int = 1,
+               decode_path: int = 0) -> ParityStats:
     """Run prefill-select (optional) and ``steps`` decode steps on both sides, comparing as it goes.
 
     The CUDA path always processes the whole workload; the oracle mirrors only the sampled ``units``
@@ -106,6 +107,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
     while the oracle still takes them one decode step at a time.  ``pattern`` cycles through call
     sizes instead: 0 = one h2o_decode_step call, n > 0 = one h2o_decode_chunk call of n tokens.
     ``split``: thread blocks (one cluster) per unit in the decode kernel, 0 = the library's choice.
+    ``decode_path``: h2o_cache_set_decode_path (0 automatic, 1 online-softmax kernel, 2 two-pass streaming kernel).
     ``group`` > 1: grouped-query attention: wl.n_heads counts the K/V heads, q and out carry n_heads * group query heads
     (drawn from the same recipe with that many heads).
     ``topk`` > 0: "Top-K" attention in decode steps on both sides (h2o_cache_set_topk); a unit whose weakest kept and
@@ -117,7 +119,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         h2o_oracle.set_topk(topk)
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
-                              chunk, chunk_path, pattern, score_mode, static_scratch, mask, split, topk=-topk, group=group)
+                              chunk, chunk_path, pattern, score_mode, static_scratch, mask, split, topk=-topk, group=group, decode_path=decode_path)
         finally:
             h2o_oracle.set_topk(0)
     topk = -topk  # (negative: the oracle already has it)
@@ -128,7 +130,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
                               chunk, chunk_path, pattern, score_mode, static_scratch, mask=(0,) + tuple(mask), split=split,
-                              topk=-topk, group=group)
+                              topk=-topk, group=group, decode_path=decode_path)
         finally:
             h2o_oracle.set_mask(0)
     if score_mode > 0:  # the oracle's ranking rule is process-wide: always put it back
@@ -136,7 +138,7 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         try:
             return run_parity(wl, gpu_cache_cls, units, steps, export_every, layer, prefill, scale, device, prefill_path,
                               chunk, chunk_path, pattern, score_mode=0 - score_mode, static_scratch=static_scratch, mask=mask,
-                              split=split, topk=-topk, group=group)
+                              split=split, topk=-topk, group=group, decode_path=decode_path)
         finally:
             h2o_oracle.set_score_mode(0)
     score_mode = -score_mode  # (negative: the oracle is already in that mode)
@@ -153,6 +155,8 @@ def run_parity(wl: Workload, gpu_cache_cls, units: Optional[Sequence[int]] = Non
         if G > 1 else gpu_cache_cls(wl.batch, H, d, wl.dtype, wl.heavy, wl.recent, softmax_scale=scale, device=0)
     gpu.set_prefill_path(prefill_path)
     gpu.set_decode_shape(split, 0)
+    if decode_path:
+        gpu.set_decode_path(decode_path)
     if topk > 0:
         gpu.set_topk(topk)
     gpu.set_score_mode(score_mode)

@@ -105,3 +105,26 @@ def test_config5_ragged_stress_scale(H2OCache):
     wl = CONFIGS["c5_ragged_32layer"]
     record(run_parity(wl, H2OCache, units=_c5_units(wl, per_class=1), export_every=32, layer=7, scale=_stress_scale(wl)),
            "c5 layer 7 scale x4")
+
+
+def test_config5_ragged_online_softmax_kernel(H2OCache):
+    """Config 5 takes the two-pass streaming step kernel by default (the cases above); the same steps on the
+    online-softmax kernel."""
+    from parity_harness import record, run_parity
+
+    wl = CONFIGS["c5_ragged_32layer"]
+    record(run_parity(wl, H2OCache, units=_c5_units(wl, per_class=1), export_every=32, layer=0, decode_path=1),
+           "c5 layer 0, online-softmax kernel")
+
+
+def test_config5_ragged_grouped_query(H2OCache):
+    """Config 5's sequences with 8 K/V heads of 4 query heads each (1024 units): tensor-core prompt kernels over the
+    group, the streaming grouped step kernel, every decode step."""
+    from parity_harness import record, run_parity
+
+    wl = CONFIGS["c5_ragged_32layer"].scaled(n_heads=8)
+    lens = np.asarray(wl.prompt_lens)
+    seqs = [int(np.argmin(lens)), int(np.argmax(lens)), int(np.argsort(lens)[len(lens) // 2])]
+    units = [s * wl.n_heads + h for s, h in zip(seqs, (0, 5, 7))]
+    record(run_parity(wl, H2OCache, units=units, export_every=32, layer=0, group=4), "c5 with 8 K/V heads x 4 query heads")
+

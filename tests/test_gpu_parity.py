@@ -531,3 +531,39 @@ def test_grouped_query_attention_argument_errors(H2OCache):
     assert pkg.lib.h2o_cache_set_mask(cache._h, 1, 4, 2) == pkg.H2O_ERR_UNSUPPORTED
     assert pkg.lib.h2o_cache_set_topk(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
     cache.close()
+
+# ---------------------------------------------------------------------------------------------------------
+# the two-pass streaming step kernel (h2o_cache_set_decode_path 2; automatic for many mid-sized units)
+# ---------------------------------------------------------------------------------------------------------
+def test_two_pass_step_kernel_ragged_fill_phase_and_edges(H2OCache):
+    """Ragged batch over several tiles with a prompt shorter than its budget (fill phase), token-by-token from an
+    empty cache, no recent window, no heavy budget, the averaged ranking, and the chunk call's per-token fallback."""
+    from parity_harness import run_parity
+
+    wl = _wl("tp", 4, 3, 128, "bf16", [300, 77, 513, 40], 48, [20, 9, 33, 30], [24, 5, 31, 30], seed=205)
+    for path in (1, 2):
+        print(run_parity(wl, H2OCache, export_every=8, decode_path=path))
+    print(run_parity(wl, H2OCache, export_every=8, decode_path=2, score_mode=1))
+    print(run_parity(wl, H2OCache, export_every=8, decode_path=2, chunk=16, chunk_path=1))
+    for heavy, recent in (([0, 0], [7, 16]), ([5, 12], [0, 0]), ([6, 1], [12, 9])):
+        wl = _wl("tpedge", 2, 2, 128, "bf16", [1, 1], 60, heavy, recent, seed=36)
+        print(run_parity(wl, H2OCache, prefill=False, export_every=5, decode_path=2))
+    wl = _wl("tplong", 1, 2, 128, "bf16", [3000], 12, [1200], [1100], seed=207)  # 72 tiles per matrix
+    print(run_parity(wl, H2OCache, export_every=4, decode_path=2))
+
+
+def test_two_pass_step_kernel_where_it_does_not_apply(H2OCache):
+    import paper_2306_14048_b200 as pkg
+
+    for args in ((1, 2, 64, "bf16"), (1, 2, 128, "f32"), (1, 2, 128, "bf16_kv4")):
+        cache = H2OCache(args[0], args[1], args[2], args[3], [8], [8])
+        assert pkg.lib.h2o_cache_set_decode_path(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
+        assert pkg.lib.h2o_cache_set_decode_path(cache._h, 3) == pkg.H2O_ERR_INVALID_ARG
+        assert pkg.lib.h2o_cache_set_decode_path(cache._h, 1) == pkg.H2O_OK
+        cache.close()
+    cache = H2OCache(1, 2, 128, "bf16", [8], [8])
+    cache.set_mask(1, 4, 2)
+    assert pkg.lib.h2o_cache_set_decode_path(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
+    cache.set_mask(0, 1, 0)
+    cache.set_decode_path(2)
+    cache.close()
