@@ -660,7 +660,7 @@ def measure_config(pkg, wl, layers, dev, local, rank, world, dist, args, steps, 
         "wall_ms_per_step_with_input_generation": wall_ms / steps,
         "clocks": clocks,
         "roofline": {
-            "kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "kernel": "decode_two_pass_kernel" if run.caches[0].decode_path() == 2 else "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": ncu_decode_traffic(wl),
             "bytes_per_launch": bytes_launch, "avg_launch_us": launch_us, "min_launch_us": dec_min * 1e3 / (S * L),
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,

@@ -282,6 +282,10 @@ int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
  * whose mean budget is at least 224 slots.
  */
 int h2o_cache_set_decode_path(h2o_cache_t* cache, int32_t path);
+/* The kind of kernel the next h2o_decode_step of this cache launches: 2 = two streaming passes, 1 = one pass
+ * (online softmax; for 4-bit slots and for grouped caches outside the streaming kernel's reach: their own
+ * one-block-per-unit kernels).  Negative: H2O_ERR_INVALID_ARG (null handle). */
+int h2o_cache_get_decode_path(h2o_cache_t* cache);
 /* h2o_decode_chunk: 0 = automatic (chunk kernel where it applies), 1 = one decode-step kernel per token. */
 int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path);
 /*

@@ -46,6 +46,7 @@ EXPORTED = (
     "h2o_cache_set_decode_shape",
     "h2o_cache_set_prefill_path",
     "h2o_cache_set_decode_path",
+    "h2o_cache_get_decode_path",
     "h2o_debug_set_early_prefetch",
     "h2o_prefill_scratch_layout",
     "h2o_strerror",
@@ -122,6 +123,8 @@ def _load() -> ctypes.CDLL:
     lib.h2o_cache_set_decode_shape.argtypes = [vp, c.c_int32, c.c_int32]
     lib.h2o_cache_set_prefill_path.restype = c.c_int
     lib.h2o_cache_set_decode_path.restype = c.c_int
+    lib.h2o_cache_get_decode_path.restype = c.c_int
+    lib.h2o_cache_get_decode_path.argtypes = [vp]
     lib.h2o_cache_set_decode_path.argtypes = [vp, c.c_int32]
     lib.h2o_cache_set_prefill_path.argtypes = [vp, c.c_int32]
     lib.h2o_prefill_scratch_layout.restype = c.c_int
@@ -323,6 +326,9 @@ class H2OCache:
 
     def set_decode_path(self, path: int):
         _check(lib.h2o_cache_set_decode_path(self._h, int(path)), "h2o_cache_set_decode_path")
+
+    def decode_path(self) -> int:
+        return int(lib.h2o_cache_get_decode_path(self._h))
 
     def set_prefill_path(self, path: int):
         _check(lib.h2o_cache_set_prefill_path(self._h, int(path)), "h2o_cache_set_prefill_path")

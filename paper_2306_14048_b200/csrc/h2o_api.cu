@@ -623,6 +623,13 @@ int h2o_cache_set_decode_path(h2o_cache_t* cache, int32_t path) {
   return H2O_OK;
 }
 
+int h2o_cache_get_decode_path(h2o_cache_t* cache) {
+  if (!cache) return H2O_ERR_INVALID_ARG;
+  if (cache->view.group > 1)
+    return h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->view.group, cache->layout.max_B) ? 2 : 1;
+  return two_pass_step(cache) ? 2 : 1;
+}
+
 int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path) {
   if (!cache || (path != 0 && path != 1)) return H2O_ERR_INVALID_ARG;
   cache->chunk_path = path;
