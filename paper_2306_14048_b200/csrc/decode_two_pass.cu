@@ -99,13 +99,15 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
 }
 
 // NW consumer warps: 8 with an 8-deep ring for launches of at most two blocks per SM, 4 with a 4-deep ring otherwise
-// (four blocks per SM hide one another's passes between the two streams and their serial ends).
-template <int G, int NW>
-__global__ void __launch_bounds__(NW * 32 + 32, NW == 8 ? 2 : 4)
+// (four blocks per SM hide one another's passes between the two streams and their serial ends).  For few units
+// neither four warps per block (256 units of 410 slots: 15.4 us against 12.3) nor eight warps capped at 56
+// registers with a 4-deep ring, so that the next launch's blocks are resident beside this launch's (14.4 us), helped.
+template <int G, int NW, int STAGES, int MINB>
+__global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                        int32_t* __restrict__ evicted_pos, int chunk, int launch_flags) {
-  constexpr int kWarps = NW, kThreads = NW * 32, kStages = NW == 8 ? 8 : 4, kStageShift = NW == 8 ? 3 : 2;
+  constexpr int kWarps = NW, kThreads = NW * 32, kStages = STAGES, kStageShift = STAGES == 8 ? 3 : 2;
   auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
@@ -426,14 +428,15 @@ size_t ring_smem(int group, int chunk, int stages) {
   return (size_t)stages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
 }
 
-template <int G, int NW>
+template <int G, int NW, int STAGES, int MINB>
 cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
                         void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  constexpr int kStages = NW == 8 ? 8 : 4;
+  constexpr int kStages = STAGES;
+  static_assert(STAGES == 4 || STAGES == 8, "ring depth");
   static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
   const size_t smem = ring_smem(G, chunk, kStages);
   static unsigned long long attr_flags = 0;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW>), 200 * 1024, &attr_flags);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)c.units);
@@ -445,7 +448,7 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, launch_flags);
 }
@@ -453,8 +456,8 @@ cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const v
 template <int G>
 cudaError_t launch_ring_g(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
                           void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  if (c.units <= 2 * sm_count()) return launch_ring<G, 8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-  return launch_ring<G, 4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  if (c.units <= 2 * sm_count()) return launch_ring<G, 8, 8, 2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_ring<G, 4, 4, 4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace
