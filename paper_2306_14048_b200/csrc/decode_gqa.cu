@@ -310,7 +310,7 @@ size_t decode_gqa_smem_bytes(int group, int max_B, int head_dim) {
 cudaError_t launch_decode_gqa(const CacheView& c, int dtype, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
                               const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   if (decode_two_pass_supported(dtype, c.head_dim, c.group, max_B))
-    return launch_decode_two_pass(c, max_B, cache_is_quiescent, all_full, q, k_new, v_new, out, evicted_pos, stream);
+    return launch_decode_two_pass(c, 1, (max_B + 3) & ~3, cache_is_quiescent, all_full, q, k_new, v_new, out, evicted_pos, stream);
   if (dtype == H2O_F32) {
     if (c.head_dim == 64) return launch_td<float, 64>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);
     return launch_td<float, 128>(c, max_B, q, k_new, v_new, out, evicted_pos, stream);

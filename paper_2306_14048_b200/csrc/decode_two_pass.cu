@@ -8,7 +8,9 @@
 // Against the online-softmax kernel of decode.cu this one reads K completely before V: the softmax is exact when
 // the values arrive, so the V pass has no running maximum to follow and no rescaling, and the scores come from the
 // tensor cores without a shuffle; the price is the pass in between and the scores of all rows in shared memory.
-// It is the faster one for launches of many waves of mid-sized and large units; it has no cluster split.
+// It is the faster one for launches of many waves of mid-sized and large units.  A unit can be split over the
+// blocks of a cluster (few long units): statistics are exchanged between the passes, partial outputs and victim
+// candidates in one exchange after the value pass.
 //
 // Shape: one thread block per unit, eight consumer warps and a producer warp.  The producer streams the unit's K
 // rows and then its V rows as 8 KB tiles (32 rows) through one bulk-copy ring, so HBM stays busy across the two
@@ -23,16 +25,21 @@
 // Tail as in the other step kernels: fp64 accumulation of the summed probabilities, victim by (score, position),
 // new row written into the freed slot.  Every wait on an mbarrier is bounded (H2O_ERR_TIMEOUT in the status word).
 #include <climits>
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "h2o_internal.cuh"
 #include "sm100_ptx.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace h2o {
 
 namespace {
 
 using namespace ptx;
+
+constexpr int kMaxSplit = 8;
 
 constexpr int kD = 128;
 constexpr int kTileRows = 32, kRowBytes = kD * 2, kTileBytes = kTileRows * kRowBytes;  // 8 KB
@@ -87,6 +94,12 @@ struct Shared {
   float part_m[kMaxWarps][8], part_l[kMaxWarps][8];  // per warp and head: softmax partials
   float m[8], inv_l[8];
   Cand wbest[kMaxWarps];
+  // Cluster exchange (a unit split over the blocks of a cluster): every block pushes its values into its peers'
+  // shared memory with remote stores, then one cluster barrier makes them visible.
+  float x_m[kMaxSplit][8], x_l[kMaxSplit][8];  // softmax statistics of every rank and head (written by that rank)
+  Cand x_cand[kMaxSplit];                      // rank 0 only: every rank's eviction candidate
+  // (the partial outputs pushed to rank 0, [kMaxSplit][G][kD] floats, live in dynamic shared memory and exist
+  //  only in launches that split a unit)
 };
 
 // D (16 x 8, fp32) += A (16 x 16, bf16, row) * B (16 x 8, bf16, col)
@@ -106,7 +119,7 @@ template <int G, int NW, int STAGES, int MINB>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                       int32_t* __restrict__ evicted_pos, int chunk, int launch_flags) {
+                       int32_t* __restrict__ evicted_pos, int split, int chunk, int launch_flags) {
   constexpr int kWarps = NW, kThreads = NW * 32, kStages = STAGES, kStageShift = STAGES == 8 ? 3 : 2;
   auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -118,9 +131,16 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   int32_t* pos_s = reinterpret_cast<int32_t*>(acc_s + chunk);
   float* p = reinterpret_cast<float*>(pos_s + chunk);
   float* red = reinterpret_cast<float*>(ring);  // [2 * kWarps][G][kD]
+  float* x_out = p + (size_t)(chunk + 4) * G;   // [kMaxSplit][G][kD], only when split > 1
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int su = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = split > 1 ? (int)cluster.block_rank() : 0;
+  // Early arrival on the cluster barrier; the matching wait comes right before the first remote store, by which
+  // time every block of the cluster has long started (its shared memory exists).
+  if (split > 1) cluster.barrier_arrive();
+  const int su = blockIdx.x / split;  // launch position of the unit; the block owns rows lo .. lo + chunk - 1 of it
+  const int lo = rank * chunk;
   const UnitMeta mt = c.meta[su];
   // Programmatic dependent launch, as in the multi-head step kernel: the inputs may come from the previous kernel
   // of the stream and are read after griddepcontrol.wait; the cache is written by this library alone, and when the
@@ -133,17 +153,17 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
-  int cnt = all_full ? 0 : c.count[su];
+  int cnt_u = all_full ? 0 : c.count[su];  // entries of the unit
   const int t = c.tpos[su];
-  int nstr = all_full ? min(B, chunk) : cnt;  // rows to stream
-  if (!H2O_IN_RANGE(u, c.units, c.status) || !H2O_IN_RANGE(nstr, min(B, chunk) + 1, c.status) ||
-      !H2O_IN_RANGE(mt.slot_off + (nstr > 0 ? nstr - 1 : 0), c.total_slots, c.status))
+  int nstr = all_full ? max(0, min(min(B, split * chunk) - lo, chunk)) : max(0, min(cnt_u - lo, chunk));  // rows to stream
+  if (!H2O_IN_RANGE(u, c.units, c.status) || !H2O_IN_RANGE(nstr, chunk + 1, c.status) ||
+      (nstr > 0 && !H2O_IN_RANGE(mt.slot_off + lo + nstr - 1, c.total_slots, c.status)))
     nstr = 0;
   const int nt = (nstr + kTileRows - 1) / kTileRows;  // tiles per matrix; the stream is K 0..nt-1, then V 0..nt-1
-  const __nv_bfloat16* Kb = reinterpret_cast<const __nv_bfloat16*>(c.K) + mt.slot_off * kD;
-  const __nv_bfloat16* Vb = reinterpret_cast<const __nv_bfloat16*>(c.V) + mt.slot_off * kD;
-  double* acc_g = c.acc + mt.slot_off;
-  int32_t* pos_g = c.pos + mt.slot_off;
+  const __nv_bfloat16* Kb = reinterpret_cast<const __nv_bfloat16*>(c.K) + (mt.slot_off + lo) * kD;
+  const __nv_bfloat16* Vb = reinterpret_cast<const __nv_bfloat16*>(c.V) + (mt.slot_off + lo) * kD;
+  double* acc_g = c.acc + mt.slot_off + lo;
+  int32_t* pos_g = c.pos + mt.slot_off + lo;
   const __nv_bfloat16* qu = q + (int64_t)u * G * kD;  // the group's query heads are consecutive
   const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
   const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
@@ -184,8 +204,9 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       bulk_load(pos_s, pos_g, (uint32_t)npad * 4u, &sh.aux);
     }
   }
-  if (all_full) cnt = c.count[su];
-  cnt = min(cnt, nstr);  // (a unit never holds more than was streamed: its budget, or the counter itself)
+  if (all_full) cnt_u = c.count[su];
+  if (!H2O_IN_RANGE(cnt_u, B + 1, c.status)) cnt_u = 0;  // (checked build) a unit never holds more than its budget
+  const int cnt = max(0, min(min(cnt_u - lo, chunk), nstr));  // occupied rows of this block
   __syncthreads();
   if (cache_is_quiescent) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -195,6 +216,14 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
 
   if (warp == kWarps) {
     // ---- producer warp: one lane keeps the ring full ------------------------------------------------------
+    // (Split unit: the warp has nothing to exchange and only keeps the cluster barriers balanced.  It must not
+    //  stand in the barrier between the passes while value tiles are still to be requested: the consumers reach
+    //  that barrier before they free the slots those tiles need.  So it completes the first barrier at once,
+    //  arrives on the second without waiting, streams, and waits afterwards.)
+    if (split > 1) {
+      cluster.barrier_wait();
+      cluster.barrier_arrive();
+    }
     if (lane == 0) {
       for (int T = kStages; T < 2 * nt; ++T) {
         if (!bar_wait(&sh.empty[T & (kStages - 1)], (uint32_t)((T >> kStageShift) - 1) & 1u)) timed_out = true;
@@ -202,12 +231,17 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       }
       if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     }
+    __syncwarp();
+    if (split > 1) {
+      cluster.barrier_wait();
+      cluster.sync();
+    }
     return;
   }
 
   // ---- consumer warps -------------------------------------------------------------------------------------
   // the new token against itself, per query head (the heads go round the warps), with plain arithmetic
-  for (int g = warp; g < G; g += kWarps) {
+  for (int g = warp; g < G && rank == 0; g += kWarps) {  // (with a split unit: the first block's entry)
     const uint2 rq = *reinterpret_cast<const uint2*>(qu + g * kD + 4 * lane);
     const uint2 rk = *reinterpret_cast<const uint2*>(ku + 4 * lane);
     float part = __uint_as_float(rq.x << 16) * __uint_as_float(rk.x << 16);
@@ -251,7 +285,7 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   consumer_sync();
 
   // ---- softmax per head over the cnt rows and the token itself: thread (x0, g) = (tid / G, tid % G) ----------
-  const int total = cnt + 1;
+  const int total = cnt + (rank == 0 ? 1 : 0);
   {
     const int g = tid % G;
     float mx = -INFINITY, sum = 0.f;
@@ -284,8 +318,34 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
 #pragma unroll
       for (int w = 0; w < kWarps; ++w)
         if (sh.part_m[w][tid] > -INFINITY) l += sh.part_l[w][tid] * expf(sh.part_m[w][tid] - m);
-      sh.m[tid] = m;
-      sh.inv_l[tid] = 1.0f / l;
+      if (split == 1) {
+        sh.m[tid] = m;
+        sh.inv_l[tid] = 1.0f / l;
+      } else {
+        sh.m[tid] = m;      // (the block's own, until the cluster's are known)
+        sh.inv_l[tid] = l;
+      }
+    }
+    if (split > 1) {
+      // the block's statistics into every block of the cluster (its own included); the value tiles keep arriving
+      // in the ring meanwhile
+      cluster.barrier_wait();  // every peer is running: its shared memory may be written
+      consumer_sync();
+      if (tid < split * G) {
+        const int dst = tid / G, g2 = tid % G;
+        *cluster.map_shared_rank(&sh.x_m[rank][g2], dst) = sh.m[g2];
+        *cluster.map_shared_rank(&sh.x_l[rank][g2], dst) = sh.inv_l[g2];
+      }
+      cluster.sync();
+      if (tid < G) {
+        float m = -INFINITY;
+        for (int rk = 0; rk < split; ++rk) m = fmaxf(m, sh.x_m[rk][tid]);
+        float l = 0.f;
+        for (int rk = 0; rk < split; ++rk)
+          if (sh.x_m[rk][tid] > -INFINITY) l += sh.x_l[rk][tid] * expf(sh.x_m[rk][tid] - m);
+        sh.m[tid] = m;
+        sh.inv_l[tid] = 1.0f / l;
+      }
     }
     consumer_sync();
     const float m = sh.m[g], inv_l = sh.inv_l[g];
@@ -351,35 +411,39 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   // (the staged scores and positions arrived long ago)
   if (nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
   consumer_sync();
+  // the block's partial outputs (normalised by the unit's sums already); rank 0 adds the new token's own value
   for (int i = tid; i < G * kD; i += kThreads) {
     const int g = i / kD, x = i % kD;
     float acc = 0.f;
 #pragma unroll
     for (int w = 0; w < 2 * kWarps; ++w) acc += red[((size_t)w * G + g) * kD + x];
-    acc = fmaf(p[cnt * G + g], __bfloat162float(vu[x]), acc);
-    out[((int64_t)u * G + g) * kD + x] = __float2bfloat16_rn(acc);
+    if (rank == 0) acc = fmaf(p[cnt * G + g], __bfloat162float(vu[x]), acc);
+    if (split == 1) out[((int64_t)u * G + g) * kD + x] = __float2bfloat16_rn(acc);
+    else *cluster.map_shared_rank(x_out + ((size_t)rank * G + g) * kD + x, 0) = acc;
   }
 
   // ---- accumulate (every head's probability), victim, in-place write ----------------------------------------
-  const bool full = cnt >= B;
+  const bool full = cnt_u >= B;
   Cand best = cand_none();
   for (int x = tid; x < cnt; x += kThreads) {
     double px = 0.0;
 #pragma unroll
     for (int g = 0; g < G; ++g) px += (double)p[x * G + g];
     const double a = acc_s[x] + px;
-    if (H2O_IN_RANGE(mt.slot_off + x, c.total_slots, c.status)) acc_g[x] = a;
+    if (H2O_IN_RANGE(mt.slot_off + lo + x, c.total_slots, c.status)) acc_g[x] = a;
     const int ps = pos_s[x];
     if (full && ps <= t - r) {
-      const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
-      const Cand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
+      const double score = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
+      const Cand cx{(unsigned long long)__double_as_longlong(score), ps, lo + x};
       if (cand_before(cx, best)) best = cx;
     }
   }
   double p_self = 0.0;
+  if (rank == 0) {
 #pragma unroll
-  for (int g = 0; g < G; ++g) p_self += (double)p[cnt * G + g];
-  if (tid == 0 && full && r == 0) {  // without a recent window the new token competes too
+    for (int g = 0; g < G; ++g) p_self += (double)p[cnt * G + g];
+  }
+  if (rank == 0 && tid == 0 && full && r == 0) {  // without a recent window the new token competes too
     const Cand cs{(unsigned long long)__double_as_longlong(p_self), t, -2};
     if (cand_before(cs, best)) best = cs;
   }
@@ -388,13 +452,27 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
   // the new token's K/V row in 16-byte pieces, fetched before the barrier so that the round trip overlaps it
   uint4 new_row = make_uint4(0, 0, 0, 0);
-  if (warp == 0) new_row = *reinterpret_cast<const uint4*>((lane < 16 ? ku : vu) + (lane & 15) * 8);
+  if (warp == 0 && rank == 0) new_row = *reinterpret_cast<const uint4*>((lane < 16 ? ku : vu) + (lane & 15) * 8);
   consumer_sync();
+  Cand b = cand_none();
+  if (warp == 0) b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+  if (split > 1) {
+    // the block's candidate to rank 0 (its partial outputs went there above); one cluster barrier for both, the
+    // last one: afterwards rank 0 works on its own memory only
+    if (warp == 0 && lane == 0) *cluster.map_shared_rank(&sh.x_cand[rank], 0) = b;
+    cluster.sync();
+    if (rank != 0) return;
+    for (int i = tid; i < G * kD; i += kThreads) {
+      float acc = 0.f;
+      for (int rk = 0; rk < split; ++rk) acc += x_out[(size_t)rk * G * kD + i];  // fixed order
+      out[(int64_t)u * G * kD + i] = __float2bfloat16_rn(acc);
+    }
+    if (warp == 0) b = warp_argmin(lane < split ? sh.x_cand[lane] : cand_none());
+  }
   if (warp == 0) {
-    const Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
     int slot, ev;
     if (!full) {
-      slot = cnt;
+      slot = cnt_u;
       ev = -1;
     } else if (b.slot == -2) {
       slot = -1;
@@ -409,7 +487,7 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
     }
     if (slot >= 0 && (!H2O_IN_RANGE(slot, B, c.status) || !H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status))) slot = -1;
     if (lane == 0) {
-      if (!full) c.count[su] = cnt + 1;
+      if (!full) c.count[su] = cnt_u + 1;
       if (slot >= 0) {
         c.acc[mt.slot_off + slot] = p_self;
         c.pos[mt.slot_off + slot] = t;
@@ -429,55 +507,64 @@ size_t ring_smem(int group, int chunk, int stages) {
 }
 
 template <int G, int NW, int STAGES, int MINB>
-cudaError_t launch_ring(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
-                        void* out, int32_t* evicted_pos, cudaStream_t stream) {
+cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
+                        const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   constexpr int kStages = STAGES;
   static_assert(STAGES == 4 || STAGES == 8, "ring depth");
   static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
-  const size_t smem = ring_smem(G, chunk, kStages);
+  const size_t smem = ring_smem(G, chunk, kStages) + (split > 1 ? (size_t)kMaxSplit * G * kD * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)c.units);
+  cfg.gridDim = dim3((unsigned)(c.units * split));
   cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = (unsigned)split;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
+  // (clusters of a launch should all be resident at once: see the step kernel of decode.cu)
+  at[2].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+  at[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = split > 1 ? 3 : 1;
   return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, launch_flags);
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, split, chunk, launch_flags);
 }
 
 template <int G>
-cudaError_t launch_ring_g(const CacheView& c, int chunk, int launch_flags, const void* q, const void* k_new, const void* v_new,
-                          void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  if (c.units <= 2 * sm_count()) return launch_ring<G, 8, 8, 2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-  return launch_ring<G, 4, 4, 4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+cudaError_t launch_ring_g(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
+                          const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  if (c.units * split <= 2 * sm_count())
+    return launch_ring<G, 8, 8, 2>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  return launch_ring<G, 4, 4, 4>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
 }
 
 }  // namespace
 
 // Does the streaming kernel serve this cache (bf16, head_dim 128, its staging within the shared memory of a block)?
-bool decode_two_pass_supported(int dtype, int head_dim, int group, int max_B) {
+// chunk: slots per thread block (the whole budget, or its share when a unit is split over a cluster).
+bool decode_two_pass_supported(int dtype, int head_dim, int group, int chunk) {
   if (dtype != H2O_BF16 || head_dim != kD || (group != 1 && group != 2 && group != 4 && group != 8)) return false;
-  return ring_smem(group, (max_B + 3) & ~3, kMaxStages) <= 190 * 1024;
+  return ring_smem(group, (chunk + 3) & ~3, kMaxStages) + (size_t)kMaxSplit * group * kD * sizeof(float) <= 190 * 1024;
 }
 
-cudaError_t launch_decode_two_pass(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
-                                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+cudaError_t launch_decode_two_pass(const CacheView& c, int split, int chunk, bool cache_is_quiescent, bool all_full,
+                                   const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                                    cudaStream_t stream) {
-  const int chunk = (max_B + 3) & ~3;
+  if (split < 1 || split > kMaxSplit || (chunk & 3) != 0) return cudaErrorInvalidValue;
   const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
   switch (c.group) {
-    case 1: return launch_ring_g<1>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-    case 2: return launch_ring_g<2>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-    case 4: return launch_ring_g<4>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
-    case 8: return launch_ring_g<8>(c, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 1: return launch_ring_g<1>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 2: return launch_ring_g<2>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 4: return launch_ring_g<4>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    case 8: return launch_ring_g<8>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -477,10 +477,11 @@ namespace {
 // mma.sync, exact softmax, V stream; decode_two_pass.cu with one query head per unit) is faster than the
 // online-softmax kernel on launches of many waves of mid-sized and large units (4096 ragged units of 26..820
 // slots: 148 -> 140.5 us; 512 units of 410 slots: 28.1 -> 20.9 us) and slower on small units (3584 units of 104
-// slots: 44.2 -> 53.9 us), equal on 256 units of 410 slots; it has no cluster split, sparse pattern or "Top-K" form.
+// slots: 44.2 -> 53.9 us), equal on 256 units of 410 slots and on 32 units of 2048 slots split over clusters of
+// eight (11.9 against 11.3 - 12.0 us), where the online kernel stays; it has no sparse pattern or "Top-K" form.
 bool two_pass_supported(const h2o_cache* cache) {
   return cache->view.group == 1 && !cache->view.kv4 && cache->view.mask_kind == 0 && cache->view.topk == 0 &&
-         h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->layout.max_B);
+         h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->chunk);
 }
 bool two_pass_step(const h2o_cache* cache) {
   if (cache->decode_path == 1 || !two_pass_supported(cache)) return false;
@@ -501,7 +502,7 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
   const bool quiescent = g_last_writer.note_and_check(static_cast<cudaStream_t>(stream), cache->view.K) && g_early_prefetch;
   const bool ring1 = two_pass_step(cache);
   const cudaError_t e =
-      ring1 ? h2o::launch_decode_two_pass(cache->view, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new, v_new, out,
+      ring1 ? h2o::launch_decode_two_pass(cache->view, cache->split, cache->chunk, quiescent, all_units_full(cache), q, k_new, v_new, out,
                                           evicted_pos, static_cast<cudaStream_t>(stream))
       : cache->view.group > 1
           ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
@@ -550,7 +551,7 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
                                        static_cast<char*>(out) + i * qstep, ev_i, st)
           : two_pass_step(cache)
-              ? h2o::launch_decode_two_pass(cache->view, cache->layout.max_B, false, all_units_full(cache),
+              ? h2o::launch_decode_two_pass(cache->view, cache->split, cache->chunk, false, all_units_full(cache),
                                             static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
                                             static_cast<const char*>(v) + off, static_cast<char*>(out) + off, ev_i, st)
           : cache->view.kv4

@@ -138,9 +138,9 @@ size_t decode_gqa_smem_bytes(int group, int max_B, int head_dim);
 cudaError_t launch_decode_gqa(const CacheView& c, int dtype, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
                               const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream);
 // The streaming form for bf16 / head_dim 128 (decode_two_pass.cu); launch_decode_gqa uses it when it is supported.
-bool decode_two_pass_supported(int dtype, int head_dim, int group, int max_B);
-cudaError_t launch_decode_two_pass(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
-                                   const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+bool decode_two_pass_supported(int dtype, int head_dim, int group, int chunk);
+cudaError_t launch_decode_two_pass(const CacheView& c, int split, int chunk, bool cache_is_quiescent, bool all_full,
+                                   const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                                    cudaStream_t stream);
 // ALU path; `rows` = attention rows + row statistics, `colsum` = column sums.
 cudaError_t launch_prefill_naive(const CacheView& c, const PrefillScratch& s, int dtype, int max_seqlen, const void* q,

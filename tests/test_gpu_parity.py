@@ -552,6 +552,19 @@ def test_two_pass_step_kernel_ragged_fill_phase_and_edges(H2OCache):
     print(run_parity(wl, H2OCache, export_every=4, decode_path=2))
 
 
+@pytest.mark.parametrize("budget,split", [(300, 2), (520, 2), (1040, 4), (2300, 8), (2048, 8)])
+def test_two_pass_step_kernel_unit_split_over_a_cluster(H2OCache, budget, split):
+    """The two-pass kernel with a unit split over a cluster: statistics exchanged between the passes, outputs and
+    candidates after the value pass.  Shares of more than 256 slots wrap the block's ring while the consumers stand
+    in the barrier between the passes (the producer warp must not wait there)."""
+    from parity_harness import run_parity
+
+    wl = _wl("tpsplit", 1, 2, 128, "bf16", [3000], 6, [budget // 2], [budget - budget // 2], seed=207)
+    print(run_parity(wl, H2OCache, export_every=2, split=split, decode_path=2))
+    wl = _wl("tpsplitfill", 1, 2, 128, "bf16", [1], 70, [20], [30], seed=208)
+    print(run_parity(wl, H2OCache, prefill=False, export_every=8, split=min(split, 2), decode_path=2))
+
+
 def test_two_pass_step_kernel_where_it_does_not_apply(H2OCache):
     import paper_2306_14048_b200 as pkg
 
