@@ -543,6 +543,13 @@ cudaError_t launch_ring_g(const CacheView& c, int split, int chunk, int launch_f
                           const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   if (c.units * split <= 2 * sm_count())
     return launch_ring<G, 8, 8, 2>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  // five blocks per SM (72 registers) where their shared memory allows it: 2048 units of 256 slots 51.1 -> 48.0 us,
+  // 3584 units of 104 slots 51.4 -> 45.6 us; with four blocks' worth of shared memory the cap only costs (config 5:
+  // 140.5 -> 142.1 us)
+  if constexpr (G == 1) {
+    if (5 * (ring_smem(G, chunk, 4) + (split > 1 ? (size_t)kMaxSplit * G * kD * sizeof(float) : 0) + 2048) <= 227 * 1024)
+      return launch_ring<G, 4, 4, 5>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+  }
   return launch_ring<G, 4, 4, 4>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
 }
 
