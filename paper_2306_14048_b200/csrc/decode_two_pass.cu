@@ -115,11 +115,14 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
 // (four blocks per SM hide one another's passes between the two streams and their serial ends).  For few units
 // neither four warps per block (256 units of 410 slots: 15.4 us against 12.3) nor eight warps capped at 56
 // registers with a 4-deep ring, so that the next launch's blocks are resident beside this launch's (14.4 us), helped.
-template <int G, int NW, int STAGES, int MINB>
+// CLUSTER: the instances that can split a unit over a cluster (the others compile that code out: its registers
+// cost the grouped four-warp instance 4 %).
+template <int G, int NW, int STAGES, int MINB, bool CLUSTER>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                       int32_t* __restrict__ evicted_pos, int split, int chunk, int launch_flags) {
+                       int32_t* __restrict__ evicted_pos, int split_arg, int chunk, int launch_flags) {
+  const int split = CLUSTER ? split_arg : 1;
   constexpr int kWarps = NW, kThreads = NW * 32, kStages = STAGES, kStageShift = STAGES == 8 ? 3 : 2;
   auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -506,7 +509,7 @@ size_t ring_smem(int group, int chunk, int stages) {
   return (size_t)stages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
 }
 
-template <int G, int NW, int STAGES, int MINB>
+template <int G, int NW, int STAGES, int MINB, bool CLUSTER = false>
 cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
                         const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   constexpr int kStages = STAGES;
@@ -514,7 +517,7 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
   static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
   const size_t smem = ring_smem(G, chunk, kStages) + (split > 1 ? (size_t)kMaxSplit * G * kD * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB>), 200 * 1024, &attr_flags);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(c.units * split));
@@ -533,7 +536,7 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
   at[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
   cfg.attrs = at;
   cfg.numAttrs = split > 1 ? 3 : 1;
-  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, split, chunk, launch_flags);
 }
@@ -541,13 +544,22 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
 template <int G>
 cudaError_t launch_ring_g(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
                           const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  if (c.units * split <= 2 * sm_count())
+  if (split > 1) {
+    if constexpr (G == 1) {
+      if (c.units * split <= 2 * sm_count())
+        return launch_ring<G, 8, 8, 2, true>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+      return launch_ring<G, 4, 4, 4, true>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    } else {
+      return cudaErrorInvalidValue;  // grouped caches are not split
+    }
+  }
+  if (c.units <= 2 * sm_count())
     return launch_ring<G, 8, 8, 2>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
   // five blocks per SM (72 registers) where their shared memory allows it: 2048 units of 256 slots 51.1 -> 48.0 us,
   // 3584 units of 104 slots 51.4 -> 45.6 us; with four blocks' worth of shared memory the cap only costs (config 5:
   // 140.5 -> 142.1 us)
   if constexpr (G == 1) {
-    if (5 * (ring_smem(G, chunk, 4) + (split > 1 ? (size_t)kMaxSplit * G * kD * sizeof(float) : 0) + 2048) <= 227 * 1024)
+    if (5 * (ring_smem(G, chunk, 4) + 2048) <= 227 * 1024)
       return launch_ring<G, 4, 4, 5>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
   }
   return launch_ring<G, 4, 4, 4>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
