@@ -15,34 +15,16 @@
 #include <climits>
 
 #include "h2o_internal.cuh"
+#include "step_common.cuh"
 
 namespace h2o {
 
 namespace {
 
+using namespace step;
+
 constexpr int kGqThreads = 256;
 constexpr int kGqWarps = kGqThreads / 32;
-
-struct GqCand {
-  unsigned long long key;  // bit pattern of the (non-negative) ranking score
-  int pos, slot;           // slot -1: none, -2: the new token itself
-};
-__device__ __forceinline__ bool gq_before(const GqCand& a, const GqCand& b) {
-  if (a.slot == -1) return false;
-  if (b.slot == -1) return true;
-  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
-}
-__device__ __forceinline__ GqCand gq_warp_min(GqCand a) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    GqCand b;
-    b.key = __shfl_xor_sync(0xffffffffu, a.key, off);
-    b.pos = __shfl_xor_sync(0xffffffffu, a.pos, off);
-    b.slot = __shfl_xor_sync(0xffffffffu, a.slot, off);
-    if (gq_before(b, a)) a = b;
-  }
-  return a;
-}
 
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kGqThreads)
@@ -53,7 +35,7 @@ decode_gqa_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_
   float* s = reinterpret_cast<float*>(dyn);                  // [G][pitch]: raw scores, then probabilities
   float* red = s + G * pitch;                                // [warps][G][D]: per-warp partial outputs
   __shared__ float sm_m[G], sm_l[G];
-  __shared__ GqCand wbest[kGqWarps];
+  __shared__ Cand wbest[kGqWarps];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sub = lane / LPR, ch = lane % LPR;
@@ -204,7 +186,7 @@ decode_gqa_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_
   const bool full = cnt >= B;
   double* acc_g = c.acc + mt.slot_off;
   const int32_t* pos_g = c.pos + mt.slot_off;
-  GqCand best{~0ull, INT_MAX, -1};
+  Cand best = cand_none();
   for (int x = tid; x < cnt; x += kGqThreads) {
     double px = 0.0;
 #pragma unroll
@@ -214,23 +196,23 @@ decode_gqa_kernel(CacheView c, const T* __restrict__ q, const T* __restrict__ k_
     const int ps = pos_g[x];
     if (full && ps <= t - r) {
       const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
-      const GqCand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
-      if (gq_before(cx, best)) best = cx;
+      const Cand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
+      if (cand_before(cx, best)) best = cx;
     }
   }
   double p_self = 0.0;
 #pragma unroll
   for (int g = 0; g < G; ++g) p_self += (double)s[g * pitch + cnt];
   if (tid == 0 && full && r == 0) {  // without a recent window the new token competes too
-    const GqCand cs{(unsigned long long)__double_as_longlong(p_self), t, -2};
-    if (gq_before(cs, best)) best = cs;
+    const Cand cs{(unsigned long long)__double_as_longlong(p_self), t, -2};
+    if (cand_before(cs, best)) best = cs;
   }
-  best = gq_warp_min(best);
+  best = warp_argmin(best);
   if (lane == 0) wbest[warp] = best;
   __syncthreads();
   if (warp == 0) {
-    GqCand b = lane < kGqWarps ? wbest[lane] : GqCand{~0ull, INT_MAX, -1};
-    b = gq_warp_min(b);
+    Cand b = lane < kGqWarps ? wbest[lane] : cand_none();
+    b = warp_argmin(b);
     int slot, ev;
     if (!full) {
       slot = cnt;

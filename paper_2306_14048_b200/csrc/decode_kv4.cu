@@ -31,11 +31,13 @@
 #include "h2o.h"
 #include "h2o_internal.cuh"
 #include "sm100_ptx.cuh"
+#include "step_common.cuh"
 
 namespace h2o {
 namespace {
 
 using namespace ptx;
+using namespace step;
 
 constexpr int kD = 128;
 constexpr int kRowBytes = 80;
@@ -45,19 +47,6 @@ constexpr int kMaxWarps = 16;             // consumer warps: 16 when a block has
 constexpr int kTileRows = 64;             // rows per tile: eight per consumer warp
 constexpr int kTileBytes = kTileRows * kRowBytes;  // 5120
 constexpr int kMaxStages = 8;             // ring depth: 2, 4 or 8 tiles (K and V) in flight
-constexpr uint32_t kSpin = 1u << 22;
-
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpin; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
 // (a & b) | c in one logic instruction
 __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
   uint32_t d;
@@ -84,28 +73,6 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
-
-struct Cand {
-  unsigned long long key;  // bit pattern of the (non-negative) ranking score
-  int pos, slot;           // slot -1: none, -2: the new token itself
-};
-__device__ __forceinline__ Cand cand_none() { return Cand{~0ull, INT_MAX, -1}; }
-__device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {
-  if (a.slot == -1) return false;
-  if (b.slot == -1) return true;
-  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
-}
-__device__ __forceinline__ Cand warp_argmin(Cand a) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    Cand b;
-    b.key = __shfl_xor_sync(0xffffffffu, a.key, off);
-    b.pos = __shfl_xor_sync(0xffffffffu, a.pos, off);
-    b.slot = __shfl_xor_sync(0xffffffffu, a.slot, off);
-    if (cand_before(b, a)) a = b;
-  }
-  return a;
-}
 
 // Quantise one group of 32 channels (bf16 inputs); codes: 16 bytes, meta = scale | zero << 16 (bf16 bits).
 __device__ __forceinline__ void quantise_group(const __nv_bfloat16* src, uint4& codes, uint32_t& meta) {

@@ -30,6 +30,7 @@
 
 #include "h2o_internal.cuh"
 #include "sm100_ptx.cuh"
+#include "step_common.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -38,6 +39,7 @@ namespace h2o {
 namespace {
 
 using namespace ptx;
+using namespace step;
 
 constexpr int kMaxSplit = 8;
 
@@ -45,49 +47,8 @@ constexpr int kD = 128;
 constexpr int kTileRows = 32, kRowBytes = kD * 2, kTileBytes = kTileRows * kRowBytes;  // 8 KB
 constexpr int kMaxStages = 8;  // ring depth: 8 tiles, or 4 for the four-warp instance (more blocks per SM)
 constexpr int kMaxWarps = 8;
-constexpr uint32_t kSpin = 1u << 22;
-
-__device__ __forceinline__ bool bar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kSpin; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
 template <int THREADS>
 __device__ __forceinline__ void consumer_sync_n() { asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory"); }
-
-struct Cand {
-  unsigned long long key;  // bit pattern of the (non-negative) ranking score
-  int pos, slot;           // slot -1: none, -2: the new token itself
-};
-__device__ __forceinline__ Cand cand_none() { return Cand{~0ull, INT_MAX, -1}; }
-__device__ __forceinline__ bool cand_before(const Cand& a, const Cand& b) {
-  if (a.slot == -1) return false;
-  if (b.slot == -1) return true;
-  return a.key < b.key || (a.key == b.key && a.pos < b.pos);
-}
-// Warp-wide minimum under the eviction order (scores are >= 0: their bit patterns order like the values).
-__device__ __forceinline__ Cand warp_argmin(const Cand& a) {
-  const bool valid = a.slot != -1;
-  const unsigned long long bits = valid ? a.key : ~0ull;
-  const unsigned hi = (unsigned)(bits >> 32), lo = (unsigned)bits;
-  const unsigned mh = __reduce_min_sync(0xffffffffu, hi);
-  const unsigned ml = __reduce_min_sync(0xffffffffu, hi == mh ? lo : 0xffffffffu);
-  const bool tie = valid && hi == mh && lo == ml;
-  const unsigned mp = __reduce_min_sync(0xffffffffu, tie ? (unsigned)a.pos : 0xffffffffu);
-  const unsigned who = __ballot_sync(0xffffffffu, tie && (unsigned)a.pos == mp);
-  if (who == 0) return cand_none();
-  Cand b;
-  b.key = ((unsigned long long)mh << 32) | ml;
-  b.pos = (int)mp;
-  b.slot = __shfl_sync(0xffffffffu, a.slot, __ffs(who) - 1);
-  return b;
-}
 
 struct Shared {
   uint64_t full[kMaxStages], empty[kMaxStages], aux;
