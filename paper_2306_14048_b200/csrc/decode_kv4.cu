@@ -21,6 +21,7 @@
 // per pair of codes, is what bounds the kernel: the logic pipe, not HBM): the scores with the query as the
 // column operand, one column per group; the values with the codes transposed as the row operand and
 // p * scale, split into a bf16 head and remainder per group, as the column operand.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -33,10 +34,14 @@
 #include "sm100_ptx.cuh"
 #include "step_common.cuh"
 
+namespace cg = cooperative_groups;
+
 namespace h2o {
 namespace {
 
 using namespace ptx;
+
+constexpr int kMaxSplit = 8;
 using namespace step;
 
 constexpr int kD = 128;
@@ -130,6 +135,11 @@ struct Shared {
   // the query as the B operand of the score products, per lane 16 words (rows padded to 20 words: 16-byte
   // reads of eight consecutive lanes then fall into different banks)
   __align__(16) uint32_t qb[32][20];
+  // Cluster exchange (a unit split over the blocks of a cluster, CLUSTER instances): every block pushes its values
+  // into its peers' shared memory with remote stores, then one cluster barrier makes them visible.
+  float x_m[kMaxSplit], x_l[kMaxSplit];  // block statistics of every rank (written by that rank)
+  float x_out[kMaxSplit][kD];            // rank 0 only: every rank's partial output, relative to its own maximum
+  Cand x_cand[kMaxSplit];                // rank 0 only: every rank's eviction candidate
 };
 
 // MINB: blocks per SM the register allocation leaves room for (the kernel wants ~96 registers a thread).
@@ -138,11 +148,15 @@ struct Shared {
 // dependency is awaited; every unit full: no counter read before the first request) and fetch the new value row
 // at the start.  In launches of many waves the same code was slower
 // (3584 units of 104 slots: 46.4 -> 48.4 us), so those instances leave it out.
-template <int MINB, int kWarps, bool EARLY>
+// CLUSTER: the instance that splits a unit over the blocks of a cluster (few long units): block `rank` owns slots
+// rank * chunk .. of the unit; statistics and partial outputs are exchanged after the stream, candidates after the
+// final probabilities, as in the step kernel of the bf16 slots.
+template <int MINB, int kWarps, bool EARLY, bool CLUSTER>
 __global__ void __launch_bounds__(kWarps * 32 + 32, MINB)
 decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
-                  int32_t* __restrict__ evicted_pos, int chunk, int stage_shift, int launch_flags) {
+                  int32_t* __restrict__ evicted_pos, int split_arg, int chunk, int stage_shift, int launch_flags) {
+  const int split = CLUSTER ? split_arg : 1;
   constexpr int kThreads = kWarps * 32;
   const int stages = 1 << stage_shift;  // ring depth: a power of two
   extern __shared__ __align__(128) unsigned char dyn[];
@@ -154,7 +168,12 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   float* p = reinterpret_cast<float*>(pos_s + chunk);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int su = blockIdx.x;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = split > 1 ? (int)cluster.block_rank() : 0;
+  // Early arrival on the cluster barrier; the matching wait comes right before the first remote store.
+  if (split > 1) cluster.barrier_arrive();
+  const int su = blockIdx.x / split;
+  const int lo = rank * chunk;  // first slot of this block
   const UnitMeta mt = c.meta[su];
   // Programmatic dependent launch, as in the step kernel of the bf16 slots: the inputs may come from the previous
   // kernel of the stream and are read after griddepcontrol.wait; the cache is written by this library alone, and
@@ -172,24 +191,24 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
   }
   KV_STAMP(13);
   const int u = mt.unit, r = mt.rwin, B = mt.kbud + mt.rwin;
-  int cnt, nstr;  // entries of the unit, rows to stream
+  int cnt_u, cnt, nstr;  // entries of the unit, of this block, rows to stream
   if constexpr (EARLY) {
-    cnt = all_full ? 0 : c.count[su];
-    nstr = all_full ? B : cnt;
+    cnt_u = all_full ? 0 : c.count[su];
+    nstr = all_full ? max(0, min(B - lo, chunk)) : max(0, min(cnt_u - lo, chunk));
   } else {
-    cnt = c.count[su];
-    nstr = cnt;
+    cnt_u = c.count[su];
+    nstr = CLUSTER ? max(0, min(cnt_u - lo, chunk)) : cnt_u;
   }
   const int t = c.tpos[su];
   // (checked build: the unit and the rows this block streams must lie inside the cache)
-  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) || !H2O_IN_RANGE(nstr, B + 1, c.status) ||
-      !H2O_IN_RANGE(mt.slot_off + (nstr > 0 ? nstr - 1 : 0), c.total_slots, c.status))
+  if (!H2O_IN_RANGE(mt.unit, c.units, c.status) || !H2O_IN_RANGE(nstr, min(B, chunk) + 1, c.status) ||
+      !H2O_IN_RANGE(mt.slot_off + lo + (nstr > 0 ? nstr - 1 : 0), c.total_slots, c.status))
     nstr = 0;
   const int ntile = (nstr + kTileRows - 1) / kTileRows;
-  unsigned char* Kb = static_cast<unsigned char*>(c.K) + mt.slot_off * kRowBytes;
-  unsigned char* Vb = static_cast<unsigned char*>(c.V) + mt.slot_off * kRowBytes;
-  double* acc_g = c.acc + mt.slot_off;
-  int32_t* pos_g = c.pos + mt.slot_off;
+  unsigned char* Kb = static_cast<unsigned char*>(c.K) + (mt.slot_off + lo) * kRowBytes;
+  unsigned char* Vb = static_cast<unsigned char*>(c.V) + (mt.slot_off + lo) * kRowBytes;
+  double* acc_g = c.acc + mt.slot_off + lo;
+  int32_t* pos_g = c.pos + mt.slot_off + lo;
   const __nv_bfloat16* qu = q + (int64_t)u * kD;
   const __nv_bfloat16* ku = k_new + (int64_t)u * kD;
   const __nv_bfloat16* vu = v_new + (int64_t)u * kD;
@@ -240,9 +259,9 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     }
   }
   if constexpr (EARLY) {
-    if (all_full) cnt = c.count[su];
+    if (all_full) cnt_u = c.count[su];
   }
-  if constexpr (EARLY) cnt = min(cnt, nstr);  // (a unit never holds more than was streamed: its budget, or the counter itself)
+  if constexpr (EARLY) cnt = max(0, min(min(cnt_u - lo, chunk), nstr));  // (never more than was streamed)
   else cnt = nstr;
   __syncthreads();
   if constexpr (EARLY) {
@@ -272,6 +291,12 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       }
       if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     }
+    __syncwarp();
+    if (split > 1) {  // the producer warp only keeps the cluster barriers balanced (both exchanges follow the stream)
+      cluster.barrier_wait();
+      cluster.sync();
+      cluster.sync();
+    }
   } else {
     // ---- consumer warps --------------------------------------------------------------------------
     // A warp takes 16 rows of a tile (with eight warps: warps 0..3 the even tiles, warps 4..7 the odd ones).
@@ -299,7 +324,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       part += __shfl_xor_sync(0xffffffffu, part, 1);
       part += __shfl_xor_sync(0xffffffffu, part, 2);
       part += __shfl_xor_sync(0xffffffffu, part, 4);
-      s_self = c.scale * part;
+      s_self = rank == 0 ? c.scale * part : -INFINITY;  // (split unit: the first block's entry)
     }
     // the query of group c4: its sum, and (warp 0) its words as B operands.  For the word w of a row
     // (channels 8 w .. 8 w + 7 of the group) the two products use k index pairs (code 0, code 4 | code 1,
@@ -493,24 +518,58 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     float l = lane < kWarps ? sh.gl[lane] * w_i : 0.f;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-    const float w_self = expf(s_self - m);
+    float w_self = s_self > -INFINITY ? expf(s_self - m) : 0.f;
     l += w_self;
-    const float inv_l = 1.0f / l;
-    if (warp == 0) {  // output: this lane's four channels
-      float res[4];
-      {
-        const uint2 raw = EARLY ? in_v : *reinterpret_cast<const uint2*>(vu + 4 * lane);  // the new token's value
-        res[0] = w_self * __uint_as_float(raw.x << 16);
-        res[1] = w_self * __uint_as_float(raw.x & 0xffff0000u);
-        res[2] = w_self * __uint_as_float(raw.y << 16);
-        res[3] = w_self * __uint_as_float(raw.y & 0xffff0000u);
-      }
+    float res[4] = {0.f, 0.f, 0.f, 0.f};
+    if (warp == 0) {  // the block's output, relative to its maximum: this lane's four channels
+      const uint2 raw = EARLY ? in_v : *reinterpret_cast<const uint2*>(vu + 4 * lane);  // the new token's value
+      res[0] = w_self * __uint_as_float(raw.x << 16);
+      res[1] = w_self * __uint_as_float(raw.x & 0xffff0000u);
+      res[2] = w_self * __uint_as_float(raw.y << 16);
+      res[3] = w_self * __uint_as_float(raw.y & 0xffff0000u);
 #pragma unroll
       for (int g2 = 0; g2 < kWarps; ++g2) {
         const float w = __shfl_sync(0xffffffffu, w_i, g2);
 #pragma unroll
         for (int i = 0; i < 4; ++i) res[i] = fmaf(sh.red[g2][4 * lane + i], w, res[i]);
       }
+    }
+    if (split > 1) {
+      const float mc = m, lc = l;
+      cluster.barrier_wait();  // every peer is running: its shared memory may be written
+      if (tid < split) {       // my statistics into every block of the cluster (my own included)
+        *cluster.map_shared_rank(&sh.x_m[rank], tid) = mc;
+        *cluster.map_shared_rank(&sh.x_l[rank], tid) = lc;
+      }
+      if (warp == 0) *reinterpret_cast<float4*>(cluster.map_shared_rank(&sh.x_out[rank][4 * lane], 0)) = make_float4(res[0], res[1], res[2], res[3]);
+      cluster.sync();
+      const float mr = lane < split ? sh.x_m[lane] : -INFINITY;
+      const float lr = lane < split ? sh.x_l[lane] : 0.f;
+      m = mr;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+      l = mr > -INFINITY ? lr * expf(mr - m) : 0.f;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+      w_self = s_self > -INFINITY ? expf(s_self - m) : 0.f;
+      if (rank == 0 && warp == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) res[i] = 0.f;
+        for (int rk = 0; rk < split; ++rk) {
+          const float mrk = sh.x_m[rk];
+          if (mrk > -INFINITY) {
+            const float w = expf(mrk - m);
+            const float4 xo = *reinterpret_cast<const float4*>(&sh.x_out[rk][4 * lane]);
+            res[0] = fmaf(xo.x, w, res[0]);
+            res[1] = fmaf(xo.y, w, res[1]);
+            res[2] = fmaf(xo.z, w, res[2]);
+            res[3] = fmaf(xo.w, w, res[3]);
+          }
+        }
+      }
+    }
+    const float inv_l = 1.0f / l;
+    if (warp == 0 && rank == 0) {
       uint2 pk;
       pk.x = Vec16<__nv_bfloat16>::pack2(res[0] * inv_l, res[1] * inv_l);
       pk.y = Vec16<__nv_bfloat16>::pack2(res[2] * inv_l, res[3] * inv_l);
@@ -519,21 +578,21 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
 
     // ---- final probabilities, accumulation (Algorithm 2: accumulated score += probability), victim search ----
     if (nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
-    const bool full = cnt >= B;
+    const bool full = cnt_u >= B;
     const float p_self = w_self * inv_l;
     Cand best = cand_none();
     for (int x = tid; x < cnt; x += kThreads) {
       const float px = expf(p[x] - m) * inv_l;
       const double a = acc_s[x] + (double)px;
-      if (H2O_IN_RANGE(mt.slot_off + x, c.total_slots, c.status)) acc_g[x] = a;
+      if (H2O_IN_RANGE(mt.slot_off + lo + x, c.total_slots, c.status)) acc_g[x] = a;
       const int ps = pos_s[x];
       if (full && ps <= t - r) {
-        const double rank = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
-        const Cand cx{(unsigned long long)__double_as_longlong(rank), ps, x};
+        const double score = c.score_mode == 1 ? a / (double)(t - ps + 1) : a;
+        const Cand cx{(unsigned long long)__double_as_longlong(score), ps, lo + x};
         if (cand_before(cx, best)) best = cx;
       }
     }
-    if (tid == 0 && full && r == 0) {  // without a recent window the new token competes too
+    if (rank == 0 && tid == 0 && full && r == 0) {  // without a recent window the new token competes too
       const Cand cs{(unsigned long long)__double_as_longlong((double)p_self), t, -2};
       if (cand_before(cs, best)) best = cs;
     }
@@ -542,11 +601,17 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
     if (timed_out) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");
     KV_STAMP(15);
-    if (warp == 0) {
-      const Cand b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+    Cand b = cand_none();
+    if (warp == 0) b = warp_argmin(lane < kWarps ? sh.wbest[lane] : cand_none());
+    if (split > 1) {
+      if (warp == 0 && lane == 0) *cluster.map_shared_rank(&sh.x_cand[rank], 0) = b;
+      cluster.sync();  // the last cluster barrier: afterwards rank 0 works on its own memory only
+      if (warp == 0 && rank == 0) b = warp_argmin(lane < split ? sh.x_cand[lane] : cand_none());
+    }
+    if (warp == 0 && rank == 0) {
       int slot, ev;
       if (!full) {
-        slot = cnt;
+        slot = cnt_u;
         ev = -1;
       } else if (b.slot == -2) {
         slot = -1;
@@ -562,7 +627,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       if (slot >= 0 && (!H2O_IN_RANGE(slot, B, c.status) || !H2O_IN_RANGE(mt.slot_off + slot, c.total_slots, c.status)))
         slot = -1;  // (checked build) never write outside the unit's slots
       if (lane == 0) {
-        if (!full) c.count[su] = cnt + 1;
+        if (!full) c.count[su] = cnt_u + 1;
         if (slot >= 0) {
           c.acc[mt.slot_off + slot] = (double)p_self;
           c.pos[mt.slot_off + slot] = t;
@@ -574,7 +639,7 @@ decode_kv4_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_b
       if (!nr_ok && lane == 0) atomicCAS(c.status, 0, H2O_ERR_TIMEOUT);
       if (nr_ok && slot >= 0 && lane < 10) {  // the quantised new row goes straight into the freed slot
         const int which = lane / 5, part = lane % 5;  // K: five 16-byte pieces, V: five
-        unsigned char* dst = (which == 0 ? Kb : Vb) + (size_t)slot * kRowBytes + 16 * part;
+        unsigned char* dst = static_cast<unsigned char*>(which == 0 ? c.K : c.V) + (size_t)(mt.slot_off + slot) * kRowBytes + 16 * part;
         *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(sh.newrow[which] + 16 * part);
       }
     }
@@ -619,55 +684,67 @@ extern "C" int h2o_debug_kv4_timers(long long* host, int n) {
 
 size_t kv4_row_bytes() { return kRowBytes; }
 
-template <int MINB, int NW, bool EARLY>
-static cudaError_t launch_kv4(const CacheView& c, int chunk, int stage_shift, size_t smem, int launch_flags, const void* q,
-                              const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+template <int MINB, int NW, bool EARLY, bool CLUSTER = false>
+static cudaError_t launch_kv4(const CacheView& c, int split, int chunk, int stage_shift, size_t smem, int launch_flags,
+                              const void* q, const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+                              cudaStream_t stream) {
   static unsigned long long attr_flags = 0;  // one word per instance, one bit per device
   {
-    cudaError_t e =
-        ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB, NW, EARLY>), 200 * 1024, &attr_flags);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_kv4_kernel<MINB, NW, EARLY, CLUSTER>),
+                                        200 * 1024, &attr_flags);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)c.units);
+  cfg.gridDim = dim3((unsigned)(c.units * (CLUSTER ? split : 1)));
   cfg.blockDim = dim3(NW * 32 + 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[3];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = (unsigned)split;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
+  // (clusters of a launch should all be resident at once: see the step kernel of decode.cu)
+  at[2].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+  at[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW, EARLY>, c, static_cast<const __nv_bfloat16*>(q),
+  cfg.numAttrs = (CLUSTER && split > 1) ? 3 : 1;
+  return cudaLaunchKernelEx(&cfg, decode_kv4_kernel<MINB, NW, EARLY, CLUSTER>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
-                            static_cast<__nv_bfloat16*>(out), evicted_pos, chunk, stage_shift, launch_flags);
+                            static_cast<__nv_bfloat16*>(out), evicted_pos, split, chunk, stage_shift, launch_flags);
 }
 
-cudaError_t launch_decode_kv4(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
+// split: thread blocks (one cluster) per unit, chunk: slots per block (a multiple of 4; the whole budget when split = 1)
+cudaError_t launch_decode_kv4(const CacheView& c, int split, int chunk, bool cache_is_quiescent, bool all_full, const void* q,
                               const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
-  const int chunk = (max_B + 3) & ~3;
+  if (split < 1 || split > kMaxSplit || (chunk & 3) != 0) return cudaErrorInvalidValue;
   const int launch_flags = (cache_is_quiescent ? 1 : 0) | (all_full ? 2 : 0);
   const int sms = sm_count();
+  const int blocks = c.units * split;
   const size_t fixed = (size_t)chunk * 16 + 16;
   auto smem_for = [&](int shift) { return ((size_t)(2 * kTileBytes) << shift) + fixed; };
   if (smem_for(1) > 200 * 1024) return cudaErrorInvalidValue;
-#define KV4_GO(M, W, EARLY, SHIFT) \
-  return launch_kv4<M, W, EARLY>(c, chunk, SHIFT, smem_for(SHIFT), launch_flags, q, k_new, v_new, out, evicted_pos, stream)
-  // Few units (at most two blocks per SM): the deepest ring that fits, since nothing else hides the load latency
+#define KV4_GO(M, W, EARLY, CL, SHIFT) \
+  return launch_kv4<M, W, EARLY, CL>(c, split, chunk, SHIFT, smem_for(SHIFT), launch_flags, q, k_new, v_new, out, evicted_pos, stream)
+  // Few blocks (at most two per SM): the deepest ring that fits, since nothing else hides the load latency
   // (eight tiles in flight against four: 13.1 -> 11.8 us per launch at 256 units of 410 slots); sixteen consumer
   // warps when a block has the SM to itself.
-  if (c.units <= 2 * sms) {
-    const bool alone = c.units <= sms;
+  if (blocks <= 2 * sms) {
+    const bool alone = blocks <= sms;
     int shift = 3;
-    while (shift > 1 && (alone ? 1 : 2) * (smem_for(shift) + 12 * 1024) > 220 * 1024) --shift;
-    if (alone) KV4_GO(1, 16, true, shift);
-    KV4_GO(2, 8, true, shift);
+    while (shift > 1 && (alone ? 1 : 2) * (smem_for(shift) + 14 * 1024) > 220 * 1024) --shift;
+    if (split > 1) KV4_GO(2, 8, true, true, shift);
+    if (alone) KV4_GO(1, 16, true, false, shift);
+    KV4_GO(2, 8, true, false, shift);
   }
-  // Many units: four consumer warps per block and four blocks per SM (96 registers a thread), whose serial
+  // Many blocks: four consumer warps per block and four blocks per SM (96 registers a thread), whose serial
   // starts and ends hide one another; a shallow ring once the blocks outnumber the resident slots.
-  if (c.units > 8 * sms) KV4_GO(4, 4, false, 1);
-  if (c.units > 4 * sms || smem_for(2) > 200 * 1024) KV4_GO(4, 4, true, 1);
-  KV4_GO(4, 4, true, 2);
+  if (split > 1) KV4_GO(4, 4, true, true, 1);
+  if (blocks > 8 * sms) KV4_GO(4, 4, false, false, 1);
+  if (blocks > 4 * sms || smem_for(2) > 200 * 1024) KV4_GO(4, 4, true, false, 1);
+  KV4_GO(4, 4, true, false, 2);
 #undef KV4_GO
 }
 

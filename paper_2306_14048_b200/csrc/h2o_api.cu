@@ -510,7 +510,7 @@ int h2o_decode_step(h2o_cache_t* cache, const void* q, const void* k_new, const 
       : cache->view.group > 1
           ? h2o::launch_decode_gqa(cache->view, cache->cfg.dtype, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
                                    v_new, out, evicted_pos, static_cast<cudaStream_t>(stream))
-      : cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, quiescent, all_units_full(cache), q, k_new,
+      : cache->view.kv4 ? h2o::launch_decode_kv4(cache->view, cache->split, cache->chunk, quiescent, all_units_full(cache), q, k_new,
                                                v_new, out, evicted_pos, static_cast<cudaStream_t>(stream))
                       : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, quiescent,
                                            all_units_full(cache), q, k_new, v_new, out, evicted_pos,
@@ -558,7 +558,7 @@ int h2o_decode_chunk(h2o_cache_t* cache, const void* q, const void* k, const voi
                                             static_cast<const char*>(q) + off, static_cast<const char*>(k) + off,
                                             static_cast<const char*>(v) + off, static_cast<char*>(out) + off, ev_i, st)
           : cache->view.kv4
-              ? h2o::launch_decode_kv4(cache->view, cache->layout.max_B, false, all_units_full(cache), static_cast<const char*>(q) + off,
+              ? h2o::launch_decode_kv4(cache->view, cache->split, cache->chunk, false, all_units_full(cache), static_cast<const char*>(q) + off,
                                        static_cast<const char*>(k) + off, static_cast<const char*>(v) + off,
                                        static_cast<char*>(out) + off, ev_i, st)
               : h2o::launch_decode(cache->view, cache->cfg.dtype, cache->split, cache->chunk, cache->stages, false,

@@ -160,7 +160,7 @@ bool decode_chunk_supported(int dtype, int head_dim, int max_B, int64_t total_sl
 cudaError_t launch_fscore(const CacheView& c, int hkind, double* out, cudaStream_t stream);
 size_t kv4_row_bytes();
 int fwd_group_units(int units, int max_seqlen);
-cudaError_t launch_decode_kv4(const CacheView& c, int max_B, bool cache_is_quiescent, bool all_full, const void* q,
+cudaError_t launch_decode_kv4(const CacheView& c, int split, int chunk, bool cache_is_quiescent, bool all_full, const void* q,
                               const void* k_new, const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream);
 cudaError_t launch_gather_kv4(const CacheView& c, const PrefillScratch& s, const void* k, const void* v, cudaStream_t stream);
 // `meta`: host copy of the unit table in launch order.

@@ -42,6 +42,8 @@ def main():
         ("sparse pattern", wl("b10", 2, 3, 128, "bf16", [400, 300], 24, [20, 30], [24, 16], 810), dict(mask=(1, 8, 3))),
         ("top-k attention", wl("b12", 2, 3, 128, "bf16", [400, 300], 24, [20, 30], [24, 16], 812), dict(topk=9)),
         ("grouped-query attention", wl("b13", 2, 2, 128, "bf16", [300, 200], 24, [20, 30], [24, 16], 813), dict(group=4)),
+        ("4-bit slots split over a cluster", wl("b15", 1, 2, 128, "bf16_kv4", [1500], 12, [300], [260], 815), dict(split=4)),
+        ("two-pass step kernel split over a cluster", wl("b16", 1, 2, 128, "bf16", [1500], 12, [300], [260], 816), dict(split=4, decode_path=2)),
         ("two-pass step kernel, fill phase", wl("b14", 3, 2, 128, "bf16", [300, 20, 513], 24, [20, 30, 33], [24, 16, 31], 814), dict(decode_path=2)),
     ]
     for name, w, kw in cases:

@@ -565,6 +565,18 @@ def test_two_pass_step_kernel_unit_split_over_a_cluster(H2OCache, budget, split)
     print(run_parity(wl, H2OCache, prefill=False, export_every=8, split=min(split, 2), decode_path=2))
 
 
+@pytest.mark.parametrize("budget,split", [(300, 2), (1040, 4), (2300, 8)])
+def test_four_bit_slots_unit_split_over_a_cluster(H2OCache, budget, split):
+    """4-bit slots with a unit split over a cluster (the library's choice for few long units): statistics and partial
+    outputs exchanged after the stream, candidates after the final probabilities; also from an empty cache."""
+    from parity_harness import run_parity
+
+    wl = _wl("k4split", 1, 2, 128, "bf16_kv4", [3000], 6, [budget // 2], [budget - budget // 2], seed=217)
+    print(run_parity(wl, H2OCache, export_every=2, split=split))
+    wl = _wl("k4splitfill", 1, 2, 128, "bf16_kv4", [1], 70, [20], [30], seed=218)
+    print(run_parity(wl, H2OCache, prefill=False, export_every=8, split=min(split, 4)))
+
+
 def test_two_pass_step_kernel_where_it_does_not_apply(H2OCache):
     import paper_2306_14048_b200 as pkg
 
