@@ -274,10 +274,10 @@ int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages
 int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
 /*
  * Which kernel runs a multi-head decode step (no counterpart in the paper; results differ by summation order
- * only): 0 = automatic, 1 = the online-softmax kernel (one pass over K and V tile pairs; the only one with a
- * cluster split, sparse patterns and "Top-K" attention), 2 = the two-pass streaming kernel (bf16, head_dim 128:
+ * only): 0 = automatic, 1 = the online-softmax kernel (one pass over K and V tile pairs; the only one with
+ * "Top-K" attention), 2 = the two-pass streaming kernel (bf16, head_dim 128:
  * K stream with the scores on the tensor cores, exact softmax, V stream; H2O_ERR_UNSUPPORTED where it does not
- * apply: other dtypes, 4-bit slots, grouped caches (which have their own form of it), a pattern or "Top-K" set,
+ * apply: other dtypes, 4-bit slots, grouped caches (which have their own form of it), "Top-K" attention set,
  * budgets whose scores do not fit shared memory).  Automatic takes 2 for launches of more than two blocks per SM
  * whose mean budget is at least 224 slots (192 from eight blocks per SM on).
  */

@@ -252,14 +252,24 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   const int total = cnt + (rank == 0 ? 1 : 0);
   {
     const int g = tid % G;
+    // a sparse pattern inside the recent window (Section 5.1: heavy hitters combined with the strided / fixed
+    // patterns) leaves keys out: logit -inf, probability 0, no score from this step; it needs the slots' positions
+    const int mask_kind = c.mask_kind;
+    if (mask_kind != 0 && nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
     float mx = -INFINITY, sum = 0.f;
     for (int x = tid / G; x < total; x += kThreads / G) {
-      const float sx = p[x * G + g];
-      if (sx > mx) {
-        sum *= expf(mx - sx);  // expf(-inf) = 0 the first time
-        mx = sx;
+      float sx = p[x * G + g];
+      if (mask_kind != 0 && x < cnt && !key_attended(mask_kind, c.mask_a, c.mask_b, pos_s[x], t, r)) {
+        sx = -INFINITY;
+        p[x * G + g] = sx;
       }
-      sum += expf(sx - mx);
+      if (sx > -INFINITY) {
+        if (sx > mx) {
+          sum *= expf(mx - sx);  // expf(-inf) = 0 the first time
+          mx = sx;
+        }
+        sum += expf(sx - mx);
+      }
     }
     // lanes of equal lane % G, then the warps
 #pragma unroll

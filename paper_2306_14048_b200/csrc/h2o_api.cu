@@ -478,9 +478,9 @@ namespace {
 // online-softmax kernel on launches of many waves of mid-sized and large units (4096 ragged units of 26..820
 // slots: 148 -> 140.5 us; 512 units of 410 slots: 28.1 -> 20.9 us) and slower on small units (3584 units of 104
 // slots: 44.2 -> 53.9 us), equal on 256 units of 410 slots and on 32 units of 2048 slots split over clusters of
-// eight (11.9 against 11.3 - 12.0 us), where the online kernel stays; it has no sparse pattern or "Top-K" form.
+// eight (11.9 against 11.3 - 12.0 us), where the online kernel stays; it has no "Top-K" form.
 bool two_pass_supported(const h2o_cache* cache) {
-  return cache->view.group == 1 && !cache->view.kv4 && cache->view.mask_kind == 0 && cache->view.topk == 0 &&
+  return cache->view.group == 1 && !cache->view.kv4 && cache->view.topk == 0 &&
          h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->chunk);
 }
 bool two_pass_step(const h2o_cache* cache) {

@@ -587,8 +587,20 @@ def test_two_pass_step_kernel_where_it_does_not_apply(H2OCache):
         assert pkg.lib.h2o_cache_set_decode_path(cache._h, 1) == pkg.H2O_OK
         cache.close()
     cache = H2OCache(1, 2, 128, "bf16", [8], [8])
-    cache.set_mask(1, 4, 2)
+    cache.set_topk(4)
     assert pkg.lib.h2o_cache_set_decode_path(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
-    cache.set_mask(0, 1, 0)
+    cache.set_topk(0)
     cache.set_decode_path(2)
     cache.close()
+
+
+@pytest.mark.parametrize("mask", [(1, 8, 3), (2, 16, 2), (1, 3, 1)])
+def test_two_pass_step_kernel_with_a_sparse_pattern(H2OCache, mask):
+    """Heavy hitters combined with the strided / fixed patterns inside the recent window, on the two-pass kernel
+    (also with a unit split over a cluster)."""
+    from parity_harness import run_parity
+
+    wl = _wl("tpmask", 3, 2, 128, "bf16", [400, 300, 90], 30, [20, 30, 10], [40, 64, 30], seed=451)
+    print(run_parity(wl, H2OCache, export_every=5, mask=mask, decode_path=2))
+    wl = _wl("tpmasksplit", 1, 2, 128, "bf16", [1500], 10, [300], [330], seed=452)
+    print(run_parity(wl, H2OCache, export_every=5, mask=mask, decode_path=2, split=4))
