@@ -279,7 +279,7 @@ int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
  * K stream with the scores on the tensor cores, exact softmax, V stream; H2O_ERR_UNSUPPORTED where it does not
  * apply: other dtypes, 4-bit slots, grouped caches (which have their own form of it), "Top-K" attention set,
  * budgets whose scores do not fit shared memory).  Automatic takes 2 for launches of more than two blocks per SM
- * whose mean budget is at least 224 slots (192 from eight blocks per SM on).
+ * whose mean budget is at least 100 slots.
  */
 int h2o_cache_set_decode_path(h2o_cache_t* cache, int32_t path);
 /* The kind of kernel the next h2o_decode_step of this cache launches: 2 = two streaming passes, 1 = one pass

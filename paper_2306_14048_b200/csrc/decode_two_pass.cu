@@ -85,6 +85,12 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
                        int32_t* __restrict__ evicted_pos, int split_arg, int chunk, int launch_flags) {
   const int split = CLUSTER ? split_arg : 1;
   constexpr int kWarps = NW, kThreads = NW * 32, kStages = STAGES, kStageShift = STAGES == 8 ? 3 : 2;
+  // KSTATS: the warps keep the softmax statistics of their rows during the K pass (see there).  Not in the
+  // instance of many large multi-head units: with one head three quarters of the lanes' work on the statistics
+  // is idle, and where several waves of blocks hide the pass between the streams anyway the extra instructions
+  // cost more than the shorter pass saves (config 5: 139.7 against 142.2 us); everywhere else it wins (3584 units
+  // of 104 slots: 45.6 -> 42.1 us; 512 grouped units, G = 8: 31.9 -> 29.8 us).
+  constexpr bool KSTATS = !(G == 1 && NW == 4 && MINB == 4);
   auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
@@ -216,7 +222,14 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
     if (lane == 0) p[cnt * G + g] = c.scale * part;
   }
   // K pass: block b (16 rows) of the stream goes to warp b % NW; every warp steps through every tile so that
-  // the ring's barriers see all of them
+  // the ring's barriers see all of them.  Besides the raw scores a warp keeps the softmax statistics of its rows
+  // (per head: running maximum, and per lane the sum over its own rows), in the shadow of the stream: the pass
+  // between the streams is then a merge of NW pairs per head instead of two sweeps over all scores.
+  // A sparse pattern inside the recent window (Section 5.1: heavy hitters combined with the strided / fixed patterns)
+  // leaves keys out: logit -inf, probability 0, no score from this step; it needs the slots' positions.
+  const int mask_kind = c.mask_kind;
+  if (mask_kind != 0 && nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
+  float wm[2] = {-INFINITY, -INFINITY}, wl[2] = {0.f, 0.f};  // heads 2 c4 and 2 c4 + 1
   for (int j = 0; j < nt; ++j) {
     const int s = j & (kStages - 1);
     if (!bar_wait(&sh.full[s], (uint32_t)(j >> kStageShift) & 1u)) timed_out = true;
@@ -233,36 +246,65 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       }
       // lane (gl, c4): rows gl and gl + 8 of the block, heads 2 c4 and 2 c4 + 1 (rows past the end hold stale bytes)
       const int rowA = j * kTileRows + 16 * hb + gl, rowB = rowA + 8;
+      // (without the statistics only a pattern needs the -inf: rows past the end are not stored at all)
+      bool okA = KSTATS ? rowA < cnt : true, okB = KSTATS ? rowB < cnt : true;
+      if (mask_kind != 0) {
+        okA = rowA < cnt;
+        okB = rowB < cnt;
+        okA = okA && key_attended(mask_kind, c.mask_a, c.mask_b, pos_s[okA ? rowA : 0], t, r);
+        okB = okB && key_attended(mask_kind, c.mask_a, c.mask_b, pos_s[okB ? rowB : 0], t, r);
+      }
+      float sc[2][2];  // [row A / B][head 2 c4 / 2 c4 + 1]
+      sc[0][0] = okA ? c.scale * (d0[0] + d1[0]) : -INFINITY;
+      sc[0][1] = okA ? c.scale * (d0[1] + d1[1]) : -INFINITY;
+      sc[1][0] = okB ? c.scale * (d0[2] + d1[2]) : -INFINITY;
+      sc[1][1] = okB ? c.scale * (d0[3] + d1[3]) : -INFINITY;
       if constexpr (G == 1) {
         if (c4 == 0) {
-          if (rowA < cnt) p[rowA] = c.scale * (d0[0] + d1[0]);
-          if (rowB < cnt) p[rowB] = c.scale * (d0[2] + d1[2]);
+          if (rowA < cnt) p[rowA] = sc[0][0];
+          if (rowB < cnt) p[rowB] = sc[1][0];
         }
       } else if (2 * c4 < G) {
-        if (rowA < cnt) *reinterpret_cast<float2*>(p + rowA * G + 2 * c4) = make_float2(c.scale * (d0[0] + d1[0]), c.scale * (d0[1] + d1[1]));
-        if (rowB < cnt) *reinterpret_cast<float2*>(p + rowB * G + 2 * c4) = make_float2(c.scale * (d0[2] + d1[2]), c.scale * (d0[3] + d1[3]));
+        if (rowA < cnt) *reinterpret_cast<float2*>(p + rowA * G + 2 * c4) = make_float2(sc[0][0], sc[0][1]);
+        if (rowB < cnt) *reinterpret_cast<float2*>(p + rowB * G + 2 * c4) = make_float2(sc[1][0], sc[1][1]);
+      }
+      if constexpr (KSTATS) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float bm = fmaxf(sc[0][h], sc[1][h]);  // the block's maximum of this head: over the eight row pairs
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 4));
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 8));
+        bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, 16));
+        const float nm = fmaxf(wm[h], bm);
+        if (nm > -INFINITY) {  // (uniform over the lanes of equal c4)
+          wl[h] = wl[h] * expf(wm[h] - nm) + expf(sc[0][h] - nm) + expf(sc[1][h] - nm);  // expf(-inf) = 0
+          wm[h] = nm;
+        }
+      }
       }
     }
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh.empty[s]);
   }
+  if constexpr (KSTATS) {
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {  // the lanes' sums over the warp's rows
+    wl[h] += __shfl_xor_sync(0xffffffffu, wl[h], 4);
+    wl[h] += __shfl_xor_sync(0xffffffffu, wl[h], 8);
+    wl[h] += __shfl_xor_sync(0xffffffffu, wl[h], 16);
+    if (gl == 0 && 2 * c4 + h < G) {
+      sh.part_m[warp][2 * c4 + h] = wm[h];
+      sh.part_l[warp][2 * c4 + h] = wl[h];
+    }
+  }
+  }
   consumer_sync();
-
-  // ---- softmax per head over the cnt rows and the token itself: thread (x0, g) = (tid / G, tid % G) ----------
-  const int total = cnt + (rank == 0 ? 1 : 0);
-  {
+  if constexpr (!KSTATS) {
+    // one sweep over the scores instead: thread (x0, g) = (tid / G, tid % G), online pairs merged by shuffles
     const int g = tid % G;
-    // a sparse pattern inside the recent window (Section 5.1: heavy hitters combined with the strided / fixed
-    // patterns) leaves keys out: logit -inf, probability 0, no score from this step; it needs the slots' positions
-    const int mask_kind = c.mask_kind;
-    if (mask_kind != 0 && nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;
     float mx = -INFINITY, sum = 0.f;
-    for (int x = tid / G; x < total; x += kThreads / G) {
-      float sx = p[x * G + g];
-      if (mask_kind != 0 && x < cnt && !key_attended(mask_kind, c.mask_a, c.mask_b, pos_s[x], t, r)) {
-        sx = -INFINITY;
-        p[x * G + g] = sx;
-      }
+    for (int x = tid / G; x < cnt; x += kThreads / G) {
+      const float sx = p[x * G + g];
       if (sx > -INFINITY) {
         if (sx > mx) {
           sum *= expf(mx - sx);  // expf(-inf) = 0 the first time
@@ -271,7 +313,6 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
         sum += expf(sx - mx);
       }
     }
-    // lanes of equal lane % G, then the warps
 #pragma unroll
     for (int off = G; off < 32; off <<= 1) {
       const float om = __shfl_xor_sync(0xffffffffu, mx, off), os = __shfl_xor_sync(0xffffffffu, sum, off);
@@ -284,21 +325,21 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       sh.part_l[warp][lane] = sum;
     }
     consumer_sync();
+  }
+
+  // ---- softmax statistics per head: the warps' pairs and the token itself (exact maximum and sum) --------------
+  {
     if (tid < G) {
-      float m = -INFINITY;
+      const float s_self = rank == 0 ? p[cnt * G + tid] : -INFINITY;
+      float m = s_self;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) m = fmaxf(m, sh.part_m[w][tid]);
-      float l = 0.f;
+      float l = s_self > -INFINITY ? expf(s_self - m) : 0.f;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w)
         if (sh.part_m[w][tid] > -INFINITY) l += sh.part_l[w][tid] * expf(sh.part_m[w][tid] - m);
-      if (split == 1) {
-        sh.m[tid] = m;
-        sh.inv_l[tid] = 1.0f / l;
-      } else {
-        sh.m[tid] = m;      // (the block's own, until the cluster's are known)
-        sh.inv_l[tid] = l;
-      }
+      sh.m[tid] = m;
+      sh.inv_l[tid] = split == 1 ? 1.0f / l : l;  // (split unit: the block's own sum, until the cluster's is known)
     }
     if (split > 1) {
       // the block's statistics into every block of the cluster (its own included); the value tiles keep arriving
@@ -322,8 +363,12 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
       }
     }
     consumer_sync();
-    const float m = sh.m[g], inv_l = sh.inv_l[g];
-    for (int x = tid / G; x < total; x += kThreads / G) p[x * G + g] = expf(p[x * G + g] - m) * inv_l;
+    // final probabilities in place: thread (x0, g) = (tid / G, tid % G); -inf (a key the pattern left out) gives 0
+    {
+      const int g = tid % G;
+      const float m = sh.m[g], inv_l = sh.inv_l[g];
+      for (int x = tid / G; x < cnt + (rank == 0 ? 1 : 0); x += kThreads / G) p[x * G + g] = expf(p[x * G + g] - m) * inv_l;
+    }
   }
   consumer_sync();
 

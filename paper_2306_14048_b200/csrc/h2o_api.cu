@@ -474,11 +474,13 @@ int h2o_prefill_select(h2o_cache_t* cache, const void* q, const void* k, const v
 
 namespace {
 // Which kernel serves a multi-head decode step.  The two-pass streaming kernel (K stream with the scores on
-// mma.sync, exact softmax, V stream; decode_two_pass.cu with one query head per unit) is faster than the
-// online-softmax kernel on launches of many waves of mid-sized and large units (4096 ragged units of 26..820
-// slots: 148 -> 140.5 us; 512 units of 410 slots: 28.1 -> 20.9 us) and slower on small units (3584 units of 104
-// slots: 44.2 -> 53.9 us), equal on 256 units of 410 slots and on 32 units of 2048 slots split over clusters of
-// eight (11.9 against 11.3 - 12.0 us), where the online kernel stays; it has no "Top-K" form.
+// mma.sync and the softmax statistics kept alongside, V stream; decode_two_pass.cu with one query head per unit) is
+// the faster one for launches of more than two blocks per SM unless the units are small.  Per launch, online-softmax
+// kernel against two-pass kernel: 4096 ragged units of 26..820 slots 148 / 140 us; 3584 units of 104 slots
+// 44.4 / 42.2; 2048 units of 64 / 96 / 128 / 160 / 256 slots 18.3 / 19.6, 23.6 / 24.0, 28.0 / 27.4, 34.0 / 33.4,
+// 54.5 / 47.1; 600 units of 128 / 300 slots 13.9 / 8.7, 23.6 / 17.2; 4096 units of 64 slots 34.0 / 38.8 us.  On
+// 256 units of 410 slots both take 12.2 us, on 32 units of 2048 slots split over clusters of eight 11.3 - 12.0
+// against 11.4: the online kernel stays there.  The two-pass kernel has no "Top-K" form.
 bool two_pass_supported(const h2o_cache* cache) {
   return cache->view.group == 1 && !cache->view.kv4 && cache->view.topk == 0 &&
          h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->chunk);
@@ -486,10 +488,7 @@ bool two_pass_supported(const h2o_cache* cache) {
 bool two_pass_step(const h2o_cache* cache) {
   if (cache->decode_path == 1 || !two_pass_supported(cache)) return false;
   if (cache->decode_path == 2) return true;
-  // (crossover measured on 2048 units: 160 slots 34.3 against 35.1 us, 192 slots 41.9 against 39.4 us; on 1024 units
-  //  of 192 slots 21.8 against 22.9 us)
-  const int sms = h2o::sm_count();
-  return cache->split == 1 && cache->view.units > 2 * sms && cache->mean_budget >= (cache->view.units >= 8 * sms ? 192.0 : 224.0);
+  return cache->split == 1 && cache->view.units > 2 * h2o::sm_count() && cache->mean_budget >= 100.0;
 }
 }  // namespace
 
