@@ -8,19 +8,20 @@
 // Against the online-softmax kernel of decode.cu this one reads K completely before V: the softmax is exact when
 // the values arrive, so the V pass has no running maximum to follow and no rescaling, and the scores come from the
 // tensor cores without a shuffle; the price is the pass in between and the scores of all rows in shared memory.
-// It is the faster one for launches of many waves of mid-sized and large units.  A unit can be split over the
+// It is the faster one for launches of more than two blocks per SM unless the units are small.  A unit can be split over the
 // blocks of a cluster (few long units): statistics are exchanged between the passes, partial outputs and victim
 // candidates in one exchange after the value pass.
 //
-// Shape: one thread block per unit, eight consumer warps and a producer warp.  The producer streams the unit's K
+// Shape: one thread block per unit (or per share of a split unit), eight or four consumer warps and a producer warp.  The producer streams the unit's K
 // rows and then its V rows as 8 KB tiles (32 rows) through one bulk-copy ring, so HBM stays busy across the two
 // passes.
 //   K pass: the scores of 16 rows x G heads are one mma.sync m16n8k16 chain (rows = M, heads = N, channels = K);
 //           a lane loads 16 bytes of a row and uses them as the k-slots of two products, the query operand is
 //           laid out to match (which channel sits in which k-slot is free as long as both operands agree).  The
-//           16-row blocks of the tiles go round the warps.  Raw scores to shared memory, [row][head].
-//   softmax per head over all rows (exact maximum and sum, as the accumulation needs the final probabilities),
-//           in place.
+//           16-row blocks of the tiles go round the warps.  Raw scores to shared memory, [row][head]; the warps
+//           keep the softmax statistics of their rows alongside (one instance computes them in a sweep afterwards).
+//   between the passes: the statistics merged per head (exact maximum and sum, as the accumulation needs the final
+//           probabilities), one sweep that turns the scores into probabilities in place.
 //   V pass: a lane holds eight channels of a row (two rows per warp and pass) and G x 8 accumulators.
 // Tail as in the other step kernels: fp64 accumulation of the summed probabilities, victim by (score, position),
 // new row written into the freed slot.  Every wait on an mbarrier is bounded (H2O_ERR_TIMEOUT in the status word).
