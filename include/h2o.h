@@ -85,8 +85,9 @@ typedef struct {
  * head attends the unit's entries with its own softmax, and a key's accumulated score grows by the SUM of the
  * probabilities the group's heads gave it; selection after the prompt and eviction use that sum.  Each K and V row
  * is read once for the whole group.  Supported: f32 / bf16 slots, budgets with G * (k_s + r_s + 1) * 4 bytes up to
- * about 160 KB; the prompt runs on the fp32-FMA kernels; sparse patterns, "Top-K" attention, 4-bit slots and the
- * host-buffer calls are not combined with it (H2O_ERR_UNSUPPORTED).
+ * about 160 KB; bf16 with head_dim 128 runs on the tensor-core prompt kernels and the streaming step kernel, the
+ * rest on the fp32-FMA prompt kernels and the plain grouped step kernel; sparse patterns, "Top-K" attention and
+ * 4-bit slots are not combined with it (H2O_ERR_UNSUPPORTED).
  */
 
 /* Bytes of device workspace h2o_cache_create needs for this configuration
@@ -217,6 +218,7 @@ int h2o_prefill_select_static(h2o_cache_t* cache, const void* q, const void* k, 
  *                            (each rounded up to 256 bytes); scratch as above.
  *   h2o_decode_step_host   : staging >= 4 tensors of [batch, n_heads, head_dim] plus
  *                            [batch, n_heads] int32 (each rounded up to 256 bytes).
+ *   (With query_group = G > 1 the q and out tensors of both calls carry n_heads * G heads.)
  * When every buffer of h2o_decode_step_host is pinned or registered host memory (which the
  * device can address) and 16-byte aligned, the kernel reads and writes it directly and no
  * copy is enqueued; the buffers must then not be touched by the host until the stream has

@@ -641,15 +641,15 @@ int h2o_cache_set_chunk_path(h2o_cache_t* cache, int32_t path) {
 
 size_t h2o_host_staging_bytes(const h2o_config_t* cfg, int64_t tokens) {
   if (check_config(cfg) != H2O_OK || tokens < 1 || tokens > INT32_MAX) return 0;
-  const size_t tensor = align_up((size_t)tokens * cfg->n_heads * cfg->head_dim * elem_size(cfg->dtype));
-  return 4 * tensor + align_up((size_t)tokens * cfg->n_heads * sizeof(int32_t));
+  const size_t kv = align_up((size_t)tokens * cfg->n_heads * cfg->head_dim * elem_size(cfg->dtype));
+  const size_t qo = align_up((size_t)tokens * cfg->n_heads * group_of(cfg) * cfg->head_dim * elem_size(cfg->dtype));
+  return 2 * qo + 2 * kv + align_up((size_t)tokens * cfg->n_heads * sizeof(int32_t));  // q, k, v, out, evicted
 }
 
 int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* k_host, const void* v_host,
                             const int32_t* cu_seqlens, void* out_host, void* staging, size_t staging_bytes,
                             void* scratch, size_t scratch_bytes, void* stream) {
   if (!cache || !q_host || !k_host || !v_host || !cu_seqlens || !out_host || !staging) return H2O_ERR_INVALID_ARG;
-  if (cache->view.group > 1) return H2O_ERR_UNSUPPORTED;  // (q / out and k / v differ in size there)
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;
   const h2o_config_t& cfg = cache->cfg;
   const int64_t total = cu_seqlens[cfg.batch];
@@ -659,20 +659,22 @@ int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* 
   DeviceGuard guard(cfg.device);
   if (!guard.ok) return H2O_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // staging: q | k | v | out; with grouped-query attention q and out carry n_heads * group heads
   const size_t bytes = (size_t)total * cfg.n_heads * cfg.head_dim * elem_size(cfg.dtype);
-  const size_t pitch = align_up(bytes);
+  const size_t qbytes = bytes * cache->view.group;
+  const size_t pitch = align_up(bytes), qpitch = align_up(qbytes);
   char* sg = static_cast<char*>(staging);
-  bool ok = cudaMemcpyAsync(sg, q_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(sg + pitch, k_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(sg + 2 * pitch, v_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  char *sq = sg, *sk = sg + qpitch, *sv = sk + pitch, *so = sv + pitch;
+  bool ok = cudaMemcpyAsync(sq, q_host, qbytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sk, k_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sv, v_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
-  const int rc = h2o_prefill_select(cache, sg, sg + pitch, sg + 2 * pitch, cu_seqlens, sg + 3 * pitch, scratch,
-                                    scratch_bytes, stream);
+  const int rc = h2o_prefill_select(cache, sq, sk, sv, cu_seqlens, so, scratch, scratch_bytes, stream);
   if (rc != H2O_OK) return rc;
-  if (cudaMemcpyAsync(out_host, sg + 3 * pitch, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+  if (cudaMemcpyAsync(out_host, so, qbytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
@@ -682,7 +684,6 @@ int h2o_prefill_select_host(h2o_cache_t* cache, const void* q_host, const void* 
 int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_new_host, const void* v_new_host,
                          void* out_host, int32_t* evicted_pos_host, void* staging, size_t staging_bytes, void* stream) {
   if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !staging) return H2O_ERR_INVALID_ARG;
-  if (cache->view.group > 1) return H2O_ERR_UNSUPPORTED;
   const h2o_config_t& cfg = cache->cfg;
   if (staging_bytes < h2o_host_staging_bytes(&cfg, cfg.batch) || (reinterpret_cast<uintptr_t>(staging) % kAlign) != 0)
     return H2O_ERR_WORKSPACE;
@@ -690,9 +691,11 @@ int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_n
   if (!guard.ok) return H2O_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t bytes = (size_t)cfg.batch * cfg.n_heads * cfg.head_dim * elem_size(cfg.dtype);
-  const size_t pitch = align_up(bytes);
+  const size_t qbytes = bytes * cache->view.group;  // q and out carry n_heads * group heads
+  const size_t pitch = align_up(bytes), qpitch = align_up(qbytes);
   char* sg = static_cast<char*>(staging);
-  int32_t* ev_dev = reinterpret_cast<int32_t*>(sg + 4 * pitch);
+  char *sq = sg, *sk = sg + qpitch, *sv = sk + pitch, *so = sv + pitch;
+  int32_t* ev_dev = reinterpret_cast<int32_t*>(so + qpitch);
   // Pinned (or registered) host memory is addressable by the device: a decode step moves only a few
   // hundred bytes per unit, so the kernel reads its inputs and writes its results straight over the
   // bus instead of paying five small copies around every launch.  Pageable buffers take the copies.
@@ -705,17 +708,16 @@ int h2o_decode_step_host(h2o_cache_t* cache, const void* q_host, const void* k_n
     if (dq && dk && dv && dout && (!evicted_pos_host || dev_ev))
       return h2o_decode_step(cache, dq, dk, dv, dout, static_cast<int32_t*>(dev_ev), stream);
   }
-  bool ok = cudaMemcpyAsync(sg, q_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(sg + pitch, k_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(sg + 2 * pitch, v_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  bool ok = cudaMemcpyAsync(sq, q_host, qbytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sk, k_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(sv, v_new_host, bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     return H2O_ERR_CUDA;
   }
-  const int rc = h2o_decode_step(cache, sg, sg + pitch, sg + 2 * pitch, sg + 3 * pitch,
-                                 evicted_pos_host ? ev_dev : nullptr, stream);
+  const int rc = h2o_decode_step(cache, sq, sk, sv, so, evicted_pos_host ? ev_dev : nullptr, stream);
   if (rc != H2O_OK) return rc;
-  ok = cudaMemcpyAsync(out_host, sg + 3 * pitch, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = cudaMemcpyAsync(out_host, so, qbytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   if (evicted_pos_host)
     ok = ok && cudaMemcpyAsync(evicted_pos_host, ev_dev, (size_t)cfg.batch * cfg.n_heads * sizeof(int32_t),
                                cudaMemcpyDeviceToHost, st) == cudaSuccess;

@@ -21,9 +21,13 @@ def pkg():
 WL = Workload("api", 3, 4, 128, "bf16", (260, 97, 513), 6, (16, 8, 20), (16, 8, 20), 1, 909)
 
 
-def _full_run(pkg, wl, host=False, reset_first=False):
-    cache = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent)
+def _full_run(pkg, wl, host=False, reset_first=False, group=1):
+    cache = pkg.H2OCache(wl.batch, wl.n_heads, wl.head_dim, wl.dtype, wl.heavy, wl.recent, query_group=group)
+    wlq = wl.scaled(n_heads=wl.n_heads * group)  # the query side carries n_heads * group heads
     q, k, v, cu = make_prompt_inputs(wl, device="cuda")
+    if group > 1:
+        q = make_prompt_inputs(wlq, device="cuda")[0]
+        reset_first = False
     if reset_first:  # dirty the cache with another prompt, then reset it
         cache.prefill_select(v, q, k, cu, torch.empty_like(q))
         cache.reset()
@@ -31,7 +35,7 @@ def _full_run(pkg, wl, host=False, reset_first=False):
     if host:
         hq, hk, hv = (x.cpu().pin_memory() for x in (q, k, v))
         ho = torch.empty_like(hq).pin_memory()
-        cache.prefill_select_host(hq, hk, hv, cu, ho)
+        cache.prefill_select_host(hq, hk, hv, cu, ho)  # (staging sized for the larger q / out of a grouped cache)
         torch.cuda.synchronize()
         outs.append(ho.float().numpy().copy())
     else:
@@ -41,6 +45,8 @@ def _full_run(pkg, wl, host=False, reset_first=False):
     evs = []
     for step in range(wl.decode_steps):
         dq, dk, dv = make_decode_inputs(wl, step, device="cuda")
+        if group > 1:
+            dq = make_decode_inputs(wlq, step, device="cuda")[0]
         if host:
             # pinned buffers are read and written by the kernel directly; pageable ones go through the staging copies
             pin = (lambda x: x.pin_memory()) if host != "pageable" else (lambda x: x)
@@ -80,6 +86,12 @@ def test_two_runs_are_bit_identical(pkg):
 @pytest.mark.parametrize("mode", ["pinned", "pageable"])
 def test_host_buffer_calls_equal_device_calls(pkg, mode):
     _identical(_full_run(pkg, WL, host=mode), _full_run(pkg, WL))
+
+
+@pytest.mark.parametrize("mode", ["pinned", "pageable"])
+def test_host_buffer_calls_with_grouped_query_heads(pkg, mode):
+    """q and out carry n_heads * group heads, k / v / evicted positions n_heads: the staging is laid out for that."""
+    _identical(_full_run(pkg, WL, host=mode, group=4), _full_run(pkg, WL, group=4))
 
 
 def test_kv4_slots_host_calls_snapshots_and_reproducibility(pkg):
