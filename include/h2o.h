@@ -86,8 +86,8 @@ typedef struct {
  * probabilities the group's heads gave it; selection after the prompt and eviction use that sum.  Each K and V row
  * is read once for the whole group.  Supported: f32 / bf16 slots, budgets with G * (k_s + r_s + 1) * 4 bytes up to
  * about 160 KB; bf16 with head_dim 128 runs on the tensor-core prompt kernels and the streaming step kernel, the
- * rest on the fp32-FMA prompt kernels and the plain grouped step kernel; sparse patterns, "Top-K" attention and
- * 4-bit slots are not combined with it (H2O_ERR_UNSUPPORTED).
+ * rest on the fp32-FMA prompt kernels and the plain grouped step kernel; "Top-K" attention and 4-bit slots are not
+ * combined with it, sparse patterns only where the streaming step kernel applies (H2O_ERR_UNSUPPORTED otherwise).
  */
 
 /* Bytes of device workspace h2o_cache_create needs for this configuration

@@ -587,7 +587,11 @@ int h2o_cache_set_mask(h2o_cache_t* cache, int32_t kind, int32_t a, int32_t b) {
   if (!cache || kind < 0 || kind > 2) return H2O_ERR_INVALID_ARG;
   if (kind != 0 && (a < 1 || b < 0 || (kind == 2 && b > a))) return H2O_ERR_INVALID_ARG;
   if (cache->phase != Phase::Empty) return H2O_ERR_STATE;  // one attention rule per generation
-  if (kind != 0 && (cache->view.kv4 || cache->view.group > 1)) return H2O_ERR_UNSUPPORTED;
+  // (4-bit slots have no pattern form; of the grouped step kernels the streaming one applies patterns)
+  if (kind != 0 && (cache->view.kv4 || (cache->view.group > 1 &&
+                                        !h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, cache->view.group,
+                                                                        cache->layout.max_B))))
+    return H2O_ERR_UNSUPPORTED;
   cache->view.mask_kind = kind;
   cache->view.mask_a = kind ? a : 1;
   cache->view.mask_b = kind ? b : 0;

@@ -515,6 +515,20 @@ def test_grouped_query_attention_long_budget_chunk_call_and_averaged_score(H2OCa
     print(run_parity(wl, H2OCache, export_every=8, group=2, score_mode=1))
 
 
+def test_grouped_query_attention_with_a_sparse_pattern(H2OCache):
+    """Grouped bf16 / head_dim 128 caches combine with the strided / fixed patterns (fp32-FMA prompt kernels with the
+    pattern over the group, streaming grouped step kernel); other grouped caches refuse a pattern."""
+    import paper_2306_14048_b200 as pkg
+    from parity_harness import run_parity
+
+    wl = _wl("gqamask", 3, 2, 128, "bf16", [400, 300, 90], 30, [20, 30, 10], [40, 64, 30], seed=461)
+    for group, mask in ((2, (1, 8, 3)), (4, (2, 16, 2)), (8, (1, 3, 1))):
+        print(run_parity(wl, H2OCache, export_every=5, mask=mask, group=group))
+    cache = H2OCache(1, 2, 64, "f32", [8], [8], query_group=2)
+    assert pkg.lib.h2o_cache_set_mask(cache._h, 1, 4, 2) == pkg.H2O_ERR_UNSUPPORTED
+    cache.close()
+
+
 def test_grouped_query_attention_argument_errors(H2OCache):
     import ctypes
 
