@@ -276,12 +276,12 @@ int h2o_cache_set_decode_shape(h2o_cache_t* cache, int32_t split, int32_t stages
 int h2o_cache_set_prefill_path(h2o_cache_t* cache, int32_t path);
 /*
  * Which kernel runs a multi-head decode step (no counterpart in the paper; results differ by summation order
- * only): 0 = automatic, 1 = the online-softmax kernel (one pass over K and V tile pairs; the only one with
- * "Top-K" attention), 2 = the two-pass streaming kernel (bf16, head_dim 128:
+ * only): 0 = automatic, 1 = the online-softmax kernel (one pass over K and V tile pairs),
+ * 2 = the two-pass streaming kernel (bf16, head_dim 128:
  * K stream with the scores on the tensor cores, exact softmax, V stream; H2O_ERR_UNSUPPORTED where it does not
- * apply: other dtypes, 4-bit slots, grouped caches (which have their own form of it), "Top-K" attention set,
+ * apply: other dtypes, 4-bit slots, grouped caches (which have their own form of it),
  * budgets whose scores do not fit shared memory).  Automatic takes 2 for launches of more than two blocks per SM
- * whose mean budget is at least 100 slots.
+ * whose mean budget is at least 100 slots; with "Top-K" attention set, for launches of at most two blocks per SM.
  */
 int h2o_cache_set_decode_path(h2o_cache_t* cache, int32_t path);
 /* The kind of kernel the next h2o_decode_step of this cache launches: 2 = two streaming passes, 1 = one pass

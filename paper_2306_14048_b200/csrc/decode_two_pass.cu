@@ -56,6 +56,10 @@ struct Shared {
   float part_m[kMaxWarps][8], part_l[kMaxWarps][8];  // per warp and head: softmax partials
   float m[8], inv_l[8];
   Cand wbest[kMaxWarps];
+  // "Top-K" attention: histogram and state of the radix select over the step's logits
+  unsigned int hist[256];
+  unsigned long long tk_prefix;
+  unsigned int tk_remaining, tk_count, tk_bin;  // tk_bin: entries in the bin the last pass chose
   // Cluster exchange (a unit split over the blocks of a cluster): every block pushes its values into its peers'
   // shared memory with remote stores, then one cluster barrier makes them visible.
   float x_m[kMaxSplit][8], x_l[kMaxSplit][8];  // softmax statistics of every rank and head (written by that rank)
@@ -79,7 +83,9 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
 // registers with a 4-deep ring, so that the next launch's blocks are resident beside this launch's (14.4 us), helped.
 // CLUSTER: the instances that can split a unit over a cluster (the others compile that code out: its registers
 // cost the grouped four-warp instance 4 %).
-template <int G, int NW, int STAGES, int MINB, bool CLUSTER>
+// TOPK: the instances with "Top-K" attention (multi-head, one block per unit): after the K pass the step keeps its
+// c.topk largest logits and drops the rest before the statistics.
+template <int G, int NW, int STAGES, int MINB, bool CLUSTER, bool TOPK>
 __global__ void __launch_bounds__(NW * 32 + 32, MINB)
 decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                        const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
@@ -91,7 +97,7 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   // is idle, and where several waves of blocks hide the pass between the streams anyway the extra instructions
   // cost more than the shorter pass saves (config 5: 139.7 against 142.2 us); everywhere else it wins (3584 units
   // of 104 slots: 45.6 -> 42.1 us; 512 grouped units, G = 8: 31.9 -> 29.8 us).
-  constexpr bool KSTATS = !(G == 1 && NW == 4 && MINB == 4);
+  constexpr bool KSTATS = !TOPK && !(G == 1 && NW == 4 && MINB == 4);  // ("Top-K": the statistics follow the selection)
   auto consumer_sync = [] { consumer_sync_n<NW * 32>(); };
   extern __shared__ __align__(128) unsigned char dyn[];
   __shared__ Shared sh;
@@ -300,6 +306,87 @@ decode_two_pass_kernel(CacheView c, const __nv_bfloat16* __restrict__ q, const _
   }
   }
   consumer_sync();
+  if constexpr (TOPK) {
+    // ---- "Top-K" attention (appendix on the Top-K baseline): keep the c.topk largest logits of the step among the
+    // kept entries the pattern allows and the token itself; equal logits: the higher position first.  The key of an
+    // entry is (order-preserving bits of its logit, position): keys are distinct, so the topk-th largest one is a
+    // threshold; it is found by a most-significant-digit radix select, 8 bits a pass, over the scores in shared
+    // memory.  What is below it gets logit -inf: probability 0, no value, no score from this step.
+    if (nstr > 0 && !bar_wait(&sh.aux, 0)) timed_out = true;  // the slots' positions
+    auto key_of = [&](int x) -> unsigned long long {  // x < cnt: cached row x; x == cnt: the token itself
+      const float sx = p[x];
+      if (!(sx > -INFINITY)) return 0ull;  // left out by the pattern: below every real key
+      unsigned int ub = __float_as_uint(sx);
+      ub = (ub & 0x80000000u) ? ~ub : (ub | 0x80000000u);
+      return ((unsigned long long)ub << 32) | (unsigned int)(x < cnt ? pos_s[x] : t);
+    };
+    const int ncand = cnt + 1;
+    if (tid == 0) {
+      sh.tk_prefix = 0ull;
+      sh.tk_remaining = (unsigned int)c.topk;
+      sh.tk_count = 0u;
+    }
+    consumer_sync();
+    {
+      unsigned int real = 0;
+      for (int x = tid; x < ncand; x += kThreads) real += key_of(x) != 0ull ? 1u : 0u;
+      real = (unsigned int)warp_sum((float)real);  // (at most 8193 per unit: exact in fp32)
+      if (lane == 0) atomicAdd(&sh.tk_count, real);
+    }
+    consumer_sync();
+    unsigned long long thr = 1ull;  // every real key
+    if (sh.tk_count > (unsigned int)c.topk) {
+      for (int pass = 0; pass < 8; ++pass) {
+        const int shift = 56 - 8 * pass;
+        for (int i = tid; i < 256; i += kThreads) sh.hist[i] = 0u;
+        consumer_sync();
+        const unsigned long long prefix = sh.tk_prefix;
+        const unsigned long long himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
+        for (int x = tid; x < ncand; x += kThreads) {
+          const unsigned long long key = key_of(x);
+          if (key != 0ull && (key & himask) == prefix) atomicAdd(&sh.hist[(unsigned int)(key >> shift) & 255u], 1u);
+        }
+        consumer_sync();
+        if (warp == 0) {  // the bin that holds the rank still looked for, scanning from the top bin down
+          const int rem = (int)sh.tk_remaining;
+          int cnts[8], tot = 0;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            cnts[i] = (int)sh.hist[255 - 8 * lane - i];
+            tot += cnts[i];
+          }
+          int incl = tot;
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += y;
+          }
+          int before = incl - tot;
+          if (before < rem && incl >= rem) {  // exactly one lane
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              if (before < rem && before + cnts[i] >= rem) {
+                sh.tk_prefix = prefix | ((unsigned long long)(255 - 8 * lane - i) << shift);
+                sh.tk_remaining = (unsigned int)(rem - before);
+                sh.tk_bin = (unsigned int)cnts[i];
+                before = rem;  // done
+              } else {
+                before += cnts[i];
+              }
+            }
+          }
+        }
+        consumer_sync();
+        // after the four passes over the logit's bits: if every entry that shares the threshold logit is wanted
+        // (nearly always: it is the only one), the positions need not be looked at
+        if (pass == 3 && sh.tk_bin == sh.tk_remaining) break;
+      }
+      thr = sh.tk_prefix;
+    }
+    for (int x = tid; x < ncand; x += kThreads)
+      if (key_of(x) < thr) p[x] = -INFINITY;
+    consumer_sync();
+  }
   if constexpr (!KSTATS) {
     // one sweep over the scores instead: thread (x0, g) = (tid / G, tid % G), online pairs merged by shuffles
     const int g = tid % G;
@@ -526,7 +613,7 @@ size_t ring_smem(int group, int chunk, int stages) {
   return (size_t)stages * kTileBytes + (size_t)chunk * 12 + (size_t)(chunk + 4) * group * sizeof(float);
 }
 
-template <int G, int NW, int STAGES, int MINB, bool CLUSTER = false>
+template <int G, int NW, int STAGES, int MINB, bool CLUSTER = false, bool TOPK = false>
 cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
                         const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
   constexpr int kStages = STAGES;
@@ -534,7 +621,7 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
   static_assert((size_t)2 * NW * G * kD * sizeof(float) <= (size_t)kStages * kTileBytes, "partial outputs reuse the ring");
   const size_t smem = ring_smem(G, chunk, kStages) + (split > 1 ? (size_t)kMaxSplit * G * kD * sizeof(float) : 0);
   static unsigned long long attr_flags = 0;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER>), 200 * 1024, &attr_flags);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER, TOPK>), 200 * 1024, &attr_flags);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(c.units * split));
@@ -553,7 +640,7 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
   at[2].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
   cfg.attrs = at;
   cfg.numAttrs = split > 1 ? 3 : 1;
-  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER>, c, static_cast<const __nv_bfloat16*>(q),
+  return cudaLaunchKernelEx(&cfg, decode_two_pass_kernel<G, NW, STAGES, MINB, CLUSTER, TOPK>, c, static_cast<const __nv_bfloat16*>(q),
                             static_cast<const __nv_bfloat16*>(k_new), static_cast<const __nv_bfloat16*>(v_new),
                             static_cast<__nv_bfloat16*>(out), evicted_pos, split, chunk, launch_flags);
 }
@@ -561,6 +648,16 @@ cudaError_t launch_ring(const CacheView& c, int split, int chunk, int launch_fla
 template <int G>
 cudaError_t launch_ring_g(const CacheView& c, int split, int chunk, int launch_flags, const void* q, const void* k_new,
                           const void* v_new, void* out, int32_t* evicted_pos, cudaStream_t stream) {
+  if (c.topk > 0) {  // "Top-K" attention: multi-head, one block per unit
+    if constexpr (G == 1) {
+      if (split != 1) return cudaErrorInvalidValue;
+      if (c.units <= 2 * sm_count())
+        return launch_ring<G, 8, 8, 2, false, true>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+      return launch_ring<G, 4, 4, 4, false, true>(c, split, chunk, launch_flags, q, k_new, v_new, out, evicted_pos, stream);
+    } else {
+      return cudaErrorInvalidValue;
+    }
+  }
   if (split > 1) {
     if constexpr (G == 1) {
       if (c.units * split <= 2 * sm_count())

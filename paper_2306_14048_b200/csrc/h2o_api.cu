@@ -480,14 +480,17 @@ namespace {
 // 44.4 / 42.2; 2048 units of 64 / 96 / 128 / 160 / 256 slots 18.3 / 19.6, 23.6 / 24.0, 28.0 / 27.4, 34.0 / 33.4,
 // 54.5 / 47.1; 600 units of 128 / 300 slots 13.9 / 8.7, 23.6 / 17.2; 4096 units of 64 slots 34.0 / 38.8 us.  On
 // 256 units of 410 slots both take 12.2 us, on 32 units of 2048 slots split over clusters of eight 11.3 - 12.0
-// against 11.4: the online kernel stays there.  The two-pass kernel has no "Top-K" form.
+// against 11.4: the online kernel stays there.
 bool two_pass_supported(const h2o_cache* cache) {
-  return cache->view.group == 1 && !cache->view.kv4 && cache->view.topk == 0 &&
+  return cache->view.group == 1 && !cache->view.kv4 && (cache->view.topk == 0 || cache->split == 1) &&
          h2o::decode_two_pass_supported(cache->cfg.dtype, cache->cfg.head_dim, 1, cache->chunk);
 }
 bool two_pass_step(const h2o_cache* cache) {
   if (cache->decode_path == 1 || !two_pass_supported(cache)) return false;
   if (cache->decode_path == 2) return true;
+  // "Top-K" attention: the selection's block barriers weigh differently on the two kernels: 256 units of 410 slots
+  // 24.0 us on the online kernel's instance against 19.4 here, 4096 ragged units 170 against 180 us
+  if (cache->view.topk > 0) return cache->view.units <= 2 * h2o::sm_count();
   return cache->split == 1 && cache->view.units > 2 * h2o::sm_count() && cache->mean_budget >= 100.0;
 }
 }  // namespace

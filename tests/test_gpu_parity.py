@@ -419,8 +419,10 @@ def test_topk_attention_ragged(H2OCache, m, dtype, d):
     from parity_harness import run_parity
 
     wl = _wl("topk", 4, 3, d, dtype, [300, 77, 513, 40], 48, [20, 9, 33, 30], [24, 5, 31, 30], seed=277 + d)
-    st = run_parity(wl, H2OCache, export_every=8, topk=m)
+    st = run_parity(wl, H2OCache, export_every=8, topk=m)  # bf16 / 128: the two-pass kernel's form (the library's choice)
     print(st)
+    if dtype == "bf16":  # the same on the online-softmax kernel's "Top-K" instance
+        print(run_parity(wl, H2OCache, export_every=8, topk=m, decode_path=1))
 
 
 @pytest.mark.parametrize("heavy,recent", [([0, 0], [7, 16]), ([5, 12], [0, 0]), ([6, 1], [12, 9])])
@@ -433,6 +435,9 @@ def test_topk_attention_edge_budgets_token_by_token(H2OCache, heavy, recent):
     for m in (1, 3):
         st = run_parity(wl, H2OCache, prefill=False, export_every=5, topk=m)
         print(st)
+    wl = _wl("topkedge2", 2, 2, 128, "bf16", [1, 1], 60, heavy, recent, seed=26)  # the two-pass kernel's form
+    for m in (1, 3):
+        print(run_parity(wl, H2OCache, prefill=False, export_every=5, topk=m))
 
 
 def test_topk_attention_long_budget_pattern_and_chunk_call(H2OCache):
@@ -601,10 +606,11 @@ def test_two_pass_step_kernel_where_it_does_not_apply(H2OCache):
         assert pkg.lib.h2o_cache_set_decode_path(cache._h, 1) == pkg.H2O_OK
         cache.close()
     cache = H2OCache(1, 2, 128, "bf16", [8], [8])
-    cache.set_topk(4)
-    assert pkg.lib.h2o_cache_set_decode_path(cache._h, 2) == pkg.H2O_ERR_UNSUPPORTED
-    cache.set_topk(0)
+    cache.set_topk(4)  # ("Top-K" attention has a form on either kernel)
     cache.set_decode_path(2)
+    assert cache.decode_path() == 2
+    cache.set_decode_path(1)
+    assert cache.decode_path() == 1
     cache.close()
 
 
